@@ -1,0 +1,246 @@
+"""CPU fp64 oracle for LongGen's efficient attention layers.  TEST INFRASTRUCTURE ONLY.
+
+Only tests, the smoke check and the benchmark's CPU-baseline leg may import this
+module.  It shares no code with the CUDA library and imports nothing from it.
+
+What it computes is masked softmax attention written out from its definition
+(paper Section 3.2: the sparse kernel skips positions whose mask value is zero, so
+the result IS masked attention, only cheaper), under the two static block
+patterns of Section 3.1 / 4.1:
+
+  * attention sink + sliding window: the first blocks plus the most recent blocks,
+  * blockwise strided: every `stride`-th block plus a few local blocks,
+
+and plain causal attention for the full-attention layers.  Every function
+materialises the explicit token-level boolean mask; nothing here is blocked,
+fused or reordered beyond "work on a slab of rows at a time", which changes no
+value.  All arithmetic is float64.
+
+Readings of points on which the paper is silent (see the design notes):
+  - the window is block-granular and counts the query's own block
+    (Section 4.1: "the first block ... and the most recent 32 blocks");
+  - the strided comb is absolute: KV block kb is retained iff kb % stride == 0;
+  - LSE is the natural log of the sum of exp of the *scaled* scores;
+  - the backward formulas are the derivatives of the definition (the paper
+    inherits them from FlashAttention and prints none).
+
+Pins (tests/test_oracle_*.py): brute-force per-row softmax, torch's dense causal
+attention and autograd in fp64, central finite differences, closed-form block
+counts, the paper's KV-cache arithmetic.  Trained-model quality: parity unpinned
+and out of scope.
+"""
+from __future__ import annotations
+
+import os
+from concurrent.futures import ThreadPoolExecutor
+from dataclasses import dataclass
+from typing import Optional, Tuple
+
+import numpy as np
+
+MODE_FULL_CAUSAL = 0
+MODE_SINK_WINDOW = 1
+MODE_STRIDED_LOCAL = 2
+
+
+@dataclass(frozen=True)
+class Pattern:
+    """Static sparse pattern (Section 3.1).  Token counts must be multiples of `block`."""
+    L: int
+    block: int
+    mode: int
+    sink_tokens: int = 0
+    window_tokens: int = 0
+    stride_blocks: int = 0
+    local_blocks: int = 0
+
+    @staticmethod
+    def of(cfg) -> "Pattern":
+        return Pattern(cfg.L, cfg.block, cfg.mode, cfg.sink_tokens, cfg.window_tokens,
+                       cfg.stride_blocks, cfg.local_blocks)
+
+
+# --------------------------------------------------------------------------- masks
+
+def allowed(p: Pattern, i, j):
+    """Token-level predicate: may query i attend key j?  i, j broadcastable int arrays.
+
+    Section 3.1 (patterns), Section 4.1 (block = 64 tokens, 1 sink block + 32 recent
+    blocks; stride in blocks)."""
+    i = np.asarray(i, dtype=np.int32)
+    j = np.asarray(j, dtype=np.int32)
+    causal = j <= i
+    if p.mode == MODE_FULL_CAUSAL:
+        return causal
+    qb = i // p.block
+    kb = j // p.block
+    if p.mode == MODE_SINK_WINDOW:
+        ns = p.sink_tokens // p.block
+        nw = p.window_tokens // p.block
+        return causal & ((kb < ns) | (qb - kb < nw))
+    if p.mode == MODE_STRIDED_LOCAL:
+        return causal & ((qb - kb < p.local_blocks) | (kb % p.stride_blocks == 0))
+    raise ValueError("unknown mode")
+
+
+def token_mask(p: Pattern, r0: int = 0, r1: Optional[int] = None) -> np.ndarray:
+    """Explicit boolean mask for query rows [r0, r1) against all L keys."""
+    r1 = p.L if r1 is None else r1
+    return allowed(p, np.arange(r0, r1)[:, None], np.arange(p.L)[None, :])
+
+
+def block_lists(p: Pattern):
+    """CSR and CSC lists of active blocks, derived from the explicit token mask.
+
+    Block (qb, kb) is active iff some allowed (i, j) lies inside it (Section 3.2: the
+    mask is kept in compressed-sparse-row form, one list shared by all heads).
+    Returns int32 arrays (row_ptr[nB+1], col_idx[nnz], col_ptr[nB+1], row_idx[nnz]);
+    rows ascending in kb, columns ascending in qb."""
+    Bs = p.block
+    nB = p.L // Bs
+    active = np.zeros((nB, nB), dtype=bool)
+
+    def one_block_row(qb):
+        m = token_mask(p, qb * Bs, (qb + 1) * Bs)                  # [Bs, L]
+        active[qb] = m.reshape(Bs, nB, Bs).any(axis=(0, 2))
+
+    # a plain parallel-for over block rows (numpy releases the GIL inside its loops)
+    with ThreadPoolExecutor(max_workers=os.cpu_count() or 1) as pool:
+        list(pool.map(one_block_row, range(nB)))
+    row_ptr = np.zeros(nB + 1, dtype=np.int32)
+    col_ptr = np.zeros(nB + 1, dtype=np.int32)
+    row_ptr[1:] = np.cumsum(active.sum(axis=1))
+    col_ptr[1:] = np.cumsum(active.sum(axis=0))
+    qb_i, kb_i = np.nonzero(active)            # row-major order: ascending qb, then kb
+    col_idx = kb_i.astype(np.int32)
+    kb_t, qb_t = np.nonzero(active.T)          # ascending kb, then qb
+    row_idx = qb_t.astype(np.int32)
+    return row_ptr, col_idx, col_ptr, row_idx
+
+
+def count_pairs(p: Pattern) -> int:
+    """Number of allowed (i, j) pairs for one head, counted from the explicit mask."""
+    Bs = p.block
+    with ThreadPoolExecutor(max_workers=os.cpu_count() or 1) as pool:
+        return sum(pool.map(lambda r0: int(token_mask(p, r0, r0 + Bs).sum()), range(0, p.L, Bs)))
+
+
+# ------------------------------------------------------------------------- forward
+
+def _softmax_rows(S: np.ndarray, M: np.ndarray):
+    """Masked softmax of score rows S under boolean mask M -> (P, LSE)."""
+    Sm = np.where(M, S, -np.inf)
+    mx = Sm.max(axis=1, keepdims=True)
+    E = np.where(M, np.exp(Sm - mx), 0.0)
+    Z = E.sum(axis=1, keepdims=True)
+    return E / Z, (mx + np.log(Z))[:, 0]
+
+
+def attn_forward(q, k, v, p: Pattern, scale: float, rows_per_slab: Optional[int] = None):
+    """O = softmax(scale*Q K^T + mask) V and LSE_i = log sum_j exp(scale*q_i.k_j).
+
+    q [Hq, L, D], k, v [Hkv, L, D] float64; query head h uses kv head h // (Hq/Hkv)
+    (grouped-query attention, Llama-2 70B).  Returns O [Hq, L, D], LSE [Hq, L].
+    rows_per_slab=None materialises the full L x L mask at once; otherwise rows are
+    taken a slab at a time and keys no row of the slab may see are dropped."""
+    Hq, L, D = q.shape
+    G = Hq // k.shape[0]
+    O = np.zeros_like(q)
+    LSE = np.zeros((Hq, L))
+    slab = L if rows_per_slab is None else rows_per_slab
+    for r0 in range(0, L, slab):
+        r1 = min(L, r0 + slab)
+        M = token_mask(p, r0, r1)
+        cols = np.nonzero(M.any(axis=0))[0]
+        Mc = M[:, cols]
+        for h in range(Hq):
+            S = scale * (q[h, r0:r1] @ k[h // G, cols].T)
+            P, lse = _softmax_rows(S, Mc)
+            O[h, r0:r1] = P @ v[h // G, cols]
+            LSE[h, r0:r1] = lse
+    return O, LSE
+
+
+def attn_backward(q, k, v, do, p: Pattern, scale: float, rows_per_slab: Optional[int] = None):
+    """Gradients of sum(O * dO) w.r.t. Q, K, V from the definition:
+
+      P = exp(S - LSE) on allowed pairs, 0 elsewhere;  dV_j = sum_i P_ij dO_i;
+      dP_ij = dO_i . v_j;  delta_i = sum_j P_ij dP_ij;  dS = P * (dP - delta);
+      dQ_i = scale * sum_j dS_ij k_j;  dK_j = scale * sum_i dS_ij q_i;
+      dK, dV of a kv head sum over the query heads of its group.
+
+    Returns (dQ [Hq,L,D], dK [Hkv,L,D], dV [Hkv,L,D], O, LSE)."""
+    Hq, L, D = q.shape
+    G = Hq // k.shape[0]
+    dQ = np.zeros_like(q)
+    dK = np.zeros_like(k)
+    dV = np.zeros_like(v)
+    O = np.zeros_like(q)
+    LSE = np.zeros((Hq, L))
+    slab = L if rows_per_slab is None else rows_per_slab
+    for r0 in range(0, L, slab):
+        r1 = min(L, r0 + slab)
+        M = token_mask(p, r0, r1)
+        cols = np.nonzero(M.any(axis=0))[0]
+        Mc = M[:, cols]
+        for h in range(Hq):
+            g = h // G
+            kc, vc = k[g, cols], v[g, cols]
+            S = scale * (q[h, r0:r1] @ kc.T)
+            P, lse = _softmax_rows(S, Mc)
+            O[h, r0:r1] = P @ vc
+            LSE[h, r0:r1] = lse
+            dOh = do[h, r0:r1]
+            dP = dOh @ vc.T
+            delta = (P * dP).sum(axis=1, keepdims=True)
+            dS = P * (dP - delta)
+            dQ[h, r0:r1] = scale * (dS @ kc)
+            dK[g, cols] += scale * (dS.T @ q[h, r0:r1])
+            dV[g, cols] += P.T @ dOh
+    return dQ, dK, dV, O, LSE
+
+
+# -------------------------------------------------------------------------- decode
+
+def decode_valid(n: int, sink: int, window: int) -> np.ndarray:
+    """Which of the first n tokens a sink + rolling-window cache still holds after n
+    appends (Section 3.2: rolling buffer for the window, sink kept beside it):
+    token j survives iff j < sink or it is among the last `window` tokens."""
+    j = np.arange(n)
+    return (j < sink) | (n - 1 - j < window)
+
+
+def decode(qv, k_lin, v_lin, n: int, sink: int, window: int, scale: float):
+    """One query token per head attends to the surviving tokens of a linear history.
+
+    qv [Hq, D]; k_lin, v_lin [Hkv, >=n, D] hold token j at index j (the oracle never
+    sees the ring layout).  Returns o [Hq, D], lse [Hq]; n == 0 gives o = 0, lse = -inf."""
+    Hq, D = qv.shape
+    G = Hq // k_lin.shape[0]
+    o = np.zeros((Hq, D))
+    lse = np.full(Hq, -np.inf)
+    if n == 0:
+        return o, lse
+    keep = np.nonzero(decode_valid(n, sink, window))[0]
+    for h in range(Hq):
+        s = scale * (k_lin[h // G, keep] @ qv[h])
+        mx = s.max()
+        e = np.exp(s - mx)
+        z = e.sum()
+        o[h] = (e / z) @ v_lin[h // G, keep]
+        lse[h] = mx + np.log(z)
+    return o, lse
+
+
+def ring_slot(j: int, sink: int, window: int) -> int:
+    """Cache slot of token j: sink tokens stay put, later ones roll (Mistral's
+    i mod W, offset past the sink)."""
+    return j if j < sink else sink + (j - sink) % window
+
+
+def ring_append_replay(cache: np.ndarray, new: np.ndarray, n_before: int, sink: int, window: int):
+    """Write tokens n_before, n_before+1, ... one at a time into `cache`
+    [sink+window, ...] in place; later writes overwrite earlier ones."""
+    for t in range(new.shape[0]):
+        cache[ring_slot(n_before + t, sink, window)] = new[t]
+    return cache

@@ -1,0 +1,417 @@
+"""Pins for the CPU oracle: each test ties it to something other than itself --
+numbers the paper prints, closed forms, textbook/library special cases, brute force
+on tiny inputs, finite differences.  No GPU needed."""
+import math
+
+import numpy as np
+import pytest
+import torch
+
+from oracle import lg_oracle as O
+from paper_2410_01485_b200 import synth
+
+
+def _read_kv(path):
+    out = {}
+    with open(path) as f:
+        for line in f:
+            line = line.split("#")[0].strip()
+            if line:
+                k, v = [s.strip() for s in line.split("=")]
+                out[k] = float(v)
+    return out
+
+
+def _rand(shape, seed):
+    return np.random.default_rng(seed).standard_normal(shape)
+
+
+TINY_PATTERNS = [
+    O.Pattern(L=32, block=4, mode=O.MODE_SINK_WINDOW, sink_tokens=4, window_tokens=8),
+    O.Pattern(L=32, block=4, mode=O.MODE_SINK_WINDOW, sink_tokens=8, window_tokens=4),
+    O.Pattern(L=48, block=8, mode=O.MODE_STRIDED_LOCAL, stride_blocks=2, local_blocks=1),
+    O.Pattern(L=40, block=4, mode=O.MODE_STRIDED_LOCAL, stride_blocks=3, local_blocks=2),
+    O.Pattern(L=24, block=8, mode=O.MODE_FULL_CAUSAL),
+]
+
+
+# ----------------------------------------------------------------- patterns / lists
+
+def test_paper_retained_tokens_and_kv_budget(golden_dir):
+    """Section 4.1 / 4.3: ~2K retained tokens per sparse layer at 128K; 69.2 GB -> 26.5 GB."""
+    g = _read_kv(golden_dir + "/paper_arithmetic.txt")
+    Bs, L = int(g["block_tokens"]), int(g["seq_len"])
+    sink = O.Pattern(L=L, block=Bs, mode=O.MODE_SINK_WINDOW, sink_tokens=int(g["sink_blocks"]) * Bs,
+                     window_tokens=int(g["local_blocks"]) * Bs)
+    last = O.allowed(sink, L - 1, np.arange(L))
+    assert last.sum() == (1 + 32) * 64 - 0  # last row of its block sees every retained token
+    assert abs(last.sum() - g["retained_tokens_approx"]) / g["retained_tokens_approx"] < 0.05
+    strided = O.Pattern(L=L, block=Bs, mode=O.MODE_STRIDED_LOCAL, stride_blocks=int(g["stride_blocks"]),
+                        local_blocks=1)
+    comb = O.allowed(strided, L - 1, np.arange(L))
+    # 2048 blocks / 64 = 32 comb blocks (+ the query's own block)
+    assert abs(comb.sum() - g["retained_tokens_approx"]) / g["retained_tokens_approx"] < 0.05
+    # KV bytes: what decode keeps per sparse layer is what the last query may see.
+    per_tok_layer = 2 * g["n_heads"] * g["head_dim"] * g["bytes_per_value"]
+    full_gb = g["n_layers"] * per_tok_layer * L / 1e9
+    assert abs(full_gb - g["kv_full_gb"]) / g["kv_full_gb"] < 0.01
+    n_sparse = g["n_layers"] - g["n_full_layers"]
+    kept = O.decode_valid(L, int(g["sink_blocks"]) * Bs, int(g["local_blocks"]) * Bs).sum()
+    assert kept == last.sum()
+    hybrid_gb = (g["n_full_layers"] * per_tok_layer * L + n_sparse * per_tok_layer * kept) / 1e9
+    assert abs(hybrid_gb - g["kv_hybrid_gb"]) < 0.06
+    assert abs(100 * (1 - hybrid_gb / full_gb) - g["kv_saving_pct"]) < 1.0
+
+
+def _nnz_closed_form(cfg):
+    nB = cfg.L // cfg.block
+    if cfg.mode == synth.MODE_FULL_CAUSAL:
+        return nB * (nB + 1) // 2
+    if cfg.mode == synth.MODE_SINK_WINDOW:
+        ns, nw = cfg.sink_tokens // cfg.block, cfg.window_tokens // cfg.block
+        return sum(min(qb + 1, nw) + min(ns, max(qb + 1 - nw, 0)) for qb in range(nB))
+    nl, s = cfg.local_blocks, cfg.stride_blocks
+    return sum(min(qb + 1, nl) + -(-max(qb - nl + 1, 0) // s) for qb in range(nB))
+
+
+@pytest.mark.parametrize("cfg", [synth.CFG1, synth.CFG2, synth.CFG2.full_causal()], ids=lambda c: c.name)
+def test_block_counts_match_closed_form(cfg, golden_dir):
+    g = _read_kv(golden_dir + "/block_counts.txt")
+    row_ptr, col_idx, col_ptr, row_idx = O.block_lists(O.Pattern.of(cfg))
+    assert int(row_ptr[-1]) == int(g[cfg.name]) == _nnz_closed_form(cfg)
+    assert len(col_idx) == len(row_idx) == int(g[cfg.name])
+
+
+def test_block_counts_golden_closed_forms_128k(golden_dir):
+    """The 128K entries of the fixture agree with the hand-derived row formulas (the
+    mask-derived lists at 128K are checked against the same numbers in the GPU tests)."""
+    g = _read_kv(golden_dir + "/block_counts.txt")
+    for cfg in (synth.CFG3, synth.CFG4, synth.PAPER_SINK):
+        assert _nnz_closed_form(cfg) == int(g[cfg.name])
+
+
+def test_block_counts_128k_scaled_down():
+    """Same patterns as the 128K configs at 1/8 of the length: counted from the mask."""
+    from dataclasses import replace
+    for cfg in (synth.CFG3, synth.CFG4, synth.PAPER_SINK, synth.PAPER_STRIDED):
+        small = replace(cfg, L=cfg.L // 8)
+        assert int(O.block_lists(O.Pattern.of(small))[0][-1]) == _nnz_closed_form(small)
+
+
+@pytest.mark.parametrize("p", TINY_PATTERNS)
+def test_lists_structure(p):
+    row_ptr, col_idx, col_ptr, row_idx = O.block_lists(p)
+    nB = p.L // p.block
+    dense = np.zeros((nB, nB), dtype=bool)
+    for qb in range(nB):
+        cols = col_idx[row_ptr[qb]:row_ptr[qb + 1]]
+        assert (np.diff(cols) > 0).all()            # ascending, no duplicates
+        assert cols[-1] == qb                       # diagonal block always active, nothing above it
+        dense[qb, cols] = True
+    # CSC is the exact transpose
+    dense_t = np.zeros((nB, nB), dtype=bool)
+    for kb in range(nB):
+        rows = row_idx[col_ptr[kb]:col_ptr[kb + 1]]
+        assert (np.diff(rows) > 0).all()
+        dense_t[rows, kb] = True
+    assert (dense == dense_t).all()
+    # brute force over token pairs with python loops
+    for qb in range(nB):
+        for kb in range(nB):
+            any_pair = any(bool(O.allowed(p, i, j)) for i in range(qb * p.block, (qb + 1) * p.block)
+                           for j in range(kb * p.block, (kb + 1) * p.block))
+            assert any_pair == dense[qb, kb]
+
+
+def test_sink_window_rows_are_sink_plus_contiguous_run():
+    """What a query sees under sink+window: the sink tokens and one contiguous run ending
+    at itself whose length lies in ((nw-1)*Bs, nw*Bs] (block-granular window, own block
+    counted) -- stated without the predicate's formula."""
+    p = O.Pattern(L=96, block=8, mode=O.MODE_SINK_WINDOW, sink_tokens=8, window_tokens=24)
+    M = O.token_mask(p)
+    for i in range(p.L):
+        seen = np.nonzero(M[i])[0]
+        assert seen[-1] == i and (seen <= i).all()
+        run = 1
+        while run < len(seen) and seen[-run - 1] == seen[-run] - 1:
+            run += 1
+        rest = seen[:-run]
+        if len(rest):                                  # the run does not reach the sink
+            assert list(rest) == list(range(8))
+            assert 16 < run <= 24
+            assert (i - run + 1) % 8 == 0              # run starts on a block boundary
+        else:
+            assert run == i + 1                        # everything up to i
+
+
+def test_strided_rows_keep_absolute_comb():
+    p = O.Pattern(L=128, block=8, mode=O.MODE_STRIDED_LOCAL, stride_blocks=4, local_blocks=2)
+    M = O.token_mask(p)
+    far = M[:, :]
+    for i in (40, 77, 127):
+        seen_blocks = sorted(set(np.nonzero(far[i])[0] // 8))
+        qb = i // 8
+        comb = [b for b in seen_blocks if b < qb - 1]
+        assert comb == [b for b in range(0, qb - 1) if b % 4 == 0]   # same comb for every query
+        assert seen_blocks[-2:] == [qb - 1, qb]
+
+
+def test_wide_window_is_full_causal():
+    L = 64
+    full = O.token_mask(O.Pattern(L=L, block=8, mode=O.MODE_FULL_CAUSAL))
+    assert (full == np.tril(np.ones((L, L), dtype=bool))).all()
+    assert (O.token_mask(O.Pattern(L=L, block=8, mode=O.MODE_SINK_WINDOW, sink_tokens=8, window_tokens=L)) == full).all()
+    assert (O.token_mask(O.Pattern(L=L, block=8, mode=O.MODE_STRIDED_LOCAL, stride_blocks=1, local_blocks=1)) == full).all()
+    assert (O.token_mask(O.Pattern(L=L, block=8, mode=O.MODE_STRIDED_LOCAL, stride_blocks=5, local_blocks=8)) == full).all()
+
+
+def test_pair_count_ratio_cfg3_scaled():
+    """Section 3.3: sparse-layer cost is a small fraction of dense when S << N.  For the
+    128K sink+window setting the exact pair ratio is 0.0625; at 1/8 length it is 8x that
+    minus edge effects -- compare the mask count with the closed form."""
+    from dataclasses import replace
+    cfg = replace(synth.CFG3, L=synth.CFG3.L // 8)
+    Bs, nB = cfg.block, cfg.L // cfg.block
+    ns, nw = 1, cfg.window_tokens // Bs
+    blocks_full = sum(min(qb + 1, nw) - 1 + min(ns, max(qb + 1 - nw, 0)) for qb in range(nB))
+    expect = blocks_full * Bs * Bs + nB * Bs * (Bs + 1) // 2
+    assert O.count_pairs(O.Pattern.of(cfg)) == expect
+    # the closed form at the full 128K length gives the 0.0625 of the measurement plan
+    nB = synth.CFG3.L // Bs
+    blocks_full = sum(min(qb + 1, nw) - 1 + min(ns, max(qb + 1 - nw, 0)) for qb in range(nB))
+    pairs = blocks_full * Bs * Bs + nB * Bs * (Bs + 1) // 2
+    assert pairs == 536674304
+    assert abs(pairs / (synth.CFG3.L * (synth.CFG3.L + 1) // 2) - 0.0625) < 5e-4
+
+
+# -------------------------------------------------------------------------- forward
+
+def _brute_forward_row(q, k, v, p, scale, h, g, i):
+    js = [j for j in range(p.L) if bool(O.allowed(p, i, j))]
+    s = [scale * sum(q[h, i, d] * k[g, j, d] for d in range(q.shape[2])) for j in js]
+    m = max(s)
+    e = [math.exp(x - m) for x in s]
+    z = sum(e)
+    o = [sum(e[t] / z * v[g, js[t], d] for t in range(len(js))) for d in range(q.shape[2])]
+    return o, m + math.log(z), e, z
+
+
+@pytest.mark.parametrize("p", TINY_PATTERNS)
+def test_forward_vs_bruteforce_rows(p):
+    Hq, Hkv, D = 4, 2, 5
+    q, k, v = _rand((Hq, p.L, D), 1), _rand((Hkv, p.L, D), 2), _rand((Hkv, p.L, D), 3)
+    scale = 0.37
+    Oo, LSE = O.attn_forward(q, k, v, p, scale)
+    for h in range(Hq):
+        for i in range(0, p.L, 3):
+            o, lse, _, _ = _brute_forward_row(q, k, v, p, scale, h, h // 2, i)
+            np.testing.assert_allclose(Oo[h, i], o, rtol=1e-12, atol=1e-13)
+            assert abs(LSE[h, i] - lse) < 1e-12
+
+
+def test_forward_full_causal_equals_torch_sdpa():
+    """Special case that reduces to a library routine: dense causal attention in fp64."""
+    Hq, Hkv, L, D = 4, 2, 48, 8
+    q, k, v = _rand((Hq, L, D), 4), _rand((Hkv, L, D), 5), _rand((Hkv, L, D), 6)
+    scale = 1 / math.sqrt(D)
+    tq, tk, tv = (torch.from_numpy(x) for x in (q, k, v))
+    ref = torch.nn.functional.scaled_dot_product_attention(
+        tq[None], tk.repeat_interleave(2, 0)[None], tv.repeat_interleave(2, 0)[None], is_causal=True, scale=scale)[0].numpy()
+    for p in (O.Pattern(L=L, block=8, mode=O.MODE_FULL_CAUSAL),
+              O.Pattern(L=L, block=8, mode=O.MODE_SINK_WINDOW, sink_tokens=8, window_tokens=L),
+              O.Pattern(L=L, block=8, mode=O.MODE_STRIDED_LOCAL, stride_blocks=1, local_blocks=1)):
+        got, lse = O.attn_forward(q, k, v, p, scale)
+        np.testing.assert_allclose(got, ref, rtol=1e-11, atol=1e-12)
+        # LSE against torch.logsumexp over the causal prefix
+        for h in (0, 3):
+            s = scale * (tq[h] @ tk[h // 2].T)
+            s = s.masked_fill(~torch.ones(L, L, dtype=torch.bool).tril(), float("-inf"))
+            np.testing.assert_allclose(lse[h], torch.logsumexp(s, dim=1).numpy(), rtol=1e-12)
+
+
+@pytest.mark.parametrize("p", TINY_PATTERNS)
+def test_forward_invariants(p):
+    Hq, Hkv, D = 2, 1, 6
+    q, k, v = _rand((Hq, p.L, D), 7), _rand((Hkv, p.L, D), 8), _rand((Hkv, p.L, D), 9)
+    scale = 0.5
+    Oo, LSE = O.attn_forward(q, k, v, p, scale)
+    # row 0 sees only key 0
+    np.testing.assert_allclose(Oo[:, 0], np.broadcast_to(v[0, 0], (Hq, D)), rtol=1e-13)
+    np.testing.assert_allclose(LSE[:, 0], scale * q[:, 0] @ k[0, 0], rtol=1e-13)
+    # LSE bounds: max <= LSE <= max + log(count)
+    M = O.token_mask(p)
+    for h in range(Hq):
+        S = np.where(M, scale * q[h] @ k[0].T, -np.inf)
+        assert (LSE[h] >= S.max(1) - 1e-12).all()
+        assert (LSE[h] <= S.max(1) + np.log(M.sum(1)) + 1e-12).all()
+        # rows of P = exp(S - LSE) sum to one
+        np.testing.assert_allclose(np.exp(S - LSE[h][:, None]).sum(1), 1.0, rtol=1e-12)
+    # all keys equal -> uniform weights -> O is the mean of the visible values
+    k_same = np.broadcast_to(k[:, :1], k.shape).copy()
+    O2, LSE2 = O.attn_forward(q, k_same, v, p, scale)
+    for i in (0, p.L // 2, p.L - 1):
+        np.testing.assert_allclose(O2[1, i], v[0, M[i]].mean(0), rtol=1e-12, atol=1e-13)
+        assert abs(LSE2[1, i] - (scale * q[1, i] @ k[0, 0] + math.log(M[i].sum()))) < 1e-12
+    # V = const vector -> O = that vector
+    v_const = np.broadcast_to(v[:, :1], v.shape).copy()
+    O3, _ = O.attn_forward(q, k, v_const, p, scale)
+    np.testing.assert_allclose(O3, np.broadcast_to(v[0, 0], O3.shape), rtol=1e-12)
+
+
+def test_masked_keys_do_not_influence_output():
+    p = O.Pattern(L=64, block=8, mode=O.MODE_SINK_WINDOW, sink_tokens=8, window_tokens=16)
+    q, k, v = _rand((1, 64, 4), 10), _rand((1, 64, 4), 11), _rand((1, 64, 4), 12)
+    O1, L1 = O.attn_forward(q, k, v, p, 0.5)
+    k2, v2 = k.copy(), v.copy()
+    k2[0, 8:16] += 100.0   # block 1: invisible to queries of blocks >= 3
+    v2[0, 8:16] -= 50.0
+    O2, L2 = O.attn_forward(q, k2, v2, p, 0.5)
+    assert (O1[0, 24:] == O2[0, 24:]).all() and (L1[0, 24:] == L2[0, 24:]).all()
+    assert not np.allclose(O1[0, 8:24], O2[0, 8:24])
+
+
+def test_slab_oracle_equals_dense_oracle():
+    for p in TINY_PATTERNS:
+        q, k, v, do = (_rand((4, p.L, 3), s) for s in (13, 14, 15, 16))
+        k, v = k[:2], v[:2]
+        a = O.attn_backward(q, k, v, do, p, 0.3)
+        b = O.attn_backward(q, k, v, do, p, 0.3, rows_per_slab=p.block)
+        c = O.attn_forward(q, k, v, p, 0.3, rows_per_slab=2 * p.block)
+        for x, y in zip(a, b):
+            np.testing.assert_allclose(x, y, rtol=1e-12, atol=1e-13)
+        np.testing.assert_allclose(a[3], c[0], rtol=1e-12, atol=1e-13)
+        np.testing.assert_allclose(a[4], c[1], rtol=1e-12, atol=1e-13)
+
+
+# ------------------------------------------------------------------------- backward
+
+def _loss(q, k, v, do, p, scale):
+    return float((O.attn_forward(q, k, v, p, scale)[0] * do).sum())
+
+
+@pytest.mark.parametrize("p", TINY_PATTERNS[:4])
+def test_backward_finite_differences(p):
+    Hq, Hkv, D = 2, 1, 3
+    q, k, v, do = _rand((Hq, p.L, D), 20), _rand((Hkv, p.L, D), 21), _rand((Hkv, p.L, D), 22), _rand((Hq, p.L, D), 23)
+    scale = 0.6
+    dQ, dK, dV, _, _ = O.attn_backward(q, k, v, do, p, scale)
+    rng = np.random.default_rng(0)
+    eps = 1e-5
+    for name, x, gx in (("q", q, dQ), ("k", k, dK), ("v", v, dV)):
+        for _ in range(12):
+            idx = tuple(rng.integers(0, s) for s in x.shape)
+            old = x[idx]
+            x[idx] = old + eps
+            up = _loss(q, k, v, do, p, scale)
+            x[idx] = old - eps
+            dn = _loss(q, k, v, do, p, scale)
+            x[idx] = old
+            fd = (up - dn) / (2 * eps)
+            assert abs(fd - gx[idx]) <= 1e-6 * max(1.0, abs(fd)), (name, idx, fd, gx[idx])
+
+
+@pytest.mark.parametrize("p", TINY_PATTERNS)
+def test_backward_equals_torch_autograd(p):
+    """Library autodiff of masked softmax attention in fp64 (GQA by repeat_interleave)."""
+    Hq, Hkv, D = 4, 2, 5
+    q, k, v, do = _rand((Hq, p.L, D), 30), _rand((Hkv, p.L, D), 31), _rand((Hkv, p.L, D), 32), _rand((Hq, p.L, D), 33)
+    scale = 0.45
+    tq, tk, tv = (torch.from_numpy(x).requires_grad_(True) for x in (q, k, v))
+    M = torch.from_numpy(O.token_mask(p))
+    s = scale * torch.einsum("hid,hjd->hij", tq, tk.repeat_interleave(2, 0))
+    pr = torch.softmax(s.masked_fill(~M, float("-inf")), dim=-1)
+    out = torch.einsum("hij,hjd->hid", pr, tv.repeat_interleave(2, 0))
+    (out * torch.from_numpy(do)).sum().backward()
+    dQ, dK, dV, Oo, _ = O.attn_backward(q, k, v, do, p, scale)
+    np.testing.assert_allclose(Oo, out.detach().numpy(), rtol=1e-11, atol=1e-12)
+    np.testing.assert_allclose(dQ, tq.grad.numpy(), rtol=1e-10, atol=1e-11)
+    np.testing.assert_allclose(dK, tk.grad.numpy(), rtol=1e-10, atol=1e-11)
+    np.testing.assert_allclose(dV, tv.grad.numpy(), rtol=1e-10, atol=1e-11)
+
+
+def test_backward_masked_keys_get_exactly_zero():
+    p = O.Pattern(L=64, block=8, mode=O.MODE_SINK_WINDOW, sink_tokens=8, window_tokens=16)
+    q, k, v, do = (_rand((2, 64, 4), s) for s in (40, 41, 42, 43))
+    do[:, :24] = 0.0      # only queries of blocks >= 3 carry gradient; they cannot see block 1
+    dQ, dK, dV, _, _ = O.attn_backward(q, k, v, do, p, 0.5)
+    assert (dK[:, 8:16] == 0).all() and (dV[:, 8:16] == 0).all()
+    assert np.abs(dK[:, 0:8]).max() > 0 and np.abs(dV[:, 16:24]).max() > 0
+    assert (dQ[:, :24] == 0).all()
+
+
+@pytest.mark.parametrize("p", TINY_PATTERNS)
+def test_backward_shift_invariances(p):
+    """softmax is invariant to adding one vector to every key, so sum_j dK_j = 0 per kv
+    head (a consequence of sum_j dS_ij = 0); and sum_j dV_j = sum_i dO_i per group."""
+    Hq, Hkv, D = 4, 2, 3
+    q, k, v, do = _rand((Hq, p.L, D), 50), _rand((Hkv, p.L, D), 51), _rand((Hkv, p.L, D), 52), _rand((Hq, p.L, D), 53)
+    dQ, dK, dV, _, _ = O.attn_backward(q, k, v, do, p, 0.7)
+    np.testing.assert_allclose(dK.sum(1), 0.0, atol=1e-11)
+    np.testing.assert_allclose(dV.sum(1), do.reshape(Hkv, 2, p.L, D).sum((1, 2)), rtol=1e-11)
+
+
+def test_backward_gqa_is_sum_of_mha_groups():
+    p = TINY_PATTERNS[3]
+    Hq, Hkv, D = 6, 2, 4
+    q, k, v, do = _rand((Hq, p.L, D), 60), _rand((Hkv, p.L, D), 61), _rand((Hkv, p.L, D), 62), _rand((Hq, p.L, D), 63)
+    dQ, dK, dV, _, _ = O.attn_backward(q, k, v, do, p, 0.5)
+    kr, vr = np.repeat(k, 3, axis=0), np.repeat(v, 3, axis=0)
+    dQm, dKm, dVm, _, _ = O.attn_backward(q, kr, vr, do, p, 0.5)
+    np.testing.assert_allclose(dQ, dQm, rtol=1e-12, atol=1e-13)
+    np.testing.assert_allclose(dK, dKm.reshape(Hkv, 3, p.L, D).sum(1), rtol=1e-12, atol=1e-13)
+    np.testing.assert_allclose(dV, dVm.reshape(Hkv, 3, p.L, D).sum(1), rtol=1e-12, atol=1e-13)
+
+
+# --------------------------------------------------------------------- decode / ring
+
+def test_decode_dense_equals_full_causal_last_row():
+    Hq, Hkv, n, D = 4, 2, 40, 8
+    q, k, v = _rand((Hq, n, D), 70), _rand((Hkv, n, D), 71), _rand((Hkv, n, D), 72)
+    Oo, LSE = O.attn_forward(q, k, v, O.Pattern(L=n, block=8, mode=O.MODE_FULL_CAUSAL), 0.35)
+    o, lse = O.decode(q[:, n - 1], k, v, n, sink=0, window=n, scale=0.35)
+    np.testing.assert_allclose(o, Oo[:, n - 1], rtol=1e-12)
+    np.testing.assert_allclose(lse, LSE[:, n - 1], rtol=1e-12)
+
+
+def test_decode_bruteforce_and_permutation_invariance():
+    Hq, Hkv, D, sink, W = 4, 2, 4, 3, 5
+    rng = np.random.default_rng(5)
+    for n in (1, 2, 3, 4, 8, 9, 23):
+        q, k, v = _rand((Hq, D), 80 + n), _rand((Hkv, n, D), 81 + n), _rand((Hkv, n, D), 82 + n)
+        o, lse = O.decode(q, k, v, n, sink, W, 0.5)
+        keep = [j for j in range(n) if j < sink or j >= n - W]
+        assert len(keep) == min(n, sink + W) or n - W < sink
+        for h in range(Hq):
+            s = [0.5 * float(q[h] @ k[h // 2, j]) for j in keep]
+            m = max(s)
+            z = sum(math.exp(x - m) for x in s)
+            ref = sum(math.exp(s[t] - m) / z * v[h // 2, keep[t]] for t in range(len(keep)))
+            np.testing.assert_allclose(o[h], ref, rtol=1e-12)
+            assert abs(lse[h] - (m + math.log(z))) < 1e-12
+        # a set function of the surviving (k, v) pairs: shuffle them inside the history
+        if n == 23:
+            perm = np.array(keep)
+            shuffled = rng.permutation(perm)
+            k2, v2 = k.copy(), v.copy()
+            k2[:, perm], v2[:, perm] = k[:, shuffled], v[:, shuffled]
+            o2, lse2 = O.decode(q, k2, v2, n, sink, W, 0.5)
+            np.testing.assert_allclose(o2, o, rtol=1e-12)
+    o0, lse0 = O.decode(_rand((Hq, D), 1), np.zeros((Hkv, 0, D)), np.zeros((Hkv, 0, D)), 0, sink, W, 0.5)
+    assert (o0 == 0).all() and np.isneginf(lse0).all()
+
+
+def test_ring_replay_holds_exactly_the_surviving_tokens():
+    sink, W = 3, 5
+    for n0, T in ((0, 1), (0, 4), (2, 3), (0, 8), (5, 20), (7, 1), (0, 31)):
+        cache = np.full((sink + W, 1), -1.0)
+        # history before: tokens 0..n0-1 appended one by one
+        O.ring_append_replay(cache, np.arange(n0, dtype=float)[:, None], 0, sink, W)
+        O.ring_append_replay(cache, np.arange(n0, n0 + T, dtype=float)[:, None], n0, sink, W)
+        n = n0 + T
+        held = sorted(int(x) for x in cache[:, 0] if x >= 0)
+        assert held == list(np.nonzero(O.decode_valid(n, sink, W))[0])
+        # every surviving token sits where the slot rule says, each slot holds one token
+        for j in held:
+            assert cache[O.ring_slot(j, sink, W), 0] == j
+        # sink slots never move; the ring holds the last W non-sink tokens
+        assert all(cache[j, 0] == j for j in range(min(n, sink)))
