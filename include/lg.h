@@ -1,0 +1,156 @@
+/*
+ * lg.h -- C ABI of the LongGen efficient-layer attention library for NVIDIA B200 (sm_100a).
+ *
+ * The library implements the attention of LongGen's sparse layers (paper Section 3.1: a
+ * static, block-wise pattern that is the same for every head -- attention sink plus
+ * sliding window, or blockwise strided plus local blocks), the plain causal attention of
+ * its full layers, and the serving side of Section 3.2 (a rolling-buffer KV cache for the
+ * window with the sink kept beside it, and a bandwidth-bound decode over it).
+ *
+ * Conventions for every entry point
+ *   - Pointers named in a signature as device pointers are device memory OWNED BY THE
+ *     CALLER; the library allocates nothing that outlives a call and keeps no state
+ *     between calls except what it writes into the caller's workspace.
+ *   - `stream` is a cudaStream_t (0 = default stream).  Calls enqueue work and return;
+ *     the return value covers validation and launch only.  A device-side wait that gave
+ *     up (every wait in the kernels is bounded) is reported by lg_last_status().
+ *   - All tensors are bf16 with the head dimension D contiguous; device pointers must be
+ *     16-byte aligned.  Results are bitwise reproducible for fixed inputs and parameters.
+ *   - No exception crosses this boundary.  A call with invalid arguments launches nothing.
+ */
+#ifndef LG_H_
+#define LG_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum {
+  LG_OK = 0,
+  LG_ERR_INVALID_ARG = -1,    /* null / misaligned pointer, inconsistent sizes              */
+  LG_ERR_UNSUPPORTED = -2,    /* valid problem outside what the kernels cover (e.g. D)      */
+  LG_ERR_WORKSPACE = -3,      /* workspace_bytes smaller than the matching *_workspace_bytes */
+  LG_ERR_CUDA = -4,           /* a CUDA runtime / driver call failed                         */
+  LG_ERR_DEVICE_TIMEOUT = -5, /* a bounded device-side wait expired (see lg_last_status)     */
+  LG_ERR_ARCH = -6            /* current device is not compute capability 10.x               */
+} lg_status;
+
+typedef enum {
+  LG_MODE_FULL_CAUSAL = 0,   /* key j visible to query i iff j <= i (the full-attention layers)  */
+  LG_MODE_SINK_WINDOW = 1,   /* Section 3.1 "Attention Sink": first blocks + most recent blocks   */
+  LG_MODE_STRIDED_LOCAL = 2  /* Section 3.1 "block sparse": every stride-th block + local blocks  */
+} lg_mode;
+
+/*
+ * Problem statement of one attention call (Sections 3.1 and 4.1).
+ * With Bs = block, qb = i / Bs, kb = j / Bs, query i may attend key j iff j <= i and
+ *   FULL_CAUSAL   : (nothing more)
+ *   SINK_WINDOW   : kb < sink_tokens/Bs  or  qb - kb < window_tokens/Bs
+ *                   (the window is block-granular and counts the query's own block:
+ *                    "the first block for sink tokens and the most recent 32 blocks")
+ *   STRIDED_LOCAL : qb - kb < local_blocks  or  kb % stride_blocks == 0
+ * Grouped-query attention: query head h reads kv head h / (Hq / Hkv).
+ */
+typedef struct {
+  int32_t B, Hq, Hkv, L, D;   /* Hq % Hkv == 0; D in {64, 128}; L % block == 0               */
+  int32_t block;              /* pattern granularity in tokens: 64 or 128                    */
+  int32_t mode;               /* lg_mode                                                     */
+  int32_t sink_tokens;        /* SINK_WINDOW: multiple of block (may be 0)                   */
+  int32_t window_tokens;      /* SINK_WINDOW: multiple of block, >= block                    */
+  int32_t stride_blocks;      /* STRIDED_LOCAL: >= 1                                         */
+  int32_t local_blocks;       /* STRIDED_LOCAL: >= 1 (the diagonal block is always active)   */
+  float   scale;              /* softmax scale; 0 selects 1/sqrt(D)                          */
+  /* Strides in ELEMENTS of (batch, head, token) for Q, K, V, O; dO and dQ use the O / Q
+     strides, dK / dV the K / V strides.  All zero selects contiguous [B, H, L, D].
+     Every stride must be a multiple of 8 elements (16 bytes).                              */
+  int64_t q_strides[3], k_strides[3], v_strides[3], o_strides[3];
+} lg_attn_params;
+
+/* ---- block-index builder (Section 3.2: the mask is kept in compressed-sparse-row form,
+ *      O(N) memory, static for all heads) ---------------------------------------------- */
+
+/* Number of active blocks (nnz) of the pattern, computed on the host; < 0 = lg_status. */
+int64_t lg_block_index_nnz(const lg_attn_params* p);
+
+/* Bytes needed for the four int32 arrays below, laid out back to back:
+ * row_ptr[nB+1], col_idx[nnz], col_ptr[nB+1], row_idx[nnz] (nB = L / block). 0 on error. */
+size_t lg_block_index_bytes(const lg_attn_params* p);
+
+/* Fill the CSR lists (for each query block, the ascending KV blocks it attends) and the
+ * CSC transpose (for each KV block, the ascending query blocks that attend it).
+ * All four arrays are DEVICE int32 arrays of the sizes above, written by a kernel on
+ * `stream`.  nnz_out_host (HOST, nullable) receives nnz.                                 */
+lg_status lg_build_block_index(const lg_attn_params* p, int32_t* row_ptr, int32_t* col_idx,
+                               int32_t* col_ptr, int32_t* row_idx, int64_t* nnz_out_host,
+                               void* stream);
+
+/* ---- training / prefill attention (Section 3.2: FlashAttention-style kernel that skips
+ *      every block whose mask is zero, in the forward and in the backward) -------------- */
+
+/* Workspace bytes for lg_sparse_attn_fwd (want_bwd == 0) or lg_sparse_attn_bwd (!= 0). */
+size_t lg_sparse_attn_workspace_bytes(const lg_attn_params* p, int want_bwd);
+
+/* O = softmax(scale * Q K^T + mask) V;  LSE_i = ln sum_j exp(scale * q_i . k_j) over the
+ * visible keys.  q [B,Hq,L,D], k, v [B,Hkv,L,D], o [B,Hq,L,D] bf16 (device);
+ * lse [B,Hq,L] fp32 contiguous (device).  workspace: device, 256-byte aligned.           */
+lg_status lg_sparse_attn_fwd(const lg_attn_params* p, const void* q, const void* k, const void* v,
+                             void* o, float* lse, void* workspace, size_t workspace_bytes,
+                             void* stream);
+
+/* Gradients of sum(O * dO): dq [B,Hq,L,D], dk, dv [B,Hkv,L,D] bf16 (device), from the
+ * forward's inputs, its outputs o and lse, and d_o [B,Hq,L,D] bf16.  dK and dV of a kv head
+ * are summed over the query heads of its group.  Keys a query may not see receive exactly
+ * zero from it.  Accumulation order is fixed (no atomics).                               */
+lg_status lg_sparse_attn_bwd(const lg_attn_params* p, const void* q, const void* k, const void* v,
+                             const void* o, const float* lse, const void* d_o,
+                             void* dq, void* dk, void* dv,
+                             void* workspace, size_t workspace_bytes, void* stream);
+
+/* ---- serving: rolling-buffer cache and decode (Section 3.2) --------------------------- */
+
+/*
+ * Cache layout: K and V each [B, Hkv, sink_tokens + window_tokens, D] bf16, contiguous.
+ * Token j of a sequence lives in slot(j) = j < sink ? j : sink + (j - sink) % window.
+ * A plain linear cache of `cap` tokens is sink_tokens = 0, window_tokens = cap.
+ */
+typedef struct {
+  int32_t B, Hq, Hkv, D;       /* D in {64, 128}; Hq % Hkv == 0                              */
+  int32_t sink_tokens;         /* >= 0                                                       */
+  int32_t window_tokens;       /* >= 1                                                       */
+  float   scale;               /* 0 selects 1/sqrt(D)                                        */
+} lg_decode_params;
+
+/* Append T_new tokens per sequence: k_new, v_new [B, Hkv, T_new, D] bf16 (device);
+ * n_tokens_before (device int64 [B]) = tokens already appended to each sequence.  The
+ * result equals appending one token at a time; writes that a later token of the same
+ * call would overwrite are skipped.                                                      */
+lg_status lg_kv_ring_append(const lg_decode_params* p, void* k_cache, void* v_cache,
+                            const void* k_new, const void* v_new, int32_t T_new,
+                            const int64_t* n_tokens_before, void* stream);
+
+size_t lg_sparse_decode_workspace_bytes(const lg_decode_params* p);
+
+/* One query token per sequence attends to every valid slot of its cache:
+ * q [B,Hq,D], o [B,Hq,D] bf16; n_tokens (device int64 [B]) counts the tokens appended so
+ * far, the current one included; slots holding no token yet are ignored; n_tokens == 0
+ * gives o = 0, lse = -inf.  lse [B,Hq] fp32 is optional (NULL to skip).                 */
+lg_status lg_sparse_decode(const lg_decode_params* p, const void* q, const void* k_cache,
+                           const void* v_cache, const int64_t* n_tokens, void* o, float* lse,
+                           void* workspace, size_t workspace_bytes, void* stream);
+
+/* ---- status ------------------------------------------------------------------------- */
+
+/* Synchronises `stream`, reads the error word the kernels keep at the start of
+ * `workspace` (attention or decode workspace) and clears it.  LG_OK, or
+ * LG_ERR_DEVICE_TIMEOUT if a bounded wait expired in a kernel that used it.              */
+lg_status lg_last_status(void* workspace, void* stream);
+
+const char* lg_status_string(lg_status s);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* LG_H_ */

@@ -1,0 +1,210 @@
+"""Thin ctypes binding of the C-ABI library (argument marshalling only).
+
+PyTorch supplies device memory and streams; every step of the attention path runs in
+the library's CUDA kernels.  There is no CPU fallback: if the shared library is missing
+or the device is not sm_100, calls raise.
+"""
+from __future__ import annotations
+
+import ctypes as C
+import os
+from typing import Optional, Tuple
+
+import torch
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(_HERE, "liblg_sparse_attn.so")
+
+LG_OK = 0
+MODE_FULL_CAUSAL, MODE_SINK_WINDOW, MODE_STRIDED_LOCAL = 0, 1, 2
+
+
+class LgError(RuntimeError):
+    def __init__(self, code: int, what: str):
+        super().__init__("%s failed: %s (%d)" % (what, status_string(code), code))
+        self.code = code
+
+
+class AttnParams(C.Structure):
+    _fields_ = [("B", C.c_int32), ("Hq", C.c_int32), ("Hkv", C.c_int32), ("L", C.c_int32), ("D", C.c_int32),
+                ("block", C.c_int32), ("mode", C.c_int32), ("sink_tokens", C.c_int32),
+                ("window_tokens", C.c_int32), ("stride_blocks", C.c_int32), ("local_blocks", C.c_int32),
+                ("scale", C.c_float),
+                ("q_strides", C.c_int64 * 3), ("k_strides", C.c_int64 * 3), ("v_strides", C.c_int64 * 3),
+                ("o_strides", C.c_int64 * 3)]
+
+
+class DecodeParams(C.Structure):
+    _fields_ = [("B", C.c_int32), ("Hq", C.c_int32), ("Hkv", C.c_int32), ("D", C.c_int32),
+                ("sink_tokens", C.c_int32), ("window_tokens", C.c_int32), ("scale", C.c_float)]
+
+
+_lib = None
+
+# every symbol include/lg.h declares: (restype, argtypes)
+_vp, _sz = C.c_void_p, C.c_size_t
+SYMBOLS = {
+    "lg_block_index_nnz": (C.c_int64, [C.POINTER(AttnParams)]),
+    "lg_block_index_bytes": (_sz, [C.POINTER(AttnParams)]),
+    "lg_build_block_index": (C.c_int, [C.POINTER(AttnParams), _vp, _vp, _vp, _vp, C.POINTER(C.c_int64), _vp]),
+    "lg_sparse_attn_workspace_bytes": (_sz, [C.POINTER(AttnParams), C.c_int]),
+    "lg_sparse_attn_fwd": (C.c_int, [C.POINTER(AttnParams), _vp, _vp, _vp, _vp, _vp, _vp, _sz, _vp]),
+    "lg_sparse_attn_bwd": (C.c_int, [C.POINTER(AttnParams)] + [_vp] * 9 + [_vp, _sz, _vp]),
+    "lg_kv_ring_append": (C.c_int, [C.POINTER(DecodeParams), _vp, _vp, _vp, _vp, C.c_int32, _vp, _vp]),
+    "lg_sparse_decode_workspace_bytes": (_sz, [C.POINTER(DecodeParams)]),
+    "lg_sparse_decode": (C.c_int, [C.POINTER(DecodeParams), _vp, _vp, _vp, _vp, _vp, _vp, _vp, _sz, _vp]),
+    "lg_last_status": (C.c_int, [_vp, _vp]),
+    "lg_status_string": (C.c_char_p, [C.c_int]),
+}
+
+
+def load_library() -> C.CDLL:
+    """Load the in-tree shared library; raises if it has not been built."""
+    global _lib
+    if _lib is None:
+        if not os.path.exists(LIB_PATH):
+            raise RuntimeError("CUDA library %s is missing: run `python -m paper_2410_01485_b200.build` "
+                               "(there is no CPU fallback)" % LIB_PATH)
+        lib = C.CDLL(LIB_PATH)
+        for name, (res, args) in SYMBOLS.items():
+            fn = getattr(lib, name)
+            fn.restype, fn.argtypes = res, args
+        _lib = lib
+    return _lib
+
+
+def status_string(code: int) -> str:
+    return load_library().lg_status_string(code).decode()
+
+
+def _check(code: int, what: str):
+    if code != LG_OK:
+        raise LgError(code, what)
+
+
+def _stream() -> int:
+    return torch.cuda.current_stream().cuda_stream
+
+
+def _strides3(t: torch.Tensor):
+    assert t.dim() == 4 and t.stride(3) == 1, "expect [B, H, L, D] with contiguous D"
+    return (C.c_int64 * 3)(t.stride(0), t.stride(1), t.stride(2))
+
+
+def attn_params(B, Hq, Hkv, L, D, block, mode, sink_tokens=0, window_tokens=0, stride_blocks=0, local_blocks=0,
+                scale=0.0) -> AttnParams:
+    p = AttnParams()
+    p.B, p.Hq, p.Hkv, p.L, p.D, p.block, p.mode = B, Hq, Hkv, L, D, block, mode
+    p.sink_tokens, p.window_tokens, p.stride_blocks, p.local_blocks = sink_tokens, window_tokens, stride_blocks, local_blocks
+    p.scale = scale
+    return p
+
+
+def params_of(cfg, scale: float = 0.0) -> AttnParams:
+    """AttnParams from a synth.AttnConfig-like object."""
+    return attn_params(cfg.B, cfg.Hq, cfg.Hkv, cfg.L, cfg.D, cfg.block, cfg.mode, cfg.sink_tokens,
+                       cfg.window_tokens, cfg.stride_blocks, cfg.local_blocks, scale)
+
+
+# ------------------------------------------------------------------------------ index
+
+def lg_block_index_nnz(p: AttnParams) -> int:
+    n = load_library().lg_block_index_nnz(C.byref(p))
+    if n < 0:
+        raise LgError(int(n), "lg_block_index_nnz")
+    return int(n)
+
+
+def lg_build_block_index(p: AttnParams, device="cuda") -> Tuple[torch.Tensor, torch.Tensor, torch.Tensor, torch.Tensor]:
+    """Returns device int32 tensors (row_ptr, col_idx, col_ptr, row_idx)."""
+    lib = load_library()
+    nnz = lg_block_index_nnz(p)
+    nB = p.L // p.block
+    assert lib.lg_block_index_bytes(C.byref(p)) == 4 * (2 * (nB + 1) + 2 * nnz)
+    row_ptr = torch.empty(nB + 1, dtype=torch.int32, device=device)
+    col_ptr = torch.empty(nB + 1, dtype=torch.int32, device=device)
+    col_idx = torch.empty(max(nnz, 1), dtype=torch.int32, device=device)
+    row_idx = torch.empty(max(nnz, 1), dtype=torch.int32, device=device)
+    out = C.c_int64(-1)
+    _check(lib.lg_build_block_index(C.byref(p), row_ptr.data_ptr(), col_idx.data_ptr(), col_ptr.data_ptr(),
+                                    row_idx.data_ptr(), C.byref(out), _stream()), "lg_build_block_index")
+    assert out.value == nnz
+    return row_ptr, col_idx[:nnz], col_ptr, row_idx[:nnz]
+
+
+# ------------------------------------------------------------------------- fwd / bwd
+
+def attn_workspace(p: AttnParams, want_bwd: bool, device="cuda") -> torch.Tensor:
+    n = load_library().lg_sparse_attn_workspace_bytes(C.byref(p), int(want_bwd))
+    if n == 0:
+        raise LgError(-1, "lg_sparse_attn_workspace_bytes")
+    return torch.empty(n, dtype=torch.uint8, device=device)
+
+
+def lg_sparse_attn_fwd(p: AttnParams, q, k, v, o=None, lse=None, workspace=None):
+    """q [B,Hq,L,D], k, v [B,Hkv,L,D] bf16 CUDA tensors -> (o bf16, lse fp32 [B,Hq,L])."""
+    lib = load_library()
+    o = torch.empty_like(q) if o is None else o
+    lse = torch.empty(q.shape[:3], dtype=torch.float32, device=q.device) if lse is None else lse
+    ws = attn_workspace(p, False, q.device) if workspace is None else workspace
+    p.q_strides, p.k_strides, p.v_strides, p.o_strides = _strides3(q), _strides3(k), _strides3(v), _strides3(o)
+    _check(lib.lg_sparse_attn_fwd(C.byref(p), q.data_ptr(), k.data_ptr(), v.data_ptr(), o.data_ptr(),
+                                  lse.data_ptr(), ws.data_ptr(), ws.numel(), _stream()), "lg_sparse_attn_fwd")
+    return o, lse
+
+
+def lg_sparse_attn_bwd(p: AttnParams, q, k, v, o, lse, d_o, dq=None, dk=None, dv=None, workspace=None):
+    """Gradients (dq, dk, dv) bf16 of sum(O * dO)."""
+    lib = load_library()
+    dq = torch.empty_like(q) if dq is None else dq
+    dk = torch.empty_like(k) if dk is None else dk
+    dv = torch.empty_like(v) if dv is None else dv
+    ws = attn_workspace(p, True, q.device) if workspace is None else workspace
+    assert d_o.stride() == o.stride() and dq.stride() == q.stride()
+    assert dk.stride() == k.stride() and dv.stride() == v.stride()
+    p.q_strides, p.k_strides, p.v_strides, p.o_strides = _strides3(q), _strides3(k), _strides3(v), _strides3(o)
+    _check(lib.lg_sparse_attn_bwd(C.byref(p), q.data_ptr(), k.data_ptr(), v.data_ptr(), o.data_ptr(),
+                                  lse.data_ptr(), d_o.data_ptr(), dq.data_ptr(), dk.data_ptr(), dv.data_ptr(),
+                                  ws.data_ptr(), ws.numel(), _stream()), "lg_sparse_attn_bwd")
+    return dq, dk, dv
+
+
+# ---------------------------------------------------------------------- decode / ring
+
+def decode_params(B, Hq, Hkv, D, sink_tokens, window_tokens, scale=0.0) -> DecodeParams:
+    p = DecodeParams()
+    p.B, p.Hq, p.Hkv, p.D, p.sink_tokens, p.window_tokens, p.scale = B, Hq, Hkv, D, sink_tokens, window_tokens, scale
+    return p
+
+
+def lg_kv_ring_append(p: DecodeParams, k_cache, v_cache, k_new, v_new, n_tokens_before):
+    """Append k_new, v_new [B,Hkv,T,D] in place; n_tokens_before int64 device [B]."""
+    assert k_cache.is_contiguous() and v_cache.is_contiguous() and k_new.is_contiguous() and v_new.is_contiguous()
+    _check(load_library().lg_kv_ring_append(C.byref(p), k_cache.data_ptr(), v_cache.data_ptr(), k_new.data_ptr(),
+                                            v_new.data_ptr(), k_new.shape[2], n_tokens_before.data_ptr(),
+                                            _stream()), "lg_kv_ring_append")
+
+
+def decode_workspace(p: DecodeParams, device="cuda") -> torch.Tensor:
+    n = load_library().lg_sparse_decode_workspace_bytes(C.byref(p))
+    if n == 0:
+        raise LgError(-1, "lg_sparse_decode_workspace_bytes")
+    return torch.empty(n, dtype=torch.uint8, device=device)
+
+
+def lg_sparse_decode(p: DecodeParams, q, k_cache, v_cache, n_tokens, o=None, lse=None, workspace=None,
+                     want_lse: bool = True):
+    """q [B,Hq,D] bf16 -> (o [B,Hq,D] bf16, lse [B,Hq] fp32 or None)."""
+    assert q.is_contiguous() and k_cache.is_contiguous() and v_cache.is_contiguous()
+    o = torch.empty_like(q) if o is None else o
+    if lse is None and want_lse:
+        lse = torch.empty(q.shape[:2], dtype=torch.float32, device=q.device)
+    ws = decode_workspace(p, q.device) if workspace is None else workspace
+    _check(load_library().lg_sparse_decode(C.byref(p), q.data_ptr(), k_cache.data_ptr(), v_cache.data_ptr(),
+                                           n_tokens.data_ptr(), o.data_ptr(), lse.data_ptr() if lse is not None else None,
+                                           ws.data_ptr(), ws.numel(), _stream()), "lg_sparse_decode")
+    return o, lse
+
+
+def lg_last_status(workspace: torch.Tensor) -> int:
+    return int(load_library().lg_last_status(workspace.data_ptr(), _stream()))

@@ -1,0 +1,282 @@
+// C-ABI entry points: validation, workspace layout, block-index builder launches.
+#include <math.h>
+#include <string.h>
+
+#include <mutex>
+
+#include "lg_common.cuh"
+#include "lg_host.h"
+#include "lg_index.cuh"
+
+namespace lg {
+
+lg_status check_arch() {
+  int dev = 0, major = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess) return LG_ERR_CUDA;
+  if (cudaDeviceGetAttribute(&major, cudaDevAttrComputeCapabilityMajor, dev) != cudaSuccess) return LG_ERR_CUDA;
+  return major == 10 ? LG_OK : LG_ERR_ARCH;
+}
+
+static bool strides_all_zero(const int64_t s[3]) { return s[0] == 0 && s[1] == 0 && s[2] == 0; }
+
+static lg_status fix_strides(const int64_t in[3], int H, int L, int D, int64_t out[3]) {
+  if (strides_all_zero(in)) {
+    out[2] = D;
+    out[1] = static_cast<int64_t>(L) * D;
+    out[0] = static_cast<int64_t>(H) * L * D;
+    return LG_OK;
+  }
+  for (int i = 0; i < 3; ++i) {
+    if (in[i] <= 0 || in[i] % 8 != 0) return LG_ERR_INVALID_ARG;
+    out[i] = in[i];
+  }
+  if (out[2] < D) return LG_ERR_INVALID_ARG;
+  return LG_OK;
+}
+
+lg_status resolve(const lg_attn_params* p, Resolved* r) {
+  if (!p || !r) return LG_ERR_INVALID_ARG;
+  if (p->B < 1 || p->Hq < 1 || p->Hkv < 1 || p->L < 1 || p->Hq % p->Hkv != 0) return LG_ERR_INVALID_ARG;
+  if (p->block != 64 && p->block != 128) return LG_ERR_INVALID_ARG;
+  if (p->L % p->block != 0) return LG_ERR_INVALID_ARG;
+  if (p->D != 64 && p->D != 128) return LG_ERR_UNSUPPORTED;
+  if (!(p->scale >= 0.f) || isinf(p->scale)) return LG_ERR_INVALID_ARG;
+  r->B = p->B; r->Hq = p->Hq; r->Hkv = p->Hkv; r->L = p->L; r->D = p->D; r->block = p->block;
+  r->mode = p->mode; r->G = p->Hq / p->Hkv;
+  r->pat.nB = p->L / p->block;
+  r->pat.mode = p->mode;
+  r->pat.ns = r->pat.nw = r->pat.stride = r->pat.nl = 0;
+  switch (p->mode) {
+    case LG_MODE_FULL_CAUSAL:
+      break;
+    case LG_MODE_SINK_WINDOW:
+      if (p->sink_tokens < 0 || p->sink_tokens % p->block != 0) return LG_ERR_INVALID_ARG;
+      if (p->window_tokens < p->block || p->window_tokens % p->block != 0) return LG_ERR_INVALID_ARG;
+      r->pat.ns = p->sink_tokens / p->block;
+      r->pat.nw = p->window_tokens / p->block;
+      break;
+    case LG_MODE_STRIDED_LOCAL:
+      if (p->stride_blocks < 1 || p->local_blocks < 1) return LG_ERR_INVALID_ARG;
+      r->pat.stride = p->stride_blocks;
+      r->pat.nl = p->local_blocks;
+      break;
+    default:
+      return LG_ERR_INVALID_ARG;
+  }
+  r->scale = p->scale > 0.f ? p->scale : 1.0f / sqrtf(static_cast<float>(p->D));
+  lg_status s;
+  if ((s = fix_strides(p->q_strides, p->Hq, p->L, p->D, r->qs)) != LG_OK) return s;
+  if ((s = fix_strides(p->k_strides, p->Hkv, p->L, p->D, r->ks)) != LG_OK) return s;
+  if ((s = fix_strides(p->v_strides, p->Hkv, p->L, p->D, r->vs)) != LG_OK) return s;
+  if ((s = fix_strides(p->o_strides, p->Hq, p->L, p->D, r->os)) != LG_OK) return s;
+  r->n_qtiles = (p->L + 127) / 128;
+  r->n_ktiles = (p->L + 127) / 128;
+  // nnz from the per-row counts of each pattern
+  int64_t nnz = 0;
+  const PatternDev& pt = r->pat;
+  for (int qb = 0; qb < pt.nB; ++qb) {
+    if (pt.mode == 0) {
+      nnz += qb + 1;
+    } else if (pt.mode == 1) {
+      const int win = qb + 1 < pt.nw ? qb + 1 : pt.nw;
+      const int below = qb + 1 - win;           // blocks older than the window
+      nnz += win + (pt.ns < below ? pt.ns : below);
+    } else {
+      const int loc = qb + 1 < pt.nl ? qb + 1 : pt.nl;
+      const int below = qb + 1 - loc;
+      nnz += loc + (below + pt.stride - 1) / pt.stride;
+    }
+  }
+  r->nnz = nnz;
+  if (nnz > 0x3fffffff || pt.nB > (1 << 20)) return LG_ERR_UNSUPPORTED;
+  return LG_OK;
+}
+
+WsLayout ws_layout(const Resolved& r, bool want_bwd) {
+  WsLayout w{};
+  size_t off = sizeof(WsHeader);
+  auto take = [&](size_t bytes) {
+    size_t o = off;
+    off = align_up(off + bytes, 256);
+    return o;
+  };
+  const size_t nB = r.pat.nB, nnz = static_cast<size_t>(r.nnz);
+  w.row_ptr = take((nB + 1) * 4);
+  w.col_idx = take(nnz * 4);
+  w.col_ptr = take((nB + 1) * 4);
+  w.row_idx = take(nnz * 4);
+  w.qt_cnt = take(r.n_qtiles * 4);
+  w.qt_ent = take(nnz * 4);
+  w.qt_order = take(r.n_qtiles * 4);
+  if (want_bwd) {
+    w.kt_cnt = take(r.n_ktiles * 4);
+    w.kt_ent = take(nnz * 4);
+    w.kt_order = take(r.n_ktiles * 4);
+    w.delta = take(static_cast<size_t>(r.B) * r.Hq * r.L * 4);
+  }
+  w.total = off;
+  return w;
+}
+
+lg_status launch_index_build(const Resolved& r, int32_t* row_ptr, int32_t* col_idx, int32_t* col_ptr,
+                             int32_t* row_idx, cudaStream_t stream) {
+  const int nB = r.pat.nB;
+  index_count_kernel<<<nB, 128, 0, stream>>>(r.pat, row_ptr, col_ptr);
+  index_scan_kernel<<<2, 1024, 0, stream>>>(row_ptr, col_ptr, nB);
+  index_fill_kernel<<<nB, 64, 0, stream>>>(r.pat, row_ptr, col_idx, col_ptr, row_idx);
+  return cudaGetLastError() == cudaSuccess ? LG_OK : LG_ERR_CUDA;
+}
+
+lg_status prepare_workspace(const Resolved& r, const WsLayout& w, uint8_t* ws, bool want_bwd,
+                            cudaStream_t stream) {
+  if (cudaMemsetAsync(ws, 0, sizeof(WsHeader), stream) != cudaSuccess) return LG_ERR_CUDA;
+  auto i32 = [&](size_t off) { return reinterpret_cast<int32_t*>(ws + off); };
+  lg_status s = launch_index_build(r, i32(w.row_ptr), i32(w.col_idx), i32(w.col_ptr), i32(w.row_idx), stream);
+  if (s != LG_OK) return s;
+  const int R = 128 / r.block;
+  tile_merge_kernel<<<(r.n_qtiles + 127) / 128, 128, 0, stream>>>(i32(w.row_ptr), i32(w.col_idx), r.pat.nB, R,
+                                                                  r.n_qtiles, i32(w.qt_cnt), i32(w.qt_ent));
+  tile_order_kernel<<<(r.n_qtiles + 127) / 128, 128, 0, stream>>>(i32(w.qt_cnt), r.n_qtiles, i32(w.qt_order));
+  if (want_bwd) {
+    tile_merge_kernel<<<(r.n_ktiles + 127) / 128, 128, 0, stream>>>(i32(w.col_ptr), i32(w.row_idx), r.pat.nB, R,
+                                                                    r.n_ktiles, i32(w.kt_cnt), i32(w.kt_ent));
+    tile_order_kernel<<<(r.n_ktiles + 127) / 128, 128, 0, stream>>>(i32(w.kt_cnt), r.n_ktiles, i32(w.kt_order));
+  }
+  return cudaGetLastError() == cudaSuccess ? LG_OK : LG_ERR_CUDA;
+}
+
+// ---- tensor maps ---------------------------------------------------------------------
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
+                                  const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
+                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+static EncodeTiledFn get_encode_fn() {
+  static EncodeTiledFn fn = nullptr;
+  static std::once_flag once;
+  std::call_once(once, [] {
+    void* p = nullptr;
+    cudaDriverEntryPointQueryResult qres;
+    if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &qres) == cudaSuccess &&
+        qres == cudaDriverEntryPointSuccess)
+      fn = reinterpret_cast<EncodeTiledFn>(p);
+  });
+  return fn;
+}
+
+lg_status make_tmap(CUtensorMap* out, const void* base, int B, int H, int L, int D, const int64_t strides[3],
+                    int box_rows) {
+  EncodeTiledFn fn = get_encode_fn();
+  if (!fn) return LG_ERR_CUDA;
+  cuuint64_t dims[4] = {static_cast<cuuint64_t>(D), static_cast<cuuint64_t>(L), static_cast<cuuint64_t>(H),
+                        static_cast<cuuint64_t>(B)};
+  cuuint64_t gstr[3] = {static_cast<cuuint64_t>(strides[2]) * 2, static_cast<cuuint64_t>(strides[1]) * 2,
+                        static_cast<cuuint64_t>(strides[0]) * 2};
+  cuuint32_t box[4] = {64, static_cast<cuuint32_t>(box_rows), 1, 1};
+  cuuint32_t estr[4] = {1, 1, 1, 1};
+  CUresult rc = fn(out, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 4, const_cast<void*>(base), dims, gstr, box, estr,
+                   CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                   CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+  return rc == CUDA_SUCCESS ? LG_OK : LG_ERR_CUDA;
+}
+
+}  // namespace lg
+
+using namespace lg;
+
+extern "C" {
+
+int64_t lg_block_index_nnz(const lg_attn_params* p) {
+  Resolved r;
+  lg_status s = resolve(p, &r);
+  return s == LG_OK ? r.nnz : static_cast<int64_t>(s);
+}
+
+size_t lg_block_index_bytes(const lg_attn_params* p) {
+  Resolved r;
+  if (resolve(p, &r) != LG_OK) return 0;
+  return (2 * (static_cast<size_t>(r.pat.nB) + 1) + 2 * static_cast<size_t>(r.nnz)) * sizeof(int32_t);
+}
+
+lg_status lg_build_block_index(const lg_attn_params* p, int32_t* row_ptr, int32_t* col_idx, int32_t* col_ptr,
+                               int32_t* row_idx, int64_t* nnz_out_host, void* stream) {
+  Resolved r;
+  lg_status s = resolve(p, &r);
+  if (s != LG_OK) return s;
+  if (!row_ptr || !col_idx || !col_ptr || !row_idx) return LG_ERR_INVALID_ARG;
+  if ((reinterpret_cast<uintptr_t>(row_ptr) | reinterpret_cast<uintptr_t>(col_idx) |
+       reinterpret_cast<uintptr_t>(col_ptr) | reinterpret_cast<uintptr_t>(row_idx)) & 3)
+    return LG_ERR_INVALID_ARG;
+  if (nnz_out_host) *nnz_out_host = r.nnz;
+  return launch_index_build(r, row_ptr, col_idx, col_ptr, row_idx, static_cast<cudaStream_t>(stream));
+}
+
+size_t lg_sparse_attn_workspace_bytes(const lg_attn_params* p, int want_bwd) {
+  Resolved r;
+  if (resolve(p, &r) != LG_OK) return 0;
+  return ws_layout(r, want_bwd != 0).total;
+}
+
+lg_status lg_sparse_attn_fwd(const lg_attn_params* p, const void* q, const void* k, const void* v, void* o,
+                             float* lse, void* workspace, size_t workspace_bytes, void* stream) {
+  Resolved r;
+  lg_status s = resolve(p, &r);
+  if (s != LG_OK) return s;
+  if (!q || !k || !v || !o || !lse || !workspace) return LG_ERR_INVALID_ARG;
+  if (!aligned16(q) || !aligned16(k) || !aligned16(v) || !aligned16(o) || !aligned16(lse)) return LG_ERR_INVALID_ARG;
+  if (reinterpret_cast<uintptr_t>(workspace) & 255) return LG_ERR_INVALID_ARG;
+  const WsLayout w = ws_layout(r, false);
+  if (workspace_bytes < w.total) return LG_ERR_WORKSPACE;
+  if ((s = check_arch()) != LG_OK) return s;
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  uint8_t* ws = static_cast<uint8_t*>(workspace);
+  if ((s = prepare_workspace(r, w, ws, false, st)) != LG_OK) return s;
+  return launch_fwd(r, w, q, k, v, o, lse, ws, st);
+}
+
+lg_status lg_sparse_attn_bwd(const lg_attn_params* p, const void* q, const void* k, const void* v, const void* o,
+                             const float* lse, const void* d_o, void* dq, void* dk, void* dv, void* workspace,
+                             size_t workspace_bytes, void* stream) {
+  Resolved r;
+  lg_status s = resolve(p, &r);
+  if (s != LG_OK) return s;
+  if (!q || !k || !v || !o || !lse || !d_o || !dq || !dk || !dv || !workspace) return LG_ERR_INVALID_ARG;
+  if (!aligned16(q) || !aligned16(k) || !aligned16(v) || !aligned16(o) || !aligned16(lse) || !aligned16(d_o) ||
+      !aligned16(dq) || !aligned16(dk) || !aligned16(dv))
+    return LG_ERR_INVALID_ARG;
+  if (reinterpret_cast<uintptr_t>(workspace) & 255) return LG_ERR_INVALID_ARG;
+  const WsLayout w = ws_layout(r, true);
+  if (workspace_bytes < w.total) return LG_ERR_WORKSPACE;
+  if ((s = check_arch()) != LG_OK) return s;
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  uint8_t* ws = static_cast<uint8_t*>(workspace);
+  if ((s = prepare_workspace(r, w, ws, true, st)) != LG_OK) return s;
+  return launch_bwd(r, w, q, k, v, o, lse, d_o, dq, dk, dv, ws, st);
+}
+
+lg_status lg_last_status(void* workspace, void* stream) {
+  if (!workspace) return LG_ERR_INVALID_ARG;
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  if (cudaStreamSynchronize(st) != cudaSuccess) return LG_ERR_CUDA;
+  unsigned int word = 0;
+  if (cudaMemcpy(&word, workspace, sizeof(word), cudaMemcpyDeviceToHost) != cudaSuccess) return LG_ERR_CUDA;
+  if (word != 0) {
+    if (cudaMemset(workspace, 0, sizeof(word)) != cudaSuccess) return LG_ERR_CUDA;
+    return LG_ERR_DEVICE_TIMEOUT;
+  }
+  return LG_OK;
+}
+
+const char* lg_status_string(lg_status s) {
+  switch (s) {
+    case LG_OK: return "ok";
+    case LG_ERR_INVALID_ARG: return "invalid argument";
+    case LG_ERR_UNSUPPORTED: return "unsupported problem";
+    case LG_ERR_WORKSPACE: return "workspace too small";
+    case LG_ERR_CUDA: return "CUDA call failed";
+    case LG_ERR_DEVICE_TIMEOUT: return "a bounded device-side wait expired";
+    case LG_ERR_ARCH: return "device is not sm_100";
+  }
+  return "unknown status";
+}
+
+}  // extern "C"

@@ -1,0 +1,88 @@
+// Launch of the backward attention kernels: delta pre-pass, dK/dV pass, dQ pass.
+#include "lg_bwd.cuh"
+#include "lg_host.h"
+
+namespace lg {
+
+template <int D, int BS>
+static lg_status launch_bwd_t(const Resolved& r, const WsLayout& w, const void* q, const void* k, const void* v,
+                              const void* o, const float* lse, const void* d_o, void* dq, void* dk, void* dv,
+                              uint8_t* ws, cudaStream_t stream) {
+  lg_status s;
+  float* delta = reinterpret_cast<float*>(ws + w.delta);
+  {
+    const int64_t rows = static_cast<int64_t>(r.B) * r.Hq * r.L;
+    const int64_t threads = rows * (D / 8);
+    const int64_t blocks = (threads + 255) / 256;
+    if (blocks > 0x7fffffff) return LG_ERR_UNSUPPORTED;
+    delta_kernel<D><<<static_cast<unsigned>(blocks), 256, 0, stream>>>(
+        static_cast<const __nv_bfloat16*>(o), static_cast<const __nv_bfloat16*>(d_o), delta, r.os[0], r.os[1],
+        r.os[2], r.Hq, r.L, rows);
+  }
+  BwdArgs a;
+  a.lse = lse;
+  a.delta = delta;
+  a.error_word = reinterpret_cast<unsigned int*>(ws);
+  a.L = r.L; a.Hq = r.Hq; a.Hkv = r.Hkv; a.G = r.G;
+  a.scale = r.scale;
+  a.scale_log2 = r.scale * 1.4426950408889634f;
+  constexpr int smem = BwdSmem<D, BS>::kTotal;
+
+  // ---- dK / dV pass -------------------------------------------------------------------
+  {
+    CUtensorMap tq, tk, tv, tdo;
+    if ((s = make_tmap(&tq, q, r.B, r.Hq, r.L, D, r.qs, BS)) != LG_OK) return s;
+    if ((s = make_tmap(&tdo, d_o, r.B, r.Hq, r.L, D, r.os, BS)) != LG_OK) return s;
+    if ((s = make_tmap(&tk, k, r.B, r.Hkv, r.L, D, r.ks, 128)) != LG_OK) return s;
+    if ((s = make_tmap(&tv, v, r.B, r.Hkv, r.L, D, r.vs, 128)) != LG_OK) return s;
+    a.tile_off = reinterpret_cast<const int32_t*>(ws + w.col_ptr);
+    a.tile_cnt = reinterpret_cast<const int32_t*>(ws + w.kt_cnt);
+    a.tile_ent = reinterpret_cast<const int32_t*>(ws + w.kt_ent);
+    a.order = reinterpret_cast<const int32_t*>(ws + w.kt_order);
+    a.out0 = static_cast<__nv_bfloat16*>(dk);
+    a.out1 = static_cast<__nv_bfloat16*>(dv);
+    for (int i = 0; i < 3; ++i) { a.s0[i] = r.ks[i]; a.s1[i] = r.vs[i]; }
+    auto kern = bwd_dkdv_kernel<D, BS>;
+    if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, smem) != cudaSuccess)
+      return LG_ERR_CUDA;
+    dim3 grid(r.B * r.Hkv, r.n_ktiles);
+    kern<<<grid, 128, smem, stream>>>(tq, tk, tv, tdo, a);
+  }
+  // ---- dQ pass ------------------------------------------------------------------------
+  {
+    CUtensorMap tq, tk, tv, tdo;
+    if ((s = make_tmap(&tq, q, r.B, r.Hq, r.L, D, r.qs, 128)) != LG_OK) return s;
+    if ((s = make_tmap(&tdo, d_o, r.B, r.Hq, r.L, D, r.os, 128)) != LG_OK) return s;
+    if ((s = make_tmap(&tk, k, r.B, r.Hkv, r.L, D, r.ks, BS)) != LG_OK) return s;
+    if ((s = make_tmap(&tv, v, r.B, r.Hkv, r.L, D, r.vs, BS)) != LG_OK) return s;
+    a.tile_off = reinterpret_cast<const int32_t*>(ws + w.row_ptr);
+    a.tile_cnt = reinterpret_cast<const int32_t*>(ws + w.qt_cnt);
+    a.tile_ent = reinterpret_cast<const int32_t*>(ws + w.qt_ent);
+    a.order = reinterpret_cast<const int32_t*>(ws + w.qt_order);
+    a.out0 = static_cast<__nv_bfloat16*>(dq);
+    a.out1 = nullptr;
+    for (int i = 0; i < 3; ++i) { a.s0[i] = r.qs[i]; a.s1[i] = 0; }
+    auto kern = bwd_dq_kernel<D, BS>;
+    if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, smem) != cudaSuccess)
+      return LG_ERR_CUDA;
+    dim3 grid(r.B * r.Hq, r.n_qtiles);
+    kern<<<grid, 128, smem, stream>>>(tq, tk, tv, tdo, a);
+  }
+  return cudaGetLastError() == cudaSuccess ? LG_OK : LG_ERR_CUDA;
+}
+
+lg_status launch_bwd(const Resolved& r, const WsLayout& w, const void* q, const void* k, const void* v,
+                     const void* o, const float* lse, const void* d_o, void* dq, void* dk, void* dv, uint8_t* ws,
+                     cudaStream_t stream) {
+  if (r.n_qtiles > 65535) return LG_ERR_UNSUPPORTED;
+#define LG_BWD_CASE(DD, BB) \
+  if (r.D == DD && r.block == BB) return launch_bwd_t<DD, BB>(r, w, q, k, v, o, lse, d_o, dq, dk, dv, ws, stream);
+  LG_BWD_CASE(128, 128)
+  LG_BWD_CASE(128, 64)
+  LG_BWD_CASE(64, 128)
+  LG_BWD_CASE(64, 64)
+#undef LG_BWD_CASE
+  return LG_ERR_UNSUPPORTED;
+}
+
+}  // namespace lg

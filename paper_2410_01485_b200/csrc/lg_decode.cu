@@ -1,0 +1,412 @@
+// Serving side of the paper's Section 3.2: a rolling-buffer KV cache for the sliding window
+// with the sink kept beside it, and a single-token decode whose only job is to stream that
+// cache from HBM as fast as possible.
+//
+// Decode layout: one CTA per (sequence, kv head, head group of <= 8 query heads, KV split).
+// Each of its 4 warps owns a contiguous run of 16-token tiles and keeps a private cp.async
+// pipeline of kStages tiles (16-byte copies into XOR-swizzled shared memory, so the HBM
+// stream never waits on arithmetic).  Scores are S^T = K Q^T and the output is
+// O^T = V^T P^T, both on mma.sync m16n8k16 (bf16 in, fp32 accumulate) with the 8 query heads
+// of the group as the N dimension, so all heads of a GQA group share every byte loaded.
+// Per-split (max, sum, O) partials go to the workspace and a second kernel merges them in
+// split order, which keeps the result bitwise reproducible.
+#include <math.h>
+
+#include "lg_common.cuh"
+#include "lg_host.h"
+
+namespace lg {
+
+constexpr int kDecWarps = 4;
+constexpr int kDecStages = 3;
+constexpr int kDecTile = 16;          // tokens per warp tile
+constexpr int kDecHeads = 8;          // query heads per CTA (mma N)
+
+struct DecodeArgs {
+  const __nv_bfloat16* q;        // [B, Hq, D]
+  const __nv_bfloat16* k_cache;  // [B, Hkv, C, D]
+  const __nv_bfloat16* v_cache;
+  const int64_t* n_tokens;       // [B]
+  float* part;                   // [B, Hkv*HG, nsplit, 8 heads, (D + 2)] : O, m, l
+  __nv_bfloat16* o;              // [B, Hq, D]
+  float* lse;                    // [B, Hq] or null
+  int Hq, Hkv, G, HG, C, nsplit;
+  float scale_log2;
+};
+
+__device__ __forceinline__ void cp_async16(uint32_t smem_addr, const void* gptr, bool valid) {
+  const int sz = valid ? 16 : 0;
+  asm volatile("cp.async.cg.shared.global [%0], [%1], 16, %2;" ::"r"(smem_addr), "l"(gptr), "r"(sz) : "memory");
+}
+__device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commit_group;" ::: "memory"); }
+template <int N>
+__device__ __forceinline__ void cp_async_wait() {
+  asm volatile("cp.async.wait_group %0;" ::"n"(N) : "memory");
+}
+__device__ __forceinline__ void ldsm_x4(uint32_t addr, uint32_t& r0, uint32_t& r1, uint32_t& r2, uint32_t& r3) {
+  asm volatile("ldmatrix.sync.aligned.m8n8.x4.shared.b16 {%0, %1, %2, %3}, [%4];"
+               : "=r"(r0), "=r"(r1), "=r"(r2), "=r"(r3)
+               : "r"(addr));
+}
+__device__ __forceinline__ void ldsm_x4_t(uint32_t addr, uint32_t& r0, uint32_t& r1, uint32_t& r2, uint32_t& r3) {
+  asm volatile("ldmatrix.sync.aligned.m8n8.x4.trans.shared.b16 {%0, %1, %2, %3}, [%4];"
+               : "=r"(r0), "=r"(r1), "=r"(r2), "=r"(r3)
+               : "r"(addr));
+}
+__device__ __forceinline__ uint32_t movmatrix_t(uint32_t x) {
+  uint32_t y;
+  asm volatile("movmatrix.sync.aligned.m8n8.trans.b16 %0, %1;" : "=r"(y) : "r"(x));
+  return y;
+}
+__device__ __forceinline__ void mma16816(float* c, uint32_t a0, uint32_t a1, uint32_t a2, uint32_t a3, uint32_t b0,
+                                         uint32_t b1) {
+  asm volatile(
+      "mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0, %1, %2, %3}, {%4, %5, %6, %7}, {%8, %9}, "
+      "{%0, %1, %2, %3};"
+      : "+f"(c[0]), "+f"(c[1]), "+f"(c[2]), "+f"(c[3])
+      : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1));
+}
+
+template <int D>
+__global__ void __launch_bounds__(kDecWarps * 32) decode_split_kernel(const DecodeArgs a) {
+  constexpr int kRowBytes = D * 2;
+  constexpr int kChunks = D / 8;                      // 16-byte chunks per row
+  constexpr int kTileBytes = kDecTile * kRowBytes;    // K (or V) bytes of one tile
+  constexpr int kCopiesPerLane = kDecTile * kChunks / 32;
+  extern __shared__ __align__(128) uint8_t dsmem[];
+
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int split = blockIdx.x, kg = blockIdx.y, b = blockIdx.z;
+  const int kvh = kg / a.HG, hg = kg % a.HG;
+  const int r = lane >> 2, c = lane & 3;
+
+  const int64_t n = a.n_tokens[b];
+  const int nvalid = static_cast<int>(n < a.C ? (n < 0 ? 0 : n) : a.C);
+  const int ntile = (nvalid + kDecTile - 1) / kDecTile;
+  const int wg = split * kDecWarps + warp, nw = a.nsplit * kDecWarps;
+  const int t_begin = static_cast<int>(static_cast<int64_t>(ntile) * wg / nw);
+  const int t_end = static_cast<int>(static_cast<int64_t>(ntile) * (wg + 1) / nw);
+
+  uint8_t* wsm = dsmem + warp * (kDecStages * 2 * kTileBytes);
+  const uint32_t wsm_u32 = smem_u32(wsm);
+  const uint8_t* kbase = reinterpret_cast<const uint8_t*>(a.k_cache) +
+                         (static_cast<int64_t>(b) * a.Hkv + kvh) * static_cast<int64_t>(a.C) * kRowBytes;
+  const uint8_t* vbase = reinterpret_cast<const uint8_t*>(a.v_cache) +
+                         (static_cast<int64_t>(b) * a.Hkv + kvh) * static_cast<int64_t>(a.C) * kRowBytes;
+
+  auto issue_tile = [&](int t) {
+    const int stage = (t - t_begin) % kDecStages;
+    const uint32_t sk = wsm_u32 + stage * 2 * kTileBytes, sv = sk + kTileBytes;
+    const int slot0 = t * kDecTile;
+#pragma unroll
+    for (int it = 0; it < kCopiesPerLane; ++it) {
+      const int ch = it * 32 + lane;
+      const int row = ch / kChunks, cc = ch % kChunks;
+      const bool valid = slot0 + row < nvalid;
+      const int64_t goff = static_cast<int64_t>(valid ? slot0 + row : 0) * kRowBytes + cc * 16;
+      const uint32_t soff = row * kRowBytes + ((cc ^ (row & 7)) * 16);
+      cp_async16(sk + soff, kbase + goff, valid);
+      cp_async16(sv + soff, vbase + goff, valid);
+    }
+  };
+
+  // Q^T fragments: b0 = Q[head r][16k + 2c, +1], b1 = Q[head r][16k + 8 + 2c, +1]
+  uint32_t qf[D / 16][2];
+  {
+    const int head = hg * kDecHeads + r;
+    const bool on = head < a.G;
+    const uint32_t* qrow = reinterpret_cast<const uint32_t*>(
+        a.q + (static_cast<int64_t>(b) * a.Hq + kvh * a.G + (on ? head : 0)) * D);
+#pragma unroll
+    for (int k = 0; k < D / 16; ++k) {
+      qf[k][0] = on ? qrow[8 * k + c] : 0u;
+      qf[k][1] = on ? qrow[8 * k + 4 + c] : 0u;
+    }
+  }
+
+  float m_run[2] = {-INFINITY, -INFINITY};   // heads 2c, 2c+1 (scaled log2 domain), warp-uniform per head
+  float l_run[2] = {0.f, 0.f};               // this thread's share of the row sums
+  float oacc[D / 16][4];
+#pragma unroll
+  for (int i = 0; i < D / 16; ++i) oacc[i][0] = oacc[i][1] = oacc[i][2] = oacc[i][3] = 0.f;
+
+#pragma unroll
+  for (int s = 0; s < kDecStages - 1; ++s) {
+    if (t_begin + s < t_end) issue_tile(t_begin + s);
+    cp_async_commit();
+  }
+
+  for (int t = t_begin; t < t_end; ++t) {
+    cp_async_wait<kDecStages - 2>();
+    __syncwarp();
+    const int stage = (t - t_begin) % kDecStages;
+    const uint32_t sk = wsm_u32 + stage * 2 * kTileBytes, sv = sk + kTileBytes;
+
+    // ---- S^T[16 tokens, 8 heads] = K Q^T ------------------------------------------------
+    float sacc[4] = {0.f, 0.f, 0.f, 0.f};
+    {
+      const int row = ((lane >> 3) & 1) * 8 + (lane & 7);
+#pragma unroll
+      for (int k = 0; k < D / 16; ++k) {
+        const int cc = 2 * k + (lane >> 4);
+        uint32_t a0, a1, a2, a3;
+        ldsm_x4(sk + row * kRowBytes + ((cc ^ (row & 7)) * 16), a0, a1, a2, a3);
+        mma16816(sacc, a0, a1, a2, a3, qf[k][0], qf[k][1]);
+      }
+    }
+    // sacc[0,1]: token r, heads 2c, 2c+1;  sacc[2,3]: token r + 8
+    const int tok0 = t * kDecTile + r;
+    const bool v0 = tok0 < nvalid, v1 = tok0 + 8 < nvalid;
+    float s00 = v0 ? sacc[0] * a.scale_log2 : -INFINITY, s01 = v0 ? sacc[1] * a.scale_log2 : -INFINITY;
+    float s10 = v1 ? sacc[2] * a.scale_log2 : -INFINITY, s11 = v1 ? sacc[3] * a.scale_log2 : -INFINITY;
+    float mx0 = fmaxf(s00, s10), mx1 = fmaxf(s01, s11);
+#pragma unroll
+    for (int o = 4; o < 32; o <<= 1) {
+      mx0 = fmaxf(mx0, __shfl_xor_sync(0xffffffffu, mx0, o));
+      mx1 = fmaxf(mx1, __shfl_xor_sync(0xffffffffu, mx1, o));
+    }
+    const float mn0 = fmaxf(m_run[0], mx0), mn1 = fmaxf(m_run[1], mx1);
+    const float mu0 = mn0 == -INFINITY ? 0.f : mn0, mu1 = mn1 == -INFINITY ? 0.f : mn1;
+    const float al0 = fast_exp2(m_run[0] - mu0), al1 = fast_exp2(m_run[1] - mu1);
+    m_run[0] = mn0; m_run[1] = mn1;
+    const float p00 = fast_exp2(s00 - mu0), p01 = fast_exp2(s01 - mu1);
+    const float p10 = fast_exp2(s10 - mu0), p11 = fast_exp2(s11 - mu1);
+    l_run[0] = l_run[0] * al0 + p00 + p10;
+    l_run[1] = l_run[1] * al1 + p01 + p11;
+    if (__any_sync(0xffffffffu, al0 != 1.f || al1 != 1.f)) {
+#pragma unroll
+      for (int i = 0; i < D / 16; ++i) {
+        oacc[i][0] *= al0; oacc[i][1] *= al1; oacc[i][2] *= al0; oacc[i][3] *= al1;
+      }
+    }
+    // P^T as the B operand: transpose the two 8x8 (token x head) fragments across the warp
+    const uint32_t pb0 = movmatrix_t(pack_bf16(p00, p01));   // tokens 2c, 2c+1 of head r
+    const uint32_t pb1 = movmatrix_t(pack_bf16(p10, p11));   // tokens 8 + 2c, +1
+
+    // ---- O^T[D, 8 heads] += V^T P^T ----------------------------------------------------
+    {
+      const int row = (lane >> 4) * 8 + (lane & 7);
+#pragma unroll
+      for (int i = 0; i < D / 16; ++i) {
+        const int cc = 2 * i + ((lane >> 3) & 1);
+        uint32_t a0, a1, a2, a3;
+        ldsm_x4_t(sv + row * kRowBytes + ((cc ^ (row & 7)) * 16), a0, a1, a2, a3);
+        mma16816(oacc[i], a0, a1, a2, a3, pb0, pb1);
+      }
+    }
+    __syncwarp();
+    if (t + kDecStages - 1 < t_end) issue_tile(t + kDecStages - 1);
+    cp_async_commit();
+  }
+  cp_async_wait<0>();
+
+  // ---- warp partial -> shared, then merge the 4 warps in warp order -----------------------
+#pragma unroll
+  for (int o = 4; o < 32; o <<= 1) {
+    l_run[0] += __shfl_xor_sync(0xffffffffu, l_run[0], o);
+    l_run[1] += __shfl_xor_sync(0xffffffffu, l_run[1], o);
+  }
+  __syncthreads();                       // everyone is done with the pipeline buffers
+  float* red = reinterpret_cast<float*>(dsmem);          // [warp][head 8][D + 2]
+  constexpr int kRec = D + 2;
+  {
+    float* mine = red + warp * kDecHeads * kRec;
+#pragma unroll
+    for (int i = 0; i < D / 16; ++i) {
+      mine[(2 * c) * kRec + 16 * i + r] = oacc[i][0];
+      mine[(2 * c + 1) * kRec + 16 * i + r] = oacc[i][1];
+      mine[(2 * c) * kRec + 16 * i + 8 + r] = oacc[i][2];
+      mine[(2 * c + 1) * kRec + 16 * i + 8 + r] = oacc[i][3];
+    }
+    if (r == 0) {
+      mine[(2 * c) * kRec + D] = m_run[0];
+      mine[(2 * c) * kRec + D + 1] = l_run[0];
+      mine[(2 * c + 1) * kRec + D] = m_run[1];
+      mine[(2 * c + 1) * kRec + D + 1] = l_run[1];
+    }
+  }
+  __syncthreads();
+  float* out = a.part + ((static_cast<int64_t>(b) * gridDim.y + kg) * a.nsplit + split) * (kDecHeads * kRec);
+  for (int idx = threadIdx.x; idx < kDecHeads * D; idx += blockDim.x) {
+    const int head = idx / D, d = idx % D;
+    float m = -INFINITY;
+#pragma unroll
+    for (int w = 0; w < kDecWarps; ++w) m = fmaxf(m, red[(w * kDecHeads + head) * kRec + D]);
+    const float mu = m == -INFINITY ? 0.f : m;
+    float acc = 0.f, l = 0.f;
+#pragma unroll
+    for (int w = 0; w < kDecWarps; ++w) {
+      const float f = fast_exp2(red[(w * kDecHeads + head) * kRec + D] - mu);
+      acc += f * red[(w * kDecHeads + head) * kRec + d];
+      l += f * red[(w * kDecHeads + head) * kRec + D + 1];
+    }
+    out[head * kRec + d] = acc;
+    if (d == 0) { out[head * kRec + D] = m; out[head * kRec + D + 1] = l; }
+  }
+}
+
+// grid = (B * Hkv * HG); 128 threads.  Merges the splits in ascending order.
+template <int D>
+__global__ void __launch_bounds__(128) decode_merge_kernel(const DecodeArgs a) {
+  constexpr int kRec = D + 2;
+  const int kg = blockIdx.x % (a.Hkv * a.HG), b = blockIdx.x / (a.Hkv * a.HG);
+  const int kvh = kg / a.HG, hg = kg % a.HG;
+  const float* part = a.part + (static_cast<int64_t>(b) * (a.Hkv * a.HG) + kg) * a.nsplit * (kDecHeads * kRec);
+  for (int idx = threadIdx.x; idx < kDecHeads * D; idx += blockDim.x) {
+    const int head = idx / D, d = idx % D;
+    const int gh = hg * kDecHeads + head;
+    if (gh >= a.G) continue;
+    float m = -INFINITY;
+    for (int s = 0; s < a.nsplit; ++s) m = fmaxf(m, part[(s * kDecHeads + head) * kRec + D]);
+    const float mu = m == -INFINITY ? 0.f : m;
+    float acc = 0.f, l = 0.f;
+    for (int s = 0; s < a.nsplit; ++s) {
+      const float f = fast_exp2(part[(s * kDecHeads + head) * kRec + D] - mu);
+      acc += f * part[(s * kDecHeads + head) * kRec + d];
+      l += f * part[(s * kDecHeads + head) * kRec + D + 1];
+    }
+    const int64_t qh = static_cast<int64_t>(b) * a.Hq + kvh * a.G + gh;
+    a.o[qh * D + d] = __float2bfloat16(l > 0.f ? acc / l : 0.f);
+    if (d == 0 && a.lse) a.lse[qh] = l > 0.f ? (m + log2f(l)) * 0.6931471805599453f : -INFINITY;
+  }
+}
+
+// ---- ring append ------------------------------------------------------------------------
+// slot(j) = j < sink ? j : sink + (j - sink) % window.  One group of D/8 threads copies one
+// K row and one V row (16 bytes per thread per row).  A token that a later token of the same
+// call would overwrite is skipped, so the outcome equals appending one at a time.
+__global__ void ring_append_kernel(__nv_bfloat16* k_cache, __nv_bfloat16* v_cache, const __nv_bfloat16* k_new,
+                                   const __nv_bfloat16* v_new, const int64_t* n_before, int B, int Hkv, int D, int T,
+                                   int sink, int window) {
+  const int per_row = D / 8;
+  const int64_t gid = static_cast<int64_t>(blockIdx.x) * blockDim.x + threadIdx.x;
+  const int64_t row_id = gid / per_row;
+  const int ch = static_cast<int>(gid % per_row);
+  const int64_t total_rows = static_cast<int64_t>(B) * Hkv * T;
+  if (row_id >= total_rows) return;
+  const int t = static_cast<int>(row_id % T);
+  const int64_t bh = row_id / T;
+  const int b = static_cast<int>(bh / Hkv);
+  const int64_t n0 = n_before[b];
+  const int64_t j = n0 + t, last = n0 + T - 1;
+  if (j >= sink && j + window <= last) return;       // overwritten later in this call
+  const int64_t slot = j < sink ? j : sink + (j - sink) % window;
+  const int64_t C = static_cast<int64_t>(sink) + window;
+  const uint4* ks = reinterpret_cast<const uint4*>(k_new + row_id * D) + ch;
+  const uint4* vs = reinterpret_cast<const uint4*>(v_new + row_id * D) + ch;
+  uint4* kd = reinterpret_cast<uint4*>(k_cache + (bh * C + slot) * D) + ch;
+  uint4* vd = reinterpret_cast<uint4*>(v_cache + (bh * C + slot) * D) + ch;
+  *kd = *ks;
+  *vd = *vs;
+}
+
+static lg_status check_decode(const lg_decode_params* p) {
+  if (!p) return LG_ERR_INVALID_ARG;
+  if (p->B < 1 || p->Hq < 1 || p->Hkv < 1 || p->Hq % p->Hkv != 0) return LG_ERR_INVALID_ARG;
+  if (p->sink_tokens < 0 || p->window_tokens < 1) return LG_ERR_INVALID_ARG;
+  if (!(p->scale >= 0.f) || isinf(p->scale)) return LG_ERR_INVALID_ARG;
+  if (p->D != 64 && p->D != 128) return LG_ERR_UNSUPPORTED;
+  if (static_cast<int64_t>(p->sink_tokens) + p->window_tokens > (1ll << 30)) return LG_ERR_UNSUPPORTED;
+  return LG_OK;
+}
+
+// Number of KV splits: enough CTAs to fill the machine a few times over, but at least
+// 4 tiles of work per warp.
+static int choose_nsplit(const lg_decode_params* p) {
+  const int C = p->sink_tokens + p->window_tokens;
+  const int HG = (p->Hq / p->Hkv + kDecHeads - 1) / kDecHeads;
+  const int64_t units = static_cast<int64_t>(p->B) * p->Hkv * HG;
+  const int64_t tiles = (C + kDecTile - 1) / kDecTile;
+  int64_t max_by_work = tiles / (kDecWarps * 4);
+  if (max_by_work < 1) max_by_work = 1;
+  int64_t want = (148 * 2 * 2 + units - 1) / units;    // about two waves of two CTAs per SM
+  if (want < 1) want = 1;
+  int64_t ns = want < max_by_work ? want : max_by_work;
+  if (ns > 256) ns = 256;
+  return static_cast<int>(ns);
+}
+
+static size_t decode_part_bytes(const lg_decode_params* p, int nsplit) {
+  const int HG = (p->Hq / p->Hkv + kDecHeads - 1) / kDecHeads;
+  return static_cast<size_t>(p->B) * p->Hkv * HG * nsplit * kDecHeads * (p->D + 2) * sizeof(float);
+}
+
+}  // namespace lg
+
+using namespace lg;
+
+extern "C" {
+
+lg_status lg_kv_ring_append(const lg_decode_params* p, void* k_cache, void* v_cache, const void* k_new,
+                            const void* v_new, int32_t T_new, const int64_t* n_tokens_before, void* stream) {
+  lg_status s = check_decode(p);
+  if (s != LG_OK) return s;
+  if (T_new < 0) return LG_ERR_INVALID_ARG;
+  if (T_new == 0) return LG_OK;
+  if (!k_cache || !v_cache || !k_new || !v_new || !n_tokens_before) return LG_ERR_INVALID_ARG;
+  if (!aligned16(k_cache) || !aligned16(v_cache) || !aligned16(k_new) || !aligned16(v_new) ||
+      (reinterpret_cast<uintptr_t>(n_tokens_before) & 7))
+    return LG_ERR_INVALID_ARG;
+  const int64_t threads = static_cast<int64_t>(p->B) * p->Hkv * T_new * (p->D / 8);
+  const int64_t blocks = (threads + 255) / 256;
+  if (blocks > 0x7fffffff) return LG_ERR_UNSUPPORTED;
+  ring_append_kernel<<<static_cast<unsigned>(blocks), 256, 0, static_cast<cudaStream_t>(stream)>>>(
+      static_cast<__nv_bfloat16*>(k_cache), static_cast<__nv_bfloat16*>(v_cache),
+      static_cast<const __nv_bfloat16*>(k_new), static_cast<const __nv_bfloat16*>(v_new), n_tokens_before, p->B,
+      p->Hkv, p->D, T_new, p->sink_tokens, p->window_tokens);
+  return cudaGetLastError() == cudaSuccess ? LG_OK : LG_ERR_CUDA;
+}
+
+size_t lg_sparse_decode_workspace_bytes(const lg_decode_params* p) {
+  if (check_decode(p) != LG_OK) return 0;
+  return sizeof(WsHeader) + align_up(decode_part_bytes(p, choose_nsplit(p)), 256);
+}
+
+lg_status lg_sparse_decode(const lg_decode_params* p, const void* q, const void* k_cache, const void* v_cache,
+                           const int64_t* n_tokens, void* o, float* lse, void* workspace, size_t workspace_bytes,
+                           void* stream) {
+  lg_status s = check_decode(p);
+  if (s != LG_OK) return s;
+  if (!q || !k_cache || !v_cache || !n_tokens || !o || !workspace) return LG_ERR_INVALID_ARG;
+  if (!aligned16(q) || !aligned16(k_cache) || !aligned16(v_cache) || !aligned16(o) ||
+      (reinterpret_cast<uintptr_t>(n_tokens) & 7) || (reinterpret_cast<uintptr_t>(lse) & 3) ||
+      (reinterpret_cast<uintptr_t>(workspace) & 255))
+    return LG_ERR_INVALID_ARG;
+  if (workspace_bytes < lg_sparse_decode_workspace_bytes(p)) return LG_ERR_WORKSPACE;
+  if ((s = check_arch()) != LG_OK) return s;
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  DecodeArgs a;
+  a.q = static_cast<const __nv_bfloat16*>(q);
+  a.k_cache = static_cast<const __nv_bfloat16*>(k_cache);
+  a.v_cache = static_cast<const __nv_bfloat16*>(v_cache);
+  a.n_tokens = n_tokens;
+  a.part = reinterpret_cast<float*>(static_cast<uint8_t*>(workspace) + sizeof(WsHeader));
+  a.o = static_cast<__nv_bfloat16*>(o);
+  a.lse = lse;
+  a.Hq = p->Hq; a.Hkv = p->Hkv; a.G = p->Hq / p->Hkv;
+  a.HG = (a.G + kDecHeads - 1) / kDecHeads;
+  a.C = p->sink_tokens + p->window_tokens;
+  a.nsplit = choose_nsplit(p);
+  const float scale = p->scale > 0.f ? p->scale : 1.0f / sqrtf(static_cast<float>(p->D));
+  a.scale_log2 = scale * 1.4426950408889634f;
+  if (a.Hkv * a.HG > 65535 || p->B > 65535) return LG_ERR_UNSUPPORTED;
+  if (cudaMemsetAsync(workspace, 0, sizeof(WsHeader), st) != cudaSuccess) return LG_ERR_CUDA;
+  dim3 grid(a.nsplit, a.Hkv * a.HG, p->B);
+  const int smem = kDecWarps * kDecStages * 2 * kDecTile * p->D * 2;
+  if (p->D == 128) {
+    if (cudaFuncSetAttribute(decode_split_kernel<128>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem) !=
+        cudaSuccess)
+      return LG_ERR_CUDA;
+    decode_split_kernel<128><<<grid, kDecWarps * 32, smem, st>>>(a);
+    decode_merge_kernel<128><<<p->B * a.Hkv * a.HG, 128, 0, st>>>(a);
+  } else {
+    if (cudaFuncSetAttribute(decode_split_kernel<64>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem) !=
+        cudaSuccess)
+      return LG_ERR_CUDA;
+    decode_split_kernel<64><<<grid, kDecWarps * 32, smem, st>>>(a);
+    decode_merge_kernel<64><<<p->B * a.Hkv * a.HG, 128, 0, st>>>(a);
+  }
+  return cudaGetLastError() == cudaSuccess ? LG_OK : LG_ERR_CUDA;
+}
+
+}  // extern "C"

@@ -1,0 +1,57 @@
+// Host-side helpers shared by the C-ABI entry points: validation, workspace layout,
+// tensor-map encoding.  Nothing here is exported.
+#pragma once
+#include <cuda.h>
+#include <cuda_runtime.h>
+#include <stddef.h>
+#include <stdint.h>
+
+#include "../../include/lg.h"
+#include "lg_pattern.h"
+
+namespace lg {
+
+inline size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
+
+struct Resolved {          // validated, defaulted copy of lg_attn_params
+  int B, Hq, Hkv, L, D, block, mode, G;
+  PatternDev pat;
+  float scale;
+  int64_t qs[3], ks[3], vs[3], os[3];
+  int n_qtiles, n_ktiles;  // ceil(L / 128)
+  int64_t nnz;
+};
+
+lg_status resolve(const lg_attn_params* p, Resolved* r);
+
+// Layout of the attention workspace (all offsets 256-byte aligned).
+struct WsLayout {
+  size_t row_ptr, col_idx, col_ptr, row_idx;     // the CSR / CSC lists
+  size_t qt_cnt, qt_ent, qt_order;               // query-tile schedules (fwd, dQ pass)
+  size_t kt_cnt, kt_ent, kt_order;               // kv-tile schedules (dK/dV pass)
+  size_t delta;                                  // fp32 [B, Hq, L] (bwd only)
+  size_t total;
+};
+WsLayout ws_layout(const Resolved& r, bool want_bwd);
+
+// Build CSR/CSC on `stream` into the given device arrays.
+lg_status launch_index_build(const Resolved& r, int32_t* row_ptr, int32_t* col_idx, int32_t* col_ptr,
+                             int32_t* row_idx, cudaStream_t stream);
+// Build lists + tile schedules inside a workspace.
+lg_status prepare_workspace(const Resolved& r, const WsLayout& w, uint8_t* ws, bool want_bwd, cudaStream_t stream);
+
+// bf16 [B, H, L, D] tensor (element strides bs, hs, ls; D contiguous) as a 4-D tensor map with
+// boxes of 64 columns x `box_rows` rows and the 128-byte swizzle.
+lg_status make_tmap(CUtensorMap* out, const void* base, int B, int H, int L, int D, const int64_t strides[3],
+                    int box_rows);
+
+lg_status check_arch();
+inline bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15) == 0; }
+
+lg_status launch_fwd(const Resolved& r, const WsLayout& w, const void* q, const void* k, const void* v, void* o,
+                     float* lse, uint8_t* ws, cudaStream_t stream);
+lg_status launch_bwd(const Resolved& r, const WsLayout& w, const void* q, const void* k, const void* v,
+                     const void* o, const float* lse, const void* d_o, void* dq, void* dk, void* dv, uint8_t* ws,
+                     cudaStream_t stream);
+
+}  // namespace lg

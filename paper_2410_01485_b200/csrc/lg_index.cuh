@@ -1,0 +1,126 @@
+// Block-index builder: CSR / CSC lists of active blocks of the static pattern (paper
+// Section 3.2: the mask lives in compressed-sparse-row form and is the same for all heads),
+// plus the per-tile schedules the attention kernels walk.
+#pragma once
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include "lg_pattern.h"
+
+namespace lg {
+
+// ---- pass 1: per-row and per-column counts -------------------------------------------
+// grid = nB blocks of 128 threads; block b counts row b and column b.
+__global__ void index_count_kernel(PatternDev p, int32_t* __restrict__ row_ptr, int32_t* __restrict__ col_ptr) {
+  const int b = blockIdx.x;
+  int rc = 0, cc = 0;
+  for (int x = threadIdx.x; x < p.nB; x += blockDim.x) {
+    rc += block_active(p, b, x) ? 1 : 0;
+    cc += block_active(p, x, b) ? 1 : 0;
+  }
+  __shared__ int s_r[4], s_c[4];
+  for (int o = 16; o > 0; o >>= 1) {
+    rc += __shfl_xor_sync(0xffffffffu, rc, o);
+    cc += __shfl_xor_sync(0xffffffffu, cc, o);
+  }
+  if ((threadIdx.x & 31) == 0) { s_r[threadIdx.x >> 5] = rc; s_c[threadIdx.x >> 5] = cc; }
+  __syncthreads();
+  if (threadIdx.x == 0) {
+    row_ptr[b + 1] = s_r[0] + s_r[1] + s_r[2] + s_r[3];
+    col_ptr[b + 1] = s_c[0] + s_c[1] + s_c[2] + s_c[3];
+  }
+}
+
+// ---- pass 2: in-place inclusive scan of ptr[1..n], ptr[0] = 0 (one block, 1024 threads;
+// blockIdx.x selects which of the two arrays) ---------------------------------------------
+__global__ void index_scan_kernel(int32_t* __restrict__ row_ptr, int32_t* __restrict__ col_ptr, int n) {
+  int32_t* ptr = blockIdx.x == 0 ? row_ptr : col_ptr;
+  __shared__ int warp_tot[32];
+  __shared__ int carry;
+  if (threadIdx.x == 0) { carry = 0; ptr[0] = 0; }
+  __syncthreads();
+  for (int base = 0; base < n; base += 1024) {
+    const int i = base + threadIdx.x;
+    int v = i < n ? ptr[i + 1] : 0;
+    for (int o = 1; o < 32; o <<= 1) {
+      int t = __shfl_up_sync(0xffffffffu, v, o);
+      if ((threadIdx.x & 31) >= o) v += t;
+    }
+    if ((threadIdx.x & 31) == 31) warp_tot[threadIdx.x >> 5] = v;
+    __syncthreads();
+    if (threadIdx.x < 32) {
+      int w = warp_tot[threadIdx.x];
+      for (int o = 1; o < 32; o <<= 1) {
+        int t = __shfl_up_sync(0xffffffffu, w, o);
+        if (threadIdx.x >= o) w += t;
+      }
+      warp_tot[threadIdx.x] = w;
+    }
+    __syncthreads();
+    const int prefix = carry + ((threadIdx.x >> 5) ? warp_tot[(threadIdx.x >> 5) - 1] : 0);
+    if (i < n) ptr[i + 1] = v + prefix;
+    __syncthreads();
+    if (threadIdx.x == 0) carry += warp_tot[31];
+    __syncthreads();
+  }
+}
+
+// ---- pass 3: fill.  grid = nB blocks of 64 threads: warp 0 writes row b (ascending kb),
+// warp 1 writes column b (ascending qb), by ordered ballot compaction. ---------------------
+__global__ void index_fill_kernel(PatternDev p, const int32_t* __restrict__ row_ptr, int32_t* __restrict__ col_idx,
+                                  const int32_t* __restrict__ col_ptr, int32_t* __restrict__ row_idx) {
+  const int b = blockIdx.x;
+  const int lane = threadIdx.x & 31;
+  const bool is_row = (threadIdx.x >> 5) == 0;
+  int32_t* out = is_row ? col_idx + row_ptr[b] : row_idx + col_ptr[b];
+  int written = 0;
+  for (int base = 0; base < p.nB; base += 32) {
+    const int x = base + lane;
+    const bool on = x < p.nB && (is_row ? block_active(p, b, x) : block_active(p, x, b));
+    const unsigned m = __ballot_sync(0xffffffffu, on);
+    if (on) out[written + __popc(m & ((1u << lane) - 1))] = x;
+    written += __popc(m);
+  }
+}
+
+// ---- tile schedules ---------------------------------------------------------------------
+// A tile groups R consecutive pattern rows (or columns).  Its schedule is the ascending
+// union of their lists; entry = idx * 4 + member_mask (bit r set: member r of the tile has
+// the block).  Entries of tile t start at ptr[R * t]; cnt[t] says how many there are.
+// One thread per tile.
+__global__ void tile_merge_kernel(const int32_t* __restrict__ ptr, const int32_t* __restrict__ idx, int nB, int R,
+                                  int n_tiles, int32_t* __restrict__ tile_cnt, int32_t* __restrict__ tile_ent) {
+  const int t = blockIdx.x * blockDim.x + threadIdx.x;
+  if (t >= n_tiles) return;
+  const int r0 = t * R;
+  int32_t* out = tile_ent + ptr[r0];
+  int n = 0;
+  if (R == 1 || r0 + 1 >= nB) {
+    for (int e = ptr[r0]; e < ptr[r0 + 1]; ++e) out[n++] = idx[e] * 4 + 1;
+  } else {  // R == 2: merge two ascending lists
+    int a = ptr[r0], ae = ptr[r0 + 1], c = ptr[r0 + 1], ce = ptr[r0 + 2];
+    while (a < ae || c < ce) {
+      const int va = a < ae ? idx[a] : 0x7fffffff;
+      const int vc = c < ce ? idx[c] : 0x7fffffff;
+      if (va == vc) { out[n++] = va * 4 + 3; ++a; ++c; }
+      else if (va < vc) { out[n++] = va * 4 + 1; ++a; }
+      else { out[n++] = vc * 4 + 2; ++c; }
+    }
+  }
+  tile_cnt[t] = n;
+}
+
+// Launch order: tiles with more work first.  order[rank] = tile; rank by (count desc, tile asc).
+__global__ void tile_order_kernel(const int32_t* __restrict__ tile_cnt, int n_tiles, int32_t* __restrict__ order) {
+  const int t = blockIdx.x * blockDim.x + threadIdx.x;
+  if (t >= n_tiles) return;
+  const int c = tile_cnt[t];
+  int rank = 0;
+  for (int u = 0; u < n_tiles; ++u) {
+    const int cu = tile_cnt[u];
+    rank += (cu > c || (cu == c && u < t)) ? 1 : 0;
+  }
+  order[rank] = t;
+}
+
+}  // namespace lg

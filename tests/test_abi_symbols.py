@@ -1,0 +1,86 @@
+"""The C-ABI library loads on a machine without a GPU and exports every symbol that
+include/lg.h declares; host-side validation rejects bad arguments without launching."""
+import ctypes as C
+import os
+import re
+
+import pytest
+
+from paper_2410_01485_b200 import binding, build
+
+
+@pytest.fixture(scope="module")
+def lib():
+    build.build()
+    return binding.load_library()
+
+
+def test_every_declared_symbol_is_exported(lib):
+    header = open(os.path.join(os.path.dirname(build.HERE), "include", "lg.h")).read()
+    header = re.sub(r"/\*.*?\*/", "", header, flags=re.S)
+    declared = set(re.findall(r"\b(lg_[a-z_0-9]+)\s*\(", header))
+    assert declared, "no declarations parsed"
+    assert declared == set(binding.SYMBOLS), (declared ^ set(binding.SYMBOLS))
+    for name in declared:
+        assert hasattr(lib, name), name
+
+
+def test_status_strings(lib):
+    assert binding.status_string(0) == "ok"
+    for code in range(-6, 0):
+        assert binding.status_string(code) not in ("ok", "unknown status")
+
+
+def _good():
+    return binding.attn_params(1, 4, 2, 512, 128, 64, binding.MODE_SINK_WINDOW, sink_tokens=64, window_tokens=128)
+
+
+def test_nnz_and_sizes_on_host(lib):
+    p = _good()
+    assert binding.lg_block_index_nnz(p) == 21      # same pattern as the tiny config
+    assert lib.lg_block_index_bytes(C.byref(p)) == 4 * (2 * 9 + 2 * 21)
+    assert lib.lg_sparse_attn_workspace_bytes(C.byref(p), 1) > lib.lg_sparse_attn_workspace_bytes(C.byref(p), 0) > 256
+    full = binding.attn_params(1, 1, 1, 32768, 128, 64, binding.MODE_FULL_CAUSAL)
+    assert binding.lg_block_index_nnz(full) == 131328
+    strided = binding.attn_params(1, 64, 8, 131072, 128, 64, binding.MODE_STRIDED_LOCAL, stride_blocks=16, local_blocks=4)
+    assert binding.lg_block_index_nnz(strided) == 139770
+
+
+@pytest.mark.parametrize("mutate", [
+    lambda p: setattr(p, "Hkv", 3),                 # Hq % Hkv != 0
+    lambda p: setattr(p, "L", 500),                 # L % block != 0
+    lambda p: setattr(p, "block", 32),
+    lambda p: setattr(p, "sink_tokens", 10),        # not a multiple of block
+    lambda p: setattr(p, "window_tokens", 0),       # window < block
+    lambda p: setattr(p, "mode", 7),
+    lambda p: setattr(p, "scale", -1.0),
+    lambda p: setattr(p, "B", 0),
+])
+def test_invalid_params_rejected(lib, mutate):
+    p = _good()
+    mutate(p)
+    assert lib.lg_block_index_nnz(C.byref(p)) == -1
+    assert lib.lg_block_index_bytes(C.byref(p)) == 0
+    assert lib.lg_sparse_attn_workspace_bytes(C.byref(p), 0) == 0
+    # fwd with (fake but aligned) pointers: rejected before anything is touched
+    assert lib.lg_sparse_attn_fwd(C.byref(p), 256, 256, 256, 256, 256, 256, 1 << 30, None) == -1
+
+
+def test_unsupported_head_dim(lib):
+    p = _good()
+    p.D = 96
+    assert lib.lg_block_index_nnz(C.byref(p)) == -2
+
+
+def test_null_misaligned_and_small_workspace(lib):
+    p = _good()
+    need = lib.lg_sparse_attn_workspace_bytes(C.byref(p), 0)
+    assert lib.lg_sparse_attn_fwd(C.byref(p), None, 256, 256, 256, 256, 256, need, None) == -1
+    assert lib.lg_sparse_attn_fwd(C.byref(p), 264, 256, 256, 256, 256, 256, need, None) == -1   # 8-byte aligned only
+    assert lib.lg_sparse_attn_fwd(C.byref(p), 256, 256, 256, 256, 256, 128, need, None) == -1   # workspace alignment
+    assert lib.lg_sparse_attn_fwd(C.byref(p), 256, 256, 256, 256, 256, 256, need - 1, None) == -3
+    assert lib.lg_sparse_attn_bwd(C.byref(p), *([256] * 9), 256, need, None) == -3              # bwd needs more
+    p.q_strides[0], p.q_strides[1], p.q_strides[2] = 4 * 512 * 128, 512 * 128, 100              # stride < D
+    assert lib.lg_sparse_attn_fwd(C.byref(p), 256, 256, 256, 256, 256, 256, need, None) == -1
+    assert lib.lg_build_block_index(C.byref(_good()), None, 256, 256, 256, None, None) == -1
+    assert lib.lg_last_status(None, None) == -1
