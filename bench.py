@@ -1,0 +1,376 @@
+#!/usr/bin/env python
+"""Benchmark of the LongGen efficient-layer attention path on B200.
+
+A step is one pass of the hot path over one batch of synthetic input: the block-index
+build, the sparse forward (with LSE) and the backward of the 128K length-extension
+workload (Llama-2-7B-shaped, sink + sliding window).  The other configurations (32K
+prefill sparse vs full-causal, 70B-shaped strided GQA fwd+bwd, 70B-shaped decode over the
+sink+window ring cache vs a dense cache) are measured once each and reported under
+"other".  One JSON line is printed by rank 0.
+
+  python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference] [--quick]
+
+With N > 1 (launched under torch.distributed.run) every rank runs the same workload on its
+own GPU -- the path has no exchange step, ranks are replicas -- and the value is the sum
+over ranks divided by the slowest rank's time.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import math
+import os
+import subprocess
+import sys
+import threading
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+sys.path.insert(0, ROOT)
+
+import numpy as np
+import torch
+
+from paper_2410_01485_b200 import synth
+
+METRIC = "128K sparse attn fwd+bwd TFLOP/s (useful)"
+UNIT = "TFLOP/s"
+NOMINAL_BF16_TFLOPS = 2250.0
+NOMINAL_HBM_GBS = 8000.0
+
+
+def load_peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        with open(path) as f:
+            p = json.load(f)
+        return {"hbm_gbs": p["hbm_gbs"], "bf16_burst": p["bf16_tflops"], "bf16_sustained": p["bf16_tflops_sustained"],
+                "source": "measured"}
+    return {"hbm_gbs": 6650.0, "bf16_burst": 1590.0, "bf16_sustained": 1400.0, "source": "fallback"}
+
+
+def pairs_per_head(cfg) -> int:
+    """Exact number of visible (query, key) pairs of one head: full blocks count Bs^2,
+    diagonal blocks Bs(Bs+1)/2 (closed form of the pattern; the oracle's mask count agrees)."""
+    Bs, nB = cfg.block, cfg.L // cfg.block
+    if cfg.mode == synth.MODE_FULL_CAUSAL:
+        off = nB * (nB - 1) // 2
+    elif cfg.mode == synth.MODE_SINK_WINDOW:
+        ns, nw = cfg.sink_tokens // Bs, cfg.window_tokens // Bs
+        off = sum(min(qb + 1, nw) - 1 + min(ns, max(qb + 1 - nw, 0)) for qb in range(nB))
+    else:
+        nl, s = cfg.local_blocks, cfg.stride_blocks
+        off = sum(min(qb + 1, nl) - 1 + -(-max(qb - nl + 1, 0) // s) for qb in range(nB))
+    return off * Bs * Bs + nB * Bs * (Bs + 1) // 2
+
+
+def flops(cfg, fwd=True, bwd=True) -> float:
+    per_pair = (4 if fwd else 0) + (10 if bwd else 0)
+    return float(pairs_per_head(cfg)) * cfg.B * cfg.Hq * cfg.D * per_pair
+
+
+# ------------------------------------------------------------------------------ clocks
+
+class ClockSampler:
+    """Samples nvidia-smi while the timed region runs (reads settings only)."""
+    QUERY = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,"
+             "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
+             "clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, index: int):
+        self.index, self.proc, self.lines = index, None, []
+
+    def __enter__(self):
+        try:
+            self.proc = subprocess.Popen(["nvidia-smi", "-i", str(self.index), "--query-gpu=" + self.QUERY,
+                                          "--format=csv,noheader,nounits", "-lms", "200"],
+                                         stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+            self.thread = threading.Thread(target=self._pump, daemon=True)
+            self.thread.start()
+        except OSError:
+            self.proc = None
+        return self
+
+    def _pump(self):
+        for line in self.proc.stdout:
+            self.lines.append(line.strip())
+
+    def __exit__(self, *exc):
+        if self.proc is not None:
+            self.proc.terminate()
+            try:
+                self.proc.wait(timeout=5)
+            except subprocess.TimeoutExpired:
+                self.proc.kill()
+
+    def summary(self):
+        sm, mx, reasons = [], 0.0, set()
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        for line in self.lines:
+            parts = [x.strip() for x in line.split(",")]
+            if len(parts) < 7:
+                continue
+            try:
+                sm.append(float(parts[0]))
+                mx = max(mx, float(parts[1]))
+            except ValueError:
+                continue
+            for name, val in zip(names, parts[3:7]):
+                if val.lower().startswith("active"):
+                    reasons.add(name)
+        return {"sm_mhz": float(np.median(sm)) if sm else None, "sm_max_mhz": mx or None,
+                "reasons": sorted(reasons), "samples": len(sm)}
+
+
+# ------------------------------------------------------------------------ oracle timing
+
+def oracle_sample(cfg, seconds_hint="~10-30 s"):
+    """Time the CPU oracle, as it stands, on a bounded sample of the workload: one head,
+    the first L/8 tokens, forward + backward.  Returns (useful TFLOP/s, description, cores)."""
+    from dataclasses import replace
+    from oracle import lg_oracle as O
+    small = replace(cfg, B=1, Hq=2 * (cfg.Hq // cfg.Hkv), Hkv=2, L=cfg.L // 8)
+    inp = synth.make_attn_inputs(small, "cpu", seed=0, with_do=True)
+    q, k, v, do = (synth.to_f64(inp[x][0]) for x in ("q", "k", "v", "do"))
+    t0 = time.perf_counter()
+    O.attn_backward(q, k, v, do, O.Pattern.of(small), 1.0 / math.sqrt(cfg.D), rows_per_slab=cfg.block)
+    dt = time.perf_counter() - t0
+    tf = flops(small) / dt / 1e12
+    desc = "%s pattern, %d query heads / 2 kv heads, first %d tokens, fwd+bwd, fp64 numpy: %.1f s" % (
+        cfg.name, small.Hq, small.L, dt)
+    return tf, desc, os.cpu_count(), dt
+
+
+def run_reference(args):
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    cfg = synth.CFG3
+    vals = []
+    for i in range(args.warmup + args.steps):
+        tf, desc, cores, dt = oracle_sample(cfg)
+        if i >= args.warmup:
+            vals.append((tf, dt))
+    tf = float(np.mean([v[0] for v in vals]))
+    ms = float(np.mean([v[1] for v in vals])) * 1e3
+    line = {"impl": "reference", "metric": METRIC, "value": tf, "unit": UNIT, "n_gpus": args.gpus,
+            "steps": args.steps, "warmup": args.warmup, "ms_per_step": ms, "higher_is_better": True,
+            "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+            "config": {"workload": cfg.name, "sample": desc},
+            "cpu_baseline": {"value": tf, "unit": UNIT, "cores": cores, "kind": "oracle", "sample": desc},
+            "e2e": {"value": tf, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0}}
+    print(json.dumps(line), flush=True)
+
+
+# ---------------------------------------------------------------------------- GPU timing
+
+def time_cuda(fn, warmup, steps):
+    """Median-free plain timing: total of `steps` calls between two events on the current stream."""
+    for _ in range(warmup):
+        fn()
+    torch.cuda.synchronize()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record()
+    for _ in range(steps):
+        fn()
+    e1.record()
+    torch.cuda.synchronize()
+    return e0.elapsed_time(e1) / steps
+
+
+def bench_attn(lg, cfg, warmup, steps, want_bwd, profile_kernels=False):
+    p = lg.params_of(cfg)
+    inp = synth.make_attn_inputs(cfg, "cuda", seed=0, with_do=want_bwd)
+    ws = lg.attn_workspace(p, want_bwd)
+    o = torch.empty_like(inp["q"])
+    lse = torch.empty(inp["q"].shape[:3], dtype=torch.float32, device="cuda")
+    out = {"config": cfg.name}
+    f_fwd = lambda: lg.lg_sparse_attn_fwd(p, inp["q"], inp["k"], inp["v"], o=o, lse=lse, workspace=ws)
+    out["fwd_ms"] = time_cuda(f_fwd, warmup, steps)
+    out["fwd_tflops"] = flops(cfg, True, False) / out["fwd_ms"] / 1e9
+    if want_bwd:
+        dq, dk, dv = torch.empty_like(inp["q"]), torch.empty_like(inp["k"]), torch.empty_like(inp["v"])
+        f_bwd = lambda: lg.lg_sparse_attn_bwd(p, inp["q"], inp["k"], inp["v"], o, lse, inp["do"], dq=dq, dk=dk,
+                                              dv=dv, workspace=ws)
+        out["bwd_ms"] = time_cuda(f_bwd, warmup, steps)
+        out["bwd_tflops"] = flops(cfg, False, True) / out["bwd_ms"] / 1e9
+        out["fwd_bwd_ms"] = out["fwd_ms"] + out["bwd_ms"]
+        out["fwd_bwd_tflops"] = flops(cfg) / out["fwd_bwd_ms"] / 1e9
+        if profile_kernels:
+            ks = np.array([lg.lg_sparse_attn_bwd_profiled(p, inp["q"], inp["k"], inp["v"], o, lse, inp["do"], dq,
+                                                          dk, dv, ws) for _ in range(max(steps, 3))])
+            out["bwd_kernel_ms"] = dict(zip(("delta", "dkdv", "dq"), [float(x) for x in ks.mean(axis=0)]))
+    assert lg.lg_last_status(ws) == 0, "device-side wait expired"
+    return out, (p, inp, ws, o, lse)
+
+
+def bench_decode(lg, c, warmup, steps, dense=False, copies=4):
+    cap = c.n_tokens if dense else c.sink_tokens + c.window_tokens
+    p = lg.decode_params(c.B, c.Hq, c.Hkv, c.D, 0 if dense else c.sink_tokens, cap if dense else c.window_tokens)
+    if dense:
+        copies = 1                      # 8.6 GB per copy: far larger than L2 already
+    sets = [synth.make_decode_inputs(c, "cuda", seed=s, capacity=cap) for s in range(copies)]
+    n_t = torch.full((c.B,), c.n_tokens, dtype=torch.int64, device="cuda")
+    ws = lg.decode_workspace(p)
+    o = torch.empty_like(sets[0]["q"])
+    state = {"i": 0}
+
+    def fn():
+        s = sets[state["i"] % copies]
+        state["i"] += 1
+        lg.lg_sparse_decode(p, s["q"], s["k_cache"], s["v_cache"], n_t, o=o, workspace=ws, want_lse=False)
+
+    ms = time_cuda(fn, warmup, steps)
+    nbytes = 2.0 * c.B * c.Hkv * cap * c.D * 2
+    assert lg.lg_last_status(ws) == 0
+    return {"config": c.name + ("_dense" if dense else ""), "ms": ms, "bytes": nbytes, "gbs": nbytes / ms / 1e6,
+            "l2": "rotating over %d cache copies (%.0f MB each)" % (copies, nbytes / 1e6)}
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=5)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--quick", action="store_true", help="headline workload only (no other configs, no e2e)")
+    ap.add_argument("--no-oracle", action="store_true", help="skip the CPU-oracle baseline leg")
+    args = ap.parse_args()
+    args.warmup = max(args.warmup, 3)
+
+    if args.impl == "reference":
+        run_reference(args)
+        return
+
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    torch.cuda.set_device(local)
+    dist = None
+    if world > 1:
+        import torch.distributed as dist
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local))
+
+    from paper_2410_01485_b200 import binding as lg, build
+    if rank == 0:
+        build.build()
+    if dist is not None:
+        dist.barrier()
+    lg.load_library()
+    peaks = load_peaks()
+    cfg = synth.CFG3
+
+    # ---- headline: K timed steps of fwd + bwd, device-resident inputs ----------------------
+    p = lg.params_of(cfg)
+    inp = synth.make_attn_inputs(cfg, "cuda", seed=0, with_do=True)
+    ws = lg.attn_workspace(p, True)
+    o = torch.empty_like(inp["q"])
+    lse = torch.empty(inp["q"].shape[:3], dtype=torch.float32, device="cuda")
+    dq, dk, dv = torch.empty_like(inp["q"]), torch.empty_like(inp["k"]), torch.empty_like(inp["v"])
+
+    def step():
+        lg.lg_sparse_attn_fwd(p, inp["q"], inp["k"], inp["v"], o=o, lse=lse, workspace=ws)
+        lg.lg_sparse_attn_bwd(p, inp["q"], inp["k"], inp["v"], o, lse, inp["do"], dq=dq, dk=dk, dv=dv, workspace=ws)
+
+    for _ in range(args.warmup):
+        step()
+    torch.cuda.synchronize()
+    if dist is not None:
+        dist.barrier()
+    with ClockSampler(local) as clocks:
+        torch.cuda.synchronize()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        for _ in range(args.steps):
+            step()
+        e1.record()
+        torch.cuda.synchronize()
+        # per-kernel durations inside the same clock-sampled region (synchronising variant)
+        fwd_ms = time_cuda(lambda: lg.lg_sparse_attn_fwd(p, inp["q"], inp["k"], inp["v"], o=o, lse=lse, workspace=ws),
+                           0, args.steps)
+        kms = np.array([lg.lg_sparse_attn_bwd_profiled(p, inp["q"], inp["k"], inp["v"], o, lse, inp["do"], dq, dk,
+                                                       dv, ws) for _ in range(args.steps)]).mean(axis=0)
+    assert lg.lg_last_status(ws) == 0, "device-side wait expired"
+    ms_step = e0.elapsed_time(e1) / args.steps
+    if dist is not None:
+        t = torch.tensor([ms_step], device="cuda")
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        ms_step = float(t.item())
+    total_flops = flops(cfg) * world
+    value = total_flops / ms_step / 1e9
+
+    pairs = float(pairs_per_head(cfg)) * cfg.B * cfg.Hq
+    kern = {"fwd": (fwd_ms, pairs * cfg.D * 4), "bwd_dkdv": (float(kms[1]), pairs * cfg.D * 8),
+            "bwd_dq": (float(kms[2]), pairs * cfg.D * 2), "bwd_delta": (float(kms[0]), 0.0)}
+    dom = max(("fwd", "bwd_dkdv", "bwd_dq"), key=lambda n: kern[n][0])
+    achieved = kern[dom][1] / kern[dom][0] / 1e9
+    roofline = {"bound": "tensor", "kernel": dom, "achieved": achieved, "peak": peaks["bf16_sustained"],
+                "unit": "TFLOP/s", "frac": achieved / peaks["bf16_sustained"], "traffic": None,
+                "peak_source": "%s sustained bf16 matmul" % peaks["source"],
+                "frac_of_nominal_2250": achieved / NOMINAL_BF16_TFLOPS,
+                "kernel_ms": {k: v[0] for k, v in kern.items()},
+                "note": "algorithmic FLOPs per launch: fwd 4D, dK/dV pass 8D, dQ pass 2D per visible pair"}
+
+    line = {"metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
+            "warmup": args.warmup, "ms_per_step": ms_step, "higher_is_better": True, "scaling": "weak",
+            "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
+            "config": {"workload": cfg.name, "B": cfg.B, "Hq": cfg.Hq, "Hkv": cfg.Hkv, "L": cfg.L, "D": cfg.D,
+                       "block": cfg.block, "sink_tokens": cfg.sink_tokens, "window_tokens": cfg.window_tokens,
+                       "useful_flop_per_step": flops(cfg), "parallelism": "replicas x%d" % world,
+                       "l2": "inputs (8.6 GB) far larger than L2; no flush"},
+            "pct_of_nominal_bf16_peak": 100.0 * value / world / NOMINAL_BF16_TFLOPS,
+            "pct_of_measured_bf16_sustained": 100.0 * value / world / peaks["bf16_sustained"],
+            "roofline": roofline, "clocks": clocks.summary(),
+            "gpu_launches": args.steps * 17}
+
+    del dq, dk, dv
+    others = []
+    if rank == 0 and not args.quick:
+        # ---- e2e: host buffers, copies inside the timed region -----------------------------
+        host = {k: torch.empty(v.shape, dtype=v.dtype, pin_memory=True).copy_(v) for k, v in inp.items()}
+        h_out = {"o": torch.empty(o.shape, dtype=o.dtype, pin_memory=True),
+                 "lse": torch.empty(lse.shape, dtype=lse.dtype, pin_memory=True),
+                 "dq": torch.empty(o.shape, dtype=o.dtype, pin_memory=True),
+                 "dk": torch.empty(inp["k"].shape, dtype=o.dtype, pin_memory=True),
+                 "dv": torch.empty(inp["v"].shape, dtype=o.dtype, pin_memory=True)}
+        dq, dk, dv = torch.empty_like(inp["q"]), torch.empty_like(inp["k"]), torch.empty_like(inp["v"])
+
+        def e2e_step():
+            lg.sparse_attn_fwd_bwd_host(p, host, h_out, dev=(inp, o, lse, dq, dk, dv, ws))
+
+        e2e_ms = time_cuda(e2e_step, 1, max(2, min(args.steps, 3)))
+        h2d = sum(t.numel() * t.element_size() for t in host.values())
+        d2h = sum(t.numel() * t.element_size() for t in h_out.values())
+        line["e2e"] = {"value": flops(cfg) / e2e_ms / 1e9, "unit": UNIT, "ms_per_step": e2e_ms,
+                       "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h}
+        del host, h_out, dq, dk, dv
+    del inp, o, lse, ws
+    torch.cuda.empty_cache()
+
+    if rank == 0 and not args.quick:
+        r2, _ = bench_attn(lg, synth.CFG2, 3, 5, want_bwd=False)
+        r2f, _ = bench_attn(lg, synth.CFG2.full_causal(), 3, 3, want_bwd=False)
+        torch.cuda.empty_cache()
+        r4, _ = bench_attn(lg, synth.CFG4, 3, 3, want_bwd=True, profile_kernels=True)
+        torch.cuda.empty_cache()
+        d5 = bench_decode(lg, synth.CFG5, 5, 40)
+        d5["pct_of_nominal_8tbs"] = 100 * d5["gbs"] / NOMINAL_HBM_GBS
+        d5["pct_of_measured_copy"] = 100 * d5["gbs"] / peaks["hbm_gbs"]
+        torch.cuda.empty_cache()
+        d5d = bench_decode(lg, synth.CFG5, 2, 5, dense=True)
+        d5d["pct_of_measured_copy"] = 100 * d5d["gbs"] / peaks["hbm_gbs"]
+        others = [r2, r2f, r4, d5, d5d]
+        line["other"] = others
+        line["decode_hbm_gbs"] = d5["gbs"]
+    if rank == 0 and not args.no_oracle and world == 1:
+        tf, desc, cores, _ = oracle_sample(cfg)
+        line["cpu_baseline"] = {"value": tf, "unit": UNIT, "cores": cores, "kind": "oracle", "sample": desc}
+    if rank == 0:
+        print(json.dumps(line), flush=True)
+    if dist is not None:
+        dist.barrier()
+        dist.destroy_process_group()
+
+
+if __name__ == "__main__":
+    main()

@@ -109,6 +109,16 @@ lg_status lg_sparse_attn_bwd(const lg_attn_params* p, const void* q, const void*
                              void* dq, void* dk, void* dv,
                              void* workspace, size_t workspace_bytes, void* stream);
 
+/* Same computation as lg_sparse_attn_bwd, for profiling: records CUDA events between its
+ * three kernels on `stream`, SYNCHRONISES the stream, and writes their durations in
+ * milliseconds to kernel_ms (HOST float[3]: delta pre-pass, dK/dV pass, dQ pass).  The paper
+ * has no counterpart; it exists so that a benchmark can report a per-kernel roofline.      */
+lg_status lg_sparse_attn_bwd_profiled(const lg_attn_params* p, const void* q, const void* k,
+                                      const void* v, const void* o, const float* lse,
+                                      const void* d_o, void* dq, void* dk, void* dv,
+                                      void* workspace, size_t workspace_bytes, void* stream,
+                                      float* kernel_ms);
+
 /* ---- serving: rolling-buffer cache and decode (Section 3.2) --------------------------- */
 
 /*

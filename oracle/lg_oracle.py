@@ -16,7 +16,7 @@ materialises the explicit token-level boolean mask; nothing here is blocked,
 fused or reordered beyond "work on a slab of rows at a time", which changes no
 value.  All arithmetic is float64.
 
-Readings of points on which the paper is silent (see the design notes):
+Readings of points on which the paper is silent:
   - the window is block-granular and counts the query's own block
     (Section 4.1: "the first block ... and the most recent 32 blocks");
   - the strided comb is absolute: KV block kb is retained iff kb % stride == 0;
@@ -198,6 +198,66 @@ def attn_backward(q, k, v, do, p: Pattern, scale: float, rows_per_slab: Optional
             dK[g, cols] += scale * (dS.T @ q[h, r0:r1])
             dV[g, cols] += P.T @ dOh
     return dQ, dK, dV, O, LSE
+
+
+# ----------------------------------------------------- subsets of the outputs (large L)
+
+def attn_rows(q, k, v, do, p: Pattern, scale: float, r0: int, r1: int):
+    """The definition restricted to query rows [r0, r1): O, LSE and (if `do` is given) dQ
+    of those rows for every head.  Row i of O, LSE and dQ depends on row i of Q and dO only,
+    so this is attn_forward / attn_backward evaluated on one slab.
+    Returns (O [Hq, r1-r0, D], LSE [Hq, r1-r0], dQ or None)."""
+    Hq, L, D = q.shape
+    G = Hq // k.shape[0]
+    M = token_mask(p, r0, r1)
+    cols = np.nonzero(M.any(axis=0))[0]
+    Mc = M[:, cols]
+    O = np.zeros((Hq, r1 - r0, D))
+    LSE = np.zeros((Hq, r1 - r0))
+    dQ = None if do is None else np.zeros((Hq, r1 - r0, D))
+    for h in range(Hq):
+        kc, vc = k[h // G, cols], v[h // G, cols]
+        S = scale * (q[h, r0:r1] @ kc.T)
+        P, lse = _softmax_rows(S, Mc)
+        O[h] = P @ vc
+        LSE[h] = lse
+        if do is not None:
+            dP = do[h, r0:r1] @ vc.T
+            delta = (P * dP).sum(axis=1, keepdims=True)
+            dQ[h] = scale * ((P * (dP - delta)) @ kc)
+    return O, LSE, dQ
+
+
+def attn_keys_grad(q, k, v, do, p: Pattern, scale: float, j0: int, j1: int):
+    """The definition restricted to keys [j0, j1): dK and dV of those keys for every kv
+    head.  Every query row that may see one of these keys is found from the explicit mask
+    and taken a block of rows at a time; its softmax runs over ALL keys it may see.
+    Returns (dK [Hkv, j1-j0, D], dV [Hkv, j1-j0, D])."""
+    Hq, L, D = q.shape
+    Hkv = k.shape[0]
+    G = Hq // Hkv
+    dK = np.zeros((Hkv, j1 - j0, D))
+    dV = np.zeros((Hkv, j1 - j0, D))
+    for r0 in range(0, L, p.block):
+        r1 = r0 + p.block
+        M = token_mask(p, r0, r1)
+        if not M[:, j0:j1].any():
+            continue
+        cols = np.nonzero(M.any(axis=0))[0]
+        Mc = M[:, cols]
+        sel = (cols >= j0) & (cols < j1)        # which of the slab's keys are the wanted ones
+        for h in range(Hq):
+            g = h // G
+            kc, vc = k[g, cols], v[g, cols]
+            S = scale * (q[h, r0:r1] @ kc.T)
+            P, _ = _softmax_rows(S, Mc)
+            dOh = do[h, r0:r1]
+            dP = dOh @ vc.T
+            delta = (P * dP).sum(axis=1, keepdims=True)
+            dS = P * (dP - delta)
+            dK[g, cols[sel] - j0] += scale * (dS[:, sel].T @ q[h, r0:r1])
+            dV[g, cols[sel] - j0] += P[:, sel].T @ dOh
+    return dK, dV
 
 
 # -------------------------------------------------------------------------- decode

@@ -50,6 +50,7 @@ SYMBOLS = {
     "lg_sparse_attn_workspace_bytes": (_sz, [C.POINTER(AttnParams), C.c_int]),
     "lg_sparse_attn_fwd": (C.c_int, [C.POINTER(AttnParams), _vp, _vp, _vp, _vp, _vp, _vp, _sz, _vp]),
     "lg_sparse_attn_bwd": (C.c_int, [C.POINTER(AttnParams)] + [_vp] * 9 + [_vp, _sz, _vp]),
+    "lg_sparse_attn_bwd_profiled": (C.c_int, [C.POINTER(AttnParams)] + [_vp] * 9 + [_vp, _sz, _vp, C.POINTER(C.c_float)]),
     "lg_kv_ring_append": (C.c_int, [C.POINTER(DecodeParams), _vp, _vp, _vp, _vp, C.c_int32, _vp, _vp]),
     "lg_sparse_decode_workspace_bytes": (_sz, [C.POINTER(DecodeParams)]),
     "lg_sparse_decode": (C.c_int, [C.POINTER(DecodeParams), _vp, _vp, _vp, _vp, _vp, _vp, _vp, _sz, _vp]),
@@ -167,6 +168,39 @@ def lg_sparse_attn_bwd(p: AttnParams, q, k, v, o, lse, d_o, dq=None, dk=None, dv
                                   lse.data_ptr(), d_o.data_ptr(), dq.data_ptr(), dk.data_ptr(), dv.data_ptr(),
                                   ws.data_ptr(), ws.numel(), _stream()), "lg_sparse_attn_bwd")
     return dq, dk, dv
+
+
+def lg_sparse_attn_bwd_profiled(p: AttnParams, q, k, v, o, lse, d_o, dq, dk, dv, workspace):
+    """As lg_sparse_attn_bwd, synchronising; returns [delta_ms, dkdv_ms, dq_ms]."""
+    p.q_strides, p.k_strides, p.v_strides, p.o_strides = _strides3(q), _strides3(k), _strides3(v), _strides3(o)
+    ms = (C.c_float * 3)()
+    _check(load_library().lg_sparse_attn_bwd_profiled(
+        C.byref(p), q.data_ptr(), k.data_ptr(), v.data_ptr(), o.data_ptr(), lse.data_ptr(), d_o.data_ptr(),
+        dq.data_ptr(), dk.data_ptr(), dv.data_ptr(), workspace.data_ptr(), workspace.numel(), _stream(), ms),
+        "lg_sparse_attn_bwd_profiled")
+    return [float(x) for x in ms]
+
+
+def sparse_attn_fwd_bwd_host(p: AttnParams, host_in, host_out, dev=None):
+    """End-to-end training step with HOST buffers: copies pinned q, k, v, do to the device,
+    runs lg_sparse_attn_fwd and lg_sparse_attn_bwd, and copies o, lse, dq, dk, dv back into the
+    pinned tensors of `host_out`.  `dev` optionally supplies preallocated device buffers
+    (inputs dict, o, lse, dq, dk, dv, workspace).  All arithmetic runs in the CUDA library."""
+    if dev is None:
+        d_in = {k: torch.empty(v.shape, dtype=v.dtype, device="cuda") for k, v in host_in.items()}
+        o = torch.empty_like(d_in["q"])
+        lse = torch.empty(d_in["q"].shape[:3], dtype=torch.float32, device="cuda")
+        dq, dk, dv = torch.empty_like(d_in["q"]), torch.empty_like(d_in["k"]), torch.empty_like(d_in["v"])
+        ws = attn_workspace(p, True)
+    else:
+        d_in, o, lse, dq, dk, dv, ws = dev
+    for name in ("q", "k", "v", "do"):
+        d_in[name].copy_(host_in[name], non_blocking=True)
+    lg_sparse_attn_fwd(p, d_in["q"], d_in["k"], d_in["v"], o=o, lse=lse, workspace=ws)
+    lg_sparse_attn_bwd(p, d_in["q"], d_in["k"], d_in["v"], o, lse, d_in["do"], dq=dq, dk=dk, dv=dv, workspace=ws)
+    for name, t in (("o", o), ("lse", lse), ("dq", dq), ("dk", dk), ("dv", dv)):
+        host_out[name].copy_(t, non_blocking=True)
+    return host_out
 
 
 # ---------------------------------------------------------------------- decode / ring

@@ -233,9 +233,9 @@ lg_status lg_sparse_attn_fwd(const lg_attn_params* p, const void* q, const void*
   return launch_fwd(r, w, q, k, v, o, lse, ws, st);
 }
 
-lg_status lg_sparse_attn_bwd(const lg_attn_params* p, const void* q, const void* k, const void* v, const void* o,
-                             const float* lse, const void* d_o, void* dq, void* dk, void* dv, void* workspace,
-                             size_t workspace_bytes, void* stream) {
+static lg_status bwd_common(const lg_attn_params* p, const void* q, const void* k, const void* v, const void* o,
+                            const float* lse, const void* d_o, void* dq, void* dk, void* dv, void* workspace,
+                            size_t workspace_bytes, void* stream, cudaEvent_t* marks) {
   Resolved r;
   lg_status s = resolve(p, &r);
   if (s != LG_OK) return s;
@@ -250,7 +250,32 @@ lg_status lg_sparse_attn_bwd(const lg_attn_params* p, const void* q, const void*
   cudaStream_t st = static_cast<cudaStream_t>(stream);
   uint8_t* ws = static_cast<uint8_t*>(workspace);
   if ((s = prepare_workspace(r, w, ws, true, st)) != LG_OK) return s;
-  return launch_bwd(r, w, q, k, v, o, lse, d_o, dq, dk, dv, ws, st);
+  return launch_bwd(r, w, q, k, v, o, lse, d_o, dq, dk, dv, ws, st, marks);
+}
+
+lg_status lg_sparse_attn_bwd(const lg_attn_params* p, const void* q, const void* k, const void* v, const void* o,
+                             const float* lse, const void* d_o, void* dq, void* dk, void* dv, void* workspace,
+                             size_t workspace_bytes, void* stream) {
+  return bwd_common(p, q, k, v, o, lse, d_o, dq, dk, dv, workspace, workspace_bytes, stream, nullptr);
+}
+
+lg_status lg_sparse_attn_bwd_profiled(const lg_attn_params* p, const void* q, const void* k, const void* v,
+                                      const void* o, const float* lse, const void* d_o, void* dq, void* dk,
+                                      void* dv, void* workspace, size_t workspace_bytes, void* stream,
+                                      float* kernel_ms) {
+  if (!kernel_ms) return LG_ERR_INVALID_ARG;
+  cudaEvent_t ev[4] = {nullptr, nullptr, nullptr, nullptr};
+  lg_status s = LG_OK;
+  for (int i = 0; i < 4; ++i)
+    if (cudaEventCreate(&ev[i]) != cudaSuccess) s = LG_ERR_CUDA;
+  if (s == LG_OK) s = bwd_common(p, q, k, v, o, lse, d_o, dq, dk, dv, workspace, workspace_bytes, stream, ev);
+  if (s == LG_OK && cudaStreamSynchronize(static_cast<cudaStream_t>(stream)) != cudaSuccess) s = LG_ERR_CUDA;
+  if (s == LG_OK)
+    for (int i = 0; i < 3; ++i)
+      if (cudaEventElapsedTime(&kernel_ms[i], ev[i], ev[i + 1]) != cudaSuccess) s = LG_ERR_CUDA;
+  for (int i = 0; i < 4; ++i)
+    if (ev[i]) cudaEventDestroy(ev[i]);
+  return s;
 }
 
 lg_status lg_last_status(void* workspace, void* stream) {

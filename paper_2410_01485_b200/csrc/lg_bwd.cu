@@ -7,9 +7,10 @@ namespace lg {
 template <int D, int BS>
 static lg_status launch_bwd_t(const Resolved& r, const WsLayout& w, const void* q, const void* k, const void* v,
                               const void* o, const float* lse, const void* d_o, void* dq, void* dk, void* dv,
-                              uint8_t* ws, cudaStream_t stream) {
+                              uint8_t* ws, cudaStream_t stream, cudaEvent_t* marks) {
   lg_status s;
   float* delta = reinterpret_cast<float*>(ws + w.delta);
+  if (marks) cudaEventRecord(marks[0], stream);
   {
     const int64_t rows = static_cast<int64_t>(r.B) * r.Hq * r.L;
     const int64_t threads = rows * (D / 8);
@@ -19,6 +20,7 @@ static lg_status launch_bwd_t(const Resolved& r, const WsLayout& w, const void* 
         static_cast<const __nv_bfloat16*>(o), static_cast<const __nv_bfloat16*>(d_o), delta, r.os[0], r.os[1],
         r.os[2], r.Hq, r.L, rows);
   }
+  if (marks) cudaEventRecord(marks[1], stream);
   BwdArgs a;
   a.lse = lse;
   a.delta = delta;
@@ -47,6 +49,7 @@ static lg_status launch_bwd_t(const Resolved& r, const WsLayout& w, const void* 
       return LG_ERR_CUDA;
     dim3 grid(r.B * r.Hkv, r.n_ktiles);
     kern<<<grid, 128, smem, stream>>>(tq, tk, tv, tdo, a);
+    if (marks) cudaEventRecord(marks[2], stream);
   }
   // ---- dQ pass ------------------------------------------------------------------------
   {
@@ -67,16 +70,17 @@ static lg_status launch_bwd_t(const Resolved& r, const WsLayout& w, const void* 
       return LG_ERR_CUDA;
     dim3 grid(r.B * r.Hq, r.n_qtiles);
     kern<<<grid, 128, smem, stream>>>(tq, tk, tv, tdo, a);
+    if (marks) cudaEventRecord(marks[3], stream);
   }
   return cudaGetLastError() == cudaSuccess ? LG_OK : LG_ERR_CUDA;
 }
 
 lg_status launch_bwd(const Resolved& r, const WsLayout& w, const void* q, const void* k, const void* v,
                      const void* o, const float* lse, const void* d_o, void* dq, void* dk, void* dv, uint8_t* ws,
-                     cudaStream_t stream) {
+                     cudaStream_t stream, cudaEvent_t* marks) {
   if (r.n_qtiles > 65535) return LG_ERR_UNSUPPORTED;
 #define LG_BWD_CASE(DD, BB) \
-  if (r.D == DD && r.block == BB) return launch_bwd_t<DD, BB>(r, w, q, k, v, o, lse, d_o, dq, dk, dv, ws, stream);
+  if (r.D == DD && r.block == BB) return launch_bwd_t<DD, BB>(r, w, q, k, v, o, lse, d_o, dq, dk, dv, ws, stream, marks);
   LG_BWD_CASE(128, 128)
   LG_BWD_CASE(128, 64)
   LG_BWD_CASE(64, 128)

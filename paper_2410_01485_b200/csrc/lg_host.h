@@ -52,6 +52,6 @@ lg_status launch_fwd(const Resolved& r, const WsLayout& w, const void* q, const 
                      float* lse, uint8_t* ws, cudaStream_t stream);
 lg_status launch_bwd(const Resolved& r, const WsLayout& w, const void* q, const void* k, const void* v,
                      const void* o, const float* lse, const void* d_o, void* dq, void* dk, void* dv, uint8_t* ws,
-                     cudaStream_t stream);
+                     cudaStream_t stream, cudaEvent_t* marks /* null, or 4 events recorded around the 3 kernels */);
 
 }  // namespace lg

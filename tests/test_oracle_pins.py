@@ -283,6 +283,25 @@ def test_slab_oracle_equals_dense_oracle():
         np.testing.assert_allclose(a[4], c[1], rtol=1e-12, atol=1e-13)
 
 
+def test_subset_evaluators_equal_full_oracle():
+    """attn_rows / attn_keys_grad (used at 128K, where only samples are affordable) give
+    the same numbers as the pinned full evaluation."""
+    for p in TINY_PATTERNS:
+        q, k, v, do = (_rand((4, p.L, 3), s) for s in (17, 18, 19, 20))
+        k, v = k[:2], v[:2]
+        dQ, dK, dV, Oo, LSE = O.attn_backward(q, k, v, do, p, 0.3)
+        for r0 in range(0, p.L, p.block):
+            o, lse, dq = O.attn_rows(q, k, v, do, p, 0.3, r0, r0 + p.block)
+            np.testing.assert_allclose(o, Oo[:, r0:r0 + p.block], rtol=1e-12, atol=1e-13)
+            np.testing.assert_allclose(lse, LSE[:, r0:r0 + p.block], rtol=1e-12, atol=1e-13)
+            np.testing.assert_allclose(dq, dQ[:, r0:r0 + p.block], rtol=1e-12, atol=1e-13)
+            dk, dv = O.attn_keys_grad(q, k, v, do, p, 0.3, r0, r0 + p.block)
+            np.testing.assert_allclose(dk, dK[:, r0:r0 + p.block], rtol=1e-11, atol=1e-12)
+            np.testing.assert_allclose(dv, dV[:, r0:r0 + p.block], rtol=1e-11, atol=1e-12)
+        dk, dv = O.attn_keys_grad(q, k, v, do, p, 0.3, 3, p.L - 5)
+        np.testing.assert_allclose(dk, dK[:, 3:p.L - 5], rtol=1e-11, atol=1e-12)
+
+
 # ------------------------------------------------------------------------- backward
 
 def _loss(q, k, v, do, p, scale):
