@@ -235,8 +235,14 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--quick", action="store_true", help="headline workload only (no other configs, no e2e)")
     ap.add_argument("--no-oracle", action="store_true", help="skip the CPU-oracle baseline leg")
+    ap.add_argument("--case", default="full", choices=["full", "small"],
+                    help="small: the headline pattern at 8 heads x 32K tokens, for profiler captures "
+                         "(implies --quick --no-oracle; its numbers are not benchmark values)")
     args = ap.parse_args()
-    args.warmup = max(args.warmup, 3)
+    if args.case == "small":
+        args.quick = args.no_oracle = True
+    else:
+        args.warmup = max(args.warmup, 3)
 
     if args.impl == "reference":
         run_reference(args)
@@ -259,6 +265,9 @@ def main():
     lg.load_library()
     peaks = load_peaks()
     cfg = synth.CFG3
+    if args.case == "small":
+        from dataclasses import replace
+        cfg = replace(cfg, name=cfg.name + "_small", Hq=8, Hkv=8, L=32768)
 
     # ---- headline: K timed steps of fwd + bwd, device-resident inputs ----------------------
     p = lg.params_of(cfg)
