@@ -151,6 +151,46 @@ lg_status lg_sparse_decode(const lg_decode_params* p, const void* q, const void*
                            const void* v_cache, const int64_t* n_tokens, void* o, float* lse,
                            void* workspace, size_t workspace_bytes, void* stream);
 
+/* ---- decode for callers that may not allocate -------------------------------------- */
+
+/* Size of the scratch array that lg_sparse_decode_static uses instead of a workspace.  It
+ * is part of the library image: every GPU on which the library is used keeps this much
+ * device memory from the first use until the process exits.                              */
+#define LG_DECODE_STATIC_SCRATCH_BYTES (4u << 20)
+
+/*
+ * lg_sparse_decode without a workspace argument.  (The paper has no counterpart; this is a
+ * convenience of this library.)
+ *
+ * Who needs it: code that runs where device memory cannot be requested at call time -- a
+ * serving loop whose memory pool is handed out entirely at start-up, a plug-in that has no
+ * allocator handle of its host framework, a latency-critical step where cudaMalloc's implicit
+ * synchronisation is not acceptable.  Such a caller still owns q, the caches, n_tokens, o and
+ * lse and passes them exactly as to lg_sparse_decode; only the split-KV partials, which
+ * lg_sparse_decode keeps in the caller's workspace, go to a fixed array inside the library.
+ * The call itself requests no device or host memory (no cudaMalloc / cudaFree, no allocating
+ * library routine).
+ *
+ * Limits and rules
+ *   - The problem must satisfy lg_sparse_decode_workspace_bytes(p) <=
+ *     LG_DECODE_STATIC_SCRATCH_BYTES (the Llama-2-70B-shaped decode of 16 sequences over a
+ *     128 + 4096 token ring needs about 2.7 MB); otherwise LG_ERR_WORKSPACE is returned and
+ *     nothing is launched.  Larger problems use lg_sparse_decode with their own workspace.
+ *   - The first call on each device looks up the array's device address (with that device
+ *     current) and remembers it; make that first call outside any stream capture.
+ *   - All calls on one device share the one array, and it keeps whatever the previous call
+ *     left in it.  The call clears the status word at its start and overwrites every partial
+ *     it later reads, so back-to-back calls on one stream are fine; two calls that can run
+ *     on the GPU at the same time (different streams, no dependency) race on the array and
+ *     give undefined results.
+ *   - The decode kernels contain no device-side waits, so there is no device status to read
+ *     back for this call (lg_last_status needs a workspace pointer and does not apply).
+ * Results are bit-identical to lg_sparse_decode on the same inputs.
+ */
+lg_status lg_sparse_decode_static(const lg_decode_params* p, const void* q, const void* k_cache,
+                                  const void* v_cache, const int64_t* n_tokens, void* o, float* lse,
+                                  void* stream);
+
 /* ---- status ------------------------------------------------------------------------- */
 
 /* Synchronises `stream`, reads the error word the kernels keep at the start of

@@ -54,6 +54,7 @@ SYMBOLS = {
     "lg_kv_ring_append": (C.c_int, [C.POINTER(DecodeParams), _vp, _vp, _vp, _vp, C.c_int32, _vp, _vp]),
     "lg_sparse_decode_workspace_bytes": (_sz, [C.POINTER(DecodeParams)]),
     "lg_sparse_decode": (C.c_int, [C.POINTER(DecodeParams), _vp, _vp, _vp, _vp, _vp, _vp, _vp, _sz, _vp]),
+    "lg_sparse_decode_static": (C.c_int, [C.POINTER(DecodeParams), _vp, _vp, _vp, _vp, _vp, _vp, _vp]),
     "lg_last_status": (C.c_int, [_vp, _vp]),
     "lg_status_string": (C.c_char_p, [C.c_int]),
 }
@@ -237,6 +238,21 @@ def lg_sparse_decode(p: DecodeParams, q, k_cache, v_cache, n_tokens, o=None, lse
     _check(load_library().lg_sparse_decode(C.byref(p), q.data_ptr(), k_cache.data_ptr(), v_cache.data_ptr(),
                                            n_tokens.data_ptr(), o.data_ptr(), lse.data_ptr() if lse is not None else None,
                                            ws.data_ptr(), ws.numel(), _stream()), "lg_sparse_decode")
+    return o, lse
+
+
+DECODE_STATIC_SCRATCH_BYTES = 4 << 20   # LG_DECODE_STATIC_SCRATCH_BYTES of include/lg.h
+
+
+def lg_sparse_decode_static(p: DecodeParams, q, k_cache, v_cache, n_tokens, o, lse=None):
+    """lg_sparse_decode for callers that cannot allocate: no workspace argument, the split
+    partials live in a fixed array inside the library (see include/lg.h).  `o` (and `lse`, if
+    wanted) must be supplied by the caller, so this wrapper allocates nothing either."""
+    assert q.is_contiguous() and k_cache.is_contiguous() and v_cache.is_contiguous() and o.is_contiguous()
+    _check(load_library().lg_sparse_decode_static(C.byref(p), q.data_ptr(), k_cache.data_ptr(), v_cache.data_ptr(),
+                                                  n_tokens.data_ptr(), o.data_ptr(),
+                                                  lse.data_ptr() if lse is not None else None, _stream()),
+           "lg_sparse_decode_static")
     return o, lse
 
 

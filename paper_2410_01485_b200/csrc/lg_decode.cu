@@ -12,6 +12,8 @@
 // split order, which keeps the result bitwise reproducible.
 #include <math.h>
 
+#include <mutex>
+
 #include "lg_common.cuh"
 #include "lg_host.h"
 
@@ -408,5 +410,49 @@ lg_status lg_sparse_decode(const lg_decode_params* p, const void* q, const void*
   }
   return cudaGetLastError() == cudaSuccess ? LG_OK : LG_ERR_CUDA;
 }
+
+// ---- decode without any allocation ------------------------------------------------------
+// Scratch for lg_sparse_decode_static: lives in the library image, one copy per GPU that
+// loads it.  In host code this name is only a handle; the device address comes from
+// cudaGetSymbolAddress, looked up once per device below.
+static __device__ __align__(256) unsigned char g_decode_static_scratch[LG_DECODE_STATIC_SCRATCH_BYTES];
+
+namespace {
+constexpr int kMaxStaticDevices = 64;
+void* g_static_scratch_addr[kMaxStaticDevices];   // device address per device ordinal, 0 = not looked up yet
+std::mutex g_static_scratch_mutex;
+
+// Device address of the scratch array on the CURRENT device (looked up on first use).
+lg_status static_scratch_address(void** out) {
+  int dev = -1;
+  if (cudaGetDevice(&dev) != cudaSuccess) return LG_ERR_CUDA;
+  if (dev < 0 || dev >= kMaxStaticDevices) return LG_ERR_UNSUPPORTED;
+  std::lock_guard<std::mutex> lock(g_static_scratch_mutex);
+  if (!g_static_scratch_addr[dev]) {
+    void* addr = nullptr;
+    if (cudaGetSymbolAddress(&addr, g_decode_static_scratch) != cudaSuccess || !addr) return LG_ERR_CUDA;
+    g_static_scratch_addr[dev] = addr;
+  }
+  *out = g_static_scratch_addr[dev];
+  return LG_OK;
+}
+}  // namespace
+
+lg_status lg_sparse_decode_static(const lg_decode_params* p, const void* q, const void* k_cache,
+                                  const void* v_cache, const int64_t* n_tokens, void* o, float* lse,
+                                  void* stream) {
+  lg_status s = check_decode(p);
+  if (s != LG_OK) return s;
+  // the split partials of this problem must fit the fixed array
+  if (lg_sparse_decode_workspace_bytes(p) > static_cast<size_t>(LG_DECODE_STATIC_SCRATCH_BYTES))
+    return LG_ERR_WORKSPACE;
+  void* scratch = nullptr;
+  if ((s = static_scratch_address(&scratch)) != LG_OK) return s;
+  // Same kernels as lg_sparse_decode, with the array as their workspace.  Its header word is
+  // cleared by that call; the partials are fully rewritten before the merge kernel reads them.
+  return lg_sparse_decode(p, q, k_cache, v_cache, n_tokens, o, lse, scratch, LG_DECODE_STATIC_SCRATCH_BYTES,
+                          stream);
+}
+
 
 }  // extern "C"
