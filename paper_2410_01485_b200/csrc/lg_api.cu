@@ -112,7 +112,7 @@ WsLayout ws_layout(const Resolved& r, bool want_bwd) {
     w.kt_cnt = take(r.n_ktiles * 4);
     w.kt_ent = take(nnz * 4);
     w.kt_order = take(r.n_ktiles * 4);
-    w.delta = take(static_cast<size_t>(r.B) * r.Hq * r.L * 4);
+    w.delta = take(static_cast<size_t>(r.B) * r.Hq * r.L * 8);   // (LSE * log2 e, delta) per query row
   }
   w.total = off;
   return w;

@@ -9,7 +9,7 @@ static lg_status launch_bwd_t(const Resolved& r, const WsLayout& w, const void* 
                               const void* o, const float* lse, const void* d_o, void* dq, void* dk, void* dv,
                               uint8_t* ws, cudaStream_t stream, cudaEvent_t* marks) {
   lg_status s;
-  float* delta = reinterpret_cast<float*>(ws + w.delta);
+  float2* stat = reinterpret_cast<float2*>(ws + w.delta);
   if (marks) cudaEventRecord(marks[0], stream);
   {
     const int64_t rows = static_cast<int64_t>(r.B) * r.Hq * r.L;
@@ -17,13 +17,12 @@ static lg_status launch_bwd_t(const Resolved& r, const WsLayout& w, const void* 
     const int64_t blocks = (threads + 255) / 256;
     if (blocks > 0x7fffffff) return LG_ERR_UNSUPPORTED;
     delta_kernel<D><<<static_cast<unsigned>(blocks), 256, 0, stream>>>(
-        static_cast<const __nv_bfloat16*>(o), static_cast<const __nv_bfloat16*>(d_o), delta, r.os[0], r.os[1],
+        static_cast<const __nv_bfloat16*>(o), static_cast<const __nv_bfloat16*>(d_o), lse, stat, r.os[0], r.os[1],
         r.os[2], r.Hq, r.L, rows);
   }
   if (marks) cudaEventRecord(marks[1], stream);
   BwdArgs a;
-  a.lse = lse;
-  a.delta = delta;
+  a.stat = stat;
   a.error_word = reinterpret_cast<unsigned int*>(ws);
   a.L = r.L; a.Hq = r.Hq; a.Hkv = r.Hkv; a.G = r.G;
   a.scale = r.scale;
@@ -48,7 +47,7 @@ static lg_status launch_bwd_t(const Resolved& r, const WsLayout& w, const void* 
     if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, smem) != cudaSuccess)
       return LG_ERR_CUDA;
     dim3 grid(r.B * r.Hkv, r.n_ktiles);
-    kern<<<grid, 128, smem, stream>>>(tq, tk, tv, tdo, a);
+    kern<<<grid, kBwdThreads, smem, stream>>>(tq, tk, tv, tdo, a);
     if (marks) cudaEventRecord(marks[2], stream);
   }
   // ---- dQ pass ------------------------------------------------------------------------
@@ -69,7 +68,7 @@ static lg_status launch_bwd_t(const Resolved& r, const WsLayout& w, const void* 
     if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, smem) != cudaSuccess)
       return LG_ERR_CUDA;
     dim3 grid(r.B * r.Hq, r.n_qtiles);
-    kern<<<grid, 128, smem, stream>>>(tq, tk, tv, tdo, a);
+    kern<<<grid, kBwdThreads, smem, stream>>>(tq, tk, tv, tdo, a);
     if (marks) cudaEventRecord(marks[3], stream);
   }
   return cudaGetLastError() == cudaSuccess ? LG_OK : LG_ERR_CUDA;

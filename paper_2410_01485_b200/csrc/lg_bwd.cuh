@@ -12,6 +12,15 @@
 //     back as bf16 over them and feed dV += P^T dO and dK += dS^T Q as TMEM A operands.
 //   * dQ pass: one CTA per tile of 128 queries of one head walks its CSR row(s):
 //     S = Q K^T, dP = dO V^T, dS over S, dQ += dS K.
+//
+// Both kernels are warp-specialised: warps 0-7 do the element-wise work (two groups of four
+// warps, each group owning 64 of the 128 columns of a step; thread = TMEM lane), warp 8
+// feeds shared memory with TMA, one thread of warp 9 issues every tcgen05.mma.  A step covers
+// 128 streamed rows: one 128-token pattern block, or two 64-token blocks side by side.  The
+// MMA order is chosen so that the tensor pipe always has independent work while the
+// exponentials of the current step are evaluated:
+//   dQ pass   : ... dQ(j-1) dP(j) S(j+1) | dQ(j) dP(j+1) S(j+2) ...      (S double-buffered)
+//   dK/dV pass: ... S(j) dK(j-1) dP(j) dV(j) | S(j+1) dK(j) dP(j+1) dV(j+1) ...
 #pragma once
 #include <cuda.h>
 #include "lg_common.cuh"
@@ -23,8 +32,7 @@ struct BwdArgs {
   const int32_t* tile_cnt;
   const int32_t* tile_ent;   // idx * 4 + member mask
   const int32_t* order;
-  const float* lse;          // [B, Hq, L]
-  const float* delta;        // [B, Hq, L]
+  const float2* stat;        // [B, Hq, L]: (LSE * log2(e), delta)
   __nv_bfloat16* out0;       // dQ   | dK
   __nv_bfloat16* out1;       // unused | dV
   unsigned int* error_word;
@@ -33,11 +41,14 @@ struct BwdArgs {
   float scale, scale_log2;
 };
 
-// ---- delta = rowsum(dO * O) ---------------------------------------------------------------
+constexpr int kBwdThreads = 320;     // 8 element-wise warps + TMA warp + MMA warp
+constexpr int kBwdEwThreads = 256;
+
+// ---- stat = (LSE * log2 e, rowsum(dO * O)) --------------------------------------------------
 template <int D>
 __global__ void delta_kernel(const __nv_bfloat16* __restrict__ o, const __nv_bfloat16* __restrict__ d_o,
-                             float* __restrict__ delta, int64_t sb, int64_t sh, int64_t sl, int Hq, int L,
-                             int64_t total_rows) {
+                             const float* __restrict__ lse, float2* __restrict__ stat, int64_t sb, int64_t sh,
+                             int64_t sl, int Hq, int L, int64_t total_rows) {
   constexpr int TPR = D / 8;   // threads per row, 16 bytes each
   const int64_t gid = static_cast<int64_t>(blockIdx.x) * blockDim.x + threadIdx.x;
   const int64_t row = gid / TPR;
@@ -61,23 +72,44 @@ __global__ void delta_kernel(const __nv_bfloat16* __restrict__ o, const __nv_bfl
   }
 #pragma unroll
   for (int s = TPR / 2; s > 0; s >>= 1) acc += __shfl_xor_sync(0xffffffffu, acc, s);
-  if (row < total_rows && ch == 0) delta[row] = acc;
+  if (row < total_rows && ch == 0) stat[row] = make_float2(lse[row] * 1.4426950408889634f, acc);
 }
+
+// Every tile in shared memory holds 128 rows of D bf16: D/64 column boxes of [128 rows x 128 B].
+template <int D>
+struct BwdTile {
+  static constexpr int kBox = 128 * 128;            // bytes of one 64-column box of 128 rows
+  static constexpr int kBytes = (D / 64) * kBox;
+};
 
 template <int D, int BS>
 struct BwdSmem {
-  static constexpr int kFixBytes = 128 * D * 2;   // Q or K (and dO or V) tile of the CTA's own 128 rows
-  static constexpr int kStgBytes = BS * D * 2;    // streamed operand tile
-  static constexpr int kVecOff = 2 * kFixBytes + 4 * kStgBytes;   // [2 stages][lse2, delta][BS] floats
-  static constexpr int kBarOff = kVecOff + 2 * 2 * BS * 4;
-  static constexpr int kTotal = kBarOff + 128 + 1024;
+  static constexpr int kTile = BwdTile<D>::kBytes;
+  static constexpr int kAStages = 3;   // operand read by the first and the last MMA of a step (K | Q)
+  static constexpr int kBStages = 2;   // operand read by adjacent MMAs (V | dO)
+  static constexpr int oFix0 = 0, oFix1 = kTile;
+  static constexpr int oA = 2 * kTile;
+  static constexpr int oB = oA + kAStages * kTile;
+  static constexpr int oStat = oB + kBStages * kTile;            // dK/dV pass: [2][128] float2
+  static constexpr int oBar = oStat + 2 * 128 * 8;
+  static constexpr int kTotal = oBar + 256;
 };
 
-// store one 128 x D fp32 accumulator tile from TMEM as bf16 rows (times `mul`)
-template <int D>
-__device__ __forceinline__ void store_acc_rows(uint32_t taddr, __nv_bfloat16* row_ptr, float mul, bool do_store) {
+// load one step (128 rows: one 128-row block, or two 64-row blocks) of a [.., L, D] tensor
+template <int D, int BS>
+__device__ __forceinline__ void tma_load_rows(uint8_t* dst, const CUtensorMap* tm, uint64_t* bar, int half,
+                                              int row, int head, int batch) {
+  // BS == 128: half is ignored (box = 128 rows); BS == 64: box = 64 rows placed at rows 64 * half
 #pragma unroll
-  for (int c = 0; c < D / 32; ++c) {
+  for (int x = 0; x < D / 64; ++x)
+    tma_load_4d(dst + x * BwdTile<D>::kBox + (BS == 64 ? half * (64 * 128) : 0), tm, bar, x * 64, row, head, batch);
+}
+
+// fp32 accumulator columns [c0, c0 + n) of this thread's TMEM lane -> bf16 row (times mul)
+template <int N>
+__device__ __forceinline__ void store_acc_cols(uint32_t taddr, __nv_bfloat16* dst, float mul, bool do_store) {
+#pragma unroll
+  for (int c = 0; c < N / 32; ++c) {
     uint32_t reg[32];
     tmem_ld32(taddr + c * 32, reg);
     tmem_ld_wait();
@@ -89,385 +121,535 @@ __device__ __forceinline__ void store_acc_rows(uint32_t taddr, __nv_bfloat16* ro
         v4.y = pack_bf16(__uint_as_float(reg[x + 2]) * mul, __uint_as_float(reg[x + 3]) * mul);
         v4.z = pack_bf16(__uint_as_float(reg[x + 4]) * mul, __uint_as_float(reg[x + 5]) * mul);
         v4.w = pack_bf16(__uint_as_float(reg[x + 6]) * mul, __uint_as_float(reg[x + 7]) * mul);
-        *reinterpret_cast<uint4*>(row_ptr + c * 32 + x) = v4;
+        *reinterpret_cast<uint4*>(dst + c * 32 + x) = v4;
       }
     }
   }
 }
 
-// ============================== dK / dV pass ==================================================
-template <int D, int BS>
-__global__ void __launch_bounds__(128, 1)
-bwd_dkdv_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUtensorMap tm_k,
-                const __grid_constant__ CUtensorMap tm_v, const __grid_constant__ CUtensorMap tm_do,
-                const BwdArgs a) {
-  using SM = BwdSmem<D, BS>;
-  constexpr int R = 128 / BS;
-  constexpr int NBOX = D / 64;
-  constexpr uint32_t kColS = 0, kColDP = BS, kColDV = 2 * BS, kColDK = 2 * BS + D;
-  constexpr uint32_t kTmemCols = (2 * BS + 2 * D) <= 256 ? 256 : 512;
-
-  extern __shared__ uint8_t smem_raw[];
-  uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
-  uint8_t* sK = smem;
-  uint8_t* sV = sK + SM::kFixBytes;
-  uint8_t* sQ = sV + SM::kFixBytes;                 // [stage]
-  uint8_t* sDO = sQ + 2 * SM::kStgBytes;            // [stage]
-  float* sVec = reinterpret_cast<float*>(smem + SM::kVecOff);
-  uint64_t* bars = reinterpret_cast<uint64_t*>(smem + SM::kBarOff);
-  uint64_t* bar_fix = bars + 0;
-  uint64_t* bar_ld = bars + 1;   // [2]
-  uint64_t* bar_s = bars + 3;
-  uint64_t* bar_o = bars + 4;
-  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 5);
-  volatile uint32_t* s_fail = tmem_slot + 1;
-
-  const int tid = threadIdx.x, warp = tid >> 5;
-  const int tile = a.order[blockIdx.y];
-  const int b = blockIdx.x / a.Hkv, hk = blockIdx.x % a.Hkv;
-  const int n_ent = a.tile_cnt[tile];
-  const int32_t* ent = a.tile_ent + a.tile_off[tile * R];
-  const int key0 = tile * 128;
-  const int n_iter = n_ent * a.G;
-
-  if (warp == 0) {
-    tmem_alloc(tmem_slot, kTmemCols);
-    tmem_relinquish();
-  }
-  if (tid == 0) {
-    *s_fail = 0;
-    mbar_init(bar_fix, 1);
-    mbar_init(bar_ld + 0, 1);
-    mbar_init(bar_ld + 1, 1);
-    mbar_init(bar_s, 1);
-    mbar_init(bar_o, 1);
-    mbar_fence_init();
-    tma_prefetch_desc(&tm_q);
-    tma_prefetch_desc(&tm_k);
-    tma_prefetch_desc(&tm_v);
-    tma_prefetch_desc(&tm_do);
-  }
+// A warp of element-wise threads finished writing tensor memory: publish it to the MMA thread.
+__device__ __forceinline__ void ew_publish(uint64_t* bar) {
+  tmem_st_wait();
   tc_fence_before();
-  __syncthreads();
-  tc_fence_after();
-  const uint32_t tmem = *tmem_slot;
-  const uint32_t lane_addr = tmem + (static_cast<uint32_t>(warp * 32) << 16);
-
-  auto issue_ld = [&](int it) {
-    const int st = it & 1;
-    const int g = it / n_ent, e = it - g * n_ent;
-    const int qb = ent[e] >> 2;
-    const int h = hk * a.G + g;
-    mbar_expect_tx(bar_ld + st, 2 * SM::kStgBytes);
-#pragma unroll
-    for (int x = 0; x < NBOX; ++x) {
-      tma_load_4d(sQ + st * SM::kStgBytes + x * (BS * 128), &tm_q, bar_ld + st, x * 64, qb * BS, h, b);
-      tma_load_4d(sDO + st * SM::kStgBytes + x * (BS * 128), &tm_do, bar_ld + st, x * 64, qb * BS, h, b);
-    }
-  };
-
-  if (tid == 0) {
-    mbar_expect_tx(bar_fix, 2 * SM::kFixBytes);
-#pragma unroll
-    for (int x = 0; x < NBOX; ++x) {
-      tma_load_4d(sK + x * (128 * 128), &tm_k, bar_fix, x * 64, key0, hk, b);
-      tma_load_4d(sV + x * (128 * 128), &tm_v, bar_fix, x * 64, key0, hk, b);
-    }
-    if (n_iter > 0) issue_ld(0);
-  }
-
-  constexpr uint32_t idesc_st = make_idesc_bf16(128, BS, 0, 0);   // S^T, dP^T: N = query block
-  constexpr uint32_t idesc_acc = make_idesc_bf16(128, D, 0, 1);   // dV, dK: B = dO / Q, MN-major
-  const int r = tid;
-  const int kj = key0 + r;                         // this thread's key
-  const int member = (R == 1) ? 0 : (r / BS);
-  bool fail = false;
-
-  for (int it = 0; it < n_iter; ++it) {
-    const int st = it & 1;
-    const int g = it / n_ent, e = it - g * n_ent;
-    const int entry = ent[e];
-    const int qb = entry >> 2;
-    const int h = hk * a.G + g;
-    // stage the per-query statistics of this block
-    if (tid < BS) {
-      const int64_t off = (static_cast<int64_t>(b) * a.Hq + h) * a.L + qb * BS + tid;
-      sVec[(st * 2 + 0) * BS + tid] = a.lse[off] * 1.4426950408889634f;
-      sVec[(st * 2 + 1) * BS + tid] = a.delta[off];
-    }
-    if (tid == 0) {
-      if (it == 0) fail |= !mbar_wait(bar_fix, 0, a.error_word, 11);
-      if (it > 0) fail |= !mbar_wait(bar_o, (it - 1) & 1, a.error_word, 12);   // MMAs of it-1 done
-      if (!fail && it + 1 < n_iter) issue_ld(it + 1);
-      fail |= !mbar_wait(bar_ld + st, (it >> 1) & 1, a.error_word, 13);
-      if (!fail) {
-        tc_fence_after();
-        const uint32_t k_base = smem_u32(sK), v_base = smem_u32(sV);
-        const uint32_t q_base = smem_u32(sQ + st * SM::kStgBytes), do_base = smem_u32(sDO + st * SM::kStgBytes);
-#pragma unroll
-        for (int k = 0; k < D / 16; ++k) {
-          const uint32_t fo = (k >> 2) * (128 * 128) + (k & 3) * 32, so = (k >> 2) * (BS * 128) + (k & 3) * 32;
-          mma_ss(tmem + kColS, make_smem_desc(k_base + fo, 16, 1024), make_smem_desc(q_base + so, 16, 1024),
-                 idesc_st, k > 0);
-        }
-#pragma unroll
-        for (int k = 0; k < D / 16; ++k) {
-          const uint32_t fo = (k >> 2) * (128 * 128) + (k & 3) * 32, so = (k >> 2) * (BS * 128) + (k & 3) * 32;
-          mma_ss(tmem + kColDP, make_smem_desc(v_base + fo, 16, 1024), make_smem_desc(do_base + so, 16, 1024),
-                 idesc_st, k > 0);
-        }
-      }
-      mma_commit(bar_s);
-    }
-    __syncthreads();   // sVec visible
-    fail |= !mbar_wait(bar_s, it & 1, a.error_word, 14);
-    tc_fence_after();
-
-    const bool need_mask = ((entry & 3) != ((1 << R) - 1)) || (qb * BS < key0 + 127);
-    const bool row_on = (entry >> member) & 1;
-    const float* lse2 = sVec + (st * 2 + 0) * BS;
-    const float* dlt = sVec + (st * 2 + 1) * BS;
-    // visible iff row_on and key <= query, i.e. column x (query qb*BS + x) >= kj - qb*BS
-    const int xmin = need_mask ? (row_on ? kj - qb * BS : BS) : 0;
-#pragma unroll
-    for (int c = 0; c < BS / 32; ++c) {
-      uint32_t sreg[32], dreg[32], preg[16], dsreg[16];
-      tmem_ld32(lane_addr + kColS + c * 32, sreg);
-      tmem_ld32(lane_addr + kColDP + c * 32, dreg);
-      tmem_ld_wait();
-#pragma unroll
-      for (int x = 0; x < 32; x += 2) {
-        const int col = c * 32 + x;
-        float p0 = fast_exp2(__uint_as_float(sreg[x]) * a.scale_log2 - lse2[col]);
-        float p1 = fast_exp2(__uint_as_float(sreg[x + 1]) * a.scale_log2 - lse2[col + 1]);
-        p0 = (col >= xmin) ? p0 : 0.f;
-        p1 = (col + 1 >= xmin) ? p1 : 0.f;
-        const float d0 = p0 * (__uint_as_float(dreg[x]) - dlt[col]);
-        const float d1 = p1 * (__uint_as_float(dreg[x + 1]) - dlt[col + 1]);
-        preg[x >> 1] = pack_bf16(p0, p1);
-        dsreg[x >> 1] = pack_bf16(d0, d1);
-      }
-      tmem_st16(lane_addr + kColS + c * 16, preg);     // P^T over the S^T columns already read
-      tmem_st16(lane_addr + kColDP + c * 16, dsreg);   // dS^T over dP^T
-    }
-    tmem_st_wait();
-    tc_fence_before();
-    if (fail) *s_fail = 1;
-    __syncthreads();
-    const bool cta_fail = *s_fail != 0;
-    if (tid == 0) {
-      tc_fence_after();
-      if (!cta_fail) {
-        const uint32_t q_base = smem_u32(sQ + st * SM::kStgBytes), do_base = smem_u32(sDO + st * SM::kStgBytes);
-#pragma unroll
-        for (int k = 0; k < BS / 16; ++k)
-          mma_ts(tmem + kColDV, tmem + kColS + k * 8, make_smem_desc(do_base + k * 2048, BS * 128, 1024), idesc_acc,
-                 (it > 0) || (k > 0));
-#pragma unroll
-        for (int k = 0; k < BS / 16; ++k)
-          mma_ts(tmem + kColDK, tmem + kColDP + k * 8, make_smem_desc(q_base + k * 2048, BS * 128, 1024), idesc_acc,
-                 (it > 0) || (k > 0));
-      }
-      mma_commit(bar_o);
-    }
-    if (cta_fail) { fail = true; break; }
-  }
-
-  if (n_iter > 0) {
-    fail |= !mbar_wait(bar_o, (n_iter - 1) & 1, a.error_word, 15);
-    tc_fence_after();
-  }
-  {
-    const bool st_ok = !fail && kj < a.L;
-    __nv_bfloat16* dk_row = a.out0 + b * a.s0[0] + hk * a.s0[1] + static_cast<int64_t>(kj) * a.s0[2];
-    __nv_bfloat16* dv_row = a.out1 + b * a.s1[0] + hk * a.s1[1] + static_cast<int64_t>(kj) * a.s1[2];
-    if (n_iter > 0) {
-      store_acc_rows<D>(lane_addr + kColDV, dv_row, 1.0f, st_ok);
-      store_acc_rows<D>(lane_addr + kColDK, dk_row, a.scale, st_ok);
-    } else if (st_ok) {
-      for (int x = 0; x < D; x += 8) {
-        *reinterpret_cast<uint4*>(dk_row + x) = make_uint4(0, 0, 0, 0);
-        *reinterpret_cast<uint4*>(dv_row + x) = make_uint4(0, 0, 0, 0);
-      }
-    }
-  }
-  tc_fence_before();
-  __syncthreads();
-  if (warp == 0) tmem_dealloc(tmem, kTmemCols);
+  __syncwarp();
+  if (lane_id() == 0) mbar_arrive(bar);
 }
 
 // ================================== dQ pass =================================================
+// TMEM columns: S[2] at 0 / 128 (dS of a step is written as bf16 over its own S), dP at 256,
+// dQ at 384.
 template <int D, int BS>
-__global__ void __launch_bounds__(128, 1)
+__global__ void __launch_bounds__(kBwdThreads, 1)
 bwd_dq_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUtensorMap tm_k,
               const __grid_constant__ CUtensorMap tm_v, const __grid_constant__ CUtensorMap tm_do,
               const BwdArgs a) {
   using SM = BwdSmem<D, BS>;
   constexpr int R = 128 / BS;
-  constexpr int NBOX = D / 64;
-  constexpr uint32_t kColS = 0, kColDP = BS, kColDQ = 2 * BS;
-  constexpr uint32_t kTmemCols = (2 * BS + D) <= 256 ? 256 : 512;
+  constexpr uint32_t kColS = 0, kColDP = 256, kColDQ = 384;
+  constexpr int kTile = SM::kTile;
+  enum { B_FIX = 0, B_KF = 1, B_KE = 4, B_VF = 7, B_VE = 9, B_SF = 11, B_DPF = 13, B_DSF = 14, B_DONE = 15,
+         B_DRAIN = 16, B_COUNT = 17 };
 
-  extern __shared__ uint8_t smem_raw[];
-  uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
-  uint8_t* sQ = smem;
-  uint8_t* sDO = sQ + SM::kFixBytes;
-  uint8_t* sK = sDO + SM::kFixBytes;                // [stage]
-  uint8_t* sV = sK + 2 * SM::kStgBytes;             // [stage]
-  uint64_t* bars = reinterpret_cast<uint64_t*>(smem + SM::kBarOff);
-  uint64_t* bar_fix = bars + 0;
-  uint64_t* bar_ld = bars + 1;
-  uint64_t* bar_s = bars + 3;
-  uint64_t* bar_o = bars + 4;
-  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 5);
-  volatile uint32_t* s_fail = tmem_slot + 1;
+  extern __shared__ __align__(1024) uint8_t smem[];
+  uint64_t* bars = reinterpret_cast<uint64_t*>(smem + SM::oBar);
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + B_COUNT);
+  const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+  if ((smem_u32(smem) & 1023u) != 0) {   // the swizzled tiles need 1024-byte alignment
+    if (tid == 0) atomicCAS(a.error_word, 0u, (2u << 24) | 20u);
+    return;
+  }
+  uint8_t* sQ = smem + SM::oFix0;
+  uint8_t* sDO = smem + SM::oFix1;
+  uint8_t* sK = smem + SM::oA;
+  uint8_t* sV = smem + SM::oB;
 
-  const int tid = threadIdx.x, warp = tid >> 5;
   const int tile = a.order[blockIdx.y];
   const int b = blockIdx.x / a.Hq, h = blockIdx.x % a.Hq, hk = h / a.G;
   const int n_ent = a.tile_cnt[tile];
   const int32_t* ent = a.tile_ent + a.tile_off[tile * R];
   const int row0 = tile * 128;
+  const int n_steps = (BS == 128) ? n_ent : (n_ent + 1) / 2;
 
-  if (warp == 0) {
-    tmem_alloc(tmem_slot, kTmemCols);
-    tmem_relinquish();
-  }
   if (tid == 0) {
-    *s_fail = 0;
-    mbar_init(bar_fix, 1);
-    mbar_init(bar_ld + 0, 1);
-    mbar_init(bar_ld + 1, 1);
-    mbar_init(bar_s, 1);
-    mbar_init(bar_o, 1);
+    mbar_init(bars + B_FIX, 1);
+    for (int i = 0; i < 3; ++i) { mbar_init(bars + B_KF + i, 1); mbar_init(bars + B_KE + i, 1); }
+    for (int i = 0; i < 2; ++i) { mbar_init(bars + B_VF + i, 1); mbar_init(bars + B_VE + i, 1); mbar_init(bars + B_SF + i, 1); }
+    mbar_init(bars + B_DPF, 1);
+    mbar_init(bars + B_DSF, 8);
+    mbar_init(bars + B_DONE, 1);
+    mbar_init(bars + B_DRAIN, 1);
     mbar_fence_init();
-    tma_prefetch_desc(&tm_q);
-    tma_prefetch_desc(&tm_k);
-    tma_prefetch_desc(&tm_v);
-    tma_prefetch_desc(&tm_do);
+  }
+  if (warp == 9) {
+    tmem_alloc(tmem_slot, 512);
+    tmem_relinquish();
   }
   tc_fence_before();
   __syncthreads();
   tc_fence_after();
   const uint32_t tmem = *tmem_slot;
-  const uint32_t lane_addr = tmem + (static_cast<uint32_t>(warp * 32) << 16);
 
-  auto issue_ld = [&](int e) {
-    const int st = e & 1;
-    const int kb = ent[e] >> 2;
-    mbar_expect_tx(bar_ld + st, 2 * SM::kStgBytes);
-#pragma unroll
-    for (int x = 0; x < NBOX; ++x) {
-      tma_load_4d(sK + st * SM::kStgBytes + x * (BS * 128), &tm_k, bar_ld + st, x * 64, kb * BS, hk, b);
-      tma_load_4d(sV + st * SM::kStgBytes + x * (BS * 128), &tm_v, bar_ld + st, x * 64, kb * BS, hk, b);
-    }
-  };
-
-  if (tid == 0) {
-    mbar_expect_tx(bar_fix, 2 * SM::kFixBytes);
-#pragma unroll
-    for (int x = 0; x < NBOX; ++x) {
-      tma_load_4d(sQ + x * (128 * 128), &tm_q, bar_fix, x * 64, row0, h, b);
-      tma_load_4d(sDO + x * (128 * 128), &tm_do, bar_fix, x * 64, row0, h, b);
-    }
-    if (n_ent > 0) issue_ld(0);
-  }
-
-  constexpr uint32_t idesc_s = make_idesc_bf16(128, BS, 0, 0);
-  constexpr uint32_t idesc_dq = make_idesc_bf16(128, D, 0, 1);
-  const int r = tid;
-  const int qi = row0 + r;
-  const int member = (R == 1) ? 0 : (r / BS);
-  float lse2 = 0.f, dlt = 0.f;
-  if (qi < a.L) {
-    const int64_t off = (static_cast<int64_t>(b) * a.Hq + h) * a.L + qi;
-    lse2 = a.lse[off] * 1.4426950408889634f;
-    dlt = a.delta[off];
-  }
-  bool fail = false;
-
-  for (int e = 0; e < n_ent; ++e) {
-    const int st = e & 1;
-    const int entry = ent[e];
-    const int kb = entry >> 2;
-    if (tid == 0) {
-      if (e == 0) fail |= !mbar_wait(bar_fix, 0, a.error_word, 21);
-      if (e > 0) fail |= !mbar_wait(bar_o, (e - 1) & 1, a.error_word, 22);
-      if (!fail && e + 1 < n_ent) issue_ld(e + 1);
-      fail |= !mbar_wait(bar_ld + st, (e >> 1) & 1, a.error_word, 23);
-      if (!fail) {
-        tc_fence_after();
-        const uint32_t q_base = smem_u32(sQ), do_base = smem_u32(sDO);
-        const uint32_t k_base = smem_u32(sK + st * SM::kStgBytes), v_base = smem_u32(sV + st * SM::kStgBytes);
-#pragma unroll
-        for (int k = 0; k < D / 16; ++k) {
-          const uint32_t fo = (k >> 2) * (128 * 128) + (k & 3) * 32, so = (k >> 2) * (BS * 128) + (k & 3) * 32;
-          mma_ss(tmem + kColS, make_smem_desc(q_base + fo, 16, 1024), make_smem_desc(k_base + so, 16, 1024),
-                 idesc_s, k > 0);
-        }
-#pragma unroll
-        for (int k = 0; k < D / 16; ++k) {
-          const uint32_t fo = (k >> 2) * (128 * 128) + (k & 3) * 32, so = (k >> 2) * (BS * 128) + (k & 3) * 32;
-          mma_ss(tmem + kColDP, make_smem_desc(do_base + fo, 16, 1024), make_smem_desc(v_base + so, 16, 1024),
-                 idesc_s, k > 0);
-        }
+  if (warp == 8) {
+    // ------------------------------ TMA producer ------------------------------------------
+    if (lane == 0) {
+      tma_prefetch_desc(&tm_q); tma_prefetch_desc(&tm_k); tma_prefetch_desc(&tm_v); tma_prefetch_desc(&tm_do);
+      mbar_expect_tx(bars + B_FIX, 2 * kTile);
+      tma_load_rows<D, 128>(sQ, &tm_q, bars + B_FIX, 0, row0, h, b);
+      tma_load_rows<D, 128>(sDO, &tm_do, bars + B_FIX, 0, row0, h, b);
+      bool ok = true;
+      int nk = 0, nv = 0;   // loads started
+      for (int j = 0; j < n_steps; ++j) {
+        const int sk = j % 3, sv = j & 1;
+        const int e0 = (BS == 128) ? j : 2 * j, e1 = min(2 * j + 1, n_ent - 1);
+        const int kb0 = ent[e0] >> 2, kb1 = (BS == 64) ? (ent[e1] >> 2) : 0;
+        if (j >= 3) ok = mbar_wait(bars + B_KE + sk, ((j / 3) - 1) & 1, a.error_word, 21);
+        if (!ok) break;
+        mbar_expect_tx(bars + B_KF + sk, kTile);
+        tma_load_rows<D, BS>(sK + sk * kTile, &tm_k, bars + B_KF + sk, 0, kb0 * BS, hk, b);
+        if (BS == 64) tma_load_rows<D, BS>(sK + sk * kTile, &tm_k, bars + B_KF + sk, 1, kb1 * BS, hk, b);
+        nk = j + 1;
+        if (j >= 2) ok = mbar_wait(bars + B_VE + sv, ((j / 2) - 1) & 1, a.error_word, 22);
+        if (!ok) break;
+        mbar_expect_tx(bars + B_VF + sv, kTile);
+        tma_load_rows<D, BS>(sV + sv * kTile, &tm_v, bars + B_VF + sv, 0, kb0 * BS, hk, b);
+        if (BS == 64) tma_load_rows<D, BS>(sV + sv * kTile, &tm_v, bars + B_VF + sv, 1, kb1 * BS, hk, b);
+        nv = j + 1;
       }
-      mma_commit(bar_s);
+      // Before leaving, make sure every copy this thread started has landed (they all have
+      // when the kernel ran normally; after a failed wait this keeps shared memory ours).
+      mbar_wait(bars + B_FIX, 0, a.error_word, 26);
+      for (int j = max(nk - 3, 0); j < nk; ++j) mbar_wait(bars + B_KF + j % 3, (j / 3) & 1, a.error_word, 27);
+      for (int j = max(nv - 2, 0); j < nv; ++j) mbar_wait(bars + B_VF + (j & 1), (j / 2) & 1, a.error_word, 28);
     }
-    fail |= !mbar_wait(bar_s, e & 1, a.error_word, 24);
-    tc_fence_after();
-
-    const bool need_mask = ((entry & 3) != ((1 << R) - 1)) || (kb * BS + BS - 1 > row0);
-    const bool row_on = (entry >> member) & 1;
-    const int jmax = need_mask ? (row_on ? qi - kb * BS : -1) : BS;   // columns <= jmax visible
+  } else if (warp == 9) {
+    // ------------------------------ MMA issuer --------------------------------------------
+    if (lane == 0) {
+      constexpr uint32_t idesc_s = make_idesc_bf16(128, 128, 0, 0);
+      constexpr uint32_t idesc_dq = make_idesc_bf16(128, D, 0, 1);
+      const uint32_t q_base = smem_u32(sQ), do_base = smem_u32(sDO), k_base = smem_u32(sK), v_base = smem_u32(sV);
+      bool ok = mbar_wait(bars + B_FIX, 0, a.error_word, 23);
+      auto issue_s = [&](int j) {
+        const int sk = j % 3;
+        ok = ok && mbar_wait(bars + B_KF + sk, (j / 3) & 1, a.error_word, 24);
+        if (ok) {
+          tc_fence_after();
 #pragma unroll
-    for (int c = 0; c < BS / 32; ++c) {
-      uint32_t sreg[32], dreg[32], dsreg[16];
-      tmem_ld32(lane_addr + kColS + c * 32, sreg);
-      tmem_ld32(lane_addr + kColDP + c * 32, dreg);
-      tmem_ld_wait();
+          for (int k = 0; k < D / 16; ++k) {
+            const uint32_t off = (k >> 2) * BwdTile<D>::kBox + (k & 3) * 32;
+            mma_ss(tmem + kColS + (j & 1) * 128, make_smem_desc(q_base + off, 16, 1024),
+                   make_smem_desc(k_base + sk * kTile + off, 16, 1024), idesc_s, k > 0);
+          }
+        }
+        mma_commit(bars + B_SF + (j & 1));
+      };
+      auto issue_dp = [&](int j) {
+        const int sv = j & 1;
+        ok = ok && mbar_wait(bars + B_VF + sv, (j / 2) & 1, a.error_word, 25);
+        if (ok) {
+          tc_fence_after();
 #pragma unroll
-      for (int x = 0; x < 32; x += 2) {
-        const int col = c * 32 + x;
-        float p0 = fast_exp2(__uint_as_float(sreg[x]) * a.scale_log2 - lse2);
-        float p1 = fast_exp2(__uint_as_float(sreg[x + 1]) * a.scale_log2 - lse2);
-        p0 = (col <= jmax) ? p0 : 0.f;
-        p1 = (col + 1 <= jmax) ? p1 : 0.f;
-        dsreg[x >> 1] = pack_bf16(p0 * (__uint_as_float(dreg[x]) - dlt), p1 * (__uint_as_float(dreg[x + 1]) - dlt));
+          for (int k = 0; k < D / 16; ++k) {
+            const uint32_t off = (k >> 2) * BwdTile<D>::kBox + (k & 3) * 32;
+            mma_ss(tmem + kColDP, make_smem_desc(do_base + off, 16, 1024),
+                   make_smem_desc(v_base + sv * kTile + off, 16, 1024), idesc_s, k > 0);
+          }
+        }
+        mma_commit(bars + B_DPF);
+        mma_commit(bars + B_VE + sv);
+      };
+      if (n_steps > 0) {
+        issue_s(0);
+        issue_dp(0);
+        if (n_steps > 1) issue_s(1);
       }
-      tmem_st16(lane_addr + kColS + c * 16, dsreg);   // dS over the S columns already read
+      for (int j = 0; j < n_steps; ++j) {
+        ok = ok && mbar_wait(bars + B_DSF, j & 1, a.error_word, 29);
+        if (ok) {
+          tc_fence_after();
+          const uint32_t kst = k_base + (j % 3) * kTile;
+#pragma unroll
+          for (int kk = 0; kk < 8; ++kk)
+            mma_ts(tmem + kColDQ, tmem + kColS + (j & 1) * 128 + (kk >> 2) * 64 + (kk & 3) * 8,
+                   make_smem_desc(kst + kk * 2048, BwdTile<D>::kBox, 1024), idesc_dq, (j > 0) || (kk > 0));
+        }
+        mma_commit(bars + B_KE + j % 3);
+        if (j + 1 < n_steps) issue_dp(j + 1);
+        if (j + 2 < n_steps) issue_s(j + 2);
+      }
+      mma_commit(bars + B_DONE);
+      mma_commit(bars + B_DRAIN);
+      mbar_wait(bars + B_DRAIN, 0, a.error_word, 30);   // nothing of ours is still running at exit
     }
-    tmem_st_wait();
-    tc_fence_before();
-    if (fail) *s_fail = 1;
-    __syncthreads();
-    const bool cta_fail = *s_fail != 0;
-    if (tid == 0) {
+  } else {
+    // ------------------------------ element-wise warps ------------------------------------
+    const int wg = warp >> 2;                               // column half
+    const int r = (warp & 3) * 32 + lane;                   // query row in the tile == TMEM lane
+    const int qi = row0 + r;
+    const int member = (R == 1) ? 0 : (r / BS);
+    const uint32_t lane_addr = tmem + (static_cast<uint32_t>((warp & 3) * 32) << 16);
+    float lse2 = 0.f, dlt = 0.f;
+    if (qi < a.L) {
+      const float2 st = a.stat[(static_cast<int64_t>(b) * a.Hq + h) * a.L + qi];
+      lse2 = st.x;
+      dlt = st.y;
+    }
+    bool ok = true;
+    for (int j = 0; j < n_steps; ++j) {
+      // which keys do my 64 columns hold, and how many of them may this row see
+      int e = (BS == 128) ? j : 2 * j + wg;
+      const bool have = e < n_ent;
+      e = have ? e : n_ent - 1;
+      const int entry = ent[e];
+      const int key0 = (entry >> 2) * BS + (BS == 128 ? 64 * wg : 0);
+      const bool on = have && ((entry >> member) & 1);
+      const int lim = on ? min(max(qi - key0 + 1, 0), 64) : 0;   // columns c < lim are visible
+
+      ok = mbar_wait(bars + B_SF + (j & 1), (j >> 1) & 1, a.error_word, 31);
+      ok = __all_sync(0xffffffffu, ok);
+      if (!ok) break;
       tc_fence_after();
-      if (!cta_fail) {
-        const uint32_t k_base = smem_u32(sK + st * SM::kStgBytes);
+      float p[64];
+      {
+        uint32_t sreg[64];
+        tmem_ld32(lane_addr + kColS + (j & 1) * 128 + wg * 64, sreg);
+        tmem_ld32(lane_addr + kColS + (j & 1) * 128 + wg * 64 + 32, sreg + 32);
+        tmem_ld_wait();
+        if (__any_sync(0xffffffffu, lim < 64)) {
 #pragma unroll
-        for (int k = 0; k < BS / 16; ++k)
-          mma_ts(tmem + kColDQ, tmem + kColS + k * 8, make_smem_desc(k_base + k * 2048, BS * 128, 1024), idesc_dq,
-                 (e > 0) || (k > 0));
+          for (int c = 0; c < 64; ++c) {
+            const float v = fast_exp2(fmaf(__uint_as_float(sreg[c]), a.scale_log2, -lse2));
+            p[c] = (c < lim) ? v : 0.f;
+          }
+        } else {
+#pragma unroll
+          for (int c = 0; c < 64; ++c) p[c] = fast_exp2(fmaf(__uint_as_float(sreg[c]), a.scale_log2, -lse2));
+        }
       }
-      mma_commit(bar_o);
+      ok = mbar_wait(bars + B_DPF, j & 1, a.error_word, 32);
+      ok = __all_sync(0xffffffffu, ok);
+      if (!ok) break;
+      tc_fence_after();
+      uint32_t dsreg[32];
+#pragma unroll
+      for (int c = 0; c < 2; ++c) {
+        uint32_t dreg[32];
+        tmem_ld32(lane_addr + kColDP + wg * 64 + c * 32, dreg);
+        tmem_ld_wait();
+#pragma unroll
+        for (int x = 0; x < 32; x += 2)
+          dsreg[c * 16 + (x >> 1)] = pack_bf16(p[c * 32 + x] * (__uint_as_float(dreg[x]) - dlt),
+                                               p[c * 32 + x + 1] * (__uint_as_float(dreg[x + 1]) - dlt));
+      }
+      tmem_st32(lane_addr + kColS + (j & 1) * 128 + wg * 64, dsreg);   // dS over my own S columns
+      ew_publish(bars + B_DSF);
     }
-    if (cta_fail) { fail = true; break; }
-  }
-
-  if (n_ent > 0) {
-    fail |= !mbar_wait(bar_o, (n_ent - 1) & 1, a.error_word, 25);
-    tc_fence_after();
-  }
-  {
-    const bool st_ok = !fail && qi < a.L;
-    __nv_bfloat16* dq_row = a.out0 + b * a.s0[0] + h * a.s0[1] + static_cast<int64_t>(qi) * a.s0[2];
-    if (n_ent > 0) store_acc_rows<D>(lane_addr + kColDQ, dq_row, a.scale, st_ok);
+    // ---- epilogue: dQ * scale -> bf16 -------------------------------------------------------
+    if (ok && n_steps > 0) {
+      ok = mbar_wait(bars + B_DONE, 0, a.error_word, 33);
+      ok = __all_sync(0xffffffffu, ok);
+    }
+    if (ok) {
+      tc_fence_after();
+      if (qi < a.L) {   // warp-uniform: L is a multiple of 64
+        __nv_bfloat16* dq_row = a.out0 + b * a.s0[0] + h * a.s0[1] + static_cast<int64_t>(qi) * a.s0[2] + wg * (D / 2);
+        if (n_steps > 0) {
+          store_acc_cols<D / 2>(lane_addr + kColDQ + wg * (D / 2), dq_row, a.scale, true);
+        } else {
+#pragma unroll
+          for (int x = 0; x < D / 2; x += 8) *reinterpret_cast<uint4*>(dq_row + x) = make_uint4(0, 0, 0, 0);
+        }
+      }
+    }
   }
   tc_fence_before();
   __syncthreads();
-  if (warp == 0) tmem_dealloc(tmem, kTmemCols);
+  if (warp == 9) tmem_dealloc(tmem, 512);
+}
+
+// ============================== dK / dV pass ==================================================
+// TMEM columns: S^T at 0 (P^T written as bf16 over it), dP^T at 128 (dS^T over it), dV at 256,
+// dK at 384.  Items = (query head of the group, entry of the tile's CSC schedule) in a fixed
+// order; a step takes one item (128-token blocks) or two (64-token blocks).
+template <int D, int BS>
+__global__ void __launch_bounds__(kBwdThreads, 1)
+bwd_dkdv_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUtensorMap tm_k,
+                const __grid_constant__ CUtensorMap tm_v, const __grid_constant__ CUtensorMap tm_do,
+                const BwdArgs a) {
+  using SM = BwdSmem<D, BS>;
+  constexpr int R = 128 / BS;
+  constexpr uint32_t kColS = 0, kColDP = 128, kColDV = 256, kColDK = 384;
+  constexpr int kTile = SM::kTile;
+  enum { B_FIX = 0, B_QF = 1, B_QE = 4, B_OF = 7, B_OE = 9, B_SF = 11, B_DPF = 12, B_PF = 13, B_DSF = 14,
+         B_DONE = 15, B_DRAIN = 16, B_STF = 17, B_COUNT = 18 };
+
+  extern __shared__ __align__(1024) uint8_t smem[];
+  uint64_t* bars = reinterpret_cast<uint64_t*>(smem + SM::oBar);
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + B_COUNT);
+  const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+  if ((smem_u32(smem) & 1023u) != 0) {
+    if (tid == 0) atomicCAS(a.error_word, 0u, (2u << 24) | 10u);
+    return;
+  }
+  uint8_t* sK = smem + SM::oFix0;
+  uint8_t* sV = smem + SM::oFix1;
+  uint8_t* sQ = smem + SM::oA;     // [3]
+  uint8_t* sDO = smem + SM::oB;    // [2]
+  float2* sStat = reinterpret_cast<float2*>(smem + SM::oStat);   // [2][128]
+
+  const int tile = a.order[blockIdx.y];
+  const int b = blockIdx.x / a.Hkv, hk = blockIdx.x % a.Hkv;
+  const int n_ent = a.tile_cnt[tile];
+  const int32_t* ent = a.tile_ent + a.tile_off[tile * R];
+  const int key0 = tile * 128;
+  const int n_items = n_ent * a.G;
+  const int n_steps = (BS == 128) ? n_items : (n_items + 1) / 2;
+
+  // item -> (query head, first query row, entry)
+  auto item_of = [&](int it, int& hq, int& qrow, int& entry) {
+    const int g = it / n_ent, e = it - g * n_ent;
+    entry = ent[e];
+    hq = hk * a.G + g;
+    qrow = (entry >> 2) * BS;
+  };
+
+  if (tid == 0) {
+    mbar_init(bars + B_FIX, 1);
+    for (int i = 0; i < 3; ++i) { mbar_init(bars + B_QF + i, 1); mbar_init(bars + B_QE + i, 1); }
+    for (int i = 0; i < 2; ++i) { mbar_init(bars + B_OF + i, 1); mbar_init(bars + B_OE + i, 1); }
+    mbar_init(bars + B_SF, 1);
+    mbar_init(bars + B_DPF, 1);
+    mbar_init(bars + B_PF, 8);
+    mbar_init(bars + B_DSF, 8);
+    mbar_init(bars + B_DONE, 1);
+    mbar_init(bars + B_DRAIN, 1);
+    mbar_init(bars + B_STF, 4);
+    mbar_fence_init();
+  }
+  if (warp == 9) {
+    tmem_alloc(tmem_slot, 512);
+    tmem_relinquish();
+  }
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  const uint32_t tmem = *tmem_slot;
+
+  if (warp == 8) {
+    // ------------------------------ TMA producer ------------------------------------------
+    if (lane == 0) {
+      tma_prefetch_desc(&tm_q); tma_prefetch_desc(&tm_k); tma_prefetch_desc(&tm_v); tma_prefetch_desc(&tm_do);
+      mbar_expect_tx(bars + B_FIX, 2 * kTile);
+      tma_load_rows<D, 128>(sK, &tm_k, bars + B_FIX, 0, key0, hk, b);
+      tma_load_rows<D, 128>(sV, &tm_v, bars + B_FIX, 0, key0, hk, b);
+      bool ok = true;
+      int nq = 0, no = 0;   // loads started
+      for (int j = 0; j < n_steps; ++j) {
+        const int sq = j % 3, so = j & 1;
+        int h0, r0, e0, h1 = 0, r1 = 0, e1;
+        item_of(BS == 128 ? j : 2 * j, h0, r0, e0);
+        if (BS == 64) item_of(min(2 * j + 1, n_items - 1), h1, r1, e1);
+        if (j >= 3) ok = mbar_wait(bars + B_QE + sq, ((j / 3) - 1) & 1, a.error_word, 11);
+        if (!ok) break;
+        mbar_expect_tx(bars + B_QF + sq, kTile);
+        tma_load_rows<D, BS>(sQ + sq * kTile, &tm_q, bars + B_QF + sq, 0, r0, h0, b);
+        if (BS == 64) tma_load_rows<D, BS>(sQ + sq * kTile, &tm_q, bars + B_QF + sq, 1, r1, h1, b);
+        nq = j + 1;
+        if (j >= 2) ok = mbar_wait(bars + B_OE + so, ((j / 2) - 1) & 1, a.error_word, 12);
+        if (!ok) break;
+        mbar_expect_tx(bars + B_OF + so, kTile);
+        tma_load_rows<D, BS>(sDO + so * kTile, &tm_do, bars + B_OF + so, 0, r0, h0, b);
+        if (BS == 64) tma_load_rows<D, BS>(sDO + so * kTile, &tm_do, bars + B_OF + so, 1, r1, h1, b);
+        no = j + 1;
+      }
+      mbar_wait(bars + B_FIX, 0, a.error_word, 16);
+      for (int j = max(nq - 3, 0); j < nq; ++j) mbar_wait(bars + B_QF + j % 3, (j / 3) & 1, a.error_word, 17);
+      for (int j = max(no - 2, 0); j < no; ++j) mbar_wait(bars + B_OF + (j & 1), (j / 2) & 1, a.error_word, 18);
+    }
+  } else if (warp == 9) {
+    // ------------------------------ MMA issuer --------------------------------------------
+    if (lane == 0) {
+      constexpr uint32_t idesc_st = make_idesc_bf16(128, 128, 0, 0);   // S^T, dP^T: N = streamed queries
+      constexpr uint32_t idesc_acc = make_idesc_bf16(128, D, 0, 1);    // dV, dK: B = dO / Q, MN-major
+      const uint32_t k_base = smem_u32(sK), v_base = smem_u32(sV), q_base = smem_u32(sQ), do_base = smem_u32(sDO);
+      bool ok = mbar_wait(bars + B_FIX, 0, a.error_word, 13);
+      auto issue_s = [&](int j) {
+        const int sq = j % 3;
+        ok = ok && mbar_wait(bars + B_QF + sq, (j / 3) & 1, a.error_word, 14);
+        if (ok) {
+          tc_fence_after();
+#pragma unroll
+          for (int k = 0; k < D / 16; ++k) {
+            const uint32_t off = (k >> 2) * BwdTile<D>::kBox + (k & 3) * 32;
+            mma_ss(tmem + kColS, make_smem_desc(k_base + off, 16, 1024),
+                   make_smem_desc(q_base + sq * kTile + off, 16, 1024), idesc_st, k > 0);
+          }
+        }
+        mma_commit(bars + B_SF);
+      };
+      auto issue_dk = [&](int j) {
+        ok = ok && mbar_wait(bars + B_DSF, j & 1, a.error_word, 15);
+        if (ok) {
+          tc_fence_after();
+          const uint32_t qst = q_base + (j % 3) * kTile;
+#pragma unroll
+          for (int kk = 0; kk < 8; ++kk)
+            mma_ts(tmem + kColDK, tmem + kColDP + (kk >> 2) * 64 + (kk & 3) * 8,
+                   make_smem_desc(qst + kk * 2048, BwdTile<D>::kBox, 1024), idesc_acc, (j > 0) || (kk > 0));
+        }
+        mma_commit(bars + B_QE + j % 3);
+      };
+      if (n_steps > 0) issue_s(0);
+      for (int j = 0; j < n_steps; ++j) {
+        const int so = j & 1;
+        if (j > 0) issue_dk(j - 1);
+        ok = ok && mbar_wait(bars + B_OF + so, (j / 2) & 1, a.error_word, 19);
+        if (ok) {
+          tc_fence_after();
+#pragma unroll
+          for (int k = 0; k < D / 16; ++k) {
+            const uint32_t off = (k >> 2) * BwdTile<D>::kBox + (k & 3) * 32;
+            mma_ss(tmem + kColDP, make_smem_desc(v_base + off, 16, 1024),
+                   make_smem_desc(do_base + so * kTile + off, 16, 1024), idesc_st, k > 0);
+          }
+        }
+        mma_commit(bars + B_DPF);
+        ok = ok && mbar_wait(bars + B_PF, j & 1, a.error_word, 9);
+        if (ok) {
+          tc_fence_after();
+          const uint32_t ost = do_base + so * kTile;
+#pragma unroll
+          for (int kk = 0; kk < 8; ++kk)
+            mma_ts(tmem + kColDV, tmem + kColS + (kk >> 2) * 64 + (kk & 3) * 8,
+                   make_smem_desc(ost + kk * 2048, BwdTile<D>::kBox, 1024), idesc_acc, (j > 0) || (kk > 0));
+        }
+        mma_commit(bars + B_OE + so);
+        if (j + 1 < n_steps) issue_s(j + 1);
+      }
+      if (n_steps > 0) issue_dk(n_steps - 1);
+      mma_commit(bars + B_DONE);
+      mma_commit(bars + B_DRAIN);
+      mbar_wait(bars + B_DRAIN, 0, a.error_word, 8);
+    }
+  } else {
+    // ------------------------------ element-wise warps ------------------------------------
+    const int wg = warp >> 2;
+    const int r = (warp & 3) * 32 + lane;                   // key row in the tile == TMEM lane
+    const int kj = key0 + r;
+    const int member = (R == 1) ? 0 : (r / BS);
+    const uint32_t lane_addr = tmem + (static_cast<uint32_t>((warp & 3) * 32) << 16);
+    const int col = tid & 127;                              // the column whose statistics I fetch
+    auto fetch_stat = [&](int j) -> float2 {
+      if (tid >= 128 || j >= n_steps) return make_float2(0.f, 0.f);
+      int it = (BS == 128) ? j : 2 * j + (col >> 6);
+      it = min(it, n_items - 1);
+      int hq, qrow, entry;
+      item_of(it, hq, qrow, entry);
+      return a.stat[(static_cast<int64_t>(b) * a.Hq + hq) * a.L + qrow + (BS == 128 ? col : (col & 63))];
+    };
+    // Statistics of step j sit in sStat[j & 1]; warps 0-3 write those of step j + 1 at the end
+    // of step j (by then every warp has left step j - 1: the dP^T of step j is only issued after
+    // all eight warps published dS^T of step j - 1) and publish them through B_STF.
+    auto publish_stat = [&](int j, float2 v) {
+      if (warp < 4) {
+        sStat[(j & 1) * 128 + col] = v;
+        __syncwarp();
+        if (lane == 0) mbar_arrive(bars + B_STF);
+      }
+    };
+    publish_stat(0, fetch_stat(0));
+    bool ok = true;
+    for (int j = 0; j < n_steps; ++j) {
+      const float2 nxt = fetch_stat(j + 1);
+      ok = mbar_wait(bars + B_STF, j & 1, a.error_word, 4);   // statistics of step j are in place
+      ok = __all_sync(0xffffffffu, ok);
+      if (!ok) break;
+      const float2* st = sStat + (j & 1) * 128 + wg * 64;
+      // which queries do my 64 columns hold, and from which of them on may this key be seen
+      int it = (BS == 128) ? j : 2 * j + wg;
+      const bool have = it < n_items;
+      it = have ? it : n_items - 1;
+      int hq, qrow, entry;
+      item_of(it, hq, qrow, entry);
+      const int q0 = qrow + (BS == 128 ? 64 * wg : 0);
+      const bool on = have && ((entry >> member) & 1);
+      const int xmin = on ? min(max(kj - q0, 0), 64) : 64;     // columns c >= xmin are visible
+
+      ok = mbar_wait(bars + B_SF, j & 1, a.error_word, 1);
+      ok = __all_sync(0xffffffffu, ok);
+      if (!ok) break;
+      tc_fence_after();
+      float p[64];
+      {
+        uint32_t sreg[64];
+        tmem_ld32(lane_addr + kColS + wg * 64, sreg);
+        tmem_ld32(lane_addr + kColS + wg * 64 + 32, sreg + 32);
+        tmem_ld_wait();
+        const bool masked = __any_sync(0xffffffffu, xmin > 0);
+#pragma unroll
+        for (int c = 0; c < 64; c += 2) {
+          const float4 s2 = *reinterpret_cast<const float4*>(st + c);   // (lse2, delta) of two columns
+          float v0 = fast_exp2(fmaf(__uint_as_float(sreg[c]), a.scale_log2, -s2.x));
+          float v1 = fast_exp2(fmaf(__uint_as_float(sreg[c + 1]), a.scale_log2, -s2.z));
+          if (masked) {
+            v0 = (c >= xmin) ? v0 : 0.f;
+            v1 = (c + 1 >= xmin) ? v1 : 0.f;
+          }
+          p[c] = v0;
+          p[c + 1] = v1;
+        }
+        uint32_t preg[32];
+#pragma unroll
+        for (int c = 0; c < 64; c += 2) preg[c >> 1] = pack_bf16(p[c], p[c + 1]);
+        tmem_st32(lane_addr + kColS + wg * 64, preg);        // P^T over my own S^T columns
+        ew_publish(bars + B_PF);
+      }
+      ok = mbar_wait(bars + B_DPF, j & 1, a.error_word, 2);
+      ok = __all_sync(0xffffffffu, ok);
+      if (!ok) break;
+      tc_fence_after();
+      uint32_t dsreg[32];
+#pragma unroll
+      for (int c = 0; c < 2; ++c) {
+        uint32_t dreg[32];
+        tmem_ld32(lane_addr + kColDP + wg * 64 + c * 32, dreg);
+        tmem_ld_wait();
+#pragma unroll
+        for (int x = 0; x < 32; x += 2) {
+          const float4 s2 = *reinterpret_cast<const float4*>(st + c * 32 + x);
+          dsreg[c * 16 + (x >> 1)] = pack_bf16(p[c * 32 + x] * (__uint_as_float(dreg[x]) - s2.y),
+                                               p[c * 32 + x + 1] * (__uint_as_float(dreg[x + 1]) - s2.w));
+        }
+      }
+      tmem_st32(lane_addr + kColDP + wg * 64, dsreg);        // dS^T over my own dP^T columns
+      ew_publish(bars + B_DSF);
+      publish_stat(j + 1, nxt);
+    }
+    // ---- epilogue: dV, dK * scale -> bf16 ---------------------------------------------------
+    if (ok && n_steps > 0) {
+      ok = mbar_wait(bars + B_DONE, 0, a.error_word, 3);
+      ok = __all_sync(0xffffffffu, ok);
+    }
+    if (ok) {
+      tc_fence_after();
+      if (kj < a.L) {
+        __nv_bfloat16* dk_row = a.out0 + b * a.s0[0] + hk * a.s0[1] + static_cast<int64_t>(kj) * a.s0[2] + wg * (D / 2);
+        __nv_bfloat16* dv_row = a.out1 + b * a.s1[0] + hk * a.s1[1] + static_cast<int64_t>(kj) * a.s1[2] + wg * (D / 2);
+        if (n_steps > 0) {
+          store_acc_cols<D / 2>(lane_addr + kColDV + wg * (D / 2), dv_row, 1.0f, true);
+          store_acc_cols<D / 2>(lane_addr + kColDK + wg * (D / 2), dk_row, a.scale, true);
+        } else {
+#pragma unroll
+          for (int x = 0; x < D / 2; x += 8) {
+            *reinterpret_cast<uint4*>(dk_row + x) = make_uint4(0, 0, 0, 0);
+            *reinterpret_cast<uint4*>(dv_row + x) = make_uint4(0, 0, 0, 0);
+          }
+        }
+      }
+    }
+  }
+  tc_fence_before();
+  __syncthreads();
+  if (warp == 9) tmem_dealloc(tmem, 512);
 }
 
 }  // namespace lg

@@ -29,7 +29,7 @@ struct WsLayout {
   size_t row_ptr, col_idx, col_ptr, row_idx;     // the CSR / CSC lists
   size_t qt_cnt, qt_ent, qt_order;               // query-tile schedules (fwd, dQ pass)
   size_t kt_cnt, kt_ent, kt_order;               // kv-tile schedules (dK/dV pass)
-  size_t delta;                                  // fp32 [B, Hq, L] (bwd only)
+  size_t delta;                                  // float2 [B, Hq, L]: (LSE * log2 e, delta) (bwd only)
   size_t total;
 };
 WsLayout ws_layout(const Resolved& r, bool want_bwd);
