@@ -71,6 +71,7 @@ lg_status resolve(const lg_attn_params* p, Resolved* r) {
   if ((s = fix_strides(p->o_strides, p->Hq, p->L, p->D, r->os)) != LG_OK) return s;
   r->n_qtiles = (p->L + 127) / 128;
   r->n_ktiles = (p->L + 127) / 128;
+  r->n_stiles = (p->L + 255) / 256;
   // nnz from the per-row counts of each pattern
   int64_t nnz = 0;
   const PatternDev& pt = r->pat;
@@ -108,6 +109,9 @@ WsLayout ws_layout(const Resolved& r, bool want_bwd) {
   w.qt_cnt = take(r.n_qtiles * 4);
   w.qt_ent = take(nnz * 4);
   w.qt_order = take(r.n_qtiles * 4);
+  w.sq_cnt = take(r.n_stiles * 4);
+  w.sq_ent = take(nnz * 4);
+  w.sq_order = take(r.n_stiles * 4);
   if (want_bwd) {
     w.kt_cnt = take(r.n_ktiles * 4);
     w.kt_ent = take(nnz * 4);
@@ -137,6 +141,9 @@ lg_status prepare_workspace(const Resolved& r, const WsLayout& w, uint8_t* ws, b
   tile_merge_kernel<<<(r.n_qtiles + 127) / 128, 128, 0, stream>>>(i32(w.row_ptr), i32(w.col_idx), r.pat.nB, R,
                                                                   r.n_qtiles, i32(w.qt_cnt), i32(w.qt_ent));
   tile_order_kernel<<<(r.n_qtiles + 127) / 128, 128, 0, stream>>>(i32(w.qt_cnt), r.n_qtiles, i32(w.qt_order));
+  tile_merge4_kernel<<<(r.n_stiles + 127) / 128, 128, 0, stream>>>(i32(w.row_ptr), i32(w.col_idx), r.pat.nB, 2 * R,
+                                                                   r.n_stiles, i32(w.sq_cnt), i32(w.sq_ent));
+  tile_order_kernel<<<(r.n_stiles + 127) / 128, 128, 0, stream>>>(i32(w.sq_cnt), r.n_stiles, i32(w.sq_order));
   if (want_bwd) {
     tile_merge_kernel<<<(r.n_ktiles + 127) / 128, 128, 0, stream>>>(i32(w.col_ptr), i32(w.row_idx), r.pat.nB, R,
                                                                     r.n_ktiles, i32(w.kt_cnt), i32(w.kt_ent));

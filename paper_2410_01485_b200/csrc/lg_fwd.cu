@@ -14,9 +14,9 @@ static lg_status launch_fwd_t(const Resolved& r, const WsLayout& w, const void* 
   if ((s = make_tmap(&tv, v, r.B, r.Hkv, r.L, D, r.vs, BS)) != LG_OK) return s;
   FwdArgs a;
   a.tile_off = reinterpret_cast<const int32_t*>(ws + w.row_ptr);
-  a.tile_cnt = reinterpret_cast<const int32_t*>(ws + w.qt_cnt);
-  a.tile_ent = reinterpret_cast<const int32_t*>(ws + w.qt_ent);
-  a.order = reinterpret_cast<const int32_t*>(ws + w.qt_order);
+  a.tile_cnt = reinterpret_cast<const int32_t*>(ws + w.sq_cnt);
+  a.tile_ent = reinterpret_cast<const int32_t*>(ws + w.sq_ent);
+  a.order = reinterpret_cast<const int32_t*>(ws + w.sq_order);
   a.o = static_cast<__nv_bfloat16*>(o);
   a.lse = lse;
   a.error_word = reinterpret_cast<unsigned int*>(ws);
@@ -24,10 +24,10 @@ static lg_status launch_fwd_t(const Resolved& r, const WsLayout& w, const void* 
   a.L = r.L; a.Hq = r.Hq; a.G = r.G;
   a.scale_log2 = r.scale * 1.4426950408889634f;
   auto kern = fwd_kernel<D, BS>;
-  constexpr int smem = FwdSmem<D, BS>::kTotal;
+  constexpr int smem = FwdSmem<D>::kTotal;
   if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, smem) != cudaSuccess) return LG_ERR_CUDA;
-  dim3 grid(r.B * r.Hq, r.n_qtiles);
-  kern<<<grid, 128, smem, stream>>>(tq, tk, tv, a);
+  dim3 grid(r.B * r.Hq, r.n_stiles);
+  kern<<<grid, kFwdThreads, smem, stream>>>(tq, tk, tv, a);
   return cudaGetLastError() == cudaSuccess ? LG_OK : LG_ERR_CUDA;
 }
 

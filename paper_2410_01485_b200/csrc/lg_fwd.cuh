@@ -1,12 +1,19 @@
 // Forward pass of block-sparse causal attention (paper Section 3.2: a FlashAttention-style
 // kernel that never loads or computes a KV block whose mask is zero), with the log-sum-exp.
 //
-// One CTA owns a tile of 128 query rows of one head and walks the tile's schedule of active
-// KV blocks.  Per block: TMA brings K and V tiles into 128-byte-swizzled shared memory,
-// tcgen05.mma computes S = Q K^T into tensor memory, the 128 softmax threads (one per query
-// row = one TMEM lane) update the running max / sum, write P as bf16 back into tensor
-// memory, and a second tcgen05.mma accumulates O += P V with P read from tensor memory and
-// V as an MN-major shared-memory operand.
+// One CTA owns a super-tile of 256 query rows of one head: two tiles ("slots") of 128 rows
+// that share every K / V tile brought into shared memory.  It walks the ascending union of
+// the slots' active KV blocks in steps of 128 keys (one 128-token block, or two 64-token
+// blocks side by side); a slot that has nothing in a step skips it.  Roles:
+//   warps 0-3 / 4-7 : softmax of slot 0 / 1 (thread = query row = TMEM lane)
+//   warp 8          : TMA producer (Q once, then the K and V rings)
+//   warp 9, lane 0  : issues every tcgen05.mma
+// Tensor memory: S of slot s at columns 128 s (P is written as bf16 over its first 64
+// columns), O of slot s at 256 + 128 s.  MMA order
+//   S0(0) S1(0) | PV0(0) S0(1) PV1(0) S1(1) | PV0(1) S0(2) PV1(1) S1(2) | ...
+// so that while one slot's softmax runs, the tensor pipe works on the other slot.
+// The running maximum is only raised (and O rescaled) when it grew by more than 2^8; until
+// then probabilities are expressed relative to the older maximum, which fp32 / bf16 hold easily.
 #pragma once
 #include <cuda.h>
 #include "lg_common.cuh"
@@ -14,10 +21,10 @@
 namespace lg {
 
 struct FwdArgs {
-  const int32_t* tile_off;   // row_ptr (CSR): entries of tile t start at tile_off[R * t]
-  const int32_t* tile_cnt;   // [n_tiles]
-  const int32_t* tile_ent;   // kb * 4 + member mask
-  const int32_t* order;      // [n_tiles] launch rank -> tile
+  const int32_t* tile_off;   // row_ptr (CSR): entries of super-tile t start at tile_off[(256 / block) * t]
+  const int32_t* tile_cnt;   // [n_super_tiles]
+  const int32_t* tile_ent;   // kb * 16 + member mask (bit r: pattern row r of the super-tile has the block)
+  const int32_t* order;      // [n_super_tiles] launch rank -> super-tile
   __nv_bfloat16* o;
   float* lse;                // [B, Hq, L]
   unsigned int* error_word;
@@ -26,228 +33,317 @@ struct FwdArgs {
   float scale_log2;          // scale * log2(e)
 };
 
-template <int D, int BS>
+constexpr int kFwdThreads = 320;
+constexpr float kFwdRescaleThreshold = 8.0f;   // log2 units
+
+template <int D>
 struct FwdSmem {
-  static constexpr int kQBytes = 128 * D * 2;
-  static constexpr int kKVBytes = BS * D * 2;
-  static constexpr int kStages = 2;
-  static constexpr int kBarOff = kQBytes + 2 * kStages * kKVBytes;
-  static constexpr int kTotal = kBarOff + 128 + 1024;   // + barriers + alignment slack
+  static constexpr int kBox = 128 * 128;               // one 64-column box of 128 rows
+  static constexpr int kTile = (D / 64) * kBox;        // 128 rows x D bf16
+  static constexpr int kKStages = 3, kVStages = 2;
+  static constexpr int oQ = 0;                         // [2 slots]
+  static constexpr int oK = 2 * kTile;
+  static constexpr int oV = oK + kKStages * kTile;
+  static constexpr int oBar = oV + kVStages * kTile;
+  static constexpr int kTotal = oBar + 256;
 };
 
 template <int D, int BS>
-__global__ void __launch_bounds__(128, 1)
+__global__ void __launch_bounds__(kFwdThreads, 1)
 fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUtensorMap tm_k,
            const __grid_constant__ CUtensorMap tm_v, const FwdArgs a) {
-  using SM = FwdSmem<D, BS>;
-  constexpr int R = 128 / BS;                 // pattern rows per query tile
-  constexpr int NBOX = D / 64;                // 64-column TMA boxes per operand row
-  constexpr uint32_t kColS = 0, kColP = BS, kColO = BS + BS / 2;
-  constexpr uint32_t kTmemCols = (BS + BS / 2 + D) <= 256 ? 256 : 512;
+  using SM = FwdSmem<D>;
+  constexpr int R4 = 256 / BS;                  // pattern rows per super-tile (2 or 4)
+  constexpr int RS = R4 / 2;                    // pattern rows per slot
+  constexpr uint32_t kSlotMask = (1u << RS) - 1u;
+  constexpr int kTile = SM::kTile;
+  constexpr uint32_t kColS = 0, kColO = 256;
+  enum { B_Q = 0, B_KF = 1, B_KE = 4, B_VF = 7, B_VE = 9, B_SF = 11, B_PF = 13, B_OD = 15, B_DRAIN = 17, B_COUNT = 18 };
 
-  extern __shared__ uint8_t smem_raw[];
-  uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
-  uint8_t* sQ = smem;
-  uint8_t* sK = sQ + SM::kQBytes;                       // [stage][box][BS rows][128 B]
-  uint8_t* sV = sK + SM::kStages * SM::kKVBytes;
-  uint64_t* bars = reinterpret_cast<uint64_t*>(smem + SM::kBarOff);
-  uint64_t* bar_q = bars + 0;
-  uint64_t* bar_kv = bars + 1;                          // [2]
-  uint64_t* bar_s = bars + 3;
-  uint64_t* bar_o = bars + 4;
-  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 5);
-  volatile uint32_t* s_fail = tmem_slot + 1;   // set by any thread whose bounded wait expired
-
-  const int tid = threadIdx.x, warp = tid >> 5;
-  const int tile = a.order[blockIdx.y];
-  const int bh = blockIdx.x;
-  const int b = bh / a.Hq, h = bh % a.Hq, hk = h / a.G;
-  const int n_ent = a.tile_cnt[tile];
-  const int32_t* ent = a.tile_ent + a.tile_off[tile * R];
-  const int row0 = tile * 128;
-
-  if (warp == 0) {
-    tmem_alloc(tmem_slot, kTmemCols);
-    tmem_relinquish();
+  extern __shared__ __align__(1024) uint8_t smem[];
+  uint64_t* bars = reinterpret_cast<uint64_t*>(smem + SM::oBar);
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + B_COUNT);
+  const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+  if ((smem_u32(smem) & 1023u) != 0) {   // the swizzled tiles need 1024-byte alignment
+    if (tid == 0) atomicCAS(a.error_word, 0u, (2u << 24) | 1u);
+    return;
   }
+  uint8_t* sQ = smem + SM::oQ;
+  uint8_t* sK = smem + SM::oK;
+  uint8_t* sV = smem + SM::oV;
+
+  const int tile = a.order[blockIdx.y];
+  const int b = blockIdx.x / a.Hq, h = blockIdx.x % a.Hq, hk = h / a.G;
+  const int n_ent = a.tile_cnt[tile];
+  const int32_t* ent = a.tile_ent + a.tile_off[tile * R4];
+  const int row0 = tile * 256;
+  const int n_steps = (BS == 128) ? n_ent : (n_ent + 1) / 2;
+
+  // union of the member masks of the blocks of step j (0 past the end)
+  auto step_mask = [&](int j) -> uint32_t {
+    if (j >= n_steps) return 0u;
+    if (BS == 128) return static_cast<uint32_t>(ent[j]) & 15u;
+    const uint32_t m0 = static_cast<uint32_t>(ent[2 * j]) & 15u;
+    const uint32_t m1 = (2 * j + 1 < n_ent) ? (static_cast<uint32_t>(ent[2 * j + 1]) & 15u) : 0u;
+    return m0 | m1;
+  };
+
   if (tid == 0) {
-    *s_fail = 0;
-    mbar_init(bar_q, 1);
-    mbar_init(bar_kv + 0, 1);
-    mbar_init(bar_kv + 1, 1);
-    mbar_init(bar_s, 1);
-    mbar_init(bar_o, 1);
+    mbar_init(bars + B_Q, 1);
+    for (int i = 0; i < 3; ++i) { mbar_init(bars + B_KF + i, 1); mbar_init(bars + B_KE + i, 1); }
+    for (int i = 0; i < 2; ++i) {
+      mbar_init(bars + B_VF + i, 1); mbar_init(bars + B_VE + i, 1);
+      mbar_init(bars + B_SF + i, 1); mbar_init(bars + B_PF + i, 4); mbar_init(bars + B_OD + i, 1);
+    }
+    mbar_init(bars + B_DRAIN, 1);
     mbar_fence_init();
-    tma_prefetch_desc(&tm_q);
-    tma_prefetch_desc(&tm_k);
-    tma_prefetch_desc(&tm_v);
+  }
+  if (warp == 9) {
+    tmem_alloc(tmem_slot, 512);
+    tmem_relinquish();
   }
   tc_fence_before();
   __syncthreads();
   tc_fence_after();
   const uint32_t tmem = *tmem_slot;
-  const uint32_t lane_addr = tmem + (static_cast<uint32_t>(warp * 32) << 16);
 
-  auto issue_kv = [&](int e) {
-    const int st = e & 1;
-    const int kb = ent[e] >> 2;
-    mbar_expect_tx(bar_kv + st, 2 * SM::kKVBytes);
+  if (warp == 8) {
+    // ------------------------------ TMA producer ------------------------------------------
+    if (lane == 0) {
+      tma_prefetch_desc(&tm_q); tma_prefetch_desc(&tm_k); tma_prefetch_desc(&tm_v);
+      mbar_expect_tx(bars + B_Q, 2 * kTile);
 #pragma unroll
-    for (int x = 0; x < NBOX; ++x) {
-      tma_load_4d(sK + st * SM::kKVBytes + x * (BS * 128), &tm_k, bar_kv + st, x * 64, kb * BS, hk, b);
-      tma_load_4d(sV + st * SM::kKVBytes + x * (BS * 128), &tm_v, bar_kv + st, x * 64, kb * BS, hk, b);
-    }
-  };
-
-  if (tid == 0) {
-    mbar_expect_tx(bar_q, SM::kQBytes);
+      for (int s = 0; s < 2; ++s)
 #pragma unroll
-    for (int x = 0; x < NBOX; ++x) tma_load_4d(sQ + x * (128 * 128), &tm_q, bar_q, x * 64, row0, h, b);
-    if (n_ent > 0) issue_kv(0);
-    if (n_ent > 1) issue_kv(1);
-  }
-
-  constexpr uint32_t idesc_s = make_idesc_bf16(128, BS, 0, 0);
-  constexpr uint32_t idesc_o = make_idesc_bf16(128, D, 0, 1);
-
-  float m_run = -INFINITY;   // running max of scale*log2e*s
-  float l_run = 0.f;
-  const int r = tid;                       // query row inside the tile == TMEM lane
-  const int qi = row0 + r;
-  const int member = (R == 1) ? 0 : (r / BS);
-  bool fail = false;
-
-  for (int e = 0; e < n_ent; ++e) {
-    const int st = e & 1;
-    const int entry = ent[e];
-    const int kb = entry >> 2;
-    if (tid == 0) {
-      if (e == 0) fail |= !mbar_wait(bar_q, 0, a.error_word, 1);
-      fail |= !mbar_wait(bar_kv + st, (e >> 1) & 1, a.error_word, 2);
-      if (!fail) {
-        tc_fence_after();
-        const uint32_t q_base = smem_u32(sQ), k_base = smem_u32(sK + st * SM::kKVBytes);
+        for (int x = 0; x < D / 64; ++x)
+          tma_load_4d(sQ + s * kTile + x * SM::kBox, &tm_q, bars + B_Q, x * 64, row0 + s * 128, h, b);
+      auto load_step = [&](uint8_t* dst, const CUtensorMap* tm, uint64_t* bar, int kb0, int kb1) {
 #pragma unroll
-        for (int k = 0; k < D / 16; ++k) {
-          const uint64_t da = make_smem_desc(q_base + (k >> 2) * (128 * 128) + (k & 3) * 32, 16, 1024);
-          const uint64_t db = make_smem_desc(k_base + (k >> 2) * (BS * 128) + (k & 3) * 32, 16, 1024);
-          mma_ss(tmem + kColS, da, db, idesc_s, k > 0);
+        for (int x = 0; x < D / 64; ++x) {
+          tma_load_4d(dst + x * SM::kBox, tm, bar, x * 64, kb0 * BS, hk, b);
+          if (BS == 64) tma_load_4d(dst + x * SM::kBox + 64 * 128, tm, bar, x * 64, kb1 * BS, hk, b);
         }
+      };
+      bool ok = true;
+      int nk = 0, nv = 0;   // loads started
+      int e_next = n_steps > 0 ? ent[0] : 0, e_next1 = (BS == 64 && n_ent > 1) ? ent[1] : e_next;
+      for (int j = 0; j < n_steps; ++j) {
+        const int sk = j % 3, sv = j & 1;
+        const int kb0 = e_next >> 4, kb1 = e_next1 >> 4;
+        if (j + 1 < n_steps) {   // fetch the next step's entries now; they are needed one step later
+          const int i0 = (BS == 128) ? j + 1 : 2 * j + 2;
+          e_next = ent[i0];
+          e_next1 = (BS == 64) ? ent[min(i0 + 1, n_ent - 1)] : e_next;
+        }
+        if (j >= 3) ok = mbar_wait(bars + B_KE + sk, ((j / 3) - 1) & 1, a.error_word, 2);
+        if (!ok) break;
+        mbar_expect_tx(bars + B_KF + sk, kTile);
+        load_step(sK + sk * kTile, &tm_k, bars + B_KF + sk, kb0, kb1);
+        nk = j + 1;
+        if (j >= 2) ok = mbar_wait(bars + B_VE + sv, ((j / 2) - 1) & 1, a.error_word, 3);
+        if (!ok) break;
+        mbar_expect_tx(bars + B_VF + sv, kTile);
+        load_step(sV + sv * kTile, &tm_v, bars + B_VF + sv, kb0, kb1);
+        nv = j + 1;
       }
-      mma_commit(bar_s);   // always commit so the other threads' wait ends
+      // every copy this thread started has landed before the CTA may exit
+      mbar_wait(bars + B_Q, 0, a.error_word, 4);
+      for (int j = max(nk - 3, 0); j < nk; ++j) mbar_wait(bars + B_KF + j % 3, (j / 3) & 1, a.error_word, 5);
+      for (int j = max(nv - 2, 0); j < nv; ++j) mbar_wait(bars + B_VF + (j & 1), (j / 2) & 1, a.error_word, 6);
     }
-    fail |= !mbar_wait(bar_s, e & 1, a.error_word, 3);
-    tc_fence_after();
+  } else if (warp == 9) {
+    // ------------------------------ MMA issuer --------------------------------------------
+    if (lane == 0) {
+      constexpr uint32_t idesc_s = make_idesc_bf16(128, 128, 0, 0);
+      constexpr uint32_t idesc_o = make_idesc_bf16(128, D, 0, 1);
+      const uint32_t hi = desc_hi(1024);
+      const uint32_t q_lo = desc_lo(smem_u32(sQ), 16), k_lo = desc_lo(smem_u32(sK), 16);
+      const uint32_t v_mn_lo = desc_lo(smem_u32(sV), SM::kBox);
+      bool ok = mbar_wait(bars + B_Q, 0, a.error_word, 7);
+      int k_ready = -1, v_ready = -1;           // last step whose K / V tile this thread has seen complete
+      int n_pv[2] = {0, 0};                     // P V products issued per slot (accumulate flag, barrier phases)
+      auto issue_s = [&](int s, int j) {
+        const int sk = j % 3;
+        if (k_ready < j) {
+          ok = ok && mbar_wait(bars + B_KF + sk, (j / 3) & 1, a.error_word, 8);
+          k_ready = j;
+        }
+        if (ok) {
+          tc_fence_after();
+          const uint32_t a_lo = q_lo + s * (kTile >> 4), b_lo = k_lo + sk * (kTile >> 4);
+#pragma unroll
+          for (int k = 0; k < D / 16; ++k) {
+            constexpr int kB = SM::kBox >> 4;
+            const uint32_t off = (k >> 2) * kB + (k & 3) * 2;
+            mma_ss2(tmem + kColS + s * 128, a_lo + off, b_lo + off, hi, idesc_s, k > 0);
+          }
+        }
+        mma_commit(bars + B_SF + s);
+      };
+      auto issue_pv = [&](int s, int j) {
+        const int sv = j & 1;
+        if (v_ready < j) {
+          ok = ok && mbar_wait(bars + B_VF + sv, (j / 2) & 1, a.error_word, 9);
+          v_ready = j;
+        }
+        ok = ok && mbar_wait(bars + B_PF + s, n_pv[s] & 1, a.error_word, 10);
+        if (ok) {
+          tc_fence_after();
+          const uint32_t b_lo = v_mn_lo + sv * (kTile >> 4);
+#pragma unroll
+          for (int kk = 0; kk < 8; ++kk)
+            mma_ts2(tmem + kColO + s * 128, tmem + kColS + s * 128 + kk * 8, b_lo + kk * (2048 >> 4), hi, idesc_o,
+                    (n_pv[s] > 0) || (kk > 0));
+        }
+        ++n_pv[s];
+        mma_commit(bars + B_OD + s);
+      };
+      uint32_t m_cur = step_mask(0), m_nxt = step_mask(1);
+      if (n_steps > 0) {
+        if (m_cur & kSlotMask) issue_s(0, 0);
+        if ((m_cur >> RS) & kSlotMask) issue_s(1, 0);
+        mma_commit(bars + B_KE + 0);
+      }
+      for (int j = 0; j < n_steps; ++j) {
+        const uint32_t m_nxt2 = step_mask(j + 2);   // read two steps ahead: off the critical path
+        const bool c0 = m_cur & kSlotMask, c1 = (m_cur >> RS) & kSlotMask;
+        const bool x0 = m_nxt & kSlotMask, x1 = (m_nxt >> RS) & kSlotMask;
+        if (c0) issue_pv(0, j);
+        if (c0 && !c1) mma_commit(bars + B_VE + (j & 1));
+        if (x0) issue_s(0, j + 1);
+        if (x0 && !x1) mma_commit(bars + B_KE + (j + 1) % 3);
+        if (c1) { issue_pv(1, j); mma_commit(bars + B_VE + (j & 1)); }
+        if (x1) { issue_s(1, j + 1); mma_commit(bars + B_KE + (j + 1) % 3); }
+        m_cur = m_nxt;
+        m_nxt = m_nxt2;
+      }
+      mma_commit(bars + B_DRAIN);
+      mbar_wait(bars + B_DRAIN, 0, a.error_word, 11);   // nothing of ours is still running at exit
+    }
+  } else {
+    // ------------------------------ softmax warps -----------------------------------------
+    const int s = warp >> 2;                                 // slot
+    const int r = (warp & 3) * 32 + lane;                    // row in the slot == TMEM lane
+    const int qi = row0 + s * 128 + r;
+    const int member = s * RS + (BS == 128 ? 0 : (r >> 6));  // pattern row of the super-tile
+    const uint32_t lane_addr = tmem + (static_cast<uint32_t>((warp & 3) * 32) << 16);
+    const uint32_t my_s = lane_addr + kColS + s * 128, my_o = lane_addr + kColO + s * 128;
+    float m_ref = -INFINITY;   // reference maximum (scaled, log2 domain) the probabilities are relative to
+    float l_run = 0.f;
+    int cnt = 0;               // steps this slot took part in
+    bool ok = true;
+    auto load_ent = [&](int j, int& e0, int& e1) {
+      if (j >= n_steps) { e0 = e1 = 0; return; }
+      if (BS == 128) { e0 = e1 = ent[j]; return; }
+      e0 = ent[2 * j];
+      e1 = (2 * j + 1 < n_ent) ? ent[2 * j + 1] : (e0 & ~15);   // odd tail: same block, nobody's member
+    };
+    int ne0, ne1;
+    load_ent(0, ne0, ne1);
+    for (int j = 0; j < n_steps; ++j) {
+      const int e0 = ne0, e1 = ne1;
+      load_ent(j + 1, ne0, ne1);
+      const uint32_t m_step = (static_cast<uint32_t>(e0) | static_cast<uint32_t>(e1)) & 15u;
+      if (((m_step >> (s * RS)) & kSlotMask) == 0) continue;          // uniform over the slot
+      // visible columns of the two 64-column halves: c < lim0, 64 + c < 64 + lim1
+      const int key0 = (e0 >> 4) * BS, key1 = (BS == 128) ? key0 + 64 : (e1 >> 4) * BS;
+      const int lim0 = ((e0 >> member) & 1) ? min(max(qi - key0 + 1, 0), 64) : 0;
+      const int lim1 = ((e1 >> member) & 1) ? min(max(qi - key1 + 1, 0), 64) : 0;
 
-    // ---- softmax on this thread's row -----------------------------------------------
-    uint32_t sreg[BS];
-#pragma unroll
-    for (int c = 0; c < BS / 32; ++c) tmem_ld32(lane_addr + kColS + c * 32, sreg + c * 32);
-    tmem_ld_wait();
-    const bool need_mask = ((entry & 3) != ((1 << R) - 1)) || (kb * BS + BS - 1 > row0);
-    float mx = -INFINITY;
-    if (need_mask) {
-      const bool row_on = (entry >> member) & 1;
-      const int jmax = row_on ? (qi - kb * BS) : -1;   // columns c <= jmax are visible
-#pragma unroll
-      for (int c = 0; c < BS; ++c) {
-        float s = __uint_as_float(sreg[c]) * a.scale_log2;
-        s = (c <= jmax) ? s : -INFINITY;
-        sreg[c] = __float_as_uint(s);
-        mx = fmaxf(mx, s);
-      }
-    } else {
-#pragma unroll
-      for (int c = 0; c < BS; ++c) {
-        const float s = __uint_as_float(sreg[c]) * a.scale_log2;
-        sreg[c] = __float_as_uint(s);
-        mx = fmaxf(mx, s);
-      }
-    }
-    const float m_new = fmaxf(m_run, mx);
-    const float m_use = (m_new == -INFINITY) ? 0.f : m_new;
-    const float alpha = fast_exp2(m_run - m_use);     // m_run = -inf -> 0
-    float rs = 0.f;
-    uint32_t preg[BS / 2];
-#pragma unroll
-    for (int c = 0; c < BS; c += 2) {
-      const float p0 = fast_exp2(__uint_as_float(sreg[c]) - m_use);
-      const float p1 = fast_exp2(__uint_as_float(sreg[c + 1]) - m_use);
-      rs += p0 + p1;
-      preg[c >> 1] = pack_bf16(p0, p1);
-    }
-    l_run = l_run * alpha + rs;
-    m_run = m_new;
-#pragma unroll
-    for (int c = 0; c < BS / 64; ++c) tmem_st32(lane_addr + kColP + c * 32, preg + c * 32);
-
-    // ---- rescale the running O (needs the previous P V product to have landed) --------
-    if (e > 0) {
-      fail |= !mbar_wait(bar_o, (e - 1) & 1, a.error_word, 4);
+      ok = mbar_wait_warp(bars + B_SF + s, cnt & 1, a.error_word, 12);
+      if (!ok) break;
       tc_fence_after();
-      if (tid == 0 && !fail && e + 1 < n_ent) issue_kv(e + 1);   // stage (e+1)&1 was freed by P V of e-1
-      if (__any_sync(0xffffffffu, alpha != 1.f)) {
-#pragma unroll
-        for (int c = 0; c < D / 32; ++c) {
-          uint32_t oreg[32];
-          tmem_ld32(lane_addr + kColO + c * 32, oreg);
-          tmem_ld_wait();
-#pragma unroll
-          for (int x = 0; x < 32; ++x) oreg[x] = __float_as_uint(__uint_as_float(oreg[x]) * alpha);
-          tmem_st32(lane_addr + kColO + c * 32, oreg);
-        }
-      }
-    }
-    tmem_st_wait();
-    tc_fence_before();
-    if (fail) *s_fail = 1;
-    __syncthreads();
-    const bool cta_fail = *s_fail != 0;   // uniform: every thread leaves the loop together
-    if (tid == 0) {
-      tc_fence_after();
-      if (!cta_fail) {
-        const uint32_t v_base = smem_u32(sV + st * SM::kKVBytes);
-#pragma unroll
-        for (int k = 0; k < BS / 16; ++k) {
-          const uint64_t db = make_smem_desc(v_base + k * 2048, BS * 128, 1024);
-          mma_ts(tmem + kColO, tmem + kColP + k * 8, db, idesc_o, (e > 0) || (k > 0));
-        }
-      }
-      mma_commit(bar_o);
-    }
-    if (cta_fail) { fail = true; break; }
-  }
-
-  // ---- epilogue: O / l -> bf16, LSE ------------------------------------------------------
-  if (n_ent > 0) {
-    fail |= !mbar_wait(bar_o, (n_ent - 1) & 1, a.error_word, 5);
-    tc_fence_after();
-  }
-  if (qi < a.L) {   // warp-uniform: L is a multiple of 64
-    const float inv_l = l_run > 0.f ? 1.f / l_run : 0.f;
-    __nv_bfloat16* orow = a.o + b * a.o_strides[0] + h * a.o_strides[1] + static_cast<int64_t>(qi) * a.o_strides[2];
-#pragma unroll
-    for (int c = 0; c < D / 32; ++c) {
-      uint32_t oreg[32];
-      tmem_ld32(lane_addr + kColO + c * 32, oreg);
+      uint32_t sreg[128];
+      tmem_ld32(my_s, sreg);
+      tmem_ld32(my_s + 32, sreg + 32);
+      tmem_ld32(my_s + 64, sreg + 64);
+      tmem_ld32(my_s + 96, sreg + 96);
       tmem_ld_wait();
+      float mx = -INFINITY;
+      if (__any_sync(0xffffffffu, (lim0 < 64) || (lim1 < 64))) {
 #pragma unroll
-      for (int x = 0; x < 32; x += 8) {
-        uint4 v4;
-        v4.x = pack_bf16(__uint_as_float(oreg[x + 0]) * inv_l, __uint_as_float(oreg[x + 1]) * inv_l);
-        v4.y = pack_bf16(__uint_as_float(oreg[x + 2]) * inv_l, __uint_as_float(oreg[x + 3]) * inv_l);
-        v4.z = pack_bf16(__uint_as_float(oreg[x + 4]) * inv_l, __uint_as_float(oreg[x + 5]) * inv_l);
-        v4.w = pack_bf16(__uint_as_float(oreg[x + 6]) * inv_l, __uint_as_float(oreg[x + 7]) * inv_l);
-        if (!fail) *reinterpret_cast<uint4*>(orow + c * 32 + x) = v4;
+        for (int c = 0; c < 64; ++c) {
+          const float v0 = (c < lim0) ? __uint_as_float(sreg[c]) : -INFINITY;
+          const float v1 = (c < lim1) ? __uint_as_float(sreg[64 + c]) : -INFINITY;
+          sreg[c] = __float_as_uint(v0);
+          sreg[64 + c] = __float_as_uint(v1);
+          mx = fmaxf(mx, fmaxf(v0, v1));
+        }
+      } else {
+#pragma unroll
+        for (int c = 0; c < 128; c += 2) mx = fmaxf(mx, fmaxf(__uint_as_float(sreg[c]), __uint_as_float(sreg[c + 1])));
       }
+      const float m_new = fmaxf(m_ref, mx * a.scale_log2);
+      // raise the reference only when it would grow by more than the threshold (or is still unset)
+      const bool raise = (m_new > m_ref + kFwdRescaleThreshold) || (m_ref == -INFINITY && m_new > -INFINITY);
+      if (__any_sync(0xffffffffu, raise)) {
+        const float alpha = raise ? fast_exp2(m_ref - m_new) : 1.f;   // m_ref = -inf -> 0
+        if (raise) { m_ref = m_new; l_run *= alpha; }
+        if (cnt > 0) {   // O already holds products: wait for the latest one, then rescale my row
+          ok = mbar_wait_warp(bars + B_OD + s, (cnt - 1) & 1, a.error_word, 13);
+          if (!ok) break;
+          tc_fence_after();
+#pragma unroll
+          for (int c = 0; c < D / 16; ++c) {
+            uint32_t oreg[16];
+            tmem_ld16(my_o + c * 16, oreg);
+            tmem_ld_wait();
+#pragma unroll
+            for (int x = 0; x < 16; ++x) oreg[x] = __float_as_uint(__uint_as_float(oreg[x]) * alpha);
+            tmem_st16(my_o + c * 16, oreg);
+          }
+        }
+      }
+      const float neg_m = (m_ref == -INFINITY) ? 0.f : -m_ref;
+      float rs0 = 0.f, rs1 = 0.f;
+#pragma unroll
+      for (int c = 0; c < 128; c += 32) {
+        uint32_t preg[16];
+#pragma unroll
+        for (int x = 0; x < 32; x += 2) {
+          const float p0 = fast_exp2(fmaf(__uint_as_float(sreg[c + x]), a.scale_log2, neg_m));      // -inf -> 0
+          const float p1 = fast_exp2(fmaf(__uint_as_float(sreg[c + x + 1]), a.scale_log2, neg_m));
+          rs0 += p0;
+          rs1 += p1;
+          preg[x >> 1] = pack_bf16(p0, p1);
+        }
+        tmem_st16(my_s + (c >> 1), preg);   // P over the S columns already in registers
+      }
+      l_run += rs0 + rs1;
+      tmem_st_wait();
+      tc_fence_before();
+      __syncwarp();
+      if (lane == 0) mbar_arrive(bars + B_PF + s);
+      ++cnt;
     }
-    if (!fail)
+    // ---- epilogue: O / l -> bf16, LSE ------------------------------------------------------
+    if (ok && cnt > 0) ok = mbar_wait_warp(bars + B_OD + s, (cnt - 1) & 1, a.error_word, 14);
+    if (ok && cnt > 0 && qi < a.L) {   // warp-uniform: L is a multiple of 64
+      tc_fence_after();
+      const float inv_l = l_run > 0.f ? 1.f / l_run : 0.f;
+      __nv_bfloat16* orow = a.o + b * a.o_strides[0] + h * a.o_strides[1] + static_cast<int64_t>(qi) * a.o_strides[2];
+#pragma unroll
+      for (int c = 0; c < D / 32; ++c) {
+        uint32_t oreg[32];
+        tmem_ld32(my_o + c * 32, oreg);
+        tmem_ld_wait();
+#pragma unroll
+        for (int x = 0; x < 32; x += 8) {
+          uint4 v4;
+          v4.x = pack_bf16(__uint_as_float(oreg[x + 0]) * inv_l, __uint_as_float(oreg[x + 1]) * inv_l);
+          v4.y = pack_bf16(__uint_as_float(oreg[x + 2]) * inv_l, __uint_as_float(oreg[x + 3]) * inv_l);
+          v4.z = pack_bf16(__uint_as_float(oreg[x + 4]) * inv_l, __uint_as_float(oreg[x + 5]) * inv_l);
+          v4.w = pack_bf16(__uint_as_float(oreg[x + 6]) * inv_l, __uint_as_float(oreg[x + 7]) * inv_l);
+          *reinterpret_cast<uint4*>(orow + c * 32 + x) = v4;
+        }
+      }
       a.lse[(static_cast<int64_t>(b) * a.Hq + h) * a.L + qi] =
-          l_run > 0.f ? (m_run + log2f(l_run)) * 0.6931471805599453f : -INFINITY;
+          l_run > 0.f ? (m_ref + log2f(l_run)) * 0.6931471805599453f : -INFINITY;
+    }
   }
   tc_fence_before();
   __syncthreads();
-  if (warp == 0) tmem_dealloc(tmem, kTmemCols);
+  if (warp == 9) tmem_dealloc(tmem, 512);
 }
 
 }  // namespace lg

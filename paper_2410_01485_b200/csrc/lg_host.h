@@ -19,6 +19,7 @@ struct Resolved {          // validated, defaulted copy of lg_attn_params
   float scale;
   int64_t qs[3], ks[3], vs[3], os[3];
   int n_qtiles, n_ktiles;  // ceil(L / 128)
+  int n_stiles;            // ceil(L / 256): super-tiles of the forward
   int64_t nnz;
 };
 
@@ -27,7 +28,8 @@ lg_status resolve(const lg_attn_params* p, Resolved* r);
 // Layout of the attention workspace (all offsets 256-byte aligned).
 struct WsLayout {
   size_t row_ptr, col_idx, col_ptr, row_idx;     // the CSR / CSC lists
-  size_t qt_cnt, qt_ent, qt_order;               // query-tile schedules (fwd, dQ pass)
+  size_t qt_cnt, qt_ent, qt_order;               // query-tile schedules (dQ pass)
+  size_t sq_cnt, sq_ent, sq_order;               // super-tile schedules (forward)
   size_t kt_cnt, kt_ent, kt_order;               // kv-tile schedules (dK/dV pass)
   size_t delta;                                  // float2 [B, Hq, L]: (LSE * log2 e, delta) (bwd only)
   size_t total;

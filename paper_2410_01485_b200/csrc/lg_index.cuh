@@ -110,6 +110,34 @@ __global__ void tile_merge_kernel(const int32_t* __restrict__ ptr, const int32_t
   tile_cnt[t] = n;
 }
 
+// The same for tiles of up to four pattern rows (the forward's super-tiles of 256 query rows):
+// entry = idx * 16 + member mask.
+__global__ void tile_merge4_kernel(const int32_t* __restrict__ ptr, const int32_t* __restrict__ idx, int nB, int R,
+                                   int n_tiles, int32_t* __restrict__ tile_cnt, int32_t* __restrict__ tile_ent) {
+  const int t = blockIdx.x * blockDim.x + threadIdx.x;
+  if (t >= n_tiles) return;
+  const int r0 = t * R;
+  int32_t* out = tile_ent + ptr[r0];
+  int cur[4], end[4];
+  for (int r = 0; r < 4; ++r) {
+    const bool have = r < R && r0 + r < nB;
+    cur[r] = have ? ptr[r0 + r] : 0;
+    end[r] = have ? ptr[r0 + r + 1] : 0;
+  }
+  int n = 0;
+  for (;;) {
+    int lo = 0x7fffffff;
+    for (int r = 0; r < 4; ++r)
+      if (cur[r] < end[r]) lo = min(lo, idx[cur[r]]);
+    if (lo == 0x7fffffff) break;
+    int mask = 0;
+    for (int r = 0; r < 4; ++r)
+      if (cur[r] < end[r] && idx[cur[r]] == lo) { mask |= 1 << r; ++cur[r]; }
+    out[n++] = lo * 16 + mask;
+  }
+  tile_cnt[t] = n;
+}
+
 // Launch order: tiles with more work first.  order[rank] = tile; rank by (count desc, tile asc).
 __global__ void tile_order_kernel(const int32_t* __restrict__ tile_cnt, int n_tiles, int32_t* __restrict__ order) {
   const int t = blockIdx.x * blockDim.x + threadIdx.x;
