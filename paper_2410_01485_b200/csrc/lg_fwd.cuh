@@ -35,6 +35,10 @@ struct FwdArgs {
 
 constexpr int kFwdThreads = 320;
 constexpr float kFwdRescaleThreshold = 8.0f;   // log2 units
+#ifndef LG_FWD_POLY_PER8
+#define LG_FWD_POLY_PER8 2
+#endif
+constexpr int kFwdPolyPer8 = LG_FWD_POLY_PER8;     // exponentials of every 8 evaluated by polynomial
 
 template <int D>
 struct FwdSmem {
@@ -260,7 +264,8 @@ fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUt
       tmem_ld32(my_s + 96, sreg + 96);
       tmem_ld_wait();
       float mx = -INFINITY;
-      if (__any_sync(0xffffffffu, (lim0 < 64) || (lim1 < 64))) {
+      const bool masked = __any_sync(0xffffffffu, (lim0 < 64) || (lim1 < 64));
+      if (masked) {
 #pragma unroll
         for (int c = 0; c < 64; ++c) {
           const float v0 = (c < lim0) ? __uint_as_float(sreg[c]) : -INFINITY;
@@ -270,8 +275,17 @@ fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUt
           mx = fmaxf(mx, fmaxf(v0, v1));
         }
       } else {
+        {   // four independent chains: a single chain of 64 dependent maxima is pure latency
+          float m0 = -INFINITY, m1 = -INFINITY, m2 = -INFINITY, m3 = -INFINITY;
 #pragma unroll
-        for (int c = 0; c < 128; c += 2) mx = fmaxf(mx, fmaxf(__uint_as_float(sreg[c]), __uint_as_float(sreg[c + 1])));
+          for (int c = 0; c < 128; c += 8) {
+            m0 = max3(m0, __uint_as_float(sreg[c + 0]), __uint_as_float(sreg[c + 1]));
+            m1 = max3(m1, __uint_as_float(sreg[c + 2]), __uint_as_float(sreg[c + 3]));
+            m2 = max3(m2, __uint_as_float(sreg[c + 4]), __uint_as_float(sreg[c + 5]));
+            m3 = max3(m3, __uint_as_float(sreg[c + 6]), __uint_as_float(sreg[c + 7]));
+          }
+          mx = fmaxf(fmaxf(m0, m1), fmaxf(m2, m3));
+        }
       }
       const float m_new = fmaxf(m_ref, mx * a.scale_log2);
       // raise the reference only when it would grow by more than the threshold (or is still unset)
@@ -296,18 +310,40 @@ fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUt
       }
       const float neg_m = (m_ref == -INFINITY) ? 0.f : -m_ref;
       float rs0 = 0.f, rs1 = 0.f;
+      if (masked) {   // steps with hidden keys: every exponential on the exact path (-inf -> 0)
 #pragma unroll
-      for (int c = 0; c < 128; c += 32) {
-        uint32_t preg[16];
+        for (int c = 0; c < 128; c += 32) {
+          uint32_t preg[16];
 #pragma unroll
-        for (int x = 0; x < 32; x += 2) {
-          const float p0 = fast_exp2(fmaf(__uint_as_float(sreg[c + x]), a.scale_log2, neg_m));      // -inf -> 0
-          const float p1 = fast_exp2(fmaf(__uint_as_float(sreg[c + x + 1]), a.scale_log2, neg_m));
-          rs0 += p0;
-          rs1 += p1;
-          preg[x >> 1] = pack_bf16(p0, p1);
+          for (int x = 0; x < 32; x += 2) {
+            const float p0 = fast_exp2(fmaf(__uint_as_float(sreg[c + x]), a.scale_log2, neg_m));
+            const float p1 = fast_exp2(fmaf(__uint_as_float(sreg[c + x + 1]), a.scale_log2, neg_m));
+            rs0 += p0;
+            rs1 += p1;
+            preg[x >> 1] = pack_bf16(p0, p1);
+          }
+          tmem_st16(my_s + (c >> 1), preg);   // P over the S columns already in registers
         }
-        tmem_st16(my_s + (c >> 1), preg);   // P over the S columns already in registers
+      } else {        // kFwdPolyPer8 of every 8 exponentials go to the FMA pipe
+        const uint64_t sc2 = f32x2(a.scale_log2, a.scale_log2), nm2 = f32x2(neg_m, neg_m);
+        uint64_t rsum[4] = {f32x2(0.f, 0.f), f32x2(0.f, 0.f), f32x2(0.f, 0.f), f32x2(0.f, 0.f)};   // independent chains
+#pragma unroll
+        for (int c = 0; c < 128; c += 32) {
+          uint32_t preg[16];
+#pragma unroll
+          for (int x = 0; x < 32; x += 2) {
+            uint64_t& rs2 = rsum[(x >> 1) & 3];
+            float x0, x1;
+            f32x2_split(fma_f32x2(f32x2(__uint_as_float(sreg[c + x]), __uint_as_float(sreg[c + x + 1])), sc2, nm2),
+                        x0, x1);
+            const float p0 = ((x & 7) < kFwdPolyPer8) ? poly_exp2(x0) : fast_exp2(x0);
+            const float p1 = (((x + 1) & 7) < kFwdPolyPer8) ? poly_exp2(x1) : fast_exp2(x1);
+            rs2 = add_f32x2(rs2, f32x2(p0, p1));
+            preg[x >> 1] = pack_bf16(p0, p1);
+          }
+          tmem_st16(my_s + (c >> 1), preg);
+        }
+        f32x2_split(add_f32x2(add_f32x2(rsum[0], rsum[1]), add_f32x2(rsum[2], rsum[3])), rs0, rs1);
       }
       l_run += rs0 + rs1;
       tmem_st_wait();
