@@ -34,6 +34,8 @@ struct DecodeArgs {
   float* lse;                    // [B, Hq] or null
   int Hq, Hkv, G, HG, C, nsplit;
   float scale_log2;
+  int B;                         // sequences (flattened path)
+  unsigned int* unit_count;      // [B * Hkv * HG] records delivered per unit (flattened path; zero between calls)
 };
 
 __device__ __forceinline__ void cp_async16(uint32_t smem_addr, const void* gptr, bool valid) {
@@ -69,26 +71,18 @@ __device__ __forceinline__ void mma16816(float* c, uint32_t a0, uint32_t a1, uin
       : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1));
 }
 
+// One segment of one (sequence, kv head, head group): warp w of the CTA streams tiles
+// [t_begin, t_end) of the cache, the four warps' partials are merged in warp order and the
+// CTA's (max, sum, O) record for its 8 heads is written to `out`.
 template <int D>
-__global__ void __launch_bounds__(kDecWarps * 32) decode_split_kernel(const DecodeArgs a) {
+__device__ __forceinline__ void decode_run_segment(const DecodeArgs& a, uint8_t* dsmem, int b, int kvh, int hg,
+                                                   int nvalid, int t_begin, int t_end, float* out) {
   constexpr int kRowBytes = D * 2;
   constexpr int kChunks = D / 8;                      // 16-byte chunks per row
   constexpr int kTileBytes = kDecTile * kRowBytes;    // K (or V) bytes of one tile
   constexpr int kCopiesPerLane = kDecTile * kChunks / 32;
-  extern __shared__ __align__(128) uint8_t dsmem[];
-
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-  const int split = blockIdx.x, kg = blockIdx.y, b = blockIdx.z;
-  const int kvh = kg / a.HG, hg = kg % a.HG;
   const int r = lane >> 2, c = lane & 3;
-
-  const int64_t n = a.n_tokens[b];
-  const int nvalid = static_cast<int>(n < a.C ? (n < 0 ? 0 : n) : a.C);
-  const int ntile = (nvalid + kDecTile - 1) / kDecTile;
-  const int wg = split * kDecWarps + warp, nw = a.nsplit * kDecWarps;
-  const int t_begin = static_cast<int>(static_cast<int64_t>(ntile) * wg / nw);
-  const int t_end = static_cast<int>(static_cast<int64_t>(ntile) * (wg + 1) / nw);
-
   uint8_t* wsm = dsmem + warp * (kDecStages * 2 * kTileBytes);
   const uint32_t wsm_u32 = smem_u32(wsm);
   const uint8_t* kbase = reinterpret_cast<const uint8_t*>(a.k_cache) +
@@ -228,7 +222,6 @@ __global__ void __launch_bounds__(kDecWarps * 32) decode_split_kernel(const Deco
     }
   }
   __syncthreads();
-  float* out = a.part + ((static_cast<int64_t>(b) * gridDim.y + kg) * a.nsplit + split) * (kDecHeads * kRec);
   for (int idx = threadIdx.x; idx < kDecHeads * D; idx += blockDim.x) {
     const int head = idx / D, d = idx % D;
     float m = -INFINITY;
@@ -244,6 +237,194 @@ __global__ void __launch_bounds__(kDecWarps * 32) decode_split_kernel(const Deco
     }
     out[head * kRec + d] = acc;
     if (d == 0) { out[head * kRec + D] = m; out[head * kRec + D + 1] = l; }
+  }
+}
+
+template <int D>
+__global__ void __launch_bounds__(kDecWarps * 32) decode_split_kernel(const DecodeArgs a) {
+  extern __shared__ __align__(128) uint8_t dsmem[];
+  const int warp = threadIdx.x >> 5;
+  const int split = blockIdx.x, kg = blockIdx.y, b = blockIdx.z;
+  const int kvh = kg / a.HG, hg = kg % a.HG;
+  const int64_t n = a.n_tokens[b];
+  const int nvalid = static_cast<int>(n < a.C ? (n < 0 ? 0 : n) : a.C);
+  const int ntile = (nvalid + kDecTile - 1) / kDecTile;
+  const int wg = split * kDecWarps + warp, nw = a.nsplit * kDecWarps;
+  const int t_begin = static_cast<int>(static_cast<int64_t>(ntile) * wg / nw);
+  const int t_end = static_cast<int>(static_cast<int64_t>(ntile) * (wg + 1) / nw);
+  constexpr int kRec = D + 2;
+  float* out = a.part + ((static_cast<int64_t>(b) * gridDim.y + kg) * a.nsplit + split) * (kDecHeads * kRec);
+  decode_run_segment<D>(a, dsmem, b, kvh, hg, nvalid, t_begin, t_end, out);
+}
+
+// ---- flattened schedule ---------------------------------------------------------------------
+// The tiles of all (sequence, kv head, head group) units form one sequence, unit after unit
+// (sequence-major); CTA c of N streams the slice [T c / N, T (c + 1) / N) of it, so every CTA
+// moves the same number of bytes whatever the mix of sequence lengths, and one wave of CTAs
+// covers the whole cache.  A slice that crosses a unit boundary is processed in segments; the
+// record of (CTA c, unit u) lives at index c + u, which grows strictly along the sequence.
+constexpr int kDecFlatMaxB = 2048;      // sequences the flattened path supports (prefix array in shared memory)
+constexpr int kDecFlatMaxCtas = 320;    // upper bound of its grid (two CTAs per SM)
+
+__device__ __forceinline__ int decode_tiles_of(const DecodeArgs& a, int b) {
+  const int64_t n = a.n_tokens[b];
+  const int nvalid = static_cast<int>(n < a.C ? (n < 0 ? 0 : n) : a.C);
+  return (nvalid + kDecTile - 1) / kDecTile;
+}
+
+// cum[b] = tiles of the sequences before b, b = 0 .. B (block of 128 threads; ends with a barrier)
+__device__ __forceinline__ void decode_build_cum(const DecodeArgs& a, int* cum) {
+  __shared__ int warp_sum[4];
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  const int ipt = (a.B + 127) / 128;
+  const int b0 = tid * ipt;
+  int local = 0;
+  for (int i = 0; i < ipt; ++i)
+    if (b0 + i < a.B) local += decode_tiles_of(a, b0 + i);
+  int incl = local;
+  for (int o = 1; o < 32; o <<= 1) {
+    const int t = __shfl_up_sync(0xffffffffu, incl, o);
+    if (lane >= o) incl += t;
+  }
+  if (lane == 31) warp_sum[warp] = incl;
+  __syncthreads();
+  int run = incl - local;
+  for (int w = 0; w < warp; ++w) run += warp_sum[w];
+  for (int i = 0; i < ipt; ++i)
+    if (b0 + i < a.B) { cum[b0 + i] = run; run += decode_tiles_of(a, b0 + i); }
+  if (tid == 127) cum[a.B] = warp_sum[0] + warp_sum[1] + warp_sum[2] + warp_sum[3];
+  __syncthreads();
+}
+
+// Merge the records of unit (b, k): CTAs first_cta .. first_cta + n_rec - 1, in that order
+// (whichever CTA happens to run this, the summation order is the same).  128 threads.
+template <int D>
+__device__ __forceinline__ void decode_merge_unit(const DecodeArgs& a, int b, int k, int64_t u, int first_cta,
+                                                  int n_rec, int64_t total, int n_cta) {
+  constexpr int kRec = D + 2;
+  const int kvh = k / a.HG, hg = k % a.HG;
+  const float* recs = a.part + (static_cast<int64_t>(first_cta) + u) * (kDecHeads * kRec);
+  // a CTA with an empty slice (possible only with fewer tiles than CTAs) wrote no record
+  const bool sparse_slices = total < n_cta;
+  auto empty_slice = [&](int c) { return total * c / n_cta == total * (c + 1) / n_cta; };
+  // Each thread owns kOut outputs (all handled together so that the loads of one record are in
+  // flight at once: the records sit in L2 and a dependent chain of loads would dominate).
+  constexpr int kOut = kDecHeads * D / 128;
+  int head[kOut], dd[kOut];
+  float m[kOut], acc[kOut], l[kOut];
+#pragma unroll
+  for (int j = 0; j < kOut; ++j) {
+    const int idx = threadIdx.x + j * 128;
+    head[j] = idx / D;
+    dd[j] = idx % D;
+    m[j] = -INFINITY;
+    acc[j] = 0.f;
+    l[j] = 0.f;
+  }
+  for (int i = 0; i < n_rec; ++i) {
+    if (sparse_slices && empty_slice(first_cta + i)) continue;
+#pragma unroll
+    for (int j = 0; j < kOut; ++j) m[j] = fmaxf(m[j], __ldcg(recs + (i * kDecHeads + head[j]) * kRec + D));
+  }
+  for (int i = 0; i < n_rec; ++i) {
+    if (sparse_slices && empty_slice(first_cta + i)) continue;
+    float rm[kOut], rl[kOut], ro[kOut];
+#pragma unroll
+    for (int j = 0; j < kOut; ++j) {
+      const float* rec = recs + (i * kDecHeads + head[j]) * kRec;
+      rm[j] = __ldcg(rec + D);
+      rl[j] = __ldcg(rec + D + 1);
+      ro[j] = __ldcg(rec + dd[j]);
+    }
+#pragma unroll
+    for (int j = 0; j < kOut; ++j) {
+      const float f = fast_exp2(rm[j] - (m[j] == -INFINITY ? 0.f : m[j]));
+      acc[j] += f * ro[j];
+      l[j] += f * rl[j];
+    }
+  }
+#pragma unroll
+  for (int j = 0; j < kOut; ++j) {
+    const int gh = hg * kDecHeads + head[j];
+    if (gh >= a.G) continue;
+    const int64_t qh = static_cast<int64_t>(b) * a.Hq + kvh * a.G + gh;
+    a.o[qh * D + dd[j]] = __float2bfloat16(l[j] > 0.f ? acc[j] / l[j] : 0.f);
+    if (dd[j] == 0 && a.lse) a.lse[qh] = l[j] > 0.f ? (m[j] + log2f(l[j])) * 0.6931471805599453f : -INFINITY;
+  }
+}
+
+template <int D>
+__global__ void __launch_bounds__(kDecWarps * 32) decode_stream_kernel(const DecodeArgs a) {
+  extern __shared__ __align__(128) uint8_t dsmem[];
+  constexpr int kPipeBytes = kDecWarps * kDecStages * 2 * kDecTile * D * 2;
+  constexpr int kRec = D + 2;
+  int* cum = reinterpret_cast<int*>(dsmem + kPipeBytes);
+  decode_build_cum(a, cum);
+  const int ups = a.Hkv * a.HG;
+  const int64_t total = static_cast<int64_t>(cum[a.B]) * ups;
+  __shared__ int s_merge[3];
+  auto start_of = [&](int64_t c) { return total * c / gridDim.x; };
+  auto cta_of = [&](int64_t f) {           // the CTA whose slice holds tile f
+    int64_t c = f * gridDim.x / total;
+    while (c + 1 < gridDim.x && start_of(c + 1) <= f) ++c;
+    while (c > 0 && start_of(c) > f) --c;
+    return static_cast<int>(c);
+  };
+  // units of sequences without tokens get their (empty) result here, spread over the CTAs
+  for (int e = 0; e < a.B; ++e) {
+    if (cum[e + 1] != cum[e]) continue;
+    for (int k = 0; k < ups; ++k) {
+      const int64_t u = static_cast<int64_t>(e) * ups + k;
+      if (u % gridDim.x == blockIdx.x) decode_merge_unit<D>(a, e, k, u, 0, 0, total, gridDim.x);
+    }
+  }
+  const int64_t f0 = start_of(blockIdx.x), f1 = start_of(blockIdx.x + 1);
+  if (f0 >= f1) return;
+  int lo = 0, hi = a.B;   // cum[lo] * ups <= f0 < cum[hi] * ups
+  while (hi - lo > 1) {
+    const int mid = (lo + hi) >> 1;
+    if (static_cast<int64_t>(cum[mid]) * ups <= f0) lo = mid; else hi = mid;
+  }
+  int b = lo;
+  const int warp = threadIdx.x >> 5;
+  int64_t pos = f0;
+  while (pos < f1) {
+    while (static_cast<int64_t>(cum[b + 1]) * ups <= pos) ++b;          // skip finished / empty sequences
+    const int nt = cum[b + 1] - cum[b];
+    const int64_t rel = pos - static_cast<int64_t>(cum[b]) * ups;
+    const int k = static_cast<int>(rel / nt), t0 = static_cast<int>(rel - static_cast<int64_t>(k) * nt);
+    const int n = static_cast<int>(min(static_cast<int64_t>(nt - t0), f1 - pos));
+    const int64_t nn = a.n_tokens[b];
+    const int nvalid = static_cast<int>(nn < a.C ? (nn < 0 ? 0 : nn) : a.C);
+    const int tb = t0 + static_cast<int>(static_cast<int64_t>(n) * warp / kDecWarps);
+    const int te = t0 + static_cast<int>(static_cast<int64_t>(n) * (warp + 1) / kDecWarps);
+    const int64_t u = static_cast<int64_t>(b) * ups + k;
+    __syncthreads();   // the previous segment's merge is done with shared memory
+    decode_run_segment<D>(a, dsmem, b, k / a.HG, k % a.HG, nvalid, tb, te,
+                          a.part + (blockIdx.x + u) * (kDecHeads * kRec));
+    // The CTA that delivers the last record of a unit merges it (records are read in index
+    // order, so the result does not depend on which CTA that is) and re-arms the counter.
+    __threadfence();
+    __syncthreads();
+    if (threadIdx.x == 0) {
+      const int64_t first = static_cast<int64_t>(cum[b]) * ups + static_cast<int64_t>(k) * nt;
+      const int c_lo = (t0 == 0) ? static_cast<int>(blockIdx.x) : cta_of(first);
+      const int c_hi = (t0 + n == nt) ? static_cast<int>(blockIdx.x) : cta_of(first + nt - 1);
+      int pieces = c_hi - c_lo + 1;
+      if (total < gridDim.x)
+        for (int c = c_lo; c <= c_hi; ++c) pieces -= (start_of(c) == start_of(c + 1)) ? 1 : 0;
+      const unsigned ticket = atomicAdd(a.unit_count + u, 1u);
+      s_merge[0] = (ticket + 1u == static_cast<unsigned>(pieces)) ? 1 : 0;
+      s_merge[1] = c_lo;
+      s_merge[2] = c_hi - c_lo + 1;
+    }
+    __syncthreads();
+    if (s_merge[0]) {
+      __threadfence();
+      decode_merge_unit<D>(a, b, k, u, s_merge[1], s_merge[2], total, gridDim.x);
+      if (threadIdx.x == 0) a.unit_count[u] = 0u;
+    }
+    pos += n;
   }
 }
 
@@ -328,6 +509,9 @@ static int choose_nsplit(const lg_decode_params* p) {
   return static_cast<int>(ns);
 }
 
+// Batches of up to kDecFlatMaxB sequences take the flattened one-wave schedule.
+static bool decode_is_flat(const lg_decode_params* p) { return p->B <= kDecFlatMaxB; }
+
 static size_t decode_part_bytes(const lg_decode_params* p, int nsplit) {
   const int HG = (p->Hq / p->Hkv + kDecHeads - 1) / kDecHeads;
   return static_cast<size_t>(p->B) * p->Hkv * HG * nsplit * kDecHeads * (p->D + 2) * sizeof(float);
@@ -361,6 +545,13 @@ lg_status lg_kv_ring_append(const lg_decode_params* p, void* k_cache, void* v_ca
 
 size_t lg_sparse_decode_workspace_bytes(const lg_decode_params* p) {
   if (check_decode(p) != LG_OK) return 0;
+  if (decode_is_flat(p)) {   // one record per (CTA, unit) pair that can occur: index CTA + unit
+    const int HG = (p->Hq / p->Hkv + kDecHeads - 1) / kDecHeads;
+    const size_t units = static_cast<size_t>(p->B) * p->Hkv * HG;
+    const size_t records = static_cast<size_t>(kDecFlatMaxCtas) + units;
+    return sizeof(WsHeader) + align_up(units * sizeof(unsigned int), 256) +
+           align_up(records * kDecHeads * (p->D + 2) * sizeof(float), 256);
+  }
   return sizeof(WsHeader) + align_up(decode_part_bytes(p, choose_nsplit(p)), 256);
 }
 
@@ -391,6 +582,39 @@ lg_status lg_sparse_decode(const lg_decode_params* p, const void* q, const void*
   a.nsplit = choose_nsplit(p);
   const float scale = p->scale > 0.f ? p->scale : 1.0f / sqrtf(static_cast<float>(p->D));
   a.scale_log2 = scale * 1.4426950408889634f;
+  a.B = p->B;
+  if (decode_is_flat(p)) {
+    int dev = 0, sms = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess ||
+        cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess)
+      return LG_ERR_CUDA;
+    // two CTAs per SM, fewer when the cache is too small to give each warp a couple of tiles
+    const int64_t units = static_cast<int64_t>(p->B) * a.Hkv * a.HG;
+    const int64_t max_tiles = units * ((a.C + kDecTile - 1) / kDecTile);
+    int64_t n_cta = (max_tiles + 2 * kDecWarps - 1) / (2 * kDecWarps);
+    if (n_cta > 2 * sms) n_cta = 2 * sms;
+    if (n_cta > kDecFlatMaxCtas) n_cta = kDecFlatMaxCtas;
+    if (n_cta < 1) n_cta = 1;
+    if (units > 0x7fffffff) return LG_ERR_UNSUPPORTED;
+    // header word and per-unit counters start at zero; the records follow them
+    const size_t count_bytes = align_up(static_cast<size_t>(units) * sizeof(unsigned int), 256);
+    a.unit_count = reinterpret_cast<unsigned int*>(static_cast<uint8_t*>(workspace) + sizeof(WsHeader));
+    a.part = reinterpret_cast<float*>(static_cast<uint8_t*>(workspace) + sizeof(WsHeader) + count_bytes);
+    if (cudaMemsetAsync(workspace, 0, sizeof(WsHeader) + count_bytes, st) != cudaSuccess) return LG_ERR_CUDA;
+    const int smem_flat = kDecWarps * kDecStages * 2 * kDecTile * p->D * 2 + (p->B + 1) * static_cast<int>(sizeof(int));
+    if (p->D == 128) {
+      if (cudaFuncSetAttribute(decode_stream_kernel<128>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem_flat) !=
+          cudaSuccess)
+        return LG_ERR_CUDA;
+      decode_stream_kernel<128><<<static_cast<unsigned>(n_cta), kDecWarps * 32, smem_flat, st>>>(a);
+    } else {
+      if (cudaFuncSetAttribute(decode_stream_kernel<64>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem_flat) !=
+          cudaSuccess)
+        return LG_ERR_CUDA;
+      decode_stream_kernel<64><<<static_cast<unsigned>(n_cta), kDecWarps * 32, smem_flat, st>>>(a);
+    }
+    return cudaGetLastError() == cudaSuccess ? LG_OK : LG_ERR_CUDA;
+  }
   if (a.Hkv * a.HG > 65535 || p->B > 65535) return LG_ERR_UNSUPPORTED;
   if (cudaMemsetAsync(workspace, 0, sizeof(WsHeader), st) != cudaSuccess) return LG_ERR_CUDA;
   dim3 grid(a.nsplit, a.Hkv * a.HG, p->B);

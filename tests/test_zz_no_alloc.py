@@ -29,7 +29,7 @@ def lib():
 
 def test_static_decode_rejects_problems_beyond_the_fixed_array(lib):
     """Host-only: the size check comes before any CUDA call, so it runs without a GPU."""
-    big = lg.decode_params(64, 64, 8, 128, 128, 1 << 20)
+    big = lg.decode_params(1024, 64, 8, 128, 128, 1 << 20)
     assert lib.lg_sparse_decode_workspace_bytes(C.byref(big)) > lg.DECODE_STATIC_SCRATCH_BYTES
     rc = lib.lg_sparse_decode_static(C.byref(big), 16, 16, 16, 16, 16, None, None)
     assert rc == -3 and "workspace" in lg.status_string(rc)
