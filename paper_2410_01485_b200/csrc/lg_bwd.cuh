@@ -148,7 +148,7 @@ bwd_dq_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ 
   constexpr uint32_t kColS = 0, kColDP = 256, kColDQ = 384;
   constexpr int kTile = SM::kTile;
   enum { B_FIX = 0, B_KF = 1, B_KE = 4, B_VF = 7, B_VE = 9, B_SF = 11, B_DPF = 13, B_DSF = 14, B_DONE = 15,
-         B_DRAIN = 16, B_COUNT = 17 };
+         B_DRAIN = 16, B_DPR = 17, B_COUNT = 18 };
 
   extern __shared__ __align__(1024) uint8_t smem[];
   uint64_t* bars = reinterpret_cast<uint64_t*>(smem + SM::oBar);
@@ -176,6 +176,7 @@ bwd_dq_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ 
     for (int i = 0; i < 2; ++i) { mbar_init(bars + B_VF + i, 1); mbar_init(bars + B_VE + i, 1); mbar_init(bars + B_SF + i, 1); }
     mbar_init(bars + B_DPF, 1);
     mbar_init(bars + B_DSF, 8);
+    mbar_init(bars + B_DPR, 8);
     mbar_init(bars + B_DONE, 1);
     mbar_init(bars + B_DRAIN, 1);
     mbar_fence_init();
@@ -263,6 +264,12 @@ bwd_dq_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ 
         if (n_steps > 1) issue_s(1);
       }
       for (int j = 0; j < n_steps; ++j) {
+        // dP of the next step goes first: it only needs the dP columns to have been read, and it
+        // is what the element-wise warps wait for next; dQ of this step follows.
+        if (j + 1 < n_steps) {
+          ok = ok && mbar_wait(bars + B_DPR, j & 1, a.error_word, 34);
+          issue_dp(j + 1);
+        }
         ok = ok && mbar_wait(bars + B_DSF, j & 1, a.error_word, 29);
         if (ok) {
           tc_fence_after();
@@ -273,7 +280,6 @@ bwd_dq_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ 
                    make_smem_desc(kst + kk * 2048, BwdTile<D>::kBox, 1024), idesc_dq, (j > 0) || (kk > 0));
         }
         mma_commit(bars + B_KE + j % 3);
-        if (j + 1 < n_steps) issue_dp(j + 1);
         if (j + 2 < n_steps) issue_s(j + 2);
       }
       mma_commit(bars + B_DONE);
@@ -330,15 +336,18 @@ bwd_dq_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ 
       if (!ok) break;
       tc_fence_after();
       uint32_t dsreg[32];
-#pragma unroll
-      for (int c = 0; c < 2; ++c) {
-        uint32_t dreg[32];
-        tmem_ld32(lane_addr + kColDP + wg * 64 + c * 32, dreg);
+      {
+        uint32_t dreg[64];
+        tmem_ld32(lane_addr + kColDP + wg * 64, dreg);
+        tmem_ld32(lane_addr + kColDP + wg * 64 + 32, dreg + 32);
         tmem_ld_wait();
+        tc_fence_before();
+        __syncwarp();
+        if (lane == 0) mbar_arrive(bars + B_DPR);   // the dP columns may be overwritten
 #pragma unroll
-        for (int x = 0; x < 32; x += 2)
-          dsreg[c * 16 + (x >> 1)] = pack_bf16(p[c * 32 + x] * (__uint_as_float(dreg[x]) - dlt),
-                                               p[c * 32 + x + 1] * (__uint_as_float(dreg[x + 1]) - dlt));
+        for (int x = 0; x < 64; x += 2)
+          dsreg[x >> 1] = pack_bf16(p[x] * (__uint_as_float(dreg[x]) - dlt),
+                                    p[x + 1] * (__uint_as_float(dreg[x + 1]) - dlt));
       }
       tmem_st32(lane_addr + kColS + (j & 1) * 128 + wg * 64, dsreg);   // dS over my own S columns
       ew_publish(bars + B_DSF);
