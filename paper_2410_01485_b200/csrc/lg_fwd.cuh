@@ -35,10 +35,6 @@ struct FwdArgs {
 
 constexpr int kFwdThreads = 320;
 constexpr float kFwdRescaleThreshold = 8.0f;   // log2 units
-#ifndef LG_FWD_POLY_PER8
-#define LG_FWD_POLY_PER8 2
-#endif
-constexpr int kFwdPolyPer8 = LG_FWD_POLY_PER8;     // exponentials of every 8 evaluated by polynomial
 
 template <int D>
 struct FwdSmem {
@@ -165,7 +161,7 @@ fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUt
       const uint32_t v_mn_lo = desc_lo(smem_u32(sV), SM::kBox);
       bool ok = mbar_wait(bars + B_Q, 0, a.error_word, 7);
       int k_ready = -1, v_ready = -1;           // last step whose K / V tile this thread has seen complete
-      int n_pv[2] = {0, 0};                     // P V products issued per slot (accumulate flag, barrier phases)
+      int n_pv0 = 0, n_pv1 = 0;                 // P V products issued per slot (accumulate flag, barrier phases)
       auto issue_s = [&](int s, int j) {
         const int sk = j % 3;
         if (k_ready < j) {
@@ -190,34 +186,40 @@ fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUt
           ok = ok && mbar_wait(bars + B_VF + sv, (j / 2) & 1, a.error_word, 9);
           v_ready = j;
         }
-        ok = ok && mbar_wait(bars + B_PF + s, n_pv[s] & 1, a.error_word, 10);
+        const int n_pv = s ? n_pv1 : n_pv0;
+        ok = ok && mbar_wait(bars + B_PF + s, n_pv & 1, a.error_word, 10);
         if (ok) {
           tc_fence_after();
           const uint32_t b_lo = v_mn_lo + sv * (kTile >> 4);
 #pragma unroll
           for (int kk = 0; kk < 8; ++kk)
             mma_ts2(tmem + kColO + s * 128, tmem + kColS + s * 128 + kk * 8, b_lo + kk * (2048 >> 4), hi, idesc_o,
-                    (n_pv[s] > 0) || (kk > 0));
+                    (n_pv > 0) || (kk > 0));
         }
-        ++n_pv[s];
+        if (s) ++n_pv1; else ++n_pv0;
         mma_commit(bars + B_OD + s);
       };
-      uint32_t m_cur = step_mask(0), m_nxt = step_mask(1);
-      if (n_steps > 0) {
-        if (m_cur & kSlotMask) issue_s(0, 0);
-        if ((m_cur >> RS) & kSlotMask) issue_s(1, 0);
-        mma_commit(bars + B_KE + 0);
-      }
-      for (int j = 0; j < n_steps; ++j) {
-        const uint32_t m_nxt2 = step_mask(j + 2);   // read two steps ahead: off the critical path
-        const bool c0 = m_cur & kSlotMask, c1 = (m_cur >> RS) & kSlotMask;
-        const bool x0 = m_nxt & kSlotMask, x1 = (m_nxt >> RS) & kSlotMask;
-        if (c0) issue_pv(0, j);
-        if (c0 && !c1) mma_commit(bars + B_VE + (j & 1));
-        if (x0) issue_s(0, j + 1);
-        if (x0 && !x1) mma_commit(bars + B_KE + (j + 1) % 3);
-        if (c1) { issue_pv(1, j); mma_commit(bars + B_VE + (j & 1)); }
-        if (x1) { issue_s(1, j + 1); mma_commit(bars + B_KE + (j + 1) % 3); }
+      // One loop body issues everything (step -1 only issues the S products of step 0): the
+      // code of this thread must stay small, it competes for the instruction caches with the
+      // softmax warps and every fetch miss is time the tensor pipe sits idle.
+      uint32_t m_cur = 0u, m_nxt = step_mask(0);
+#pragma unroll 1
+      for (int j = -1; j < n_steps; ++j) {
+        const uint32_t m_nxt2 = step_mask(j + 2);   // read ahead: off the critical path
+#pragma unroll 1
+        for (int s = 0; s < 2; ++s) {
+          const bool cur = (m_cur >> (s * RS)) & kSlotMask, nxt = (m_nxt >> (s * RS)) & kSlotMask;
+          const bool cur_other_later = (s == 0) && ((m_cur >> RS) & kSlotMask);   // slot 1 still needs V(j)
+          const bool nxt_other_later = (s == 0) && ((m_nxt >> RS) & kSlotMask);   // slot 1 still needs K(j+1)
+          if (cur) {
+            issue_pv(s, j);
+            if (!cur_other_later) mma_commit(bars + B_VE + (j & 1));
+          }
+          if (nxt) {
+            issue_s(s, j + 1);
+            if (!nxt_other_later) mma_commit(bars + B_KE + (j + 1) % 3);
+          }
+        }
         m_cur = m_nxt;
         m_nxt = m_nxt2;
       }
@@ -257,32 +259,28 @@ fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUt
       ok = mbar_wait_warp(bars + B_SF + s, cnt & 1, a.error_word, 12);
       if (!ok) break;
       tc_fence_after();
-      uint32_t sreg[128];
-      tmem_ld32(my_s, sreg);
-      tmem_ld32(my_s + 32, sreg + 32);
-      tmem_ld32(my_s + 64, sreg + 64);
-      tmem_ld32(my_s + 96, sreg + 96);
-      tmem_ld_wait();
+      // The row is walked in two halves of 64 columns, twice (maximum, then exponentials),
+      // re-reading tensor memory instead of holding 128 values: compact loops keep the softmax
+      // code resident in the instruction caches, which matters more than the extra reads.
       float mx = -INFINITY;
-      const bool masked = __any_sync(0xffffffffu, (lim0 < 64) || (lim1 < 64));
-      if (masked) {
+#pragma unroll 1
+      for (int hf = 0; hf < 2; ++hf) {
+        uint32_t v[64];
+        tmem_ld32(my_s + hf * 64, v);
+        tmem_ld32(my_s + hf * 64 + 32, v + 32);
+        tmem_ld_wait();
+        const int lim = hf ? lim1 : lim0;   // visible columns of this half
+        if (__any_sync(0xffffffffu, lim < 64)) {
 #pragma unroll
-        for (int c = 0; c < 64; ++c) {
-          const float v0 = (c < lim0) ? __uint_as_float(sreg[c]) : -INFINITY;
-          const float v1 = (c < lim1) ? __uint_as_float(sreg[64 + c]) : -INFINITY;
-          sreg[c] = __float_as_uint(v0);
-          sreg[64 + c] = __float_as_uint(v1);
-          mx = fmaxf(mx, fmaxf(v0, v1));
-        }
-      } else {
-        {   // four independent chains: a single chain of 64 dependent maxima is pure latency
-          float m0 = -INFINITY, m1 = -INFINITY, m2 = -INFINITY, m3 = -INFINITY;
+          for (int x = 0; x < 64; ++x) mx = fmaxf(mx, (x < lim) ? __uint_as_float(v[x]) : -INFINITY);
+        } else {
+          float m0 = mx, m1 = -INFINITY, m2 = -INFINITY, m3 = -INFINITY;
 #pragma unroll
-          for (int c = 0; c < 128; c += 8) {
-            m0 = max3(m0, __uint_as_float(sreg[c + 0]), __uint_as_float(sreg[c + 1]));
-            m1 = max3(m1, __uint_as_float(sreg[c + 2]), __uint_as_float(sreg[c + 3]));
-            m2 = max3(m2, __uint_as_float(sreg[c + 4]), __uint_as_float(sreg[c + 5]));
-            m3 = max3(m3, __uint_as_float(sreg[c + 6]), __uint_as_float(sreg[c + 7]));
+          for (int x = 0; x < 64; x += 8) {
+            m0 = max3(m0, __uint_as_float(v[x + 0]), __uint_as_float(v[x + 1]));
+            m1 = max3(m1, __uint_as_float(v[x + 2]), __uint_as_float(v[x + 3]));
+            m2 = max3(m2, __uint_as_float(v[x + 4]), __uint_as_float(v[x + 5]));
+            m3 = max3(m3, __uint_as_float(v[x + 6]), __uint_as_float(v[x + 7]));
           }
           mx = fmaxf(fmaxf(m0, m1), fmaxf(m2, m3));
         }
@@ -297,7 +295,7 @@ fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUt
           ok = mbar_wait_warp(bars + B_OD + s, (cnt - 1) & 1, a.error_word, 13);
           if (!ok) break;
           tc_fence_after();
-#pragma unroll
+#pragma unroll 1
           for (int c = 0; c < D / 16; ++c) {
             uint32_t oreg[16];
             tmem_ld16(my_o + c * 16, oreg);
@@ -310,40 +308,32 @@ fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUt
       }
       const float neg_m = (m_ref == -INFINITY) ? 0.f : -m_ref;
       float rs0 = 0.f, rs1 = 0.f;
-      if (masked) {   // steps with hidden keys: every exponential on the exact path (-inf -> 0)
+#pragma unroll 1
+      for (int hf = 0; hf < 2; ++hf) {
+        uint32_t v[64], preg[32];
+        tmem_ld32(my_s + hf * 64, v);
+        tmem_ld32(my_s + hf * 64 + 32, v + 32);
+        tmem_ld_wait();
+        const int lim = hf ? lim1 : lim0;
+        if (__any_sync(0xffffffffu, lim < 64)) {
 #pragma unroll
-        for (int c = 0; c < 128; c += 32) {
-          uint32_t preg[16];
-#pragma unroll
-          for (int x = 0; x < 32; x += 2) {
-            const float p0 = fast_exp2(fmaf(__uint_as_float(sreg[c + x]), a.scale_log2, neg_m));
-            const float p1 = fast_exp2(fmaf(__uint_as_float(sreg[c + x + 1]), a.scale_log2, neg_m));
-            rs0 += p0;
-            rs1 += p1;
-            preg[x >> 1] = pack_bf16(p0, p1);
-          }
-          tmem_st16(my_s + (c >> 1), preg);   // P over the S columns already in registers
+          for (int x = 0; x < 64; ++x)
+            v[x] = (x < lim) ? v[x] : 0xff800000u;   // -inf: the exponential below gives exactly 0
         }
-      } else {        // kFwdPolyPer8 of every 8 exponentials go to the FMA pipe
-        const uint64_t sc2 = f32x2(a.scale_log2, a.scale_log2), nm2 = f32x2(neg_m, neg_m);
-        uint64_t rsum[4] = {f32x2(0.f, 0.f), f32x2(0.f, 0.f), f32x2(0.f, 0.f), f32x2(0.f, 0.f)};   // independent chains
+        float q0 = 0.f, q1 = 0.f, q2 = 0.f, q3 = 0.f;   // independent partial sums
 #pragma unroll
-        for (int c = 0; c < 128; c += 32) {
-          uint32_t preg[16];
-#pragma unroll
-          for (int x = 0; x < 32; x += 2) {
-            uint64_t& rs2 = rsum[(x >> 1) & 3];
-            float x0, x1;
-            f32x2_split(fma_f32x2(f32x2(__uint_as_float(sreg[c + x]), __uint_as_float(sreg[c + x + 1])), sc2, nm2),
-                        x0, x1);
-            const float p0 = ((x & 7) < kFwdPolyPer8) ? poly_exp2(x0) : fast_exp2(x0);
-            const float p1 = (((x + 1) & 7) < kFwdPolyPer8) ? poly_exp2(x1) : fast_exp2(x1);
-            rs2 = add_f32x2(rs2, f32x2(p0, p1));
-            preg[x >> 1] = pack_bf16(p0, p1);
-          }
-          tmem_st16(my_s + (c >> 1), preg);
+        for (int x = 0; x < 64; x += 4) {
+          const float p0 = fast_exp2(fmaf(__uint_as_float(v[x]), a.scale_log2, neg_m));
+          const float p1 = fast_exp2(fmaf(__uint_as_float(v[x + 1]), a.scale_log2, neg_m));
+          const float p2 = fast_exp2(fmaf(__uint_as_float(v[x + 2]), a.scale_log2, neg_m));
+          const float p3 = fast_exp2(fmaf(__uint_as_float(v[x + 3]), a.scale_log2, neg_m));
+          q0 += p0; q1 += p1; q2 += p2; q3 += p3;
+          preg[x >> 1] = pack_bf16(p0, p1);
+          preg[(x >> 1) + 1] = pack_bf16(p2, p3);
         }
-        f32x2_split(add_f32x2(add_f32x2(rsum[0], rsum[1]), add_f32x2(rsum[2], rsum[3])), rs0, rs1);
+        rs0 += q0 + q2;
+        rs1 += q1 + q3;
+        tmem_st32(my_s + hf * 32, preg);   // P over S columns that were already read
       }
       l_run += rs0 + rs1;
       tmem_st_wait();
