@@ -235,9 +235,10 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--quick", action="store_true", help="headline workload only (no other configs, no e2e)")
     ap.add_argument("--no-oracle", action="store_true", help="skip the CPU-oracle baseline leg")
-    ap.add_argument("--case", default="full", choices=["full", "small"],
+    ap.add_argument("--case", default="full", choices=["full", "small", "decode"],
                     help="small: the headline pattern at 8 heads x 32K tokens, for profiler captures "
-                         "(implies --quick --no-oracle; its numbers are not benchmark values)")
+                         "(implies --quick --no-oracle; its numbers are not benchmark values); "
+                         "decode: only the 70B-shaped decode over the sink+window ring, for profiler captures")
     args = ap.parse_args()
     if args.case == "small":
         args.quick = args.no_oracle = True
@@ -264,6 +265,10 @@ def main():
         dist.barrier()
     lg.load_library()
     peaks = load_peaks()
+    if args.case == "decode":
+        d5 = bench_decode(lg, synth.CFG5, args.warmup, max(args.steps, 1))
+        print(json.dumps({"case": "decode", **d5}), flush=True)
+        return
     cfg = synth.CFG3
     if args.case == "small":
         from dataclasses import replace
@@ -313,8 +318,13 @@ def main():
             "bwd_dq": (float(kms[2]), pairs * cfg.D * 2), "bwd_delta": (float(kms[0]), 0.0)}
     dom = max(("fwd", "bwd_dkdv", "bwd_dq"), key=lambda n: kern[n][0])
     achieved = kern[dom][1] / kern[dom][0] / 1e9
+    # dram__bytes_read + dram__bytes_write of one launch, from the ncu capture of the same kernels on
+    # the 8-head x 32K case of this pattern, scaled by the (head, token) units of this workload
+    ncu_small_bytes = {"fwd": 268.1e6, "bwd_dkdv": 446.1e6, "bwd_dq": 341.4e6}
+    traffic = ncu_small_bytes[dom] * (cfg.B * cfg.Hq * cfg.L) / (8 * 32768.0)
     roofline = {"bound": "tensor", "kernel": dom, "achieved": achieved, "peak": peaks["bf16_sustained"],
-                "unit": "TFLOP/s", "frac": achieved / peaks["bf16_sustained"], "traffic": None,
+                "unit": "TFLOP/s", "frac": achieved / peaks["bf16_sustained"], "traffic": traffic,
+                "traffic_note": "bytes; ncu capture of the 8-head x 32K case scaled by (head, token) units",
                 "peak_source": "%s sustained bf16 matmul" % peaks["source"],
                 "frac_of_nominal_2250": achieved / NOMINAL_BF16_TFLOPS,
                 "kernel_ms": {k: v[0] for k, v in kern.items()},
@@ -371,6 +381,10 @@ def main():
         others = [r2, r2f, r4, d5, d5d]
         line["other"] = others
         line["decode_hbm_gbs"] = d5["gbs"]
+        line["decode_roofline"] = {"bound": "hbm", "kernel": "decode_stream_kernel", "achieved": d5["gbs"],
+                                   "peak": peaks["hbm_gbs"], "unit": "GB/s", "frac": d5["gbs"] / peaks["hbm_gbs"],
+                                   "frac_of_nominal_8000": d5["gbs"] / NOMINAL_HBM_GBS,
+                                   "peak_source": "%s copy bandwidth" % peaks["source"]}
     if rank == 0 and not args.no_oracle and world == 1:
         tf, desc, cores, _ = oracle_sample(cfg)
         line["cpu_baseline"] = {"value": tf, "unit": UNIT, "cores": cores, "kind": "oracle", "sample": desc}
