@@ -378,7 +378,12 @@ def main():
         torch.cuda.empty_cache()
         d5d = bench_decode(lg, synth.CFG5, 2, 5, dense=True)
         d5d["pct_of_measured_copy"] = 100 * d5d["gbs"] / peaks["hbm_gbs"]
-        others = [r2, r2f, r4, d5, d5d]
+        # the paper's own pattern settings (Section 4.1) on the Llama-2-7B shape at 128K
+        rp1, _ = bench_attn(lg, synth.PAPER_SINK, 3, 3, want_bwd=True)
+        torch.cuda.empty_cache()
+        rp2, _ = bench_attn(lg, synth.PAPER_STRIDED, 3, 3, want_bwd=True)
+        torch.cuda.empty_cache()
+        others = [r2, r2f, r4, d5, d5d, rp1, rp2]
         line["other"] = others
         line["decode_hbm_gbs"] = d5["gbs"]
         line["decode_roofline"] = {"bound": "hbm", "kernel": "decode_stream_kernel", "achieved": d5["gbs"],

@@ -116,6 +116,8 @@ WsLayout ws_layout(const Resolved& r, bool want_bwd) {
     w.kt_cnt = take(r.n_ktiles * 4);
     w.kt_ent = take(nnz * 4);
     w.kt_order = take(r.n_ktiles * 4);
+    w.kt_cols = take(static_cast<size_t>(r.n_ktiles) * 2 * 4);
+    w.kt_off = take((static_cast<size_t>(r.n_ktiles) + 1) * 4);
     w.delta = take(static_cast<size_t>(r.B) * r.Hq * r.L * 8);   // (LSE * log2 e, delta) per query row
   }
   w.total = off;
@@ -145,9 +147,13 @@ lg_status prepare_workspace(const Resolved& r, const WsLayout& w, uint8_t* ws, b
                                                                    r.n_stiles, i32(w.sq_cnt), i32(w.sq_ent));
   tile_order_kernel<<<(r.n_stiles + 127) / 128, 128, 0, stream>>>(i32(w.sq_cnt), r.n_stiles, i32(w.sq_order));
   if (want_bwd) {
-    tile_merge_kernel<<<(r.n_ktiles + 127) / 128, 128, 0, stream>>>(i32(w.col_ptr), i32(w.row_idx), r.pat.nB, R,
-                                                                    r.n_ktiles, i32(w.kt_cnt), i32(w.kt_ent));
-    tile_order_kernel<<<(r.n_ktiles + 127) / 128, 128, 0, stream>>>(i32(w.kt_cnt), r.n_ktiles, i32(w.kt_order));
+    const int nB = r.pat.nB, nt = r.n_ktiles;
+    kv_tile_cols_kernel<<<(nt * R + 127) / 128, 128, 0, stream>>>(i32(w.col_ptr), nB, R, nt, i32(w.kt_cols));
+    kv_tile_len_kernel<<<(nt + 127) / 128, 128, 0, stream>>>(i32(w.col_ptr), i32(w.kt_cols), R, nt, i32(w.kt_off));
+    index_scan_kernel<<<1, 1024, 0, stream>>>(i32(w.kt_off), i32(w.kt_off), nt);
+    kv_tile_merge_kernel<<<(nt + 127) / 128, 128, 0, stream>>>(i32(w.col_ptr), i32(w.row_idx), i32(w.kt_cols),
+                                                               i32(w.kt_off), R, nt, i32(w.kt_cnt), i32(w.kt_ent));
+    tile_order_kernel<<<(nt + 127) / 128, 128, 0, stream>>>(i32(w.kt_cnt), nt, i32(w.kt_order));
   }
   return cudaGetLastError() == cudaSuccess ? LG_OK : LG_ERR_CUDA;
 }

@@ -34,9 +34,10 @@ static lg_status launch_bwd_t(const Resolved& r, const WsLayout& w, const void* 
     CUtensorMap tq, tk, tv, tdo;
     if ((s = make_tmap(&tq, q, r.B, r.Hq, r.L, D, r.qs, BS)) != LG_OK) return s;
     if ((s = make_tmap(&tdo, d_o, r.B, r.Hq, r.L, D, r.os, BS)) != LG_OK) return s;
-    if ((s = make_tmap(&tk, k, r.B, r.Hkv, r.L, D, r.ks, 128)) != LG_OK) return s;
-    if ((s = make_tmap(&tv, v, r.B, r.Hkv, r.L, D, r.vs, 128)) != LG_OK) return s;
-    a.tile_off = reinterpret_cast<const int32_t*>(ws + w.col_ptr);
+    if ((s = make_tmap(&tk, k, r.B, r.Hkv, r.L, D, r.ks, BS)) != LG_OK) return s;
+    if ((s = make_tmap(&tv, v, r.B, r.Hkv, r.L, D, r.vs, BS)) != LG_OK) return s;
+    a.tile_off = reinterpret_cast<const int32_t*>(ws + w.kt_off);
+    a.tile_cols = reinterpret_cast<const int32_t*>(ws + w.kt_cols);
     a.tile_cnt = reinterpret_cast<const int32_t*>(ws + w.kt_cnt);
     a.tile_ent = reinterpret_cast<const int32_t*>(ws + w.kt_ent);
     a.order = reinterpret_cast<const int32_t*>(ws + w.kt_order);
@@ -58,6 +59,7 @@ static lg_status launch_bwd_t(const Resolved& r, const WsLayout& w, const void* 
     if ((s = make_tmap(&tk, k, r.B, r.Hkv, r.L, D, r.ks, BS)) != LG_OK) return s;
     if ((s = make_tmap(&tv, v, r.B, r.Hkv, r.L, D, r.vs, BS)) != LG_OK) return s;
     a.tile_off = reinterpret_cast<const int32_t*>(ws + w.row_ptr);
+    a.tile_cols = nullptr;
     a.tile_cnt = reinterpret_cast<const int32_t*>(ws + w.qt_cnt);
     a.tile_ent = reinterpret_cast<const int32_t*>(ws + w.qt_ent);
     a.order = reinterpret_cast<const int32_t*>(ws + w.qt_order);

@@ -28,7 +28,8 @@
 namespace lg {
 
 struct BwdArgs {
-  const int32_t* tile_off;   // CSR row_ptr (dQ pass) or CSC col_ptr (dK/dV pass)
+  const int32_t* tile_off;   // dQ pass: CSR row_ptr (tile t starts at tile_off[R t]); dK/dV pass: start per tile
+  const int32_t* tile_cols;  // dK/dV pass: pattern column of each member of a kv tile (-1: none)
   const int32_t* tile_cnt;
   const int32_t* tile_ent;   // idx * 4 + member mask
   const int32_t* order;
@@ -408,8 +409,9 @@ bwd_dkdv_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
   const int tile = a.order[blockIdx.y];
   const int b = blockIdx.x / a.Hkv, hk = blockIdx.x % a.Hkv;
   const int n_ent = a.tile_cnt[tile];
-  const int32_t* ent = a.tile_ent + a.tile_off[tile * R];
-  const int key0 = tile * 128;
+  const int32_t* ent = a.tile_ent + a.tile_off[tile];
+  // key blocks of the tile's members (with 64-token blocks the two members need not be neighbours)
+  const int kb_a = a.tile_cols[R * tile], kb_b = (R == 2) ? a.tile_cols[R * tile + 1] : -1;
   const int n_items = n_ent * a.G;
   const int n_steps = (BS == 128) ? n_items : (n_items + 1) / 2;
 
@@ -448,8 +450,12 @@ bwd_dkdv_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
     if (lane == 0) {
       tma_prefetch_desc(&tm_q); tma_prefetch_desc(&tm_k); tma_prefetch_desc(&tm_v); tma_prefetch_desc(&tm_do);
       mbar_expect_tx(bars + B_FIX, 2 * kTile);
-      tma_load_rows<D, 128>(sK, &tm_k, bars + B_FIX, 0, key0, hk, b);
-      tma_load_rows<D, 128>(sV, &tm_v, bars + B_FIX, 0, key0, hk, b);
+      tma_load_rows<D, BS>(sK, &tm_k, bars + B_FIX, 0, kb_a * BS, hk, b);
+      tma_load_rows<D, BS>(sV, &tm_v, bars + B_FIX, 0, kb_a * BS, hk, b);
+      if (R == 2) {   // second member (a missing one re-loads the first; its rows are never stored)
+        tma_load_rows<D, BS>(sK, &tm_k, bars + B_FIX, 1, (kb_b >= 0 ? kb_b : kb_a) * BS, hk, b);
+        tma_load_rows<D, BS>(sV, &tm_v, bars + B_FIX, 1, (kb_b >= 0 ? kb_b : kb_a) * BS, hk, b);
+      }
       bool ok = true;
       int nq = 0, no = 0;   // loads started
       for (int j = 0; j < n_steps; ++j) {
@@ -543,8 +549,9 @@ bwd_dkdv_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
     // ------------------------------ element-wise warps ------------------------------------
     const int wg = warp >> 2;
     const int r = (warp & 3) * 32 + lane;                   // key row in the tile == TMEM lane
-    const int kj = key0 + r;
     const int member = (R == 1) ? 0 : (r / BS);
+    const int kb_mine = (R == 2 && member) ? kb_b : kb_a;
+    const int kj = kb_mine * BS + (R == 2 ? (r & (BS - 1)) : r);   // this thread's key (kb_mine < 0: none)
     const uint32_t lane_addr = tmem + (static_cast<uint32_t>((warp & 3) * 32) << 16);
     const int col = tid & 127;                              // the column whose statistics I fetch
     auto fetch_stat = [&](int j) -> float2 {
@@ -640,7 +647,7 @@ bwd_dkdv_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
     }
     if (ok) {
       tc_fence_after();
-      if (kj < a.L) {
+      if (kb_mine >= 0) {
         __nv_bfloat16* dk_row = a.out0 + b * a.s0[0] + hk * a.s0[1] + static_cast<int64_t>(kj) * a.s0[2] + wg * (D / 2);
         __nv_bfloat16* dv_row = a.out1 + b * a.s1[0] + hk * a.s1[1] + static_cast<int64_t>(kj) * a.s1[2] + wg * (D / 2);
         if (n_steps > 0) {

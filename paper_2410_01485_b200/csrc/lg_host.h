@@ -31,6 +31,7 @@ struct WsLayout {
   size_t qt_cnt, qt_ent, qt_order;               // query-tile schedules (dQ pass)
   size_t sq_cnt, sq_ent, sq_order;               // super-tile schedules (forward)
   size_t kt_cnt, kt_ent, kt_order;               // kv-tile schedules (dK/dV pass)
+  size_t kt_cols, kt_off;                        // members of each kv tile, start of its schedule
   size_t delta;                                  // float2 [B, Hq, L]: (LSE * log2 e, delta) (bwd only)
   size_t total;
 };

@@ -151,4 +151,60 @@ __global__ void tile_order_kernel(const int32_t* __restrict__ tile_cnt, int n_ti
   order[rank] = t;
 }
 
+// ---- kv tiles of the dK/dV pass ------------------------------------------------------------
+// A kv tile holds R pattern columns (R = 128 / block).  With R = 2 the two columns of a tile
+// should have similar lists: a comb column of the strided pattern is attended by every later
+// query block and its neighbour by a handful, so pairing neighbours would leave half of every
+// MMA idle.  Columns are therefore ranked by list length (longest first, ties by index) and
+// consecutive ranks share a tile.  cols[R * t + m] = pattern column of member m (-1: none).
+__global__ void kv_tile_cols_kernel(const int32_t* __restrict__ col_ptr, int nB, int R, int n_tiles,
+                                    int32_t* __restrict__ cols) {
+  const int c = blockIdx.x * blockDim.x + threadIdx.x;
+  if (c < n_tiles * R && c >= nB) cols[c] = -1;          // padding member of the last tile
+  if (c >= nB) return;
+  if (R == 1) { cols[c] = c; return; }
+  const int len = col_ptr[c + 1] - col_ptr[c];
+  int rank = 0;
+  for (int u = 0; u < nB; ++u) {
+    const int lu = col_ptr[u + 1] - col_ptr[u];
+    rank += (lu > len || (lu == len && u < c)) ? 1 : 0;
+  }
+  cols[rank] = c;
+}
+
+// upper bound of a tile's schedule length, written to off[t + 1] (off[0] = 0) for the scan
+__global__ void kv_tile_len_kernel(const int32_t* __restrict__ col_ptr, const int32_t* __restrict__ cols, int R,
+                                   int n_tiles, int32_t* __restrict__ off) {
+  const int t = blockIdx.x * blockDim.x + threadIdx.x;
+  if (t >= n_tiles) return;
+  int n = 0;
+  for (int m = 0; m < R; ++m) {
+    const int c = cols[R * t + m];
+    if (c >= 0) n += col_ptr[c + 1] - col_ptr[c];
+  }
+  off[t + 1] = n;
+  if (t == 0) off[0] = 0;
+}
+
+// ascending union of the members' CSC lists; entry = query block * 4 + member mask
+__global__ void kv_tile_merge_kernel(const int32_t* __restrict__ col_ptr, const int32_t* __restrict__ row_idx,
+                                     const int32_t* __restrict__ cols, const int32_t* __restrict__ off, int R,
+                                     int n_tiles, int32_t* __restrict__ tile_cnt, int32_t* __restrict__ tile_ent) {
+  const int t = blockIdx.x * blockDim.x + threadIdx.x;
+  if (t >= n_tiles) return;
+  int32_t* out = tile_ent + off[t];
+  const int ca = cols[R * t], cb = (R == 2) ? cols[R * t + 1] : -1;
+  int a = ca >= 0 ? col_ptr[ca] : 0, ae = ca >= 0 ? col_ptr[ca + 1] : 0;
+  int c = cb >= 0 ? col_ptr[cb] : 0, ce = cb >= 0 ? col_ptr[cb + 1] : 0;
+  int n = 0;
+  while (a < ae || c < ce) {
+    const int va = a < ae ? row_idx[a] : 0x7fffffff;
+    const int vc = c < ce ? row_idx[c] : 0x7fffffff;
+    if (va == vc) { out[n++] = va * 4 + 3; ++a; ++c; }
+    else if (va < vc) { out[n++] = va * 4 + 1; ++a; }
+    else { out[n++] = vc * 4 + 2; ++c; }
+  }
+  tile_cnt[t] = n;
+}
+
 }  // namespace lg
