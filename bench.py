@@ -178,6 +178,20 @@ def time_cuda(fn, warmup, steps):
     return e0.elapsed_time(e1) / steps
 
 
+def max_over_ranks(ms: float, dist, device) -> float:
+    """Step time of the job = the slowest rank's device time (ranks are independent replicas)."""
+    if dist is None:
+        return ms
+    t = torch.tensor([ms], dtype=torch.float64, device=device)
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return float(t.item())
+
+
+def aggregate_value(flops_per_rank: float, world: int, ms_step: float) -> float:
+    """Whole-job useful TFLOP/s: every rank does the same work in the time of the slowest one."""
+    return flops_per_rank * world / ms_step / 1e9
+
+
 def bench_attn(lg, cfg, warmup, steps, want_bwd, profile_kernels=False):
     p = lg.params_of(cfg)
     inp = synth.make_attn_inputs(cfg, "cuda", seed=0, with_do=want_bwd)
@@ -305,13 +319,8 @@ def main():
         kms = np.array([lg.lg_sparse_attn_bwd_profiled(p, inp["q"], inp["k"], inp["v"], o, lse, inp["do"], dq, dk,
                                                        dv, ws) for _ in range(args.steps)]).mean(axis=0)
     assert lg.lg_last_status(ws) == 0, "device-side wait expired"
-    ms_step = e0.elapsed_time(e1) / args.steps
-    if dist is not None:
-        t = torch.tensor([ms_step], device="cuda")
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        ms_step = float(t.item())
-    total_flops = flops(cfg) * world
-    value = total_flops / ms_step / 1e9
+    ms_step = max_over_ranks(e0.elapsed_time(e1) / args.steps, dist, "cuda")
+    value = aggregate_value(flops(cfg), world, ms_step)
 
     pairs = float(pairs_per_head(cfg)) * cfg.B * cfg.Hq
     kern = {"fwd": (fwd_ms, pairs * cfg.D * 4), "bwd_dkdv": (float(kms[1]), pairs * cfg.D * 8),
