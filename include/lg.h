@@ -50,7 +50,10 @@ typedef enum {
  *   FULL_CAUSAL   : (nothing more)
  *   SINK_WINDOW   : kb < sink_tokens/Bs  or  qb - kb < window_tokens/Bs
  *                   (the window is block-granular and counts the query's own block:
- *                    "the first block for sink tokens and the most recent 32 blocks")
+ *                    "the first block for sink tokens and the most recent 32 blocks");
+ *                   with window_exact != 0 the second condition is i - j < window_tokens,
+ *                   the token-exact window of the rolling-buffer cache (Section 3.2), so
+ *                   that a model can be trained on exactly the keys lg_sparse_decode reads
  *   STRIDED_LOCAL : qb - kb < local_blocks  or  kb % stride_blocks == 0
  * Grouped-query attention: query head h reads kv head h / (Hq / Hkv).
  */
@@ -62,6 +65,7 @@ typedef struct {
   int32_t window_tokens;      /* SINK_WINDOW: multiple of block, >= block                    */
   int32_t stride_blocks;      /* STRIDED_LOCAL: >= 1                                         */
   int32_t local_blocks;       /* STRIDED_LOCAL: >= 1 (the diagonal block is always active)   */
+  int32_t window_exact;       /* SINK_WINDOW: 0 = block-granular window, 1 = token-exact     */
   float   scale;              /* softmax scale; 0 selects 1/sqrt(D)                          */
   /* Strides in ELEMENTS of (batch, head, token) for Q, K, V, O; dO and dQ use the O / Q
      strides, dK / dV the K / V strides.  All zero selects contiguous [B, H, L, D].

@@ -18,7 +18,9 @@ value.  All arithmetic is float64.
 
 Readings of points on which the paper is silent:
   - the window is block-granular and counts the query's own block
-    (Section 4.1: "the first block ... and the most recent 32 blocks");
+    (Section 4.1: "the first block ... and the most recent 32 blocks"); with
+    window_exact it is the token-exact window of the rolling-buffer cache
+    (Section 3.2), i - j < window_tokens, which is what the decode attends;
   - the strided comb is absolute: KV block kb is retained iff kb % stride == 0;
   - LSE is the natural log of the sum of exp of the *scaled* scores;
   - the backward formulas are the derivatives of the definition (the paper
@@ -53,11 +55,12 @@ class Pattern:
     window_tokens: int = 0
     stride_blocks: int = 0
     local_blocks: int = 0
+    window_exact: bool = False   # sink + window only: the window edge is token-exact (i - j < window_tokens)
 
     @staticmethod
     def of(cfg) -> "Pattern":
         return Pattern(cfg.L, cfg.block, cfg.mode, cfg.sink_tokens, cfg.window_tokens,
-                       cfg.stride_blocks, cfg.local_blocks)
+                       cfg.stride_blocks, cfg.local_blocks, bool(getattr(cfg, "window_exact", False)))
 
 
 # --------------------------------------------------------------------------- masks
@@ -77,6 +80,10 @@ def allowed(p: Pattern, i, j):
     if p.mode == MODE_SINK_WINDOW:
         ns = p.sink_tokens // p.block
         nw = p.window_tokens // p.block
+        if p.window_exact:
+            # the Mistral-style window the paper cites for serving (Section 3.2): the last
+            # window_tokens tokens, the query's own included; sink blocks as before
+            return causal & ((kb < ns) | (i - j < p.window_tokens))
         return causal & ((kb < ns) | (qb - kb < nw))
     if p.mode == MODE_STRIDED_LOCAL:
         return causal & ((qb - kb < p.local_blocks) | (kb % p.stride_blocks == 0))

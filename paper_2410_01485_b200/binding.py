@@ -29,7 +29,7 @@ class AttnParams(C.Structure):
     _fields_ = [("B", C.c_int32), ("Hq", C.c_int32), ("Hkv", C.c_int32), ("L", C.c_int32), ("D", C.c_int32),
                 ("block", C.c_int32), ("mode", C.c_int32), ("sink_tokens", C.c_int32),
                 ("window_tokens", C.c_int32), ("stride_blocks", C.c_int32), ("local_blocks", C.c_int32),
-                ("scale", C.c_float),
+                ("window_exact", C.c_int32), ("scale", C.c_float),
                 ("q_strides", C.c_int64 * 3), ("k_strides", C.c_int64 * 3), ("v_strides", C.c_int64 * 3),
                 ("o_strides", C.c_int64 * 3)]
 
@@ -94,18 +94,20 @@ def _strides3(t: torch.Tensor):
 
 
 def attn_params(B, Hq, Hkv, L, D, block, mode, sink_tokens=0, window_tokens=0, stride_blocks=0, local_blocks=0,
-                scale=0.0) -> AttnParams:
+                scale=0.0, window_exact=False) -> AttnParams:
     p = AttnParams()
     p.B, p.Hq, p.Hkv, p.L, p.D, p.block, p.mode = B, Hq, Hkv, L, D, block, mode
     p.sink_tokens, p.window_tokens, p.stride_blocks, p.local_blocks = sink_tokens, window_tokens, stride_blocks, local_blocks
     p.scale = scale
+    p.window_exact = int(bool(window_exact))
     return p
 
 
 def params_of(cfg, scale: float = 0.0) -> AttnParams:
     """AttnParams from a synth.AttnConfig-like object."""
     return attn_params(cfg.B, cfg.Hq, cfg.Hkv, cfg.L, cfg.D, cfg.block, cfg.mode, cfg.sink_tokens,
-                       cfg.window_tokens, cfg.stride_blocks, cfg.local_blocks, scale)
+                       cfg.window_tokens, cfg.stride_blocks, cfg.local_blocks, scale,
+                       getattr(cfg, "window_exact", False))
 
 
 # ------------------------------------------------------------------------------ index

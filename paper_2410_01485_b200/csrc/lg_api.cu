@@ -46,14 +46,18 @@ lg_status resolve(const lg_attn_params* p, Resolved* r) {
   r->pat.nB = p->L / p->block;
   r->pat.mode = p->mode;
   r->pat.ns = r->pat.nw = r->pat.stride = r->pat.nl = 0;
+  r->exact_w = 0;
   switch (p->mode) {
     case LG_MODE_FULL_CAUSAL:
       break;
     case LG_MODE_SINK_WINDOW:
       if (p->sink_tokens < 0 || p->sink_tokens % p->block != 0) return LG_ERR_INVALID_ARG;
       if (p->window_tokens < p->block || p->window_tokens % p->block != 0) return LG_ERR_INVALID_ARG;
+      if (p->window_exact != 0 && p->window_exact != 1) return LG_ERR_INVALID_ARG;
       r->pat.ns = p->sink_tokens / p->block;
-      r->pat.nw = p->window_tokens / p->block;
+      // a token-exact window of W tokens reaches into one more block (partially)
+      r->pat.nw = p->window_tokens / p->block + (p->window_exact ? 1 : 0);
+      r->exact_w = p->window_exact ? p->window_tokens : 0;
       break;
     case LG_MODE_STRIDED_LOCAL:
       if (p->stride_blocks < 1 || p->local_blocks < 1) return LG_ERR_INVALID_ARG;

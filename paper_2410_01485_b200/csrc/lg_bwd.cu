@@ -25,6 +25,7 @@ static lg_status launch_bwd_t(const Resolved& r, const WsLayout& w, const void* 
   a.stat = stat;
   a.error_word = reinterpret_cast<unsigned int*>(ws);
   a.L = r.L; a.Hq = r.Hq; a.Hkv = r.Hkv; a.G = r.G;
+  a.exact_w = r.exact_w; a.ns = r.pat.ns;
   a.scale = r.scale;
   a.scale_log2 = r.scale * 1.4426950408889634f;
   constexpr int smem = BwdSmem<D, BS>::kTotal;

@@ -39,6 +39,7 @@ struct BwdArgs {
   unsigned int* error_word;
   int64_t s0[3], s1[3];      // strides of out0 / out1 (batch, head, token; elements)
   int L, Hq, Hkv, G;
+  int exact_w, ns;           // token-exact window (0: off) and number of sink blocks
   float scale, scale_log2;
 };
 
@@ -309,7 +310,8 @@ bwd_dq_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ 
       const int entry = ent[e];
       const int key0 = (entry >> 2) * BS + (BS == 128 ? 64 * wg : 0);
       const bool on = have && ((entry >> member) & 1);
-      const int lim = on ? min(max(qi - key0 + 1, 0), 64) : 0;   // columns c < lim are visible
+      const int lim = on ? min(max(qi - key0 + 1, 0), 64) : 0;   // columns lo <= c < lim are visible
+      const int lo = (a.exact_w > 0 && (entry >> 2) >= a.ns) ? min(max(qi - a.exact_w + 1 - key0, 0), 64) : 0;
 
       ok = mbar_wait(bars + B_SF + (j & 1), (j >> 1) & 1, a.error_word, 31);
       ok = __all_sync(0xffffffffu, ok);
@@ -321,11 +323,11 @@ bwd_dq_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ 
         tmem_ld32(lane_addr + kColS + (j & 1) * 128 + wg * 64, sreg);
         tmem_ld32(lane_addr + kColS + (j & 1) * 128 + wg * 64 + 32, sreg + 32);
         tmem_ld_wait();
-        if (__any_sync(0xffffffffu, lim < 64)) {
+        if (__any_sync(0xffffffffu, lim < 64 || lo > 0)) {
 #pragma unroll
           for (int c = 0; c < 64; ++c) {
             const float v = fast_exp2(fmaf(__uint_as_float(sreg[c]), a.scale_log2, -lse2));
-            p[c] = (c < lim) ? v : 0.f;
+            p[c] = (c < lim && c >= lo) ? v : 0.f;
           }
         } else {
 #pragma unroll
@@ -588,7 +590,8 @@ bwd_dkdv_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
       item_of(it, hq, qrow, entry);
       const int q0 = qrow + (BS == 128 ? 64 * wg : 0);
       const bool on = have && ((entry >> member) & 1);
-      const int xmin = on ? min(max(kj - q0, 0), 64) : 64;     // columns c >= xmin are visible
+      const int xmin = on ? min(max(kj - q0, 0), 64) : 64;     // columns xmin <= c < xmax are visible
+      const int xmax = (a.exact_w > 0 && kb_mine >= a.ns) ? min(max(kj + a.exact_w - q0, 0), 64) : 64;
 
       ok = mbar_wait(bars + B_SF, j & 1, a.error_word, 1);
       ok = __all_sync(0xffffffffu, ok);
@@ -600,15 +603,15 @@ bwd_dkdv_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
         tmem_ld32(lane_addr + kColS + wg * 64, sreg);
         tmem_ld32(lane_addr + kColS + wg * 64 + 32, sreg + 32);
         tmem_ld_wait();
-        const bool masked = __any_sync(0xffffffffu, xmin > 0);
+        const bool masked = __any_sync(0xffffffffu, xmin > 0 || xmax < 64);
 #pragma unroll
         for (int c = 0; c < 64; c += 2) {
           const float4 s2 = *reinterpret_cast<const float4*>(st + c);   // (lse2, delta) of two columns
           float v0 = fast_exp2(fmaf(__uint_as_float(sreg[c]), a.scale_log2, -s2.x));
           float v1 = fast_exp2(fmaf(__uint_as_float(sreg[c + 1]), a.scale_log2, -s2.z));
           if (masked) {
-            v0 = (c >= xmin) ? v0 : 0.f;
-            v1 = (c + 1 >= xmin) ? v1 : 0.f;
+            v0 = (c >= xmin && c < xmax) ? v0 : 0.f;
+            v1 = (c + 1 >= xmin && c + 1 < xmax) ? v1 : 0.f;
           }
           p[c] = v0;
           p[c + 1] = v1;

@@ -22,6 +22,7 @@ static lg_status launch_fwd_t(const Resolved& r, const WsLayout& w, const void* 
   a.error_word = reinterpret_cast<unsigned int*>(ws);
   for (int i = 0; i < 3; ++i) a.o_strides[i] = r.os[i];
   a.L = r.L; a.Hq = r.Hq; a.G = r.G;
+  a.exact_w = r.exact_w; a.ns = r.pat.ns;
   a.scale_log2 = r.scale * 1.4426950408889634f;
   auto kern = fwd_kernel<D, BS>;
   constexpr int smem = FwdSmem<D>::kTotal;

@@ -30,6 +30,7 @@ struct FwdArgs {
   unsigned int* error_word;
   int64_t o_strides[3];      // batch, head, token (elements)
   int L, Hq, G;              // G = Hq / Hkv
+  int exact_w, ns;           // token-exact window (0: off) and number of sink blocks
   float scale_log2;          // scale * log2(e)
 };
 
@@ -251,10 +252,13 @@ fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUt
       load_ent(j + 1, ne0, ne1);
       const uint32_t m_step = (static_cast<uint32_t>(e0) | static_cast<uint32_t>(e1)) & 15u;
       if (((m_step >> (s * RS)) & kSlotMask) == 0) continue;          // uniform over the slot
-      // visible columns of the two 64-column halves: c < lim0, 64 + c < 64 + lim1
+      // visible columns of the two 64-column halves: lo0 <= c < lim0 and lo1 <= c < lim1 (the lower
+      // bound only exists with a token-exact window, on blocks outside the sink)
       const int key0 = (e0 >> 4) * BS, key1 = (BS == 128) ? key0 + 64 : (e1 >> 4) * BS;
       const int lim0 = ((e0 >> member) & 1) ? min(max(qi - key0 + 1, 0), 64) : 0;
       const int lim1 = ((e1 >> member) & 1) ? min(max(qi - key1 + 1, 0), 64) : 0;
+      const int lo0 = (a.exact_w > 0 && (e0 >> 4) >= a.ns) ? min(max(qi - a.exact_w + 1 - key0, 0), 64) : 0;
+      const int lo1 = (a.exact_w > 0 && (e1 >> 4) >= a.ns) ? min(max(qi - a.exact_w + 1 - key1, 0), 64) : 0;
 
       ok = mbar_wait_warp(bars + B_SF + s, cnt & 1, a.error_word, 12);
       if (!ok) break;
@@ -269,10 +273,10 @@ fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUt
         tmem_ld32(my_s + hf * 64, v);
         tmem_ld32(my_s + hf * 64 + 32, v + 32);
         tmem_ld_wait();
-        const int lim = hf ? lim1 : lim0;   // visible columns of this half
-        if (__any_sync(0xffffffffu, lim < 64)) {
+        const int lim = hf ? lim1 : lim0, lo = hf ? lo1 : lo0;   // visible columns of this half
+        if (__any_sync(0xffffffffu, lim < 64 || lo > 0)) {
 #pragma unroll
-          for (int x = 0; x < 64; ++x) mx = fmaxf(mx, (x < lim) ? __uint_as_float(v[x]) : -INFINITY);
+          for (int x = 0; x < 64; ++x) mx = fmaxf(mx, (x < lim && x >= lo) ? __uint_as_float(v[x]) : -INFINITY);
         } else {
           float m0 = mx, m1 = -INFINITY, m2 = -INFINITY, m3 = -INFINITY;
 #pragma unroll
@@ -314,11 +318,11 @@ fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUt
         tmem_ld32(my_s + hf * 64, v);
         tmem_ld32(my_s + hf * 64 + 32, v + 32);
         tmem_ld_wait();
-        const int lim = hf ? lim1 : lim0;
-        if (__any_sync(0xffffffffu, lim < 64)) {
+        const int lim = hf ? lim1 : lim0, lo = hf ? lo1 : lo0;
+        if (__any_sync(0xffffffffu, lim < 64 || lo > 0)) {
 #pragma unroll
           for (int x = 0; x < 64; ++x)
-            v[x] = (x < lim) ? v[x] : 0xff800000u;   // -inf: the exponential below gives exactly 0
+            v[x] = (x < lim && x >= lo) ? v[x] : 0xff800000u;   // -inf: the exponential below gives exactly 0
         }
         float q0 = 0.f, q1 = 0.f, q2 = 0.f, q3 = 0.f;   // independent partial sums
 #pragma unroll

@@ -17,6 +17,7 @@ struct Resolved {          // validated, defaulted copy of lg_attn_params
   int B, Hq, Hkv, L, D, block, mode, G;
   PatternDev pat;
   float scale;
+  int exact_w;             // token-exact window length in tokens (0: block-granular)
   int64_t qs[3], ks[3], vs[3], os[3];
   int n_qtiles, n_ktiles;  // ceil(L / 128)
   int n_stiles;            // ceil(L / 256): super-tiles of the forward

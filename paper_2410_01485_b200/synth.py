@@ -37,6 +37,7 @@ class AttnConfig:
     stride_blocks: int = 0
     local_blocks: int = 0
     backward: bool = True
+    window_exact: bool = False   # sink + window: token-exact window edge (matches the decode's ring)
 
     def full_causal(self) -> "AttnConfig":
         return replace(self, name=self.name + "_full", mode=MODE_FULL_CAUSAL)

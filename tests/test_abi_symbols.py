@@ -55,6 +55,7 @@ def test_nnz_and_sizes_on_host(lib):
     lambda p: setattr(p, "mode", 7),
     lambda p: setattr(p, "scale", -1.0),
     lambda p: setattr(p, "B", 0),
+    lambda p: setattr(p, "window_exact", 2),      # only 0 or 1
 ])
 def test_invalid_params_rejected(lib, mutate):
     p = _good()

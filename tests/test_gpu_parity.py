@@ -51,11 +51,18 @@ SMALL = [
     replace(synth.CFG1, name="window_ge_L", L=512, sink_tokens=0, window_tokens=512, Hq=3, Hkv=1, D=128),
     replace(synth.CFG1, name="strided_bs128", mode=synth.MODE_STRIDED_LOCAL, stride_blocks=3, local_blocks=1,
             block=128, L=1536, D=64, Hq=2, Hkv=2),
+    # token-exact window edge (the mask the rolling-buffer decode applies)
+    replace(synth.CFG1, name="exact_bs64", window_exact=True, D=128, L=640),
+    replace(synth.CFG1, name="exact_bs128_gqa2", window_exact=True, block=128, sink_tokens=128, window_tokens=256,
+            L=1280, D=128, Hq=4, Hkv=2),
+    replace(synth.CFG1, name="exact_no_sink_ragged", window_exact=True, sink_tokens=0, window_tokens=64, L=64 * 7, D=64),
 ]
 
 
 @pytest.mark.parametrize("cfg", SMALL + [synth.CFG2, synth.CFG2.full_causal(), synth.CFG3, synth.CFG4,
-                                         synth.PAPER_SINK, synth.PAPER_STRIDED], ids=lambda c: c.name)
+                                         synth.PAPER_SINK, synth.PAPER_STRIDED,
+                                         replace(synth.PAPER_SINK, name="paper_sink_exact", window_exact=True)],
+                         ids=lambda c: c.name)
 def test_block_index_bit_exact(lg, cfg):
     got = lg.lg_build_block_index(lg.params_of(cfg))
     torch.cuda.synchronize()
@@ -132,6 +139,28 @@ def test_strided_inputs(lg):
     o2, lse2 = lg.lg_sparse_attn_fwd(lg.params_of(cfg), q_view, k_view, v_view, o=o2)
     torch.cuda.synchronize()
     assert torch.equal(o1, o2.contiguous()) and torch.equal(lse1, lse2)
+
+
+def test_exact_window_training_mask_is_the_decode_mask(lg):
+    """With window_exact the last query row of the forward and a decode over the ring built from the
+    same keys read exactly the same tokens: the two CUDA paths must agree (and both match the oracle)."""
+    cfg = replace(synth.CFG1, name="exact_vs_decode", window_exact=True, L=1024, D=128, Hq=8, Hkv=1,
+                  sink_tokens=64, window_tokens=256)
+    inp = synth.make_attn_inputs(cfg, "cuda", seed=4)
+    o, lse = lg.lg_sparse_attn_fwd(lg.params_of(cfg), inp["q"], inp["k"], inp["v"])
+    dp = lg.decode_params(1, cfg.Hq, cfg.Hkv, cfg.D, cfg.sink_tokens, cfg.window_tokens)
+    kc = torch.zeros(1, cfg.Hkv, cfg.sink_tokens + cfg.window_tokens, cfg.D, device="cuda", dtype=torch.bfloat16)
+    vc = torch.zeros_like(kc)
+    lg.lg_kv_ring_append(dp, kc, vc, inp["k"].contiguous(), inp["v"].contiguous(),
+                         torch.zeros(1, dtype=torch.int64, device="cuda"))
+    qd = inp["q"][:, :, cfg.L - 1].contiguous()
+    od, lsed = lg.lg_sparse_decode(dp, qd, kc, vc, torch.full((1,), cfg.L, dtype=torch.int64, device="cuda"))
+    torch.cuda.synchronize()
+    assert (od.float() - o[:, :, cfg.L - 1].float()).abs().max().item() <= 2 ** -7   # two bf16 roundings
+    assert (lsed - lse[:, :, cfg.L - 1]).abs().max().item() <= 1e-4
+    oo, ll = O.decode(synth.to_f64(qd[0]), synth.to_f64(inp["k"][0]), synth.to_f64(inp["v"][0]), cfg.L,
+                      cfg.sink_tokens, cfg.window_tokens, 1.0 / np.sqrt(cfg.D))
+    _assert_close(synth.to_f64(o[0, :, cfg.L - 1]), oo, TOL_O, "exact-window last row")
 
 
 # ------------------------------------------------------------------------ full-size configs

@@ -434,3 +434,80 @@ def test_ring_replay_holds_exactly_the_surviving_tokens():
             assert cache[O.ring_slot(j, sink, W), 0] == j
         # sink slots never move; the ring holds the last W non-sink tokens
         assert all(cache[j, 0] == j for j in range(min(n, sink)))
+
+
+# --------------------------------------------------------- token-exact window (window_exact)
+
+def _exact(L=512, block=64, sink=64, window=128):
+    return O.Pattern(L, block, O.MODE_SINK_WINDOW, sink_tokens=sink, window_tokens=window, window_exact=True)
+
+
+def test_exact_window_predicate_bruteforce():
+    """Plain loops over token pairs: j <= i and (j in a sink block or i - j < W)."""
+    p = _exact(L=320, block=64, sink=64, window=128)
+    m = O.token_mask(p)
+    for i in range(p.L):
+        for j in range(p.L):
+            want = j <= i and (j < p.sink_tokens or i - j < p.window_tokens)
+            assert bool(m[i, j]) == want, (i, j)
+
+
+@pytest.mark.parametrize("block,sink,window", [(64, 64, 128), (128, 128, 256), (64, 0, 64), (64, 128, 64)])
+def test_exact_window_row_counts_and_block_counts(block, sink, window):
+    """Late rows see exactly sink + W keys; the exact window reaches one block further back than
+    the block-granular one, so nnz follows the closed form with nw + 1 window blocks."""
+    L = 16 * block
+    p = _exact(L, block, sink, window)
+    m = O.token_mask(p)
+    for i in range(sink + window, L):
+        assert m[i].sum() == sink + window
+    nB, ns, nw1 = L // block, sink // block, window // block + 1
+    nnz = sum(min(qb + 1, nw1) + min(ns, max(qb + 1 - nw1, 0)) for qb in range(nB))
+    row_ptr, col_idx, col_ptr, row_idx = O.block_lists(p)
+    assert row_ptr[-1] == nnz == len(col_idx) == len(row_idx)
+    # it contains the block-granular pattern with the same sizes, and nothing older than W tokens
+    coarse = O.token_mask(O.Pattern(L, block, O.MODE_SINK_WINDOW, sink_tokens=sink, window_tokens=window))
+    i, j = np.nonzero(m & ~coarse)
+    assert ((i - j) < window).all() and ((i // block) - (j // block) == window // block).all()
+    i, j = np.nonzero(coarse & ~m)
+    assert ((i - j) >= window).all()
+
+
+def test_exact_window_wide_is_full_causal():
+    p = _exact(L=256, block=64, sink=0, window=256)
+    assert np.array_equal(O.token_mask(p), np.tril(np.ones((256, 256), dtype=bool)))
+
+
+def test_exact_window_last_row_equals_decode():
+    """The decode oracle (written separately: survivors of a linear history) attends exactly the keys
+    the exact-window mask gives the last query row, so the two must agree on that row."""
+    rng = np.random.default_rng(5)
+    L, D, sink, window = 448, 32, 64, 128
+    q = rng.standard_normal((2, L, D))
+    k = rng.standard_normal((1, L, D))
+    v = rng.standard_normal((1, L, D))
+    p = _exact(L, 64, sink, window)
+    scale = 1.0 / math.sqrt(D)
+    o, lse = O.attn_forward(q, k, v, p, scale)
+    for n in (L, L - 37, sink + window + 1):
+        od, ld = O.decode(q[:, n - 1], k, v, n, sink, window, scale)
+        np.testing.assert_allclose(od, o[:, n - 1], rtol=0, atol=1e-12)
+        np.testing.assert_allclose(ld, lse[:, n - 1], rtol=0, atol=1e-12)
+
+
+def test_exact_window_backward_finite_differences():
+    rng = np.random.default_rng(6)
+    L, D = 192, 8
+    p = _exact(L, 64, 64, 64)
+    q, k, v, do = (rng.standard_normal((1, L, D)) for _ in range(4))
+    scale = 0.3
+    dQ, dK, dV, _, _ = O.attn_backward(q, k, v, do, p, scale)
+    f = lambda q_, k_, v_: float((O.attn_forward(q_, k_, v_, p, scale)[0] * do).sum())
+    eps = 1e-6
+    for arr, grad in ((q, dQ), (k, dK), (v, dV)):
+        for idx in [(0, 3, 1), (0, 100, 5), (0, 191, 7), (0, 64, 0)]:
+            a0 = arr[idx]
+            arr[idx] = a0 + eps; fp = f(q, k, v)
+            arr[idx] = a0 - eps; fm = f(q, k, v)
+            arr[idx] = a0
+            assert abs((fp - fm) / (2 * eps) - grad[idx]) < 1e-6
