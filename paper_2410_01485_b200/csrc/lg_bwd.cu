@@ -71,7 +71,7 @@ static lg_status launch_bwd_t(const Resolved& r, const WsLayout& w, const void* 
     if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, smem) != cudaSuccess)
       return LG_ERR_CUDA;
     dim3 grid(r.B * r.Hq, r.n_qtiles);
-    kern<<<grid, kBwdThreads, smem, stream>>>(tq, tk, tv, tdo, a);
+    kern<<<grid, kDqThreads, smem, stream>>>(tq, tk, tv, tdo, a);
     if (marks) cudaEventRecord(marks[3], stream);
   }
   return cudaGetLastError() == cudaSuccess ? LG_OK : LG_ERR_CUDA;

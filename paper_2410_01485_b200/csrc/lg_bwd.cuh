@@ -139,9 +139,17 @@ __device__ __forceinline__ void ew_publish(uint64_t* bar) {
 
 // ================================== dQ pass =================================================
 // TMEM columns: S[2] at 0 / 128 (dS of a step is written as bf16 over its own S), dP at 256,
-// dQ at 384.
+// dQ at 384.  Sixteen element-wise warps (four column groups of 32) and TWO issuing threads on
+// different scheduler partitions: thread A issues S and dQ (they alias the same columns, so their
+// order must stay with one thread), thread B issues dP (its only hazard is the element-wise read
+// of the previous dP, signalled by a barrier).  The two never have to wait for one another.
+constexpr int kDqEwWarps = 16;
+constexpr int kDqTmaWarp = 16, kDqMmaWarpA = 17, kDqMmaWarpB = 18;
+constexpr int kDqThreads = 19 * 32;
+constexpr int kDqCols = 128 / (kDqEwWarps / 4);   // columns of a step per element-wise thread
+
 template <int D, int BS>
-__global__ void __launch_bounds__(kBwdThreads, 1)
+__global__ void __launch_bounds__(kDqThreads, 1)
 bwd_dq_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUtensorMap tm_k,
               const __grid_constant__ CUtensorMap tm_v, const __grid_constant__ CUtensorMap tm_do,
               const BwdArgs a) {
@@ -150,7 +158,7 @@ bwd_dq_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ 
   constexpr uint32_t kColS = 0, kColDP = 256, kColDQ = 384;
   constexpr int kTile = SM::kTile;
   enum { B_FIX = 0, B_KF = 1, B_KE = 4, B_VF = 7, B_VE = 9, B_SF = 11, B_DPF = 13, B_DSF = 14, B_DONE = 15,
-         B_DRAIN = 16, B_DPR = 17, B_COUNT = 18 };
+         B_DRAIN = 16, B_DPR = 18, B_COUNT = 19 };
 
   extern __shared__ __align__(1024) uint8_t smem[];
   uint64_t* bars = reinterpret_cast<uint64_t*>(smem + SM::oBar);
@@ -175,15 +183,17 @@ bwd_dq_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ 
   if (tid == 0) {
     mbar_init(bars + B_FIX, 1);
     for (int i = 0; i < 3; ++i) { mbar_init(bars + B_KF + i, 1); mbar_init(bars + B_KE + i, 1); }
-    for (int i = 0; i < 2; ++i) { mbar_init(bars + B_VF + i, 1); mbar_init(bars + B_VE + i, 1); mbar_init(bars + B_SF + i, 1); }
+    for (int i = 0; i < 2; ++i) {
+      mbar_init(bars + B_VF + i, 1); mbar_init(bars + B_VE + i, 1); mbar_init(bars + B_SF + i, 1);
+      mbar_init(bars + B_DRAIN + i, 1);
+    }
     mbar_init(bars + B_DPF, 1);
-    mbar_init(bars + B_DSF, 8);
-    mbar_init(bars + B_DPR, 8);
+    mbar_init(bars + B_DSF, kDqEwWarps);
+    mbar_init(bars + B_DPR, kDqEwWarps);
     mbar_init(bars + B_DONE, 1);
-    mbar_init(bars + B_DRAIN, 1);
     mbar_fence_init();
   }
-  if (warp == 9) {
+  if (warp == kDqMmaWarpA) {
     tmem_alloc(tmem_slot, 512);
     tmem_relinquish();
   }
@@ -192,7 +202,7 @@ bwd_dq_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ 
   tc_fence_after();
   const uint32_t tmem = *tmem_slot;
 
-  if (warp == 8) {
+  if (warp == kDqTmaWarp) {
     // ------------------------------ TMA producer ------------------------------------------
     if (lane == 0) {
       tma_prefetch_desc(&tm_q); tma_prefetch_desc(&tm_k); tma_prefetch_desc(&tm_v); tma_prefetch_desc(&tm_do);
@@ -201,10 +211,15 @@ bwd_dq_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ 
       tma_load_rows<D, 128>(sDO, &tm_do, bars + B_FIX, 0, row0, h, b);
       bool ok = true;
       int nk = 0, nv = 0;   // loads started
+      int e_cur0 = n_steps > 0 ? ent[0] : 0, e_cur1 = (BS == 64 && n_ent > 1) ? ent[1] : e_cur0;
       for (int j = 0; j < n_steps; ++j) {
         const int sk = j % 3, sv = j & 1;
-        const int e0 = (BS == 128) ? j : 2 * j, e1 = min(2 * j + 1, n_ent - 1);
-        const int kb0 = ent[e0] >> 2, kb1 = (BS == 64) ? (ent[e1] >> 2) : 0;
+        const int kb0 = e_cur0 >> 2, kb1 = e_cur1 >> 2;
+        if (j + 1 < n_steps) {   // next step's entries: read now, used one step later
+          const int i0 = (BS == 128) ? j + 1 : 2 * j + 2;
+          e_cur0 = ent[i0];
+          e_cur1 = (BS == 64) ? ent[min(i0 + 1, n_ent - 1)] : e_cur0;
+        }
         if (j >= 3) ok = mbar_wait(bars + B_KE + sk, ((j / 3) - 1) & 1, a.error_word, 21);
         if (!ok) break;
         mbar_expect_tx(bars + B_KF + sk, kTile);
@@ -224,73 +239,82 @@ bwd_dq_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ 
       for (int j = max(nk - 3, 0); j < nk; ++j) mbar_wait(bars + B_KF + j % 3, (j / 3) & 1, a.error_word, 27);
       for (int j = max(nv - 2, 0); j < nv; ++j) mbar_wait(bars + B_VF + (j & 1), (j / 2) & 1, a.error_word, 28);
     }
-  } else if (warp == 9) {
-    // ------------------------------ MMA issuer --------------------------------------------
+  } else if (warp == kDqMmaWarpA) {
+    // ------------------------------ MMA issuer A: S and dQ ---------------------------------
     if (lane == 0) {
       constexpr uint32_t idesc_s = make_idesc_bf16(128, 128, 0, 0);
       constexpr uint32_t idesc_dq = make_idesc_bf16(128, D, 0, 1);
-      const uint32_t q_base = smem_u32(sQ), do_base = smem_u32(sDO), k_base = smem_u32(sK), v_base = smem_u32(sV);
+      const uint32_t hi = desc_hi(1024);
+      const uint32_t q_lo = desc_lo(smem_u32(sQ), 16), k_lo = desc_lo(smem_u32(sK), 16);
+      const uint32_t k_mn_lo = desc_lo(smem_u32(sK), BwdTile<D>::kBox);   // K tile as an MN-major operand
       bool ok = mbar_wait(bars + B_FIX, 0, a.error_word, 23);
       auto issue_s = [&](int j) {
         const int sk = j % 3;
         ok = ok && mbar_wait(bars + B_KF + sk, (j / 3) & 1, a.error_word, 24);
         if (ok) {
           tc_fence_after();
+          const uint32_t b_lo = k_lo + sk * (kTile >> 4), d_s = tmem + kColS + (j & 1) * 128;
 #pragma unroll
           for (int k = 0; k < D / 16; ++k) {
-            const uint32_t off = (k >> 2) * BwdTile<D>::kBox + (k & 3) * 32;
-            mma_ss(tmem + kColS + (j & 1) * 128, make_smem_desc(q_base + off, 16, 1024),
-                   make_smem_desc(k_base + sk * kTile + off, 16, 1024), idesc_s, k > 0);
+            constexpr int kB = BwdTile<D>::kBox >> 4;
+            const uint32_t off = (k >> 2) * kB + (k & 3) * 2;          // (bytes >> 4) of K slice k
+            mma_ss2(d_s, q_lo + off, b_lo + off, hi, idesc_s, k > 0);
           }
         }
         mma_commit(bars + B_SF + (j & 1));
       };
-      auto issue_dp = [&](int j) {
-        const int sv = j & 1;
-        ok = ok && mbar_wait(bars + B_VF + sv, (j / 2) & 1, a.error_word, 25);
-        if (ok) {
-          tc_fence_after();
+#pragma unroll 1
+      for (int j = -2; j < n_steps; ++j) {   // steps -2 and -1 only issue S(0) and S(1)
+        if (j >= 0) {
+          ok = ok && mbar_wait(bars + B_DSF, j & 1, a.error_word, 29);
+          if (ok) {
+            tc_fence_after();
+            const uint32_t b_lo = k_mn_lo + (j % 3) * (kTile >> 4), a_t = tmem + kColS + (j & 1) * 128;
 #pragma unroll
-          for (int k = 0; k < D / 16; ++k) {
-            const uint32_t off = (k >> 2) * BwdTile<D>::kBox + (k & 3) * 32;
-            mma_ss(tmem + kColDP, make_smem_desc(do_base + off, 16, 1024),
-                   make_smem_desc(v_base + sv * kTile + off, 16, 1024), idesc_s, k > 0);
+            for (int kk = 0; kk < 8; ++kk)
+              mma_ts2(tmem + kColDQ, a_t + (kk >> 1) * kDqCols + (kk & 1) * 8, b_lo + kk * (2048 >> 4), hi, idesc_dq,
+                      (j > 0) || (kk > 0));
           }
+          mma_commit(bars + B_KE + j % 3);
         }
-        mma_commit(bars + B_DPF);
-        mma_commit(bars + B_VE + sv);
-      };
-      if (n_steps > 0) {
-        issue_s(0);
-        issue_dp(0);
-        if (n_steps > 1) issue_s(1);
-      }
-      for (int j = 0; j < n_steps; ++j) {
-        // dP of the next step goes first: it only needs the dP columns to have been read, and it
-        // is what the element-wise warps wait for next; dQ of this step follows.
-        if (j + 1 < n_steps) {
-          ok = ok && mbar_wait(bars + B_DPR, j & 1, a.error_word, 34);
-          issue_dp(j + 1);
-        }
-        ok = ok && mbar_wait(bars + B_DSF, j & 1, a.error_word, 29);
-        if (ok) {
-          tc_fence_after();
-          const uint32_t kst = k_base + (j % 3) * kTile;
-#pragma unroll
-          for (int kk = 0; kk < 8; ++kk)
-            mma_ts(tmem + kColDQ, tmem + kColS + (j & 1) * 128 + (kk >> 2) * 64 + (kk & 3) * 8,
-                   make_smem_desc(kst + kk * 2048, BwdTile<D>::kBox, 1024), idesc_dq, (j > 0) || (kk > 0));
-        }
-        mma_commit(bars + B_KE + j % 3);
         if (j + 2 < n_steps) issue_s(j + 2);
       }
       mma_commit(bars + B_DONE);
       mma_commit(bars + B_DRAIN);
       mbar_wait(bars + B_DRAIN, 0, a.error_word, 30);   // nothing of ours is still running at exit
     }
+  } else if (warp == kDqMmaWarpB) {
+    // ------------------------------ MMA issuer B: dP ---------------------------------------
+    if (lane == 0) {
+      constexpr uint32_t idesc_s = make_idesc_bf16(128, 128, 0, 0);
+      const uint32_t hi = desc_hi(1024);
+      const uint32_t do_lo = desc_lo(smem_u32(sDO), 16), v_lo = desc_lo(smem_u32(sV), 16);
+      bool ok = mbar_wait(bars + B_FIX, 0, a.error_word, 35);
+#pragma unroll 1
+      for (int j = 0; j < n_steps; ++j) {
+        const int sv = j & 1;
+        if (j > 0) ok = ok && mbar_wait(bars + B_DPR, (j - 1) & 1, a.error_word, 34);   // dP(j-1) was read
+        ok = ok && mbar_wait(bars + B_VF + sv, (j / 2) & 1, a.error_word, 25);
+        if (ok) {
+          tc_fence_after();
+          const uint32_t b_lo = v_lo + sv * (kTile >> 4);
+#pragma unroll
+          for (int k = 0; k < D / 16; ++k) {
+            constexpr int kB = BwdTile<D>::kBox >> 4;
+            const uint32_t off = (k >> 2) * kB + (k & 3) * 2;
+            mma_ss2(tmem + kColDP, do_lo + off, b_lo + off, hi, idesc_s, k > 0);
+          }
+        }
+        mma_commit(bars + B_DPF);
+        mma_commit(bars + B_VE + sv);
+      }
+      mma_commit(bars + B_DRAIN + 1);
+      mbar_wait(bars + B_DRAIN + 1, 0, a.error_word, 36);
+    }
   } else {
     // ------------------------------ element-wise warps ------------------------------------
-    const int wg = warp >> 2;                               // column half
+    constexpr int C = kDqCols;
+    const int g = warp >> 2;                                // column group of C columns
     const int r = (warp & 3) * 32 + lane;                   // query row in the tile == TMEM lane
     const int qi = row0 + r;
     const int member = (R == 1) ? 0 : (r / BS);
@@ -301,59 +325,66 @@ bwd_dq_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ 
       lse2 = st.x;
       dlt = st.y;
     }
+    // entry of the step: read one step ahead so that the load is off the critical path
+    auto entry_of = [&](int j, bool& have) {
+      int e = (BS == 128) ? j : 2 * j + (g >> 1);
+      have = e < n_ent;
+      return ent[min(e, n_ent - 1)];
+    };
+    bool have = false, have_next = false;
+    int entry = n_steps > 0 ? entry_of(0, have) : 0;
     bool ok = true;
+#pragma unroll 1
     for (int j = 0; j < n_steps; ++j) {
-      // which keys do my 64 columns hold, and how many of them may this row see
-      int e = (BS == 128) ? j : 2 * j + wg;
-      const bool have = e < n_ent;
-      e = have ? e : n_ent - 1;
-      const int entry = ent[e];
-      const int key0 = (entry >> 2) * BS + (BS == 128 ? 64 * wg : 0);
+      const int entry_next = (j + 1 < n_steps) ? entry_of(j + 1, have_next) : 0;
+      // which keys do my C columns hold, and how many of them may this row see
+      const int key0 = (entry >> 2) * BS + (BS == 128 ? C * g : C * (g & 1));
       const bool on = have && ((entry >> member) & 1);
-      const int lim = on ? min(max(qi - key0 + 1, 0), 64) : 0;   // columns lo <= c < lim are visible
-      const int lo = (a.exact_w > 0 && (entry >> 2) >= a.ns) ? min(max(qi - a.exact_w + 1 - key0, 0), 64) : 0;
+      const int lim = on ? min(max(qi - key0 + 1, 0), C) : 0;   // columns lo <= c < lim are visible
+      const int lo = (a.exact_w > 0 && (entry >> 2) >= a.ns) ? min(max(qi - a.exact_w + 1 - key0, 0), C) : 0;
+      const uint32_t s_addr = lane_addr + kColS + (j & 1) * 128 + g * C;
 
       ok = mbar_wait(bars + B_SF + (j & 1), (j >> 1) & 1, a.error_word, 31);
       ok = __all_sync(0xffffffffu, ok);
       if (!ok) break;
       tc_fence_after();
-      float p[64];
+      float p[C];
       {
-        uint32_t sreg[64];
-        tmem_ld32(lane_addr + kColS + (j & 1) * 128 + wg * 64, sreg);
-        tmem_ld32(lane_addr + kColS + (j & 1) * 128 + wg * 64 + 32, sreg + 32);
+        uint32_t sreg[C];
+        tmem_ld32(s_addr, sreg);
         tmem_ld_wait();
-        if (__any_sync(0xffffffffu, lim < 64 || lo > 0)) {
+        if (__any_sync(0xffffffffu, lim < C || lo > 0)) {
 #pragma unroll
-          for (int c = 0; c < 64; ++c) {
+          for (int c = 0; c < C; ++c) {
             const float v = fast_exp2(fmaf(__uint_as_float(sreg[c]), a.scale_log2, -lse2));
             p[c] = (c < lim && c >= lo) ? v : 0.f;
           }
         } else {
 #pragma unroll
-          for (int c = 0; c < 64; ++c) p[c] = fast_exp2(fmaf(__uint_as_float(sreg[c]), a.scale_log2, -lse2));
+          for (int c = 0; c < C; ++c) p[c] = fast_exp2(fmaf(__uint_as_float(sreg[c]), a.scale_log2, -lse2));
         }
       }
       ok = mbar_wait(bars + B_DPF, j & 1, a.error_word, 32);
       ok = __all_sync(0xffffffffu, ok);
       if (!ok) break;
       tc_fence_after();
-      uint32_t dsreg[32];
+      uint32_t dsreg[C / 2];
       {
-        uint32_t dreg[64];
-        tmem_ld32(lane_addr + kColDP + wg * 64, dreg);
-        tmem_ld32(lane_addr + kColDP + wg * 64 + 32, dreg + 32);
+        uint32_t dreg[C];
+        tmem_ld32(lane_addr + kColDP + g * C, dreg);
         tmem_ld_wait();
         tc_fence_before();
         __syncwarp();
         if (lane == 0) mbar_arrive(bars + B_DPR);   // the dP columns may be overwritten
 #pragma unroll
-        for (int x = 0; x < 64; x += 2)
+        for (int x = 0; x < C; x += 2)
           dsreg[x >> 1] = pack_bf16(p[x] * (__uint_as_float(dreg[x]) - dlt),
                                     p[x + 1] * (__uint_as_float(dreg[x + 1]) - dlt));
       }
-      tmem_st32(lane_addr + kColS + (j & 1) * 128 + wg * 64, dsreg);   // dS over my own S columns
+      tmem_st16(s_addr, dsreg);   // dS over my own S columns
       ew_publish(bars + B_DSF);
+      entry = entry_next;
+      have = have_next;
     }
     // ---- epilogue: dQ * scale -> bf16 -------------------------------------------------------
     if (ok && n_steps > 0) {
@@ -362,20 +393,21 @@ bwd_dq_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ 
     }
     if (ok) {
       tc_fence_after();
-      if (qi < a.L) {   // warp-uniform: L is a multiple of 64
-        __nv_bfloat16* dq_row = a.out0 + b * a.s0[0] + h * a.s0[1] + static_cast<int64_t>(qi) * a.s0[2] + wg * (D / 2);
+      constexpr int kEpi = 32;                     // output columns per thread
+      if (qi < a.L && g * kEpi < D) {              // warp-uniform: L is a multiple of 64
+        __nv_bfloat16* dq_row = a.out0 + b * a.s0[0] + h * a.s0[1] + static_cast<int64_t>(qi) * a.s0[2] + g * kEpi;
         if (n_steps > 0) {
-          store_acc_cols<D / 2>(lane_addr + kColDQ + wg * (D / 2), dq_row, a.scale, true);
+          store_acc_cols<kEpi>(lane_addr + kColDQ + g * kEpi, dq_row, a.scale, true);
         } else {
 #pragma unroll
-          for (int x = 0; x < D / 2; x += 8) *reinterpret_cast<uint4*>(dq_row + x) = make_uint4(0, 0, 0, 0);
+          for (int x = 0; x < kEpi; x += 8) *reinterpret_cast<uint4*>(dq_row + x) = make_uint4(0, 0, 0, 0);
         }
       }
     }
   }
   tc_fence_before();
   __syncthreads();
-  if (warp == 9) tmem_dealloc(tmem, 512);
+  if (warp == kDqMmaWarpA) tmem_dealloc(tmem, 512);
 }
 
 // ============================== dK / dV pass ==================================================
