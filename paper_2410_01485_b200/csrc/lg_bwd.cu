@@ -49,7 +49,7 @@ static lg_status launch_bwd_t(const Resolved& r, const WsLayout& w, const void* 
     if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, smem) != cudaSuccess)
       return LG_ERR_CUDA;
     dim3 grid(r.B * r.Hkv, r.n_ktiles);
-    kern<<<grid, kBwdThreads, smem, stream>>>(tq, tk, tv, tdo, a);
+    kern<<<grid, kKvThreads, smem, stream>>>(tq, tk, tv, tdo, a);
     if (marks) cudaEventRecord(marks[2], stream);
   }
   // ---- dQ pass ------------------------------------------------------------------------

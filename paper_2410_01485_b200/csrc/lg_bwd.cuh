@@ -13,14 +13,16 @@
 //   * dQ pass: one CTA per tile of 128 queries of one head walks its CSR row(s):
 //     S = Q K^T, dP = dO V^T, dS over S, dQ += dS K.
 //
-// Both kernels are warp-specialised: warps 0-7 do the element-wise work (two groups of four
-// warps, each group owning 64 of the 128 columns of a step; thread = TMEM lane), warp 8
-// feeds shared memory with TMA, one thread of warp 9 issues every tcgen05.mma.  A step covers
-// 128 streamed rows: one 128-token pattern block, or two 64-token blocks side by side.  The
-// MMA order is chosen so that the tensor pipe always has independent work while the
-// exponentials of the current step are evaluated:
-//   dQ pass   : ... dQ(j-1) dP(j) S(j+1) | dQ(j) dP(j+1) S(j+2) ...      (S double-buffered)
-//   dK/dV pass: ... S(j) dK(j-1) dP(j) dV(j) | S(j+1) dK(j) dP(j+1) dV(j+1) ...
+// Both kernels are warp-specialised: warps 0-15 do the element-wise work (four groups of four
+// warps, each group owning 32 of the 128 columns of a step; thread = TMEM lane), warp 16
+// feeds shared memory with TMA, one thread each of warps 17 and 18 issues tcgen05.mma.  The two
+// issuing threads sit on different scheduler partitions of the SM: issuing an MMA is slowed by
+// fp32 arithmetic of other warps on the issuer's partition, and two queues halve what each has
+// to push through.  MMAs whose operands alias in tensor memory stay on one thread, so that the
+// queue order is the only synchronisation they need.  A step covers 128 streamed rows: one
+// 128-token pattern block, or two 64-token blocks side by side.
+//   dQ pass   : thread A: S(j+2) after dQ(j) (S double-buffered, dS over S)   thread B: dP(j)
+//   dK/dV pass: thread A: dV(j) then S^T(j+1) (P^T over S^T)     thread B: dK(j-1) then dP^T(j)
 #pragma once
 #include <cuda.h>
 #include "lg_common.cuh"
@@ -42,9 +44,6 @@ struct BwdArgs {
   int exact_w, ns;           // token-exact window (0: off) and number of sink blocks
   float scale, scale_log2;
 };
-
-constexpr int kBwdThreads = 320;     // 8 element-wise warps + TMA warp + MMA warp
-constexpr int kBwdEwThreads = 256;
 
 // ---- stat = (LSE * log2 e, rowsum(dO * O)) --------------------------------------------------
 template <int D>
@@ -163,7 +162,8 @@ bwd_dq_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ 
   extern __shared__ __align__(1024) uint8_t smem[];
   uint64_t* bars = reinterpret_cast<uint64_t*>(smem + SM::oBar);
   uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + B_COUNT);
-  const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+  const int tid = threadIdx.x, lane = tid & 31;
+  const int warp = __shfl_sync(0xffffffffu, tid >> 5, 0);   // same value, known to be warp-uniform
   if ((smem_u32(smem) & 1023u) != 0) {   // the swizzled tiles need 1024-byte alignment
     if (tid == 0) atomicCAS(a.error_word, 0u, (2u << 24) | 20u);
     return;
@@ -241,7 +241,10 @@ bwd_dq_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ 
     }
   } else if (warp == kDqMmaWarpA) {
     // ------------------------------ MMA issuer A: S and dQ ---------------------------------
-    if (lane == 0) {
+    {
+      // The whole warp runs the loop (so that addresses and descriptors stay warp-uniform values);
+      // one elected lane issues.
+      const bool lead = elect_one();
       constexpr uint32_t idesc_s = make_idesc_bf16(128, 128, 0, 0);
       constexpr uint32_t idesc_dq = make_idesc_bf16(128, D, 0, 1);
       const uint32_t hi = desc_hi(1024);
@@ -258,10 +261,10 @@ bwd_dq_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ 
           for (int k = 0; k < D / 16; ++k) {
             constexpr int kB = BwdTile<D>::kBox >> 4;
             const uint32_t off = (k >> 2) * kB + (k & 3) * 2;          // (bytes >> 4) of K slice k
-            mma_ss2(d_s, q_lo + off, b_lo + off, hi, idesc_s, k > 0);
+            if (lead) mma_ss2(d_s, q_lo + off, b_lo + off, hi, idesc_s, k > 0);
           }
         }
-        mma_commit(bars + B_SF + (j & 1));
+        if (lead) mma_commit(bars + B_SF + (j & 1));
       };
 #pragma unroll 1
       for (int j = -2; j < n_steps; ++j) {   // steps -2 and -1 only issue S(0) and S(1)
@@ -272,20 +275,20 @@ bwd_dq_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ 
             const uint32_t b_lo = k_mn_lo + (j % 3) * (kTile >> 4), a_t = tmem + kColS + (j & 1) * 128;
 #pragma unroll
             for (int kk = 0; kk < 8; ++kk)
-              mma_ts2(tmem + kColDQ, a_t + (kk >> 1) * kDqCols + (kk & 1) * 8, b_lo + kk * (2048 >> 4), hi, idesc_dq,
+              if (lead) mma_ts2(tmem + kColDQ, a_t + (kk >> 1) * kDqCols + (kk & 1) * 8, b_lo + kk * (2048 >> 4), hi, idesc_dq,
                       (j > 0) || (kk > 0));
           }
-          mma_commit(bars + B_KE + j % 3);
+          if (lead) mma_commit(bars + B_KE + j % 3);
         }
         if (j + 2 < n_steps) issue_s(j + 2);
       }
-      mma_commit(bars + B_DONE);
-      mma_commit(bars + B_DRAIN);
+      if (lead) { mma_commit(bars + B_DONE); mma_commit(bars + B_DRAIN); }
       mbar_wait(bars + B_DRAIN, 0, a.error_word, 30);   // nothing of ours is still running at exit
     }
   } else if (warp == kDqMmaWarpB) {
     // ------------------------------ MMA issuer B: dP ---------------------------------------
-    if (lane == 0) {
+    {
+      const bool lead = elect_one();
       constexpr uint32_t idesc_s = make_idesc_bf16(128, 128, 0, 0);
       const uint32_t hi = desc_hi(1024);
       const uint32_t do_lo = desc_lo(smem_u32(sDO), 16), v_lo = desc_lo(smem_u32(sV), 16);
@@ -302,13 +305,12 @@ bwd_dq_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ 
           for (int k = 0; k < D / 16; ++k) {
             constexpr int kB = BwdTile<D>::kBox >> 4;
             const uint32_t off = (k >> 2) * kB + (k & 3) * 2;
-            mma_ss2(tmem + kColDP, do_lo + off, b_lo + off, hi, idesc_s, k > 0);
+            if (lead) mma_ss2(tmem + kColDP, do_lo + off, b_lo + off, hi, idesc_s, k > 0);
           }
         }
-        mma_commit(bars + B_DPF);
-        mma_commit(bars + B_VE + sv);
+        if (lead) { mma_commit(bars + B_DPF); mma_commit(bars + B_VE + sv); }
       }
-      mma_commit(bars + B_DRAIN + 1);
+      if (lead) mma_commit(bars + B_DRAIN + 1);
       mbar_wait(bars + B_DRAIN + 1, 0, a.error_word, 36);
     }
   } else {
@@ -411,11 +413,23 @@ bwd_dq_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ 
 }
 
 // ============================== dK / dV pass ==================================================
-// TMEM columns: S^T at 0 (P^T written as bf16 over it), dP^T at 128 (dS^T over it), dV at 256,
-// dK at 384.  Items = (query head of the group, entry of the tile's CSC schedule) in a fixed
-// order; a step takes one item (128-token blocks) or two (64-token blocks).
+// Items = (query head of the group, entry of the tile's CSC schedule) in a fixed order; a step
+// streams 128 query rows (one item with 128-token blocks, two with 64-token blocks) and is
+// worked in two half-steps of 64 queries.  TMEM columns: S^T of the even / odd half-step at
+// 0 / 64 (P^T written as bf16 over it), dP^T at 128 / 192 (dS^T over it), dV at 256, dK at 384:
+// both score tiles are double-buffered, so the S^T of the next half-step is computed while the
+// exponentials of this one are evaluated.  Sixteen element-wise warps (four groups of 16
+// streamed queries) and two issuing threads on different scheduler partitions: thread A issues
+// S^T and dV (dV reads P^T from the S^T columns, so the S^T that overwrites them follows it in
+// the same queue), thread B issues dP^T and dK likewise.
+constexpr int kKvEwWarps = 16;
+constexpr int kKvTmaWarp = 16, kKvMmaWarpA = 17, kKvMmaWarpB = 18;
+constexpr int kKvThreads = 19 * 32;
+constexpr int kKvHalf = 64;                                // queries of a half-step
+constexpr int kKvCols = kKvHalf / (kKvEwWarps / 4);        // queries of a half-step per element-wise thread
+
 template <int D, int BS>
-__global__ void __launch_bounds__(kBwdThreads, 1)
+__global__ void __launch_bounds__(kKvThreads, 1)
 bwd_dkdv_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUtensorMap tm_k,
                 const __grid_constant__ CUtensorMap tm_v, const __grid_constant__ CUtensorMap tm_do,
                 const BwdArgs a) {
@@ -423,13 +437,15 @@ bwd_dkdv_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
   constexpr int R = 128 / BS;
   constexpr uint32_t kColS = 0, kColDP = 128, kColDV = 256, kColDK = 384;
   constexpr int kTile = SM::kTile;
-  enum { B_FIX = 0, B_QF = 1, B_QE = 4, B_OF = 7, B_OE = 9, B_SF = 11, B_DPF = 12, B_PF = 13, B_DSF = 14,
-         B_DONE = 15, B_DRAIN = 16, B_STF = 17, B_COUNT = 18 };
+  enum { B_FIX = 0, B_QF = 1, B_QE = 4, B_OF = 7, B_OE = 9, B_SF = 11, B_DPF = 13, B_PF = 15, B_DSF = 17,
+         B_DONE = 19, B_DRAIN = 20, B_STF = 22, B_STE = 24, B_COUNT = 26 };
 
   extern __shared__ __align__(1024) uint8_t smem[];
   uint64_t* bars = reinterpret_cast<uint64_t*>(smem + SM::oBar);
   uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + B_COUNT);
-  const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+  int32_t* sEnt = reinterpret_cast<int32_t*>(bars + B_COUNT + 1);   // [2][2]: entries of a step's items
+  const int tid = threadIdx.x, lane = tid & 31;
+  const int warp = __shfl_sync(0xffffffffu, tid >> 5, 0);   // same value, known to be warp-uniform
   if ((smem_u32(smem) & 1023u) != 0) {
     if (tid == 0) atomicCAS(a.error_word, 0u, (2u << 24) | 10u);
     return;
@@ -447,30 +463,30 @@ bwd_dkdv_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
   // key blocks of the tile's members (with 64-token blocks the two members need not be neighbours)
   const int kb_a = a.tile_cols[R * tile], kb_b = (R == 2) ? a.tile_cols[R * tile + 1] : -1;
   const int n_items = n_ent * a.G;
-  const int n_steps = (BS == 128) ? n_items : (n_items + 1) / 2;
+  const int n_hs = (BS == 128) ? 2 * n_items : n_items;    // half-steps
+  const int n_steps = (n_hs + 1) / 2;                      // 128-row tiles streamed
+  // half-step hs belongs to step hs >> 1 and is its last one when:
+  auto closes_step = [&](int hs) { return (hs & 1) || hs == n_hs - 1; };
 
-  // item -> (query head, first query row, entry)
-  auto item_of = [&](int it, int& hq, int& qrow, int& entry) {
-    const int g = it / n_ent, e = it - g * n_ent;
-    entry = ent[e];
-    hq = hk * a.G + g;
-    qrow = (entry >> 2) * BS;
-  };
 
   if (tid == 0) {
     mbar_init(bars + B_FIX, 1);
     for (int i = 0; i < 3; ++i) { mbar_init(bars + B_QF + i, 1); mbar_init(bars + B_QE + i, 1); }
-    for (int i = 0; i < 2; ++i) { mbar_init(bars + B_OF + i, 1); mbar_init(bars + B_OE + i, 1); }
-    mbar_init(bars + B_SF, 1);
-    mbar_init(bars + B_DPF, 1);
-    mbar_init(bars + B_PF, 8);
-    mbar_init(bars + B_DSF, 8);
-    mbar_init(bars + B_DONE, 1);
-    mbar_init(bars + B_DRAIN, 1);
-    mbar_init(bars + B_STF, 4);
+    for (int i = 0; i < 2; ++i) {
+      mbar_init(bars + B_OF + i, 1);
+      mbar_init(bars + B_OE + i, 2);      // dP^T (thread B) and dV (thread A) both read the dO tile
+      mbar_init(bars + B_SF + i, 1);
+      mbar_init(bars + B_DPF + i, 1);
+      mbar_init(bars + B_PF + i, kKvEwWarps);
+      mbar_init(bars + B_DSF + i, kKvEwWarps);
+      mbar_init(bars + B_DRAIN + i, 1);
+      mbar_init(bars + B_STF + i, 1);
+      mbar_init(bars + B_STE + i, kKvEwWarps);
+    }
+    mbar_init(bars + B_DONE, 2);          // the last dV and the last dK
     mbar_fence_init();
   }
-  if (warp == 9) {
+  if (warp == kKvMmaWarpA) {
     tmem_alloc(tmem_slot, 512);
     tmem_relinquish();
   }
@@ -479,7 +495,7 @@ bwd_dkdv_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
   tc_fence_after();
   const uint32_t tmem = *tmem_slot;
 
-  if (warp == 8) {
+  if (warp == kKvTmaWarp) {
     // ------------------------------ TMA producer ------------------------------------------
     if (lane == 0) {
       tma_prefetch_desc(&tm_q); tma_prefetch_desc(&tm_k); tma_prefetch_desc(&tm_v); tma_prefetch_desc(&tm_do);
@@ -490,13 +506,40 @@ bwd_dkdv_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
         tma_load_rows<D, BS>(sK, &tm_k, bars + B_FIX, 1, (kb_b >= 0 ? kb_b : kb_a) * BS, hk, b);
         tma_load_rows<D, BS>(sV, &tm_v, bars + B_FIX, 1, (kb_b >= 0 ? kb_b : kb_a) * BS, hk, b);
       }
+      // Besides the tiles, each step gets the softmax statistics of its 128 queries and the
+      // schedule entries of its items, so that the element-wise warps read neither global memory
+      // nor the schedule.  Items run query head by query head through the tile's entries.
       bool ok = true;
-      int nq = 0, no = 0;   // loads started
+      int nq = 0, no = 0, nst = 0;   // loads started
+      int grp = 0, e = 0;            // (query head within the group, entry) of the next item
+      auto next_item = [&](int& hq, int& qrow, int& entry) {
+        entry = ent[e];
+        hq = hk * a.G + grp;
+        qrow = (entry >> 2) * BS;
+        if (++e == n_ent) { e = 0; ++grp; }
+      };
       for (int j = 0; j < n_steps; ++j) {
         const int sq = j % 3, so = j & 1;
-        int h0, r0, e0, h1 = 0, r1 = 0, e1;
-        item_of(BS == 128 ? j : 2 * j, h0, r0, e0);
-        if (BS == 64) item_of(min(2 * j + 1, n_items - 1), h1, r1, e1);
+        int h0, r0, e0, h1, r1, e1;
+        next_item(h0, r0, e0);
+        h1 = h0; r1 = r0; e1 = e0;                              // a missing second item repeats the first
+        if (BS == 64 && 2 * j + 1 < n_items) next_item(h1, r1, e1);
+        if (j >= 2) ok = mbar_wait(bars + B_STE + so, ((j / 2) - 1) & 1, a.error_word, 40);
+        if (!ok) break;
+        sEnt[so * 2] = e0;
+        sEnt[so * 2 + 1] = e1;
+        mbar_expect_tx(bars + B_STF + so, 128 * 8);             // (release: publishes the entries as well)
+        {
+          const float2* st0 = a.stat + (static_cast<int64_t>(b) * a.Hq + h0) * a.L + r0;
+          const float2* st1 = a.stat + (static_cast<int64_t>(b) * a.Hq + h1) * a.L + r1;
+          if (BS == 128) {
+            bulk_load(sStat + so * 128, st0, 128 * 8, bars + B_STF + so);
+          } else {
+            bulk_load(sStat + so * 128, st0, 64 * 8, bars + B_STF + so);
+            bulk_load(sStat + so * 128 + 64, st1, 64 * 8, bars + B_STF + so);
+          }
+        }
+        nst = j + 1;
         if (j >= 3) ok = mbar_wait(bars + B_QE + sq, ((j / 3) - 1) & 1, a.error_word, 11);
         if (!ok) break;
         mbar_expect_tx(bars + B_QF + sq, kTile);
@@ -513,131 +556,146 @@ bwd_dkdv_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
       mbar_wait(bars + B_FIX, 0, a.error_word, 16);
       for (int j = max(nq - 3, 0); j < nq; ++j) mbar_wait(bars + B_QF + j % 3, (j / 3) & 1, a.error_word, 17);
       for (int j = max(no - 2, 0); j < no; ++j) mbar_wait(bars + B_OF + (j & 1), (j / 2) & 1, a.error_word, 18);
+      for (int j = max(nst - 2, 0); j < nst; ++j) mbar_wait(bars + B_STF + (j & 1), (j / 2) & 1, a.error_word, 41);
     }
-  } else if (warp == 9) {
-    // ------------------------------ MMA issuer --------------------------------------------
-    if (lane == 0) {
-      constexpr uint32_t idesc_st = make_idesc_bf16(128, 128, 0, 0);   // S^T, dP^T: N = streamed queries
-      constexpr uint32_t idesc_acc = make_idesc_bf16(128, D, 0, 1);    // dV, dK: B = dO / Q, MN-major
-      const uint32_t k_base = smem_u32(sK), v_base = smem_u32(sV), q_base = smem_u32(sQ), do_base = smem_u32(sDO);
+  } else if (warp == kKvMmaWarpA) {
+    // ------------------------------ MMA issuer A: S^T and dV -------------------------------
+    {
+      // The whole warp runs the loop (so that addresses and descriptors stay warp-uniform values);
+      // one elected lane issues.
+      const bool lead = elect_one();
+      constexpr uint32_t idesc_st = make_idesc_bf16(128, kKvHalf, 0, 0);   // S^T: N = queries of a half-step
+      constexpr uint32_t idesc_acc = make_idesc_bf16(128, D, 0, 1);        // dV: B = dO, MN-major
+      constexpr uint32_t kHalfRows = (kKvHalf * 128) >> 4;                 // 64 rows of a box, in 16-byte units
+      const uint32_t hi = desc_hi(1024);
+      const uint32_t k_lo = desc_lo(smem_u32(sK), 16), q_lo = desc_lo(smem_u32(sQ), 16);
+      const uint32_t do_mn_lo = desc_lo(smem_u32(sDO), BwdTile<D>::kBox);
       bool ok = mbar_wait(bars + B_FIX, 0, a.error_word, 13);
-      auto issue_s = [&](int j) {
-        const int sq = j % 3;
-        ok = ok && mbar_wait(bars + B_QF + sq, (j / 3) & 1, a.error_word, 14);
-        if (ok) {
-          tc_fence_after();
+#pragma unroll 1
+      for (int hs = -2; hs < n_hs; ++hs) {   // half-steps -2 and -1 only issue S^T(0) and S^T(1)
+        if (hs >= 0) {
+          const int j = hs >> 1, half = hs & 1, so = j & 1;
+          if (half == 0) ok = ok && mbar_wait(bars + B_OF + so, (j / 2) & 1, a.error_word, 19);
+          ok = ok && mbar_wait(bars + B_PF + half, j & 1, a.error_word, 9);
+          if (ok) {
+            tc_fence_after();
+            const uint32_t b_lo = do_mn_lo + so * (kTile >> 4) + half * 4 * (2048 >> 4);
+            const uint32_t a_t = tmem + kColS + half * kKvHalf;
 #pragma unroll
-          for (int k = 0; k < D / 16; ++k) {
-            const uint32_t off = (k >> 2) * BwdTile<D>::kBox + (k & 3) * 32;
-            mma_ss(tmem + kColS, make_smem_desc(k_base + off, 16, 1024),
-                   make_smem_desc(q_base + sq * kTile + off, 16, 1024), idesc_st, k > 0);
+            for (int kk = 0; kk < kKvHalf / 16; ++kk)
+              if (lead) mma_ts2(tmem + kColDV, a_t + kk * kKvCols, b_lo + kk * (2048 >> 4), hi, idesc_acc, (hs > 0) || (kk > 0));
           }
+          if (lead && closes_step(hs)) mma_commit(bars + B_OE + so);
         }
-        mma_commit(bars + B_SF);
-      };
-      auto issue_dk = [&](int j) {
-        ok = ok && mbar_wait(bars + B_DSF, j & 1, a.error_word, 15);
-        if (ok) {
-          tc_fence_after();
-          const uint32_t qst = q_base + (j % 3) * kTile;
+        const int hn = hs + 2;
+        if (hn < n_hs) {
+          const int j = hn >> 1, half = hn & 1, sq = j % 3;
+          if (half == 0) ok = ok && mbar_wait(bars + B_QF + sq, (j / 3) & 1, a.error_word, 14);
+          if (ok) {
+            tc_fence_after();
+            const uint32_t b_lo = q_lo + sq * (kTile >> 4) + half * kHalfRows;
 #pragma unroll
-          for (int kk = 0; kk < 8; ++kk)
-            mma_ts(tmem + kColDK, tmem + kColDP + (kk >> 2) * 64 + (kk & 3) * 8,
-                   make_smem_desc(qst + kk * 2048, BwdTile<D>::kBox, 1024), idesc_acc, (j > 0) || (kk > 0));
-        }
-        mma_commit(bars + B_QE + j % 3);
-      };
-      if (n_steps > 0) issue_s(0);
-      for (int j = 0; j < n_steps; ++j) {
-        const int so = j & 1;
-        if (j > 0) issue_dk(j - 1);
-        ok = ok && mbar_wait(bars + B_OF + so, (j / 2) & 1, a.error_word, 19);
-        if (ok) {
-          tc_fence_after();
-#pragma unroll
-          for (int k = 0; k < D / 16; ++k) {
-            const uint32_t off = (k >> 2) * BwdTile<D>::kBox + (k & 3) * 32;
-            mma_ss(tmem + kColDP, make_smem_desc(v_base + off, 16, 1024),
-                   make_smem_desc(do_base + so * kTile + off, 16, 1024), idesc_st, k > 0);
+            for (int k = 0; k < D / 16; ++k) {
+              constexpr int kB = BwdTile<D>::kBox >> 4;
+              const uint32_t off = (k >> 2) * kB + (k & 3) * 2;
+              if (lead) mma_ss2(tmem + kColS + half * kKvHalf, k_lo + off, b_lo + off, hi, idesc_st, k > 0);
+            }
           }
+          if (lead) mma_commit(bars + B_SF + half);
         }
-        mma_commit(bars + B_DPF);
-        ok = ok && mbar_wait(bars + B_PF, j & 1, a.error_word, 9);
-        if (ok) {
-          tc_fence_after();
-          const uint32_t ost = do_base + so * kTile;
-#pragma unroll
-          for (int kk = 0; kk < 8; ++kk)
-            mma_ts(tmem + kColDV, tmem + kColS + (kk >> 2) * 64 + (kk & 3) * 8,
-                   make_smem_desc(ost + kk * 2048, BwdTile<D>::kBox, 1024), idesc_acc, (j > 0) || (kk > 0));
-        }
-        mma_commit(bars + B_OE + so);
-        if (j + 1 < n_steps) issue_s(j + 1);
       }
-      if (n_steps > 0) issue_dk(n_steps - 1);
-      mma_commit(bars + B_DONE);
-      mma_commit(bars + B_DRAIN);
+      if (lead) { mma_commit(bars + B_DONE); mma_commit(bars + B_DRAIN); }
       mbar_wait(bars + B_DRAIN, 0, a.error_word, 8);
+    }
+  } else if (warp == kKvMmaWarpB) {
+    // ------------------------------ MMA issuer B: dP^T and dK ------------------------------
+    {
+      const bool lead = elect_one();
+      constexpr uint32_t idesc_st = make_idesc_bf16(128, kKvHalf, 0, 0);
+      constexpr uint32_t idesc_acc = make_idesc_bf16(128, D, 0, 1);        // dK: B = Q, MN-major
+      constexpr uint32_t kHalfRows = (kKvHalf * 128) >> 4;
+      const uint32_t hi = desc_hi(1024);
+      const uint32_t v_lo = desc_lo(smem_u32(sV), 16), do_lo = desc_lo(smem_u32(sDO), 16);
+      const uint32_t q_mn_lo = desc_lo(smem_u32(sQ), BwdTile<D>::kBox);
+      bool ok = mbar_wait(bars + B_FIX, 0, a.error_word, 5);
+#pragma unroll 1
+      for (int hs = -2; hs < n_hs; ++hs) {   // half-steps -2 and -1 only issue dP^T(0) and dP^T(1)
+        if (hs >= 0) {
+          const int j = hs >> 1, half = hs & 1, sq = j % 3;
+          ok = ok && mbar_wait(bars + B_DSF + half, j & 1, a.error_word, 15);
+          if (ok) {
+            tc_fence_after();
+            const uint32_t b_lo = q_mn_lo + sq * (kTile >> 4) + half * 4 * (2048 >> 4);
+            const uint32_t a_t = tmem + kColDP + half * kKvHalf;
+#pragma unroll
+            for (int kk = 0; kk < kKvHalf / 16; ++kk)
+              if (lead) mma_ts2(tmem + kColDK, a_t + kk * kKvCols, b_lo + kk * (2048 >> 4), hi, idesc_acc, (hs > 0) || (kk > 0));
+          }
+          if (lead && closes_step(hs)) mma_commit(bars + B_QE + sq);
+        }
+        const int hn = hs + 2;
+        if (hn < n_hs) {
+          const int j = hn >> 1, half = hn & 1, so = j & 1;
+          if (half == 0) ok = ok && mbar_wait(bars + B_OF + so, (j / 2) & 1, a.error_word, 6);
+          if (ok) {
+            tc_fence_after();
+            const uint32_t b_lo = do_lo + so * (kTile >> 4) + half * kHalfRows;
+#pragma unroll
+            for (int k = 0; k < D / 16; ++k) {
+              constexpr int kB = BwdTile<D>::kBox >> 4;
+              const uint32_t off = (k >> 2) * kB + (k & 3) * 2;
+              if (lead) mma_ss2(tmem + kColDP + half * kKvHalf, v_lo + off, b_lo + off, hi, idesc_st, k > 0);
+            }
+          }
+          if (lead) {
+            mma_commit(bars + B_DPF + half);
+            if (closes_step(hn)) mma_commit(bars + B_OE + so);
+          }
+        }
+      }
+      if (lead) { mma_commit(bars + B_DONE); mma_commit(bars + B_DRAIN + 1); }
+      mbar_wait(bars + B_DRAIN + 1, 0, a.error_word, 7);
     }
   } else {
     // ------------------------------ element-wise warps ------------------------------------
-    const int wg = warp >> 2;
+    constexpr int C = kKvCols;
+    const int g = warp >> 2;                                // group of C streamed queries
     const int r = (warp & 3) * 32 + lane;                   // key row in the tile == TMEM lane
     const int member = (R == 1) ? 0 : (r / BS);
     const int kb_mine = (R == 2 && member) ? kb_b : kb_a;
     const int kj = kb_mine * BS + (R == 2 ? (r & (BS - 1)) : r);   // this thread's key (kb_mine < 0: none)
     const uint32_t lane_addr = tmem + (static_cast<uint32_t>((warp & 3) * 32) << 16);
-    const int col = tid & 127;                              // the column whose statistics I fetch
-    auto fetch_stat = [&](int j) -> float2 {
-      if (tid >= 128 || j >= n_steps) return make_float2(0.f, 0.f);
-      int it = (BS == 128) ? j : 2 * j + (col >> 6);
-      it = min(it, n_items - 1);
-      int hq, qrow, entry;
-      item_of(it, hq, qrow, entry);
-      return a.stat[(static_cast<int64_t>(b) * a.Hq + hq) * a.L + qrow + (BS == 128 ? col : (col & 63))];
-    };
-    // Statistics of step j sit in sStat[j & 1]; warps 0-3 write those of step j + 1 at the end
-    // of step j (by then every warp has left step j - 1: the dP^T of step j is only issued after
-    // all eight warps published dS^T of step j - 1) and publish them through B_STF.
-    auto publish_stat = [&](int j, float2 v) {
-      if (warp < 4) {
-        sStat[(j & 1) * 128 + col] = v;
-        __syncwarp();
-        if (lane == 0) mbar_arrive(bars + B_STF);
-      }
-    };
-    publish_stat(0, fetch_stat(0));
     bool ok = true;
-    for (int j = 0; j < n_steps; ++j) {
-      const float2 nxt = fetch_stat(j + 1);
-      ok = mbar_wait(bars + B_STF, j & 1, a.error_word, 4);   // statistics of step j are in place
-      ok = __all_sync(0xffffffffu, ok);
-      if (!ok) break;
-      const float2* st = sStat + (j & 1) * 128 + wg * 64;
-      // which queries do my 64 columns hold, and from which of them on may this key be seen
-      int it = (BS == 128) ? j : 2 * j + wg;
-      const bool have = it < n_items;
-      it = have ? it : n_items - 1;
-      int hq, qrow, entry;
-      item_of(it, hq, qrow, entry);
-      const int q0 = qrow + (BS == 128 ? 64 * wg : 0);
-      const bool on = have && ((entry >> member) & 1);
-      const int xmin = on ? min(max(kj - q0, 0), 64) : 64;     // columns xmin <= c < xmax are visible
-      const int xmax = (a.exact_w > 0 && kb_mine >= a.ns) ? min(max(kj + a.exact_w - q0, 0), 64) : 64;
+#pragma unroll 1
+    for (int hs = 0; hs < n_hs; ++hs) {
+      const int j = hs >> 1, half = hs & 1;
+      if (half == 0) {
+        ok = mbar_wait(bars + B_STF + (j & 1), (j >> 1) & 1, a.error_word, 4);   // statistics and entries of step j
+        ok = __all_sync(0xffffffffu, ok);
+        if (!ok) break;
+      }
+      const float2* st = sStat + (j & 1) * 128 + half * kKvHalf + g * C;
+      // the queries my columns hold, and from which of them on this key may be seen
+      const int entry = sEnt[(j & 1) * 2 + (BS == 64 ? half : 0)];
+      const int q0 = (entry >> 2) * BS + (BS == 128 ? kKvHalf * half : 0) + C * g;
+      const bool on = (entry >> member) & 1;
+      const int xmin = on ? min(max(kj - q0, 0), C) : C;      // columns xmin <= c < xmax are visible
+      const int xmax = (a.exact_w > 0 && kb_mine >= a.ns) ? min(max(kj + a.exact_w - q0, 0), C) : C;
+      const uint32_t s_addr = lane_addr + kColS + half * kKvHalf + g * C;
+      const uint32_t dp_addr = lane_addr + kColDP + half * kKvHalf + g * C;
 
-      ok = mbar_wait(bars + B_SF, j & 1, a.error_word, 1);
+      ok = mbar_wait(bars + B_SF + half, j & 1, a.error_word, 1);
       ok = __all_sync(0xffffffffu, ok);
       if (!ok) break;
       tc_fence_after();
-      float p[64];
+      float p[C];
       {
-        uint32_t sreg[64];
-        tmem_ld32(lane_addr + kColS + wg * 64, sreg);
-        tmem_ld32(lane_addr + kColS + wg * 64 + 32, sreg + 32);
+        uint32_t sreg[C];
+        tmem_ld16(s_addr, sreg);
         tmem_ld_wait();
-        const bool masked = __any_sync(0xffffffffu, xmin > 0 || xmax < 64);
+        const bool masked = __any_sync(0xffffffffu, xmin > 0 || xmax < C);
 #pragma unroll
-        for (int c = 0; c < 64; c += 2) {
+        for (int c = 0; c < C; c += 2) {
           const float4 s2 = *reinterpret_cast<const float4*>(st + c);   // (lse2, delta) of two columns
           float v0 = fast_exp2(fmaf(__uint_as_float(sreg[c]), a.scale_log2, -s2.x));
           float v1 = fast_exp2(fmaf(__uint_as_float(sreg[c + 1]), a.scale_log2, -s2.z));
@@ -648,49 +706,52 @@ bwd_dkdv_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
           p[c] = v0;
           p[c + 1] = v1;
         }
-        uint32_t preg[32];
+        uint32_t preg[C / 2];
 #pragma unroll
-        for (int c = 0; c < 64; c += 2) preg[c >> 1] = pack_bf16(p[c], p[c + 1]);
-        tmem_st32(lane_addr + kColS + wg * 64, preg);        // P^T over my own S^T columns
-        ew_publish(bars + B_PF);
+        for (int c = 0; c < C; c += 2) preg[c >> 1] = pack_bf16(p[c], p[c + 1]);
+        tmem_st8(s_addr, preg);                               // P^T over my own S^T columns
+        ew_publish(bars + B_PF + half);
       }
-      ok = mbar_wait(bars + B_DPF, j & 1, a.error_word, 2);
+      ok = mbar_wait(bars + B_DPF + half, j & 1, a.error_word, 2);
       ok = __all_sync(0xffffffffu, ok);
       if (!ok) break;
       tc_fence_after();
-      uint32_t dsreg[32];
-#pragma unroll
-      for (int c = 0; c < 2; ++c) {
-        uint32_t dreg[32];
-        tmem_ld32(lane_addr + kColDP + wg * 64 + c * 32, dreg);
+      uint32_t dsreg[C / 2];
+      {
+        uint32_t dreg[C];
+        tmem_ld16(dp_addr, dreg);
         tmem_ld_wait();
 #pragma unroll
-        for (int x = 0; x < 32; x += 2) {
-          const float4 s2 = *reinterpret_cast<const float4*>(st + c * 32 + x);
-          dsreg[c * 16 + (x >> 1)] = pack_bf16(p[c * 32 + x] * (__uint_as_float(dreg[x]) - s2.y),
-                                               p[c * 32 + x + 1] * (__uint_as_float(dreg[x + 1]) - s2.w));
+        for (int x = 0; x < C; x += 2) {
+          const float4 s2 = *reinterpret_cast<const float4*>(st + x);
+          dsreg[x >> 1] = pack_bf16(p[x] * (__uint_as_float(dreg[x]) - s2.y),
+                                    p[x + 1] * (__uint_as_float(dreg[x + 1]) - s2.w));
         }
       }
-      tmem_st32(lane_addr + kColDP + wg * 64, dsreg);        // dS^T over my own dP^T columns
-      ew_publish(bars + B_DSF);
-      publish_stat(j + 1, nxt);
+      tmem_st8(dp_addr, dsreg);                               // dS^T over my own dP^T columns
+      ew_publish(bars + B_DSF + half);
+      if (closes_step(hs)) {   // this warp is done with the statistics of step j
+        __syncwarp();
+        if (lane == 0) mbar_arrive(bars + B_STE + (j & 1));
+      }
     }
     // ---- epilogue: dV, dK * scale -> bf16 ---------------------------------------------------
-    if (ok && n_steps > 0) {
+    if (ok && n_hs > 0) {
       ok = mbar_wait(bars + B_DONE, 0, a.error_word, 3);
       ok = __all_sync(0xffffffffu, ok);
     }
     if (ok) {
       tc_fence_after();
-      if (kb_mine >= 0) {
-        __nv_bfloat16* dk_row = a.out0 + b * a.s0[0] + hk * a.s0[1] + static_cast<int64_t>(kj) * a.s0[2] + wg * (D / 2);
-        __nv_bfloat16* dv_row = a.out1 + b * a.s1[0] + hk * a.s1[1] + static_cast<int64_t>(kj) * a.s1[2] + wg * (D / 2);
-        if (n_steps > 0) {
-          store_acc_cols<D / 2>(lane_addr + kColDV + wg * (D / 2), dv_row, 1.0f, true);
-          store_acc_cols<D / 2>(lane_addr + kColDK + wg * (D / 2), dk_row, a.scale, true);
+      constexpr int kEpi = 32;                               // output columns per thread
+      if (kb_mine >= 0 && g * kEpi < D) {
+        __nv_bfloat16* dk_row = a.out0 + b * a.s0[0] + hk * a.s0[1] + static_cast<int64_t>(kj) * a.s0[2] + g * kEpi;
+        __nv_bfloat16* dv_row = a.out1 + b * a.s1[0] + hk * a.s1[1] + static_cast<int64_t>(kj) * a.s1[2] + g * kEpi;
+        if (n_hs > 0) {
+          store_acc_cols<kEpi>(lane_addr + kColDV + g * kEpi, dv_row, 1.0f, true);
+          store_acc_cols<kEpi>(lane_addr + kColDK + g * kEpi, dk_row, a.scale, true);
         } else {
 #pragma unroll
-          for (int x = 0; x < D / 2; x += 8) {
+          for (int x = 0; x < kEpi; x += 8) {
             *reinterpret_cast<uint4*>(dk_row + x) = make_uint4(0, 0, 0, 0);
             *reinterpret_cast<uint4*>(dv_row + x) = make_uint4(0, 0, 0, 0);
           }
@@ -700,7 +761,7 @@ bwd_dkdv_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
   }
   tc_fence_before();
   __syncthreads();
-  if (warp == 9) tmem_dealloc(tmem, 512);
+  if (warp == kKvMmaWarpA) tmem_dealloc(tmem, 512);
 }
 
 }  // namespace lg
