@@ -35,7 +35,7 @@ struct BwdArgs {
   const int32_t* tile_cnt;
   const int32_t* tile_ent;   // idx * 4 + member mask
   const int32_t* order;
-  const float2* stat;        // [B, Hq, L]: (LSE * log2(e), delta)
+  const float2* stat;        // [B, Hq, L / 2] x (-LSE2 of rows 2i, 2i+1, -delta of rows 2i, 2i+1), LSE2 = LSE * log2(e)
   __nv_bfloat16* out0;       // dQ   | dK
   __nv_bfloat16* out1;       // unused | dV
   unsigned int* error_word;
@@ -45,7 +45,9 @@ struct BwdArgs {
   float scale, scale_log2;
 };
 
-// ---- stat = (LSE * log2 e, rowsum(dO * O)) --------------------------------------------------
+// ---- stat = -(LSE * log2 e) and -rowsum(dO * O), stored negated (they are only ever subtracted)
+// and with the rows paired, (a_2i, a_2i+1, b_2i, b_2i+1), so that two neighbouring rows feed one
+// packed fp32x2 instruction --------------------------------------------------------------------
 template <int D>
 __global__ void delta_kernel(const __nv_bfloat16* __restrict__ o, const __nv_bfloat16* __restrict__ d_o,
                              const float* __restrict__ lse, float2* __restrict__ stat, int64_t sb, int64_t sh,
@@ -73,7 +75,11 @@ __global__ void delta_kernel(const __nv_bfloat16* __restrict__ o, const __nv_bfl
   }
 #pragma unroll
   for (int s = TPR / 2; s > 0; s >>= 1) acc += __shfl_xor_sync(0xffffffffu, acc, s);
-  if (row < total_rows && ch == 0) stat[row] = make_float2(lse[row] * 1.4426950408889634f, acc);
+  if (row < total_rows && ch == 0) {
+    float* f = reinterpret_cast<float*>(stat) + (row >> 1) * 4 + (row & 1);
+    f[0] = -lse[row] * 1.4426950408889634f;
+    f[2] = -acc;
+  }
 }
 
 // Every tile in shared memory holds 128 rows of D bf16: D/64 column boxes of [128 rows x 128 B].
@@ -321,11 +327,12 @@ bwd_dq_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ 
     const int qi = row0 + r;
     const int member = (R == 1) ? 0 : (r / BS);
     const uint32_t lane_addr = tmem + (static_cast<uint32_t>((warp & 3) * 32) << 16);
-    float lse2 = 0.f, dlt = 0.f;
+    float nlse2 = 0.f, ndlt = 0.f;   // -LSE2 and -delta of my row
     if (qi < a.L) {
-      const float2 st = a.stat[(static_cast<int64_t>(b) * a.Hq + h) * a.L + qi];
-      lse2 = st.x;
-      dlt = st.y;
+      const int64_t row = (static_cast<int64_t>(b) * a.Hq + h) * a.L + qi;
+      const float* f = reinterpret_cast<const float*>(a.stat) + (row >> 1) * 4 + (row & 1);
+      nlse2 = f[0];
+      ndlt = f[2];
     }
     // entry of the step: read one step ahead so that the load is off the critical path
     auto entry_of = [&](int j, bool& have) {
@@ -358,12 +365,12 @@ bwd_dq_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ 
         if (__any_sync(0xffffffffu, lim < C || lo > 0)) {
 #pragma unroll
           for (int c = 0; c < C; ++c) {
-            const float v = fast_exp2(fmaf(__uint_as_float(sreg[c]), a.scale_log2, -lse2));
+            const float v = fast_exp2(fmaf(__uint_as_float(sreg[c]), a.scale_log2, nlse2));
             p[c] = (c < lim && c >= lo) ? v : 0.f;
           }
         } else {
 #pragma unroll
-          for (int c = 0; c < C; ++c) p[c] = fast_exp2(fmaf(__uint_as_float(sreg[c]), a.scale_log2, -lse2));
+          for (int c = 0; c < C; ++c) p[c] = fast_exp2(fmaf(__uint_as_float(sreg[c]), a.scale_log2, nlse2));
         }
       }
       ok = mbar_wait(bars + B_DPF, j & 1, a.error_word, 32);
@@ -380,8 +387,8 @@ bwd_dq_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ 
         if (lane == 0) mbar_arrive(bars + B_DPR);   // the dP columns may be overwritten
 #pragma unroll
         for (int x = 0; x < C; x += 2)
-          dsreg[x >> 1] = pack_bf16(p[x] * (__uint_as_float(dreg[x]) - dlt),
-                                    p[x + 1] * (__uint_as_float(dreg[x + 1]) - dlt));
+          dsreg[x >> 1] = pack_bf16(p[x] * (__uint_as_float(dreg[x]) + ndlt),
+                                    p[x + 1] * (__uint_as_float(dreg[x + 1]) + ndlt));
       }
       tmem_st16(s_addr, dsreg);   // dS over my own S columns
       ew_publish(bars + B_DSF);
@@ -422,9 +429,12 @@ bwd_dq_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ 
 // streamed queries) and two issuing threads on different scheduler partitions: thread A issues
 // S^T and dV (dV reads P^T from the S^T columns, so the S^T that overwrites them follows it in
 // the same queue), thread B issues dP^T and dK likewise.
-constexpr int kKvEwWarps = 16;
-constexpr int kKvTmaWarp = 16, kKvMmaWarpA = 17, kKvMmaWarpB = 18;
-constexpr int kKvThreads = 19 * 32;
+#ifndef LG_KV_EW_WARPS
+#define LG_KV_EW_WARPS 16
+#endif
+constexpr int kKvEwWarps = LG_KV_EW_WARPS;
+constexpr int kKvTmaWarp = kKvEwWarps, kKvMmaWarpA = kKvEwWarps + 1, kKvMmaWarpB = kKvEwWarps + 2;
+constexpr int kKvThreads = (kKvEwWarps + 3) * 32;
 constexpr int kKvHalf = 64;                                // queries of a half-step
 constexpr int kKvCols = kKvHalf / (kKvEwWarps / 4);        // queries of a half-step per element-wise thread
 
@@ -583,7 +593,7 @@ bwd_dkdv_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
             const uint32_t a_t = tmem + kColS + half * kKvHalf;
 #pragma unroll
             for (int kk = 0; kk < kKvHalf / 16; ++kk)
-              if (lead) mma_ts2(tmem + kColDV, a_t + kk * kKvCols, b_lo + kk * (2048 >> 4), hi, idesc_acc, (hs > 0) || (kk > 0));
+              if (lead) mma_ts2(tmem + kColDV, a_t + (kk * 16 / kKvCols) * kKvCols + (kk * 16 % kKvCols) / 2, b_lo + kk * (2048 >> 4), hi, idesc_acc, (hs > 0) || (kk > 0));
           }
           if (lead && closes_step(hs)) mma_commit(bars + B_OE + so);
         }
@@ -629,7 +639,7 @@ bwd_dkdv_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
             const uint32_t a_t = tmem + kColDP + half * kKvHalf;
 #pragma unroll
             for (int kk = 0; kk < kKvHalf / 16; ++kk)
-              if (lead) mma_ts2(tmem + kColDK, a_t + kk * kKvCols, b_lo + kk * (2048 >> 4), hi, idesc_acc, (hs > 0) || (kk > 0));
+              if (lead) mma_ts2(tmem + kColDK, a_t + (kk * 16 / kKvCols) * kKvCols + (kk * 16 % kKvCols) / 2, b_lo + kk * (2048 >> 4), hi, idesc_acc, (hs > 0) || (kk > 0));
           }
           if (lead && closes_step(hs)) mma_commit(bars + B_QE + sq);
         }
@@ -665,6 +675,7 @@ bwd_dkdv_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
     const int kb_mine = (R == 2 && member) ? kb_b : kb_a;
     const int kj = kb_mine * BS + (R == 2 ? (r & (BS - 1)) : r);   // this thread's key (kb_mine < 0: none)
     const uint32_t lane_addr = tmem + (static_cast<uint32_t>((warp & 3) * 32) << 16);
+    const uint64_t scale2 = f32x2(a.scale_log2, a.scale_log2);
     bool ok = true;
 #pragma unroll 1
     for (int hs = 0; hs < n_hs; ++hs) {
@@ -674,7 +685,8 @@ bwd_dkdv_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
         ok = __all_sync(0xffffffffu, ok);
         if (!ok) break;
       }
-      const float2* st = sStat + (j & 1) * 128 + half * kKvHalf + g * C;
+      // (-LSE2_c, -LSE2_c+1, -delta_c, -delta_c+1) of my column pairs
+      const float4* st = reinterpret_cast<const float4*>(sStat + (j & 1) * 128 + half * kKvHalf + g * C);
       // the queries my columns hold, and from which of them on this key may be seen
       const int entry = sEnt[(j & 1) * 2 + (BS == 64 ? half : 0)];
       const int q0 = (entry >> 2) * BS + (BS == 128 ? kKvHalf * half : 0) + C * g;
@@ -691,14 +703,16 @@ bwd_dkdv_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
       float p[C];
       {
         uint32_t sreg[C];
-        tmem_ld16(s_addr, sreg);
+        if constexpr (C == 16) tmem_ld16(s_addr, sreg); else tmem_ld32(s_addr, sreg);
         tmem_ld_wait();
         const bool masked = __any_sync(0xffffffffu, xmin > 0 || xmax < C);
 #pragma unroll
         for (int c = 0; c < C; c += 2) {
-          const float4 s2 = *reinterpret_cast<const float4*>(st + c);   // (lse2, delta) of two columns
-          float v0 = fast_exp2(fmaf(__uint_as_float(sreg[c]), a.scale_log2, -s2.x));
-          float v1 = fast_exp2(fmaf(__uint_as_float(sreg[c + 1]), a.scale_log2, -s2.z));
+          const float4 s4 = st[c >> 1];
+          float x0, x1;
+          f32x2_split(fma_f32x2(f32x2(__uint_as_float(sreg[c]), __uint_as_float(sreg[c + 1])), scale2,
+                                f32x2(s4.x, s4.y)), x0, x1);
+          float v0 = fast_exp2(x0), v1 = fast_exp2(x1);
           if (masked) {
             v0 = (c >= xmin && c < xmax) ? v0 : 0.f;
             v1 = (c + 1 >= xmin && c + 1 < xmax) ? v1 : 0.f;
@@ -709,7 +723,7 @@ bwd_dkdv_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
         uint32_t preg[C / 2];
 #pragma unroll
         for (int c = 0; c < C; c += 2) preg[c >> 1] = pack_bf16(p[c], p[c + 1]);
-        tmem_st8(s_addr, preg);                               // P^T over my own S^T columns
+        if constexpr (C == 16) tmem_st8(s_addr, preg); else tmem_st16(s_addr, preg);                               // P^T over my own S^T columns
         ew_publish(bars + B_PF + half);
       }
       ok = mbar_wait(bars + B_DPF + half, j & 1, a.error_word, 2);
@@ -719,16 +733,19 @@ bwd_dkdv_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
       uint32_t dsreg[C / 2];
       {
         uint32_t dreg[C];
-        tmem_ld16(dp_addr, dreg);
+        if constexpr (C == 16) tmem_ld16(dp_addr, dreg); else tmem_ld32(dp_addr, dreg);
         tmem_ld_wait();
 #pragma unroll
         for (int x = 0; x < C; x += 2) {
-          const float4 s2 = *reinterpret_cast<const float4*>(st + x);
-          dsreg[x >> 1] = pack_bf16(p[x] * (__uint_as_float(dreg[x]) - s2.y),
-                                    p[x + 1] * (__uint_as_float(dreg[x + 1]) - s2.w));
+          const float4 s4 = st[x >> 1];
+          float d0, d1;
+          f32x2_split(mul_f32x2(f32x2(p[x], p[x + 1]),
+                                add_f32x2(f32x2(__uint_as_float(dreg[x]), __uint_as_float(dreg[x + 1])),
+                                          f32x2(s4.z, s4.w))), d0, d1);
+          dsreg[x >> 1] = pack_bf16(d0, d1);
         }
       }
-      tmem_st8(dp_addr, dsreg);                               // dS^T over my own dP^T columns
+      if constexpr (C == 16) tmem_st8(dp_addr, dsreg); else tmem_st16(dp_addr, dsreg);                               // dS^T over my own dP^T columns
       ew_publish(bars + B_DSF + half);
       if (closes_step(hs)) {   // this warp is done with the statistics of step j
         __syncwarp();
