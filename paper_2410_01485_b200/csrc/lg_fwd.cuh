@@ -4,16 +4,20 @@
 // One CTA owns a super-tile of 256 query rows of one head: two tiles ("slots") of 128 rows
 // that share every K / V tile brought into shared memory.  It walks the ascending union of
 // the slots' active KV blocks in steps of 128 keys (one 128-token block, or two 64-token
-// blocks side by side); a slot that has nothing in a step skips it.  Roles:
+// blocks side by side), each step in two halves of 64 keys; a slot skips the halves none of
+// its rows can see.  Roles:
 //   warps 0-3 / 4-7 : softmax of slot 0 / 1 (thread = query row = TMEM lane)
 //   warp 8          : TMA producer (Q once, then the K and V rings)
-//   warp 9, lane 0  : issues every tcgen05.mma
-// Tensor memory: S of slot s at columns 128 s (P is written as bf16 over its first 64
-// columns), O of slot s at 256 + 128 s.  MMA order
-//   S0(0) S1(0) | PV0(0) S0(1) PV1(0) S1(1) | PV0(1) S0(2) PV1(1) S1(2) | ...
-// so that while one slot's softmax runs, the tensor pipe works on the other slot.
-// The running maximum is only raised (and O rescaled) when it grew by more than 2^8; until
-// then probabilities are expressed relative to the older maximum, which fp32 / bf16 hold easily.
+//   warps 9 / 10    : issue the tcgen05.mma of slot 0 / 1 (warp-uniform code, one elected lane;
+//                     the two warps sit on different scheduler partitions of the SM)
+// Tensor memory: S of slot s, half h at columns 128 s + 64 h (P is written as bf16 over the
+// first 32 of them), O of slot s at 256 + 128 s.  Per slot the issue order is
+//   S_0(0) S_1(0) | PV_0(0) S_0(1) | PV_1(0) S_1(1) | PV_0(1) S_0(2) | ...
+// so the two halves of a slot form a double buffer: while the softmax works on one half the
+// tensor pipe computes the other, and the second slot fills what is left.  The online softmax
+// advances half by half.  The running maximum is only raised (and O rescaled) when it grew by
+// more than 2^8; until then probabilities are expressed relative to the older maximum, which
+// fp32 / bf16 hold easily.
 #pragma once
 #include <cuda.h>
 #include "lg_common.cuh"
@@ -34,8 +38,13 @@ struct FwdArgs {
   float scale_log2;          // scale * log2(e)
 };
 
-constexpr int kFwdThreads = 320;
+constexpr int kFwdTmaWarp = 8, kFwdMmaWarp0 = 9;
+constexpr int kFwdThreads = 11 * 32;
 constexpr float kFwdRescaleThreshold = 8.0f;   // log2 units
+// Of every 8 exponentials, this many are evaluated on the FMA pipe instead of the exponential unit.
+#ifndef LG_FWD_POLY
+#define LG_FWD_POLY 0
+#endif
 
 template <int D>
 struct FwdSmem {
@@ -59,12 +68,17 @@ fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUt
   constexpr uint32_t kSlotMask = (1u << RS) - 1u;
   constexpr int kTile = SM::kTile;
   constexpr uint32_t kColS = 0, kColO = 256;
-  enum { B_Q = 0, B_KF = 1, B_KE = 4, B_VF = 7, B_VE = 9, B_SF = 11, B_PF = 13, B_OD = 15, B_DRAIN = 17, B_COUNT = 18 };
+  // SF / PF / OD are indexed [slot * 2 + half].  A parity wait is only meaningful while the barrier
+  // is at most one phase behind the waiter; per half buffer that holds by construction (the S
+  // product that re-fills a half is queued behind the P V product that read it), which is why
+  // "O is complete" is tracked per half as well.
+  enum { B_Q = 0, B_KF = 1, B_KE = 4, B_VF = 7, B_VE = 9, B_SF = 11, B_PF = 15, B_OD = 19, B_DRAIN = 23, B_COUNT = 25 };
 
   extern __shared__ __align__(1024) uint8_t smem[];
   uint64_t* bars = reinterpret_cast<uint64_t*>(smem + SM::oBar);
   uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + B_COUNT);
-  const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+  const int tid = threadIdx.x, lane = tid & 31;
+  const int warp = __shfl_sync(0xffffffffu, tid >> 5, 0);   // same value, known to be warp-uniform
   if ((smem_u32(smem) & 1023u) != 0) {   // the swizzled tiles need 1024-byte alignment
     if (tid == 0) atomicCAS(a.error_word, 0u, (2u << 24) | 1u);
     return;
@@ -80,26 +94,25 @@ fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUt
   const int row0 = tile * 256;
   const int n_steps = (BS == 128) ? n_ent : (n_ent + 1) / 2;
 
-  // union of the member masks of the blocks of step j (0 past the end)
-  auto step_mask = [&](int j) -> uint32_t {
-    if (j >= n_steps) return 0u;
-    if (BS == 128) return static_cast<uint32_t>(ent[j]) & 15u;
-    const uint32_t m0 = static_cast<uint32_t>(ent[2 * j]) & 15u;
-    const uint32_t m1 = (2 * j + 1 < n_ent) ? (static_cast<uint32_t>(ent[2 * j + 1]) & 15u) : 0u;
-    return m0 | m1;
+  // entries of the two halves of step j (0: nobody's member, also past the end)
+  auto load_ent = [&](int j, int& e0, int& e1) {
+    if (j >= n_steps) { e0 = e1 = 0; return; }
+    if (BS == 128) { e0 = e1 = ent[j]; return; }
+    e0 = ent[2 * j];
+    e1 = (2 * j + 1 < n_ent) ? ent[2 * j + 1] : 0;   // odd tail: no second block
   };
 
   if (tid == 0) {
     mbar_init(bars + B_Q, 1);
-    for (int i = 0; i < 3; ++i) { mbar_init(bars + B_KF + i, 1); mbar_init(bars + B_KE + i, 1); }
+    for (int i = 0; i < 3; ++i) { mbar_init(bars + B_KF + i, 1); mbar_init(bars + B_KE + i, 2); }   // both issuers release
     for (int i = 0; i < 2; ++i) {
-      mbar_init(bars + B_VF + i, 1); mbar_init(bars + B_VE + i, 1);
-      mbar_init(bars + B_SF + i, 1); mbar_init(bars + B_PF + i, 4); mbar_init(bars + B_OD + i, 1);
+      mbar_init(bars + B_VF + i, 1); mbar_init(bars + B_VE + i, 2);
+      mbar_init(bars + B_DRAIN + i, 1);
     }
-    mbar_init(bars + B_DRAIN, 1);
+    for (int i = 0; i < 4; ++i) { mbar_init(bars + B_SF + i, 1); mbar_init(bars + B_PF + i, 4); mbar_init(bars + B_OD + i, 1); }
     mbar_fence_init();
   }
-  if (warp == 9) {
+  if (warp == kFwdMmaWarp0) {
     tmem_alloc(tmem_slot, 512);
     tmem_relinquish();
   }
@@ -108,7 +121,7 @@ fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUt
   tc_fence_after();
   const uint32_t tmem = *tmem_slot;
 
-  if (warp == 8) {
+  if (warp == kFwdTmaWarp) {
     // ------------------------------ TMA producer ------------------------------------------
     if (lane == 0) {
       tma_prefetch_desc(&tm_q); tma_prefetch_desc(&tm_k); tma_prefetch_desc(&tm_v);
@@ -152,81 +165,78 @@ fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUt
       for (int j = max(nk - 3, 0); j < nk; ++j) mbar_wait(bars + B_KF + j % 3, (j / 3) & 1, a.error_word, 5);
       for (int j = max(nv - 2, 0); j < nv; ++j) mbar_wait(bars + B_VF + (j & 1), (j / 2) & 1, a.error_word, 6);
     }
-  } else if (warp == 9) {
-    // ------------------------------ MMA issuer --------------------------------------------
-    if (lane == 0) {
-      constexpr uint32_t idesc_s = make_idesc_bf16(128, 128, 0, 0);
-      constexpr uint32_t idesc_o = make_idesc_bf16(128, D, 0, 1);
-      const uint32_t hi = desc_hi(1024);
-      const uint32_t q_lo = desc_lo(smem_u32(sQ), 16), k_lo = desc_lo(smem_u32(sK), 16);
-      const uint32_t v_mn_lo = desc_lo(smem_u32(sV), SM::kBox);
-      bool ok = mbar_wait(bars + B_Q, 0, a.error_word, 7);
-      int k_ready = -1, v_ready = -1;           // last step whose K / V tile this thread has seen complete
-      int n_pv0 = 0, n_pv1 = 0;                 // P V products issued per slot (accumulate flag, barrier phases)
-      auto issue_s = [&](int s, int j) {
-        const int sk = j % 3;
-        if (k_ready < j) {
-          ok = ok && mbar_wait(bars + B_KF + sk, (j / 3) & 1, a.error_word, 8);
-          k_ready = j;
-        }
-        if (ok) {
-          tc_fence_after();
-          const uint32_t a_lo = q_lo + s * (kTile >> 4), b_lo = k_lo + sk * (kTile >> 4);
-#pragma unroll
-          for (int k = 0; k < D / 16; ++k) {
-            constexpr int kB = SM::kBox >> 4;
-            const uint32_t off = (k >> 2) * kB + (k & 3) * 2;
-            mma_ss2(tmem + kColS + s * 128, a_lo + off, b_lo + off, hi, idesc_s, k > 0);
-          }
-        }
-        mma_commit(bars + B_SF + s);
-      };
-      auto issue_pv = [&](int s, int j) {
-        const int sv = j & 1;
-        if (v_ready < j) {
-          ok = ok && mbar_wait(bars + B_VF + sv, (j / 2) & 1, a.error_word, 9);
-          v_ready = j;
-        }
-        const int n_pv = s ? n_pv1 : n_pv0;
-        ok = ok && mbar_wait(bars + B_PF + s, n_pv & 1, a.error_word, 10);
-        if (ok) {
-          tc_fence_after();
-          const uint32_t b_lo = v_mn_lo + sv * (kTile >> 4);
-#pragma unroll
-          for (int kk = 0; kk < 8; ++kk)
-            mma_ts2(tmem + kColO + s * 128, tmem + kColS + s * 128 + kk * 8, b_lo + kk * (2048 >> 4), hi, idesc_o,
-                    (n_pv > 0) || (kk > 0));
-        }
-        if (s) ++n_pv1; else ++n_pv0;
-        mma_commit(bars + B_OD + s);
-      };
-      // One loop body issues everything (step -1 only issues the S products of step 0): the
-      // code of this thread must stay small, it competes for the instruction caches with the
-      // softmax warps and every fetch miss is time the tensor pipe sits idle.
-      uint32_t m_cur = 0u, m_nxt = step_mask(0);
+  } else if (warp == kFwdMmaWarp0 || warp == kFwdMmaWarp0 + 1) {
+    // ------------------------------ MMA issuer of one slot --------------------------------
+    // The whole warp runs the loop (addresses and descriptors stay warp-uniform values); one
+    // elected lane issues.  Both issuers arrive once per step on the K / V "empty" barriers,
+    // whether or not their slot used the step, and only after having seen the step's tile
+    // arrive: an idle issuer can then never be a whole ring turn ahead of the other one.
+    const int s = warp - kFwdMmaWarp0;
+    const bool lead = elect_one();
+    constexpr uint32_t idesc_s = make_idesc_bf16(128, 64, 0, 0);
+    constexpr uint32_t idesc_o = make_idesc_bf16(128, D, 0, 1);
+    constexpr uint32_t kHalfRows = (64 * 128) >> 4;   // 64 rows of a box, in 16-byte units
+    const uint32_t hi = desc_hi(1024);
+    const uint32_t q_lo = desc_lo(smem_u32(sQ), 16) + s * (kTile >> 4), k_lo = desc_lo(smem_u32(sK), 16);
+    const uint32_t v_mn_lo = desc_lo(smem_u32(sV), SM::kBox);
+    const uint32_t t_s = tmem + kColS + s * 128, t_o = tmem + kColO + s * 128;
+    bool ok = mbar_wait(bars + B_Q, 0, a.error_word, 7);
+    int n_pv = 0;                 // P V products issued (accumulate flag)
+    int pf0 = 0, pf1 = 0;         // uses of the two half buffers whose P V product was issued (barrier phases)
+    int ce0 = 0, ce1 = 0, ne0, ne1, nn0, nn1;
+    load_ent(0, ne0, ne1);
+    load_ent(1, nn0, nn1);
 #pragma unroll 1
-      for (int j = -1; j < n_steps; ++j) {
-        const uint32_t m_nxt2 = step_mask(j + 2);   // read ahead: off the critical path
-#pragma unroll 1
-        for (int s = 0; s < 2; ++s) {
-          const bool cur = (m_cur >> (s * RS)) & kSlotMask, nxt = (m_nxt >> (s * RS)) & kSlotMask;
-          const bool cur_other_later = (s == 0) && ((m_cur >> RS) & kSlotMask);   // slot 1 still needs V(j)
-          const bool nxt_other_later = (s == 0) && ((m_nxt >> RS) & kSlotMask);   // slot 1 still needs K(j+1)
-          if (cur) {
-            issue_pv(s, j);
-            if (!cur_other_later) mma_commit(bars + B_VE + (j & 1));
+    for (int j = -1; j < n_steps; ++j) {   // step -1 only issues the S products of step 0
+      bool v_seen = false, k_seen = false;
+#pragma unroll
+      for (int hf = 0; hf < 2; ++hf) {
+        const int ce = hf ? ce1 : ce0, ne = hf ? ne1 : ne0;
+        if ((static_cast<uint32_t>(ce) >> (s * RS)) & kSlotMask) {           // P V of half hf of step j
+          const int sv = j & 1;
+          if (!v_seen) { ok = ok && mbar_wait(bars + B_VF + sv, (j / 2) & 1, a.error_word, 9); v_seen = true; }
+          ok = ok && mbar_wait(bars + B_PF + s * 2 + hf, (hf ? pf1 : pf0) & 1, a.error_word, 10);
+          if (ok) {
+            tc_fence_after();
+            const uint32_t b_lo = v_mn_lo + sv * (kTile >> 4) + hf * 4 * (2048 >> 4);
+#pragma unroll
+            for (int kk = 0; kk < 4; ++kk)
+              if (lead) mma_ts2(t_o, t_s + hf * 64 + kk * 8, b_lo + kk * (2048 >> 4), hi, idesc_o, (n_pv > 0) || (kk > 0));
           }
-          if (nxt) {
-            issue_s(s, j + 1);
-            if (!nxt_other_later) mma_commit(bars + B_KE + (j + 1) % 3);
-          }
+          if (lead) mma_commit(bars + B_OD + s * 2 + hf);
+          ++n_pv;
+          if (hf) ++pf1; else ++pf0;
         }
-        m_cur = m_nxt;
-        m_nxt = m_nxt2;
+        if (hf == 1 && j >= 0) {
+          if (!v_seen) ok = ok && mbar_wait(bars + B_VF + (j & 1), (j / 2) & 1, a.error_word, 9);
+          if (lead) mma_commit(bars + B_VE + (j & 1));
+        }
+        if ((static_cast<uint32_t>(ne) >> (s * RS)) & kSlotMask) {           // S of half hf of step j + 1
+          const int sk = (j + 1) % 3;
+          if (!k_seen) { ok = ok && mbar_wait(bars + B_KF + sk, ((j + 1) / 3) & 1, a.error_word, 8); k_seen = true; }
+          if (ok) {
+            tc_fence_after();
+            const uint32_t b_lo = k_lo + sk * (kTile >> 4) + hf * kHalfRows;
+#pragma unroll
+            for (int k = 0; k < D / 16; ++k) {
+              constexpr int kB = SM::kBox >> 4;
+              const uint32_t off = (k >> 2) * kB + (k & 3) * 2;
+              if (lead) mma_ss2(t_s + hf * 64, q_lo + off, b_lo + off, hi, idesc_s, k > 0);
+            }
+          }
+          if (lead) mma_commit(bars + B_SF + s * 2 + hf);
+        }
+        if (hf == 1 && j + 1 < n_steps) {
+          if (!k_seen) ok = ok && mbar_wait(bars + B_KF + (j + 1) % 3, ((j + 1) / 3) & 1, a.error_word, 8);
+          if (lead) mma_commit(bars + B_KE + (j + 1) % 3);
+        }
       }
-      mma_commit(bars + B_DRAIN);
-      mbar_wait(bars + B_DRAIN, 0, a.error_word, 11);   // nothing of ours is still running at exit
+      ce0 = ne0; ce1 = ne1;
+      ne0 = nn0; ne1 = nn1;
+      load_ent(j + 3, nn0, nn1);   // read ahead: off the critical path
     }
+    if (lead) mma_commit(bars + B_DRAIN + s);
+    mbar_wait(bars + B_DRAIN + s, 0, a.error_word, 11);   // nothing of ours is still running at exit
   } else {
     // ------------------------------ softmax warps -----------------------------------------
     const int s = warp >> 2;                                 // slot
@@ -237,48 +247,46 @@ fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUt
     const uint32_t my_s = lane_addr + kColS + s * 128, my_o = lane_addr + kColO + s * 128;
     float m_ref = -INFINITY;   // reference maximum (scaled, log2 domain) the probabilities are relative to
     float l_run = 0.f;
-    int cnt = 0;               // steps this slot took part in
-    bool ok = true;
-    auto load_ent = [&](int j, int& e0, int& e1) {
-      if (j >= n_steps) { e0 = e1 = 0; return; }
-      if (BS == 128) { e0 = e1 = ent[j]; return; }
-      e0 = ent[2 * j];
-      e1 = (2 * j + 1 < n_ent) ? ent[2 * j + 1] : (e0 & ~15);   // odd tail: same block, nobody's member
+    int p0 = 0, p1 = 0;        // P tiles published per half buffer (barrier phases)
+    // every P V product issued so far has completed (at most one per half can still be running)
+    auto wait_o = [&](uint32_t site) {
+      bool w = true;
+      if (p0 > 0) w = mbar_wait_warp(bars + B_OD + s * 2, (p0 - 1) & 1, a.error_word, site);
+      if (w && p1 > 0) w = mbar_wait_warp(bars + B_OD + s * 2 + 1, (p1 - 1) & 1, a.error_word, site);
+      return w;
     };
+    bool ok = true;
     int ne0, ne1;
     load_ent(0, ne0, ne1);
-    for (int j = 0; j < n_steps; ++j) {
+#pragma unroll 1
+    for (int j = 0; j < n_steps && ok; ++j) {
       const int e0 = ne0, e1 = ne1;
       load_ent(j + 1, ne0, ne1);
-      const uint32_t m_step = (static_cast<uint32_t>(e0) | static_cast<uint32_t>(e1)) & 15u;
-      if (((m_step >> (s * RS)) & kSlotMask) == 0) continue;          // uniform over the slot
-      // visible columns of the two 64-column halves: lo0 <= c < lim0 and lo1 <= c < lim1 (the lower
-      // bound only exists with a token-exact window, on blocks outside the sink)
-      const int key0 = (e0 >> 4) * BS, key1 = (BS == 128) ? key0 + 64 : (e1 >> 4) * BS;
-      const int lim0 = ((e0 >> member) & 1) ? min(max(qi - key0 + 1, 0), 64) : 0;
-      const int lim1 = ((e1 >> member) & 1) ? min(max(qi - key1 + 1, 0), 64) : 0;
-      const int lo0 = (a.exact_w > 0 && (e0 >> 4) >= a.ns) ? min(max(qi - a.exact_w + 1 - key0, 0), 64) : 0;
-      const int lo1 = (a.exact_w > 0 && (e1 >> 4) >= a.ns) ? min(max(qi - a.exact_w + 1 - key1, 0), 64) : 0;
-
-      ok = mbar_wait_warp(bars + B_SF + s, cnt & 1, a.error_word, 12);
-      if (!ok) break;
-      tc_fence_after();
-      // The row is walked in two halves of 64 columns, twice (maximum, then exponentials),
-      // re-reading tensor memory instead of holding 128 values: compact loops keep the softmax
-      // code resident in the instruction caches, which matters more than the extra reads.
-      float mx = -INFINITY;
-#pragma unroll 1
+#pragma unroll
       for (int hf = 0; hf < 2; ++hf) {
+        const int e = hf ? e1 : e0;
+        if (((static_cast<uint32_t>(e) >> (s * RS)) & kSlotMask) == 0) continue;   // uniform over the slot
+        // visible columns of this half: lo <= c < lim (the lower bound only exists with a
+        // token-exact window, on blocks outside the sink)
+        const int key0 = (e >> 4) * BS + (BS == 128 ? 64 * hf : 0);
+        const int lim = ((e >> member) & 1) ? min(max(qi - key0 + 1, 0), 64) : 0;
+        const int lo = (a.exact_w > 0 && (e >> 4) >= a.ns) ? min(max(qi - a.exact_w + 1 - key0, 0), 64) : 0;
+
+        ok = mbar_wait_warp(bars + B_SF + s * 2 + hf, (hf ? p1 : p0) & 1, a.error_word, 12);
+        if (!ok) break;
+        tc_fence_after();
         uint32_t v[64];
         tmem_ld32(my_s + hf * 64, v);
         tmem_ld32(my_s + hf * 64 + 32, v + 32);
         tmem_ld_wait();
-        const int lim = hf ? lim1 : lim0, lo = hf ? lo1 : lo0;   // visible columns of this half
         if (__any_sync(0xffffffffu, lim < 64 || lo > 0)) {
 #pragma unroll
-          for (int x = 0; x < 64; ++x) mx = fmaxf(mx, (x < lim && x >= lo) ? __uint_as_float(v[x]) : -INFINITY);
-        } else {
-          float m0 = mx, m1 = -INFINITY, m2 = -INFINITY, m3 = -INFINITY;
+          for (int x = 0; x < 64; ++x)
+            v[x] = (x < lim && x >= lo) ? v[x] : 0xff800000u;   // -inf: the exponential below gives exactly 0
+        }
+        float mx;
+        {
+          float m0 = -INFINITY, m1 = -INFINITY, m2 = -INFINITY, m3 = -INFINITY;
 #pragma unroll
           for (int x = 0; x < 64; x += 8) {
             m0 = max3(m0, __uint_as_float(v[x + 0]), __uint_as_float(v[x + 1]));
@@ -288,67 +296,57 @@ fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUt
           }
           mx = fmaxf(fmaxf(m0, m1), fmaxf(m2, m3));
         }
-      }
-      const float m_new = fmaxf(m_ref, mx * a.scale_log2);
-      // raise the reference only when it would grow by more than the threshold (or is still unset)
-      const bool raise = (m_new > m_ref + kFwdRescaleThreshold) || (m_ref == -INFINITY && m_new > -INFINITY);
-      if (__any_sync(0xffffffffu, raise)) {
-        const float alpha = raise ? fast_exp2(m_ref - m_new) : 1.f;   // m_ref = -inf -> 0
-        if (raise) { m_ref = m_new; l_run *= alpha; }
-        if (cnt > 0) {   // O already holds products: wait for the latest one, then rescale my row
-          ok = mbar_wait_warp(bars + B_OD + s, (cnt - 1) & 1, a.error_word, 13);
-          if (!ok) break;
-          tc_fence_after();
+        const float m_new = fmaxf(m_ref, mx * a.scale_log2);
+        // raise the reference only when it would grow by more than the threshold (or is still unset)
+        const bool raise = (m_new > m_ref + kFwdRescaleThreshold) || (m_ref == -INFINITY && m_new > -INFINITY);
+        if (__any_sync(0xffffffffu, raise)) {
+          const float alpha = raise ? fast_exp2(m_ref - m_new) : 1.f;   // m_ref = -inf -> 0
+          if (raise) { m_ref = m_new; l_run *= alpha; }
+          if (p0 + p1 > 0) {   // O already holds products: wait for them, then rescale my row
+            ok = wait_o(13);
+            if (!ok) break;
+            tc_fence_after();
 #pragma unroll 1
-          for (int c = 0; c < D / 16; ++c) {
-            uint32_t oreg[16];
-            tmem_ld16(my_o + c * 16, oreg);
-            tmem_ld_wait();
+            for (int c = 0; c < D / 16; ++c) {
+              uint32_t oreg[16];
+              tmem_ld16(my_o + c * 16, oreg);
+              tmem_ld_wait();
 #pragma unroll
-            for (int x = 0; x < 16; ++x) oreg[x] = __float_as_uint(__uint_as_float(oreg[x]) * alpha);
-            tmem_st16(my_o + c * 16, oreg);
+              for (int x = 0; x < 16; ++x) oreg[x] = __float_as_uint(__uint_as_float(oreg[x]) * alpha);
+              tmem_st16(my_o + c * 16, oreg);
+            }
           }
         }
-      }
-      const float neg_m = (m_ref == -INFINITY) ? 0.f : -m_ref;
-      float rs0 = 0.f, rs1 = 0.f;
-#pragma unroll 1
-      for (int hf = 0; hf < 2; ++hf) {
-        uint32_t v[64], preg[32];
-        tmem_ld32(my_s + hf * 64, v);
-        tmem_ld32(my_s + hf * 64 + 32, v + 32);
-        tmem_ld_wait();
-        const int lim = hf ? lim1 : lim0, lo = hf ? lo1 : lo0;
-        if (__any_sync(0xffffffffu, lim < 64 || lo > 0)) {
-#pragma unroll
-          for (int x = 0; x < 64; ++x)
-            v[x] = (x < lim && x >= lo) ? v[x] : 0xff800000u;   // -inf: the exponential below gives exactly 0
-        }
+        const float neg_m = (m_ref == -INFINITY) ? 0.f : -m_ref;
+        uint32_t preg[32];
         float q0 = 0.f, q1 = 0.f, q2 = 0.f, q3 = 0.f;   // independent partial sums
 #pragma unroll
         for (int x = 0; x < 64; x += 4) {
-          const float p0 = fast_exp2(fmaf(__uint_as_float(v[x]), a.scale_log2, neg_m));
-          const float p1 = fast_exp2(fmaf(__uint_as_float(v[x + 1]), a.scale_log2, neg_m));
-          const float p2 = fast_exp2(fmaf(__uint_as_float(v[x + 2]), a.scale_log2, neg_m));
-          const float p3 = fast_exp2(fmaf(__uint_as_float(v[x + 3]), a.scale_log2, neg_m));
+          const float x0 = fmaf(__uint_as_float(v[x]), a.scale_log2, neg_m);
+          const float x1 = fmaf(__uint_as_float(v[x + 1]), a.scale_log2, neg_m);
+          const float x2 = fmaf(__uint_as_float(v[x + 2]), a.scale_log2, neg_m);
+          const float x3 = fmaf(__uint_as_float(v[x + 3]), a.scale_log2, neg_m);
+          // a share of the exponentials goes to the FMA pipe (the exponential unit delivers 16 per clock and SM)
+          const float p0 = ((x & 7) + 0 < LG_FWD_POLY) ? poly_exp2(x0) : fast_exp2(x0);
+          const float p1 = ((x & 7) + 1 < LG_FWD_POLY) ? poly_exp2(x1) : fast_exp2(x1);
+          const float p2 = ((x & 7) + 2 < LG_FWD_POLY) ? poly_exp2(x2) : fast_exp2(x2);
+          const float p3 = ((x & 7) + 3 < LG_FWD_POLY) ? poly_exp2(x3) : fast_exp2(x3);
           q0 += p0; q1 += p1; q2 += p2; q3 += p3;
           preg[x >> 1] = pack_bf16(p0, p1);
           preg[(x >> 1) + 1] = pack_bf16(p2, p3);
         }
-        rs0 += q0 + q2;
-        rs1 += q1 + q3;
-        tmem_st32(my_s + hf * 32, preg);   // P over S columns that were already read
+        l_run += (q0 + q2) + (q1 + q3);
+        tmem_st32(my_s + hf * 64, preg);   // P over the first columns of this half's S
+        tmem_st_wait();
+        tc_fence_before();
+        __syncwarp();
+        if (lane == 0) mbar_arrive(bars + B_PF + s * 2 + hf);
+        if (hf) ++p1; else ++p0;
       }
-      l_run += rs0 + rs1;
-      tmem_st_wait();
-      tc_fence_before();
-      __syncwarp();
-      if (lane == 0) mbar_arrive(bars + B_PF + s);
-      ++cnt;
     }
     // ---- epilogue: O / l -> bf16, LSE ------------------------------------------------------
-    if (ok && cnt > 0) ok = mbar_wait_warp(bars + B_OD + s, (cnt - 1) & 1, a.error_word, 14);
-    if (ok && cnt > 0 && qi < a.L) {   // warp-uniform: L is a multiple of 64
+    if (ok) ok = wait_o(14);
+    if (ok && p0 + p1 > 0 && qi < a.L) {   // warp-uniform: L is a multiple of 64
       tc_fence_after();
       const float inv_l = l_run > 0.f ? 1.f / l_run : 0.f;
       __nv_bfloat16* orow = a.o + b * a.o_strides[0] + h * a.o_strides[1] + static_cast<int64_t>(qi) * a.o_strides[2];
@@ -373,7 +371,7 @@ fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUt
   }
   tc_fence_before();
   __syncthreads();
-  if (warp == 9) tmem_dealloc(tmem, 512);
+  if (warp == kFwdMmaWarp0) tmem_dealloc(tmem, 512);
 }
 
 }  // namespace lg
