@@ -28,7 +28,8 @@ Readings of points on which the paper is silent:
 
 Pins (tests/test_oracle_*.py): brute-force per-row softmax, torch's dense causal
 attention and autograd in fp64, central finite differences, closed-form block
-counts, the paper's KV-cache arithmetic.  Trained-model quality: parity unpinned
+counts, the paper's KV-cache arithmetic; the chunk-against-cache function (T decode
+steps) against the rows of the mask-based forward and against explicit loops.  Trained-model quality: parity unpinned
 and out of scope.
 """
 from __future__ import annotations
@@ -296,6 +297,22 @@ def decode(qv, k_lin, v_lin, n: int, sink: int, window: int, scale: float):
         z = e.sum()
         o[h] = (e / z) @ v_lin[h // G, keep]
         lse[h] = mx + np.log(z)
+    return o, lse
+
+
+def chunk_prefill(q_chunk, k_lin, v_lin, n_before: int, sink: int, window: int, scale: float):
+    """A chunk of T new tokens served against a sink + rolling-window cache (Section 3.2: in
+    serving the sparse layers keep only the sink and the last `window` tokens).  By definition
+    the result is what T successive decode steps give: token n_before + t is appended and then
+    attends to whatever the cache holds at that moment.
+
+    q_chunk [Hq, T, D]; k_lin, v_lin [Hkv, >= n_before + T, D] hold token j at index j (the
+    oracle never sees the ring layout).  Returns o [Hq, T, D], lse [Hq, T]."""
+    Hq, T, D = q_chunk.shape
+    o = np.zeros((Hq, T, D))
+    lse = np.full((Hq, T), -np.inf)
+    for t in range(T):
+        o[:, t], lse[:, t] = decode(q_chunk[:, t], k_lin, v_lin, n_before + t + 1, sink, window, scale)
     return o, lse
 
 

@@ -511,3 +511,60 @@ def test_exact_window_backward_finite_differences():
             arr[idx] = a0 - eps; fm = f(q, k, v)
             arr[idx] = a0
             assert abs((fp - fm) / (2 * eps) - grad[idx]) < 1e-6
+
+
+# --------------------------------------------------------------------- chunked prefill
+
+def test_chunk_prefill_equals_exact_window_rows():
+    """Serving a chunk against the cache gives the rows the token-exact sink + window mask gives those
+    positions in one pass over the whole sequence (the mask-based forward shares no code with the
+    decode-based chunk function): before the ring is full, exactly at the fill point, and long after."""
+    rng = np.random.default_rng(11)
+    L, D, sink, window = 640, 16, 64, 128
+    q = rng.standard_normal((4, L, D))
+    k = rng.standard_normal((2, L, D))
+    v = rng.standard_normal((2, L, D))
+    scale = 1.0 / math.sqrt(D)
+    o, lse = O.attn_forward(q, k, v, _exact(L, 64, sink, window), scale)
+    for n0, T in ((0, 64), (64, 128), (128, 64), (192, 128), (320, 192), (576, 64), (37, 5)):
+        oc, lc = O.chunk_prefill(q[:, n0:n0 + T], k, v, n0, sink, window, scale)
+        np.testing.assert_allclose(oc, o[:, n0:n0 + T], rtol=0, atol=1e-12)
+        np.testing.assert_allclose(lc, lse[:, n0:n0 + T], rtol=0, atol=1e-12)
+
+
+def test_chunk_prefill_bruteforce_tiny():
+    """Written out with loops: token i sees the sink tokens and the last `window` tokens up to itself."""
+    rng = np.random.default_rng(12)
+    Hq, Hkv, D, sink, window, n0, T = 2, 1, 4, 2, 3, 7, 4
+    q = rng.standard_normal((Hq, T, D))
+    k = rng.standard_normal((Hkv, n0 + T, D))
+    v = rng.standard_normal((Hkv, n0 + T, D))
+    o, lse = O.chunk_prefill(q, k, v, n0, sink, window, 0.7)
+    for h in range(Hq):
+        for t in range(T):
+            i = n0 + t
+            js = [j for j in range(i + 1) if j < sink or i - j < window]
+            w = [math.exp(0.7 * float(np.dot(q[h, t], k[0, j]))) for j in js]
+            z = sum(w)
+            ref = sum(wj / z * v[0, j] for wj, j in zip(w, js))
+            np.testing.assert_allclose(o[h, t], ref, rtol=1e-12, atol=1e-12)
+            assert abs(lse[h, t] - math.log(z)) < 1e-12
+
+
+def test_chunk_prefill_ignores_evicted_tokens():
+    """Tokens that fell out of the ring before the chunk arrived cannot influence it."""
+    rng = np.random.default_rng(13)
+    Hq, Hkv, D, sink, window, n0, T = 2, 2, 8, 4, 16, 40, 8
+    q = rng.standard_normal((Hq, T, D))
+    k = rng.standard_normal((Hkv, n0 + T, D))
+    v = rng.standard_normal((Hkv, n0 + T, D))
+    o, lse = O.chunk_prefill(q, k, v, n0, sink, window, 0.3)
+    k2, v2 = k.copy(), v.copy()
+    gone = slice(sink, n0 - window + 1)      # evicted before the chunk's first token attends
+    k2[:, gone] = 99.0
+    v2[:, gone] = -99.0
+    o2, lse2 = O.chunk_prefill(q, k2, v2, n0, sink, window, 0.3)
+    assert np.array_equal(o, o2) and np.array_equal(lse, lse2)
+    k2[:, n0 - window + 1] += 1.0            # the oldest token the first chunk token still sees
+    o3, _ = O.chunk_prefill(q, k2, v2, n0, sink, window, 0.3)
+    assert not np.array_equal(o3[:, 0], o[:, 0]) and np.array_equal(o3[:, 1:], o[:, 1:])
