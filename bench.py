@@ -261,6 +261,27 @@ def bench_decode(lg, c, warmup, steps, dense=False, copies=4, graph=True):
     return out
 
 
+def bench_chunk_prefill(lg, c, T, warmup, steps):
+    """A chunk of T tokens served against the full sink + window ring of the decode configuration."""
+    p = lg.decode_params(1, c.Hq, c.Hkv, c.D, c.sink_tokens, c.window_tokens)
+    cap = c.sink_tokens + c.window_tokens
+    gen = torch.Generator(device="cuda").manual_seed(0)
+    mk = lambda *shape: torch.randn(*shape, generator=gen, device="cuda").to(torch.bfloat16)
+    q, kc, vc = mk(1, c.Hq, T, c.D), mk(1, c.Hkv, T, c.D), mk(1, c.Hkv, T, c.D)
+    k_cache, v_cache = mk(1, c.Hkv, cap, c.D), mk(1, c.Hkv, cap, c.D)
+    n0 = c.n_tokens - T
+    ws = lg.chunk_prefill_workspace(p, T, n0)
+    o = torch.empty_like(q)
+    lse = torch.empty(1, c.Hq, T, dtype=torch.float32, device="cuda")
+    ms = time_cuda(lambda: lg.lg_chunk_prefill(p, q, kc, vc, k_cache, v_cache, n0, o=o, lse=lse, workspace=ws),
+                   warmup, steps)
+    assert lg.lg_last_status(ws) == 0
+    pairs = float(T) * cap          # every chunk token sees the sink and a full window
+    flop = 4.0 * c.D * pairs * c.Hq
+    return {"config": "%s_chunk_prefill_T%d" % (c.name, T), "ms": ms, "tflops": flop / ms / 1e9,
+            "note": "ring linearisation + block-index build + forward, one sequence"}
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -412,7 +433,8 @@ def main():
         torch.cuda.empty_cache()
         rp2, _ = bench_attn(lg, synth.PAPER_STRIDED, 3, 3, want_bwd=True)
         torch.cuda.empty_cache()
-        others = [r2, r2f, r4, d5, d5d, rp1, rp2]
+        cp = bench_chunk_prefill(lg, synth.CFG5, 8192, 3, 10)
+        others = [r2, r2f, r4, d5, d5d, rp1, rp2, cp]
         line["other"] = others
         line["decode_hbm_gbs"] = d5["gbs"]
         line["decode_roofline"] = {"bound": "hbm", "kernel": "decode_stream_kernel", "achieved": d5["gbs"],

@@ -155,6 +155,33 @@ lg_status lg_sparse_decode(const lg_decode_params* p, const void* q, const void*
                            const void* v_cache, const int64_t* n_tokens, void* o, float* lse,
                            void* workspace, size_t workspace_bytes, void* stream);
 
+/* ---- a chunk of new tokens served against the cache (Section 3.2: in serving, the sparse
+ *      layers keep only the sink and the most recent window of K,V) ---------------------- */
+
+/*
+ * T new tokens of every sequence attend to what the sink + window ring holds and, causally,
+ * to themselves: the token at position i sees the sink tokens and the positions j with
+ * 0 <= i - j < window_tokens.  That is what T single-token steps (append, then lg_sparse_decode)
+ * would have seen; the chunk is NOT appended by this call (use lg_kv_ring_append afterwards).
+ * It is the step that prefills a long prompt chunk by chunk with a cache of fixed size.
+ *
+ * q_chunk, o [B,Hq,T,D]; k_chunk, v_chunk [B,Hkv,T,D]; caches as above (may be NULL when
+ * n_tokens_before == 0); all bf16, contiguous, device.  lse [B,Hq,T] fp32 (device).
+ * n_tokens_before (HOST value, the same for every sequence) = tokens appended so far.
+ * Limits: sink_tokens, window_tokens and T are multiples of 64 (window_tokens >= 64), and
+ * while the ring is not yet full (n_tokens_before < sink + window) n_tokens_before is a
+ * multiple of 64 too; otherwise LG_ERR_UNSUPPORTED.  The call copies the ring's tokens in
+ * time order, followed by the chunk, into the workspace and runs the sparse forward kernel
+ * with the token-exact window over them, for the chunk's rows only.  workspace: device,
+ * 256-byte aligned, lg_chunk_prefill_workspace_bytes() bytes (0 = invalid arguments);
+ * lg_last_status(workspace, stream) reports a device-side timeout as for the forward.
+ */
+size_t lg_chunk_prefill_workspace_bytes(const lg_decode_params* p, int32_t T, int64_t n_tokens_before);
+lg_status lg_chunk_prefill(const lg_decode_params* p, const void* q_chunk, const void* k_chunk,
+                           const void* v_chunk, const void* k_cache, const void* v_cache, int32_t T,
+                           int64_t n_tokens_before, void* o, float* lse, void* workspace,
+                           size_t workspace_bytes, void* stream);
+
 /* ---- decode for callers that may not allocate -------------------------------------- */
 
 /* Size of the scratch array that lg_sparse_decode_static uses instead of a workspace.  It

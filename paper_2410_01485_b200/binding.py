@@ -54,6 +54,9 @@ SYMBOLS = {
     "lg_kv_ring_append": (C.c_int, [C.POINTER(DecodeParams), _vp, _vp, _vp, _vp, C.c_int32, _vp, _vp]),
     "lg_sparse_decode_workspace_bytes": (_sz, [C.POINTER(DecodeParams)]),
     "lg_sparse_decode": (C.c_int, [C.POINTER(DecodeParams), _vp, _vp, _vp, _vp, _vp, _vp, _vp, _sz, _vp]),
+    "lg_chunk_prefill_workspace_bytes": (_sz, [C.POINTER(DecodeParams), C.c_int32, C.c_int64]),
+    "lg_chunk_prefill": (C.c_int, [C.POINTER(DecodeParams), _vp, _vp, _vp, _vp, _vp, C.c_int32, C.c_int64, _vp, _vp,
+                                   _vp, _sz, _vp]),
     "lg_sparse_decode_static": (C.c_int, [C.POINTER(DecodeParams), _vp, _vp, _vp, _vp, _vp, _vp, _vp]),
     "lg_last_status": (C.c_int, [_vp, _vp]),
     "lg_status_string": (C.c_char_p, [C.c_int]),
@@ -240,6 +243,30 @@ def lg_sparse_decode(p: DecodeParams, q, k_cache, v_cache, n_tokens, o=None, lse
     _check(load_library().lg_sparse_decode(C.byref(p), q.data_ptr(), k_cache.data_ptr(), v_cache.data_ptr(),
                                            n_tokens.data_ptr(), o.data_ptr(), lse.data_ptr() if lse is not None else None,
                                            ws.data_ptr(), ws.numel(), _stream()), "lg_sparse_decode")
+    return o, lse
+
+
+def chunk_prefill_workspace(p: DecodeParams, T: int, n_tokens_before: int, device="cuda") -> torch.Tensor:
+    n = load_library().lg_chunk_prefill_workspace_bytes(C.byref(p), T, n_tokens_before)
+    if n == 0:
+        raise LgError(-1, "lg_chunk_prefill_workspace_bytes")
+    return torch.empty(n, dtype=torch.uint8, device=device)
+
+
+def lg_chunk_prefill(p: DecodeParams, q_chunk, k_chunk, v_chunk, k_cache, v_cache, n_tokens_before: int,
+                     o=None, lse=None, workspace=None):
+    """q_chunk [B,Hq,T,D], k_chunk, v_chunk [B,Hkv,T,D] bf16 against the ring caches (None while empty);
+    n_tokens_before is a host integer.  Returns (o [B,Hq,T,D] bf16, lse [B,Hq,T] fp32)."""
+    assert q_chunk.is_contiguous() and k_chunk.is_contiguous() and v_chunk.is_contiguous()
+    assert k_cache is None or (k_cache.is_contiguous() and v_cache.is_contiguous())
+    T = q_chunk.shape[2]
+    o = torch.empty_like(q_chunk) if o is None else o
+    lse = torch.empty(q_chunk.shape[:3], dtype=torch.float32, device=q_chunk.device) if lse is None else lse
+    ws = chunk_prefill_workspace(p, T, n_tokens_before, q_chunk.device) if workspace is None else workspace
+    _check(load_library().lg_chunk_prefill(
+        C.byref(p), q_chunk.data_ptr(), k_chunk.data_ptr(), v_chunk.data_ptr(),
+        k_cache.data_ptr() if k_cache is not None else None, v_cache.data_ptr() if v_cache is not None else None,
+        T, n_tokens_before, o.data_ptr(), lse.data_ptr(), ws.data_ptr(), ws.numel(), _stream()), "lg_chunk_prefill")
     return o, lse
 
 

@@ -76,6 +76,8 @@ lg_status resolve(const lg_attn_params* p, Resolved* r) {
   r->n_qtiles = (p->L + 127) / 128;
   r->n_ktiles = (p->L + 127) / 128;
   r->n_stiles = (p->L + 255) / 256;
+  r->q_start = 0;
+  r->Lq = p->L;
   // nnz from the per-row counts of each pattern
   int64_t nnz = 0;
   const PatternDev& pt = r->pat;
@@ -196,6 +198,89 @@ lg_status make_tmap(CUtensorMap* out, const void* base, int B, int H, int L, int
   return rc == CUDA_SUCCESS ? LG_OK : LG_ERR_CUDA;
 }
 
+
+// ---- chunk served against a sink + window ring ----------------------------------------------
+// Time-ordered copy of what the ring holds, followed by the chunk: K_lin, V_lin [B, Hkv, Lc, D]
+// with Lc = kept + T.  Row v < kept is the cache slot of position
+//   v                                   (v < sink: the sink never moves)
+//   n_before - (kept - sink) + v - sink (the kept window tokens, oldest first),
+// row v >= kept is chunk token v - kept.  One 16-byte copy per thread.
+__global__ void ring_linearise_kernel(const __nv_bfloat16* __restrict__ k_cache, const __nv_bfloat16* __restrict__ v_cache,
+                                      const __nv_bfloat16* __restrict__ k_chunk, const __nv_bfloat16* __restrict__ v_chunk,
+                                      __nv_bfloat16* __restrict__ k_lin, __nv_bfloat16* __restrict__ v_lin, int B, int Hkv,
+                                      int D, int sink, int window, int kept, int T, int64_t n_before) {
+  const int cpr = D / 8;   // 16-byte chunks per row
+  const int Lc = kept + T;
+  const int64_t gid = static_cast<int64_t>(blockIdx.x) * blockDim.x + threadIdx.x;
+  const int64_t total = static_cast<int64_t>(B) * Hkv * Lc * cpr;
+  if (gid >= total) return;
+  const int c = static_cast<int>(gid % cpr);
+  const int v = static_cast<int>((gid / cpr) % Lc);
+  const int64_t bh = gid / (static_cast<int64_t>(cpr) * Lc);
+  const __nv_bfloat16 *ksrc, *vsrc;
+  if (v < kept) {
+    const int64_t pos = v < sink ? v : n_before - (kept - sink) + (v - sink);
+    const int64_t slot = pos < sink ? pos : sink + (pos - sink) % window;
+    const int64_t off = (bh * (sink + window) + slot) * D + c * 8;
+    ksrc = k_cache + off;
+    vsrc = v_cache + off;
+  } else {
+    const int64_t off = (bh * T + (v - kept)) * D + c * 8;
+    ksrc = k_chunk + off;
+    vsrc = v_chunk + off;
+  }
+  const int64_t dst = (bh * Lc + v) * D + c * 8;
+  *reinterpret_cast<uint4*>(k_lin + dst) = *reinterpret_cast<const uint4*>(ksrc);
+  *reinterpret_cast<uint4*>(v_lin + dst) = *reinterpret_cast<const uint4*>(vsrc);
+}
+
+struct ChunkPlan {
+  lg_attn_params ap;     // exact-window sink + window attention over the kept tokens and the chunk
+  Resolved r;
+  WsLayout w;
+  int kept;              // tokens the ring holds = first query row
+  size_t lin_bytes;      // one of K_lin / V_lin
+  size_t o_k, o_v, total;
+};
+
+static lg_status plan_chunk(const lg_decode_params* p, int32_t T, int64_t n_before, ChunkPlan* c) {
+  if (!p) return LG_ERR_INVALID_ARG;
+  if (p->B <= 0 || p->Hq <= 0 || p->Hkv <= 0 || p->Hq % p->Hkv != 0) return LG_ERR_INVALID_ARG;
+  if (p->D != 64 && p->D != 128) return LG_ERR_UNSUPPORTED;
+  if (p->sink_tokens < 0 || p->window_tokens < 64 || T <= 0 || n_before < 0) return LG_ERR_INVALID_ARG;
+  // the attention kernel works on 64-token blocks: sink, window, chunk and (while the ring is
+  // not yet full) the fill level must be multiples of 64
+  if (p->sink_tokens % 64 || p->window_tokens % 64 || T % 64) return LG_ERR_UNSUPPORTED;
+  const int64_t cap = static_cast<int64_t>(p->sink_tokens) + p->window_tokens;
+  const int64_t kept = n_before < cap ? n_before : cap;
+  if (kept % 64) return LG_ERR_UNSUPPORTED;
+  if (kept + T > (1 << 24)) return LG_ERR_UNSUPPORTED;
+  c->kept = static_cast<int>(kept);
+  lg_attn_params& ap = c->ap;
+  memset(&ap, 0, sizeof(ap));
+  ap.B = p->B; ap.Hq = p->Hq; ap.Hkv = p->Hkv; ap.D = p->D;
+  ap.L = c->kept + T;
+  ap.block = 64;
+  ap.mode = LG_MODE_SINK_WINDOW;
+  ap.sink_tokens = p->sink_tokens;
+  ap.window_tokens = p->window_tokens;
+  ap.window_exact = 1;
+  ap.scale = p->scale;
+  // Q and O hold the chunk's T rows only
+  ap.q_strides[0] = ap.o_strides[0] = static_cast<int64_t>(p->Hq) * T * p->D;
+  ap.q_strides[1] = ap.o_strides[1] = static_cast<int64_t>(T) * p->D;
+  ap.q_strides[2] = ap.o_strides[2] = p->D;
+  lg_status s = resolve(&ap, &c->r);
+  if (s != LG_OK) return s;
+  c->r.q_start = c->kept;
+  c->r.Lq = T;
+  c->w = ws_layout(c->r, false);
+  c->lin_bytes = align_up(static_cast<size_t>(p->B) * p->Hkv * ap.L * p->D * sizeof(__nv_bfloat16), 256);
+  c->o_k = align_up(c->w.total, 256);
+  c->o_v = c->o_k + c->lin_bytes;
+  c->total = c->o_v + c->lin_bytes;
+  return LG_OK;
+}
 }  // namespace lg
 
 using namespace lg;
@@ -293,6 +378,40 @@ lg_status lg_sparse_attn_bwd_profiled(const lg_attn_params* p, const void* q, co
   for (int i = 0; i < 4; ++i)
     if (ev[i]) cudaEventDestroy(ev[i]);
   return s;
+}
+
+size_t lg_chunk_prefill_workspace_bytes(const lg_decode_params* p, int32_t T, int64_t n_tokens_before) {
+  ChunkPlan c;
+  return plan_chunk(p, T, n_tokens_before, &c) == LG_OK ? c.total : 0;
+}
+
+lg_status lg_chunk_prefill(const lg_decode_params* p, const void* q_chunk, const void* k_chunk, const void* v_chunk,
+                           const void* k_cache, const void* v_cache, int32_t T, int64_t n_tokens_before, void* o,
+                           float* lse, void* workspace, size_t workspace_bytes, void* stream) {
+  ChunkPlan c;
+  lg_status s = plan_chunk(p, T, n_tokens_before, &c);
+  if (s != LG_OK) return s;
+  if (!q_chunk || !k_chunk || !v_chunk || !o || !lse || !workspace) return LG_ERR_INVALID_ARG;
+  if (c.kept > 0 && (!k_cache || !v_cache)) return LG_ERR_INVALID_ARG;
+  if (!aligned16(q_chunk) || !aligned16(k_chunk) || !aligned16(v_chunk) || !aligned16(k_cache) ||
+      !aligned16(v_cache) || !aligned16(o) || !aligned16(lse) || (reinterpret_cast<uintptr_t>(workspace) & 255))
+    return LG_ERR_INVALID_ARG;
+  if (workspace_bytes < c.total) return LG_ERR_WORKSPACE;
+  if ((s = check_arch()) != LG_OK) return s;
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  uint8_t* ws = static_cast<uint8_t*>(workspace);
+  __nv_bfloat16* k_lin = reinterpret_cast<__nv_bfloat16*>(ws + c.o_k);
+  __nv_bfloat16* v_lin = reinterpret_cast<__nv_bfloat16*>(ws + c.o_v);
+  const int64_t threads = static_cast<int64_t>(p->B) * p->Hkv * c.ap.L * (p->D / 8);
+  const int64_t blocks = (threads + 255) / 256;
+  if (blocks > 0x7fffffff) return LG_ERR_UNSUPPORTED;
+  ring_linearise_kernel<<<static_cast<unsigned>(blocks), 256, 0, st>>>(
+      static_cast<const __nv_bfloat16*>(k_cache), static_cast<const __nv_bfloat16*>(v_cache),
+      static_cast<const __nv_bfloat16*>(k_chunk), static_cast<const __nv_bfloat16*>(v_chunk), k_lin, v_lin, p->B,
+      p->Hkv, p->D, p->sink_tokens, p->window_tokens, c.kept, T, n_tokens_before);
+  if (cudaGetLastError() != cudaSuccess) return LG_ERR_CUDA;
+  if ((s = prepare_workspace(c.r, c.w, ws, false, st)) != LG_OK) return s;
+  return launch_fwd(c.r, c.w, q_chunk, k_lin, v_lin, o, lse, ws, st);
 }
 
 lg_status lg_last_status(void* workspace, void* stream) {

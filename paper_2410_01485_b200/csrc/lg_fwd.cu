@@ -9,7 +9,7 @@ static lg_status launch_fwd_t(const Resolved& r, const WsLayout& w, const void* 
                               void* o, float* lse, uint8_t* ws, cudaStream_t stream) {
   CUtensorMap tq, tk, tv;
   lg_status s;
-  if ((s = make_tmap(&tq, q, r.B, r.Hq, r.L, D, r.qs, 128)) != LG_OK) return s;
+  if ((s = make_tmap(&tq, q, r.B, r.Hq, r.Lq, D, r.qs, 128)) != LG_OK) return s;
   if ((s = make_tmap(&tk, k, r.B, r.Hkv, r.L, D, r.ks, BS)) != LG_OK) return s;
   if ((s = make_tmap(&tv, v, r.B, r.Hkv, r.L, D, r.vs, BS)) != LG_OK) return s;
   FwdArgs a;
@@ -22,6 +22,7 @@ static lg_status launch_fwd_t(const Resolved& r, const WsLayout& w, const void* 
   a.error_word = reinterpret_cast<unsigned int*>(ws);
   for (int i = 0; i < 3; ++i) a.o_strides[i] = r.os[i];
   a.L = r.L; a.Hq = r.Hq; a.G = r.G;
+  a.q_start = r.q_start; a.Lq = r.Lq;
   a.exact_w = r.exact_w; a.ns = r.pat.ns;
   a.scale_log2 = r.scale * 1.4426950408889634f;
   auto kern = fwd_kernel<D, BS>;

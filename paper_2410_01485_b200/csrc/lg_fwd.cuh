@@ -34,6 +34,8 @@ struct FwdArgs {
   unsigned int* error_word;
   int64_t o_strides[3];      // batch, head, token (elements)
   int L, Hq, G;              // G = Hq / Hkv
+  int q_start, Lq;           // queries exist for rows [q_start, q_start + Lq) of the L key positions only
+                             // (a chunk served against a cache); Q, O, LSE are indexed by row - q_start
   int exact_w, ns;           // token-exact window (0: off) and number of sink blocks
   float scale_log2;          // scale * log2(e)
 };
@@ -93,6 +95,7 @@ fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUt
   const int32_t* ent = a.tile_ent + a.tile_off[tile * R4];
   const int row0 = tile * 256;
   const int n_steps = (BS == 128) ? n_ent : (n_ent + 1) / 2;
+  if (row0 + 256 <= a.q_start) return;   // no query lives in this super-tile (uniform over the CTA)
 
   // entries of the two halves of step j (0: nobody's member, also past the end)
   auto load_ent = [&](int j, int& e0, int& e1) {
@@ -130,7 +133,8 @@ fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUt
       for (int s = 0; s < 2; ++s)
 #pragma unroll
         for (int x = 0; x < D / 64; ++x)
-          tma_load_4d(sQ + s * kTile + x * SM::kBox, &tm_q, bars + B_Q, x * 64, row0 + s * 128, h, b);
+          // rows before q_start lie outside the tensor and arrive as zeros (their results are never stored)
+          tma_load_4d(sQ + s * kTile + x * SM::kBox, &tm_q, bars + B_Q, x * 64, row0 + s * 128 - a.q_start, h, b);
       auto load_step = [&](uint8_t* dst, const CUtensorMap* tm, uint64_t* bar, int kb0, int kb1) {
 #pragma unroll
         for (int x = 0; x < D / 64; ++x) {
@@ -346,10 +350,11 @@ fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUt
     }
     // ---- epilogue: O / l -> bf16, LSE ------------------------------------------------------
     if (ok) ok = wait_o(14);
-    if (ok && p0 + p1 > 0 && qi < a.L) {   // warp-uniform: L is a multiple of 64
+    if (ok && p0 + p1 > 0 && qi < a.L && qi >= a.q_start) {   // warp-uniform: L and q_start are multiples of 64
       tc_fence_after();
       const float inv_l = l_run > 0.f ? 1.f / l_run : 0.f;
-      __nv_bfloat16* orow = a.o + b * a.o_strides[0] + h * a.o_strides[1] + static_cast<int64_t>(qi) * a.o_strides[2];
+      __nv_bfloat16* orow =
+          a.o + b * a.o_strides[0] + h * a.o_strides[1] + static_cast<int64_t>(qi - a.q_start) * a.o_strides[2];
 #pragma unroll
       for (int c = 0; c < D / 32; ++c) {
         uint32_t oreg[32];
@@ -365,7 +370,7 @@ fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUt
           *reinterpret_cast<uint4*>(orow + c * 32 + x) = v4;
         }
       }
-      a.lse[(static_cast<int64_t>(b) * a.Hq + h) * a.L + qi] =
+      a.lse[(static_cast<int64_t>(b) * a.Hq + h) * a.Lq + qi - a.q_start] =
           l_run > 0.f ? (m_ref + log2f(l_run)) * 0.6931471805599453f : -INFINITY;
     }
   }

@@ -21,6 +21,7 @@ struct Resolved {          // validated, defaulted copy of lg_attn_params
   int64_t qs[3], ks[3], vs[3], os[3];
   int n_qtiles, n_ktiles;  // ceil(L / 128)
   int n_stiles;            // ceil(L / 256): super-tiles of the forward
+  int q_start, Lq;         // forward only: queries exist for rows [q_start, q_start + Lq) (0, L by default)
   int64_t nnz;
 };
 

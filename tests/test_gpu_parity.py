@@ -347,3 +347,88 @@ def test_decode_dense_comparator_matches_sparse_on_same_tokens(lg):
     od, lsed = lg.lg_sparse_decode(pd, q, kc, vc, torch.full((B,), sink + W, dtype=torch.int64, device="cuda"))
     torch.cuda.synchronize()
     assert torch.equal(od, o) and torch.equal(lsed, lse)
+
+
+# ------------------------------------------------------------------------- chunk served against the ring
+
+def _chunk_prefill_case(lg, B, Hq, Hkv, D, sink, W, n0, T, seed=0, heads=None):
+    """History of n0 tokens appended to the ring (lg_kv_ring_append, checked byte-exact elsewhere), then
+    a chunk of T tokens served against it; compared with the oracle's T decode steps on the linear history."""
+    p = lg.decode_params(B, Hq, Hkv, D, sink, W)
+    g = torch.Generator(device="cuda").manual_seed(seed)
+    hist_k = torch.randn(B, Hkv, n0 + T, D, generator=g, device="cuda").to(torch.bfloat16)
+    hist_v = torch.randn(B, Hkv, n0 + T, D, generator=g, device="cuda").to(torch.bfloat16)
+    q = torch.randn(B, Hq, T, D, generator=g, device="cuda").to(torch.bfloat16)
+    kc = torch.full((B, Hkv, sink + W, D), float("nan"), device="cuda", dtype=torch.bfloat16)   # unused slots must not be read
+    vc = torch.full((B, Hkv, sink + W, D), float("nan"), device="cuda", dtype=torch.bfloat16)
+    if n0 > 0:
+        nb = torch.zeros(B, dtype=torch.int64, device="cuda")
+        lg.lg_kv_ring_append(p, kc, vc, hist_k[:, :, :n0].contiguous(), hist_v[:, :, :n0].contiguous(), nb)
+    ws = lg.chunk_prefill_workspace(p, T, n0)
+    o, lse = lg.lg_chunk_prefill(p, q, hist_k[:, :, n0:].contiguous(), hist_v[:, :, n0:].contiguous(), kc, vc, n0,
+                                 workspace=ws)
+    assert lg.lg_last_status(ws) == 0
+    scale = 1.0 / np.sqrt(D)
+    G = Hq // Hkv
+    worst = 0.0
+    for b in range(B):
+        hs = list(range(Hq)) if heads is None else heads
+        oo = np.zeros((len(hs), T, D))
+        ll = np.zeros((len(hs), T))
+        for x, h in enumerate(hs):   # one query head at a time, with its kv head
+            oo[x:x + 1], ll[x:x + 1] = O.chunk_prefill(synth.to_f64(q[b][h:h + 1]),
+                                                       synth.to_f64(hist_k[b][h // G:h // G + 1]),
+                                                       synth.to_f64(hist_v[b][h // G:h // G + 1]), n0, sink, W, scale)
+        worst = max(worst, _assert_close(synth.to_f64(o[b][hs]), oo, TOL_O, "chunk o"))
+        assert np.abs(synth.to_f64(lse[b][hs]) - ll).max() <= TOL_LSE
+    return o, lse, q, hist_k, hist_v, p
+
+
+@pytest.mark.parametrize("args", [
+    (1, 2, 2, 64, 64, 128, 0, 64),          # empty cache: plain causal start
+    (2, 4, 2, 128, 64, 128, 64, 128),       # ring not yet full (fill level a multiple of 64)
+    (1, 4, 1, 128, 64, 128, 192, 64),       # exactly full
+    (2, 4, 2, 128, 64, 128, 1000, 192),     # wrapped ring, odd fill level, chunk longer than the window
+    (1, 8, 2, 64, 0, 256, 777, 320),        # no sink; chunk spans two super-tiles with a ragged second one
+    (1, 2, 2, 128, 128, 512, 5003, 448),    # first super-tile half below the first query row (640 = 2.5 x 256)
+], ids=str)
+def test_chunk_prefill_small(lg, args):
+    _chunk_prefill_case(lg, *args)
+
+
+def test_chunk_prefill_equals_decode_steps_on_gpu(lg):
+    """Serving consistency on the GPU itself: the chunk's rows equal what appending one token at a time and
+    decoding gives (two different kernels, same cache)."""
+    B, Hq, Hkv, D, sink, W, n0, T = 1, 8, 2, 128, 64, 256, 900, 64
+    o, lse, q, hist_k, hist_v, p = _chunk_prefill_case(lg, B, Hq, Hkv, D, sink, W, n0, T, seed=3)
+    kc = torch.zeros((B, Hkv, sink + W, D), device="cuda", dtype=torch.bfloat16)
+    vc = torch.zeros_like(kc)
+    lg.lg_kv_ring_append(p, kc, vc, hist_k[:, :, :n0].contiguous(), hist_v[:, :, :n0].contiguous(),
+                         torch.zeros(B, dtype=torch.int64, device="cuda"))
+    for t in (0, 1, 31, 63):
+        # bring the ring to position n0 + t (inclusive), then decode that token
+        kc2, vc2 = kc.clone(), vc.clone()
+        lg.lg_kv_ring_append(p, kc2, vc2, hist_k[:, :, n0:n0 + t + 1].contiguous(), hist_v[:, :, n0:n0 + t + 1].contiguous(),
+                             torch.full((B,), n0, dtype=torch.int64, device="cuda"))
+        od, ld = lg.lg_sparse_decode(p, q[:, :, t].contiguous(), kc2, vc2,
+                                     torch.full((B,), n0 + t + 1, dtype=torch.int64, device="cuda"))
+        assert (od.float() - o[:, :, t].float()).abs().max() <= 1e-2
+        assert (ld - lse[:, :, t]).abs().max() <= 1e-3
+
+
+def test_chunk_prefill_cfg5_shape(lg):
+    """Llama-2-70B-shaped ring (128 sink + 4096 window, 64 query heads over 8 kv heads) at context 131072, a
+    2048-token chunk; sampled heads against the oracle."""
+    c = synth.CFG5
+    _chunk_prefill_case(lg, 1, c.Hq, c.Hkv, c.D, c.sink_tokens, c.window_tokens, 20000, 2048, seed=1, heads=[0, 37])
+
+
+def test_chunk_prefill_rejects_unsupported(lg):
+    p = lg.decode_params(1, 2, 2, 128, 64, 128)
+    L = lg.load_library()
+    import ctypes as C
+    assert L.lg_chunk_prefill_workspace_bytes(C.byref(p), 60, 0) == 0        # chunk not a multiple of 64
+    assert L.lg_chunk_prefill_workspace_bytes(C.byref(p), 64, 100) == 0      # ring not full, ragged fill level
+    assert L.lg_chunk_prefill_workspace_bytes(C.byref(p), 64, 1000) > 0      # full ring: any fill level
+    p2 = lg.decode_params(1, 2, 2, 128, 32, 128)
+    assert L.lg_chunk_prefill_workspace_bytes(C.byref(p2), 64, 0) == 0       # sink not a multiple of 64
