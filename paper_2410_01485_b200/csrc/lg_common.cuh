@@ -14,9 +14,6 @@ struct WsHeader {
 };
 static_assert(sizeof(WsHeader) == 256, "header size");
 
-#ifndef LG_WAIT_SLEEP_NS
-#define LG_WAIT_SLEEP_NS 0
-#endif
 constexpr long long kWaitLimitCycles = 4000000000ll;   // ~2 s of SM clock: a wait that long gave up
 
 __device__ __forceinline__ uint32_t smem_u32(const void* p) {
@@ -70,9 +67,6 @@ static __device__ __noinline__ bool mbar_wait_slow(uint64_t* bar, uint32_t parit
 #pragma unroll 1
     for (int it = 0; it < 256; ++it) {
       if (mbar_try_wait(bar, parity)) return true;
-#if LG_WAIT_SLEEP_NS > 0
-      __nanosleep(LG_WAIT_SLEEP_NS);   // a polling warp would otherwise take issue slots from the working warps
-#endif
     }
     if (clock64() - t0 > kWaitLimitCycles) break;
   }
@@ -275,20 +269,6 @@ __device__ __forceinline__ float fast_exp2(float x) {
   float y;
   asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
   return y;
-}
-// 2^x evaluated on the FMA pipe (the exponential unit delivers 16 results per clock and SM,
-// which is what bounds a softmax over 128-wide tiles): round x to the nearest integer n with
-// the 1.5 * 2^23 trick, degree-3 polynomial for 2^(x - n) on [-0.5, 0.5] (relative error
-// below 8e-5, far inside bf16's 2^-9), exponent patched in with an integer add.
-// Valid for x <= 127; x below -126 (including -inf) gives about 2^-126, not 0.
-__device__ __forceinline__ float poly_exp2(float x) {
-  x = fmaxf(x, -126.f);
-  const float t = x + 12582912.f;
-  const float f = x - (t - 12582912.f);
-  float p = fmaf(0.05517033f, f, 0.24260782f);
-  p = fmaf(p, f, 0.69326091f);
-  p = fmaf(p, f, 0.9999283f);
-  return __int_as_float(__float_as_int(p) + (__float_as_int(t) << 23));
 }
 // packed pairs of fp32 (one instruction for two lanes of work on sm_100)
 __device__ __forceinline__ uint64_t f32x2(float lo, float hi) {

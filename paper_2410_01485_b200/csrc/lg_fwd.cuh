@@ -43,11 +43,6 @@ struct FwdArgs {
 constexpr int kFwdTmaWarp = 8, kFwdMmaWarp0 = 9;
 constexpr int kFwdThreads = 11 * 32;
 constexpr float kFwdRescaleThreshold = 8.0f;   // log2 units
-// Of every 8 exponentials, this many are evaluated on the FMA pipe instead of the exponential unit.
-#ifndef LG_FWD_POLY
-#define LG_FWD_POLY 0
-#endif
-
 template <int D>
 struct FwdSmem {
   static constexpr int kBox = 128 * 128;               // one 64-column box of 128 rows
@@ -330,11 +325,7 @@ fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUt
           const float x1 = fmaf(__uint_as_float(v[x + 1]), a.scale_log2, neg_m);
           const float x2 = fmaf(__uint_as_float(v[x + 2]), a.scale_log2, neg_m);
           const float x3 = fmaf(__uint_as_float(v[x + 3]), a.scale_log2, neg_m);
-          // a share of the exponentials goes to the FMA pipe (the exponential unit delivers 16 per clock and SM)
-          const float p0 = ((x & 7) + 0 < LG_FWD_POLY) ? poly_exp2(x0) : fast_exp2(x0);
-          const float p1 = ((x & 7) + 1 < LG_FWD_POLY) ? poly_exp2(x1) : fast_exp2(x1);
-          const float p2 = ((x & 7) + 2 < LG_FWD_POLY) ? poly_exp2(x2) : fast_exp2(x2);
-          const float p3 = ((x & 7) + 3 < LG_FWD_POLY) ? poly_exp2(x3) : fast_exp2(x3);
+          const float p0 = fast_exp2(x0), p1 = fast_exp2(x1), p2 = fast_exp2(x2), p3 = fast_exp2(x3);
           q0 += p0; q1 += p1; q2 += p2; q3 += p3;
           preg[x >> 1] = pack_bf16(p0, p1);
           preg[(x >> 1) + 1] = pack_bf16(p2, p3);
