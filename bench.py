@@ -390,7 +390,7 @@ def main():
             "pct_of_nominal_bf16_peak": 100.0 * value / world / NOMINAL_BF16_TFLOPS,
             "pct_of_measured_bf16_sustained": 100.0 * value / world / peaks["bf16_sustained"],
             "roofline": roofline, "clocks": clocks.summary(),
-            "gpu_launches": args.steps * 20}
+            "gpu_launches": args.steps * 19}
 
     del dq, dk, dv
     others = []

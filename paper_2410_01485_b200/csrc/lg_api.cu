@@ -146,14 +146,16 @@ lg_status prepare_workspace(const Resolved& r, const WsLayout& w, uint8_t* ws, b
   lg_status s = launch_index_build(r, i32(w.row_ptr), i32(w.col_idx), i32(w.col_ptr), i32(w.row_idx), stream);
   if (s != LG_OK) return s;
   const int R = 128 / r.block;
-  tile_merge_kernel<<<(r.n_qtiles + 127) / 128, 128, 0, stream>>>(i32(w.row_ptr), i32(w.col_idx), r.pat.nB, R,
-                                                                  r.n_qtiles, i32(w.qt_cnt), i32(w.qt_ent));
-  tile_order_kernel<<<(r.n_qtiles + 127) / 128, 128, 0, stream>>>(i32(w.qt_cnt), r.n_qtiles, i32(w.qt_order));
-  tile_merge4_kernel<<<(r.n_stiles + 127) / 128, 128, 0, stream>>>(i32(w.row_ptr), i32(w.col_idx), r.pat.nB, 2 * R,
-                                                                   r.n_stiles, i32(w.sq_cnt), i32(w.sq_ent));
-  tile_order_kernel<<<(r.n_stiles + 127) / 128, 128, 0, stream>>>(i32(w.sq_cnt), r.n_stiles, i32(w.sq_order));
+  if (!want_bwd) {   // the forward walks super-tiles of 256 rows; the backward passes have their own schedules
+    tile_merge4_kernel<<<(r.n_stiles + 127) / 128, 128, 0, stream>>>(i32(w.row_ptr), i32(w.col_idx), r.pat.nB, 2 * R,
+                                                                     r.n_stiles, i32(w.sq_cnt), i32(w.sq_ent));
+    tile_order_kernel<<<(r.n_stiles + 127) / 128, 128, 0, stream>>>(i32(w.sq_cnt), r.n_stiles, i32(w.sq_order));
+  }
   if (want_bwd) {
     const int nB = r.pat.nB, nt = r.n_ktiles;
+    tile_merge_kernel<<<(r.n_qtiles + 127) / 128, 128, 0, stream>>>(i32(w.row_ptr), i32(w.col_idx), nB, R, r.n_qtiles,
+                                                                    i32(w.qt_cnt), i32(w.qt_ent));
+    tile_order_kernel<<<(r.n_qtiles + 127) / 128, 128, 0, stream>>>(i32(w.qt_cnt), r.n_qtiles, i32(w.qt_order));
     kv_tile_cols_kernel<<<(nt * R + 127) / 128, 128, 0, stream>>>(i32(w.col_ptr), nB, R, nt, i32(w.kt_cols));
     kv_tile_len_kernel<<<(nt + 127) / 128, 128, 0, stream>>>(i32(w.col_ptr), i32(w.kt_cols), R, nt, i32(w.kt_off));
     index_scan_kernel<<<1, 1024, 0, stream>>>(i32(w.kt_off), i32(w.kt_off), nt);
