@@ -124,7 +124,7 @@ WsLayout ws_layout(const Resolved& r, bool want_bwd) {
     w.kt_order = take(r.n_ktiles * 4);
     w.kt_cols = take(static_cast<size_t>(r.n_ktiles) * 2 * 4);
     w.kt_off = take((static_cast<size_t>(r.n_ktiles) + 1) * 4);
-    w.delta = take(static_cast<size_t>(r.B) * r.Hq * r.L * 8);   // (LSE * log2 e, delta) per query row
+    w.delta = take(static_cast<size_t>(r.B) * r.Hq * r.L * 8);   // two planes: -LSE * log2 e and -delta per query row
   }
   w.total = off;
   return w;

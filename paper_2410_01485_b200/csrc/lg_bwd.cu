@@ -9,7 +9,7 @@ static lg_status launch_bwd_t(const Resolved& r, const WsLayout& w, const void* 
                               const void* o, const float* lse, const void* d_o, void* dq, void* dk, void* dv,
                               uint8_t* ws, cudaStream_t stream, cudaEvent_t* marks) {
   lg_status s;
-  float2* stat = reinterpret_cast<float2*>(ws + w.delta);
+  float* stat = reinterpret_cast<float*>(ws + w.delta);
   if (marks) cudaEventRecord(marks[0], stream);
   {
     const int64_t rows = static_cast<int64_t>(r.B) * r.Hq * r.L;
@@ -23,6 +23,7 @@ static lg_status launch_bwd_t(const Resolved& r, const WsLayout& w, const void* 
   if (marks) cudaEventRecord(marks[1], stream);
   BwdArgs a;
   a.stat = stat;
+  a.stat_plane = static_cast<int64_t>(r.B) * r.Hq * r.L;
   a.error_word = reinterpret_cast<unsigned int*>(ws);
   a.L = r.L; a.Hq = r.Hq; a.Hkv = r.Hkv; a.G = r.G;
   a.exact_w = r.exact_w; a.ns = r.pat.ns;

@@ -35,7 +35,8 @@ struct BwdArgs {
   const int32_t* tile_cnt;
   const int32_t* tile_ent;   // idx * 4 + member mask
   const int32_t* order;
-  const float2* stat;        // [B, Hq, L / 2] x (-LSE2 of rows 2i, 2i+1, -delta of rows 2i, 2i+1), LSE2 = LSE * log2(e)
+  const float* stat;         // two planes of [B, Hq, L] floats: -LSE * log2(e), then -delta
+  int64_t stat_plane;        // floats per plane
   __nv_bfloat16* out0;       // dQ   | dK
   __nv_bfloat16* out1;       // unused | dV
   unsigned int* error_word;
@@ -45,12 +46,12 @@ struct BwdArgs {
   float scale, scale_log2;
 };
 
-// ---- stat = -(LSE * log2 e) and -rowsum(dO * O), stored negated (they are only ever subtracted)
-// and with the rows paired, (a_2i, a_2i+1, b_2i, b_2i+1), so that two neighbouring rows feed one
-// packed fp32x2 instruction --------------------------------------------------------------------
+// ---- stat = -(LSE * log2 e) and -rowsum(dO * O), stored negated (they are only ever subtracted),
+// each in a plane of its own: the dK/dV pass fetches four neighbouring queries' values of one kind
+// with a single 16-byte shared-memory load ---------------------------------------------------------
 template <int D>
 __global__ void delta_kernel(const __nv_bfloat16* __restrict__ o, const __nv_bfloat16* __restrict__ d_o,
-                             const float* __restrict__ lse, float2* __restrict__ stat, int64_t sb, int64_t sh,
+                             const float* __restrict__ lse, float* __restrict__ stat, int64_t sb, int64_t sh,
                              int64_t sl, int Hq, int L, int64_t total_rows) {
   constexpr int TPR = D / 8;   // threads per row, 16 bytes each
   const int64_t gid = static_cast<int64_t>(blockIdx.x) * blockDim.x + threadIdx.x;
@@ -76,9 +77,8 @@ __global__ void delta_kernel(const __nv_bfloat16* __restrict__ o, const __nv_bfl
 #pragma unroll
   for (int s = TPR / 2; s > 0; s >>= 1) acc += __shfl_xor_sync(0xffffffffu, acc, s);
   if (row < total_rows && ch == 0) {
-    float* f = reinterpret_cast<float*>(stat) + (row >> 1) * 4 + (row & 1);
-    f[0] = -lse[row] * 1.4426950408889634f;
-    f[2] = -acc;
+    stat[row] = -lse[row] * 1.4426950408889634f;
+    stat[total_rows + row] = -acc;
   }
 }
 
@@ -97,7 +97,7 @@ struct BwdSmem {
   static constexpr int oFix0 = 0, oFix1 = kTile;
   static constexpr int oA = 2 * kTile;
   static constexpr int oB = oA + kAStages * kTile;
-  static constexpr int oStat = oB + kBStages * kTile;            // dK/dV pass: [2][128] float2
+  static constexpr int oStat = oB + kBStages * kTile;            // dK/dV pass: [2 stages][2 planes][128] floats
   static constexpr int oBar = oStat + 2 * 128 * 8;
   static constexpr int kTotal = oBar + 256;
 };
@@ -330,9 +330,8 @@ bwd_dq_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ 
     float nlse2 = 0.f, ndlt = 0.f;   // -LSE2 and -delta of my row
     if (qi < a.L) {
       const int64_t row = (static_cast<int64_t>(b) * a.Hq + h) * a.L + qi;
-      const float* f = reinterpret_cast<const float*>(a.stat) + (row >> 1) * 4 + (row & 1);
-      nlse2 = f[0];
-      ndlt = f[2];
+      nlse2 = a.stat[row];
+      ndlt = a.stat[a.stat_plane + row];
     }
     // entry of the step: read one step ahead so that the load is off the critical path
     auto entry_of = [&](int j, bool& have) {
@@ -464,7 +463,7 @@ bwd_dkdv_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
   uint8_t* sV = smem + SM::oFix1;
   uint8_t* sQ = smem + SM::oA;     // [3]
   uint8_t* sDO = smem + SM::oB;    // [2]
-  float2* sStat = reinterpret_cast<float2*>(smem + SM::oStat);   // [2][128]
+  float* sStat = reinterpret_cast<float*>(smem + SM::oStat);   // [2 stages][-LSE2 | -delta][128 queries]
 
   const int tile = a.order[blockIdx.y];
   const int b = blockIdx.x / a.Hkv, hk = blockIdx.x % a.Hkv;
@@ -538,15 +537,19 @@ bwd_dkdv_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
         if (!ok) break;
         sEnt[so * 2] = e0;
         sEnt[so * 2 + 1] = e1;
-        mbar_expect_tx(bars + B_STF + so, 128 * 8);             // (release: publishes the entries as well)
+        mbar_expect_tx(bars + B_STF + so, 2 * 128 * 4);         // (release: publishes the entries as well)
         {
-          const float2* st0 = a.stat + (static_cast<int64_t>(b) * a.Hq + h0) * a.L + r0;
-          const float2* st1 = a.stat + (static_cast<int64_t>(b) * a.Hq + h1) * a.L + r1;
-          if (BS == 128) {
-            bulk_load(sStat + so * 128, st0, 128 * 8, bars + B_STF + so);
-          } else {
-            bulk_load(sStat + so * 128, st0, 64 * 8, bars + B_STF + so);
-            bulk_load(sStat + so * 128 + 64, st1, 64 * 8, bars + B_STF + so);
+          const float* st0 = a.stat + (static_cast<int64_t>(b) * a.Hq + h0) * a.L + r0;
+          const float* st1 = a.stat + (static_cast<int64_t>(b) * a.Hq + h1) * a.L + r1;
+#pragma unroll
+          for (int pl = 0; pl < 2; ++pl) {
+            float* dst = sStat + (so * 2 + pl) * 128;
+            if (BS == 128) {
+              bulk_load(dst, st0 + pl * a.stat_plane, 128 * 4, bars + B_STF + so);
+            } else {
+              bulk_load(dst, st0 + pl * a.stat_plane, 64 * 4, bars + B_STF + so);
+              bulk_load(dst + 64, st1 + pl * a.stat_plane, 64 * 4, bars + B_STF + so);
+            }
           }
         }
         nst = j + 1;
@@ -685,8 +688,9 @@ bwd_dkdv_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
         ok = __all_sync(0xffffffffu, ok);
         if (!ok) break;
       }
-      // (-LSE2_c, -LSE2_c+1, -delta_c, -delta_c+1) of my column pairs
-      const float4* st = reinterpret_cast<const float4*>(sStat + (j & 1) * 128 + half * kKvHalf + g * C);
+      // -LSE2 and -delta of my C queries, four to a load
+      const float4* st_l = reinterpret_cast<const float4*>(sStat + (j & 1) * 256 + half * kKvHalf + g * C);
+      const float4* st_d = st_l + 128 / 4;
       // the queries my columns hold, and from which of them on this key may be seen
       const int entry = sEnt[(j & 1) * 2 + (BS == 64 ? half : 0)];
       const int q0 = (entry >> 2) * BS + (BS == 128 ? kKvHalf * half : 0) + C * g;
@@ -707,18 +711,24 @@ bwd_dkdv_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
         tmem_ld_wait();
         const bool masked = __any_sync(0xffffffffu, xmin > 0 || xmax < C);
 #pragma unroll
-        for (int c = 0; c < C; c += 2) {
-          const float4 s4 = st[c >> 1];
-          float x0, x1;
+        for (int c = 0; c < C; c += 4) {
+          const float4 l4 = st_l[c >> 2];
+          float x0, x1, x2, x3;
           f32x2_split(fma_f32x2(f32x2(__uint_as_float(sreg[c]), __uint_as_float(sreg[c + 1])), scale2,
-                                f32x2(s4.x, s4.y)), x0, x1);
-          float v0 = fast_exp2(x0), v1 = fast_exp2(x1);
+                                f32x2(l4.x, l4.y)), x0, x1);
+          f32x2_split(fma_f32x2(f32x2(__uint_as_float(sreg[c + 2]), __uint_as_float(sreg[c + 3])), scale2,
+                                f32x2(l4.z, l4.w)), x2, x3);
+          float v0 = fast_exp2(x0), v1 = fast_exp2(x1), v2 = fast_exp2(x2), v3 = fast_exp2(x3);
           if (masked) {
             v0 = (c >= xmin && c < xmax) ? v0 : 0.f;
             v1 = (c + 1 >= xmin && c + 1 < xmax) ? v1 : 0.f;
+            v2 = (c + 2 >= xmin && c + 2 < xmax) ? v2 : 0.f;
+            v3 = (c + 3 >= xmin && c + 3 < xmax) ? v3 : 0.f;
           }
           p[c] = v0;
           p[c + 1] = v1;
+          p[c + 2] = v2;
+          p[c + 3] = v3;
         }
         uint32_t preg[C / 2];
 #pragma unroll
@@ -736,13 +746,17 @@ bwd_dkdv_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
         if constexpr (C == 16) tmem_ld16(dp_addr, dreg); else tmem_ld32(dp_addr, dreg);
         tmem_ld_wait();
 #pragma unroll
-        for (int x = 0; x < C; x += 2) {
-          const float4 s4 = st[x >> 1];
-          float d0, d1;
+        for (int x = 0; x < C; x += 4) {
+          const float4 d4 = st_d[x >> 2];
+          float d0, d1, d2, d3;
           f32x2_split(mul_f32x2(f32x2(p[x], p[x + 1]),
                                 add_f32x2(f32x2(__uint_as_float(dreg[x]), __uint_as_float(dreg[x + 1])),
-                                          f32x2(s4.z, s4.w))), d0, d1);
+                                          f32x2(d4.x, d4.y))), d0, d1);
+          f32x2_split(mul_f32x2(f32x2(p[x + 2], p[x + 3]),
+                                add_f32x2(f32x2(__uint_as_float(dreg[x + 2]), __uint_as_float(dreg[x + 3])),
+                                          f32x2(d4.z, d4.w))), d2, d3);
           dsreg[x >> 1] = pack_bf16(d0, d1);
+          dsreg[(x >> 1) + 1] = pack_bf16(d2, d3);
         }
       }
       if constexpr (C == 16) tmem_st8(dp_addr, dsreg); else tmem_st16(dp_addr, dsreg);                               // dS^T over my own dP^T columns

@@ -34,7 +34,7 @@ struct WsLayout {
   size_t sq_cnt, sq_ent, sq_order;               // super-tile schedules (forward)
   size_t kt_cnt, kt_ent, kt_order;               // kv-tile schedules (dK/dV pass)
   size_t kt_cols, kt_off;                        // members of each kv tile, start of its schedule
-  size_t delta;                                  // float2 [B, Hq, L]: (LSE * log2 e, delta) (bwd only)
+  size_t delta;                                  // 2 x float [B, Hq, L]: -LSE * log2 e, then -delta (bwd only)
   size_t total;
 };
 WsLayout ws_layout(const Resolved& r, bool want_bwd);
