@@ -434,7 +434,11 @@ bwd_dq_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ 
 constexpr int kKvEwWarps = LG_KV_EW_WARPS;
 constexpr int kKvTmaWarp = kKvEwWarps, kKvMmaWarpA = kKvEwWarps + 1, kKvMmaWarpB = kKvEwWarps + 2;
 constexpr int kKvThreads = (kKvEwWarps + 3) * 32;
-constexpr int kKvHalf = 64;                                // queries of a half-step
+#ifndef LG_KV_HALF
+#define LG_KV_HALF 64
+#endif
+constexpr int kKvHalf = LG_KV_HALF;                        // queries of a (half-)step: 64, or 128 = whole steps, single buffers
+constexpr int kKvNB = 128 / kKvHalf;                       // (half-)steps per step = score buffers in rotation
 constexpr int kKvCols = kKvHalf / (kKvEwWarps / 4);        // queries of a half-step per element-wise thread
 
 template <int D, int BS>
@@ -472,10 +476,10 @@ bwd_dkdv_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
   // key blocks of the tile's members (with 64-token blocks the two members need not be neighbours)
   const int kb_a = a.tile_cols[R * tile], kb_b = (R == 2) ? a.tile_cols[R * tile + 1] : -1;
   const int n_items = n_ent * a.G;
-  const int n_hs = (BS == 128) ? 2 * n_items : n_items;    // half-steps
-  const int n_steps = (n_hs + 1) / 2;                      // 128-row tiles streamed
-  // half-step hs belongs to step hs >> 1 and is its last one when:
-  auto closes_step = [&](int hs) { return (hs & 1) || hs == n_hs - 1; };
+  const int n_hs = (BS == 128) ? kKvNB * n_items : (kKvNB == 2 ? n_items : (n_items + 1) / 2);    // half-steps
+  const int n_steps = (n_hs + kKvNB - 1) / kKvNB;          // 128-row tiles streamed
+  // half-step hs belongs to step hs / kKvNB and is its last one when:
+  auto closes_step = [&](int hs) { return (hs % kKvNB == kKvNB - 1) || hs == n_hs - 1; };
 
 
   if (tid == 0) {
@@ -531,7 +535,7 @@ bwd_dkdv_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
         const int sq = j % 3, so = j & 1;
         int h0, r0, e0, h1, r1, e1;
         next_item(h0, r0, e0);
-        h1 = h0; r1 = r0; e1 = e0;                              // a missing second item repeats the first
+        h1 = h0; r1 = r0; e1 = e0 & ~3;                         // a missing second item repeats the first block, as nobody's member
         if (BS == 64 && 2 * j + 1 < n_items) next_item(h1, r1, e1);
         if (j >= 2) ok = mbar_wait(bars + B_STE + so, ((j / 2) - 1) & 1, a.error_word, 40);
         if (!ok) break;
@@ -585,14 +589,14 @@ bwd_dkdv_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
       const uint32_t do_mn_lo = desc_lo(smem_u32(sDO), BwdTile<D>::kBox);
       bool ok = mbar_wait(bars + B_FIX, 0, a.error_word, 13);
 #pragma unroll 1
-      for (int hs = -2; hs < n_hs; ++hs) {   // half-steps -2 and -1 only issue S^T(0) and S^T(1)
+      for (int hs = -kKvNB; hs < n_hs; ++hs) {   // the first kKvNB rounds only issue S^T
         if (hs >= 0) {
-          const int j = hs >> 1, half = hs & 1, so = j & 1;
+          const int j = hs / kKvNB, half = hs % kKvNB, so = j & 1;
           if (half == 0) ok = ok && mbar_wait(bars + B_OF + so, (j / 2) & 1, a.error_word, 19);
           ok = ok && mbar_wait(bars + B_PF + half, j & 1, a.error_word, 9);
           if (ok) {
             tc_fence_after();
-            const uint32_t b_lo = do_mn_lo + so * (kTile >> 4) + half * 4 * (2048 >> 4);
+            const uint32_t b_lo = do_mn_lo + so * (kTile >> 4) + half * (kKvHalf / 16) * (2048 >> 4);
             const uint32_t a_t = tmem + kColS + half * kKvHalf;
 #pragma unroll
             for (int kk = 0; kk < kKvHalf / 16; ++kk)
@@ -600,9 +604,9 @@ bwd_dkdv_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
           }
           if (lead && closes_step(hs)) mma_commit(bars + B_OE + so);
         }
-        const int hn = hs + 2;
+        const int hn = hs + kKvNB;
         if (hn < n_hs) {
-          const int j = hn >> 1, half = hn & 1, sq = j % 3;
+          const int j = hn / kKvNB, half = hn % kKvNB, sq = j % 3;
           if (half == 0) ok = ok && mbar_wait(bars + B_QF + sq, (j / 3) & 1, a.error_word, 14);
           if (ok) {
             tc_fence_after();
@@ -632,13 +636,13 @@ bwd_dkdv_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
       const uint32_t q_mn_lo = desc_lo(smem_u32(sQ), BwdTile<D>::kBox);
       bool ok = mbar_wait(bars + B_FIX, 0, a.error_word, 5);
 #pragma unroll 1
-      for (int hs = -2; hs < n_hs; ++hs) {   // half-steps -2 and -1 only issue dP^T(0) and dP^T(1)
+      for (int hs = -kKvNB; hs < n_hs; ++hs) {   // the first kKvNB rounds only issue dP^T
         if (hs >= 0) {
-          const int j = hs >> 1, half = hs & 1, sq = j % 3;
+          const int j = hs / kKvNB, half = hs % kKvNB, sq = j % 3;
           ok = ok && mbar_wait(bars + B_DSF + half, j & 1, a.error_word, 15);
           if (ok) {
             tc_fence_after();
-            const uint32_t b_lo = q_mn_lo + sq * (kTile >> 4) + half * 4 * (2048 >> 4);
+            const uint32_t b_lo = q_mn_lo + sq * (kTile >> 4) + half * (kKvHalf / 16) * (2048 >> 4);
             const uint32_t a_t = tmem + kColDP + half * kKvHalf;
 #pragma unroll
             for (int kk = 0; kk < kKvHalf / 16; ++kk)
@@ -646,9 +650,9 @@ bwd_dkdv_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
           }
           if (lead && closes_step(hs)) mma_commit(bars + B_QE + sq);
         }
-        const int hn = hs + 2;
+        const int hn = hs + kKvNB;
         if (hn < n_hs) {
-          const int j = hn >> 1, half = hn & 1, so = j & 1;
+          const int j = hn / kKvNB, half = hn % kKvNB, so = j & 1;
           if (half == 0) ok = ok && mbar_wait(bars + B_OF + so, (j / 2) & 1, a.error_word, 6);
           if (ok) {
             tc_fence_after();
@@ -682,7 +686,7 @@ bwd_dkdv_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
     bool ok = true;
 #pragma unroll 1
     for (int hs = 0; hs < n_hs; ++hs) {
-      const int j = hs >> 1, half = hs & 1;
+      const int j = hs / kKvNB, half = hs % kKvNB;
       if (half == 0) {
         ok = mbar_wait(bars + B_STF + (j & 1), (j >> 1) & 1, a.error_word, 4);   // statistics and entries of step j
         ok = __all_sync(0xffffffffu, ok);
@@ -692,8 +696,9 @@ bwd_dkdv_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
       const float4* st_l = reinterpret_cast<const float4*>(sStat + (j & 1) * 256 + half * kKvHalf + g * C);
       const float4* st_d = st_l + 128 / 4;
       // the queries my columns hold, and from which of them on this key may be seen
-      const int entry = sEnt[(j & 1) * 2 + (BS == 64 ? half : 0)];
-      const int q0 = (entry >> 2) * BS + (BS == 128 ? kKvHalf * half : 0) + C * g;
+      const int col0 = half * kKvHalf + g * C;                 // my first column within the step's 128 queries
+      const int entry = sEnt[(j & 1) * 2 + (BS == 64 ? col0 / 64 : 0)];
+      const int q0 = (entry >> 2) * BS + (BS == 128 ? col0 : col0 % 64);
       const bool on = (entry >> member) & 1;
       const int xmin = on ? min(max(kj - q0, 0), C) : C;      // columns xmin <= c < xmax are visible
       const int xmax = (a.exact_w > 0 && kb_mine >= a.ns) ? min(max(kj + a.exact_w - q0, 0), C) : C;
