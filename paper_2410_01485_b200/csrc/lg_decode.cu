@@ -594,6 +594,10 @@ lg_status lg_sparse_decode(const lg_decode_params* p, const void* q, const void*
     int64_t n_cta = (max_tiles + 2 * kDecWarps - 1) / (2 * kDecWarps);
     if (n_cta > 2 * sms) n_cta = 2 * sms;
     if (n_cta > kDecFlatMaxCtas) n_cta = kDecFlatMaxCtas;
+    // A whole number of CTAs per unit when that costs at most a quarter of the CTAs: with equal
+    // lengths every slice then lies inside one unit (one pipeline fill, one record, one ticket per
+    // CTA instead of two); with mixed lengths the slices fall where they fall, as before.
+    if (units > 0 && n_cta > units && (n_cta / units) * units * 4 >= n_cta * 3) n_cta = (n_cta / units) * units;
     if (n_cta < 1) n_cta = 1;
     if (units > 0x7fffffff) return LG_ERR_UNSUPPORTED;
     // header word and per-unit counters start at zero; the records follow them
