@@ -147,13 +147,20 @@ lg_status lg_kv_ring_append(const lg_decode_params* p, void* k_cache, void* v_ca
 
 size_t lg_sparse_decode_workspace_bytes(const lg_decode_params* p);
 
+/* A decode workspace must be zero-filled once before its first use (this call, or any memset);
+ * every lg_sparse_decode call leaves it ready for the next one, so a serving loop pays no
+ * clearing per token.  (The first bytes hold the status word and one arrival counter per
+ * (sequence, kv head, head group); the CTA that completes a unit resets its counter.)  Call it
+ * again after a launch that failed.                                                       */
+lg_status lg_sparse_decode_workspace_init(void* workspace, size_t workspace_bytes, void* stream);
+
 /* One query token per sequence attends to every valid slot of its cache:
  * q [B,Hq,D], o [B,Hq,D] bf16; n_tokens (device int64 [B]) counts the tokens appended so
  * far, the current one included; slots holding no token yet are ignored; n_tokens == 0
  * gives o = 0, lse = -inf.  lse [B,Hq] fp32 is optional (NULL to skip).                 */
 lg_status lg_sparse_decode(const lg_decode_params* p, const void* q, const void* k_cache,
                            const void* v_cache, const int64_t* n_tokens, void* o, float* lse,
-                           void* workspace, size_t workspace_bytes, void* stream);
+                           void* workspace /* initialised, see above */, size_t workspace_bytes, void* stream);
 
 /* ---- a chunk of new tokens served against the cache (Section 3.2: in serving, the sparse
  *      layers keep only the sink and the most recent window of K,V) ---------------------- */
@@ -210,8 +217,9 @@ lg_status lg_chunk_prefill(const lg_decode_params* p, const void* q_chunk, const
  *   - The first call on each device looks up the array's device address (with that device
  *     current) and remembers it; make that first call outside any stream capture.
  *   - All calls on one device share the one array, and it keeps whatever the previous call
- *     left in it.  The call clears the status word at its start and overwrites every partial
- *     it later reads, so back-to-back calls on one stream are fine; two calls that can run
+ *     left in it.  The array starts zero-filled (it is a static object), every call resets the
+ *     arrival counters it used and overwrites every partial it later reads, so back-to-back
+ *     calls on one stream are fine; two calls that can run
  *     on the GPU at the same time (different streams, no dependency) race on the array and
  *     give undefined results.
  *   - The decode kernels contain no device-side waits, so there is no device status to read

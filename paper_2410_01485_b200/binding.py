@@ -53,6 +53,7 @@ SYMBOLS = {
     "lg_sparse_attn_bwd_profiled": (C.c_int, [C.POINTER(AttnParams)] + [_vp] * 9 + [_vp, _sz, _vp, C.POINTER(C.c_float)]),
     "lg_kv_ring_append": (C.c_int, [C.POINTER(DecodeParams), _vp, _vp, _vp, _vp, C.c_int32, _vp, _vp]),
     "lg_sparse_decode_workspace_bytes": (_sz, [C.POINTER(DecodeParams)]),
+    "lg_sparse_decode_workspace_init": (C.c_int, [_vp, _sz, _vp]),
     "lg_sparse_decode": (C.c_int, [C.POINTER(DecodeParams), _vp, _vp, _vp, _vp, _vp, _vp, _vp, _sz, _vp]),
     "lg_chunk_prefill_workspace_bytes": (_sz, [C.POINTER(DecodeParams), C.c_int32, C.c_int64]),
     "lg_chunk_prefill": (C.c_int, [C.POINTER(DecodeParams), _vp, _vp, _vp, _vp, _vp, C.c_int32, C.c_int64, _vp, _vp,
@@ -226,10 +227,14 @@ def lg_kv_ring_append(p: DecodeParams, k_cache, v_cache, k_new, v_new, n_tokens_
 
 
 def decode_workspace(p: DecodeParams, device="cuda") -> torch.Tensor:
+    """A workspace ready for lg_sparse_decode (allocated and zero-filled through the library's own call)."""
     n = load_library().lg_sparse_decode_workspace_bytes(C.byref(p))
     if n == 0:
         raise LgError(-1, "lg_sparse_decode_workspace_bytes")
-    return torch.empty(n, dtype=torch.uint8, device=device)
+    ws = torch.empty(n, dtype=torch.uint8, device=device)
+    _check(load_library().lg_sparse_decode_workspace_init(ws.data_ptr(), ws.numel(), _stream()),
+           "lg_sparse_decode_workspace_init")
+    return ws
 
 
 def lg_sparse_decode(p: DecodeParams, q, k_cache, v_cache, n_tokens, o=None, lse=None, workspace=None,

@@ -555,6 +555,12 @@ size_t lg_sparse_decode_workspace_bytes(const lg_decode_params* p) {
   return sizeof(WsHeader) + align_up(decode_part_bytes(p, choose_nsplit(p)), 256);
 }
 
+lg_status lg_sparse_decode_workspace_init(void* workspace, size_t workspace_bytes, void* stream) {
+  if (!workspace || (reinterpret_cast<uintptr_t>(workspace) & 255)) return LG_ERR_INVALID_ARG;
+  return cudaMemsetAsync(workspace, 0, workspace_bytes, static_cast<cudaStream_t>(stream)) == cudaSuccess ? LG_OK
+                                                                                                           : LG_ERR_CUDA;
+}
+
 lg_status lg_sparse_decode(const lg_decode_params* p, const void* q, const void* k_cache, const void* v_cache,
                            const int64_t* n_tokens, void* o, float* lse, void* workspace, size_t workspace_bytes,
                            void* stream) {
@@ -600,11 +606,11 @@ lg_status lg_sparse_decode(const lg_decode_params* p, const void* q, const void*
     if (units > 0 && n_cta > units && (n_cta / units) * units * 4 >= n_cta * 3) n_cta = (n_cta / units) * units;
     if (n_cta < 1) n_cta = 1;
     if (units > 0x7fffffff) return LG_ERR_UNSUPPORTED;
-    // header word and per-unit counters start at zero; the records follow them
+    // header word and per-unit counters are zero on entry (the caller zero-filled the workspace once,
+    // and the CTA that merges a unit re-arms its counter); the records follow them
     const size_t count_bytes = align_up(static_cast<size_t>(units) * sizeof(unsigned int), 256);
     a.unit_count = reinterpret_cast<unsigned int*>(static_cast<uint8_t*>(workspace) + sizeof(WsHeader));
     a.part = reinterpret_cast<float*>(static_cast<uint8_t*>(workspace) + sizeof(WsHeader) + count_bytes);
-    if (cudaMemsetAsync(workspace, 0, sizeof(WsHeader) + count_bytes, st) != cudaSuccess) return LG_ERR_CUDA;
     const int smem_flat = kDecWarps * kDecStages * 2 * kDecTile * p->D * 2 + (p->B + 1) * static_cast<int>(sizeof(int));
     if (p->D == 128) {
       if (cudaFuncSetAttribute(decode_stream_kernel<128>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem_flat) !=
@@ -676,8 +682,8 @@ lg_status lg_sparse_decode_static(const lg_decode_params* p, const void* q, cons
     return LG_ERR_WORKSPACE;
   void* scratch = nullptr;
   if ((s = static_scratch_address(&scratch)) != LG_OK) return s;
-  // Same kernels as lg_sparse_decode, with the array as their workspace.  Its header word is
-  // cleared by that call; the partials are fully rewritten before the merge kernel reads them.
+  // Same kernels as lg_sparse_decode, with the array as their workspace: a static array starts
+  // zero-filled, and every call leaves its counters at zero again.
   return lg_sparse_decode(p, q, k_cache, v_cache, n_tokens, o, lse, scratch, LG_DECODE_STATIC_SCRATCH_BYTES,
                           stream);
 }

@@ -432,3 +432,25 @@ def test_chunk_prefill_rejects_unsupported(lg):
     assert L.lg_chunk_prefill_workspace_bytes(C.byref(p), 64, 1000) > 0      # full ring: any fill level
     p2 = lg.decode_params(1, 2, 2, 128, 32, 128)
     assert L.lg_chunk_prefill_workspace_bytes(C.byref(p2), 64, 0) == 0       # sink not a multiple of 64
+
+
+def test_decode_workspace_is_reusable_without_clearing(lg):
+    """A decode workspace is zero-filled once (lg_sparse_decode_workspace_init) and then reused by calls
+    with different lengths and batch contents without any clearing in between; a dirty buffer becomes
+    usable through the same init call."""
+    B, Hq, Hkv, D, sink, W = 3, 16, 2, 128, 64, 512
+    p = lg.decode_params(B, Hq, Hkv, D, sink, W)
+    import ctypes as C
+    n = lg.load_library().lg_sparse_decode_workspace_bytes(C.byref(p))
+    ws = torch.full((n,), 0xAB, dtype=torch.uint8, device="cuda")          # dirty
+    lg._check(lg.load_library().lg_sparse_decode_workspace_init(ws.data_ptr(), ws.numel(), lg._stream()), "init")
+    g = torch.Generator(device="cuda").manual_seed(5)
+    kc = torch.randn(B, Hkv, sink + W, D, generator=g, device="cuda").to(torch.bfloat16)
+    vc = torch.randn(B, Hkv, sink + W, D, generator=g, device="cuda").to(torch.bfloat16)
+    q = torch.randn(B, Hq, D, generator=g, device="cuda").to(torch.bfloat16)
+    for ns in ([5000, 17, 300], [1, 576, 0], [64, 64, 9000], [5000, 17, 300]):
+        n_t = torch.tensor(ns, dtype=torch.int64, device="cuda")
+        o1, l1 = lg.lg_sparse_decode(p, q, kc, vc, n_t, workspace=ws)          # reused, never cleared
+        o2, l2 = lg.lg_sparse_decode(p, q, kc, vc, n_t)                        # fresh workspace
+        assert lg.lg_last_status(ws) == 0
+        assert torch.equal(o1, o2) and torch.equal(l1, l2)
