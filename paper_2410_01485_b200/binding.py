@@ -188,26 +188,79 @@ def lg_sparse_attn_bwd_profiled(p: AttnParams, q, k, v, o, lse, d_o, dq, dk, dv,
     return [float(x) for x in ms]
 
 
-def sparse_attn_fwd_bwd_host(p: AttnParams, host_in, host_out, dev=None):
+def sparse_attn_fwd_bwd_host(p: AttnParams, host_in, host_out, dev=None, head_groups: int = 4):
     """End-to-end training step with HOST buffers: copies pinned q, k, v, do to the device,
     runs lg_sparse_attn_fwd and lg_sparse_attn_bwd, and copies o, lse, dq, dk, dv back into the
     pinned tensors of `host_out`.  `dev` optionally supplies preallocated device buffers
-    (inputs dict, o, lse, dq, dk, dv, workspace).  All arithmetic runs in the CUDA library."""
+    (inputs dict, o, lse, dq, dk, dv, workspace or list of workspaces).  All arithmetic runs in
+    the CUDA library.
+
+    Heads are independent, so with B == 1 the step is cut into `head_groups` groups of kv heads
+    (with their query heads) that move through three streams: while one group computes, the next
+    one's inputs arrive and the previous one's results leave, and the two copy directions share the
+    link.  The library calls are the same, on strided views of the full tensors."""
     if dev is None:
         d_in = {k: torch.empty(v.shape, dtype=v.dtype, device="cuda") for k, v in host_in.items()}
         o = torch.empty_like(d_in["q"])
         lse = torch.empty(d_in["q"].shape[:3], dtype=torch.float32, device="cuda")
         dq, dk, dv = torch.empty_like(d_in["q"]), torch.empty_like(d_in["k"]), torch.empty_like(d_in["v"])
-        ws = attn_workspace(p, True)
+        ws = None
     else:
         d_in, o, lse, dq, dk, dv, ws = dev
-    for name in ("q", "k", "v", "do"):
-        d_in[name].copy_(host_in[name], non_blocking=True)
-    lg_sparse_attn_fwd(p, d_in["q"], d_in["k"], d_in["v"], o=o, lse=lse, workspace=ws)
-    lg_sparse_attn_bwd(p, d_in["q"], d_in["k"], d_in["v"], o, lse, d_in["do"], dq=dq, dk=dk, dv=dv, workspace=ws)
-    for name, t in (("o", o), ("lse", lse), ("dq", dq), ("dk", dk), ("dv", dv)):
-        host_out[name].copy_(t, non_blocking=True)
+    n_groups = head_groups if (p.B == 1 and head_groups > 1 and p.Hkv % head_groups == 0) else 1
+    if n_groups == 1:
+        ws = attn_workspace(p, True) if ws is None else (ws[0] if isinstance(ws, (list, tuple)) else ws)
+        for name in ("q", "k", "v", "do"):
+            d_in[name].copy_(host_in[name], non_blocking=True)
+        lg_sparse_attn_fwd(p, d_in["q"], d_in["k"], d_in["v"], o=o, lse=lse, workspace=ws)
+        lg_sparse_attn_bwd(p, d_in["q"], d_in["k"], d_in["v"], o, lse, d_in["do"], dq=dq, dk=dk, dv=dv, workspace=ws)
+        for name, t in (("o", o), ("lse", lse), ("dq", dq), ("dk", dk), ("dv", dv)):
+            host_out[name].copy_(t, non_blocking=True)
+        return host_out
+
+    G = p.Hq // p.Hkv
+    kv_per = p.Hkv // n_groups
+    pg = attn_params(p.B, kv_per * G, kv_per, p.L, p.D, p.block, p.mode, p.sink_tokens, p.window_tokens,
+                     p.stride_blocks, p.local_blocks, p.scale, bool(p.window_exact))
+    if not isinstance(ws, (list, tuple)) or len(ws) < n_groups:
+        ws = [attn_workspace(pg, True) for _ in range(n_groups)]   # groups overlap in time: one workspace each
+    cur = torch.cuda.current_stream()
+    s_in, s_cmp, s_out = (_side_stream(i) for i in range(3))
+    for st in (s_in, s_cmp, s_out):
+        st.wait_stream(cur)
+    for g in range(n_groups):
+        kv = slice(g * kv_per, (g + 1) * kv_per)
+        qh = slice(g * kv_per * G, (g + 1) * kv_per * G)
+        sl = {"q": qh, "k": kv, "v": kv, "do": qh}
+        ev_in, ev_cmp = torch.cuda.Event(), torch.cuda.Event()
+        with torch.cuda.stream(s_in):
+            for name in ("q", "k", "v", "do"):
+                d_in[name][:, sl[name]].copy_(host_in[name][:, sl[name]], non_blocking=True)
+            ev_in.record()
+        with torch.cuda.stream(s_cmp):
+            s_cmp.wait_event(ev_in)
+            qg, kg, vg, dog = (d_in[n][:, sl[n]] for n in ("q", "k", "v", "do"))
+            og, lg_ = o[:, qh], lse[:, qh]
+            lg_sparse_attn_fwd(pg, qg, kg, vg, o=og, lse=lg_, workspace=ws[g])
+            lg_sparse_attn_bwd(pg, qg, kg, vg, og, lg_, dog, dq=dq[:, qh], dk=dk[:, kv], dv=dv[:, kv], workspace=ws[g])
+            ev_cmp.record()
+        with torch.cuda.stream(s_out):
+            s_out.wait_event(ev_cmp)
+            for name, t, hs in (("o", o, qh), ("lse", lse, qh), ("dq", dq, qh), ("dk", dk, kv), ("dv", dv, kv)):
+                host_out[name][:, hs].copy_(t[:, hs], non_blocking=True)
+    for st in (s_in, s_cmp, s_out):
+        cur.wait_stream(st)
     return host_out
+
+
+_side_streams = {}
+
+
+def _side_stream(i: int) -> "torch.cuda.Stream":
+    key = (torch.cuda.current_device(), i)
+    if key not in _side_streams:
+        _side_streams[key] = torch.cuda.Stream()
+    return _side_streams[key]
 
 
 # ---------------------------------------------------------------------- decode / ring
