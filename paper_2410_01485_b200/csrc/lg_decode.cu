@@ -19,7 +19,11 @@
 
 namespace lg {
 
-constexpr int kDecWarps = 4;
+#ifndef LG_DEC_WARPS
+#define LG_DEC_WARPS 8
+#endif
+constexpr int kDecWarps = LG_DEC_WARPS;   // warps per CTA, each with its own pipeline of tiles
+constexpr int kDecThreads = kDecWarps * 32;
 constexpr int kDecStages = 3;
 constexpr int kDecTile = 16;          // tokens per warp tile
 constexpr int kDecHeads = 8;          // query heads per CTA (mma N)
@@ -76,7 +80,7 @@ __device__ __forceinline__ void mma16816(float* c, uint32_t a0, uint32_t a1, uin
 // CTA's (max, sum, O) record for its 8 heads is written to `out`.
 template <int D>
 __device__ __forceinline__ void decode_run_segment(const DecodeArgs& a, uint8_t* dsmem, int b, int kvh, int hg,
-                                                   int nvalid, int t_begin, int t_end, float* out) {
+                                                   int nvalid, int t_begin, int t_end, float* out, bool direct) {
   constexpr int kRowBytes = D * 2;
   constexpr int kChunks = D / 8;                      // 16-byte chunks per row
   constexpr int kTileBytes = kDecTile * kRowBytes;    // K (or V) bytes of one tile
@@ -196,7 +200,9 @@ __device__ __forceinline__ void decode_run_segment(const DecodeArgs& a, uint8_t*
   }
   cp_async_wait<0>();
 
-  // ---- warp partial -> shared, then merge the 4 warps in warp order -----------------------
+  // ---- warp partial -> shared, then merge the warps in warp order.  `direct`: this segment is the
+  // whole unit, so the merged result is final and goes straight to o / lse; otherwise it is the
+  // CTA's record for the cross-CTA merge ------------------------------------------------------
 #pragma unroll
   for (int o = 4; o < 32; o <<= 1) {
     l_run[0] += __shfl_xor_sync(0xffffffffu, l_run[0], o);
@@ -235,8 +241,17 @@ __device__ __forceinline__ void decode_run_segment(const DecodeArgs& a, uint8_t*
       acc += f * red[(w * kDecHeads + head) * kRec + d];
       l += f * red[(w * kDecHeads + head) * kRec + D + 1];
     }
-    out[head * kRec + d] = acc;
-    if (d == 0) { out[head * kRec + D] = m; out[head * kRec + D + 1] = l; }
+    if (direct) {
+      const int gh = hg * kDecHeads + head;
+      if (gh < a.G) {
+        const int64_t qh = static_cast<int64_t>(b) * a.Hq + kvh * a.G + gh;
+        a.o[qh * D + d] = __float2bfloat16(l > 0.f ? acc / l : 0.f);
+        if (d == 0 && a.lse) a.lse[qh] = l > 0.f ? (m + log2f(l)) * 0.6931471805599453f : -INFINITY;
+      }
+    } else {
+      out[head * kRec + d] = acc;
+      if (d == 0) { out[head * kRec + D] = m; out[head * kRec + D + 1] = l; }
+    }
   }
 }
 
@@ -254,7 +269,7 @@ __global__ void __launch_bounds__(kDecWarps * 32) decode_split_kernel(const Deco
   const int t_end = static_cast<int>(static_cast<int64_t>(ntile) * (wg + 1) / nw);
   constexpr int kRec = D + 2;
   float* out = a.part + ((static_cast<int64_t>(b) * gridDim.y + kg) * a.nsplit + split) * (kDecHeads * kRec);
-  decode_run_segment<D>(a, dsmem, b, kvh, hg, nvalid, t_begin, t_end, out);
+  decode_run_segment<D>(a, dsmem, b, kvh, hg, nvalid, t_begin, t_end, out, false);
 }
 
 // ---- flattened schedule ---------------------------------------------------------------------
@@ -272,11 +287,11 @@ __device__ __forceinline__ int decode_tiles_of(const DecodeArgs& a, int b) {
   return (nvalid + kDecTile - 1) / kDecTile;
 }
 
-// cum[b] = tiles of the sequences before b, b = 0 .. B (block of 128 threads; ends with a barrier)
+// cum[b] = tiles of the sequences before b, b = 0 .. B (block of kDecThreads threads; ends with a barrier)
 __device__ __forceinline__ void decode_build_cum(const DecodeArgs& a, int* cum) {
-  __shared__ int warp_sum[4];
+  __shared__ int warp_sum[kDecWarps];
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-  const int ipt = (a.B + 127) / 128;
+  const int ipt = (a.B + kDecThreads - 1) / kDecThreads;
   const int b0 = tid * ipt;
   int local = 0;
   for (int i = 0; i < ipt; ++i)
@@ -292,12 +307,12 @@ __device__ __forceinline__ void decode_build_cum(const DecodeArgs& a, int* cum) 
   for (int w = 0; w < warp; ++w) run += warp_sum[w];
   for (int i = 0; i < ipt; ++i)
     if (b0 + i < a.B) { cum[b0 + i] = run; run += decode_tiles_of(a, b0 + i); }
-  if (tid == 127) cum[a.B] = warp_sum[0] + warp_sum[1] + warp_sum[2] + warp_sum[3];
+  if (tid == kDecThreads - 1) cum[a.B] = run;   // the last thread's running total is the grand total
   __syncthreads();
 }
 
 // Merge the records of unit (b, k): CTAs first_cta .. first_cta + n_rec - 1, in that order
-// (whichever CTA happens to run this, the summation order is the same).  128 threads.
+// (whichever CTA happens to run this, the summation order is the same).  kDecThreads threads.
 template <int D>
 __device__ __forceinline__ void decode_merge_unit(const DecodeArgs& a, int b, int k, int64_t u, int first_cta,
                                                   int n_rec, int64_t total, int n_cta) {
@@ -309,12 +324,12 @@ __device__ __forceinline__ void decode_merge_unit(const DecodeArgs& a, int b, in
   auto empty_slice = [&](int c) { return total * c / n_cta == total * (c + 1) / n_cta; };
   // Each thread owns kOut outputs (all handled together so that the loads of one record are in
   // flight at once: the records sit in L2 and a dependent chain of loads would dominate).
-  constexpr int kOut = kDecHeads * D / 128;
+  constexpr int kOut = kDecHeads * D / kDecThreads;
   int head[kOut], dd[kOut];
   float m[kOut], acc[kOut], l[kOut];
 #pragma unroll
   for (int j = 0; j < kOut; ++j) {
-    const int idx = threadIdx.x + j * 128;
+    const int idx = threadIdx.x + j * kDecThreads;
     head[j] = idx / D;
     dd[j] = idx % D;
     m[j] = -INFINITY;
@@ -400,8 +415,11 @@ __global__ void __launch_bounds__(kDecWarps * 32) decode_stream_kernel(const Dec
     const int te = t0 + static_cast<int>(static_cast<int64_t>(n) * (warp + 1) / kDecWarps);
     const int64_t u = static_cast<int64_t>(b) * ups + k;
     __syncthreads();   // the previous segment's merge is done with shared memory
+    const bool direct = (t0 == 0 && n == nt);   // my segment is the whole unit: no record, no ticket
     decode_run_segment<D>(a, dsmem, b, k / a.HG, k % a.HG, nvalid, tb, te,
-                          a.part + (blockIdx.x + u) * (kDecHeads * kRec));
+                          a.part + (blockIdx.x + u) * (kDecHeads * kRec), direct);
+    pos += n;
+    if (direct) continue;
     // The CTA that delivers the last record of a unit merges it (records are read in index
     // order, so the result does not depend on which CTA that is) and re-arms the counter.
     __threadfence();
@@ -424,7 +442,6 @@ __global__ void __launch_bounds__(kDecWarps * 32) decode_stream_kernel(const Dec
       decode_merge_unit<D>(a, b, k, u, s_merge[1], s_merge[2], total, gridDim.x);
       if (threadIdx.x == 0) a.unit_count[u] = 0u;
     }
-    pos += n;
   }
 }
 
@@ -594,11 +611,14 @@ lg_status lg_sparse_decode(const lg_decode_params* p, const void* q, const void*
     if (cudaGetDevice(&dev) != cudaSuccess ||
         cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess)
       return LG_ERR_CUDA;
-    // two CTAs per SM, fewer when the cache is too small to give each warp a couple of tiles
+    // as many CTAs per SM as shared memory allows (at most two), fewer when the cache is too small to
+    // give each warp a couple of tiles
     const int64_t units = static_cast<int64_t>(p->B) * a.Hkv * a.HG;
     const int64_t max_tiles = units * ((a.C + kDecTile - 1) / kDecTile);
     int64_t n_cta = (max_tiles + 2 * kDecWarps - 1) / (2 * kDecWarps);
-    if (n_cta > 2 * sms) n_cta = 2 * sms;
+    const int64_t pipe_bytes = static_cast<int64_t>(kDecWarps) * kDecStages * 2 * kDecTile * p->D * 2;
+    const int per_sm = pipe_bytes * 2 + 4096 <= 227 * 1024 ? 2 : 1;
+    if (n_cta > per_sm * sms) n_cta = per_sm * sms;
     if (n_cta > kDecFlatMaxCtas) n_cta = kDecFlatMaxCtas;
     // A whole number of CTAs per unit when that costs at most a quarter of the CTAs: with equal
     // lengths every slice then lies inside one unit (one pipeline fill, one record, one ticket per
