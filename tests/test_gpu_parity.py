@@ -1,6 +1,6 @@
 """Parity of the CUDA path (through the C ABI) with the CPU fp64 oracle on a B200.
 
-Tolerances are the ones the task states: max-abs 1e-2 on O, 2e-2 on dQ/dK/dV, 1e-3 on LSE,
+Tolerances: max-abs 1e-2 on O, 2e-2 on dQ/dK/dV, 1e-3 on LSE,
 lists and ring contents bit-exact.  Outputs are bf16, whose grid spacing exceeds those
 bounds once |x| >= 4 (O) or |x| >= 8 (gradients): there the half-ulp bound 2^-8 * |x| of
 the output format itself is added, so the check is |err| <= tol + 2^-8 * |reference|.
