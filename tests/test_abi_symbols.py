@@ -85,3 +85,27 @@ def test_null_misaligned_and_small_workspace(lib):
     assert lib.lg_sparse_attn_fwd(C.byref(p), 256, 256, 256, 256, 256, 256, need, None) == -1
     assert lib.lg_build_block_index(C.byref(_good()), None, 256, 256, 256, None, None) == -1
     assert lib.lg_last_status(None, None) == -1
+
+
+def test_chunk_prefill_planning_on_host(lib):
+    """Sizes and limits of a chunk served against the ring are decided on the host."""
+    p = binding.decode_params(1, 4, 2, 128, 64, 128)
+    sz = lib.lg_chunk_prefill_workspace_bytes
+    assert sz(C.byref(p), 60, 0) == 0          # chunk not a multiple of 64
+    assert sz(C.byref(p), 64, 100) == 0        # ring not yet full: the fill level must be a multiple of 64
+    assert sz(C.byref(p), 64, -1) == 0
+    full, more = sz(C.byref(p), 64, 1000), sz(C.byref(p), 128, 1000)
+    assert 0 < full < more                     # a full ring: any fill level; longer chunk, more room
+    assert sz(C.byref(p), 64, 192) == full     # exactly full = full
+    assert sz(C.byref(p), 64, 64) < full       # fewer kept tokens, smaller copy
+    assert sz(C.byref(binding.decode_params(1, 4, 2, 128, 32, 128)), 64, 0) == 0    # sink not a multiple of 64
+    assert sz(C.byref(binding.decode_params(1, 4, 2, 96, 64, 128)), 64, 0) == 0     # head dimension
+    # argument checks come before any CUDA call
+    assert lib.lg_chunk_prefill(C.byref(p), None, 256, 256, 256, 256, 64, 1000, 256, 256, 256, full, None) == -1
+    assert lib.lg_chunk_prefill(C.byref(p), 256, 256, 256, 256, 256, 64, 1000, 256, 256, 128, full, None) == -1   # workspace alignment
+    assert lib.lg_chunk_prefill(C.byref(p), 256, 256, 256, 256, 256, 64, 1000, 256, 256, 256, full - 1, None) == -3
+
+
+def test_decode_workspace_init_rejects_bad_pointers(lib):
+    assert lib.lg_sparse_decode_workspace_init(None, 1024, None) == -1
+    assert lib.lg_sparse_decode_workspace_init(128, 1024, None) == -1   # not 256-byte aligned
