@@ -230,6 +230,18 @@ lg_status lg_sparse_decode_static(const lg_decode_params* p, const void* q, cons
                                   const void* v_cache, const int64_t* n_tokens, void* o, float* lse,
                                   void* stream);
 
+/* ---- self-test of the error path -------------------------------------------------------- */
+
+/* (The paper has no counterpart; this exists so that the error path can be exercised without
+ * breaking anything.)  Every device-side wait of the kernels has a time limit; when one expires,
+ * the waiting thread writes its site into the status word at the start of the workspace, all
+ * roles leave their loops, and lg_last_status() reports LG_ERR_DEVICE_TIMEOUT.  This call runs a
+ * one-warp kernel whose only wait can never be satisfied and whose limit is about a millisecond:
+ * afterwards lg_last_status(workspace, stream) must return LG_ERR_DEVICE_TIMEOUT once (and LG_OK
+ * on the next call), and the CUDA context is as usable as before.  workspace: device, 256-byte
+ * aligned, at least 256 bytes.                                                              */
+lg_status lg_selftest_wait_timeout(void* workspace, void* stream);
+
 /* ---- status ------------------------------------------------------------------------- */
 
 /* Synchronises `stream`, reads the error word the kernels keep at the start of

@@ -59,6 +59,7 @@ SYMBOLS = {
     "lg_chunk_prefill": (C.c_int, [C.POINTER(DecodeParams), _vp, _vp, _vp, _vp, _vp, C.c_int32, C.c_int64, _vp, _vp,
                                    _vp, _sz, _vp]),
     "lg_sparse_decode_static": (C.c_int, [C.POINTER(DecodeParams), _vp, _vp, _vp, _vp, _vp, _vp, _vp]),
+    "lg_selftest_wait_timeout": (C.c_int, [_vp, _vp]),
     "lg_last_status": (C.c_int, [_vp, _vp]),
     "lg_status_string": (C.c_char_p, [C.c_int]),
 }
@@ -341,6 +342,11 @@ def lg_sparse_decode_static(p: DecodeParams, q, k_cache, v_cache, n_tokens, o, l
                                                   lse.data_ptr() if lse is not None else None, _stream()),
            "lg_sparse_decode_static")
     return o, lse
+
+
+def lg_selftest_wait_timeout(workspace: torch.Tensor) -> None:
+    """Launch the one-warp kernel whose bounded wait must expire (see include/lg.h)."""
+    _check(load_library().lg_selftest_wait_timeout(workspace.data_ptr(), _stream()), "lg_selftest_wait_timeout")
 
 
 def lg_last_status(workspace: torch.Tensor) -> int:

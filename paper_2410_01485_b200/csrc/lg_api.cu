@@ -283,6 +283,18 @@ static lg_status plan_chunk(const lg_decode_params* p, int32_t T, int64_t n_befo
   c->total = c->o_v + c->lin_bytes;
   return LG_OK;
 }
+
+// ---- self-test of the bounded wait -----------------------------------------------------------
+// One thread waits on a barrier nobody will ever arrive at, with a limit of about a millisecond:
+// the wait gives up, records its site in the error word and the kernel ends normally.
+__global__ void wait_selftest_kernel(unsigned int* error_word, long long limit_cycles) {
+  __shared__ uint64_t bar;
+  if (threadIdx.x == 0) {
+    mbar_init(&bar, 1);
+    mbar_fence_init();
+    if (!mbar_try_wait(&bar, 0)) mbar_wait_slow(&bar, 0, error_word, 99, limit_cycles);
+  }
+}
 }  // namespace lg
 
 using namespace lg;
@@ -414,6 +426,16 @@ lg_status lg_chunk_prefill(const lg_decode_params* p, const void* q_chunk, const
   if (cudaGetLastError() != cudaSuccess) return LG_ERR_CUDA;
   if ((s = prepare_workspace(c.r, c.w, ws, false, st)) != LG_OK) return s;
   return launch_fwd(c.r, c.w, q_chunk, k_lin, v_lin, o, lse, ws, st);
+}
+
+lg_status lg_selftest_wait_timeout(void* workspace, void* stream) {
+  if (!workspace || (reinterpret_cast<uintptr_t>(workspace) & 255)) return LG_ERR_INVALID_ARG;
+  lg_status s = check_arch();
+  if (s != LG_OK) return s;
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  if (cudaMemsetAsync(workspace, 0, sizeof(WsHeader), st) != cudaSuccess) return LG_ERR_CUDA;
+  wait_selftest_kernel<<<1, 32, 0, st>>>(static_cast<unsigned int*>(workspace), 2000000ll);
+  return cudaGetLastError() == cudaSuccess ? LG_OK : LG_ERR_CUDA;
 }
 
 lg_status lg_last_status(void* workspace, void* stream) {

@@ -61,14 +61,14 @@ __device__ __forceinline__ bool mbar_try_wait(uint64_t* bar, uint32_t parity) {
 // never completed; callers then skip the rest of their work and fall through to cleanup.
 // The first probe is inlined: a wait that is already satisfied costs one try_wait.
 static __device__ __noinline__ bool mbar_wait_slow(uint64_t* bar, uint32_t parity, unsigned int* error_word,
-                                                   uint32_t site) {
+                                                   uint32_t site, long long limit_cycles = kWaitLimitCycles) {
   const long long t0 = clock64();
   for (;;) {
 #pragma unroll 1
     for (int it = 0; it < 256; ++it) {
       if (mbar_try_wait(bar, parity)) return true;
     }
-    if (clock64() - t0 > kWaitLimitCycles) break;
+    if (clock64() - t0 > limit_cycles) break;
   }
   if (error_word) atomicCAS(error_word, 0u, (1u << 24) | site);
   return false;

@@ -475,3 +475,19 @@ def test_host_buffer_step_equals_device_calls(lg):
         torch.cuda.synchronize()
         for name, ref in (("o", o), ("lse", lse), ("dq", dq), ("dk", dk), ("dv", dv)):
             assert torch.equal(h_out[name], ref.cpu()), (groups, name)
+
+
+def test_expired_wait_is_reported_and_leaves_the_context_usable(lg):
+    """The error path end to end, without breaking anything: a wait that cannot be satisfied gives up after
+    its limit, the status word carries it to the host once, and the same workspace then serves a forward."""
+    cfg = synth.CFG1
+    p = lg.params_of(cfg)
+    ws = lg.attn_workspace(p, False)
+    lg.lg_selftest_wait_timeout(ws)
+    assert lg.lg_last_status(ws) == -5          # LG_ERR_DEVICE_TIMEOUT
+    assert lg.lg_last_status(ws) == 0           # reported once, then cleared
+    inp = synth.make_attn_inputs(cfg, "cuda", seed=0, with_do=False)
+    o, lse = lg.lg_sparse_attn_fwd(p, inp["q"], inp["k"], inp["v"], workspace=ws)
+    assert lg.lg_last_status(ws) == 0
+    Oo, LSE = O.attn_forward(*(synth.to_f64(inp[x][0]) for x in ("q", "k", "v")), O.Pattern.of(cfg), 1.0 / np.sqrt(cfg.D))[:2]
+    _assert_close(synth.to_f64(o[0]), Oo, TOL_O, "O")
