@@ -24,12 +24,15 @@ Readings of points on which the paper is silent:
   - the strided comb is absolute: KV block kb is retained iff kb % stride == 0;
   - LSE is the natural log of the sum of exp of the *scaled* scores;
   - the backward formulas are the derivatives of the definition (the paper
-    inherits them from FlashAttention and prints none).
+    inherits them from FlashAttention and prints none);
+  - documents packed into one sample: the paper masks nothing across them; the
+    optional doc_start array adds "no key of an earlier document" to the pattern.
 
 Pins (tests/test_oracle_*.py): brute-force per-row softmax, torch's dense causal
 attention and autograd in fp64, central finite differences, closed-form block
 counts, the paper's KV-cache arithmetic; the chunk-against-cache function (T decode
-steps) against the rows of the mask-based forward and against explicit loops.  Trained-model quality: parity unpinned
+steps) against the rows of the mask-based forward and against explicit loops; the
+document option against torch attention run on each document separately.  Trained-model quality: parity unpinned
 and out of scope.
 """
 from __future__ import annotations
@@ -57,6 +60,11 @@ class Pattern:
     stride_blocks: int = 0
     local_blocks: int = 0
     window_exact: bool = False   # sink + window only: the window edge is token-exact (i - j < window_tokens)
+    # packed documents (Section 4.1 packs documents, each opened by <bos>, into one training sample):
+    # doc_start[i] = position of the first token of the document that token i belongs to; when given,
+    # a query sees no key of an earlier document.  The paper describes no such masking; it is an
+    # option on top of the static pattern, which itself stays in absolute positions.
+    doc_start: Optional[np.ndarray] = None
 
     @staticmethod
     def of(cfg) -> "Pattern":
@@ -74,6 +82,8 @@ def allowed(p: Pattern, i, j):
     i = np.asarray(i, dtype=np.int32)
     j = np.asarray(j, dtype=np.int32)
     causal = j <= i
+    if p.doc_start is not None:
+        causal = causal & (j >= np.asarray(p.doc_start, dtype=np.int32)[i])
     if p.mode == MODE_FULL_CAUSAL:
         return causal
     qb = i // p.block

@@ -119,6 +119,20 @@ def make_decode_inputs(cfg: DecodeConfig, device="cpu", seed: int = 0, capacity:
     }
 
 
+def make_doc_start(L: int, seed: int = 0, mean_len: int = 700, device="cpu") -> torch.Tensor:
+    """doc_start[i] (int32 [L]) for documents packed back to back into a sample of L tokens: lengths are
+    drawn from a seeded exponential distribution with the given mean (a few long documents, many short
+    ones, as in a web corpus), at least 1 token each; the last document is cut at L."""
+    gen = torch.Generator().manual_seed(seed)
+    out = torch.empty(L, dtype=torch.int32)
+    pos = 0
+    while pos < L:
+        n = max(1, int(-mean_len * torch.log(1.0 - torch.rand(1, generator=gen)).item()))
+        out[pos:pos + n] = pos
+        pos += n
+    return out.to(device)
+
+
 def to_f64(t: torch.Tensor):
     """Exact widening of a bf16/fp32 tensor to a float64 numpy array (host)."""
     return t.detach().to("cpu").to(torch.float64).numpy()

@@ -568,3 +568,64 @@ def test_chunk_prefill_ignores_evicted_tokens():
     k2[:, n0 - window + 1] += 1.0            # the oldest token the first chunk token still sees
     o3, _ = O.chunk_prefill(q, k2, v2, n0, sink, window, 0.3)
     assert not np.array_equal(o3[:, 0], o[:, 0]) and np.array_equal(o3[:, 1:], o[:, 1:])
+
+
+# --------------------------------------------------------------------- packed documents
+
+def _doc_bounds(L, cuts):
+    ds = np.zeros(L, dtype=np.int32)
+    for a, b in zip(cuts[:-1], cuts[1:]):
+        ds[a:b] = a
+    return ds
+
+
+def test_documents_full_causal_equals_torch_per_document():
+    """Full causal attention with the document option is plain causal attention run on every document by
+    itself: forward and all three gradients against torch (fp64 SDPA / autograd), document by document."""
+    rng = np.random.default_rng(21)
+    L, D, cuts = 320, 16, [0, 37, 38, 130, 256, 320]      # one-token document, block-straddling cuts
+    q = rng.standard_normal((2, L, D)); k = rng.standard_normal((1, L, D)); v = rng.standard_normal((1, L, D))
+    do = rng.standard_normal((2, L, D))
+    scale = 0.31
+    p = O.Pattern(L, 64, O.MODE_FULL_CAUSAL, doc_start=_doc_bounds(L, cuts))
+    dQ, dK, dV, Oo, LSE = O.attn_backward(q, k, v, do, p, scale)
+    for a, b in zip(cuts[:-1], cuts[1:]):
+        tq = torch.tensor(q[:, a:b], requires_grad=True); tk = torch.tensor(k[:, a:b], requires_grad=True)
+        tv = torch.tensor(v[:, a:b], requires_grad=True)
+        s = scale * tq @ tk.expand(2, -1, -1).transpose(1, 2)
+        s = s.masked_fill(~torch.tril(torch.ones(b - a, b - a, dtype=torch.bool)), float("-inf"))
+        out = torch.softmax(s, dim=-1) @ tv.expand(2, -1, -1)
+        (out * torch.tensor(do[:, a:b])).sum().backward()
+        np.testing.assert_allclose(Oo[:, a:b], out.detach().numpy(), rtol=0, atol=1e-12)
+        np.testing.assert_allclose(LSE[:, a:b], torch.logsumexp(s, dim=-1).detach().numpy(), rtol=0, atol=1e-12)
+        np.testing.assert_allclose(dQ[:, a:b], tq.grad.numpy(), rtol=0, atol=1e-11)
+        np.testing.assert_allclose(dK[:, a:b], tk.grad.numpy(), rtol=0, atol=1e-11)
+        np.testing.assert_allclose(dV[:, a:b], tv.grad.numpy(), rtol=0, atol=1e-11)
+
+
+def test_documents_with_window_are_the_pattern_and_the_document_mask():
+    """With a sparse pattern the option only removes pairs: allowed = pattern AND same document, written out
+    with loops; and an exact window without sink is translation invariant, so each document by itself
+    (positions restarting at 0) gives the same rows."""
+    L, cuts = 256, [0, 100, 101, 256]
+    ds = _doc_bounds(L, cuts)
+    for base in (O.Pattern(L, 64, O.MODE_SINK_WINDOW, sink_tokens=64, window_tokens=128),
+                 O.Pattern(L, 64, O.MODE_STRIDED_LOCAL, stride_blocks=2, local_blocks=1),
+                 O.Pattern(L, 64, O.MODE_SINK_WINDOW, sink_tokens=0, window_tokens=64, window_exact=True)):
+        withd = O.Pattern(base.L, base.block, base.mode, base.sink_tokens, base.window_tokens, base.stride_blocks,
+                          base.local_blocks, base.window_exact, doc_start=ds)
+        m0, m1 = O.token_mask(base), O.token_mask(withd)
+        for i in range(L):
+            for j in range(L):
+                assert m1[i, j] == (m0[i, j] and j >= ds[i])
+    rng = np.random.default_rng(22)
+    D = 8
+    q = rng.standard_normal((1, L, D)); k = rng.standard_normal((1, L, D)); v = rng.standard_normal((1, L, D))
+    o, lse = O.attn_forward(q, k, v, withd, 0.4)[:2]
+    for a, b in zip(cuts[:-1], cuts[1:]):
+        n = b - a
+        npad = (n + 63) // 64 * 64          # the per-document run needs a multiple of the block
+        pad = lambda x: np.concatenate([x[:, a:b], np.zeros((1, npad - n, D))], axis=1)
+        od, ld = O.attn_forward(pad(q), pad(k), pad(v), O.Pattern(npad, 64, O.MODE_SINK_WINDOW, 0, 64, window_exact=True), 0.4)[:2]
+        np.testing.assert_allclose(o[:, a:b], od[:, :n], rtol=0, atol=1e-12)
+        np.testing.assert_allclose(lse[:, a:b], ld[:, :n], rtol=0, atol=1e-12)
