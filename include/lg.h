@@ -71,6 +71,14 @@ typedef struct {
      strides, dK / dV the K / V strides.  All zero selects contiguous [B, H, L, D].
      Every stride must be a multiple of 8 elements (16 bytes).                              */
   int64_t q_strides[3], k_strides[3], v_strides[3], o_strides[3];
+  /* Packed documents (optional; the paper packs documents, each opened by <bos>, into one
+     sample and describes no masking between them): NULL, or a DEVICE int32 array [B, L],
+     contiguous, with doc_start[b][i] = position of the first token of the document token i
+     belongs to (non-decreasing in i, <= i).  When given, a query sees no key of an earlier
+     document, on top of the pattern (which stays in absolute positions: the sink blocks are
+     those of the sample, so only its first document sees them).  The block lists are those
+     of the pattern alone; blocks that the documents empty are computed and masked.          */
+  const int32_t* doc_start;
 } lg_attn_params;
 
 /* ---- block-index builder (Section 3.2: the mask is kept in compressed-sparse-row form,

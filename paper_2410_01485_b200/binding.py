@@ -31,7 +31,7 @@ class AttnParams(C.Structure):
                 ("window_tokens", C.c_int32), ("stride_blocks", C.c_int32), ("local_blocks", C.c_int32),
                 ("window_exact", C.c_int32), ("scale", C.c_float),
                 ("q_strides", C.c_int64 * 3), ("k_strides", C.c_int64 * 3), ("v_strides", C.c_int64 * 3),
-                ("o_strides", C.c_int64 * 3)]
+                ("o_strides", C.c_int64 * 3), ("doc_start", C.c_void_p)]
 
 
 class DecodeParams(C.Structure):
@@ -99,8 +99,14 @@ def _strides3(t: torch.Tensor):
 
 
 def attn_params(B, Hq, Hkv, L, D, block, mode, sink_tokens=0, window_tokens=0, stride_blocks=0, local_blocks=0,
-                scale=0.0, window_exact=False) -> AttnParams:
+                scale=0.0, window_exact=False, doc_start=None) -> AttnParams:
+    """doc_start: optional CUDA int32 tensor [B, L] (first position of each token's document); the params
+    object keeps a reference to it."""
     p = AttnParams()
+    if doc_start is not None:
+        assert doc_start.dtype == torch.int32 and doc_start.is_contiguous() and tuple(doc_start.shape) == (B, L)
+        p.doc_start = doc_start.data_ptr()
+        p._doc_start_ref = doc_start
     p.B, p.Hq, p.Hkv, p.L, p.D, p.block, p.mode = B, Hq, Hkv, L, D, block, mode
     p.sink_tokens, p.window_tokens, p.stride_blocks, p.local_blocks = sink_tokens, window_tokens, stride_blocks, local_blocks
     p.scale = scale
@@ -108,11 +114,11 @@ def attn_params(B, Hq, Hkv, L, D, block, mode, sink_tokens=0, window_tokens=0, s
     return p
 
 
-def params_of(cfg, scale: float = 0.0) -> AttnParams:
+def params_of(cfg, scale: float = 0.0, doc_start=None) -> AttnParams:
     """AttnParams from a synth.AttnConfig-like object."""
     return attn_params(cfg.B, cfg.Hq, cfg.Hkv, cfg.L, cfg.D, cfg.block, cfg.mode, cfg.sink_tokens,
                        cfg.window_tokens, cfg.stride_blocks, cfg.local_blocks, scale,
-                       getattr(cfg, "window_exact", False))
+                       getattr(cfg, "window_exact", False), doc_start)
 
 
 # ------------------------------------------------------------------------------ index

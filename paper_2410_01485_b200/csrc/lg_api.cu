@@ -78,6 +78,8 @@ lg_status resolve(const lg_attn_params* p, Resolved* r) {
   r->n_stiles = (p->L + 255) / 256;
   r->q_start = 0;
   r->Lq = p->L;
+  if (reinterpret_cast<uintptr_t>(p->doc_start) & 3) return LG_ERR_INVALID_ARG;
+  r->doc_start = p->doc_start;
   // nnz from the per-row counts of each pattern
   int64_t nnz = 0;
   const PatternDev& pt = r->pat;
@@ -124,6 +126,7 @@ WsLayout ws_layout(const Resolved& r, bool want_bwd) {
     w.kt_order = take(r.n_ktiles * 4);
     w.kt_cols = take(static_cast<size_t>(r.n_ktiles) * 2 * 4);
     w.kt_off = take((static_cast<size_t>(r.n_ktiles) + 1) * 4);
+    if (r.doc_start) w.doc_end = take(static_cast<size_t>(r.B) * r.L * 4);
     w.delta = take(static_cast<size_t>(r.B) * r.Hq * r.L * 8);   // two planes: -LSE * log2 e and -delta per query row
   }
   w.total = off;
@@ -162,6 +165,10 @@ lg_status prepare_workspace(const Resolved& r, const WsLayout& w, uint8_t* ws, b
     kv_tile_merge_kernel<<<(nt + 127) / 128, 128, 0, stream>>>(i32(w.col_ptr), i32(w.row_idx), i32(w.kt_cols),
                                                                i32(w.kt_off), R, nt, i32(w.kt_cnt), i32(w.kt_ent));
     tile_order_kernel<<<(nt + 127) / 128, 128, 0, stream>>>(i32(w.kt_cnt), nt, i32(w.kt_order));
+    if (r.doc_start) {
+      const int64_t n = static_cast<int64_t>(r.B) * r.L;
+      doc_end_kernel<<<static_cast<unsigned>((n + 255) / 256), 256, 0, stream>>>(r.doc_start, i32(w.doc_end), r.B, r.L);
+    }
   }
   return cudaGetLastError() == cudaSuccess ? LG_OK : LG_ERR_CUDA;
 }

@@ -27,6 +27,8 @@ static lg_status launch_bwd_t(const Resolved& r, const WsLayout& w, const void* 
   a.error_word = reinterpret_cast<unsigned int*>(ws);
   a.L = r.L; a.Hq = r.Hq; a.Hkv = r.Hkv; a.G = r.G;
   a.exact_w = r.exact_w; a.ns = r.pat.ns;
+  a.doc_start = r.doc_start;
+  a.doc_end = r.doc_start ? reinterpret_cast<const int32_t*>(ws + w.doc_end) : nullptr;
   a.scale = r.scale;
   a.scale_log2 = r.scale * 1.4426950408889634f;
   constexpr int smem = BwdSmem<D, BS>::kTotal;

@@ -43,6 +43,8 @@ struct BwdArgs {
   int64_t s0[3], s1[3];      // strides of out0 / out1 (batch, head, token; elements)
   int L, Hq, Hkv, G;
   int exact_w, ns;           // token-exact window (0: off) and number of sink blocks
+  const int32_t* doc_start;  // [B, L] first position of each token's document, or null
+  const int32_t* doc_end;    // [B, L] end of each token's document (null together with doc_start)
   float scale, scale_log2;
 };
 
@@ -333,6 +335,7 @@ bwd_dq_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ 
       nlse2 = a.stat[row];
       ndlt = a.stat[a.stat_plane + row];
     }
+    const int dstart = (a.doc_start && qi < a.L) ? a.doc_start[static_cast<int64_t>(b) * a.L + qi] : 0;   // start of my document
     // entry of the step: read one step ahead so that the load is off the critical path
     auto entry_of = [&](int j, bool& have) {
       int e = (BS == 128) ? j : 2 * j + (g >> 1);
@@ -349,7 +352,8 @@ bwd_dq_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ 
       const int key0 = (entry >> 2) * BS + (BS == 128 ? C * g : C * (g & 1));
       const bool on = have && ((entry >> member) & 1);
       const int lim = on ? min(max(qi - key0 + 1, 0), C) : 0;   // columns lo <= c < lim are visible
-      const int lo = (a.exact_w > 0 && (entry >> 2) >= a.ns) ? min(max(qi - a.exact_w + 1 - key0, 0), C) : 0;
+      const int lo_abs = (a.exact_w > 0 && (entry >> 2) >= a.ns) ? max(dstart, qi - a.exact_w + 1) : dstart;
+      const int lo = min(max(lo_abs - key0, 0), C);
       const uint32_t s_addr = lane_addr + kColS + (j & 1) * 128 + g * C;
 
       ok = mbar_wait(bars + B_SF + (j & 1), (j >> 1) & 1, a.error_word, 31);
@@ -681,6 +685,8 @@ bwd_dkdv_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
     const int member = (R == 1) ? 0 : (r / BS);
     const int kb_mine = (R == 2 && member) ? kb_b : kb_a;
     const int kj = kb_mine * BS + (R == 2 ? (r & (BS - 1)) : r);   // this thread's key (kb_mine < 0: none)
+    // end of my key's document: queries from there on do not see it (no documents: never)
+    const int dend = (a.doc_end && kb_mine >= 0 && kj < a.L) ? a.doc_end[static_cast<int64_t>(b) * a.L + kj] : (1 << 30);
     const uint32_t lane_addr = tmem + (static_cast<uint32_t>((warp & 3) * 32) << 16);
     const uint64_t scale2 = f32x2(a.scale_log2, a.scale_log2);
     bool ok = true;
@@ -701,7 +707,8 @@ bwd_dkdv_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
       const int q0 = (entry >> 2) * BS + (BS == 128 ? col0 : col0 % 64);
       const bool on = (entry >> member) & 1;
       const int xmin = on ? min(max(kj - q0, 0), C) : C;      // columns xmin <= c < xmax are visible
-      const int xmax = (a.exact_w > 0 && kb_mine >= a.ns) ? min(max(kj + a.exact_w - q0, 0), C) : C;
+      const int hi_abs = (a.exact_w > 0 && kb_mine >= a.ns) ? min(dend, kj + a.exact_w) : dend;   // first query that no longer sees me
+      const int xmax = min(max(hi_abs - q0, 0), C);
       const uint32_t s_addr = lane_addr + kColS + half * kKvHalf + g * C;
       const uint32_t dp_addr = lane_addr + kColDP + half * kKvHalf + g * C;
 

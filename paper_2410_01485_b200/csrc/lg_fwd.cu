@@ -24,6 +24,7 @@ static lg_status launch_fwd_t(const Resolved& r, const WsLayout& w, const void* 
   a.L = r.L; a.Hq = r.Hq; a.G = r.G;
   a.q_start = r.q_start; a.Lq = r.Lq;
   a.exact_w = r.exact_w; a.ns = r.pat.ns;
+  a.doc_start = r.doc_start;
   a.scale_log2 = r.scale * 1.4426950408889634f;
   auto kern = fwd_kernel<D, BS>;
   constexpr int smem = FwdSmem<D>::kTotal;

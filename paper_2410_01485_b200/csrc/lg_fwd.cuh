@@ -37,6 +37,7 @@ struct FwdArgs {
   int q_start, Lq;           // queries exist for rows [q_start, q_start + Lq) of the L key positions only
                              // (a chunk served against a cache); Q, O, LSE are indexed by row - q_start
   int exact_w, ns;           // token-exact window (0: off) and number of sink blocks
+  const int32_t* doc_start;  // [B, L] first position of each query's document, or null
   float scale_log2;          // scale * log2(e)
 };
 
@@ -244,6 +245,9 @@ fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUt
     const int member = s * RS + (BS == 128 ? 0 : (r >> 6));  // pattern row of the super-tile
     const uint32_t lane_addr = tmem + (static_cast<uint32_t>((warp & 3) * 32) << 16);
     const uint32_t my_s = lane_addr + kColS + s * 128, my_o = lane_addr + kColO + s * 128;
+    // lowest key position this row may see outside what the pattern already excludes: the start of its
+    // document (0 without documents)
+    const int dstart = (a.doc_start && qi < a.L && qi >= a.q_start) ? a.doc_start[static_cast<int64_t>(b) * a.L + qi] : 0;
     float m_ref = -INFINITY;   // reference maximum (scaled, log2 domain) the probabilities are relative to
     float l_run = 0.f;
     int p0 = 0, p1 = 0;        // P tiles published per half buffer (barrier phases)
@@ -269,7 +273,8 @@ fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUt
         // token-exact window, on blocks outside the sink)
         const int key0 = (e >> 4) * BS + (BS == 128 ? 64 * hf : 0);
         const int lim = ((e >> member) & 1) ? min(max(qi - key0 + 1, 0), 64) : 0;
-        const int lo = (a.exact_w > 0 && (e >> 4) >= a.ns) ? min(max(qi - a.exact_w + 1 - key0, 0), 64) : 0;
+        const int lo_abs = (a.exact_w > 0 && (e >> 4) >= a.ns) ? max(dstart, qi - a.exact_w + 1) : dstart;
+        const int lo = min(max(lo_abs - key0, 0), 64);
 
         ok = mbar_wait_warp(bars + B_SF + s * 2 + hf, (hf ? p1 : p0) & 1, a.error_word, 12);
         if (!ok) break;

@@ -22,6 +22,7 @@ struct Resolved {          // validated, defaulted copy of lg_attn_params
   int n_qtiles, n_ktiles;  // ceil(L / 128)
   int n_stiles;            // ceil(L / 256): super-tiles of the forward
   int q_start, Lq;         // forward only: queries exist for rows [q_start, q_start + Lq) (0, L by default)
+  const int32_t* doc_start;  // device [B, L] or null: first position of each token's document
   int64_t nnz;
 };
 
@@ -34,6 +35,7 @@ struct WsLayout {
   size_t sq_cnt, sq_ent, sq_order;               // super-tile schedules (forward)
   size_t kt_cnt, kt_ent, kt_order;               // kv-tile schedules (dK/dV pass)
   size_t kt_cols, kt_off;                        // members of each kv tile, start of its schedule
+  size_t doc_end;                                // int32 [B, L]: end of each token's document (bwd with documents only)
   size_t delta;                                  // 2 x float [B, Hq, L]: -LSE * log2 e, then -delta (bwd only)
   size_t total;
 };

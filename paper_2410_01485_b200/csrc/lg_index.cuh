@@ -207,4 +207,20 @@ __global__ void kv_tile_merge_kernel(const int32_t* __restrict__ col_ptr, const 
   tile_cnt[t] = n;
 }
 
+// doc_end[b][j] = end (one past the last token) of the document token j belongs to, from
+// doc_start[b][i] = first token of token i's document (non-decreasing): the first i > j whose
+// document starts after j, found by bisection, or L.
+__global__ void doc_end_kernel(const int32_t* __restrict__ doc_start, int32_t* __restrict__ doc_end, int B, int L) {
+  const int64_t gid = static_cast<int64_t>(blockIdx.x) * blockDim.x + threadIdx.x;
+  if (gid >= static_cast<int64_t>(B) * L) return;
+  const int j = static_cast<int>(gid % L);
+  const int32_t* ds = doc_start + (gid - j);
+  int lo = j, hi = L;            // ds[lo] <= j (its own document); ds[hi] > j, with ds[L] taken as +inf
+  while (hi - lo > 1) {
+    const int mid = (lo + hi) >> 1;
+    if (ds[mid] > j) hi = mid; else lo = mid;
+  }
+  doc_end[gid] = hi;
+}
+
 }  // namespace lg

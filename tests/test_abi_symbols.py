@@ -109,3 +109,13 @@ def test_chunk_prefill_planning_on_host(lib):
 def test_decode_workspace_init_rejects_bad_pointers(lib):
     assert lib.lg_sparse_decode_workspace_init(None, 1024, None) == -1
     assert lib.lg_sparse_decode_workspace_init(128, 1024, None) == -1   # not 256-byte aligned
+
+
+def test_document_array_must_be_aligned(lib):
+    p = _good()
+    need = lib.lg_sparse_attn_workspace_bytes(C.byref(p), 1)
+    p.doc_start = 258                          # not 4-byte aligned
+    assert lib.lg_sparse_attn_workspace_bytes(C.byref(p), 1) == 0
+    p.doc_start = 256
+    assert lib.lg_sparse_attn_workspace_bytes(C.byref(p), 1) > need      # the backward keeps the documents' ends
+    assert lib.lg_sparse_attn_workspace_bytes(C.byref(p), 0) == lib.lg_sparse_attn_workspace_bytes(C.byref(_good()), 0)

@@ -165,9 +165,9 @@ def test_exact_window_training_mask_is_the_decode_mask(lg):
 
 # ------------------------------------------------------------------------ full-size configs
 
-def _check_rows(lg, cfg, inp, o, lse, dq, heads, slabs):
+def _check_rows(lg, cfg, inp, o, lse, dq, heads, slabs, pat=None):
     scale = 1.0 / np.sqrt(cfg.D)
-    pat = O.Pattern.of(cfg)
+    pat = O.Pattern.of(cfg) if pat is None else pat
     G = cfg.Hq // cfg.Hkv
     for h in heads:
         q = synth.to_f64(inp["q"][0, h:h + 1])
@@ -183,9 +183,9 @@ def _check_rows(lg, cfg, inp, o, lse, dq, heads, slabs):
                 _assert_close(synth.to_f64(dq[0, h, r0:r1]), dQ[0], TOL_G, "dQ h%d r%d" % (h, r0))
 
 
-def _check_keys(cfg, inp, dk, dv, kv_heads, key_ranges):
+def _check_keys(cfg, inp, dk, dv, kv_heads, key_ranges, pat=None):
     scale = 1.0 / np.sqrt(cfg.D)
-    pat = O.Pattern.of(cfg)
+    pat = O.Pattern.of(cfg) if pat is None else pat
     G = cfg.Hq // cfg.Hkv
     for g in kv_heads:
         q = synth.to_f64(inp["q"][0, g * G:(g + 1) * G])
@@ -491,3 +491,69 @@ def test_expired_wait_is_reported_and_leaves_the_context_usable(lg):
     assert lg.lg_last_status(ws) == 0
     Oo, LSE = O.attn_forward(*(synth.to_f64(inp[x][0]) for x in ("q", "k", "v")), O.Pattern.of(cfg), 1.0 / np.sqrt(cfg.D))[:2]
     _assert_close(synth.to_f64(o[0]), Oo, TOL_O, "O")
+
+
+# ------------------------------------------------------------------------- packed documents
+
+DOC_CASES = [
+    replace(synth.CFG1, name="docs_full_causal", mode=synth.MODE_FULL_CAUSAL, L=1024, D=128, Hq=4, Hkv=2),
+    replace(synth.CFG1, name="docs_sink_window", L=1024, D=128),
+    replace(synth.CFG1, name="docs_window_bs128", block=128, sink_tokens=0, window_tokens=256, L=1536, D=64),
+    replace(synth.CFG1, name="docs_exact_window", window_exact=True, sink_tokens=0, window_tokens=128, L=768, D=128),
+    replace(synth.CFG1, name="docs_strided_gqa4_b2", mode=synth.MODE_STRIDED_LOCAL, stride_blocks=4, local_blocks=2,
+            L=1024, D=128, Hq=4, Hkv=1, B=2),
+]
+
+
+@pytest.mark.parametrize("cfg", DOC_CASES, ids=lambda c: c.name)
+def test_documents_fwd_bwd_parity(lg, cfg):
+    """Packed documents (no key of an earlier document) on top of every pattern: forward and backward against
+    the oracle; document lengths are seeded, differ per batch element, and include very short documents."""
+    ds = torch.stack([synth.make_doc_start(cfg.L, seed=7 + b, mean_len=150) for b in range(cfg.B)]).cuda()
+    first = int((ds[0] == 0).sum())                        # cut the first document of sequence 0 into 1 + 2 + rest
+    assert first > 3
+    ds[0, 1:3] = 1
+    ds[0, 3:first] = 3
+    assert bool((ds[:, 1:] >= ds[:, :-1]).all())           # doc_start is non-decreasing
+    p = lg.params_of(cfg, doc_start=ds)
+    inp = synth.make_attn_inputs(cfg, "cuda", seed=1, with_do=True)
+    ws = lg.attn_workspace(p, True)
+    o, lse = lg.lg_sparse_attn_fwd(p, inp["q"], inp["k"], inp["v"], workspace=ws)
+    assert lg.lg_last_status(ws) == 0
+    dq, dk, dv = lg.lg_sparse_attn_bwd(p, inp["q"], inp["k"], inp["v"], o, lse, inp["do"], workspace=ws)
+    assert lg.lg_last_status(ws) == 0
+    scale = 1.0 / np.sqrt(cfg.D)
+    for b in range(cfg.B):
+        pat = replace(O.Pattern.of(cfg), doc_start=ds[b].cpu().numpy())
+        q, k, v, do = (synth.to_f64(inp[x][b]) for x in ("q", "k", "v", "do"))
+        dQ, dK, dV, Oo, LSE = O.attn_backward(q, k, v, do, pat, scale, rows_per_slab=cfg.block)
+        _assert_close(synth.to_f64(o[b]), Oo, TOL_O, "O")
+        assert np.abs(synth.to_f64(lse[b]) - LSE).max() <= TOL_LSE
+        _assert_close(synth.to_f64(dq[b]), dQ, TOL_G, "dQ")
+        _assert_close(synth.to_f64(dk[b]), dK, TOL_G, "dK")
+        _assert_close(synth.to_f64(dv[b]), dV, TOL_G, "dV")
+    # without the array the same call is the plain pattern (the pointer is optional)
+    p0 = lg.params_of(cfg)
+    o0, _ = lg.lg_sparse_attn_fwd(p0, inp["q"], inp["k"], inp["v"])
+    assert not torch.equal(o0, o)
+
+
+def test_documents_32k_sampled(lg):
+    """The 128K training pattern (sink 128 + window 4096, 128-token blocks) on 8 heads x 32K tokens of packed
+    documents: row slabs and key ranges around document boundaries against the oracle."""
+    cfg = replace(synth.CFG3, name="docs_32k", Hq=8, Hkv=8, L=32768)
+    ds = synth.make_doc_start(cfg.L, seed=3, mean_len=3000)
+    starts = sorted(set(int(x) for x in ds.tolist()))
+    assert len(starts) > 4
+    p = lg.params_of(cfg, doc_start=ds.view(1, -1).cuda())
+    inp = synth.make_attn_inputs(cfg, "cuda", seed=4)
+    ws = lg.attn_workspace(p, True)
+    o, lse = lg.lg_sparse_attn_fwd(p, inp["q"], inp["k"], inp["v"], workspace=ws)
+    dq, dk, dv = lg.lg_sparse_attn_bwd(p, inp["q"], inp["k"], inp["v"], o, lse, inp["do"], workspace=ws)
+    assert lg.lg_last_status(ws) == 0
+    pat = replace(O.Pattern.of(cfg), doc_start=ds.numpy())
+    b1, b2 = starts[1], starts[len(starts) // 2]           # two document boundaries
+    slabs = [0, (b1 // 128) * 128, (b2 // 128) * 128, min((b2 // 128) * 128 + 4096, cfg.L - 128), cfg.L - 128]
+    _check_rows(lg, cfg, inp, o, lse, dq, heads=[0, 5], slabs=slabs, pat=pat)
+    keys = [(0, 128), ((b2 // 128) * 128 - 128, (b2 // 128) * 128 + 128), (cfg.L - 128, cfg.L)]
+    _check_keys(cfg, inp, dk, dv, kv_heads=[3], key_ranges=keys, pat=pat)
