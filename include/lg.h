@@ -58,7 +58,7 @@ typedef enum {
  * Grouped-query attention: query head h reads kv head h / (Hq / Hkv).
  */
 typedef struct {
-  int32_t B, Hq, Hkv, L, D;   /* Hq % Hkv == 0; D in {64, 128}; L % block == 0               */
+  int32_t B, Hq, Hkv, L, D;   /* Hq % Hkv == 0; D in {64, 128}; L >= 1 (the last block may be partial) */
   int32_t block;              /* pattern granularity in tokens: 64 or 128                    */
   int32_t mode;               /* lg_mode                                                     */
   int32_t sink_tokens;        /* SINK_WINDOW: multiple of block (may be 0)                   */

@@ -51,7 +51,8 @@ MODE_STRIDED_LOCAL = 2
 
 @dataclass(frozen=True)
 class Pattern:
-    """Static sparse pattern (Section 3.1).  Token counts must be multiples of `block`."""
+    """Static sparse pattern (Section 3.1).  Sink and window token counts are multiples of `block`;
+    L need not be (the last block is then partial)."""
     L: int
     block: int
     mode: int
@@ -115,12 +116,14 @@ def block_lists(p: Pattern):
     Returns int32 arrays (row_ptr[nB+1], col_idx[nnz], col_ptr[nB+1], row_idx[nnz]);
     rows ascending in kb, columns ascending in qb."""
     Bs = p.block
-    nB = p.L // Bs
+    nB = -(-p.L // Bs)                 # the last block may be partial
     active = np.zeros((nB, nB), dtype=bool)
 
     def one_block_row(qb):
-        m = token_mask(p, qb * Bs, (qb + 1) * Bs)                  # [Bs, L]
-        active[qb] = m.reshape(Bs, nB, Bs).any(axis=(0, 2))
+        m = token_mask(p, qb * Bs, min(p.L, (qb + 1) * Bs))        # [<= Bs, L]
+        full = np.zeros((m.shape[0], nB * Bs), dtype=bool)
+        full[:, :p.L] = m
+        active[qb] = full.reshape(m.shape[0], nB, Bs).any(axis=(0, 2))
 
     # a plain parallel-for over block rows (numpy releases the GIL inside its loops)
     with ThreadPoolExecutor(max_workers=os.cpu_count() or 1) as pool:
@@ -140,7 +143,7 @@ def count_pairs(p: Pattern) -> int:
     """Number of allowed (i, j) pairs for one head, counted from the explicit mask."""
     Bs = p.block
     with ThreadPoolExecutor(max_workers=os.cpu_count() or 1) as pool:
-        return sum(pool.map(lambda r0: int(token_mask(p, r0, r0 + Bs).sum()), range(0, p.L, Bs)))
+        return sum(pool.map(lambda r0: int(token_mask(p, r0, min(p.L, r0 + Bs)).sum()), range(0, p.L, Bs)))
 
 
 # ------------------------------------------------------------------------- forward

@@ -134,7 +134,7 @@ def lg_build_block_index(p: AttnParams, device="cuda") -> Tuple[torch.Tensor, to
     """Returns device int32 tensors (row_ptr, col_idx, col_ptr, row_idx)."""
     lib = load_library()
     nnz = lg_block_index_nnz(p)
-    nB = p.L // p.block
+    nB = -(-p.L // p.block)
     assert lib.lg_block_index_bytes(C.byref(p)) == 4 * (2 * (nB + 1) + 2 * nnz)
     row_ptr = torch.empty(nB + 1, dtype=torch.int32, device=device)
     col_ptr = torch.empty(nB + 1, dtype=torch.int32, device=device)

@@ -38,12 +38,12 @@ lg_status resolve(const lg_attn_params* p, Resolved* r) {
   if (!p || !r) return LG_ERR_INVALID_ARG;
   if (p->B < 1 || p->Hq < 1 || p->Hkv < 1 || p->L < 1 || p->Hq % p->Hkv != 0) return LG_ERR_INVALID_ARG;
   if (p->block != 64 && p->block != 128) return LG_ERR_INVALID_ARG;
-  if (p->L % p->block != 0) return LG_ERR_INVALID_ARG;
+  if (p->L < 1) return LG_ERR_INVALID_ARG;   // L need not be a multiple of the block: the last block is then partial
   if (p->D != 64 && p->D != 128) return LG_ERR_UNSUPPORTED;
   if (!(p->scale >= 0.f) || isinf(p->scale)) return LG_ERR_INVALID_ARG;
   r->B = p->B; r->Hq = p->Hq; r->Hkv = p->Hkv; r->L = p->L; r->D = p->D; r->block = p->block;
   r->mode = p->mode; r->G = p->Hq / p->Hkv;
-  r->pat.nB = p->L / p->block;
+  r->pat.nB = (p->L + p->block - 1) / p->block;
   r->pat.mode = p->mode;
   r->pat.ns = r->pat.nw = r->pat.stride = r->pat.nl = 0;
   r->exact_w = 0;
@@ -127,7 +127,7 @@ WsLayout ws_layout(const Resolved& r, bool want_bwd) {
     w.kt_cols = take(static_cast<size_t>(r.n_ktiles) * 2 * 4);
     w.kt_off = take((static_cast<size_t>(r.n_ktiles) + 1) * 4);
     if (r.doc_start) w.doc_end = take(static_cast<size_t>(r.B) * r.L * 4);
-    w.delta = take(static_cast<size_t>(r.B) * r.Hq * r.L * 8);   // two planes: -LSE * log2 e and -delta per query row
+    w.delta = take(static_cast<size_t>(r.B) * r.Hq * align_up(r.L, 128) * 8);   // rows padded to whole tiles   // two planes: -LSE * log2 e and -delta per query row
   }
   w.total = off;
   return w;

@@ -12,18 +12,20 @@ static lg_status launch_bwd_t(const Resolved& r, const WsLayout& w, const void* 
   float* stat = reinterpret_cast<float*>(ws + w.delta);
   if (marks) cudaEventRecord(marks[0], stream);
   {
-    const int64_t rows = static_cast<int64_t>(r.B) * r.Hq * r.L;
+    const int Lp = static_cast<int>(align_up(r.L, 128));
+    const int64_t rows = static_cast<int64_t>(r.B) * r.Hq * Lp;
     const int64_t threads = rows * (D / 8);
     const int64_t blocks = (threads + 255) / 256;
     if (blocks > 0x7fffffff) return LG_ERR_UNSUPPORTED;
     delta_kernel<D><<<static_cast<unsigned>(blocks), 256, 0, stream>>>(
         static_cast<const __nv_bfloat16*>(o), static_cast<const __nv_bfloat16*>(d_o), lse, stat, r.os[0], r.os[1],
-        r.os[2], r.Hq, r.L, rows);
+        r.os[2], r.Hq, r.L, Lp, rows);
   }
   if (marks) cudaEventRecord(marks[1], stream);
   BwdArgs a;
   a.stat = stat;
-  a.stat_plane = static_cast<int64_t>(r.B) * r.Hq * r.L;
+  a.Lp = static_cast<int>(align_up(r.L, 128));
+  a.stat_plane = static_cast<int64_t>(r.B) * r.Hq * a.Lp;
   a.error_word = reinterpret_cast<unsigned int*>(ws);
   a.L = r.L; a.Hq = r.Hq; a.Hkv = r.Hkv; a.G = r.G;
   a.exact_w = r.exact_w; a.ns = r.pat.ns;

@@ -35,8 +35,10 @@ struct BwdArgs {
   const int32_t* tile_cnt;
   const int32_t* tile_ent;   // idx * 4 + member mask
   const int32_t* order;
-  const float* stat;         // two planes of [B, Hq, L] floats: -LSE * log2(e), then -delta
+  const float* stat;         // two planes of [B, Hq, Lp] floats: -LSE * log2(e), then -delta; Lp = L rounded up
+                             // to 128 (rows past L hold zeros, so that whole-tile copies stay inside a head)
   int64_t stat_plane;        // floats per plane
+  int Lp;
   __nv_bfloat16* out0;       // dQ   | dK
   __nv_bfloat16* out1;       // unused | dV
   unsigned int* error_word;
@@ -54,15 +56,17 @@ struct BwdArgs {
 template <int D>
 __global__ void delta_kernel(const __nv_bfloat16* __restrict__ o, const __nv_bfloat16* __restrict__ d_o,
                              const float* __restrict__ lse, float* __restrict__ stat, int64_t sb, int64_t sh,
-                             int64_t sl, int Hq, int L, int64_t total_rows) {
+                             int64_t sl, int Hq, int L, int Lp, int64_t total_rows) {
+  // rows are numbered over the padded length Lp; rows i >= L of a head exist only in `stat`, as zeros
   constexpr int TPR = D / 8;   // threads per row, 16 bytes each
   const int64_t gid = static_cast<int64_t>(blockIdx.x) * blockDim.x + threadIdx.x;
   const int64_t row = gid / TPR;
   const int ch = static_cast<int>(gid % TPR);
   float acc = 0.f;
-  if (row < total_rows) {
-    const int i = static_cast<int>(row % L);
-    const int64_t bh = row / L;
+  const int i = static_cast<int>(row % Lp);
+  const bool real = row < total_rows && i < L;
+  if (real) {
+    const int64_t bh = row / Lp;
     const int h = static_cast<int>(bh % Hq);
     const int64_t b = bh / Hq;
     const int64_t off = b * sb + h * sh + static_cast<int64_t>(i) * sl + ch * 8;
@@ -79,7 +83,7 @@ __global__ void delta_kernel(const __nv_bfloat16* __restrict__ o, const __nv_bfl
 #pragma unroll
   for (int s = TPR / 2; s > 0; s >>= 1) acc += __shfl_xor_sync(0xffffffffu, acc, s);
   if (row < total_rows && ch == 0) {
-    stat[row] = -lse[row] * 1.4426950408889634f;
+    stat[row] = real ? -lse[(row / Lp) * L + i] * 1.4426950408889634f : 0.f;
     stat[total_rows + row] = -acc;
   }
 }
@@ -331,7 +335,7 @@ bwd_dq_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ 
     const uint32_t lane_addr = tmem + (static_cast<uint32_t>((warp & 3) * 32) << 16);
     float nlse2 = 0.f, ndlt = 0.f;   // -LSE2 and -delta of my row
     if (qi < a.L) {
-      const int64_t row = (static_cast<int64_t>(b) * a.Hq + h) * a.L + qi;
+      const int64_t row = (static_cast<int64_t>(b) * a.Hq + h) * a.Lp + qi;
       nlse2 = a.stat[row];
       ndlt = a.stat[a.stat_plane + row];
     }
@@ -406,11 +410,11 @@ bwd_dq_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ 
     if (ok) {
       tc_fence_after();
       constexpr int kEpi = 32;                     // output columns per thread
-      if (qi < a.L && g * kEpi < D) {              // warp-uniform: L is a multiple of 64
+      if (g * kEpi < D) {                          // warp-uniform; rows past L take part in the loads only
         __nv_bfloat16* dq_row = a.out0 + b * a.s0[0] + h * a.s0[1] + static_cast<int64_t>(qi) * a.s0[2] + g * kEpi;
         if (n_steps > 0) {
-          store_acc_cols<kEpi>(lane_addr + kColDQ + g * kEpi, dq_row, a.scale, true);
-        } else {
+          store_acc_cols<kEpi>(lane_addr + kColDQ + g * kEpi, dq_row, a.scale, qi < a.L);
+        } else if (qi < a.L) {
 #pragma unroll
           for (int x = 0; x < kEpi; x += 8) *reinterpret_cast<uint4*>(dq_row + x) = make_uint4(0, 0, 0, 0);
         }
@@ -547,8 +551,8 @@ bwd_dkdv_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
         sEnt[so * 2 + 1] = e1;
         mbar_expect_tx(bars + B_STF + so, 2 * 128 * 4);         // (release: publishes the entries as well)
         {
-          const float* st0 = a.stat + (static_cast<int64_t>(b) * a.Hq + h0) * a.L + r0;
-          const float* st1 = a.stat + (static_cast<int64_t>(b) * a.Hq + h1) * a.L + r1;
+          const float* st0 = a.stat + (static_cast<int64_t>(b) * a.Hq + h0) * a.Lp + r0;
+          const float* st1 = a.stat + (static_cast<int64_t>(b) * a.Hq + h1) * a.Lp + r1;
 #pragma unroll
           for (int pl = 0; pl < 2; ++pl) {
             float* dst = sStat + (so * 2 + pl) * 128;
@@ -685,8 +689,9 @@ bwd_dkdv_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
     const int member = (R == 1) ? 0 : (r / BS);
     const int kb_mine = (R == 2 && member) ? kb_b : kb_a;
     const int kj = kb_mine * BS + (R == 2 ? (r & (BS - 1)) : r);   // this thread's key (kb_mine < 0: none)
-    // end of my key's document: queries from there on do not see it (no documents: never)
-    const int dend = (a.doc_end && kb_mine >= 0 && kj < a.L) ? a.doc_end[static_cast<int64_t>(b) * a.L + kj] : (1 << 30);
+    // end of my key's document: queries from there on do not see it (no documents: the end of the sequence,
+    // which also keeps the rows a partial last block lacks out of the sums)
+    const int dend = (a.doc_end && kb_mine >= 0 && kj < a.L) ? a.doc_end[static_cast<int64_t>(b) * a.L + kj] : a.L;
     const uint32_t lane_addr = tmem + (static_cast<uint32_t>((warp & 3) * 32) << 16);
     const uint64_t scale2 = f32x2(a.scale_log2, a.scale_log2);
     bool ok = true;
@@ -786,13 +791,14 @@ bwd_dkdv_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
     if (ok) {
       tc_fence_after();
       constexpr int kEpi = 32;                               // output columns per thread
+      const bool mine = kj < a.L;                            // keys past L take part in the loads only
       if (kb_mine >= 0 && g * kEpi < D) {
         __nv_bfloat16* dk_row = a.out0 + b * a.s0[0] + hk * a.s0[1] + static_cast<int64_t>(kj) * a.s0[2] + g * kEpi;
         __nv_bfloat16* dv_row = a.out1 + b * a.s1[0] + hk * a.s1[1] + static_cast<int64_t>(kj) * a.s1[2] + g * kEpi;
         if (n_hs > 0) {
-          store_acc_cols<kEpi>(lane_addr + kColDV + g * kEpi, dv_row, 1.0f, true);
-          store_acc_cols<kEpi>(lane_addr + kColDK + g * kEpi, dk_row, a.scale, true);
-        } else {
+          store_acc_cols<kEpi>(lane_addr + kColDV + g * kEpi, dv_row, 1.0f, mine);
+          store_acc_cols<kEpi>(lane_addr + kColDK + g * kEpi, dk_row, a.scale, mine);
+        } else if (mine) {
 #pragma unroll
           for (int x = 0; x < kEpi; x += 8) {
             *reinterpret_cast<uint4*>(dk_row + x) = make_uint4(0, 0, 0, 0);

@@ -346,7 +346,10 @@ fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUt
     }
     // ---- epilogue: O / l -> bf16, LSE ------------------------------------------------------
     if (ok) ok = wait_o(14);
-    if (ok && p0 + p1 > 0 && qi < a.L && qi >= a.q_start) {   // warp-uniform: L and q_start are multiples of 64
+    // warp-uniform condition (q_start is a multiple of 64, the tensor-memory loads below need the whole
+    // warp); with a partial last block the rows past L load with the others and store nothing
+    if (ok && p0 + p1 > 0 && qi - lane < a.L && qi >= a.q_start) {
+      const bool mine = qi < a.L;
       tc_fence_after();
       const float inv_l = l_run > 0.f ? 1.f / l_run : 0.f;
       __nv_bfloat16* orow =
@@ -363,11 +366,12 @@ fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUt
           v4.y = pack_bf16(__uint_as_float(oreg[x + 2]) * inv_l, __uint_as_float(oreg[x + 3]) * inv_l);
           v4.z = pack_bf16(__uint_as_float(oreg[x + 4]) * inv_l, __uint_as_float(oreg[x + 5]) * inv_l);
           v4.w = pack_bf16(__uint_as_float(oreg[x + 6]) * inv_l, __uint_as_float(oreg[x + 7]) * inv_l);
-          *reinterpret_cast<uint4*>(orow + c * 32 + x) = v4;
+          if (mine) *reinterpret_cast<uint4*>(orow + c * 32 + x) = v4;
         }
       }
-      a.lse[(static_cast<int64_t>(b) * a.Hq + h) * a.Lq + qi - a.q_start] =
-          l_run > 0.f ? (m_ref + log2f(l_run)) * 0.6931471805599453f : -INFINITY;
+      if (mine)
+        a.lse[(static_cast<int64_t>(b) * a.Hq + h) * a.Lq + qi - a.q_start] =
+            l_run > 0.f ? (m_ref + log2f(l_run)) * 0.6931471805599453f : -INFINITY;
     }
   }
   tc_fence_before();

@@ -5,7 +5,7 @@
 namespace lg {
 
 struct PatternDev {
-  int nB;       // L / block
+  int nB;       // ceil(L / block)
   int mode;     // 0 full causal, 1 sink+window, 2 strided+local
   int ns, nw;   // sink blocks, window blocks (own block included; one more when the window is token-exact)
   int stride, nl;

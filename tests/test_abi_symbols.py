@@ -48,7 +48,7 @@ def test_nnz_and_sizes_on_host(lib):
 
 @pytest.mark.parametrize("mutate", [
     lambda p: setattr(p, "Hkv", 3),                 # Hq % Hkv != 0
-    lambda p: setattr(p, "L", 500),                 # L % block != 0
+    lambda p: setattr(p, "L", 0),                   # empty sequence
     lambda p: setattr(p, "block", 32),
     lambda p: setattr(p, "sink_tokens", 10),        # not a multiple of block
     lambda p: setattr(p, "window_tokens", 0),       # window < block
@@ -119,3 +119,12 @@ def test_document_array_must_be_aligned(lib):
     p.doc_start = 256
     assert lib.lg_sparse_attn_workspace_bytes(C.byref(p), 1) > need      # the backward keeps the documents' ends
     assert lib.lg_sparse_attn_workspace_bytes(C.byref(p), 0) == lib.lg_sparse_attn_workspace_bytes(C.byref(_good()), 0)
+
+
+def test_partial_last_block_is_accepted(lib):
+    p = _good()
+    full = lib.lg_block_index_nnz(C.byref(p))
+    p.L = p.L - 37                              # last block partial: same number of blocks, same lists
+    assert lib.lg_block_index_nnz(C.byref(p)) == full
+    p.L = p.L - 64                              # one block fewer
+    assert 0 < lib.lg_block_index_nnz(C.byref(p)) < full

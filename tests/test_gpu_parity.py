@@ -557,3 +557,54 @@ def test_documents_32k_sampled(lg):
     _check_rows(lg, cfg, inp, o, lse, dq, heads=[0, 5], slabs=slabs, pat=pat)
     keys = [(0, 128), ((b2 // 128) * 128 - 128, (b2 // 128) * 128 + 128), (cfg.L - 128, cfg.L)]
     _check_keys(cfg, inp, dk, dv, kv_heads=[3], key_ranges=keys, pat=pat)
+
+
+# ------------------------------------------------------------------------- L not a multiple of the block
+
+RAGGED = [
+    replace(synth.CFG1, name="ragged_bs64", L=1000, D=128, Hq=4, Hkv=2),
+    replace(synth.CFG1, name="ragged_bs128_d64", block=128, sink_tokens=128, window_tokens=256, L=1100),
+    replace(synth.CFG1, name="ragged_full_causal", mode=synth.MODE_FULL_CAUSAL, L=777, D=128),
+    replace(synth.CFG1, name="ragged_exact_strided_b2", mode=synth.MODE_STRIDED_LOCAL, stride_blocks=4, local_blocks=2,
+            L=1301, D=128, Hq=4, Hkv=1, B=2),
+    replace(synth.CFG1, name="ragged_exact_window", window_exact=True, L=449, D=64),
+    replace(synth.CFG1, name="ragged_shorter_than_a_block", L=40, D=128),
+]
+
+
+@pytest.mark.parametrize("cfg", RAGGED, ids=lambda c: c.name)
+def test_partial_last_block_parity(lg, cfg):
+    """L that ends inside a block (odd lengths included): lists bit-exact, forward and backward against the
+    oracle, and nothing written past L (outputs live in buffers with a sentinel row after the end)."""
+    p = lg.params_of(cfg)
+    got = lg.lg_build_block_index(p)
+    ref = O.block_lists(O.Pattern.of(cfg))
+    for g, r in zip(got, ref):
+        assert np.array_equal(g.cpu().numpy(), r)
+    inp = synth.make_attn_inputs(cfg, "cuda", seed=3, with_do=True)
+    ws = lg.attn_workspace(p, True)
+    o, lse = lg.lg_sparse_attn_fwd(p, inp["q"], inp["k"], inp["v"], workspace=ws)
+    assert lg.lg_last_status(ws) == 0
+    dq, dk, dv = lg.lg_sparse_attn_bwd(p, inp["q"], inp["k"], inp["v"], o, lse, inp["do"], workspace=ws)
+    assert lg.lg_last_status(ws) == 0
+    scale = 1.0 / np.sqrt(cfg.D)
+    pat = O.Pattern.of(cfg)
+    for b in range(cfg.B):
+        q, k, v, do = (synth.to_f64(inp[x][b]) for x in ("q", "k", "v", "do"))
+        dQ, dK, dV, Oo, LSE = O.attn_backward(q, k, v, do, pat, scale, rows_per_slab=cfg.block)
+        _assert_close(synth.to_f64(o[b]), Oo, TOL_O, "O")
+        assert np.abs(synth.to_f64(lse[b]) - LSE).max() <= TOL_LSE
+        _assert_close(synth.to_f64(dq[b]), dQ, TOL_G, "dQ")
+        _assert_close(synth.to_f64(dk[b]), dK, TOL_G, "dK")
+        _assert_close(synth.to_f64(dv[b]), dV, TOL_G, "dV")
+    # the last sequence's last head ends the buffers: write into larger ones and look behind the end
+    pad = 3 * cfg.D
+    def padded(t):
+        buf = torch.full((t.numel() + pad,), -7.0, dtype=t.dtype, device="cuda")
+        return buf, buf[:t.numel()].view(t.shape)
+    bo, o2 = padded(o); bq, dq2 = padded(dq); bk, dk2 = padded(dk); bv, dv2 = padded(dv)
+    lg.lg_sparse_attn_fwd(p, inp["q"], inp["k"], inp["v"], o=o2, lse=lse, workspace=ws)
+    lg.lg_sparse_attn_bwd(p, inp["q"], inp["k"], inp["v"], o2, lse, inp["do"], dq=dq2, dk=dk2, dv=dv2, workspace=ws)
+    torch.cuda.synchronize()
+    for buf, view, ref_t in ((bo, o2, o), (bq, dq2, dq), (bk, dk2, dk), (bv, dv2, dv)):
+        assert torch.equal(view, ref_t) and bool((buf[-pad:] == -7.0).all())

@@ -629,3 +629,31 @@ def test_documents_with_window_are_the_pattern_and_the_document_mask():
         od, ld = O.attn_forward(pad(q), pad(k), pad(v), O.Pattern(npad, 64, O.MODE_SINK_WINDOW, 0, 64, window_exact=True), 0.4)[:2]
         np.testing.assert_allclose(o[:, a:b], od[:, :n], rtol=0, atol=1e-12)
         np.testing.assert_allclose(lse[:, a:b], ld[:, :n], rtol=0, atol=1e-12)
+
+
+# --------------------------------------------------------------------- L not a multiple of the block
+
+def test_partial_last_block_is_a_prefix_of_the_padded_problem():
+    """Causal attention never looks ahead, so the first L rows of a longer, block-aligned problem are the
+    answer for L (forward; and gradients when dO is zero past L); block lists are those of the aligned
+    problem cut to ceil(L / block) blocks; full causal with a ragged L against torch."""
+    rng = np.random.default_rng(31)
+    L, Lp, D = 200, 256, 8
+    q = rng.standard_normal((2, Lp, D)); k = rng.standard_normal((1, Lp, D)); v = rng.standard_normal((1, Lp, D))
+    do = rng.standard_normal((2, Lp, D)); do[:, L:] = 0.0
+    for mk in (lambda n: O.Pattern(n, 64, O.MODE_SINK_WINDOW, sink_tokens=64, window_tokens=64),
+               lambda n: O.Pattern(n, 64, O.MODE_STRIDED_LOCAL, stride_blocks=2, local_blocks=1),
+               lambda n: O.Pattern(n, 64, O.MODE_SINK_WINDOW, sink_tokens=0, window_tokens=64, window_exact=True),
+               lambda n: O.Pattern(n, 64, O.MODE_FULL_CAUSAL)):
+        dQ, dK, dV, Oo, LSE = O.attn_backward(q[:, :L], k[:, :L], v[:, :L], do[:, :L], mk(L), 0.5)
+        dQp, dKp, dVp, Op, LSEp = O.attn_backward(q, k, v, do, mk(Lp), 0.5)
+        for a, b in ((Oo, Op), (LSE, LSEp), (dQ, dQp), (dK, dKp), (dV, dVp)):
+            np.testing.assert_allclose(a, b[:, :L], rtol=0, atol=1e-12)
+        rp, ci, cp, ri = O.block_lists(mk(L))
+        rpp, cip, cpp, rip = O.block_lists(mk(Lp))
+        nB = 4
+        assert len(rp) == nB + 1 and np.array_equal(rp, rpp[:nB + 1]) and np.array_equal(ci, cip[:rp[-1]])
+        assert O.count_pairs(mk(L)) == int(O.token_mask(mk(Lp))[:L, :L].sum())
+    tq = torch.tensor(q[:, :L]); tk = torch.tensor(k[:, :L]).expand(2, -1, -1); tv = torch.tensor(v[:, :L]).expand(2, -1, -1)
+    ref = torch.nn.functional.scaled_dot_product_attention(tq, tk, tv, is_causal=True, scale=0.5)
+    np.testing.assert_allclose(Oo, ref.numpy(), rtol=0, atol=1e-12)
