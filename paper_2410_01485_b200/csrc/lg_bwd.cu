@@ -13,13 +13,12 @@ static lg_status launch_bwd_t(const Resolved& r, const WsLayout& w, const void* 
   if (marks) cudaEventRecord(marks[0], stream);
   {
     const int Lp = static_cast<int>(align_up(r.L, 128));
-    const int64_t rows = static_cast<int64_t>(r.B) * r.Hq * Lp;
-    const int64_t threads = rows * (D / 8);
-    const int64_t blocks = (threads + 255) / 256;
-    if (blocks > 0x7fffffff) return LG_ERR_UNSUPPORTED;
-    delta_kernel<D><<<static_cast<unsigned>(blocks), 256, 0, stream>>>(
+    const int n_bh = r.B * r.Hq;
+    const int rows_per_block = 256 / (D / 8);
+    dim3 grid((Lp + rows_per_block - 1) / rows_per_block, n_bh < 65535 ? n_bh : 65535);
+    delta_kernel<D><<<grid, 256, 0, stream>>>(
         static_cast<const __nv_bfloat16*>(o), static_cast<const __nv_bfloat16*>(d_o), lse, stat, r.os[0], r.os[1],
-        r.os[2], r.Hq, r.L, Lp, rows);
+        r.os[2], r.Hq, n_bh, r.L, Lp, static_cast<int64_t>(n_bh) * Lp);
   }
   if (marks) cudaEventRecord(marks[1], stream);
   BwdArgs a;

@@ -56,35 +56,34 @@ struct BwdArgs {
 template <int D>
 __global__ void delta_kernel(const __nv_bfloat16* __restrict__ o, const __nv_bfloat16* __restrict__ d_o,
                              const float* __restrict__ lse, float* __restrict__ stat, int64_t sb, int64_t sh,
-                             int64_t sl, int Hq, int L, int Lp, int64_t total_rows) {
-  // rows are numbered over the padded length Lp; rows i >= L of a head exist only in `stat`, as zeros
+                             int64_t sl, int Hq, int n_bh, int L, int Lp, int64_t plane) {
+  // grid.x walks the padded rows of a head (rows i >= L exist only in `stat`, as zeros), grid.y the heads
   constexpr int TPR = D / 8;   // threads per row, 16 bytes each
-  const int64_t gid = static_cast<int64_t>(blockIdx.x) * blockDim.x + threadIdx.x;
-  const int64_t row = gid / TPR;
-  const int ch = static_cast<int>(gid % TPR);
-  float acc = 0.f;
-  const int i = static_cast<int>(row % Lp);
-  const bool real = row < total_rows && i < L;
-  if (real) {
-    const int64_t bh = row / Lp;
-    const int h = static_cast<int>(bh % Hq);
-    const int64_t b = bh / Hq;
-    const int64_t off = b * sb + h * sh + static_cast<int64_t>(i) * sl + ch * 8;
-    const uint4 ov = *reinterpret_cast<const uint4*>(o + off);
-    const uint4 dv = *reinterpret_cast<const uint4*>(d_o + off);
-    const __nv_bfloat162* op = reinterpret_cast<const __nv_bfloat162*>(&ov);
-    const __nv_bfloat162* dp = reinterpret_cast<const __nv_bfloat162*>(&dv);
+  const int i = blockIdx.x * (blockDim.x / TPR) + threadIdx.x / TPR;
+  const int ch = threadIdx.x % TPR;
+  for (int bh = blockIdx.y; bh < n_bh; bh += gridDim.y) {
+    float acc = 0.f;
+    const bool real = i < L;
+    if (real) {
+      const int h = bh % Hq, b = bh / Hq;
+      const int64_t off = b * sb + h * sh + static_cast<int64_t>(i) * sl + ch * 8;
+      const uint4 ov = *reinterpret_cast<const uint4*>(o + off);
+      const uint4 dv = *reinterpret_cast<const uint4*>(d_o + off);
+      const __nv_bfloat162* op = reinterpret_cast<const __nv_bfloat162*>(&ov);
+      const __nv_bfloat162* dp = reinterpret_cast<const __nv_bfloat162*>(&dv);
 #pragma unroll
-    for (int x = 0; x < 4; ++x) {
-      const float2 a = __bfloat1622float2(op[x]), c = __bfloat1622float2(dp[x]);
-      acc += a.x * c.x + a.y * c.y;
+      for (int x = 0; x < 4; ++x) {
+        const float2 a = __bfloat1622float2(op[x]), c = __bfloat1622float2(dp[x]);
+        acc += a.x * c.x + a.y * c.y;
+      }
     }
-  }
 #pragma unroll
-  for (int s = TPR / 2; s > 0; s >>= 1) acc += __shfl_xor_sync(0xffffffffu, acc, s);
-  if (row < total_rows && ch == 0) {
-    stat[row] = real ? -lse[(row / Lp) * L + i] * 1.4426950408889634f : 0.f;
-    stat[total_rows + row] = -acc;
+    for (int s = TPR / 2; s > 0; s >>= 1) acc += __shfl_xor_sync(0xffffffffu, acc, s);
+    if (i < Lp && ch == 0) {
+      const int64_t row = static_cast<int64_t>(bh) * Lp + i;
+      stat[row] = real ? -lse[static_cast<int64_t>(bh) * L + i] * 1.4426950408889634f : 0.f;
+      stat[plane + row] = -acc;
+    }
   }
 }
 
