@@ -183,9 +183,8 @@ lg_status lg_sparse_decode(const lg_decode_params* p, const void* q, const void*
  * q_chunk, o [B,Hq,T,D]; k_chunk, v_chunk [B,Hkv,T,D]; caches as above (may be NULL when
  * n_tokens_before == 0); all bf16, contiguous, device.  lse [B,Hq,T] fp32 (device).
  * n_tokens_before (HOST value, the same for every sequence) = tokens appended so far.
- * Limits: sink_tokens, window_tokens and T are multiples of 64 (window_tokens >= 64), and
- * while the ring is not yet full (n_tokens_before < sink + window) n_tokens_before is a
- * multiple of 64 too; otherwise LG_ERR_UNSUPPORTED.  The call copies the ring's tokens in
+ * Limits: sink_tokens and window_tokens are multiples of 64 (window_tokens >= 64), otherwise
+ * LG_ERR_UNSUPPORTED; T >= 1 and n_tokens_before >= 0 are free.  The call copies the ring's tokens in
  * time order, followed by the chunk, into the workspace and runs the sparse forward kernel
  * with the token-exact window over them, for the chunk's rows only.  workspace: device,
  * 256-byte aligned, lg_chunk_prefill_workspace_bytes() bytes (0 = invalid arguments);

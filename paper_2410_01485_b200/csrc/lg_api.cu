@@ -257,12 +257,11 @@ static lg_status plan_chunk(const lg_decode_params* p, int32_t T, int64_t n_befo
   if (p->B <= 0 || p->Hq <= 0 || p->Hkv <= 0 || p->Hq % p->Hkv != 0) return LG_ERR_INVALID_ARG;
   if (p->D != 64 && p->D != 128) return LG_ERR_UNSUPPORTED;
   if (p->sink_tokens < 0 || p->window_tokens < 64 || T <= 0 || n_before < 0) return LG_ERR_INVALID_ARG;
-  // the attention kernel works on 64-token blocks: sink, window, chunk and (while the ring is
-  // not yet full) the fill level must be multiples of 64
-  if (p->sink_tokens % 64 || p->window_tokens % 64 || T % 64) return LG_ERR_UNSUPPORTED;
+  // the pattern is made of 64-token blocks: sink and window must be multiples of 64; the chunk and
+  // the fill level of the ring may be anything
+  if (p->sink_tokens % 64 || p->window_tokens % 64) return LG_ERR_UNSUPPORTED;
   const int64_t cap = static_cast<int64_t>(p->sink_tokens) + p->window_tokens;
   const int64_t kept = n_before < cap ? n_before : cap;
-  if (kept % 64) return LG_ERR_UNSUPPORTED;
   if (kept + T > (1 << 24)) return LG_ERR_UNSUPPORTED;
   c->kept = static_cast<int>(kept);
   lg_attn_params& ap = c->ap;

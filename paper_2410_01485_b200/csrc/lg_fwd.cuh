@@ -346,10 +346,10 @@ fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUt
     }
     // ---- epilogue: O / l -> bf16, LSE ------------------------------------------------------
     if (ok) ok = wait_o(14);
-    // warp-uniform condition (q_start is a multiple of 64, the tensor-memory loads below need the whole
-    // warp); with a partial last block the rows past L load with the others and store nothing
-    if (ok && p0 + p1 > 0 && qi - lane < a.L && qi >= a.q_start) {
-      const bool mine = qi < a.L;
+    // warp-uniform condition (the tensor-memory loads below need the whole warp): some row of the warp
+    // is a real query; rows past L or before q_start load with the others and store nothing
+    if (ok && p0 + p1 > 0 && qi - lane < a.L && qi - lane + 32 > a.q_start) {
+      const bool mine = qi < a.L && qi >= a.q_start;
       tc_fence_after();
       const float inv_l = l_run > 0.f ? 1.f / l_run : 0.f;
       __nv_bfloat16* orow =

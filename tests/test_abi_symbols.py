@@ -91,9 +91,9 @@ def test_chunk_prefill_planning_on_host(lib):
     """Sizes and limits of a chunk served against the ring are decided on the host."""
     p = binding.decode_params(1, 4, 2, 128, 64, 128)
     sz = lib.lg_chunk_prefill_workspace_bytes
-    assert sz(C.byref(p), 60, 0) == 0          # chunk not a multiple of 64
-    assert sz(C.byref(p), 64, 100) == 0        # ring not yet full: the fill level must be a multiple of 64
-    assert sz(C.byref(p), 64, -1) == 0
+    assert sz(C.byref(p), 0, 0) == 0 and sz(C.byref(p), 64, -1) == 0
+    assert sz(C.byref(p), 60, 0) > 0           # neither the chunk nor the fill level need be a multiple of 64
+    assert sz(C.byref(p), 64, 100) > sz(C.byref(p), 64, 64)
     full, more = sz(C.byref(p), 64, 1000), sz(C.byref(p), 128, 1000)
     assert 0 < full < more                     # a full ring: any fill level; longer chunk, more room
     assert sz(C.byref(p), 64, 192) == full     # exactly full = full

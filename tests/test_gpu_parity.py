@@ -391,6 +391,9 @@ def _chunk_prefill_case(lg, B, Hq, Hkv, D, sink, W, n0, T, seed=0, heads=None):
     (2, 4, 2, 128, 64, 128, 1000, 192),     # wrapped ring, odd fill level, chunk longer than the window
     (1, 8, 2, 64, 0, 256, 777, 320),        # no sink; chunk spans two super-tiles with a ragged second one
     (1, 2, 2, 128, 128, 512, 5003, 448),    # first super-tile half below the first query row (640 = 2.5 x 256)
+    (2, 4, 2, 128, 64, 128, 100, 37),       # ring not yet full at an odd level, odd chunk
+    (1, 4, 1, 64, 64, 256, 1000, 77),       # full ring, odd chunk
+    (1, 2, 1, 128, 0, 128, 7, 1),           # a single token (what the decode computes)
 ], ids=str)
 def test_chunk_prefill_small(lg, args):
     _chunk_prefill_case(lg, *args)
@@ -424,14 +427,12 @@ def test_chunk_prefill_cfg5_shape(lg):
 
 
 def test_chunk_prefill_rejects_unsupported(lg):
-    p = lg.decode_params(1, 2, 2, 128, 64, 128)
     L = lg.load_library()
     import ctypes as C
-    assert L.lg_chunk_prefill_workspace_bytes(C.byref(p), 60, 0) == 0        # chunk not a multiple of 64
-    assert L.lg_chunk_prefill_workspace_bytes(C.byref(p), 64, 100) == 0      # ring not full, ragged fill level
-    assert L.lg_chunk_prefill_workspace_bytes(C.byref(p), 64, 1000) > 0      # full ring: any fill level
     p2 = lg.decode_params(1, 2, 2, 128, 32, 128)
     assert L.lg_chunk_prefill_workspace_bytes(C.byref(p2), 64, 0) == 0       # sink not a multiple of 64
+    p3 = lg.decode_params(1, 2, 2, 128, 64, 100)
+    assert L.lg_chunk_prefill_workspace_bytes(C.byref(p3), 64, 0) == 0       # window not a multiple of 64
 
 
 def test_decode_workspace_is_reusable_without_clearing(lg):
