@@ -14,15 +14,18 @@
 //     S = Q K^T, dP = dO V^T, dS over S, dQ += dS K.
 //
 // Both kernels are warp-specialised: warps 0-15 do the element-wise work (four groups of four
-// warps, each group owning 32 of the 128 columns of a step; thread = TMEM lane), warp 16
-// feeds shared memory with TMA, one thread each of warps 17 and 18 issues tcgen05.mma.  The two
-// issuing threads sit on different scheduler partitions of the SM: issuing an MMA is slowed by
-// fp32 arithmetic of other warps on the issuer's partition, and two queues halve what each has
-// to push through.  MMAs whose operands alias in tensor memory stay on one thread, so that the
-// queue order is the only synchronisation they need.  A step covers 128 streamed rows: one
-// 128-token pattern block, or two 64-token blocks side by side.
-//   dQ pass   : thread A: S(j+2) after dQ(j) (S double-buffered, dS over S)   thread B: dP(j)
-//   dK/dV pass: thread A: dV(j) then S^T(j+1) (P^T over S^T)     thread B: dK(j-1) then dP^T(j)
+// warps; thread = TMEM lane, each group owns a quarter of the columns in work), warp 16 feeds
+// shared memory with TMA, warps 17 and 18 issue tcgen05.mma (the whole warp runs the loop with
+// warp-uniform values, one elected lane issues).  The two issuing warps sit on different scheduler
+// partitions of the SM: issuing an MMA is slowed by other warps' arithmetic on the issuer's
+// partition, and two queues halve what each has to push through.  MMAs whose operands alias in
+// tensor memory stay on one warp, so that the queue order is the only synchronisation they need.
+// A step covers 128 streamed rows: one 128-token pattern block, or two 64-token blocks side by
+// side; the dK/dV pass works it in two half-steps of 64 queries whose score buffers alternate.
+//   dQ pass   : warp A: dQ(j) then S(j+2) (S double-buffered, dS over S)   warp B: dP(j+1) once dP(j) is read
+//   dK/dV pass: warp A: dV(h) then S^T(h+2) (P^T over S^T)       warp B: dK(h) then dP^T(h+2)   (h: half-step)
+// Options folded into the masks: a token-exact window edge, packed documents (no key of an earlier
+// document), and a sequence length that ends inside a block.
 #pragma once
 #include <cuda.h>
 #include "lg_common.cuh"

@@ -2,14 +2,18 @@
 // with the sink kept beside it, and a single-token decode whose only job is to stream that
 // cache from HBM as fast as possible.
 //
-// Decode layout: one CTA per (sequence, kv head, head group of <= 8 query heads, KV split).
-// Each of its 4 warps owns a contiguous run of 16-token tiles and keeps a private cp.async
-// pipeline of kStages tiles (16-byte copies into XOR-swizzled shared memory, so the HBM
-// stream never waits on arithmetic).  Scores are S^T = K Q^T and the output is
-// O^T = V^T P^T, both on mma.sync m16n8k16 (bf16 in, fp32 accumulate) with the 8 query heads
-// of the group as the N dimension, so all heads of a GQA group share every byte loaded.
-// Per-split (max, sum, O) partials go to the workspace and a second kernel merges them in
-// split order, which keeps the result bitwise reproducible.
+// Decode layout: the 16-token tiles of all (sequence, kv head, head group of <= 8 query heads)
+// units form one sequence that is cut into equal slices, one per CTA, so that a single wave of
+// CTAs streams the whole cache whatever the mix of lengths.  Each of a CTA's warps owns a
+// contiguous run of tiles and keeps a private cp.async pipeline of kDecStages tiles (16-byte
+// copies into XOR-swizzled shared memory, so the HBM stream never waits on arithmetic).  Scores
+// are S^T = K Q^T and the output is O^T = V^T P^T, both on mma.sync m16n8k16 (bf16 in, fp32
+// accumulate) with the 8 query heads of the group as the N dimension, so all heads of a GQA group
+// share every byte loaded.  The warps' (max, sum, O) are merged in warp order in shared memory; a
+// CTA whose slice is a whole unit writes the result itself, otherwise the CTAs of a unit leave
+// records in the workspace and the one that arrives last merges them in index order.  Either way
+// the summation order is fixed, so results are bitwise reproducible.  (Batches of more than
+// kDecFlatMaxB sequences use a per-unit split grid and a separate merge kernel.)
 #include <math.h>
 
 #include <mutex>
