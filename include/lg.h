@@ -76,8 +76,10 @@ typedef struct {
      contiguous, with doc_start[b][i] = position of the first token of the document token i
      belongs to (non-decreasing in i, <= i).  When given, a query sees no key of an earlier
      document, on top of the pattern (which stays in absolute positions: the sink blocks are
-     those of the sample, so only its first document sees them).  The block lists are those
-     of the pattern alone; blocks that the documents empty are computed and masked.          */
+     those of the sample, so only its first document sees them).  With B == 1 the calls drop
+     every key block that ends before the earliest document of a query block starts; with
+     B > 1 the lists are shared by the sequences and stay the pattern's own (what the
+     documents empty is computed and masked).  lg_build_block_index ignores this field.      */
   const int32_t* doc_start;
 } lg_attn_params;
 

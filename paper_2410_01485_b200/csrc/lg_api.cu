@@ -46,6 +46,8 @@ lg_status resolve(const lg_attn_params* p, Resolved* r) {
   r->pat.nB = (p->L + p->block - 1) / p->block;
   r->pat.mode = p->mode;
   r->pat.ns = r->pat.nw = r->pat.stride = r->pat.nl = 0;
+  r->pat.doc_start = nullptr;
+  r->pat.block = p->block;
   r->exact_w = 0;
   switch (p->mode) {
     case LG_MODE_FULL_CAUSAL:
@@ -146,7 +148,11 @@ lg_status prepare_workspace(const Resolved& r, const WsLayout& w, uint8_t* ws, b
                             cudaStream_t stream) {
   if (cudaMemsetAsync(ws, 0, sizeof(WsHeader), stream) != cudaSuccess) return LG_ERR_CUDA;
   auto i32 = [&](size_t off) { return reinterpret_cast<int32_t*>(ws + off); };
-  lg_status s = launch_index_build(r, i32(w.row_ptr), i32(w.col_idx), i32(w.col_ptr), i32(w.row_idx), stream);
+  // The lists are shared by all sequences of the batch, so documents can only prune them when there
+  // is one sequence (the usual case for long packed samples); otherwise they stay the pattern's own.
+  Resolved rl = r;
+  if (r.doc_start && r.B == 1) rl.pat.doc_start = r.doc_start;
+  lg_status s = launch_index_build(rl, i32(w.row_ptr), i32(w.col_idx), i32(w.col_ptr), i32(w.row_idx), stream);
   if (s != LG_OK) return s;
   const int R = 128 / r.block;
   if (!want_bwd) {   // the forward walks super-tiles of 256 rows; the backward passes have their own schedules
