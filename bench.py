@@ -450,7 +450,27 @@ def main():
                "attention_prefill_speedup": 32 * rpf["fwd_ms"] / (12 * rpf["fwd_ms"] + 20 * rp1["fwd_ms"]),
                "note": "attention kernels only, Llama-2-7B shape at 128K; the paper's 1.55x (training) and 1.67x "
                        "(prefill) are end-to-end model numbers on other hardware"}
-        others = [r2, r2f, r4, d5, d5d, rp1, rp2, cp, mix]
+        # packed documents (exponential lengths, 8K tokens on average) on the headline pattern and on full
+        # causal attention: one sequence, so the documents also prune the block lists
+        ds = synth.make_doc_start(cfg.L, seed=0, mean_len=8192).view(1, -1).cuda()
+        docs = {"config": "cfg3_packed_documents_mean8k", "documents": int(ds.unique().numel())}
+        for name, c in (("sink_window", cfg), ("full_causal", cfg.full_causal())):
+            pd_ = lg.params_of(c, doc_start=ds)
+            inp_d = synth.make_attn_inputs(c, "cuda", seed=0, with_do=True)
+            ws_d = lg.attn_workspace(pd_, True)
+            o_d = torch.empty_like(inp_d["q"])
+            lse_d = torch.empty(inp_d["q"].shape[:3], dtype=torch.float32, device="cuda")
+            g_d = [torch.empty_like(inp_d[x]) for x in ("q", "k", "v")]
+
+            def step_d():
+                lg.lg_sparse_attn_fwd(pd_, inp_d["q"], inp_d["k"], inp_d["v"], o=o_d, lse=lse_d, workspace=ws_d)
+                lg.lg_sparse_attn_bwd(pd_, inp_d["q"], inp_d["k"], inp_d["v"], o_d, lse_d, inp_d["do"], dq=g_d[0],
+                                      dk=g_d[1], dv=g_d[2], workspace=ws_d)
+            docs[name + "_fwd_bwd_ms"] = time_cuda(step_d, 2, 3)
+            assert lg.lg_last_status(ws_d) == 0
+            del inp_d, ws_d, o_d, lse_d, g_d
+            torch.cuda.empty_cache()
+        others = [r2, r2f, r4, d5, d5d, rp1, rp2, cp, mix, docs]
         line["other"] = others
         line["decode_hbm_gbs"] = d5["gbs"]
         line["decode_roofline"] = {"bound": "hbm", "kernel": "decode_stream_kernel", "achieved": d5["gbs"],
