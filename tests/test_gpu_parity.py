@@ -609,3 +609,33 @@ def test_partial_last_block_parity(lg, cfg):
     torch.cuda.synchronize()
     for buf, view, ref_t in ((bo, o2, o), (bq, dq2, dq), (bk, dk2, dk), (bv, dv2, dv)):
         assert torch.equal(view, ref_t) and bool((buf[-pad:] == -7.0).all())
+
+
+def test_serving_flow_prefill_in_chunks_equals_training_mask(lg):
+    """A prompt prefilled chunk by chunk through the ring (lg_chunk_prefill, then lg_kv_ring_append) gives,
+    row for row, what one pass of the training kernel with the token-exact window gives on the whole prompt;
+    a decode step after the last chunk continues it."""
+    B, Hq, Hkv, D, sink, W, L = 1, 8, 2, 128, 64, 256, 1536
+    cfg = replace(synth.CFG1, name="flow", B=B, Hq=Hq, Hkv=Hkv, L=L, D=D, block=64, sink_tokens=sink, window_tokens=W,
+                  window_exact=True)
+    inp = synth.make_attn_inputs(cfg, "cuda", seed=9, with_do=False)
+    o_ref, lse_ref = lg.lg_sparse_attn_fwd(lg.params_of(cfg), inp["q"], inp["k"], inp["v"])
+    p = lg.decode_params(B, Hq, Hkv, D, sink, W)
+    kc = torch.zeros(B, Hkv, sink + W, D, dtype=torch.bfloat16, device="cuda")
+    vc = torch.zeros_like(kc)
+    pos = 0
+    for T in (320, 64, 500, 37, 614):     # ends at 1535: the last token is left for the decode
+        sl = slice(pos, pos + T)
+        o, lse = lg.lg_chunk_prefill(p, inp["q"][:, :, sl].contiguous(), inp["k"][:, :, sl].contiguous(),
+                                     inp["v"][:, :, sl].contiguous(), kc, vc, pos)
+        assert (o.float() - o_ref[:, :, sl].float()).abs().max() <= 1e-2
+        assert (lse - lse_ref[:, :, sl]).abs().max() <= 1e-3
+        lg.lg_kv_ring_append(p, kc, vc, inp["k"][:, :, sl].contiguous(), inp["v"][:, :, sl].contiguous(),
+                             torch.full((B,), pos, dtype=torch.int64, device="cuda"))
+        pos += T
+    assert pos == L - 1
+    lg.lg_kv_ring_append(p, kc, vc, inp["k"][:, :, pos:].contiguous(), inp["v"][:, :, pos:].contiguous(),
+                         torch.full((B,), pos, dtype=torch.int64, device="cuda"))
+    od, ld = lg.lg_sparse_decode(p, inp["q"][:, :, pos].contiguous(), kc, vc, torch.full((B,), L, dtype=torch.int64, device="cuda"))
+    assert (od.float() - o_ref[:, :, pos].float()).abs().max() <= 1e-2
+    assert (ld - lse_ref[:, :, pos]).abs().max() <= 1e-3
