@@ -639,3 +639,40 @@ def test_serving_flow_prefill_in_chunks_equals_training_mask(lg):
     od, ld = lg.lg_sparse_decode(p, inp["q"][:, :, pos].contiguous(), kc, vc, torch.full((B,), L, dtype=torch.int64, device="cuda"))
     assert (od.float() - o_ref[:, :, pos].float()).abs().max() <= 1e-2
     assert (ld - lse_ref[:, :, pos]).abs().max() <= 1e-3
+
+
+def test_decode_large_batch_uses_the_split_grid(lg):
+    """More than 2048 sequences take the per-unit split grid with its separate merge kernel: same results
+    (sampled sequences against the oracle), empty sequences included."""
+    B, Hq, Hkv, D, sink, W = 2100, 4, 2, 64, 8, 120
+    p = lg.decode_params(B, Hq, Hkv, D, sink, W)
+    g = torch.Generator(device="cuda").manual_seed(11)
+    nmax = 300
+    hist_k = torch.randn(B, Hkv, nmax, D, generator=g, device="cuda").to(torch.bfloat16)
+    hist_v = torch.randn(B, Hkv, nmax, D, generator=g, device="cuda").to(torch.bfloat16)
+    q = torch.randn(B, Hq, D, generator=g, device="cuda").to(torch.bfloat16)
+    ns = [(37 * b) % (nmax + 1) for b in range(B)]          # 0 .. 300, mixed
+    kc = torch.zeros(B, Hkv, sink + W, D, dtype=torch.bfloat16, device="cuda")
+    vc = torch.zeros_like(kc)
+    # fill each ring with its first ns[b] tokens: one append of nmax tokens would overshoot, so append by length class
+    for n in sorted(set(ns)):
+        if n == 0:
+            continue
+        idx = torch.tensor([b for b in range(B) if ns[b] == n], device="cuda")
+        pk = lg.decode_params(len(idx), Hq, Hkv, D, sink, W)
+        kk, vv = kc[idx].contiguous(), vc[idx].contiguous()
+        lg.lg_kv_ring_append(pk, kk, vv, hist_k[idx][:, :, :n].contiguous(), hist_v[idx][:, :, :n].contiguous(),
+                             torch.zeros(len(idx), dtype=torch.int64, device="cuda"))
+        kc[idx], vc[idx] = kk, vv
+    n_t = torch.tensor(ns, dtype=torch.int64, device="cuda")
+    ws = lg.decode_workspace(p)
+    o, lse = lg.lg_sparse_decode(p, q, kc, vc, n_t, workspace=ws)
+    assert lg.lg_last_status(ws) == 0
+    scale = 1.0 / np.sqrt(D)
+    for b in (0, 1, 8, 57, 1000, 2048, 2099):
+        oo, ll = O.decode(synth.to_f64(q[b]), synth.to_f64(hist_k[b]), synth.to_f64(hist_v[b]), ns[b], sink, W, scale)
+        _assert_close(synth.to_f64(o[b]), oo, TOL_O, "decode o")
+        if ns[b] > 0:
+            assert np.abs(synth.to_f64(lse[b]) - ll).max() <= TOL_LSE
+        else:
+            assert torch.isneginf(lse[b]).all() and (o[b] == 0).all()
