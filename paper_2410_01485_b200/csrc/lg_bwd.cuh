@@ -187,6 +187,9 @@ bwd_dq_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ 
   uint8_t* sK = smem + SM::oA;
   uint8_t* sV = smem + SM::oB;
 
+  // has a wait already given up in this call?  (read now, so that it travels with the schedule loads below)
+  unsigned int abort_word = 0;
+  if (tid == 0) abort_word = *reinterpret_cast<volatile unsigned int*>(a.error_word);
   const int tile = a.order[blockIdx.y];
   const int b = blockIdx.x / a.Hq, h = blockIdx.x % a.Hq, hk = h / a.G;
   const int n_ent = a.tile_cnt[tile];
@@ -206,6 +209,7 @@ bwd_dq_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ 
     mbar_init(bars + B_DPR, kDqEwWarps);
     mbar_init(bars + B_DONE, 1);
     mbar_fence_init();
+    tmem_slot[1] = abort_word;
   }
   if (warp == kDqMmaWarpA) {
     tmem_alloc(tmem_slot, 512);
@@ -215,6 +219,10 @@ bwd_dq_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ 
   __syncthreads();
   tc_fence_after();
   const uint32_t tmem = *tmem_slot;
+  if (tmem_slot[1] != 0) {   // after a failed wait the rest of the grid does nothing: the call ends in seconds, not minutes
+    if (warp == kDqMmaWarpA) tmem_dealloc(tmem, 512);
+    return;
+  }
 
   if (warp == kDqTmaWarp) {
     // ------------------------------ TMA producer ------------------------------------------
@@ -479,6 +487,9 @@ bwd_dkdv_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
   uint8_t* sDO = smem + SM::oB;    // [2]
   float* sStat = reinterpret_cast<float*>(smem + SM::oStat);   // [2 stages][-LSE2 | -delta][128 queries]
 
+  // has a wait already given up in this call?  (read now, so that it travels with the schedule loads below)
+  unsigned int abort_word = 0;
+  if (tid == 0) abort_word = *reinterpret_cast<volatile unsigned int*>(a.error_word);
   const int tile = a.order[blockIdx.y];
   const int b = blockIdx.x / a.Hkv, hk = blockIdx.x % a.Hkv;
   const int n_ent = a.tile_cnt[tile];
@@ -508,6 +519,7 @@ bwd_dkdv_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
     }
     mbar_init(bars + B_DONE, 2);          // the last dV and the last dK
     mbar_fence_init();
+    tmem_slot[1] = abort_word;
   }
   if (warp == kKvMmaWarpA) {
     tmem_alloc(tmem_slot, 512);
@@ -517,6 +529,10 @@ bwd_dkdv_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
   __syncthreads();
   tc_fence_after();
   const uint32_t tmem = *tmem_slot;
+  if (tmem_slot[1] != 0) {   // after a failed wait the rest of the grid does nothing: the call ends in seconds, not minutes
+    if (warp == kKvMmaWarpA) tmem_dealloc(tmem, 512);
+    return;
+  }
 
   if (warp == kKvTmaWarp) {
     // ------------------------------ TMA producer ------------------------------------------

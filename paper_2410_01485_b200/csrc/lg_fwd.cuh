@@ -85,6 +85,9 @@ fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUt
   uint8_t* sK = smem + SM::oK;
   uint8_t* sV = smem + SM::oV;
 
+  // has a wait already given up in this call?  (read now, so that it travels with the schedule loads below)
+  unsigned int abort_word = 0;
+  if (tid == 0) abort_word = *reinterpret_cast<volatile unsigned int*>(a.error_word);
   const int tile = a.order[blockIdx.y];
   const int b = blockIdx.x / a.Hq, h = blockIdx.x % a.Hq, hk = h / a.G;
   const int n_ent = a.tile_cnt[tile];
@@ -110,6 +113,7 @@ fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUt
     }
     for (int i = 0; i < 4; ++i) { mbar_init(bars + B_SF + i, 1); mbar_init(bars + B_PF + i, 4); mbar_init(bars + B_OD + i, 1); }
     mbar_fence_init();
+    tmem_slot[1] = abort_word;
   }
   if (warp == kFwdMmaWarp0) {
     tmem_alloc(tmem_slot, 512);
@@ -119,6 +123,10 @@ fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUt
   __syncthreads();
   tc_fence_after();
   const uint32_t tmem = *tmem_slot;
+  if (tmem_slot[1] != 0) {   // after a failed wait the rest of the grid does nothing: the call ends in seconds, not minutes
+    if (warp == kFwdMmaWarp0) tmem_dealloc(tmem, 512);
+    return;
+  }
 
   if (warp == kFwdTmaWarp) {
     // ------------------------------ TMA producer ------------------------------------------
