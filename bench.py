@@ -369,7 +369,7 @@ def main():
     achieved = kern[dom][1] / kern[dom][0] / 1e9
     # dram__bytes_read + dram__bytes_write of one launch, from the ncu capture of the same kernels on
     # the 8-head x 32K case of this pattern, scaled by the (head, token) units of this workload
-    ncu_small_bytes = {"fwd": 266.6e6, "bwd_dkdv": 450.8e6, "bwd_dq": 342.2e6}
+    ncu_small_bytes = {"fwd": 266.5e6, "bwd_dkdv": 451.4e6, "bwd_dq": 341.2e6}
     traffic = ncu_small_bytes[dom] * (cfg.B * cfg.Hq * cfg.L) / (8 * 32768.0)
     roofline = {"bound": "tensor", "kernel": dom, "achieved": achieved, "peak": peaks["bf16_sustained"],
                 "unit": "TFLOP/s", "frac": achieved / peaks["bf16_sustained"], "traffic": traffic,
