@@ -76,10 +76,11 @@ typedef struct {
      contiguous, with doc_start[b][i] = position of the first token of the document token i
      belongs to (non-decreasing in i, <= i).  When given, a query sees no key of an earlier
      document, on top of the pattern (which stays in absolute positions: the sink blocks are
-     those of the sample, so only its first document sees them).  With B == 1 the calls drop
-     every key block that ends before the earliest document of a query block starts; with
-     B > 1 the lists are shared by the sequences and stay the pattern's own (what the
-     documents empty is computed and masked).  lg_build_block_index ignores this field.      */
+     those of the sample, so only its first document sees them).  The calls drop every key
+     block that ends before the earliest document of a query block starts; as the lists then
+     differ between sequences, a call with B > 1 runs sequence by sequence (its workspace is
+     B slices of the B == 1 size; lg_sparse_attn_bwd_profiled does not take that case).
+     lg_build_block_index ignores this field.                                                */
   const int32_t* doc_start;
 } lg_attn_params;
 

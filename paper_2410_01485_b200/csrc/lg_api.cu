@@ -82,6 +82,7 @@ lg_status resolve(const lg_attn_params* p, Resolved* r) {
   r->Lq = p->L;
   if (reinterpret_cast<uintptr_t>(p->doc_start) & 3) return LG_ERR_INVALID_ARG;
   r->doc_start = p->doc_start;
+  r->error_word = nullptr;
   // nnz from the per-row counts of each pattern
   int64_t nnz = 0;
   const PatternDev& pt = r->pat;
@@ -307,6 +308,33 @@ __global__ void wait_selftest_kernel(unsigned int* error_word, long long limit_c
     if (!mbar_try_wait(&bar, 0)) mbar_wait_slow(&bar, 0, error_word, 99, limit_cycles);
   }
 }
+
+// ---- packed documents with several sequences ------------------------------------------------
+// The block lists are shared by the sequences of a call, and documents prune them per sequence;
+// with documents and B > 1 a call therefore runs sequence by sequence, each with its own lists in
+// its own slice of the workspace (long packed samples fill the GPU one at a time).  The status
+// word of the call stays the first word of the whole workspace.
+static bool per_sequence(const Resolved& r) { return r.doc_start != nullptr && r.B > 1; }
+
+static Resolved one_sequence(const Resolved& r, int b, void* workspace) {
+  Resolved r1 = r;
+  r1.B = 1;
+  r1.doc_start = r.doc_start + static_cast<int64_t>(b) * r.L;
+  r1.error_word = static_cast<unsigned int*>(workspace);
+  return r1;
+}
+
+static size_t attn_workspace_total(const Resolved& r, bool want_bwd) {
+  if (!per_sequence(r)) return ws_layout(r, want_bwd).total;
+  return align_up(ws_layout(one_sequence(r, 0, nullptr), want_bwd).total, 256) * r.B;
+}
+
+template <typename T>
+static T* seq_ptr(T* base, int b, int64_t batch_stride_elems) {   // bf16 tensors: 2 bytes per element
+  return base ? reinterpret_cast<T*>(reinterpret_cast<uint8_t*>(const_cast<void*>(static_cast<const void*>(base))) +
+                                     static_cast<int64_t>(b) * batch_stride_elems * 2)
+              : nullptr;
+}
 }  // namespace lg
 
 using namespace lg;
@@ -341,7 +369,7 @@ lg_status lg_build_block_index(const lg_attn_params* p, int32_t* row_ptr, int32_
 size_t lg_sparse_attn_workspace_bytes(const lg_attn_params* p, int want_bwd) {
   Resolved r;
   if (resolve(p, &r) != LG_OK) return 0;
-  return ws_layout(r, want_bwd != 0).total;
+  return attn_workspace_total(r, want_bwd != 0);
 }
 
 lg_status lg_sparse_attn_fwd(const lg_attn_params* p, const void* q, const void* k, const void* v, void* o,
@@ -352,11 +380,24 @@ lg_status lg_sparse_attn_fwd(const lg_attn_params* p, const void* q, const void*
   if (!q || !k || !v || !o || !lse || !workspace) return LG_ERR_INVALID_ARG;
   if (!aligned16(q) || !aligned16(k) || !aligned16(v) || !aligned16(o) || !aligned16(lse)) return LG_ERR_INVALID_ARG;
   if (reinterpret_cast<uintptr_t>(workspace) & 255) return LG_ERR_INVALID_ARG;
-  const WsLayout w = ws_layout(r, false);
-  if (workspace_bytes < w.total) return LG_ERR_WORKSPACE;
+  if (workspace_bytes < attn_workspace_total(r, false)) return LG_ERR_WORKSPACE;
   if ((s = check_arch()) != LG_OK) return s;
   cudaStream_t st = static_cast<cudaStream_t>(stream);
   uint8_t* ws = static_cast<uint8_t*>(workspace);
+  if (per_sequence(r)) {
+    const size_t per = attn_workspace_total(r, false) / r.B;
+    for (int b = 0; b < r.B; ++b) {
+      const Resolved r1 = one_sequence(r, b, workspace);
+      const WsLayout w1 = ws_layout(r1, false);
+      uint8_t* wsb = ws + b * per;
+      if ((s = prepare_workspace(r1, w1, wsb, false, st)) != LG_OK) return s;
+      s = launch_fwd(r1, w1, seq_ptr(q, b, r.qs[0]), seq_ptr(k, b, r.ks[0]), seq_ptr(v, b, r.vs[0]),
+                     seq_ptr(o, b, r.os[0]), lse + static_cast<int64_t>(b) * r.Hq * r.L, wsb, st);
+      if (s != LG_OK) return s;
+    }
+    return LG_OK;
+  }
+  const WsLayout w = ws_layout(r, false);
   if ((s = prepare_workspace(r, w, ws, false, st)) != LG_OK) return s;
   return launch_fwd(r, w, q, k, v, o, lse, ws, st);
 }
@@ -372,11 +413,26 @@ static lg_status bwd_common(const lg_attn_params* p, const void* q, const void* 
       !aligned16(dq) || !aligned16(dk) || !aligned16(dv))
     return LG_ERR_INVALID_ARG;
   if (reinterpret_cast<uintptr_t>(workspace) & 255) return LG_ERR_INVALID_ARG;
-  const WsLayout w = ws_layout(r, true);
-  if (workspace_bytes < w.total) return LG_ERR_WORKSPACE;
+  if (workspace_bytes < attn_workspace_total(r, true)) return LG_ERR_WORKSPACE;
   if ((s = check_arch()) != LG_OK) return s;
   cudaStream_t st = static_cast<cudaStream_t>(stream);
   uint8_t* ws = static_cast<uint8_t*>(workspace);
+  if (per_sequence(r)) {
+    if (marks) return LG_ERR_UNSUPPORTED;   // the per-kernel timing variant covers one launch of each kernel
+    const size_t per = attn_workspace_total(r, true) / r.B;
+    for (int b = 0; b < r.B; ++b) {
+      const Resolved r1 = one_sequence(r, b, workspace);
+      const WsLayout w1 = ws_layout(r1, true);
+      uint8_t* wsb = ws + b * per;
+      if ((s = prepare_workspace(r1, w1, wsb, true, st)) != LG_OK) return s;
+      s = launch_bwd(r1, w1, seq_ptr(q, b, r.qs[0]), seq_ptr(k, b, r.ks[0]), seq_ptr(v, b, r.vs[0]),
+                     seq_ptr(o, b, r.os[0]), lse + static_cast<int64_t>(b) * r.Hq * r.L, seq_ptr(d_o, b, r.os[0]),
+                     seq_ptr(dq, b, r.qs[0]), seq_ptr(dk, b, r.ks[0]), seq_ptr(dv, b, r.vs[0]), wsb, st, nullptr);
+      if (s != LG_OK) return s;
+    }
+    return LG_OK;
+  }
+  const WsLayout w = ws_layout(r, true);
   if ((s = prepare_workspace(r, w, ws, true, st)) != LG_OK) return s;
   return launch_bwd(r, w, q, k, v, o, lse, d_o, dq, dk, dv, ws, st, marks);
 }

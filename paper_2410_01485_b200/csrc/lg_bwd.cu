@@ -25,7 +25,7 @@ static lg_status launch_bwd_t(const Resolved& r, const WsLayout& w, const void* 
   a.stat = stat;
   a.Lp = static_cast<int>(align_up(r.L, 128));
   a.stat_plane = static_cast<int64_t>(r.B) * r.Hq * a.Lp;
-  a.error_word = reinterpret_cast<unsigned int*>(ws);
+  a.error_word = r.error_word ? r.error_word : reinterpret_cast<unsigned int*>(ws);
   a.L = r.L; a.Hq = r.Hq; a.Hkv = r.Hkv; a.G = r.G;
   a.exact_w = r.exact_w; a.ns = r.pat.ns;
   a.doc_start = r.doc_start;

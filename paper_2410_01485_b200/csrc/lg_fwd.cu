@@ -19,7 +19,7 @@ static lg_status launch_fwd_t(const Resolved& r, const WsLayout& w, const void* 
   a.order = reinterpret_cast<const int32_t*>(ws + w.sq_order);
   a.o = static_cast<__nv_bfloat16*>(o);
   a.lse = lse;
-  a.error_word = reinterpret_cast<unsigned int*>(ws);
+  a.error_word = r.error_word ? r.error_word : reinterpret_cast<unsigned int*>(ws);
   for (int i = 0; i < 3; ++i) a.o_strides[i] = r.os[i];
   a.L = r.L; a.Hq = r.Hq; a.G = r.G;
   a.q_start = r.q_start; a.Lq = r.Lq;

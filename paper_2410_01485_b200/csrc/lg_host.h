@@ -23,6 +23,7 @@ struct Resolved {          // validated, defaulted copy of lg_attn_params
   int n_stiles;            // ceil(L / 256): super-tiles of the forward
   int q_start, Lq;         // forward only: queries exist for rows [q_start, q_start + Lq) (0, L by default)
   const int32_t* doc_start;  // device [B, L] or null: first position of each token's document
+  unsigned int* error_word;  // status word of the call when it is not the start of `ws` (null: it is)
   int64_t nnz;
 };
 
