@@ -228,7 +228,8 @@ def sparse_attn_fwd_bwd_host(p: AttnParams, host_in, host_out, dev=None, head_gr
     G = p.Hq // p.Hkv
     kv_per = p.Hkv // n_groups
     pg = attn_params(p.B, kv_per * G, kv_per, p.L, p.D, p.block, p.mode, p.sink_tokens, p.window_tokens,
-                     p.stride_blocks, p.local_blocks, p.scale, bool(p.window_exact))
+                     p.stride_blocks, p.local_blocks, p.scale, bool(p.window_exact),
+                     getattr(p, "_doc_start_ref", None))
     if not isinstance(ws, (list, tuple)) or len(ws) < n_groups:
         ws = [attn_workspace(pg, True) for _ in range(n_groups)]   # groups overlap in time: one workspace each
     cur = torch.cuda.current_stream()

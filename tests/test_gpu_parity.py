@@ -476,6 +476,14 @@ def test_host_buffer_step_equals_device_calls(lg):
         torch.cuda.synchronize()
         for name, ref in (("o", o), ("lse", lse), ("dq", dq), ("dk", dk), ("dv", dv)):
             assert torch.equal(h_out[name], ref.cpu()), (groups, name)
+    # packed documents travel with the parameters into every head group
+    ds = synth.make_doc_start(cfg.L, seed=1, mean_len=200).view(1, -1).cuda()
+    pd = lg.params_of(cfg, doc_start=ds)
+    od, lsed = lg.lg_sparse_attn_fwd(pd, inp["q"], inp["k"], inp["v"])
+    assert not torch.equal(od, o)
+    lg.sparse_attn_fwd_bwd_host(lg.params_of(cfg, doc_start=ds), host, h_out, head_groups=4)
+    torch.cuda.synchronize()
+    assert torch.equal(h_out["o"], od.cpu()) and torch.equal(h_out["lse"], lsed.cpu())
 
 
 def test_expired_wait_is_reported_and_leaves_the_context_usable(lg):
