@@ -128,3 +128,14 @@ def test_partial_last_block_is_accepted(lib):
     assert lib.lg_block_index_nnz(C.byref(p)) == full
     p.L = p.L - 64                              # one block fewer
     assert 0 < lib.lg_block_index_nnz(C.byref(p)) < full
+
+
+def test_documents_with_several_sequences_take_a_workspace_slice_each(lib):
+    p = _good()
+    p.B = 1
+    p.doc_start = 256
+    one = lib.lg_sparse_attn_workspace_bytes(C.byref(p), 1)
+    p.B = 3
+    assert lib.lg_sparse_attn_workspace_bytes(C.byref(p), 1) == 3 * one
+    p.doc_start = None
+    assert lib.lg_sparse_attn_workspace_bytes(C.byref(p), 1) < 3 * one      # shared lists without documents
