@@ -49,8 +49,8 @@ typedef enum {
  * With Bs = block, qb = i / Bs, kb = j / Bs, query i may attend key j iff j <= i and
  *   FULL_CAUSAL   : (nothing more)
  *   SINK_WINDOW   : kb < sink_tokens/Bs  or  qb - kb < window_tokens/Bs
- *                   (the window is block-granular and counts the query's own block:
- *                    "the first block for sink tokens and the most recent 32 blocks");
+ *                   (the window is block-granular and counts the query's own block: Section 4.1
+ *                    keeps one sink block and the 32 latest blocks, the query's included);
  *                   with window_exact != 0 the second condition is i - j < window_tokens,
  *                   the token-exact window of the rolling-buffer cache (Section 3.2), so
  *                   that a model can be trained on exactly the keys lg_sparse_decode reads

@@ -18,7 +18,7 @@ value.  All arithmetic is float64.
 
 Readings of points on which the paper is silent:
   - the window is block-granular and counts the query's own block
-    (Section 4.1: "the first block ... and the most recent 32 blocks"); with
+    (Section 4.1 keeps one sink block and the 32 latest blocks); with
     window_exact it is the token-exact window of the rolling-buffer cache
     (Section 3.2), i - j < window_tokens, which is what the decode attends;
   - the strided comb is absolute: KV block kb is retained iff kb % stride == 0;
