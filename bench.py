@@ -403,7 +403,7 @@ def main():
                  "dv": torch.empty(inp["v"].shape, dtype=o.dtype, pin_memory=True)}
         dq, dk, dv = torch.empty_like(inp["q"]), torch.empty_like(inp["k"]), torch.empty_like(inp["v"])
 
-        n_grp = next((g for g in (8, 4, 2) if cfg.B == 1 and cfg.Hkv % g == 0), 1)
+        n_grp = next((g for g in (16, 8, 4, 2) if cfg.B == 1 and cfg.Hkv % g == 0), 1)
         pg = lg.params_of(replace(cfg, Hq=cfg.Hq // n_grp, Hkv=cfg.Hkv // n_grp))
         ws_g = [lg.attn_workspace(pg, True) for _ in range(n_grp)] if n_grp > 1 else ws
 
