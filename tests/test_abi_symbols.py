@@ -139,3 +139,13 @@ def test_documents_with_several_sequences_take_a_workspace_slice_each(lib):
     assert lib.lg_sparse_attn_workspace_bytes(C.byref(p), 1) == 3 * one
     p.doc_start = None
     assert lib.lg_sparse_attn_workspace_bytes(C.byref(p), 1) < 3 * one      # shared lists without documents
+
+
+def test_missing_library_fails_loudly(tmp_path, monkeypatch):
+    """There is no CPU path: without the built CUDA library every call raises, naming the build step."""
+    monkeypatch.setattr(binding, "_lib", None)
+    monkeypatch.setattr(binding, "LIB_PATH", str(tmp_path / "nothing_here.so"))
+    with pytest.raises(RuntimeError, match="no CPU fallback"):
+        binding.load_library()
+    with pytest.raises(RuntimeError):
+        binding.lg_block_index_nnz(_good())
