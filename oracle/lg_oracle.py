@@ -260,7 +260,7 @@ def attn_keys_grad(q, k, v, do, p: Pattern, scale: float, j0: int, j1: int):
     dK = np.zeros((Hkv, j1 - j0, D))
     dV = np.zeros((Hkv, j1 - j0, D))
     for r0 in range(0, L, p.block):
-        r1 = r0 + p.block
+        r1 = min(L, r0 + p.block)          # the last block may be partial
         M = token_mask(p, r0, r1)
         if not M[:, j0:j1].any():
             continue

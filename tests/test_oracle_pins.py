@@ -300,6 +300,19 @@ def test_subset_evaluators_equal_full_oracle():
             np.testing.assert_allclose(dv, dV[:, r0:r0 + p.block], rtol=1e-11, atol=1e-12)
         dk, dv = O.attn_keys_grad(q, k, v, do, p, 0.3, 3, p.L - 5)
         np.testing.assert_allclose(dk, dK[:, 3:p.L - 5], rtol=1e-11, atol=1e-12)
+    # a sequence that ends inside a block: the last slab of rows is shorter than a block
+    for p in (O.Pattern(L=30, block=4, mode=O.MODE_SINK_WINDOW, sink_tokens=4, window_tokens=8),
+              O.Pattern(L=43, block=8, mode=O.MODE_STRIDED_LOCAL, stride_blocks=2, local_blocks=1)):
+        q, k, v, do = (_rand((4, p.L, 3), s) for s in (27, 28, 29, 30))
+        k, v = k[:2], v[:2]
+        dQ, dK, dV, Oo, LSE = O.attn_backward(q, k, v, do, p, 0.3)
+        for j0, j1 in ((0, p.L), (p.L - 3, p.L), (5, p.L - 1)):
+            dk, dv = O.attn_keys_grad(q, k, v, do, p, 0.3, j0, j1)
+            np.testing.assert_allclose(dk, dK[:, j0:j1], rtol=1e-11, atol=1e-12)
+            np.testing.assert_allclose(dv, dV[:, j0:j1], rtol=1e-11, atol=1e-12)
+        o, lse, dq = O.attn_rows(q, k, v, do, p, 0.3, p.L - 5, p.L)
+        np.testing.assert_allclose(o, Oo[:, p.L - 5:], rtol=1e-12, atol=1e-13)
+        np.testing.assert_allclose(dq, dQ[:, p.L - 5:], rtol=1e-12, atol=1e-13)
 
 
 # ------------------------------------------------------------------------- backward
