@@ -125,19 +125,21 @@ class ClockSampler:
 
 # ------------------------------------------------------------------------ oracle timing
 
-def oracle_sample(cfg, seconds_hint="~10-30 s"):
-    """Time the CPU oracle, as it stands, on a bounded sample of the workload: one head,
-    the first L/8 tokens, forward + backward.  Returns (useful TFLOP/s, description, cores)."""
+def oracle_sample(cfg, fraction=8):
+    """Time the CPU oracle, as it stands, on a bounded sample of the workload: two kv heads with
+    their query heads, the first L/fraction tokens, forward + backward.  The value is the sample's
+    own rate (its own useful FLOPs / its own time): it is not extrapolated to the whole workload.
+    Returns (useful TFLOP/s, description, cores, seconds)."""
     from oracle import lg_oracle as O
-    small = replace(cfg, B=1, Hq=2 * (cfg.Hq // cfg.Hkv), Hkv=2, L=cfg.L // 8)
+    small = replace(cfg, B=1, Hq=2 * (cfg.Hq // cfg.Hkv), Hkv=2, L=cfg.L // fraction)
     inp = synth.make_attn_inputs(small, "cpu", seed=0, with_do=True)
     q, k, v, do = (synth.to_f64(inp[x][0]) for x in ("q", "k", "v", "do"))
     t0 = time.perf_counter()
     O.attn_backward(q, k, v, do, O.Pattern.of(small), 1.0 / math.sqrt(cfg.D), rows_per_slab=cfg.block)
     dt = time.perf_counter() - t0
     tf = flops(small) / dt / 1e12
-    desc = "%s pattern, %d query heads / 2 kv heads, first %d tokens, fwd+bwd, fp64 numpy: %.1f s" % (
-        cfg.name, small.Hq, small.L, dt)
+    desc = ("sample, not extrapolated: %s pattern, %d query heads / 2 kv heads, first %d of %d tokens, fwd+bwd, "
+            "fp64 numpy, %.1f s" % (cfg.name, small.Hq, small.L, cfg.L, dt))
     return tf, desc, os.cpu_count(), dt
 
 
@@ -192,10 +194,43 @@ def aggregate_value(flops_per_rank: float, world: int, ms_step: float) -> float:
     return flops_per_rank * world / ms_step / 1e9
 
 
+def bwd_kernel_ms(lg, p, inp, o, lse, dq, dk, dv, ws, reps):
+    """Mean durations (ms) of the backward's three kernels: the caller's events are recorded between them
+    by lg_sparse_attn_bwd_marked; nothing synchronises inside the library."""
+    ev = lg.timing_events(4)
+    acc = np.zeros(3)
+    for _ in range(reps):
+        lg.lg_sparse_attn_bwd_marked(p, inp["q"], inp["k"], inp["v"], o, lse, inp["do"], dq, dk, dv, ws, ev)
+        torch.cuda.synchronize()
+        acc += [ev[i].elapsed_time(ev[i + 1]) for i in range(3)]
+    return acc / reps
+
+
+def dram_traffic_record(kernel: str):
+    """DRAM bytes per launch of `kernel` from the committed ncu summary, or None when the kernel sources
+    have changed since that capture (the record carries a hash of them)."""
+    import hashlib
+    path = os.path.join(ROOT, "profiles", "dram_traffic_cfg3_small.json")
+    if not os.path.exists(path):
+        return None, "no record"
+    with open(path) as f:
+        rec = json.load(f)
+    h = hashlib.sha256()
+    for name in rec["sources"]:
+        with open(os.path.join(ROOT, name), "rb") as f:
+            h.update(f.read())
+    if h.hexdigest() != rec["sources_sha256"]:
+        return None, "kernel sources changed since the capture %s" % rec["capture"]
+    if kernel not in rec["dram_bytes_per_launch"]:
+        return None, "kernel not in the capture %s" % rec["capture"]
+    return rec, rec["capture"]
+
+
 def bench_attn(lg, cfg, warmup, steps, want_bwd, profile_kernels=False):
     p = lg.params_of(cfg)
     inp = synth.make_attn_inputs(cfg, "cuda", seed=0, with_do=want_bwd)
     ws = lg.attn_workspace(p, want_bwd)
+    lg.lg_sparse_attn_prepare(p, ws, want_bwd)       # lists and schedules once; the timed calls launch attention kernels only
     o = torch.empty_like(inp["q"])
     lse = torch.empty(inp["q"].shape[:3], dtype=torch.float32, device="cuda")
     out = {"config": cfg.name}
@@ -211,9 +246,8 @@ def bench_attn(lg, cfg, warmup, steps, want_bwd, profile_kernels=False):
         out["fwd_bwd_ms"] = out["fwd_ms"] + out["bwd_ms"]
         out["fwd_bwd_tflops"] = flops(cfg) / out["fwd_bwd_ms"] / 1e9
         if profile_kernels:
-            ks = np.array([lg.lg_sparse_attn_bwd_profiled(p, inp["q"], inp["k"], inp["v"], o, lse, inp["do"], dq,
-                                                          dk, dv, ws) for _ in range(max(steps, 3))])
-            out["bwd_kernel_ms"] = dict(zip(("delta", "dkdv", "dq"), [float(x) for x in ks.mean(axis=0)]))
+            ks = bwd_kernel_ms(lg, p, inp, o, lse, dq, dk, dv, ws, max(steps, 3))
+            out["bwd_kernel_ms"] = dict(zip(("delta", "dkdv", "dq"), [float(x) for x in ks]))
     assert lg.lg_last_status(ws) == 0, "device-side wait expired"
     return out, (p, inp, ws, o, lse)
 
@@ -336,6 +370,10 @@ def main():
     lse = torch.empty(inp["q"].shape[:3], dtype=torch.float32, device="cuda")
     dq, dk, dv = torch.empty_like(inp["q"]), torch.empty_like(inp["k"]), torch.empty_like(inp["v"])
 
+    # The block lists and tile schedules are static (same pattern, same L every step): built once here,
+    # timed by itself, and every step below launches the four attention kernels only.
+    index_ms = time_cuda(lambda: lg.lg_sparse_attn_prepare(p, ws, True), 1, 3)
+
     def step():
         lg.lg_sparse_attn_fwd(p, inp["q"], inp["k"], inp["v"], o=o, lse=lse, workspace=ws)
         lg.lg_sparse_attn_bwd(p, inp["q"], inp["k"], inp["v"], o, lse, inp["do"], dq=dq, dk=dk, dv=dv, workspace=ws)
@@ -347,49 +385,63 @@ def main():
         dist.barrier()
     with ClockSampler(local) as clocks:
         torch.cuda.synchronize()
+        launches0 = lg.kernel_launches()
         e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
         e0.record()
         for _ in range(args.steps):
             step()
         e1.record()
         torch.cuda.synchronize()
-        # per-kernel durations inside the same clock-sampled region (synchronising variant)
+        launches = lg.kernel_launches() - launches0
+        # per-kernel durations inside the same clock-sampled region
         fwd_ms = time_cuda(lambda: lg.lg_sparse_attn_fwd(p, inp["q"], inp["k"], inp["v"], o=o, lse=lse, workspace=ws),
                            0, args.steps)
-        kms = np.array([lg.lg_sparse_attn_bwd_profiled(p, inp["q"], inp["k"], inp["v"], o, lse, inp["do"], dq, dk,
-                                                       dv, ws) for _ in range(args.steps)]).mean(axis=0)
+        kms = bwd_kernel_ms(lg, p, inp, o, lse, dq, dk, dv, ws, args.steps)
     assert lg.lg_last_status(ws) == 0, "device-side wait expired"
     ms_step = max_over_ranks(e0.elapsed_time(e1) / args.steps, dist, "cuda")
     value = aggregate_value(flops(cfg), world, ms_step)
+    clk = clocks.summary()
 
     pairs = float(pairs_per_head(cfg)) * cfg.B * cfg.Hq
     kern = {"fwd": (fwd_ms, pairs * cfg.D * 4), "bwd_dkdv": (float(kms[1]), pairs * cfg.D * 8),
             "bwd_dq": (float(kms[2]), pairs * cfg.D * 2), "bwd_delta": (float(kms[0]), 0.0)}
     dom = max(("fwd", "bwd_dkdv", "bwd_dq"), key=lambda n: kern[n][0])
     achieved = kern[dom][1] / kern[dom][0] / 1e9
-    # dram__bytes_read + dram__bytes_write of one launch, from the ncu capture of the same kernels on
-    # the 8-head x 32K case of this pattern, scaled by the (head, token) units of this workload
-    ncu_small_bytes = {"fwd": 266.5e6, "bwd_dkdv": 451.4e6, "bwd_dq": 341.2e6}
-    traffic = ncu_small_bytes[dom] * (cfg.B * cfg.Hq * cfg.L) / (8 * 32768.0)
+    # dram__bytes_read + dram__bytes_write of one launch come from the committed ncu summary of the same kernels
+    # on the 8-head x 32K case of this pattern, scaled by the (head, token) units of this workload; null once
+    # the kernel sources differ from the ones that were captured
+    rec, rec_note = dram_traffic_record(dom)
+    traffic = None
+    if rec is not None:
+        traffic = rec["dram_bytes_per_launch"][dom] * (cfg.B * cfg.Hq * cfg.L) / float(rec["units_head_tokens"])
+    kernel_ms = {k: v[0] for k, v in kern.items()}
+    kernel_ms["index_build_once"] = index_ms
     roofline = {"bound": "tensor", "kernel": dom, "achieved": achieved, "peak": peaks["bf16_sustained"],
                 "unit": "TFLOP/s", "frac": achieved / peaks["bf16_sustained"], "traffic": traffic,
-                "traffic_note": "bytes; ncu capture of the 8-head x 32K case scaled by (head, token) units",
+                "traffic_note": "bytes per launch; " + rec_note,
                 "peak_source": "%s sustained bf16 matmul" % peaks["source"],
                 "frac_of_nominal_2250": achieved / NOMINAL_BF16_TFLOPS,
-                "kernel_ms": {k: v[0] for k, v in kern.items()},
+                "kernel_ms": kernel_ms,
                 "note": "algorithmic FLOPs per launch: fwd 4D, dK/dV pass 8D, dQ pass 2D per visible pair"}
 
+    mhz = clk.get("sm_mhz")
     line = {"metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
             "warmup": args.warmup, "ms_per_step": ms_step, "higher_is_better": True, "scaling": "weak",
             "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
             "config": {"workload": cfg.name, "B": cfg.B, "Hq": cfg.Hq, "Hkv": cfg.Hkv, "L": cfg.L, "D": cfg.D,
                        "block": cfg.block, "sink_tokens": cfg.sink_tokens, "window_tokens": cfg.window_tokens,
                        "useful_flop_per_step": flops(cfg), "parallelism": "replicas x%d" % world,
-                       "l2": "inputs (8.6 GB) far larger than L2; no flush"},
+                       "l2": "inputs (8.6 GB) far larger than L2; no flush",
+                       "lists": "block lists and tile schedules built once before the timed region "
+                                "(lg_sparse_attn_prepare, %.3f ms); a step = forward + backward kernels" % index_ms},
             "pct_of_nominal_bf16_peak": 100.0 * value / world / NOMINAL_BF16_TFLOPS,
             "pct_of_measured_bf16_sustained": 100.0 * value / world / peaks["bf16_sustained"],
-            "roofline": roofline, "clocks": clocks.summary(),
-            "gpu_launches": args.steps * 19}
+            "roofline": roofline, "clocks": clk,
+            "kernel_ms": kernel_ms,
+            "kernel_ms_x_sm_mhz": {k: v * mhz for k, v in kernel_ms.items()} if mhz else None,
+            "gpu_launches": launches,
+            "gpu_launches_note": "counted by the library (lg_debug_kernel_launches) around the timed region: "
+                                 "%.1f per step" % (launches / float(args.steps))}
 
     del dq, dk, dv
     others = []
@@ -403,19 +455,21 @@ def main():
                  "dv": torch.empty(inp["v"].shape, dtype=o.dtype, pin_memory=True)}
         dq, dk, dv = torch.empty_like(inp["q"]), torch.empty_like(inp["k"]), torch.empty_like(inp["v"])
 
-        n_grp = next((g for g in (16, 8, 4, 2) if cfg.B == 1 and cfg.Hkv % g == 0), 1)
-        pg = lg.params_of(replace(cfg, Hq=cfg.Hq // n_grp, Hkv=cfg.Hkv // n_grp))
-        ws_g = [lg.attn_workspace(pg, True) for _ in range(n_grp)] if n_grp > 1 else ws
+        n_grp = next((g for g in (16, 8, 4, 2) if cfg.Hkv % g == 0), 1)
+        p_host = lg.params_of(cfg)
+        ws_g = lg.host_step_workspace(p_host, n_grp)
 
         def e2e_step():
-            # the library's host-buffer call: head groups pipelined over copy-in / compute / copy-out streams
-            lg.sparse_attn_fwd_bwd_host(p, host, h_out, dev=(inp, o, lse, dq, dk, dv, ws_g), head_groups=n_grp)
+            # the library's host-buffer entry point (C ABI): head groups pipelined over copy-in / compute /
+            # copy-out streams inside the call
+            lg.sparse_attn_fwd_bwd_host(p_host, host, h_out, dev=(inp, o, lse, dq, dk, dv, ws_g), head_groups=n_grp)
 
         e2e_ms = time_cuda(e2e_step, 1, max(2, min(args.steps, 3)))
         h2d = sum(t.numel() * t.element_size() for t in host.values())
         d2h = sum(t.numel() * t.element_size() for t in h_out.values())
         line["e2e"] = {"value": flops(cfg) / e2e_ms / 1e9, "unit": UNIT, "ms_per_step": e2e_ms,
                        "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
+                       "entry_point": "lg_sparse_attn_fwd_bwd_host (C ABI, host pointers)",
                        "pipeline": "%d head groups over copy-in / compute / copy-out streams" % n_grp}
         del host, h_out, dq, dk, dv, ws_g
     del inp, o, lse, ws
@@ -478,7 +532,7 @@ def main():
                                    "frac_of_nominal_8000": d5["gbs"] / NOMINAL_HBM_GBS,
                                    "peak_source": "%s copy bandwidth" % peaks["source"]}
     if rank == 0 and not args.no_oracle and world == 1:
-        tf, desc, cores, _ = oracle_sample(cfg)
+        tf, desc, cores, _ = oracle_sample(cfg, fraction=4)
         line["cpu_baseline"] = {"value": tf, "unit": UNIT, "cores": cores, "kind": "oracle", "sample": desc}
     if rank == 0:
         print(json.dumps(line), flush=True)

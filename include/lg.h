@@ -66,6 +66,9 @@ typedef struct {
   int32_t stride_blocks;      /* STRIDED_LOCAL: >= 1                                         */
   int32_t local_blocks;       /* STRIDED_LOCAL: >= 1 (the diagonal block is always active)   */
   int32_t window_exact;       /* SINK_WINDOW: 0 = block-granular window, 1 = token-exact     */
+  int32_t lists_prepared;     /* 0: the call builds the block lists itself (any workspace);
+                                 1: the workspace was filled by lg_sparse_attn_prepare() for
+                                 this pattern and the call only launches its attention kernels */
   float   scale;              /* softmax scale; 0 selects 1/sqrt(D)                          */
   /* Strides in ELEMENTS of (batch, head, token) for Q, K, V, O; dO and dQ use the O / Q
      strides, dK / dV the K / V strides.  All zero selects contiguous [B, H, L, D].
@@ -79,7 +82,7 @@ typedef struct {
      those of the sample, so only its first document sees them).  The calls drop every key
      block that ends before the earliest document of a query block starts; as the lists then
      differ between sequences, a call with B > 1 runs sequence by sequence (its workspace is
-     B slices of the B == 1 size; lg_sparse_attn_bwd_profiled does not take that case).
+     B slices of the B == 1 size).
      lg_build_block_index ignores this field.                                                */
   const int32_t* doc_start;
 } lg_attn_params;
@@ -108,6 +111,22 @@ lg_status lg_build_block_index(const lg_attn_params* p, int32_t* row_ptr, int32_
 /* Workspace bytes for lg_sparse_attn_fwd (want_bwd == 0) or lg_sparse_attn_bwd (!= 0). */
 size_t lg_sparse_attn_workspace_bytes(const lg_attn_params* p, int want_bwd);
 
+/* Build the block lists and the kernels' tile schedules once (Section 3.2: the mask is static
+ * and the same for all heads, so nothing has to be rebuilt from step to step).  Afterwards
+ * lg_sparse_attn_fwd (and, with want_bwd != 0, lg_sparse_attn_bwd) called with the same
+ * workspace, the same pattern (L, block, mode, sink / window / stride / local counts,
+ * window_exact, doc_start pointer) and lists_prepared = 1 launch their attention kernels only:
+ * one kernel for the forward, three for the backward.  The lists do not depend on the head
+ * counts, on D or on the strides.  With doc_start the lists also depend on the CONTENTS of that
+ * array: prepare again whenever they change.  The workspace keeps a fingerprint of what it was
+ * prepared for; a call with lists_prepared = 1 whose pattern does not match it launches kernels
+ * that do nothing, and lg_last_status() then returns LG_ERR_WORKSPACE.  In this mode the status
+ * word is not cleared from call to call: a failure stays visible until lg_last_status() reads it,
+ * and calls made in between do nothing.  workspace: device, 256-byte aligned,
+ * lg_sparse_attn_workspace_bytes(p, want_bwd) bytes.                                       */
+lg_status lg_sparse_attn_prepare(const lg_attn_params* p, void* workspace, size_t workspace_bytes,
+                                 int want_bwd, void* stream);
+
 /* O = softmax(scale * Q K^T + mask) V;  LSE_i = ln sum_j exp(scale * q_i . k_j) over the
  * visible keys.  q [B,Hq,L,D], k, v [B,Hkv,L,D], o [B,Hq,L,D] bf16 (device);
  * lse [B,Hq,L] fp32 contiguous (device).  workspace: device, 256-byte aligned.           */
@@ -124,15 +143,63 @@ lg_status lg_sparse_attn_bwd(const lg_attn_params* p, const void* q, const void*
                              void* dq, void* dk, void* dv,
                              void* workspace, size_t workspace_bytes, void* stream);
 
-/* Same computation as lg_sparse_attn_bwd, for profiling: records CUDA events between its
- * three kernels on `stream`, SYNCHRONISES the stream, and writes their durations in
- * milliseconds to kernel_ms (HOST float[3]: delta pre-pass, dK/dV pass, dQ pass).  The paper
- * has no counterpart; it exists so that a benchmark can report a per-kernel roofline.      */
-lg_status lg_sparse_attn_bwd_profiled(const lg_attn_params* p, const void* q, const void* k,
-                                      const void* v, const void* o, const float* lse,
-                                      const void* d_o, void* dq, void* dk, void* dv,
-                                      void* workspace, size_t workspace_bytes, void* stream,
-                                      float* kernel_ms);
+/* Same computation as lg_sparse_attn_bwd; in addition the CUDA events of the caller are recorded on
+ * `stream` around its kernels: events[0] before the first one, events[1] after the pre-pass
+ * (delta), events[2] after the dK/dV pass, events[3] after the dQ pass.  `events` is a HOST array
+ * of four cudaEvent_t created by the caller (with timing enabled if durations are wanted).  The
+ * call creates nothing and does not synchronise; the caller reads the events when the stream has
+ * passed them.  With doc_start and B > 1 (sequence-by-sequence execution) the events bracket the
+ * first sequence only.  (The paper has no counterpart; a benchmark uses it to report per-kernel
+ * durations.)                                                                              */
+lg_status lg_sparse_attn_bwd_marked(const lg_attn_params* p, const void* q, const void* k,
+                                    const void* v, const void* o, const float* lse,
+                                    const void* d_o, void* dq, void* dk, void* dv,
+                                    void* workspace, size_t workspace_bytes, void* stream,
+                                    void* const* events);
+
+/* ---- a whole training step on HOST buffers ---------------------------------------------- */
+
+/*
+ * Forward + backward of one attention call whose inputs and results live in HOST memory (pinned,
+ * for the copies to overlap): q, k, v, d_o are copied to the device, lg_sparse_attn_fwd and
+ * lg_sparse_attn_bwd run there, and o, lse, dq, dk, dv are copied back.  (The paper has no
+ * counterpart: its kernels sit inside a trainer whose activations are already on the GPU; this is
+ * the end-to-end form of the same two calls for a caller who holds host tensors.)
+ *
+ * Heads are independent, so the step is cut into `head_groups` groups of kv heads (with their
+ * query heads) that move through three streams: while one group computes on `stream_compute`, the
+ * next one's inputs arrive on `stream_in` and the previous one's results leave on `stream_out`;
+ * the two copy directions share the link.  head_groups must divide Hkv (1 = no pipelining).
+ *
+ *   host tensors   : contiguous [B,H,L,D] bf16 (lse_host [B,Hq,L] fp32); the strides in `p` are
+ *                    ignored.  doc_start in `p` (a DEVICE array, as always) is honoured.
+ *   dev            : DEVICE staging buffers of the same shapes, owned by the caller, and one
+ *                    workspace of lg_sparse_attn_fwd_bwd_host_workspace_bytes() bytes (256-byte
+ *                    aligned), which the call cuts into one slice per group.
+ *   streams        : three cudaStream_t of the caller.  The call waits for nothing that was
+ *                    enqueued on them before; it creates a few timing-less CUDA events for the
+ *                    hand-over between the streams and destroys them before returning.  On
+ *                    return everything is enqueued; the host results are complete when
+ *                    stream_out is idle (stream_in and stream_compute are then idle too).
+ * Results are bit-identical to the two device calls on the whole tensors.  lg_last_status() on
+ * dev->workspace reports a device-side failure of any group.
+ */
+typedef struct {
+  void* q; void* k; void* v; void* d_o;      /* inputs  [B,Hq,L,D], [B,Hkv,L,D] x2, [B,Hq,L,D] */
+  void* o; float* lse; void* dq; void* dk; void* dv;
+  void* workspace;
+  size_t workspace_bytes;
+} lg_device_step_buffers;
+
+size_t lg_sparse_attn_fwd_bwd_host_workspace_bytes(const lg_attn_params* p, int head_groups);
+
+lg_status lg_sparse_attn_fwd_bwd_host(const lg_attn_params* p,
+                                      const void* q_host, const void* k_host, const void* v_host,
+                                      const void* d_o_host,
+                                      void* o_host, float* lse_host, void* dq_host, void* dk_host,
+                                      void* dv_host,
+                                      const lg_device_step_buffers* dev, int head_groups,
+                                      void* stream_in, void* stream_compute, void* stream_out);
 
 /* ---- serving: rolling-buffer cache and decode (Section 3.2) --------------------------- */
 
@@ -254,12 +321,20 @@ lg_status lg_selftest_wait_timeout(void* workspace, void* stream);
 
 /* ---- status ------------------------------------------------------------------------- */
 
-/* Synchronises `stream`, reads the error word the kernels keep at the start of
- * `workspace` (attention or decode workspace) and clears it.  LG_OK, or
- * LG_ERR_DEVICE_TIMEOUT if a bounded wait expired in a kernel that used it.              */
+/* Synchronises `stream`, reads the status words the kernels keep at the start of
+ * `workspace` (attention or decode workspace) and clears them.  LG_OK;
+ * LG_ERR_DEVICE_TIMEOUT if a bounded wait expired in a kernel that used the workspace since
+ * the last call of this function (a later call on the same workspace does not hide it);
+ * LG_ERR_WORKSPACE if a call with lists_prepared = 1 found lists of another pattern.       */
 lg_status lg_last_status(void* workspace, void* stream);
 
 const char* lg_status_string(lg_status s);
+
+/* Diagnostic (the paper has no counterpart): the number of CUDA kernels this library has launched
+ * in the calling process so far, over all entry points and devices.  A benchmark takes the
+ * difference around its timed region.  The counter is the one piece of process-wide state the
+ * library keeps besides the fixed array of lg_sparse_decode_static; nothing depends on it.   */
+int64_t lg_debug_kernel_launches(void);
 
 #ifdef __cplusplus
 }

@@ -29,9 +29,15 @@ class AttnParams(C.Structure):
     _fields_ = [("B", C.c_int32), ("Hq", C.c_int32), ("Hkv", C.c_int32), ("L", C.c_int32), ("D", C.c_int32),
                 ("block", C.c_int32), ("mode", C.c_int32), ("sink_tokens", C.c_int32),
                 ("window_tokens", C.c_int32), ("stride_blocks", C.c_int32), ("local_blocks", C.c_int32),
-                ("window_exact", C.c_int32), ("scale", C.c_float),
+                ("window_exact", C.c_int32), ("lists_prepared", C.c_int32), ("scale", C.c_float),
                 ("q_strides", C.c_int64 * 3), ("k_strides", C.c_int64 * 3), ("v_strides", C.c_int64 * 3),
                 ("o_strides", C.c_int64 * 3), ("doc_start", C.c_void_p)]
+
+
+class DeviceStepBuffers(C.Structure):
+    _fields_ = [("q", C.c_void_p), ("k", C.c_void_p), ("v", C.c_void_p), ("d_o", C.c_void_p),
+                ("o", C.c_void_p), ("lse", C.c_void_p), ("dq", C.c_void_p), ("dk", C.c_void_p), ("dv", C.c_void_p),
+                ("workspace", C.c_void_p), ("workspace_bytes", C.c_size_t)]
 
 
 class DecodeParams(C.Structure):
@@ -48,9 +54,12 @@ SYMBOLS = {
     "lg_block_index_bytes": (_sz, [C.POINTER(AttnParams)]),
     "lg_build_block_index": (C.c_int, [C.POINTER(AttnParams), _vp, _vp, _vp, _vp, C.POINTER(C.c_int64), _vp]),
     "lg_sparse_attn_workspace_bytes": (_sz, [C.POINTER(AttnParams), C.c_int]),
+    "lg_sparse_attn_prepare": (C.c_int, [C.POINTER(AttnParams), _vp, _sz, C.c_int, _vp]),
     "lg_sparse_attn_fwd": (C.c_int, [C.POINTER(AttnParams), _vp, _vp, _vp, _vp, _vp, _vp, _sz, _vp]),
     "lg_sparse_attn_bwd": (C.c_int, [C.POINTER(AttnParams)] + [_vp] * 9 + [_vp, _sz, _vp]),
-    "lg_sparse_attn_bwd_profiled": (C.c_int, [C.POINTER(AttnParams)] + [_vp] * 9 + [_vp, _sz, _vp, C.POINTER(C.c_float)]),
+    "lg_sparse_attn_bwd_marked": (C.c_int, [C.POINTER(AttnParams)] + [_vp] * 9 + [_vp, _sz, _vp, C.POINTER(_vp)]),
+    "lg_sparse_attn_fwd_bwd_host_workspace_bytes": (_sz, [C.POINTER(AttnParams), C.c_int]),
+    "lg_sparse_attn_fwd_bwd_host": (C.c_int, [C.POINTER(AttnParams)] + [_vp] * 9 + [_vp, C.c_int, _vp, _vp, _vp]),
     "lg_kv_ring_append": (C.c_int, [C.POINTER(DecodeParams), _vp, _vp, _vp, _vp, C.c_int32, _vp, _vp]),
     "lg_sparse_decode_workspace_bytes": (_sz, [C.POINTER(DecodeParams)]),
     "lg_sparse_decode_workspace_init": (C.c_int, [_vp, _sz, _vp]),
@@ -62,6 +71,7 @@ SYMBOLS = {
     "lg_selftest_wait_timeout": (C.c_int, [_vp, _vp]),
     "lg_last_status": (C.c_int, [_vp, _vp]),
     "lg_status_string": (C.c_char_p, [C.c_int]),
+    "lg_debug_kernel_launches": (C.c_int64, []),
 }
 
 
@@ -156,6 +166,16 @@ def attn_workspace(p: AttnParams, want_bwd: bool, device="cuda") -> torch.Tensor
     return torch.empty(n, dtype=torch.uint8, device=device)
 
 
+def lg_sparse_attn_prepare(p: AttnParams, workspace: torch.Tensor, want_bwd: bool) -> AttnParams:
+    """Build lists and schedules once into `workspace`; sets p.lists_prepared so that later forward /
+    backward calls with this params object and workspace launch their attention kernels only."""
+    p.lists_prepared = 0
+    _check(load_library().lg_sparse_attn_prepare(C.byref(p), workspace.data_ptr(), workspace.numel(), int(want_bwd),
+                                                 _stream()), "lg_sparse_attn_prepare")
+    p.lists_prepared = 1
+    return p
+
+
 def lg_sparse_attn_fwd(p: AttnParams, q, k, v, o=None, lse=None, workspace=None):
     """q [B,Hq,L,D], k, v [B,Hkv,L,D] bf16 CUDA tensors -> (o bf16, lse fp32 [B,Hq,L])."""
     lib = load_library()
@@ -184,78 +204,68 @@ def lg_sparse_attn_bwd(p: AttnParams, q, k, v, o, lse, d_o, dq=None, dk=None, dv
     return dq, dk, dv
 
 
-def lg_sparse_attn_bwd_profiled(p: AttnParams, q, k, v, o, lse, d_o, dq, dk, dv, workspace):
-    """As lg_sparse_attn_bwd, synchronising; returns [delta_ms, dkdv_ms, dq_ms]."""
+def lg_sparse_attn_bwd_marked(p: AttnParams, q, k, v, o, lse, d_o, dq, dk, dv, workspace, events):
+    """As lg_sparse_attn_bwd; records the caller's four torch.cuda.Event objects (timing enabled, each
+    recorded once before so that its handle exists) around the delta, dK/dV and dQ kernels.  Does not
+    synchronise: read event durations after the stream has passed them."""
     p.q_strides, p.k_strides, p.v_strides, p.o_strides = _strides3(q), _strides3(k), _strides3(v), _strides3(o)
-    ms = (C.c_float * 3)()
-    _check(load_library().lg_sparse_attn_bwd_profiled(
+    assert len(events) == 4
+    ev = (C.c_void_p * 4)(*[e.cuda_event for e in events])
+    _check(load_library().lg_sparse_attn_bwd_marked(
         C.byref(p), q.data_ptr(), k.data_ptr(), v.data_ptr(), o.data_ptr(), lse.data_ptr(), d_o.data_ptr(),
-        dq.data_ptr(), dk.data_ptr(), dv.data_ptr(), workspace.data_ptr(), workspace.numel(), _stream(), ms),
-        "lg_sparse_attn_bwd_profiled")
-    return [float(x) for x in ms]
+        dq.data_ptr(), dk.data_ptr(), dv.data_ptr(), workspace.data_ptr(), workspace.numel(), _stream(), ev),
+        "lg_sparse_attn_bwd_marked")
+
+
+def timing_events(n: int = 4):
+    """n CUDA events with timing, each recorded once so that the driver object behind it exists."""
+    evs = [torch.cuda.Event(enable_timing=True) for _ in range(n)]
+    for e in evs:
+        e.record()
+    return evs
+
+
+def host_step_workspace(p: AttnParams, head_groups: int, device="cuda") -> torch.Tensor:
+    n = load_library().lg_sparse_attn_fwd_bwd_host_workspace_bytes(C.byref(p), head_groups)
+    if n == 0:
+        raise LgError(-1, "lg_sparse_attn_fwd_bwd_host_workspace_bytes")
+    return torch.empty(n, dtype=torch.uint8, device=device)
+
+
+def host_step_groups(p: AttnParams, head_groups: int) -> int:
+    """The number of head groups a step can be cut into: `head_groups` if it divides Hkv, else 1."""
+    return head_groups if (head_groups > 1 and p.Hkv % head_groups == 0) else 1
 
 
 def sparse_attn_fwd_bwd_host(p: AttnParams, host_in, host_out, dev=None, head_groups: int = 4):
-    """End-to-end training step with HOST buffers: copies pinned q, k, v, do to the device,
-    runs lg_sparse_attn_fwd and lg_sparse_attn_bwd, and copies o, lse, dq, dk, dv back into the
-    pinned tensors of `host_out`.  `dev` optionally supplies preallocated device buffers
-    (inputs dict, o, lse, dq, dk, dv, workspace or list of workspaces).  All arithmetic runs in
-    the CUDA library.
-
-    Heads are independent, so with B == 1 the step is cut into `head_groups` groups of kv heads
-    (with their query heads) that move through three streams: while one group computes, the next
-    one's inputs arrive and the previous one's results leave, and the two copy directions share the
-    link.  The library calls are the same, on strided views of the full tensors."""
+    """End-to-end training step with HOST buffers through lg_sparse_attn_fwd_bwd_host: pinned q, k, v, do
+    go to the device, forward and backward run there, and o, lse, dq, dk, dv come back into the pinned
+    tensors of `host_out`; head groups are pipelined over three streams inside the library call.
+    `dev` optionally supplies preallocated device buffers (inputs dict, o, lse, dq, dk, dv, workspace of
+    host_step_workspace(p, groups) bytes).  This wrapper only marshals pointers and streams."""
+    n_groups = host_step_groups(p, head_groups)
     if dev is None:
         d_in = {k: torch.empty(v.shape, dtype=v.dtype, device="cuda") for k, v in host_in.items()}
         o = torch.empty_like(d_in["q"])
         lse = torch.empty(d_in["q"].shape[:3], dtype=torch.float32, device="cuda")
         dq, dk, dv = torch.empty_like(d_in["q"]), torch.empty_like(d_in["k"]), torch.empty_like(d_in["v"])
-        ws = None
+        ws = host_step_workspace(p, n_groups)
     else:
         d_in, o, lse, dq, dk, dv, ws = dev
-    n_groups = head_groups if (p.B == 1 and head_groups > 1 and p.Hkv % head_groups == 0) else 1
-    if n_groups == 1:
-        ws = attn_workspace(p, True) if ws is None else (ws[0] if isinstance(ws, (list, tuple)) else ws)
-        for name in ("q", "k", "v", "do"):
-            d_in[name].copy_(host_in[name], non_blocking=True)
-        lg_sparse_attn_fwd(p, d_in["q"], d_in["k"], d_in["v"], o=o, lse=lse, workspace=ws)
-        lg_sparse_attn_bwd(p, d_in["q"], d_in["k"], d_in["v"], o, lse, d_in["do"], dq=dq, dk=dk, dv=dv, workspace=ws)
-        for name, t in (("o", o), ("lse", lse), ("dq", dq), ("dk", dk), ("dv", dv)):
-            host_out[name].copy_(t, non_blocking=True)
-        return host_out
-
-    G = p.Hq // p.Hkv
-    kv_per = p.Hkv // n_groups
-    pg = attn_params(p.B, kv_per * G, kv_per, p.L, p.D, p.block, p.mode, p.sink_tokens, p.window_tokens,
-                     p.stride_blocks, p.local_blocks, p.scale, bool(p.window_exact),
-                     getattr(p, "_doc_start_ref", None))
-    if not isinstance(ws, (list, tuple)) or len(ws) < n_groups:
-        ws = [attn_workspace(pg, True) for _ in range(n_groups)]   # groups overlap in time: one workspace each
+    for t in list(host_in.values()) + list(host_out.values()) + list(d_in.values()) + [o, lse, dq, dk, dv]:
+        assert t.is_contiguous()
+    bufs = DeviceStepBuffers(d_in["q"].data_ptr(), d_in["k"].data_ptr(), d_in["v"].data_ptr(), d_in["do"].data_ptr(),
+                             o.data_ptr(), lse.data_ptr(), dq.data_ptr(), dk.data_ptr(), dv.data_ptr(),
+                             ws.data_ptr(), ws.numel())
     cur = torch.cuda.current_stream()
     s_in, s_cmp, s_out = (_side_stream(i) for i in range(3))
     for st in (s_in, s_cmp, s_out):
         st.wait_stream(cur)
-    for g in range(n_groups):
-        kv = slice(g * kv_per, (g + 1) * kv_per)
-        qh = slice(g * kv_per * G, (g + 1) * kv_per * G)
-        sl = {"q": qh, "k": kv, "v": kv, "do": qh}
-        ev_in, ev_cmp = torch.cuda.Event(), torch.cuda.Event()
-        with torch.cuda.stream(s_in):
-            for name in ("q", "k", "v", "do"):
-                d_in[name][:, sl[name]].copy_(host_in[name][:, sl[name]], non_blocking=True)
-            ev_in.record()
-        with torch.cuda.stream(s_cmp):
-            s_cmp.wait_event(ev_in)
-            qg, kg, vg, dog = (d_in[n][:, sl[n]] for n in ("q", "k", "v", "do"))
-            og, lg_ = o[:, qh], lse[:, qh]
-            lg_sparse_attn_fwd(pg, qg, kg, vg, o=og, lse=lg_, workspace=ws[g])
-            lg_sparse_attn_bwd(pg, qg, kg, vg, og, lg_, dog, dq=dq[:, qh], dk=dk[:, kv], dv=dv[:, kv], workspace=ws[g])
-            ev_cmp.record()
-        with torch.cuda.stream(s_out):
-            s_out.wait_event(ev_cmp)
-            for name, t, hs in (("o", o, qh), ("lse", lse, qh), ("dq", dq, qh), ("dk", dk, kv), ("dv", dv, kv)):
-                host_out[name][:, hs].copy_(t[:, hs], non_blocking=True)
+    _check(load_library().lg_sparse_attn_fwd_bwd_host(
+        C.byref(p), host_in["q"].data_ptr(), host_in["k"].data_ptr(), host_in["v"].data_ptr(), host_in["do"].data_ptr(),
+        host_out["o"].data_ptr(), host_out["lse"].data_ptr(), host_out["dq"].data_ptr(), host_out["dk"].data_ptr(),
+        host_out["dv"].data_ptr(), C.byref(bufs), n_groups, s_in.cuda_stream, s_cmp.cuda_stream, s_out.cuda_stream),
+        "lg_sparse_attn_fwd_bwd_host")
     for st in (s_in, s_cmp, s_out):
         cur.wait_stream(st)
     return host_out
@@ -354,6 +364,11 @@ def lg_sparse_decode_static(p: DecodeParams, q, k_cache, v_cache, n_tokens, o, l
 def lg_selftest_wait_timeout(workspace: torch.Tensor) -> None:
     """Launch the one-warp kernel whose bounded wait must expire (see include/lg.h)."""
     _check(load_library().lg_selftest_wait_timeout(workspace.data_ptr(), _stream()), "lg_selftest_wait_timeout")
+
+
+def kernel_launches() -> int:
+    """Kernels launched by the library in this process so far (diagnostic counter)."""
+    return int(load_library().lg_debug_kernel_launches())
 
 
 def lg_last_status(workspace: torch.Tensor) -> int:

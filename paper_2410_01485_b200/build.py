@@ -9,7 +9,7 @@ from concurrent.futures import ThreadPoolExecutor
 HERE = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(HERE, "csrc")
 LIB = os.path.join(HERE, "liblg_sparse_attn.so")
-SOURCES = ["lg_api.cu", "lg_fwd.cu", "lg_bwd.cu", "lg_decode.cu"]
+SOURCES = ["lg_api.cu", "lg_fwd.cu", "lg_bwd.cu", "lg_decode.cu", "lg_host_step.cu"]
 NVCC_FLAGS = ["-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",
               "-Xcompiler", "-fPIC", "--expt-relaxed-constexpr", "-Xptxas", "-v"]
 

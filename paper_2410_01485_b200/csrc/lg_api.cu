@@ -2,6 +2,7 @@
 #include <math.h>
 #include <string.h>
 
+#include <atomic>
 #include <mutex>
 
 #include "lg_common.cuh"
@@ -9,6 +10,9 @@
 #include "lg_index.cuh"
 
 namespace lg {
+
+static std::atomic<long long> g_kernel_launches{0};
+void note_launch() { g_kernel_launches.fetch_add(1, std::memory_order_relaxed); }
 
 lg_status check_arch() {
   int dev = 0, major = 0;
@@ -83,6 +87,9 @@ lg_status resolve(const lg_attn_params* p, Resolved* r) {
   if (reinterpret_cast<uintptr_t>(p->doc_start) & 3) return LG_ERR_INVALID_ARG;
   r->doc_start = p->doc_start;
   r->error_word = nullptr;
+  if (p->lists_prepared != 0 && p->lists_prepared != 1) return LG_ERR_INVALID_ARG;
+  r->lists_prepared = p->lists_prepared;
+  r->expect_fp = r->expect_fp2 = 0;
   // nnz from the per-row counts of each pattern
   int64_t nnz = 0;
   const PatternDev& pt = r->pat;
@@ -139,15 +146,43 @@ WsLayout ws_layout(const Resolved& r, bool want_bwd) {
 lg_status launch_index_build(const Resolved& r, int32_t* row_ptr, int32_t* col_idx, int32_t* col_ptr,
                              int32_t* row_idx, cudaStream_t stream) {
   const int nB = r.pat.nB;
-  index_count_kernel<<<nB, 128, 0, stream>>>(r.pat, row_ptr, col_ptr);
-  index_scan_kernel<<<2, 1024, 0, stream>>>(row_ptr, col_ptr, nB);
-  index_fill_kernel<<<nB, 64, 0, stream>>>(r.pat, row_ptr, col_idx, col_ptr, row_idx);
+  index_count_kernel<<<nB, 128, 0, stream>>>(r.pat, row_ptr, col_ptr); note_launch();
+  index_scan_kernel<<<2, 1024, 0, stream>>>(row_ptr, col_ptr, nB); note_launch();
+  index_fill_kernel<<<nB, 64, 0, stream>>>(r.pat, row_ptr, col_idx, col_ptr, row_idx); note_launch();
   return cudaGetLastError() == cudaSuccess ? LG_OK : LG_ERR_CUDA;
 }
 
-lg_status prepare_workspace(const Resolved& r, const WsLayout& w, uint8_t* ws, bool want_bwd,
-                            cudaStream_t stream) {
-  if (cudaMemsetAsync(ws, 0, sizeof(WsHeader), stream) != cudaSuccess) return LG_ERR_CUDA;
+// Which lists a workspace holds: FNV-1a over everything the lists and schedules depend on.
+unsigned long long pattern_fingerprint(const Resolved& r, bool has_bwd) {
+  unsigned long long h = 1469598103934665603ull;
+  auto mix = [&](unsigned long long v) {
+    for (int i = 0; i < 8; ++i) { h ^= (v >> (8 * i)) & 0xffu; h *= 1099511628211ull; }
+  };
+  mix(static_cast<unsigned long long>(r.L)); mix(r.block); mix(r.mode); mix(r.pat.ns); mix(r.pat.nw);
+  mix(r.pat.stride); mix(r.pat.nl); mix(r.exact_w); mix(has_bwd ? 1 : 0);
+  mix(reinterpret_cast<uintptr_t>(r.doc_start)); mix(r.doc_start ? r.B : 0);
+  return h ? h : 1;
+}
+
+// Start of a call that (re)builds the lists: a header that was never initialised is reset, an
+// error word nobody has read yet moves to `latched`, and the fingerprint is withdrawn until the
+// lists are whole again.
+__global__ void header_begin_kernel(WsHeader* h) {
+  if (h->magic != kWsMagic) { h->magic = kWsMagic; h->latched = 0; }
+  else if (h->error_word != 0 && h->latched == 0) h->latched = h->error_word;
+  h->error_word = 0;
+  h->fingerprint = 0;
+}
+__global__ void header_stamp_kernel(WsHeader* h, unsigned long long fp) { h->fingerprint = fp; }
+
+lg_status begin_workspace(uint8_t* ws, cudaStream_t stream) {
+  header_begin_kernel<<<1, 1, 0, stream>>>(reinterpret_cast<WsHeader*>(ws)); note_launch();
+  return cudaGetLastError() == cudaSuccess ? LG_OK : LG_ERR_CUDA;
+}
+
+// what: bit 0 = the forward's super-tile schedule, bit 1 = the backward's schedules
+lg_status prepare_workspace(const Resolved& r, const WsLayout& w, uint8_t* ws, int what, cudaStream_t stream) {
+  const bool want_fwd = (what & 1) != 0, want_bwd = (what & 2) != 0;
   auto i32 = [&](size_t off) { return reinterpret_cast<int32_t*>(ws + off); };
   // The lists are shared by all sequences of the batch, so documents can only prune them when there
   // is one sequence (the usual case for long packed samples); otherwise they stay the pattern's own.
@@ -156,25 +191,25 @@ lg_status prepare_workspace(const Resolved& r, const WsLayout& w, uint8_t* ws, b
   lg_status s = launch_index_build(rl, i32(w.row_ptr), i32(w.col_idx), i32(w.col_ptr), i32(w.row_idx), stream);
   if (s != LG_OK) return s;
   const int R = 128 / r.block;
-  if (!want_bwd) {   // the forward walks super-tiles of 256 rows; the backward passes have their own schedules
+  if (want_fwd) {   // the forward walks super-tiles of 256 rows; the backward passes have their own schedules
     tile_merge4_kernel<<<(r.n_stiles + 127) / 128, 128, 0, stream>>>(i32(w.row_ptr), i32(w.col_idx), r.pat.nB, 2 * R,
-                                                                     r.n_stiles, i32(w.sq_cnt), i32(w.sq_ent));
-    tile_order_kernel<<<(r.n_stiles + 127) / 128, 128, 0, stream>>>(i32(w.sq_cnt), r.n_stiles, i32(w.sq_order));
+                                                                     r.n_stiles, i32(w.sq_cnt), i32(w.sq_ent)); note_launch();
+    tile_order_kernel<<<(r.n_stiles + 127) / 128, 128, 0, stream>>>(i32(w.sq_cnt), r.n_stiles, i32(w.sq_order)); note_launch();
   }
   if (want_bwd) {
     const int nB = r.pat.nB, nt = r.n_ktiles;
     tile_merge_kernel<<<(r.n_qtiles + 127) / 128, 128, 0, stream>>>(i32(w.row_ptr), i32(w.col_idx), nB, R, r.n_qtiles,
-                                                                    i32(w.qt_cnt), i32(w.qt_ent));
-    tile_order_kernel<<<(r.n_qtiles + 127) / 128, 128, 0, stream>>>(i32(w.qt_cnt), r.n_qtiles, i32(w.qt_order));
-    kv_tile_cols_kernel<<<(nt * R + 127) / 128, 128, 0, stream>>>(i32(w.col_ptr), nB, R, nt, i32(w.kt_cols));
-    kv_tile_len_kernel<<<(nt + 127) / 128, 128, 0, stream>>>(i32(w.col_ptr), i32(w.kt_cols), R, nt, i32(w.kt_off));
-    index_scan_kernel<<<1, 1024, 0, stream>>>(i32(w.kt_off), i32(w.kt_off), nt);
+                                                                    i32(w.qt_cnt), i32(w.qt_ent)); note_launch();
+    tile_order_kernel<<<(r.n_qtiles + 127) / 128, 128, 0, stream>>>(i32(w.qt_cnt), r.n_qtiles, i32(w.qt_order)); note_launch();
+    kv_tile_cols_kernel<<<(nt * R + 127) / 128, 128, 0, stream>>>(i32(w.col_ptr), nB, R, nt, i32(w.kt_cols)); note_launch();
+    kv_tile_len_kernel<<<(nt + 127) / 128, 128, 0, stream>>>(i32(w.col_ptr), i32(w.kt_cols), R, nt, i32(w.kt_off)); note_launch();
+    index_scan_kernel<<<1, 1024, 0, stream>>>(i32(w.kt_off), i32(w.kt_off), nt); note_launch();
     kv_tile_merge_kernel<<<(nt + 127) / 128, 128, 0, stream>>>(i32(w.col_ptr), i32(w.row_idx), i32(w.kt_cols),
-                                                               i32(w.kt_off), R, nt, i32(w.kt_cnt), i32(w.kt_ent));
-    tile_order_kernel<<<(nt + 127) / 128, 128, 0, stream>>>(i32(w.kt_cnt), nt, i32(w.kt_order));
+                                                               i32(w.kt_off), R, nt, i32(w.kt_cnt), i32(w.kt_ent)); note_launch();
+    tile_order_kernel<<<(nt + 127) / 128, 128, 0, stream>>>(i32(w.kt_cnt), nt, i32(w.kt_order)); note_launch();
     if (r.doc_start) {
       const int64_t n = static_cast<int64_t>(r.B) * r.L;
-      doc_end_kernel<<<static_cast<unsigned>((n + 255) / 256), 256, 0, stream>>>(r.doc_start, i32(w.doc_end), r.B, r.L);
+      doc_end_kernel<<<static_cast<unsigned>((n + 255) / 256), 256, 0, stream>>>(r.doc_start, i32(w.doc_end), r.B, r.L); note_launch();
     }
   }
   return cudaGetLastError() == cudaSuccess ? LG_OK : LG_ERR_CUDA;
@@ -320,7 +355,7 @@ static Resolved one_sequence(const Resolved& r, int b, void* workspace) {
   Resolved r1 = r;
   r1.B = 1;
   r1.doc_start = r.doc_start + static_cast<int64_t>(b) * r.L;
-  r1.error_word = static_cast<unsigned int*>(workspace);
+  r1.error_word = r.error_word ? r.error_word : static_cast<unsigned int*>(workspace);
   return r1;
 }
 
@@ -372,11 +407,32 @@ size_t lg_sparse_attn_workspace_bytes(const lg_attn_params* p, int want_bwd) {
   return attn_workspace_total(r, want_bwd != 0);
 }
 
-lg_status lg_sparse_attn_fwd(const lg_attn_params* p, const void* q, const void* k, const void* v, void* o,
-                             float* lse, void* workspace, size_t workspace_bytes, void* stream) {
+lg_status lg_sparse_attn_prepare(const lg_attn_params* p, void* workspace, size_t workspace_bytes, int want_bwd,
+                                 void* stream) {
   Resolved r;
   lg_status s = resolve(p, &r);
   if (s != LG_OK) return s;
+  if (!workspace || (reinterpret_cast<uintptr_t>(workspace) & 255)) return LG_ERR_INVALID_ARG;
+  if (per_sequence(r)) return LG_ERR_UNSUPPORTED;   // lists per sequence: those calls build them themselves
+  if (workspace_bytes < attn_workspace_total(r, want_bwd != 0)) return LG_ERR_WORKSPACE;
+  if ((s = check_arch()) != LG_OK) return s;
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  uint8_t* ws = static_cast<uint8_t*>(workspace);
+  if ((s = begin_workspace(ws, st)) != LG_OK) return s;
+  if ((s = prepare_workspace(r, ws_layout(r, want_bwd != 0), ws, want_bwd ? 3 : 1, st)) != LG_OK) return s;
+  header_stamp_kernel<<<1, 1, 0, st>>>(reinterpret_cast<WsHeader*>(ws), pattern_fingerprint(r, want_bwd != 0)); note_launch();
+  return cudaGetLastError() == cudaSuccess ? LG_OK : LG_ERR_CUDA;
+}
+
+}  // extern "C"
+
+namespace lg {
+lg_status attn_fwd_entry(const lg_attn_params* p, const void* q, const void* k, const void* v, void* o, float* lse,
+                         void* workspace, size_t workspace_bytes, void* stream, unsigned int* status_word) {
+  Resolved r;
+  lg_status s = resolve(p, &r);
+  if (s != LG_OK) return s;
+  r.error_word = status_word;
   if (!q || !k || !v || !o || !lse || !workspace) return LG_ERR_INVALID_ARG;
   if (!aligned16(q) || !aligned16(k) || !aligned16(v) || !aligned16(o) || !aligned16(lse)) return LG_ERR_INVALID_ARG;
   if (reinterpret_cast<uintptr_t>(workspace) & 255) return LG_ERR_INVALID_ARG;
@@ -384,13 +440,20 @@ lg_status lg_sparse_attn_fwd(const lg_attn_params* p, const void* q, const void*
   if ((s = check_arch()) != LG_OK) return s;
   cudaStream_t st = static_cast<cudaStream_t>(stream);
   uint8_t* ws = static_cast<uint8_t*>(workspace);
+  if (r.lists_prepared) {   // lists and schedules are in the workspace (the kernel checks the fingerprint)
+    if (per_sequence(r)) return LG_ERR_UNSUPPORTED;
+    r.expect_fp = pattern_fingerprint(r, false);
+    r.expect_fp2 = pattern_fingerprint(r, true);
+    return launch_fwd(r, ws_layout(r, false), q, k, v, o, lse, ws, st);
+  }
+  if ((s = begin_workspace(ws, st)) != LG_OK) return s;
   if (per_sequence(r)) {
     const size_t per = attn_workspace_total(r, false) / r.B;
     for (int b = 0; b < r.B; ++b) {
       const Resolved r1 = one_sequence(r, b, workspace);
       const WsLayout w1 = ws_layout(r1, false);
       uint8_t* wsb = ws + b * per;
-      if ((s = prepare_workspace(r1, w1, wsb, false, st)) != LG_OK) return s;
+      if ((s = prepare_workspace(r1, w1, wsb, 1, st)) != LG_OK) return s;
       s = launch_fwd(r1, w1, seq_ptr(q, b, r.qs[0]), seq_ptr(k, b, r.ks[0]), seq_ptr(v, b, r.vs[0]),
                      seq_ptr(o, b, r.os[0]), lse + static_cast<int64_t>(b) * r.Hq * r.L, wsb, st);
       if (s != LG_OK) return s;
@@ -398,16 +461,17 @@ lg_status lg_sparse_attn_fwd(const lg_attn_params* p, const void* q, const void*
     return LG_OK;
   }
   const WsLayout w = ws_layout(r, false);
-  if ((s = prepare_workspace(r, w, ws, false, st)) != LG_OK) return s;
+  if ((s = prepare_workspace(r, w, ws, 1, st)) != LG_OK) return s;
   return launch_fwd(r, w, q, k, v, o, lse, ws, st);
 }
 
-static lg_status bwd_common(const lg_attn_params* p, const void* q, const void* k, const void* v, const void* o,
-                            const float* lse, const void* d_o, void* dq, void* dk, void* dv, void* workspace,
-                            size_t workspace_bytes, void* stream, cudaEvent_t* marks) {
+lg_status attn_bwd_entry(const lg_attn_params* p, const void* q, const void* k, const void* v, const void* o,
+                         const float* lse, const void* d_o, void* dq, void* dk, void* dv, void* workspace,
+                         size_t workspace_bytes, void* stream, cudaEvent_t* marks, unsigned int* status_word) {
   Resolved r;
   lg_status s = resolve(p, &r);
   if (s != LG_OK) return s;
+  r.error_word = status_word;
   if (!q || !k || !v || !o || !lse || !d_o || !dq || !dk || !dv || !workspace) return LG_ERR_INVALID_ARG;
   if (!aligned16(q) || !aligned16(k) || !aligned16(v) || !aligned16(o) || !aligned16(lse) || !aligned16(d_o) ||
       !aligned16(dq) || !aligned16(dk) || !aligned16(dv))
@@ -417,49 +481,57 @@ static lg_status bwd_common(const lg_attn_params* p, const void* q, const void* 
   if ((s = check_arch()) != LG_OK) return s;
   cudaStream_t st = static_cast<cudaStream_t>(stream);
   uint8_t* ws = static_cast<uint8_t*>(workspace);
+  if (r.lists_prepared) {
+    if (per_sequence(r)) return LG_ERR_UNSUPPORTED;
+    r.expect_fp = r.expect_fp2 = pattern_fingerprint(r, true);
+    return launch_bwd(r, ws_layout(r, true), q, k, v, o, lse, d_o, dq, dk, dv, ws, st, marks);
+  }
+  if ((s = begin_workspace(ws, st)) != LG_OK) return s;
   if (per_sequence(r)) {
-    if (marks) return LG_ERR_UNSUPPORTED;   // the per-kernel timing variant covers one launch of each kernel
     const size_t per = attn_workspace_total(r, true) / r.B;
     for (int b = 0; b < r.B; ++b) {
       const Resolved r1 = one_sequence(r, b, workspace);
       const WsLayout w1 = ws_layout(r1, true);
       uint8_t* wsb = ws + b * per;
-      if ((s = prepare_workspace(r1, w1, wsb, true, st)) != LG_OK) return s;
+      if ((s = prepare_workspace(r1, w1, wsb, 2, st)) != LG_OK) return s;
       s = launch_bwd(r1, w1, seq_ptr(q, b, r.qs[0]), seq_ptr(k, b, r.ks[0]), seq_ptr(v, b, r.vs[0]),
                      seq_ptr(o, b, r.os[0]), lse + static_cast<int64_t>(b) * r.Hq * r.L, seq_ptr(d_o, b, r.os[0]),
-                     seq_ptr(dq, b, r.qs[0]), seq_ptr(dk, b, r.ks[0]), seq_ptr(dv, b, r.vs[0]), wsb, st, nullptr);
+                     seq_ptr(dq, b, r.qs[0]), seq_ptr(dk, b, r.ks[0]), seq_ptr(dv, b, r.vs[0]), wsb, st,
+                     b == 0 ? marks : nullptr);
       if (s != LG_OK) return s;
     }
     return LG_OK;
   }
   const WsLayout w = ws_layout(r, true);
-  if ((s = prepare_workspace(r, w, ws, true, st)) != LG_OK) return s;
+  if ((s = prepare_workspace(r, w, ws, 2, st)) != LG_OK) return s;
   return launch_bwd(r, w, q, k, v, o, lse, d_o, dq, dk, dv, ws, st, marks);
+}
+
+}  // namespace lg
+
+extern "C" {
+
+lg_status lg_sparse_attn_fwd(const lg_attn_params* p, const void* q, const void* k, const void* v, void* o,
+                             float* lse, void* workspace, size_t workspace_bytes, void* stream) {
+  return attn_fwd_entry(p, q, k, v, o, lse, workspace, workspace_bytes, stream, nullptr);
 }
 
 lg_status lg_sparse_attn_bwd(const lg_attn_params* p, const void* q, const void* k, const void* v, const void* o,
                              const float* lse, const void* d_o, void* dq, void* dk, void* dv, void* workspace,
                              size_t workspace_bytes, void* stream) {
-  return bwd_common(p, q, k, v, o, lse, d_o, dq, dk, dv, workspace, workspace_bytes, stream, nullptr);
+  return attn_bwd_entry(p, q, k, v, o, lse, d_o, dq, dk, dv, workspace, workspace_bytes, stream, nullptr, nullptr);
 }
 
-lg_status lg_sparse_attn_bwd_profiled(const lg_attn_params* p, const void* q, const void* k, const void* v,
-                                      const void* o, const float* lse, const void* d_o, void* dq, void* dk,
-                                      void* dv, void* workspace, size_t workspace_bytes, void* stream,
-                                      float* kernel_ms) {
-  if (!kernel_ms) return LG_ERR_INVALID_ARG;
-  cudaEvent_t ev[4] = {nullptr, nullptr, nullptr, nullptr};
-  lg_status s = LG_OK;
-  for (int i = 0; i < 4; ++i)
-    if (cudaEventCreate(&ev[i]) != cudaSuccess) s = LG_ERR_CUDA;
-  if (s == LG_OK) s = bwd_common(p, q, k, v, o, lse, d_o, dq, dk, dv, workspace, workspace_bytes, stream, ev);
-  if (s == LG_OK && cudaStreamSynchronize(static_cast<cudaStream_t>(stream)) != cudaSuccess) s = LG_ERR_CUDA;
-  if (s == LG_OK)
-    for (int i = 0; i < 3; ++i)
-      if (cudaEventElapsedTime(&kernel_ms[i], ev[i], ev[i + 1]) != cudaSuccess) s = LG_ERR_CUDA;
-  for (int i = 0; i < 4; ++i)
-    if (ev[i]) cudaEventDestroy(ev[i]);
-  return s;
+lg_status lg_sparse_attn_bwd_marked(const lg_attn_params* p, const void* q, const void* k, const void* v,
+                                    const void* o, const float* lse, const void* d_o, void* dq, void* dk, void* dv,
+                                    void* workspace, size_t workspace_bytes, void* stream, void* const* events) {
+  if (!events) return LG_ERR_INVALID_ARG;
+  cudaEvent_t ev[4];
+  for (int i = 0; i < 4; ++i) {
+    if (!events[i]) return LG_ERR_INVALID_ARG;
+    ev[i] = static_cast<cudaEvent_t>(events[i]);
+  }
+  return attn_bwd_entry(p, q, k, v, o, lse, d_o, dq, dk, dv, workspace, workspace_bytes, stream, ev, nullptr);
 }
 
 size_t lg_chunk_prefill_workspace_bytes(const lg_decode_params* p, int32_t T, int64_t n_tokens_before) {
@@ -490,9 +562,10 @@ lg_status lg_chunk_prefill(const lg_decode_params* p, const void* q_chunk, const
   ring_linearise_kernel<<<static_cast<unsigned>(blocks), 256, 0, st>>>(
       static_cast<const __nv_bfloat16*>(k_cache), static_cast<const __nv_bfloat16*>(v_cache),
       static_cast<const __nv_bfloat16*>(k_chunk), static_cast<const __nv_bfloat16*>(v_chunk), k_lin, v_lin, p->B,
-      p->Hkv, p->D, p->sink_tokens, p->window_tokens, c.kept, T, n_tokens_before);
+      p->Hkv, p->D, p->sink_tokens, p->window_tokens, c.kept, T, n_tokens_before); note_launch();
   if (cudaGetLastError() != cudaSuccess) return LG_ERR_CUDA;
-  if ((s = prepare_workspace(c.r, c.w, ws, false, st)) != LG_OK) return s;
+  if ((s = begin_workspace(ws, st)) != LG_OK) return s;
+  if ((s = prepare_workspace(c.r, c.w, ws, 1, st)) != LG_OK) return s;
   return launch_fwd(c.r, c.w, q_chunk, k_lin, v_lin, o, lse, ws, st);
 }
 
@@ -501,8 +574,8 @@ lg_status lg_selftest_wait_timeout(void* workspace, void* stream) {
   lg_status s = check_arch();
   if (s != LG_OK) return s;
   cudaStream_t st = static_cast<cudaStream_t>(stream);
-  if (cudaMemsetAsync(workspace, 0, sizeof(WsHeader), st) != cudaSuccess) return LG_ERR_CUDA;
-  wait_selftest_kernel<<<1, 32, 0, st>>>(static_cast<unsigned int*>(workspace), 2000000ll);
+  if (cudaMemsetAsync(workspace, 0, 2 * sizeof(unsigned int), st) != cudaSuccess) return LG_ERR_CUDA;   // the status words only
+  wait_selftest_kernel<<<1, 32, 0, st>>>(static_cast<unsigned int*>(workspace), 2000000ll); note_launch();
   return cudaGetLastError() == cudaSuccess ? LG_OK : LG_ERR_CUDA;
 }
 
@@ -510,14 +583,17 @@ lg_status lg_last_status(void* workspace, void* stream) {
   if (!workspace) return LG_ERR_INVALID_ARG;
   cudaStream_t st = static_cast<cudaStream_t>(stream);
   if (cudaStreamSynchronize(st) != cudaSuccess) return LG_ERR_CUDA;
-  unsigned int word = 0;
-  if (cudaMemcpy(&word, workspace, sizeof(word), cudaMemcpyDeviceToHost) != cudaSuccess) return LG_ERR_CUDA;
-  if (word != 0) {
+  unsigned int word[2] = {0, 0};   // error word of the latest call, and one an earlier call left unread
+  if (cudaMemcpy(word, workspace, sizeof(word), cudaMemcpyDeviceToHost) != cudaSuccess) return LG_ERR_CUDA;
+  if (word[0] != 0 || word[1] != 0) {
     if (cudaMemset(workspace, 0, sizeof(word)) != cudaSuccess) return LG_ERR_CUDA;
-    return LG_ERR_DEVICE_TIMEOUT;
+    const unsigned int first = word[1] != 0 ? word[1] : word[0];
+    return (first >> 24) == 3u ? LG_ERR_WORKSPACE : LG_ERR_DEVICE_TIMEOUT;
   }
   return LG_OK;
 }
+
+int64_t lg_debug_kernel_launches(void) { return g_kernel_launches.load(std::memory_order_relaxed); }
 
 const char* lg_status_string(lg_status s) {
   switch (s) {

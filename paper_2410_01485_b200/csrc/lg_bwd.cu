@@ -18,7 +18,7 @@ static lg_status launch_bwd_t(const Resolved& r, const WsLayout& w, const void* 
     dim3 grid((Lp + rows_per_block - 1) / rows_per_block, n_bh < 65535 ? n_bh : 65535);
     delta_kernel<D><<<grid, 256, 0, stream>>>(
         static_cast<const __nv_bfloat16*>(o), static_cast<const __nv_bfloat16*>(d_o), lse, stat, r.os[0], r.os[1],
-        r.os[2], r.Hq, n_bh, r.L, Lp, static_cast<int64_t>(n_bh) * Lp);
+        r.os[2], r.Hq, n_bh, r.L, Lp, static_cast<int64_t>(n_bh) * Lp); note_launch();
   }
   if (marks) cudaEventRecord(marks[1], stream);
   BwdArgs a;
@@ -26,6 +26,8 @@ static lg_status launch_bwd_t(const Resolved& r, const WsLayout& w, const void* 
   a.Lp = static_cast<int>(align_up(r.L, 128));
   a.stat_plane = static_cast<int64_t>(r.B) * r.Hq * a.Lp;
   a.error_word = r.error_word ? r.error_word : reinterpret_cast<unsigned int*>(ws);
+  a.expect_fp = r.expect_fp;
+  a.expect_fp2 = r.expect_fp2;
   a.L = r.L; a.Hq = r.Hq; a.Hkv = r.Hkv; a.G = r.G;
   a.exact_w = r.exact_w; a.ns = r.pat.ns;
   a.doc_start = r.doc_start;
@@ -53,7 +55,7 @@ static lg_status launch_bwd_t(const Resolved& r, const WsLayout& w, const void* 
     if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, smem) != cudaSuccess)
       return LG_ERR_CUDA;
     dim3 grid(r.B * r.Hkv, r.n_ktiles);
-    kern<<<grid, kKvThreads, smem, stream>>>(tq, tk, tv, tdo, a);
+    kern<<<grid, kKvThreads, smem, stream>>>(tq, tk, tv, tdo, a); note_launch();
     if (marks) cudaEventRecord(marks[2], stream);
   }
   // ---- dQ pass ------------------------------------------------------------------------
@@ -75,7 +77,7 @@ static lg_status launch_bwd_t(const Resolved& r, const WsLayout& w, const void* 
     if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, smem) != cudaSuccess)
       return LG_ERR_CUDA;
     dim3 grid(r.B * r.Hq, r.n_qtiles);
-    kern<<<grid, kDqThreads, smem, stream>>>(tq, tk, tv, tdo, a);
+    kern<<<grid, kDqThreads, smem, stream>>>(tq, tk, tv, tdo, a); note_launch();
     if (marks) cudaEventRecord(marks[3], stream);
   }
   return cudaGetLastError() == cudaSuccess ? LG_OK : LG_ERR_CUDA;

@@ -44,7 +44,8 @@ struct BwdArgs {
   int Lp;
   __nv_bfloat16* out0;       // dQ   | dK
   __nv_bfloat16* out1;       // unused | dV
-  unsigned int* error_word;
+  unsigned int* error_word;  // first word of the workspace header
+  unsigned long long expect_fp, expect_fp2;   // fingerprints of the lists this call was told the workspace holds (0: built by the call itself)
   int64_t s0[3], s1[3];      // strides of out0 / out1 (batch, head, token; elements)
   int L, Hq, Hkv, G;
   int exact_w, ns;           // token-exact window (0: off) and number of sink blocks
@@ -182,6 +183,7 @@ bwd_dq_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ 
     if (tid == 0) atomicCAS(a.error_word, 0u, (2u << 24) | 20u);
     return;
   }
+  if (!lists_match(a.error_word, a.expect_fp, a.expect_fp2, 20u)) return;
   uint8_t* sQ = smem + SM::oFix0;
   uint8_t* sDO = smem + SM::oFix1;
   uint8_t* sK = smem + SM::oA;
@@ -481,6 +483,7 @@ bwd_dkdv_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
     if (tid == 0) atomicCAS(a.error_word, 0u, (2u << 24) | 10u);
     return;
   }
+  if (!lists_match(a.error_word, a.expect_fp, a.expect_fp2, 10u)) return;
   uint8_t* sK = smem + SM::oFix0;
   uint8_t* sV = smem + SM::oFix1;
   uint8_t* sQ = smem + SM::oA;     // [3]

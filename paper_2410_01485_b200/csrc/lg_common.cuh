@@ -9,10 +9,26 @@ namespace lg {
 
 // ---- workspace header (first 256 bytes of every workspace) ---------------------------
 struct WsHeader {
-  unsigned int error_word;     // 0 = ok; else (code << 24) | site
-  unsigned int pad[63];
+  unsigned int error_word;         // 0 = ok; else (code << 24) | site.  code 1: a wait gave up, 2: shared memory
+                                   // misaligned, 3: the workspace does not hold the lists the call was told it holds
+  unsigned int latched;            // an error word that a later call found unread and kept for lg_last_status
+  unsigned long long magic;        // kWsMagic once the header has been initialised by a call
+  unsigned long long fingerprint;  // which pattern the lists and schedules below were built for (0: none)
+  unsigned int pad[58];
 };
+constexpr unsigned long long kWsMagic = 0x4c47575348445231ull;   // "LGWSHDR1"
 static_assert(sizeof(WsHeader) == 256, "header size");
+
+// A call that was told its workspace holds prepared lists checks, before it reads any of them,
+// that the header carries a fingerprint it accepts; otherwise the CTA records code 3 and returns.
+__device__ __forceinline__ bool lists_match(unsigned int* error_word, unsigned long long fp, unsigned long long fp2,
+                                            unsigned int site) {
+  if (fp == 0) return true;
+  const unsigned long long have = reinterpret_cast<const volatile WsHeader*>(error_word)->fingerprint;
+  if (have == fp || have == fp2) return true;
+  if (threadIdx.x == 0) atomicCAS(error_word, 0u, (3u << 24) | site);
+  return false;
+}
 
 constexpr long long kWaitLimitCycles = 4000000000ll;   // ~2 s of SM clock: a wait that long gave up
 

@@ -560,7 +560,7 @@ lg_status lg_kv_ring_append(const lg_decode_params* p, void* k_cache, void* v_ca
   ring_append_kernel<<<static_cast<unsigned>(blocks), 256, 0, static_cast<cudaStream_t>(stream)>>>(
       static_cast<__nv_bfloat16*>(k_cache), static_cast<__nv_bfloat16*>(v_cache),
       static_cast<const __nv_bfloat16*>(k_new), static_cast<const __nv_bfloat16*>(v_new), n_tokens_before, p->B,
-      p->Hkv, p->D, T_new, p->sink_tokens, p->window_tokens);
+      p->Hkv, p->D, T_new, p->sink_tokens, p->window_tokens); note_launch();
   return cudaGetLastError() == cudaSuccess ? LG_OK : LG_ERR_CUDA;
 }
 
@@ -640,12 +640,12 @@ lg_status lg_sparse_decode(const lg_decode_params* p, const void* q, const void*
       if (cudaFuncSetAttribute(decode_stream_kernel<128>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem_flat) !=
           cudaSuccess)
         return LG_ERR_CUDA;
-      decode_stream_kernel<128><<<static_cast<unsigned>(n_cta), kDecWarps * 32, smem_flat, st>>>(a);
+      decode_stream_kernel<128><<<static_cast<unsigned>(n_cta), kDecWarps * 32, smem_flat, st>>>(a); note_launch();
     } else {
       if (cudaFuncSetAttribute(decode_stream_kernel<64>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem_flat) !=
           cudaSuccess)
         return LG_ERR_CUDA;
-      decode_stream_kernel<64><<<static_cast<unsigned>(n_cta), kDecWarps * 32, smem_flat, st>>>(a);
+      decode_stream_kernel<64><<<static_cast<unsigned>(n_cta), kDecWarps * 32, smem_flat, st>>>(a); note_launch();
     }
     return cudaGetLastError() == cudaSuccess ? LG_OK : LG_ERR_CUDA;
   }
@@ -657,14 +657,14 @@ lg_status lg_sparse_decode(const lg_decode_params* p, const void* q, const void*
     if (cudaFuncSetAttribute(decode_split_kernel<128>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem) !=
         cudaSuccess)
       return LG_ERR_CUDA;
-    decode_split_kernel<128><<<grid, kDecWarps * 32, smem, st>>>(a);
-    decode_merge_kernel<128><<<p->B * a.Hkv * a.HG, 128, 0, st>>>(a);
+    decode_split_kernel<128><<<grid, kDecWarps * 32, smem, st>>>(a); note_launch();
+    decode_merge_kernel<128><<<p->B * a.Hkv * a.HG, 128, 0, st>>>(a); note_launch();
   } else {
     if (cudaFuncSetAttribute(decode_split_kernel<64>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem) !=
         cudaSuccess)
       return LG_ERR_CUDA;
-    decode_split_kernel<64><<<grid, kDecWarps * 32, smem, st>>>(a);
-    decode_merge_kernel<64><<<p->B * a.Hkv * a.HG, 128, 0, st>>>(a);
+    decode_split_kernel<64><<<grid, kDecWarps * 32, smem, st>>>(a); note_launch();
+    decode_merge_kernel<64><<<p->B * a.Hkv * a.HG, 128, 0, st>>>(a); note_launch();
   }
   return cudaGetLastError() == cudaSuccess ? LG_OK : LG_ERR_CUDA;
 }

@@ -20,6 +20,8 @@ static lg_status launch_fwd_t(const Resolved& r, const WsLayout& w, const void* 
   a.o = static_cast<__nv_bfloat16*>(o);
   a.lse = lse;
   a.error_word = r.error_word ? r.error_word : reinterpret_cast<unsigned int*>(ws);
+  a.expect_fp = r.expect_fp;
+  a.expect_fp2 = r.expect_fp2;
   for (int i = 0; i < 3; ++i) a.o_strides[i] = r.os[i];
   a.L = r.L; a.Hq = r.Hq; a.G = r.G;
   a.q_start = r.q_start; a.Lq = r.Lq;
@@ -30,7 +32,7 @@ static lg_status launch_fwd_t(const Resolved& r, const WsLayout& w, const void* 
   constexpr int smem = FwdSmem<D>::kTotal;
   if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, smem) != cudaSuccess) return LG_ERR_CUDA;
   dim3 grid(r.B * r.Hq, r.n_stiles);
-  kern<<<grid, kFwdThreads, smem, stream>>>(tq, tk, tv, a);
+  kern<<<grid, kFwdThreads, smem, stream>>>(tq, tk, tv, a); note_launch();
   return cudaGetLastError() == cudaSuccess ? LG_OK : LG_ERR_CUDA;
 }
 

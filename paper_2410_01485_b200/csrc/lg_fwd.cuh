@@ -31,7 +31,8 @@ struct FwdArgs {
   const int32_t* order;      // [n_super_tiles] launch rank -> super-tile
   __nv_bfloat16* o;
   float* lse;                // [B, Hq, L]
-  unsigned int* error_word;
+  unsigned int* error_word;  // first word of the workspace header
+  unsigned long long expect_fp, expect_fp2;   // fingerprints of the lists this call was told the workspace holds (0: built by the call itself)
   int64_t o_strides[3];      // batch, head, token (elements)
   int L, Hq, G;              // G = Hq / Hkv
   int q_start, Lq;           // queries exist for rows [q_start, q_start + Lq) of the L key positions only
@@ -81,6 +82,7 @@ fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUt
     if (tid == 0) atomicCAS(a.error_word, 0u, (2u << 24) | 1u);
     return;
   }
+  if (!lists_match(a.error_word, a.expect_fp, a.expect_fp2, 1u)) return;
   uint8_t* sQ = smem + SM::oQ;
   uint8_t* sK = smem + SM::oK;
   uint8_t* sV = smem + SM::oV;

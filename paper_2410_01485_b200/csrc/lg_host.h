@@ -13,6 +13,10 @@ namespace lg {
 
 inline size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
 
+// Diagnostic only: how many kernels the library has launched in this process (read through
+// lg_debug_kernel_launches); nothing in the library depends on it.
+void note_launch();
+
 struct Resolved {          // validated, defaulted copy of lg_attn_params
   int B, Hq, Hkv, L, D, block, mode, G;
   PatternDev pat;
@@ -24,6 +28,8 @@ struct Resolved {          // validated, defaulted copy of lg_attn_params
   int q_start, Lq;         // forward only: queries exist for rows [q_start, q_start + Lq) (0, L by default)
   const int32_t* doc_start;  // device [B, L] or null: first position of each token's document
   unsigned int* error_word;  // status word of the call when it is not the start of `ws` (null: it is)
+  int lists_prepared;        // the caller says the workspace already holds this pattern's lists
+  unsigned long long expect_fp, expect_fp2;   // fingerprints the kernels accept in the header (0: no check)
   int64_t nnz;
 };
 
@@ -46,7 +52,8 @@ WsLayout ws_layout(const Resolved& r, bool want_bwd);
 lg_status launch_index_build(const Resolved& r, int32_t* row_ptr, int32_t* col_idx, int32_t* col_ptr,
                              int32_t* row_idx, cudaStream_t stream);
 // Build lists + tile schedules inside a workspace.
-lg_status prepare_workspace(const Resolved& r, const WsLayout& w, uint8_t* ws, bool want_bwd, cudaStream_t stream);
+// `what`: bit 0 = the forward's schedule, bit 1 = the backward's schedules.
+lg_status prepare_workspace(const Resolved& r, const WsLayout& w, uint8_t* ws, int what, cudaStream_t stream);
 
 // bf16 [B, H, L, D] tensor (element strides bs, hs, ls; D contiguous) as a 4-D tensor map with
 // boxes of 64 columns x `box_rows` rows and the 128-byte swizzle.
@@ -61,5 +68,13 @@ lg_status launch_fwd(const Resolved& r, const WsLayout& w, const void* q, const 
 lg_status launch_bwd(const Resolved& r, const WsLayout& w, const void* q, const void* k, const void* v,
                      const void* o, const float* lse, const void* d_o, void* dq, void* dk, void* dv, uint8_t* ws,
                      cudaStream_t stream, cudaEvent_t* marks /* null, or 4 events recorded around the 3 kernels */);
+
+// The forward / backward entry points with the status word of the call redirected (null: the start
+// of `workspace`): a step that runs several calls on slices of one workspace reports through one word.
+lg_status attn_fwd_entry(const lg_attn_params* p, const void* q, const void* k, const void* v, void* o, float* lse,
+                         void* workspace, size_t workspace_bytes, void* stream, unsigned int* status_word);
+lg_status attn_bwd_entry(const lg_attn_params* p, const void* q, const void* k, const void* v, const void* o,
+                         const float* lse, const void* d_o, void* dq, void* dk, void* dv, void* workspace,
+                         size_t workspace_bytes, void* stream, cudaEvent_t* marks, unsigned int* status_word);
 
 }  // namespace lg

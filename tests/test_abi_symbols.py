@@ -67,6 +67,58 @@ def test_invalid_params_rejected(lib, mutate):
     assert lib.lg_sparse_attn_fwd(C.byref(p), 256, 256, 256, 256, 256, 256, 1 << 30, None) == -1
 
 
+def test_header_compiles_as_c(tmp_path):
+    """include/lg.h is a C header: a C translation unit that includes it and takes the address of an entry
+    point compiles with the C compiler (no C++ construct has slipped in)."""
+    import shutil
+    import subprocess
+    cc = shutil.which("gcc") or shutil.which("cc")
+    if cc is None:
+        pytest.skip("no C compiler")
+    src = tmp_path / "use_lg.c"
+    src.write_text('#include "lg.h"\n'
+                   'lg_status (*fwd)(const lg_attn_params*, const void*, const void*, const void*, void*, float*,\n'
+                   '                 void*, size_t, void*) = lg_sparse_attn_fwd;\n'
+                   'int main(void) { lg_attn_params p; lg_decode_params d; lg_device_step_buffers b;\n'
+                   '  (void)p; (void)d; (void)b; return sizeof(p) == 0; }\n')
+    inc = os.path.join(os.path.dirname(build.HERE), "include")
+    res = subprocess.run([cc, "-std=c99", "-Wall", "-Werror", "-pedantic", "-I", inc, "-c", str(src), "-o",
+                          str(tmp_path / "use_lg.o")], capture_output=True, text=True)
+    assert res.returncode == 0, res.stderr
+
+
+def test_prepare_and_host_step_validation(lib):
+    """The entry points added around the plain forward / backward reject bad arguments on the host."""
+    p = _good()
+    need = lib.lg_sparse_attn_workspace_bytes(C.byref(p), 1)
+    assert lib.lg_sparse_attn_prepare(C.byref(p), None, need, 1, None) == -1
+    assert lib.lg_sparse_attn_prepare(C.byref(p), 128, need, 1, None) == -1          # workspace alignment
+    assert lib.lg_sparse_attn_prepare(C.byref(p), 256, need - 1, 1, None) == -3
+    p.lists_prepared = 2
+    assert lib.lg_sparse_attn_workspace_bytes(C.byref(p), 1) == 0                      # only 0 or 1
+    p.lists_prepared = 0
+    p.doc_start, p.B = 256, 2                                                          # lists per sequence: no prepare
+    assert lib.lg_sparse_attn_prepare(C.byref(p), 256, 1 << 30, 1, None) == -2
+    # host step: group count must divide Hkv; sizes grow with the number of groups
+    p = _good()
+    sz = lib.lg_sparse_attn_fwd_bwd_host_workspace_bytes
+    assert sz(C.byref(p), 0) == 0 and sz(C.byref(p), 3) == 0
+    assert 0 < sz(C.byref(p), 1) and sz(C.byref(p), 2) > 0
+    bufs = binding.DeviceStepBuffers(*([256] * 10), sz(C.byref(p), 2) - 1)
+    args = [C.byref(p)] + [256] * 9 + [C.byref(bufs), 2, None, None, None]
+    assert lib.lg_sparse_attn_fwd_bwd_host(*args) == -3                               # workspace too small
+    bufs.workspace_bytes = sz(C.byref(p), 2)
+    bufs.dq = None
+    assert lib.lg_sparse_attn_fwd_bwd_host(*args) == -1                               # a staging buffer is missing
+    args[3] = None
+    assert lib.lg_sparse_attn_fwd_bwd_host(*args) == -1                               # a host tensor is missing
+    # marked backward: the four events are mandatory
+    ev = (C.c_void_p * 4)(1, 2, 3, None)
+    assert lib.lg_sparse_attn_bwd_marked(C.byref(p), *([256] * 9), 256, need, None, None) == -1
+    assert lib.lg_sparse_attn_bwd_marked(C.byref(p), *([256] * 9), 256, need, None, ev) == -1
+    assert lib.lg_debug_kernel_launches() >= 0
+
+
 def test_unsupported_head_dim(lib):
     p = _good()
     p.D = 96

@@ -38,6 +38,10 @@ def test_gpu_arm_line_on_the_small_case():
     assert d["n_gpus"] == 1 and d["steps"] == 2 and d["dtype"] == "bf16" and d["data"] == "synthetic"
     r = d["roofline"]
     assert r["bound"] == "tensor" and r["unit"] == "TFLOP/s" and 0 < r["frac"] < 1.5
-    assert abs(r["frac"] - r["achieved"] / r["peak"]) < 1e-9 and r["traffic"] > 0
-    assert set(r["kernel_ms"]) == {"fwd", "bwd_dkdv", "bwd_dq", "bwd_delta"}
-    assert d["gpu_launches"] == 2 * 19 and d["value"] > 0 and "workload" in d["config"]
+    assert abs(r["frac"] - r["achieved"] / r["peak"]) < 1e-9
+    assert r["traffic"] is None or r["traffic"] > 0            # null once the kernels differ from the captured ones
+    assert set(d["kernel_ms"]) == {"fwd", "bwd_dkdv", "bwd_dq", "bwd_delta", "index_build_once"}
+    assert all(v > 0 for v in d["kernel_ms"].values()) and d["kernel_ms"] == r["kernel_ms"]
+    # the lists are built once before the timed region: a step launches the forward kernel and the
+    # backward's three (delta, dK/dV, dQ), counted by the library itself
+    assert d["gpu_launches"] == 2 * 4 and d["value"] > 0 and "workload" in d["config"]
