@@ -10,7 +10,9 @@
  * Conventions for every entry point
  *   - Pointers named in a signature as device pointers are device memory OWNED BY THE
  *     CALLER; the library allocates nothing that outlives a call and keeps no state
- *     between calls except what it writes into the caller's workspace.
+ *     between calls except what it writes into the caller's workspace.  Two exceptions, both
+ *     documented where they are declared: the fixed scratch array of lg_sparse_decode_static
+ *     (shared by all its calls on a device) and a diagnostic launch counter.
  *   - `stream` is a cudaStream_t (0 = default stream).  Calls enqueue work and return;
  *     the return value covers validation and launch only.  A device-side wait that gave
  *     up (every wait in the kernels is bounded) is reported by lg_last_status().
@@ -212,13 +214,23 @@ typedef struct {
   int32_t B, Hq, Hkv, D;       /* D in {64, 128}; Hq % Hkv == 0                              */
   int32_t sink_tokens;         /* >= 0                                                       */
   int32_t window_tokens;       /* >= 1                                                       */
+  int32_t block_tokens;        /* 0: the query attends every token the cache holds (the token-exact
+                                  window of Section 3.2's rolling buffer, the same keys as
+                                  window_exact = 1 in training).  Bs > 0: the block-granular window
+                                  of Section 4.1 that the default training mask uses -- the query at
+                                  position n - 1 attends the sink and the tokens j with
+                                  (n-1)/Bs - j/Bs < window_tokens/Bs; sink_tokens and window_tokens
+                                  must be multiples of Bs.  The cache layout is the same either way
+                                  (the ring still holds window_tokens tokens; up to Bs - 1 of the
+                                  oldest are then read but not attended).  lg_kv_ring_append
+                                  ignores this field.                                         */
   float   scale;               /* 0 selects 1/sqrt(D)                                        */
 } lg_decode_params;
 
 /* Append T_new tokens per sequence: k_new, v_new [B, Hkv, T_new, D] bf16 (device);
  * n_tokens_before (device int64 [B]) = tokens already appended to each sequence.  The
  * result equals appending one token at a time; writes that a later token of the same
- * call would overwrite are skipped.                                                      */
+ * call would overwrite are skipped.  A sequence whose count is negative is left untouched. */
 lg_status lg_kv_ring_append(const lg_decode_params* p, void* k_cache, void* v_cache,
                             const void* k_new, const void* v_new, int32_t T_new,
                             const int64_t* n_tokens_before, void* stream);
@@ -301,11 +313,18 @@ lg_status lg_chunk_prefill(const lg_decode_params* p, const void* q_chunk, const
  *     give undefined results.
  *   - The decode kernels contain no device-side waits, so there is no device status to read
  *     back for this call (lg_last_status needs a workspace pointer and does not apply).
+ *   - If a launch on the array ends abnormally (a CUDA error reported for the stream, the
+ *     process interrupted in mid-kernel and the context kept), arrival counters in the array may
+ *     be left non-zero, and later calls would then merge too early or never.  The workspace
+ *     variant is repaired by lg_sparse_decode_workspace_init; this array by
+ *     lg_sparse_decode_static_reset(stream), which clears it with one memset on `stream`
+ *     (no allocation either) and may be called at any time no static call is in flight.
  * Results are bit-identical to lg_sparse_decode on the same inputs.
  */
 lg_status lg_sparse_decode_static(const lg_decode_params* p, const void* q, const void* k_cache,
                                   const void* v_cache, const int64_t* n_tokens, void* o, float* lse,
                                   void* stream);
+lg_status lg_sparse_decode_static_reset(void* stream);
 
 /* ---- self-test of the error path -------------------------------------------------------- */
 

@@ -261,9 +261,11 @@ def attn_keys_grad(q, k, v, do, p: Pattern, scale: float, j0: int, j1: int):
     dV = np.zeros((Hkv, j1 - j0, D))
     for r0 in range(0, L, p.block):
         r1 = min(L, r0 + p.block)          # the last block may be partial
-        M = token_mask(p, r0, r1)
-        if not M[:, j0:j1].any():
+        # does any row of this slab see one of the wanted keys?  (the explicit mask, on those columns only,
+        # before the slab's whole mask is materialised)
+        if not allowed(p, np.arange(r0, r1)[:, None], np.arange(j0, j1)[None, :]).any():
             continue
+        M = token_mask(p, r0, r1)
         cols = np.nonzero(M.any(axis=0))[0]
         Mc = M[:, cols]
         sel = (cols >= j0) & (cols < j1)        # which of the slab's keys are the wanted ones
@@ -283,16 +285,25 @@ def attn_keys_grad(q, k, v, do, p: Pattern, scale: float, j0: int, j1: int):
 
 # -------------------------------------------------------------------------- decode
 
-def decode_valid(n: int, sink: int, window: int) -> np.ndarray:
-    """Which of the first n tokens a sink + rolling-window cache still holds after n
-    appends (Section 3.2: rolling buffer for the window, sink kept beside it):
-    token j survives iff j < sink or it is among the last `window` tokens."""
+def decode_valid(n: int, sink: int, window: int, block_tokens: int = 0) -> np.ndarray:
+    """Which of the first n tokens the query token n - 1 attends to in serving.
+
+    block_tokens == 0: every token a sink + rolling-window cache still holds after n appends
+    (Section 3.2: rolling buffer for the window, sink kept beside it): token j survives iff
+    j < sink or it is among the last `window` tokens.
+    block_tokens == Bs > 0: the block-granular window the sparse layers are trained with
+    (Section 4.1 counts the local context in blocks, the query's own block included): token j
+    is attended iff j < sink or floor((n-1)/Bs) - floor(j/Bs) < window/Bs.  These are tokens
+    the cache holds (a subset: up to Bs - 1 of the oldest window tokens are left out)."""
     j = np.arange(n)
+    if block_tokens:
+        return (j < sink) | ((n - 1) // block_tokens - j // block_tokens < window // block_tokens)
     return (j < sink) | (n - 1 - j < window)
 
 
-def decode(qv, k_lin, v_lin, n: int, sink: int, window: int, scale: float):
-    """One query token per head attends to the surviving tokens of a linear history.
+def decode(qv, k_lin, v_lin, n: int, sink: int, window: int, scale: float, block_tokens: int = 0):
+    """One query token per head attends to the surviving tokens of a linear history
+    (block_tokens: see decode_valid).
 
     qv [Hq, D]; k_lin, v_lin [Hkv, >=n, D] hold token j at index j (the oracle never
     sees the ring layout).  Returns o [Hq, D], lse [Hq]; n == 0 gives o = 0, lse = -inf."""
@@ -302,7 +313,7 @@ def decode(qv, k_lin, v_lin, n: int, sink: int, window: int, scale: float):
     lse = np.full(Hq, -np.inf)
     if n == 0:
         return o, lse
-    keep = np.nonzero(decode_valid(n, sink, window))[0]
+    keep = np.nonzero(decode_valid(n, sink, window, block_tokens))[0]
     for h in range(Hq):
         s = scale * (k_lin[h // G, keep] @ qv[h])
         mx = s.max()
@@ -313,7 +324,7 @@ def decode(qv, k_lin, v_lin, n: int, sink: int, window: int, scale: float):
     return o, lse
 
 
-def chunk_prefill(q_chunk, k_lin, v_lin, n_before: int, sink: int, window: int, scale: float):
+def chunk_prefill(q_chunk, k_lin, v_lin, n_before: int, sink: int, window: int, scale: float, block_tokens: int = 0):
     """A chunk of T new tokens served against a sink + rolling-window cache (Section 3.2: in
     serving the sparse layers keep only the sink and the last `window` tokens).  By definition
     the result is what T successive decode steps give: token n_before + t is appended and then
@@ -325,7 +336,7 @@ def chunk_prefill(q_chunk, k_lin, v_lin, n_before: int, sink: int, window: int, 
     o = np.zeros((Hq, T, D))
     lse = np.full((Hq, T), -np.inf)
     for t in range(T):
-        o[:, t], lse[:, t] = decode(q_chunk[:, t], k_lin, v_lin, n_before + t + 1, sink, window, scale)
+        o[:, t], lse[:, t] = decode(q_chunk[:, t], k_lin, v_lin, n_before + t + 1, sink, window, scale, block_tokens)
     return o, lse
 
 

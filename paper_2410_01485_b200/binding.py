@@ -42,7 +42,8 @@ class DeviceStepBuffers(C.Structure):
 
 class DecodeParams(C.Structure):
     _fields_ = [("B", C.c_int32), ("Hq", C.c_int32), ("Hkv", C.c_int32), ("D", C.c_int32),
-                ("sink_tokens", C.c_int32), ("window_tokens", C.c_int32), ("scale", C.c_float)]
+                ("sink_tokens", C.c_int32), ("window_tokens", C.c_int32), ("block_tokens", C.c_int32),
+                ("scale", C.c_float)]
 
 
 _lib = None
@@ -68,6 +69,7 @@ SYMBOLS = {
     "lg_chunk_prefill": (C.c_int, [C.POINTER(DecodeParams), _vp, _vp, _vp, _vp, _vp, C.c_int32, C.c_int64, _vp, _vp,
                                    _vp, _sz, _vp]),
     "lg_sparse_decode_static": (C.c_int, [C.POINTER(DecodeParams), _vp, _vp, _vp, _vp, _vp, _vp, _vp]),
+    "lg_sparse_decode_static_reset": (C.c_int, [_vp]),
     "lg_selftest_wait_timeout": (C.c_int, [_vp, _vp]),
     "lg_last_status": (C.c_int, [_vp, _vp]),
     "lg_status_string": (C.c_char_p, [C.c_int]),
@@ -283,9 +285,11 @@ def _side_stream(i: int) -> "torch.cuda.Stream":
 
 # ---------------------------------------------------------------------- decode / ring
 
-def decode_params(B, Hq, Hkv, D, sink_tokens, window_tokens, scale=0.0) -> DecodeParams:
+def decode_params(B, Hq, Hkv, D, sink_tokens, window_tokens, scale=0.0, block_tokens=0) -> DecodeParams:
+    """block_tokens: 0 = attend every token the cache holds; Bs = the block-granular window of training."""
     p = DecodeParams()
     p.B, p.Hq, p.Hkv, p.D, p.sink_tokens, p.window_tokens, p.scale = B, Hq, Hkv, D, sink_tokens, window_tokens, scale
+    p.block_tokens = block_tokens
     return p
 
 

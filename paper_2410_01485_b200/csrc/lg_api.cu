@@ -53,6 +53,7 @@ lg_status resolve(const lg_attn_params* p, Resolved* r) {
   r->pat.doc_start = nullptr;
   r->pat.block = p->block;
   r->exact_w = 0;
+  r->win_block = r->win_phase = 0;
   switch (p->mode) {
     case LG_MODE_FULL_CAUSAL:
       break;
@@ -302,6 +303,9 @@ static lg_status plan_chunk(const lg_decode_params* p, int32_t T, int64_t n_befo
   // the pattern is made of 64-token blocks: sink and window must be multiples of 64; the chunk and
   // the fill level of the ring may be anything
   if (p->sink_tokens % 64 || p->window_tokens % 64) return LG_ERR_UNSUPPORTED;
+  if (p->block_tokens < 0) return LG_ERR_INVALID_ARG;
+  if (p->block_tokens > 0 && (p->window_tokens % p->block_tokens || p->sink_tokens % p->block_tokens))
+    return LG_ERR_INVALID_ARG;
   const int64_t cap = static_cast<int64_t>(p->sink_tokens) + p->window_tokens;
   const int64_t kept = n_before < cap ? n_before : cap;
   if (kept + T > (1 << 24)) return LG_ERR_UNSUPPORTED;
@@ -324,6 +328,12 @@ static lg_status plan_chunk(const lg_decode_params* p, int32_t T, int64_t n_befo
   if (s != LG_OK) return s;
   c->r.q_start = c->kept;
   c->r.Lq = T;
+  // Block-aligned window: every non-sink row v of the virtual sequence (kept tokens, then the chunk) is the
+  // token at position v + (n_before - kept), so the block-granular edge of the real positions is a
+  // block-aligned edge in coordinates shifted by that amount.  The lists stay those of the token-exact
+  // window, which contains it.
+  c->r.win_block = p->block_tokens;
+  c->r.win_phase = p->block_tokens > 0 ? static_cast<int>((n_before - kept) % p->block_tokens) : 0;
   c->w = ws_layout(c->r, false);
   c->lin_bytes = align_up(static_cast<size_t>(p->B) * p->Hkv * ap.L * p->D * sizeof(__nv_bfloat16), 256);
   c->o_k = align_up(c->w.total, 256);
@@ -390,6 +400,7 @@ size_t lg_block_index_bytes(const lg_attn_params* p) {
 
 lg_status lg_build_block_index(const lg_attn_params* p, int32_t* row_ptr, int32_t* col_idx, int32_t* col_ptr,
                                int32_t* row_idx, int64_t* nnz_out_host, void* stream) {
+  LG_RANGE("lg_build_block_index");
   Resolved r;
   lg_status s = resolve(p, &r);
   if (s != LG_OK) return s;
@@ -409,6 +420,7 @@ size_t lg_sparse_attn_workspace_bytes(const lg_attn_params* p, int want_bwd) {
 
 lg_status lg_sparse_attn_prepare(const lg_attn_params* p, void* workspace, size_t workspace_bytes, int want_bwd,
                                  void* stream) {
+  LG_RANGE("lg_sparse_attn_prepare");
   Resolved r;
   lg_status s = resolve(p, &r);
   if (s != LG_OK) return s;
@@ -513,18 +525,21 @@ extern "C" {
 
 lg_status lg_sparse_attn_fwd(const lg_attn_params* p, const void* q, const void* k, const void* v, void* o,
                              float* lse, void* workspace, size_t workspace_bytes, void* stream) {
+  LG_RANGE("lg_sparse_attn_fwd");
   return attn_fwd_entry(p, q, k, v, o, lse, workspace, workspace_bytes, stream, nullptr);
 }
 
 lg_status lg_sparse_attn_bwd(const lg_attn_params* p, const void* q, const void* k, const void* v, const void* o,
                              const float* lse, const void* d_o, void* dq, void* dk, void* dv, void* workspace,
                              size_t workspace_bytes, void* stream) {
+  LG_RANGE("lg_sparse_attn_bwd");
   return attn_bwd_entry(p, q, k, v, o, lse, d_o, dq, dk, dv, workspace, workspace_bytes, stream, nullptr, nullptr);
 }
 
 lg_status lg_sparse_attn_bwd_marked(const lg_attn_params* p, const void* q, const void* k, const void* v,
                                     const void* o, const float* lse, const void* d_o, void* dq, void* dk, void* dv,
                                     void* workspace, size_t workspace_bytes, void* stream, void* const* events) {
+  LG_RANGE("lg_sparse_attn_bwd_marked");
   if (!events) return LG_ERR_INVALID_ARG;
   cudaEvent_t ev[4];
   for (int i = 0; i < 4; ++i) {
@@ -542,6 +557,7 @@ size_t lg_chunk_prefill_workspace_bytes(const lg_decode_params* p, int32_t T, in
 lg_status lg_chunk_prefill(const lg_decode_params* p, const void* q_chunk, const void* k_chunk, const void* v_chunk,
                            const void* k_cache, const void* v_cache, int32_t T, int64_t n_tokens_before, void* o,
                            float* lse, void* workspace, size_t workspace_bytes, void* stream) {
+  LG_RANGE("lg_chunk_prefill");
   ChunkPlan c;
   lg_status s = plan_chunk(p, T, n_tokens_before, &c);
   if (s != LG_OK) return s;
@@ -570,6 +586,7 @@ lg_status lg_chunk_prefill(const lg_decode_params* p, const void* q_chunk, const
 }
 
 lg_status lg_selftest_wait_timeout(void* workspace, void* stream) {
+  LG_RANGE("lg_selftest_wait_timeout");
   if (!workspace || (reinterpret_cast<uintptr_t>(workspace) & 255)) return LG_ERR_INVALID_ARG;
   lg_status s = check_arch();
   if (s != LG_OK) return s;
@@ -580,6 +597,7 @@ lg_status lg_selftest_wait_timeout(void* workspace, void* stream) {
 }
 
 lg_status lg_last_status(void* workspace, void* stream) {
+  LG_RANGE("lg_last_status");
   if (!workspace) return LG_ERR_INVALID_ARG;
   cudaStream_t st = static_cast<cudaStream_t>(stream);
   if (cudaStreamSynchronize(st) != cudaSuccess) return LG_ERR_CUDA;

@@ -125,19 +125,7 @@ __device__ __forceinline__ void bulk_load(void* smem_dst, const void* gsrc, uint
                "l"(gsrc), "r"(bytes), "r"(smem_u32(bar))
                : "memory");
 }
-__device__ __forceinline__ void tma_store_4d(const void* tmap, const void* smem_src, int c0, int c1, int c2,
-                                             int c3) {
-  asm volatile("cp.async.bulk.tensor.4d.global.shared::cta.bulk_group [%0, {%2, %3, %4, %5}], [%1];" ::"l"(
-                   reinterpret_cast<uint64_t>(tmap)),
-               "r"(smem_u32(smem_src)), "r"(c0), "r"(c1), "r"(c2), "r"(c3)
-               : "memory");
-}
-__device__ __forceinline__ void tma_store_commit() { asm volatile("cp.async.bulk.commit_group;" ::: "memory"); }
-__device__ __forceinline__ void tma_store_wait_all() { asm volatile("cp.async.bulk.wait_group 0;" ::: "memory"); }
-__device__ __forceinline__ void tma_store_wait_read() {
-  asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory");
-}
-// generic-proxy smem writes -> visible to the async proxy (TMA store, tcgen05.mma operands)
+// generic-proxy smem writes -> visible to the async proxy (tcgen05.mma operands read from shared memory)
 __device__ __forceinline__ void fence_proxy_async_smem() {
   asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
 }
@@ -158,18 +146,6 @@ __device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence:
 __device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
 
 // ---- tcgen05: descriptors -------------------------------------------------------------
-// Shared-memory matrix descriptor, 128-byte swizzle, rows of 128 bytes packed in groups of
-// 8 (1024-byte atoms).  `lbo_bytes` is the distance between 64-element column groups for an
-// MN-major operand (ignored for K-major); `sbo_bytes` the distance between 8-row groups.
-__device__ __forceinline__ uint64_t make_smem_desc(uint32_t smem_addr, uint32_t lbo_bytes, uint32_t sbo_bytes) {
-  uint64_t d = 0;
-  d |= static_cast<uint64_t>((smem_addr & 0x3FFFF) >> 4);
-  d |= static_cast<uint64_t>((lbo_bytes >> 4) & 0x3FFF) << 16;
-  d |= static_cast<uint64_t>((sbo_bytes >> 4) & 0x3FFF) << 32;
-  d |= 1ull << 46;   // descriptor version for this architecture
-  d |= 2ull << 61;   // 128-byte swizzle
-  return d;
-}
 // Instruction descriptor for kind::f16 with bf16 operands and fp32 accumulation.
 // a_mn / b_mn: operand is MN-major (1) or K-major (0).
 __host__ __device__ constexpr uint32_t make_idesc_bf16(int M, int N, int a_mn, int b_mn) {
@@ -178,30 +154,13 @@ __host__ __device__ constexpr uint32_t make_idesc_bf16(int M, int N, int a_mn, i
          (static_cast<uint32_t>(M >> 4) << 24);
 }
 
-// D[tmem] (+)= A[smem] * B[smem]
-__device__ __forceinline__ void mma_ss(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t idesc,
-                                       uint32_t accumulate) {
-  asm volatile(
-      "{\n\t.reg .pred p;\n\t"
-      "setp.ne.b32 p, %4, 0;\n\t"
-      "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}" ::"r"(d_tmem),
-      "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate)
-      : "memory");
-}
-// D[tmem] (+)= A[tmem] * B[smem]
-__device__ __forceinline__ void mma_ts(uint32_t d_tmem, uint32_t a_tmem, uint64_t b_desc, uint32_t idesc,
-                                       uint32_t accumulate) {
-  asm volatile(
-      "{\n\t.reg .pred p;\n\t"
-      "setp.ne.b32 p, %4, 0;\n\t"
-      "tcgen05.mma.cta_group::1.kind::f16 [%0], [%1], %2, %3, p;\n\t}" ::"r"(d_tmem),
-      "r"(a_tmem), "l"(b_desc), "r"(idesc), "r"(accumulate)
-      : "memory");
-}
-// The same two instructions with the descriptors given as (low word, high word).  The high word
-// of a descriptor (stride fields, version, swizzle) is constant for an operand kind and the low
-// word is (address >> 4) | (leading-dimension field << 16), so stepping through the K slices of a
-// tile costs the issuing thread one 32-bit add per operand.
+// Shared-memory matrix descriptors (128-byte swizzle, rows of 128 bytes packed in groups of 8 =
+// 1024-byte atoms), given as (low word, high word).  The high word (stride between 8-row groups,
+// descriptor version, swizzle mode) is constant for an operand kind and the low word is
+// (address >> 4) | (leading-dimension field << 16) -- the leading dimension being the distance
+// between 64-element column groups of an MN-major operand (ignored for K-major) -- so stepping
+// through the K slices of a tile costs the issuing thread one 32-bit add per operand.
+// mma_ss2: D[tmem] (+)= A[smem] * B[smem];  mma_ts2: D[tmem] (+)= A[tmem] * B[smem].
 __device__ __forceinline__ uint32_t desc_hi(uint32_t sbo_bytes) {
   return ((sbo_bytes >> 4) & 0x3FFF) | (1u << 14) | (2u << 29);
 }
@@ -319,13 +278,6 @@ __device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
   uint32_t r;
   asm("cvt.rn.bf16x2.f32 %0, %1, %2;" : "=r"(r) : "f"(hi), "f"(lo));
   return r;
-}
-
-// Byte offset of element (row, col) inside a [rows x 64] bf16 tile stored with 128-byte
-// rows and the 128-byte swizzle TMA applies (16-byte chunk index XOR row % 8).
-__device__ __forceinline__ uint32_t swz128_offset(uint32_t row, uint32_t col) {
-  uint32_t chunk = (col >> 3) ^ (row & 7);
-  return row * 128 + chunk * 16 + (col & 7) * 2;
 }
 
 }  // namespace lg

@@ -42,6 +42,7 @@ struct DecodeArgs {
   float* lse;                    // [B, Hq] or null
   int Hq, Hkv, G, HG, C, nsplit;
   float scale_log2;
+  int sink, block_tokens;        // sink slots; block of the block-aligned window (0: every held token is attended)
   int B;                         // sequences (flattened path)
   unsigned int* unit_count;      // [B * Hkv * HG] records delivered per unit (flattened path; zero between calls)
 };
@@ -97,6 +98,31 @@ __device__ __forceinline__ void decode_run_segment(const DecodeArgs& a, uint8_t*
                          (static_cast<int64_t>(b) * a.Hkv + kvh) * static_cast<int64_t>(a.C) * kRowBytes;
   const uint8_t* vbase = reinterpret_cast<const uint8_t*>(a.v_cache) +
                          (static_cast<int64_t>(b) * a.Hkv + kvh) * static_cast<int64_t>(a.C) * kRowBytes;
+
+  // Block-aligned window (block_tokens = Bs > 0): the query at position n - 1 attends, besides the sink,
+  // the tokens j with floor((n-1)/Bs) - floor(j/Bs) < W/Bs.  The ring holds the last W tokens, up to
+  // Bs - 1 more: those oldest ones occupy ex_cnt consecutive (cyclic) ring slots from ring offset ex0
+  // and are masked out of the scores (they are still streamed with their tiles).
+  int ex0 = 0, ex_cnt = 0;
+  const int ring_w = a.C - a.sink;
+  if (a.block_tokens > 0) {
+    const int64_t n = a.n_tokens[b];
+    if (n > a.C) {                                  // before the ring has wrapped nothing is left out
+      const int64_t first_held = n - ring_w;        // oldest window token in the ring (>= sink here)
+      const int64_t first_kept = ((n - 1) / a.block_tokens - ring_w / a.block_tokens + 1) * a.block_tokens;
+      if (first_kept > first_held) {
+        ex_cnt = static_cast<int>(first_kept - first_held);
+        ex0 = static_cast<int>((first_held - a.sink) % ring_w);
+      }
+    }
+  }
+  auto attended = [&](int slot) {
+    if (slot >= nvalid) return false;
+    if (ex_cnt == 0 || slot < a.sink) return true;
+    int d = slot - a.sink - ex0;
+    if (d < 0) d += ring_w;
+    return d >= ex_cnt;
+  };
 
   auto issue_tile = [&](int t) {
     const int stage = (t - t_begin) % kDecStages;
@@ -160,7 +186,7 @@ __device__ __forceinline__ void decode_run_segment(const DecodeArgs& a, uint8_t*
     }
     // sacc[0,1]: token r, heads 2c, 2c+1;  sacc[2,3]: token r + 8
     const int tok0 = t * kDecTile + r;
-    const bool v0 = tok0 < nvalid, v1 = tok0 + 8 < nvalid;
+    const bool v0 = attended(tok0), v1 = attended(tok0 + 8);
     float s00 = v0 ? sacc[0] * a.scale_log2 : -INFINITY, s01 = v0 ? sacc[1] * a.scale_log2 : -INFINITY;
     float s10 = v1 ? sacc[2] * a.scale_log2 : -INFINITY, s11 = v1 ? sacc[3] * a.scale_log2 : -INFINITY;
     float mx0 = fmaxf(s00, s10), mx1 = fmaxf(s01, s11);
@@ -492,6 +518,7 @@ __global__ void ring_append_kernel(__nv_bfloat16* k_cache, __nv_bfloat16* v_cach
   const int64_t bh = row_id / T;
   const int b = static_cast<int>(bh / Hkv);
   const int64_t n0 = n_before[b];
+  if (n0 < 0) return;                                  // a negative count addresses nothing: the sequence is skipped
   const int64_t j = n0 + t, last = n0 + T - 1;
   if (j >= sink && j + window <= last) return;       // overwritten later in this call
   const int64_t slot = j < sink ? j : sink + (j - sink) % window;
@@ -508,6 +535,9 @@ static lg_status check_decode(const lg_decode_params* p) {
   if (!p) return LG_ERR_INVALID_ARG;
   if (p->B < 1 || p->Hq < 1 || p->Hkv < 1 || p->Hq % p->Hkv != 0) return LG_ERR_INVALID_ARG;
   if (p->sink_tokens < 0 || p->window_tokens < 1) return LG_ERR_INVALID_ARG;
+  if (p->block_tokens < 0) return LG_ERR_INVALID_ARG;
+  if (p->block_tokens > 0 && (p->window_tokens % p->block_tokens != 0 || p->sink_tokens % p->block_tokens != 0))
+    return LG_ERR_INVALID_ARG;                         // the block-aligned window counts whole blocks
   if (!(p->scale >= 0.f) || isinf(p->scale)) return LG_ERR_INVALID_ARG;
   if (p->D != 64 && p->D != 128) return LG_ERR_UNSUPPORTED;
   if (static_cast<int64_t>(p->sink_tokens) + p->window_tokens > (1ll << 30)) return LG_ERR_UNSUPPORTED;
@@ -546,6 +576,7 @@ extern "C" {
 
 lg_status lg_kv_ring_append(const lg_decode_params* p, void* k_cache, void* v_cache, const void* k_new,
                             const void* v_new, int32_t T_new, const int64_t* n_tokens_before, void* stream) {
+  LG_RANGE("lg_kv_ring_append");
   lg_status s = check_decode(p);
   if (s != LG_OK) return s;
   if (T_new < 0) return LG_ERR_INVALID_ARG;
@@ -577,6 +608,7 @@ size_t lg_sparse_decode_workspace_bytes(const lg_decode_params* p) {
 }
 
 lg_status lg_sparse_decode_workspace_init(void* workspace, size_t workspace_bytes, void* stream) {
+  LG_RANGE("lg_sparse_decode_workspace_init");
   if (!workspace || (reinterpret_cast<uintptr_t>(workspace) & 255)) return LG_ERR_INVALID_ARG;
   return cudaMemsetAsync(workspace, 0, workspace_bytes, static_cast<cudaStream_t>(stream)) == cudaSuccess ? LG_OK
                                                                                                            : LG_ERR_CUDA;
@@ -585,6 +617,7 @@ lg_status lg_sparse_decode_workspace_init(void* workspace, size_t workspace_byte
 lg_status lg_sparse_decode(const lg_decode_params* p, const void* q, const void* k_cache, const void* v_cache,
                            const int64_t* n_tokens, void* o, float* lse, void* workspace, size_t workspace_bytes,
                            void* stream) {
+  LG_RANGE("lg_sparse_decode");
   lg_status s = check_decode(p);
   if (s != LG_OK) return s;
   if (!q || !k_cache || !v_cache || !n_tokens || !o || !workspace) return LG_ERR_INVALID_ARG;
@@ -606,6 +639,8 @@ lg_status lg_sparse_decode(const lg_decode_params* p, const void* q, const void*
   a.Hq = p->Hq; a.Hkv = p->Hkv; a.G = p->Hq / p->Hkv;
   a.HG = (a.G + kDecHeads - 1) / kDecHeads;
   a.C = p->sink_tokens + p->window_tokens;
+  a.sink = p->sink_tokens;
+  a.block_tokens = p->block_tokens;
   a.nsplit = choose_nsplit(p);
   const float scale = p->scale > 0.f ? p->scale : 1.0f / sqrtf(static_cast<float>(p->D));
   a.scale_log2 = scale * 1.4426950408889634f;
@@ -699,6 +734,7 @@ lg_status static_scratch_address(void** out) {
 lg_status lg_sparse_decode_static(const lg_decode_params* p, const void* q, const void* k_cache,
                                   const void* v_cache, const int64_t* n_tokens, void* o, float* lse,
                                   void* stream) {
+  LG_RANGE("lg_sparse_decode_static");
   lg_status s = check_decode(p);
   if (s != LG_OK) return s;
   // the split partials of this problem must fit the fixed array
@@ -712,5 +748,14 @@ lg_status lg_sparse_decode_static(const lg_decode_params* p, const void* q, cons
                           stream);
 }
 
+lg_status lg_sparse_decode_static_reset(void* stream) {
+  LG_RANGE("lg_sparse_decode_static_reset");
+  void* scratch = nullptr;
+  lg_status s = static_scratch_address(&scratch);
+  if (s != LG_OK) return s;
+  return cudaMemsetAsync(scratch, 0, LG_DECODE_STATIC_SCRATCH_BYTES, static_cast<cudaStream_t>(stream)) == cudaSuccess
+             ? LG_OK
+             : LG_ERR_CUDA;
+}
 
 }  // extern "C"

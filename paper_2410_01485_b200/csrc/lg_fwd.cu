@@ -26,6 +26,7 @@ static lg_status launch_fwd_t(const Resolved& r, const WsLayout& w, const void* 
   a.L = r.L; a.Hq = r.Hq; a.G = r.G;
   a.q_start = r.q_start; a.Lq = r.Lq;
   a.exact_w = r.exact_w; a.ns = r.pat.ns;
+  a.win_block = r.win_block; a.win_phase = r.win_phase;
   a.doc_start = r.doc_start;
   a.scale_log2 = r.scale * 1.4426950408889634f;
   auto kern = fwd_kernel<D, BS>;

@@ -38,6 +38,10 @@ struct FwdArgs {
   int q_start, Lq;           // queries exist for rows [q_start, q_start + Lq) of the L key positions only
                              // (a chunk served against a cache); Q, O, LSE are indexed by row - q_start
   int exact_w, ns;           // token-exact window (0: off) and number of sink blocks
+  int win_block, win_phase;  // with exact_w: the window edge is block-aligned in shifted coordinates instead --
+                             // row i keeps the keys j with (i + phase) / win_block - (j + phase) / win_block
+                             // < exact_w / win_block (a chunk served against a ring whose first kept token
+                             // is `phase` tokens into the sequence); win_block = 0: token-exact edge
   const int32_t* doc_start;  // [B, L] first position of each query's document, or null
   float scale_log2;          // scale * log2(e)
 };
@@ -258,6 +262,10 @@ fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUt
     // lowest key position this row may see outside what the pattern already excludes: the start of its
     // document (0 without documents)
     const int dstart = (a.doc_start && qi < a.L && qi >= a.q_start) ? a.doc_start[static_cast<int64_t>(b) * a.L + qi] : 0;
+    // oldest key position the window lets this row see (blocks outside the sink)
+    const int win_lo = a.win_block > 0
+                           ? ((qi + a.win_phase) / a.win_block - a.exact_w / a.win_block + 1) * a.win_block - a.win_phase
+                           : qi - a.exact_w + 1;
     float m_ref = -INFINITY;   // reference maximum (scaled, log2 domain) the probabilities are relative to
     float l_run = 0.f;
     int p0 = 0, p1 = 0;        // P tiles published per half buffer (barrier phases)
@@ -283,7 +291,7 @@ fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUt
         // token-exact window, on blocks outside the sink)
         const int key0 = (e >> 4) * BS + (BS == 128 ? 64 * hf : 0);
         const int lim = ((e >> member) & 1) ? min(max(qi - key0 + 1, 0), 64) : 0;
-        const int lo_abs = (a.exact_w > 0 && (e >> 4) >= a.ns) ? max(dstart, qi - a.exact_w + 1) : dstart;
+        const int lo_abs = (a.exact_w > 0 && (e >> 4) >= a.ns) ? max(dstart, win_lo) : dstart;
         const int lo = min(max(lo_abs - key0, 0), 64);
 
         ok = mbar_wait_warp(bars + B_SF + s * 2 + hf, (hf ? p1 : p0) & 1, a.error_word, 12);

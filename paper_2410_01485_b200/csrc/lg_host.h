@@ -9,6 +9,21 @@
 #include "../../include/lg.h"
 #include "lg_pattern.h"
 
+// Optional NVTX ranges around every entry point (build with -DLG_NVTX; the NVTX headers are
+// self-contained and cost nothing when no tool is attached).
+#ifdef LG_NVTX
+#include <nvtx3/nvToolsExt.h>
+namespace lg {
+struct NvtxRange {
+  explicit NvtxRange(const char* name) { nvtxRangePushA(name); }
+  ~NvtxRange() { nvtxRangePop(); }
+};
+}  // namespace lg
+#define LG_RANGE(name) ::lg::NvtxRange lg_nvtx_range_(name)
+#else
+#define LG_RANGE(name) ((void)0)
+#endif
+
 namespace lg {
 
 inline size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
@@ -22,6 +37,7 @@ struct Resolved {          // validated, defaulted copy of lg_attn_params
   PatternDev pat;
   float scale;
   int exact_w;             // token-exact window length in tokens (0: block-granular)
+  int win_block, win_phase;  // forward only, with exact_w: block-aligned window edge in coordinates shifted by win_phase (0: off)
   int64_t qs[3], ks[3], vs[3], os[3];
   int n_qtiles, n_ktiles;  // ceil(L / 128)
   int n_stiles;            // ceil(L / 256): super-tiles of the forward

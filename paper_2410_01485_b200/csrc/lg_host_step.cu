@@ -66,6 +66,7 @@ lg_status lg_sparse_attn_fwd_bwd_host(const lg_attn_params* p, const void* q_hos
                                       const void* v_host, const void* d_o_host, void* o_host, float* lse_host,
                                       void* dq_host, void* dk_host, void* dv_host, const lg_device_step_buffers* dev,
                                       int head_groups, void* stream_in, void* stream_compute, void* stream_out) {
+  LG_RANGE("lg_sparse_attn_fwd_bwd_host");
   if (!p || !dev) return LG_ERR_INVALID_ARG;
   GroupPlan g;
   lg_status s = plan_groups(p, head_groups, &g);

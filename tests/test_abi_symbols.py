@@ -158,6 +158,17 @@ def test_chunk_prefill_planning_on_host(lib):
     assert lib.lg_chunk_prefill(C.byref(p), 256, 256, 256, 256, 256, 64, 1000, 256, 256, 256, full - 1, None) == -3
 
 
+def test_block_aligned_decode_params_are_validated(lib):
+    ok = binding.decode_params(1, 8, 1, 128, 64, 256, block_tokens=64)
+    assert lib.lg_sparse_decode_workspace_bytes(C.byref(ok)) > 0
+    for bad in (binding.decode_params(1, 8, 1, 128, 64, 256, block_tokens=-1),
+                binding.decode_params(1, 8, 1, 128, 64, 200, block_tokens=64),      # window not whole blocks
+                binding.decode_params(1, 8, 1, 128, 32, 256, block_tokens=64)):     # sink not whole blocks
+        assert lib.lg_sparse_decode_workspace_bytes(C.byref(bad)) == 0
+        assert lib.lg_sparse_decode(C.byref(bad), 256, 256, 256, 256, 256, None, 256, 1 << 20, None) == -1
+    assert lib.lg_chunk_prefill_workspace_bytes(C.byref(binding.decode_params(1, 4, 2, 128, 64, 128, block_tokens=48)), 64, 0) == 0
+
+
 def test_decode_workspace_init_rejects_bad_pointers(lib):
     assert lib.lg_sparse_decode_workspace_init(None, 1024, None) == -1
     assert lib.lg_sparse_decode_workspace_init(128, 1024, None) == -1   # not 256-byte aligned

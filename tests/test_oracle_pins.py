@@ -432,6 +432,32 @@ def test_decode_bruteforce_and_permutation_invariance():
     assert (o0 == 0).all() and np.isneginf(lse0).all()
 
 
+def test_block_aligned_decode_is_the_training_masks_row():
+    """With block_tokens the serving mask is the block-granular training mask (Section 4.1: the local
+    context is counted in blocks): the decode at position n - 1 equals row n - 1 of the mask-based forward
+    under the default (block-granular) pattern, for every n, and its keys are tokens the ring still holds."""
+    Hq, Hkv, D, Bs, sink, W = 4, 2, 6, 4, 4, 12
+    L = 61
+    q, k, v = _rand((Hq, L, D), 90), _rand((Hkv, L, D), 91), _rand((Hkv, L, D), 92)
+    pat = O.Pattern(L=L, block=Bs, mode=O.MODE_SINK_WINDOW, sink_tokens=sink, window_tokens=W)
+    Oo, LSE = O.attn_forward(q, k, v, pat, 0.4)
+    for n in range(1, L + 1):
+        o, lse = O.decode(q[:, n - 1], k, v, n, sink, W, 0.4, block_tokens=Bs)
+        np.testing.assert_allclose(o, Oo[:, n - 1], rtol=1e-12, atol=1e-13)
+        np.testing.assert_allclose(lse, LSE[:, n - 1], rtol=1e-12, atol=1e-13)
+        aligned, held = O.decode_valid(n, sink, W, Bs), O.decode_valid(n, sink, W)
+        assert (aligned <= held).all()                       # a subset of what the cache holds
+        assert held.sum() - aligned.sum() == (0 if n <= sink + W else Bs - 1 - (n - 1) % Bs)
+        # written out with loops
+        i = n - 1
+        assert [j for j in range(n) if j < sink or i // Bs - j // Bs < W // Bs] == list(np.nonzero(aligned)[0])
+    # the chunk function is T such steps
+    n0, T = 23, 9
+    oc, lc = O.chunk_prefill(q[:, n0:n0 + T], k, v, n0, sink, W, 0.4, block_tokens=Bs)
+    np.testing.assert_allclose(oc, Oo[:, n0:n0 + T], rtol=1e-12, atol=1e-13)
+    np.testing.assert_allclose(lc, LSE[:, n0:n0 + T], rtol=1e-12, atol=1e-13)
+
+
 def test_ring_replay_holds_exactly_the_surviving_tokens():
     sink, W = 3, 5
     for n0, T in ((0, 1), (0, 4), (2, 3), (0, 8), (5, 20), (7, 1), (0, 31)):
