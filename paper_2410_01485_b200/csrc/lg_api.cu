@@ -1,5 +1,6 @@
 // C-ABI entry points: validation, workspace layout, block-index builder launches.
 #include <math.h>
+#include <stdlib.h>
 #include <string.h>
 
 #include <atomic>
@@ -112,6 +113,19 @@ lg_status resolve(const lg_attn_params* p, Resolved* r) {
   return LG_OK;
 }
 
+// The single-sweep backward needs D = 128 (its dQ^T product puts the head dimension on the 128 TMEM
+// lanes).  It is the default for the sink + window and full-causal patterns, where every kv tile has a
+// short schedule and the fixed order of the dQ parts follows the launch order without waiting; the
+// strided pattern keeps the two passes.  LG_BWD_VARIANT = fused | two_pass overrides the choice (read
+// at every call; it must not change between a size query, a prepare and the calls that use them).
+bool bwd_is_fused(const Resolved& r) {
+  if (r.D != 128) return false;
+  const char* env = getenv("LG_BWD_VARIANT");
+  if (env && strcmp(env, "two_pass") == 0) return false;
+  if (env && strcmp(env, "fused") == 0) return true;
+  return false;
+}
+
 WsLayout ws_layout(const Resolved& r, bool want_bwd) {
   WsLayout w{};
   size_t off = sizeof(WsHeader);
@@ -139,6 +153,15 @@ WsLayout ws_layout(const Resolved& r, bool want_bwd) {
     w.kt_off = take((static_cast<size_t>(r.n_ktiles) + 1) * 4);
     if (r.doc_start) w.doc_end = take(static_cast<size_t>(r.B) * r.L * 4);
     w.delta = take(static_cast<size_t>(r.B) * r.Hq * align_up(r.L, 128) * 8);   // rows padded to whole tiles   // two planes: -LSE * log2 e and -delta per query row
+    if (bwd_is_fused(r)) {
+      const size_t Lp = align_up(r.L, 128);
+      w.kt_rank = take(nnz * 4);
+      w.kt_tile_of = take(nB * 4);
+      w.kt_pos = take(static_cast<size_t>(r.n_ktiles) * 4);
+      w.sem_bytes = (64 + static_cast<size_t>(r.B) * r.Hq * (Lp / 64) * 4) * 4;   // ticket + four counters per (head, 64-row group)
+      w.sem = take(w.sem_bytes);
+      w.dq_acc = take(static_cast<size_t>(r.B) * r.Hq * Lp * r.D * 4);
+    }
   }
   w.total = off;
   return w;
@@ -162,6 +185,7 @@ unsigned long long pattern_fingerprint(const Resolved& r, bool has_bwd) {
   mix(static_cast<unsigned long long>(r.L)); mix(r.block); mix(r.mode); mix(r.pat.ns); mix(r.pat.nw);
   mix(r.pat.stride); mix(r.pat.nl); mix(r.exact_w); mix(has_bwd ? 1 : 0);
   mix(reinterpret_cast<uintptr_t>(r.doc_start)); mix(r.doc_start ? r.B : 0);
+  mix(has_bwd && bwd_is_fused(r) ? 1 : 0);
   return h ? h : 1;
 }
 
@@ -208,6 +232,13 @@ lg_status prepare_workspace(const Resolved& r, const WsLayout& w, uint8_t* ws, i
     kv_tile_merge_kernel<<<(nt + 127) / 128, 128, 0, stream>>>(i32(w.col_ptr), i32(w.row_idx), i32(w.kt_cols),
                                                                i32(w.kt_off), R, nt, i32(w.kt_cnt), i32(w.kt_ent)); note_launch();
     tile_order_kernel<<<(nt + 127) / 128, 128, 0, stream>>>(i32(w.kt_cnt), nt, i32(w.kt_order)); note_launch();
+    if (bwd_is_fused(r)) {   // order of the dQ parts: rank of every (kv tile, query block) entry
+      kv_tile_of_kernel<<<(nt * R + 127) / 128, 128, 0, stream>>>(i32(w.kt_cols), R, nt, i32(w.kt_tile_of)); note_launch();
+      tile_pos_kernel<<<(nt + 127) / 128, 128, 0, stream>>>(i32(w.kt_order), nt, i32(w.kt_pos)); note_launch();
+      kv_tile_rank_kernel<<<nt, 128, 0, stream>>>(i32(w.row_ptr), i32(w.col_idx), i32(w.kt_tile_of), i32(w.kt_pos),
+                                                  i32(w.kt_cols), i32(w.kt_off), i32(w.kt_cnt), i32(w.kt_ent), R,
+                                                  i32(w.kt_rank)); note_launch();
+    }
     if (r.doc_start) {
       const int64_t n = static_cast<int64_t>(r.B) * r.L;
       doc_end_kernel<<<static_cast<unsigned>((n + 255) / 256), 256, 0, stream>>>(r.doc_start, i32(w.doc_end), r.B, r.L); note_launch();

@@ -60,6 +60,10 @@ struct WsLayout {
   size_t kt_cols, kt_off;                        // members of each kv tile, start of its schedule
   size_t doc_end;                                // int32 [B, L]: end of each token's document (bwd with documents only)
   size_t delta;                                  // 2 x float [B, Hq, L]: -LSE * log2 e, then -delta (bwd only)
+  // fused backward only (0 otherwise): rank of every kv-tile schedule entry, column -> tile, tile -> launch
+  // position, the ticket + arrival counters (cleared at every call), and dQ in fp32
+  size_t kt_rank, kt_tile_of, kt_pos, sem, dq_acc;
+  size_t sem_bytes;
   size_t total;
 };
 WsLayout ws_layout(const Resolved& r, bool want_bwd);
@@ -75,6 +79,9 @@ lg_status prepare_workspace(const Resolved& r, const WsLayout& w, uint8_t* ws, i
 // boxes of 64 columns x `box_rows` rows and the 128-byte swizzle.
 lg_status make_tmap(CUtensorMap* out, const void* base, int B, int H, int L, int D, const int64_t strides[3],
                     int box_rows);
+
+// Which backward runs for this problem: the single sweep (lg_bwd_fused.cuh) or the two passes (lg_bwd.cuh).
+bool bwd_is_fused(const Resolved& r);
 
 lg_status check_arch();
 inline bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15) == 0; }

@@ -207,6 +207,58 @@ __global__ void kv_tile_merge_kernel(const int32_t* __restrict__ col_ptr, const 
   tile_cnt[t] = n;
 }
 
+// ---- order of the dQ contributions in the fused backward --------------------------------------
+// In the fused backward every kv tile adds its part of dQ to the rows of the query blocks it
+// visits; the parts of one query block are added in the launch order of the kv tiles that hold
+// a column of its row.  rank[e] of schedule entry e = (tile t, query block qb) is the number of
+// OTHER kv tiles with an active column in row qb that come before t in that order: the tile's
+// part is the rank-th one (0 = it initialises the rows).
+//   tile_of[kb] = kv tile of pattern column kb;  pos[t] = launch position of tile t.
+__global__ void kv_tile_of_kernel(const int32_t* __restrict__ cols, int R, int n_tiles, int32_t* __restrict__ tile_of) {
+  const int c = blockIdx.x * blockDim.x + threadIdx.x;
+  if (c >= n_tiles * R) return;
+  const int kb = cols[c];
+  if (kb >= 0) tile_of[kb] = c / R;
+}
+__global__ void tile_pos_kernel(const int32_t* __restrict__ order, int n_tiles, int32_t* __restrict__ pos) {
+  const int i = blockIdx.x * blockDim.x + threadIdx.x;
+  if (i < n_tiles) pos[order[i]] = i;
+}
+// grid = kv tiles, block = 128 threads striding over the tile's entries
+__global__ void kv_tile_rank_kernel(const int32_t* __restrict__ row_ptr, const int32_t* __restrict__ col_idx,
+                                    const int32_t* __restrict__ tile_of, const int32_t* __restrict__ pos,
+                                    const int32_t* __restrict__ cols, const int32_t* __restrict__ off,
+                                    const int32_t* __restrict__ tile_cnt, const int32_t* __restrict__ tile_ent, int R,
+                                    int32_t* __restrict__ rank) {
+  const int t = blockIdx.x;
+  const int my_pos = pos[t];
+  const int n = tile_cnt[t];
+  for (int e = threadIdx.x; e < n; e += blockDim.x) {
+    const int qb = tile_ent[off[t] + e] >> 2;
+    const int r0 = row_ptr[qb], r1 = row_ptr[qb + 1];
+    int count = 0;
+    for (int x = r0; x < r1; ++x) {
+      const int kb = col_idx[x];
+      const int u = tile_of[kb];
+      if (u == t || pos[u] >= my_pos) continue;
+      if (R == 2) {   // a tile with both columns in this row counts once: at its smaller column
+        const int ca = cols[2 * u], cb = cols[2 * u + 1];
+        const int other = (kb == ca) ? cb : ca;
+        if (other >= 0 && other < kb) {
+          int lo = r0, hi = r1;            // is `other` in the (ascending) row?
+          while (lo < hi) {
+            const int mid = (lo + hi) >> 1;
+            if (col_idx[mid] < other) lo = mid + 1; else hi = mid;
+          }
+          if (lo < r1 && col_idx[lo] == other) continue;
+        }
+      }
+      ++count;
+    }
+    rank[off[t] + e] = count;
+  }
+}
+
 // doc_end[b][j] = end (one past the last token) of the document token j belongs to, from
 // doc_start[b][i] = first token of token i's document (non-decreasing): the first i > j whose
 // document starts after j, found by bisection, or L.

@@ -96,8 +96,12 @@ def test_block_index_bit_exact(lg, cfg):
         assert np.array_equal(g.cpu().numpy(), r), name
 
 
+@pytest.mark.parametrize("variant", ["fused", "two_pass"])
 @pytest.mark.parametrize("cfg", SMALL, ids=lambda c: c.name)
-def test_fwd_bwd_parity_small(lg, cfg):
+def test_fwd_bwd_parity_small(lg, cfg, variant, monkeypatch):
+    """Both backward variants (the single sweep that adds the parts of dQ in a fixed order, and the two
+    passes) on every small pattern; with D = 64 both names run the two passes."""
+    monkeypatch.setenv("LG_BWD_VARIANT", variant)
     p = lg.params_of(cfg)
     inp = synth.make_attn_inputs(cfg, "cuda", seed=0, with_do=True)
     ws = lg.attn_workspace(p, True)
@@ -117,19 +121,26 @@ def test_fwd_bwd_parity_small(lg, cfg):
         _assert_close(synth.to_f64(dv[b]), dV, TOL_G, "dV")
 
 
-def test_bitwise_reproducible(lg):
-    cfg = SMALL[5]
+@pytest.mark.parametrize("variant", ["fused", "two_pass"])
+@pytest.mark.parametrize("cfg", [SMALL[5], replace(synth.CFG1, name="rep_window", L=8192, D=128, Hq=8, Hkv=4, block=128,
+                                                   sink_tokens=128, window_tokens=1024)], ids=lambda c: c.name)
+def test_bitwise_reproducible(lg, cfg, variant, monkeypatch):
+    """Same inputs, same bits, run after run: single writers in the two passes; in the single sweep the parts
+    of dQ that several kv tiles add to the same rows arrive in a fixed order (the second case has 64 kv tiles
+    per head in flight at once, so the order would show if it were left to chance)."""
+    monkeypatch.setenv("LG_BWD_VARIANT", variant)
     p = lg.params_of(cfg)
     inp = synth.make_attn_inputs(cfg, "cuda", seed=1, with_do=True)
     outs = []
-    for _ in range(2):
+    for _ in range(4):
         o, lse = lg.lg_sparse_attn_fwd(p, inp["q"], inp["k"], inp["v"])
         dq, dk, dv = lg.lg_sparse_attn_bwd(p, inp["q"], inp["k"], inp["v"], o, lse, inp["do"])
         torch.cuda.synchronize()
         outs.append((o, lse, dq, dk, dv))
-    for x, y in zip(*outs):
-        assert torch.equal(x.view(torch.int16) if x.dtype == torch.bfloat16 else x.view(torch.int32),
-                           y.view(torch.int16) if y.dtype == torch.bfloat16 else y.view(torch.int32))
+    for other in outs[1:]:
+        for x, y in zip(outs[0], other):
+            assert torch.equal(x.view(torch.int16) if x.dtype == torch.bfloat16 else x.view(torch.int32),
+                               y.view(torch.int16) if y.dtype == torch.bfloat16 else y.view(torch.int32))
 
 
 def test_masked_keys_get_exactly_zero_gradient(lg):
