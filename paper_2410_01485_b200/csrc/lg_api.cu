@@ -113,17 +113,29 @@ lg_status resolve(const lg_attn_params* p, Resolved* r) {
   return LG_OK;
 }
 
-// The single-sweep backward needs D = 128 (its dQ^T product puts the head dimension on the 128 TMEM
-// lanes).  It is the default for the sink + window and full-causal patterns, where every kv tile has a
-// short schedule and the fixed order of the dQ parts follows the launch order without waiting; the
-// strided pattern keeps the two passes.  LG_BWD_VARIANT = fused | two_pass overrides the choice (read
-// at every call; it must not change between a size query, a prepare and the calls that use them).
-bool bwd_is_fused(const Resolved& r) {
-  if (r.D != 128) return false;
+// Three backward variants compute the same gradients (see BwdVariant).  The two passes run everywhere.
+// Keeping dS trades workspace and HBM traffic (2 bytes per visible pair, written once and read once, on
+// a memory system the attention kernels otherwise leave idle) for the two recomputed products of the dQ
+// pass; it is the default where it applies: 128-token blocks, no per-sequence lists, and a dS buffer of
+// at most LG_KEEP_DS_MAX_GB (default 48) gigabytes.  The single sweep needs D = 128 and is only chosen
+// explicitly: its ordered fp32 additions into dQ cost more than the recomputation they save.
+// LG_BWD_VARIANT = two_pass | keep_ds | fused overrides the choice (read at every call; it must not
+// change between a size query, a prepare and the calls that use them).
+size_t ds_buffer_bytes(const Resolved& r) {
+  return static_cast<size_t>(r.B) * r.Hq * static_cast<size_t>(r.nnz) * (r.block / 64) * (128 * 128);
+}
+
+BwdVariant bwd_variant(const Resolved& r) {
   const char* env = getenv("LG_BWD_VARIANT");
-  if (env && strcmp(env, "two_pass") == 0) return false;
-  if (env && strcmp(env, "fused") == 0) return true;
-  return false;
+  if (env && strcmp(env, "two_pass") == 0) return kBwdTwoPass;
+  if (env && strcmp(env, "fused") == 0) return r.D == 128 ? kBwdFused : kBwdTwoPass;
+  // the stored tiles are addressed by 32-bit row coordinates of a tensor map
+  const bool can_keep = r.block == 128 && !(r.doc_start != nullptr && r.B > 1) &&
+                        ds_buffer_bytes(r) / 128 < (1ull << 31);
+  if (env && strcmp(env, "keep_ds") == 0) return can_keep ? kBwdKeepDs : kBwdTwoPass;
+  double max_gb = 48.0;
+  if (const char* m = getenv("LG_KEEP_DS_MAX_GB")) max_gb = atof(m);
+  return (can_keep && static_cast<double>(ds_buffer_bytes(r)) <= max_gb * 1e9) ? kBwdKeepDs : kBwdTwoPass;
 }
 
 WsLayout ws_layout(const Resolved& r, bool want_bwd) {
@@ -162,6 +174,7 @@ WsLayout ws_layout(const Resolved& r, bool want_bwd) {
       w.sem = take(w.sem_bytes);
       w.dq_acc = take(static_cast<size_t>(r.B) * r.Hq * Lp * r.D * 4);
     }
+    if (bwd_variant(r) == kBwdKeepDs) w.ds_buf = take(ds_buffer_bytes(r));
   }
   w.total = off;
   return w;
@@ -185,7 +198,7 @@ unsigned long long pattern_fingerprint(const Resolved& r, bool has_bwd) {
   mix(static_cast<unsigned long long>(r.L)); mix(r.block); mix(r.mode); mix(r.pat.ns); mix(r.pat.nw);
   mix(r.pat.stride); mix(r.pat.nl); mix(r.exact_w); mix(has_bwd ? 1 : 0);
   mix(reinterpret_cast<uintptr_t>(r.doc_start)); mix(r.doc_start ? r.B : 0);
-  mix(has_bwd && bwd_is_fused(r) ? 1 : 0);
+  mix(has_bwd ? static_cast<int>(bwd_variant(r)) : 0);
   return h ? h : 1;
 }
 
@@ -281,6 +294,20 @@ lg_status make_tmap(CUtensorMap* out, const void* base, int B, int H, int L, int
   return rc == CUDA_SUCCESS ? LG_OK : LG_ERR_CUDA;
 }
 
+
+// dS^T buffer of the backward that keeps dS: rows of 64 bf16 (128 bytes), boxes of 128 rows, 128-byte swizzle
+lg_status make_tmap_ds(CUtensorMap* out, const void* base, int64_t rows) {
+  EncodeTiledFn fn = get_encode_fn();
+  if (!fn) return LG_ERR_CUDA;
+  cuuint64_t dims[2] = {64, static_cast<cuuint64_t>(rows)};
+  cuuint64_t gstr[1] = {128};
+  cuuint32_t box[2] = {64, 128};
+  cuuint32_t estr[2] = {1, 1};
+  CUresult rc = fn(out, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(base), dims, gstr, box, estr,
+                   CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                   CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+  return rc == CUDA_SUCCESS ? LG_OK : LG_ERR_CUDA;
+}
 
 // ---- chunk served against a sink + window ring ----------------------------------------------
 // Time-ordered copy of what the ring holds, followed by the chunk: K_lin, V_lin [B, Hkv, Lc, D]

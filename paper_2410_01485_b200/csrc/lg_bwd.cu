@@ -34,7 +34,10 @@ static lg_status launch_bwd_t(const Resolved& r, const WsLayout& w, const void* 
   a.doc_end = r.doc_start ? reinterpret_cast<const int32_t*>(ws + w.doc_end) : nullptr;
   a.scale = r.scale;
   a.scale_log2 = r.scale * 1.4426950408889634f;
+  a.ds_nnz = r.nnz;
+  a.aux0 = a.aux1 = a.aux2 = nullptr;
   constexpr int smem = BwdSmem<D, BS>::kTotal;
+  const BwdVariant variant = bwd_variant(r);
 
   if constexpr (D == 128) {
     if (bwd_is_fused(r)) {
@@ -92,12 +95,49 @@ static lg_status launch_bwd_t(const Resolved& r, const WsLayout& w, const void* 
     a.out0 = static_cast<__nv_bfloat16*>(dk);
     a.out1 = static_cast<__nv_bfloat16*>(dv);
     for (int i = 0; i < 3; ++i) { a.s0[i] = r.ks[i]; a.s1[i] = r.vs[i]; }
-    auto kern = bwd_dkdv_kernel<D, BS>;
-    if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, smem) != cudaSuccess)
-      return LG_ERR_CUDA;
     dim3 grid(r.B * r.Hkv, r.n_ktiles);
-    kern<<<grid, kKvThreads, smem, stream>>>(tq, tk, tv, tdo, a); note_launch();
+    if (variant == kBwdKeepDs) {
+      CUtensorMap tds;
+      if ((s = make_tmap_ds(&tds, ws + w.ds_buf, static_cast<int64_t>(ds_buffer_bytes(r) / 128))) != LG_OK) return s;
+      auto kern = bwd_dkdv_kernel<D, BS, true>;
+      constexpr int smem_k = BwdSmem<D, BS, true>::kTotal;
+      if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, smem_k) != cudaSuccess)
+        return LG_ERR_CUDA;
+      kern<<<grid, kKvThreads + 32, smem_k, stream>>>(tq, tk, tv, tdo, tds, a); note_launch();
+    } else {
+      auto kern = bwd_dkdv_kernel<D, BS, false>;
+      if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, smem) != cudaSuccess)
+        return LG_ERR_CUDA;
+      kern<<<grid, kKvThreads, smem, stream>>>(tq, tk, tv, tdo, tq /* unused */, a); note_launch();
+    }
     if (marks) cudaEventRecord(marks[2], stream);
+  }
+  if constexpr (BS == 128) {
+    if (variant == kBwdKeepDs) {
+      // ---- dQ = scale * dS K from the kept tiles ------------------------------------------
+      CUtensorMap tk, tds;
+      if ((s = make_tmap(&tk, k, r.B, r.Hkv, r.L, D, r.ks, 128)) != LG_OK) return s;
+      if ((s = make_tmap_ds(&tds, ws + w.ds_buf, static_cast<int64_t>(ds_buffer_bytes(r) / 128))) != LG_OK) return s;
+      a.tile_off = reinterpret_cast<const int32_t*>(ws + w.row_ptr);
+      a.tile_ent = reinterpret_cast<const int32_t*>(ws + w.col_idx);
+      a.tile_cols = nullptr;
+      a.tile_cnt = nullptr;
+      a.order = reinterpret_cast<const int32_t*>(ws + w.qt_order);
+      a.aux0 = reinterpret_cast<const int32_t*>(ws + w.col_ptr);
+      a.aux1 = reinterpret_cast<const int32_t*>(ws + w.row_idx);
+      a.aux2 = reinterpret_cast<const int32_t*>(ws + w.kt_off);
+      a.out0 = static_cast<__nv_bfloat16*>(dq);
+      a.out1 = nullptr;
+      for (int i = 0; i < 3; ++i) { a.s0[i] = r.qs[i]; a.s1[i] = 0; }
+      auto kern = bwd_dq_from_ds_kernel<D>;
+      constexpr int smem_q = DqDsSmem<D>::kTotal;
+      if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, smem_q) != cudaSuccess)
+        return LG_ERR_CUDA;
+      dim3 grid(r.B * r.Hq, r.n_qtiles);
+      kern<<<grid, kDq2Threads, smem_q, stream>>>(tk, tds, a); note_launch();
+      if (marks) cudaEventRecord(marks[3], stream);
+      return cudaGetLastError() == cudaSuccess ? LG_OK : LG_ERR_CUDA;
+    }
   }
   // ---- dQ pass ------------------------------------------------------------------------
   {

@@ -52,6 +52,13 @@ struct BwdArgs {
   const int32_t* doc_start;  // [B, L] first position of each token's document, or null
   const int32_t* doc_end;    // [B, L] end of each token's document (null together with doc_start)
   float scale, scale_log2;
+  // dK/dV pass that also keeps dS (see bwd_dkdv_kernel): dS^T of every half-step of 64 queries goes to
+  // ds_buf as a tile of [128 keys][64 queries] bf16; tile index = ((b * Hq + h) * ds_nnz + schedule
+  // position of the (kv tile, query block) entry) * (block / 64) + half.  The dQ pass then reads them back.
+  int64_t ds_nnz;
+  const int32_t* aux0;       // dQ-from-dS pass: col_ptr (CSC)        } to find where a (query block, key block)
+  const int32_t* aux1;       //                  row_idx (CSC)        } pair sits in its kv tile's schedule
+  const int32_t* aux2;       //                  start of each kv tile's schedule
 };
 
 // ---- stat = -(LSE * log2 e) and -rowsum(dO * O), stored negated (they are only ever subtracted),
@@ -98,17 +105,20 @@ struct BwdTile {
   static constexpr int kBytes = (D / 64) * kBox;
 };
 
-template <int D, int BS>
+template <int D, int BS, bool kSpill = false>
 struct BwdSmem {
   static constexpr int kTile = BwdTile<D>::kBytes;
-  static constexpr int kAStages = 3;   // operand read by the first and the last MMA of a step (K | Q)
+  static constexpr int kDs = 128 * 128;                          // a dS^T tile: 128 keys x 64 queries bf16
+  static constexpr int kAStages = kSpill ? 2 : 3;   // operand read by the first and the last MMA of a step (K | Q)
   static constexpr int kBStages = 2;   // operand read by adjacent MMAs (V | dO)
   static constexpr int oFix0 = 0, oFix1 = kTile;
   static constexpr int oA = 2 * kTile;
   static constexpr int oB = oA + kAStages * kTile;
-  static constexpr int oStat = oB + kBStages * kTile;            // dK/dV pass: [2 stages][2 planes][128] floats
+  static constexpr int oDS = oB + kBStages * kTile;              // [2] dS^T tiles on their way to global memory (kSpill)
+  static constexpr int oStat = oDS + (kSpill ? 2 * kDs : 0);     // dK/dV pass: [2 stages][2 planes][128] floats
   static constexpr int oBar = oStat + 2 * 128 * 8;
-  static constexpr int kTotal = oBar + 256;
+  static constexpr int kBarBytes = 512;                          // mbarriers, the TMEM slot and the step's schedule entries
+  static constexpr int kTotal = oBar + kBarBytes;
 };
 
 // load one step (128 rows: one 128-row block, or two 64-row blocks) of a [.., L, D] tensor
@@ -461,22 +471,28 @@ constexpr int kKvHalf = LG_KV_HALF;                        // queries of a (half
 constexpr int kKvNB = 128 / kKvHalf;                       // (half-)steps per step = score buffers in rotation
 constexpr int kKvCols = kKvHalf / (kKvEwWarps / 4);        // queries of a half-step per element-wise thread
 
-template <int D, int BS>
-__global__ void __launch_bounds__(kKvThreads, 1)
+// kSpill: the pass also writes dS^T (bf16) of every half-step to global memory (tm_ds: the buffer as
+// rows of 64 queries, boxes of 128 key rows, 128-byte swizzle), so that the dQ pass is one product per
+// step, dQ += dS K, instead of recomputing S and dP (bwd_dq_from_ds_kernel).  The element-wise warps put
+// dS^T into shared memory as well as tensor memory; the thread that issues dK sends the tile on its way.
+template <int D, int BS, bool kSpill>
+__global__ void __launch_bounds__(kKvThreads + (kSpill ? 32 : 0), 1)
 bwd_dkdv_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUtensorMap tm_k,
                 const __grid_constant__ CUtensorMap tm_v, const __grid_constant__ CUtensorMap tm_do,
-                const BwdArgs a) {
-  using SM = BwdSmem<D, BS>;
+                const __grid_constant__ CUtensorMap tm_ds, const BwdArgs a) {
+  using SM = BwdSmem<D, BS, kSpill>;
+  constexpr int kQS = SM::kAStages;
   constexpr int R = 128 / BS;
   constexpr uint32_t kColS = 0, kColDP = 128, kColDV = 256, kColDK = 384;
   constexpr int kTile = SM::kTile;
   enum { B_FIX = 0, B_QF = 1, B_QE = 4, B_OF = 7, B_OE = 9, B_SF = 11, B_DPF = 13, B_PF = 15, B_DSF = 17,
-         B_DONE = 19, B_DRAIN = 20, B_STF = 22, B_STE = 24, B_COUNT = 26 };
+         B_DONE = 19, B_DRAIN = 20, B_STF = 22, B_STE = 24, B_DSE = 26, B_DSS = 28, B_COUNT = 30 };
 
   extern __shared__ __align__(1024) uint8_t smem[];
   uint64_t* bars = reinterpret_cast<uint64_t*>(smem + SM::oBar);
   uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + B_COUNT);
   int32_t* sEnt = reinterpret_cast<int32_t*>(bars + B_COUNT + 1);   // [2][2]: entries of a step's items
+  static_assert((B_COUNT + 1) * 8 + 16 <= SM::kBarBytes, "barrier area too small");
   const int tid = threadIdx.x, lane = tid & 31;
   const int warp = __shfl_sync(0xffffffffu, tid >> 5, 0);   // same value, known to be warp-uniform
   if ((smem_u32(smem) & 1023u) != 0) {
@@ -488,6 +504,7 @@ bwd_dkdv_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
   uint8_t* sV = smem + SM::oFix1;
   uint8_t* sQ = smem + SM::oA;     // [3]
   uint8_t* sDO = smem + SM::oB;    // [2]
+  uint8_t* sDS = smem + SM::oDS;   // [2] (kSpill)
   float* sStat = reinterpret_cast<float*>(smem + SM::oStat);   // [2 stages][-LSE2 | -delta][128 queries]
 
   // has a wait already given up in this call?  (read now, so that it travels with the schedule loads below)
@@ -508,7 +525,7 @@ bwd_dkdv_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
 
   if (tid == 0) {
     mbar_init(bars + B_FIX, 1);
-    for (int i = 0; i < 3; ++i) { mbar_init(bars + B_QF + i, 1); mbar_init(bars + B_QE + i, 1); }
+    for (int i = 0; i < 3; ++i) { mbar_init(bars + B_QF + i, 1); mbar_init(bars + B_QE + i, 1); }   // (kQS of them are used)
     for (int i = 0; i < 2; ++i) {
       mbar_init(bars + B_OF + i, 1);
       mbar_init(bars + B_OE + i, 2);      // dP^T (thread B) and dV (thread A) both read the dO tile
@@ -519,6 +536,8 @@ bwd_dkdv_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
       mbar_init(bars + B_DRAIN + i, 1);
       mbar_init(bars + B_STF + i, 1);
       mbar_init(bars + B_STE + i, kKvEwWarps);
+      mbar_init(bars + B_DSE + i, 1);
+      mbar_init(bars + B_DSS + i, kKvEwWarps);
     }
     mbar_init(bars + B_DONE, 2);          // the last dV and the last dK
     mbar_fence_init();
@@ -561,7 +580,7 @@ bwd_dkdv_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
         if (++e == n_ent) { e = 0; ++grp; }
       };
       for (int j = 0; j < n_steps; ++j) {
-        const int sq = j % 3, so = j & 1;
+        const int sq = j % kQS, so = j & 1;
         int h0, r0, e0, h1, r1, e1;
         next_item(h0, r0, e0);
         h1 = h0; r1 = r0; e1 = e0 & ~3;                         // a missing second item repeats the first block, as nobody's member
@@ -586,7 +605,7 @@ bwd_dkdv_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
           }
         }
         nst = j + 1;
-        if (j >= 3) ok = mbar_wait(bars + B_QE + sq, ((j / 3) - 1) & 1, a.error_word, 11);
+        if (j >= kQS) ok = mbar_wait(bars + B_QE + sq, ((j / kQS) - 1) & 1, a.error_word, 11);
         if (!ok) break;
         mbar_expect_tx(bars + B_QF + sq, kTile);
         tma_load_rows<D, BS>(sQ + sq * kTile, &tm_q, bars + B_QF + sq, 0, r0, h0, b);
@@ -600,7 +619,7 @@ bwd_dkdv_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
         no = j + 1;
       }
       mbar_wait(bars + B_FIX, 0, a.error_word, 16);
-      for (int j = max(nq - 3, 0); j < nq; ++j) mbar_wait(bars + B_QF + j % 3, (j / 3) & 1, a.error_word, 17);
+      for (int j = max(nq - kQS, 0); j < nq; ++j) mbar_wait(bars + B_QF + j % kQS, (j / kQS) & 1, a.error_word, 17);
       for (int j = max(no - 2, 0); j < no; ++j) mbar_wait(bars + B_OF + (j & 1), (j / 2) & 1, a.error_word, 18);
       for (int j = max(nst - 2, 0); j < nst; ++j) mbar_wait(bars + B_STF + (j & 1), (j / 2) & 1, a.error_word, 41);
     }
@@ -635,8 +654,8 @@ bwd_dkdv_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
         }
         const int hn = hs + kKvNB;
         if (hn < n_hs) {
-          const int j = hn / kKvNB, half = hn % kKvNB, sq = j % 3;
-          if (half == 0) ok = ok && mbar_wait(bars + B_QF + sq, (j / 3) & 1, a.error_word, 14);
+          const int j = hn / kKvNB, half = hn % kKvNB, sq = j % kQS;
+          if (half == 0) ok = ok && mbar_wait(bars + B_QF + sq, (j / kQS) & 1, a.error_word, 14);
           if (ok) {
             tc_fence_after();
             const uint32_t b_lo = q_lo + sq * (kTile >> 4) + half * kHalfRows;
@@ -667,7 +686,7 @@ bwd_dkdv_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
 #pragma unroll 1
       for (int hs = -kKvNB; hs < n_hs; ++hs) {   // the first kKvNB rounds only issue dP^T
         if (hs >= 0) {
-          const int j = hs / kKvNB, half = hs % kKvNB, sq = j % 3;
+          const int j = hs / kKvNB, half = hs % kKvNB, sq = j % kQS;
           ok = ok && mbar_wait(bars + B_DSF + half, j & 1, a.error_word, 15);
           if (ok) {
             tc_fence_after();
@@ -701,6 +720,36 @@ bwd_dkdv_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
       }
       if (lead) { mma_commit(bars + B_DONE); mma_commit(bars + B_DRAIN + 1); }
       mbar_wait(bars + B_DRAIN + 1, 0, a.error_word, 7);
+    }
+  } else if (kSpill && warp == kKvMmaWarpB + 1) {
+    // ------------------------------ store warp: dS^T tiles -> global memory (kSpill) ----------
+    // The element-wise warps leave dS^T of every half-step in shared memory as well; this thread sends the
+    // tile on its way and tells them when its buffer may be written again.  Items = (query head g of the
+    // group, entry e) in schedule order; one tile of 64 queries per half-step.
+    if (lane == 0) {
+      uint64_t evict_first;
+      // (written once, read once by the dQ pass: marked evict-first so that the stream does not push the
+      // Q / dO tiles, which every kv tile of a window re-reads, out of the L2)
+      asm volatile("createpolicy.fractional.L2::evict_first.b64 %0, 1.0;" : "=l"(evict_first));
+      bool ok = true;
+      for (int hs = 0; hs < n_hs && ok; ++hs) {
+        const int j = hs / kKvNB, half = hs % kKvNB;
+        ok = mbar_wait(bars + B_DSS + half, j & 1, a.error_word, 43);
+        if (!ok) break;
+        const int item = (BS == 128) ? j : hs;
+        const int g = item / n_ent, e = item - g * n_ent;
+        const int64_t tile_idx = ((static_cast<int64_t>(b) * a.Hq + hk * a.G + g) * a.ds_nnz + a.tile_off[tile] + e) *
+                                     (BS / 64) + (BS == 128 ? half : 0);
+        asm volatile("cp.async.bulk.tensor.2d.global.shared::cta.bulk_group.L2::cache_hint [%0, {%2, %3}], [%1], %4;" ::"l"(
+                         reinterpret_cast<uint64_t>(&tm_ds)), "r"(smem_u32(sDS + half * SM::kDs)), "r"(0),
+                     "r"(static_cast<int>(tile_idx * 128)), "l"(evict_first) : "memory");
+        asm volatile("cp.async.bulk.commit_group;" ::: "memory");
+        if (hs >= 1) {   // the tile of the half-step before this one has been read out of its buffer
+          asm volatile("cp.async.bulk.wait_group.read 1;" ::: "memory");
+          mbar_arrive(bars + B_DSE + ((hs - 1) & 1));
+        }
+      }
+      asm volatile("cp.async.bulk.wait_group 0;" ::: "memory");   // my stores have left shared memory and landed
     }
   } else {
     // ------------------------------ element-wise warps ------------------------------------
@@ -798,6 +847,25 @@ bwd_dkdv_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
         }
       }
       if constexpr (C == 16) tmem_st8(dp_addr, dsreg); else tmem_st16(dp_addr, dsreg);                               // dS^T over my own dP^T columns
+      if constexpr (kSpill) {
+        static_assert(!kSpill || (C == 16 && kKvNB == 2), "the spilled tile is laid out for half-steps of 64 queries");
+        // ... and into this half's tile in shared memory: my 16 queries are two 16-byte chunks of my key's
+        // 128-byte row (128-byte swizzle, the layout the stored tensor map expects).  The tile is free once
+        // the store of the half-step two before this one has read it.
+        if (j >= 1) {
+          ok = mbar_wait(bars + B_DSE + half, (j - 1) & 1, a.error_word, 42);
+          ok = __all_sync(0xffffffffu, ok);
+          if (!ok) break;
+        }
+        const uint32_t base = smem_u32(sDS) + half * SM::kDs + r * 128;
+        asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(base + (((2 * g) ^ (r & 7)) << 4)), "r"(dsreg[0]),
+                     "r"(dsreg[1]), "r"(dsreg[2]), "r"(dsreg[3]) : "memory");
+        asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(base + (((2 * g + 1) ^ (r & 7)) << 4)), "r"(dsreg[4]),
+                     "r"(dsreg[5]), "r"(dsreg[6]), "r"(dsreg[7]) : "memory");
+        fence_proxy_async_smem();
+        __syncwarp();
+        if (lane == 0) mbar_arrive(bars + B_DSS + half);
+      }
       ew_publish(bars + B_DSF + half);
       if (closes_step(hs)) {   // this warp is done with the statistics of step j
         __syncwarp();
@@ -832,6 +900,165 @@ bwd_dkdv_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
   tc_fence_before();
   __syncthreads();
   if (warp == kKvMmaWarpA) tmem_dealloc(tmem, 512);
+}
+
+// ============================== dQ from the kept dS ===========================================
+// dQ(128 queries x D) = scale * sum over the active key blocks of dS(128 queries x 128 keys) K(128 keys x D),
+// with dS^T read back from the tiles the dK/dV pass left in global memory (two tiles of 64 queries per
+// step): one product per step, no exponentials, nothing recomputed.  The kernel is a plain pipelined
+// contraction -- warp 4 loads (three stages of dS^T + K), warp 5 issues, warps 0-3 write the result --
+// and is bound by the HBM reads of dS.  128-token blocks only.
+template <int D>
+struct DqDsSmem {
+  static constexpr int kTile = BwdTile<D>::kBytes;
+  static constexpr int kDs2 = 2 * 128 * 128;                   // dS^T of a step: two tiles of [128 keys][64 queries]
+  static constexpr int kStages = 3;
+  static constexpr int oA = 0;
+  static constexpr int oK = kStages * kDs2;
+  static constexpr int oBar = oK + kStages * kTile;
+  static constexpr int kTotal = oBar + 512;
+};
+constexpr int kDq2Threads = 6 * 32;
+
+template <int D>
+__global__ void __launch_bounds__(kDq2Threads, 1)
+bwd_dq_from_ds_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__ CUtensorMap tm_ds, const BwdArgs a) {
+  using SM = DqDsSmem<D>;
+  constexpr int kSt = SM::kStages;
+  constexpr int kTile = SM::kTile;
+  enum { B_F = 0, B_E = kSt, B_DONE = 2 * kSt, B_COUNT = 2 * kSt + 1 };
+  extern __shared__ __align__(1024) uint8_t smem[];
+  uint64_t* bars = reinterpret_cast<uint64_t*>(smem + SM::oBar);
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + B_COUNT);
+  const int tid = threadIdx.x, lane = tid & 31;
+  const int warp = __shfl_sync(0xffffffffu, tid >> 5, 0);
+  if ((smem_u32(smem) & 1023u) != 0) {
+    if (tid == 0) atomicCAS(a.error_word, 0u, (2u << 24) | 80u);
+    return;
+  }
+  if (!lists_match(a.error_word, a.expect_fp, a.expect_fp2, 80u)) return;
+  unsigned int abort_word = 0;
+  if (tid == 0) abort_word = *reinterpret_cast<volatile unsigned int*>(a.error_word);
+  const int t = a.order[blockIdx.y];                       // query tile = query block (128 rows)
+  const int b = blockIdx.x / a.Hq, h = blockIdx.x % a.Hq, hk = h / a.G;
+  const int e0 = a.tile_off[t], n_ent = a.tile_off[t + 1] - e0;   // CSR row of the block
+  const int32_t* cols = a.tile_ent + e0;                    // its key blocks, ascending
+  if (tid == 0) {
+    for (int i = 0; i < kSt; ++i) { mbar_init(bars + B_F + i, 1); mbar_init(bars + B_E + i, 1); }
+    mbar_init(bars + B_DONE, 1);
+    mbar_fence_init();
+    tmem_slot[1] = abort_word;
+  }
+  if (warp == 5) {
+    tmem_alloc(tmem_slot, D);
+    tmem_relinquish();
+  }
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  const uint32_t tmem = *tmem_slot;
+  if (tmem_slot[1] != 0) {
+    if (warp == 5) tmem_dealloc(tmem, D);
+    return;
+  }
+  if (warp == 4) {
+    // ------------------------------ TMA producer ------------------------------------------
+    // Where a (query block, key block) pair sits in the key block's schedule takes a bisection of its
+    // CSC column: a chain of dependent loads.  The whole warp does 32 entries at a time, one chunk ahead
+    // of the lane that issues the copies, so that the chain is never on the critical path.
+    int32_t* sSlot = reinterpret_cast<int32_t*>(bars + B_COUNT + 1);   // [2][32] schedule positions
+    auto find_chunk = [&](int c) {
+      const int x = c * 32 + lane;
+      if (x < n_ent) {
+        const int kb = cols[x];
+        int lo = a.aux0[kb], hi = a.aux0[kb + 1];
+        const int c0 = lo;
+        while (lo < hi) {
+          const int mid = (lo + hi) >> 1;
+          if (a.aux1[mid] < t) lo = mid + 1; else hi = mid;
+        }
+        sSlot[(c & 1) * 32 + lane] = a.aux2[kb] + (lo - c0);
+      }
+    };
+    if (lane == 0) { tma_prefetch_desc(&tm_k); tma_prefetch_desc(&tm_ds); }
+    uint64_t evict_first;
+    asm volatile("createpolicy.fractional.L2::evict_first.b64 %0, 1.0;" : "=l"(evict_first));   // dS tiles are read once
+    bool ok = true;
+    int nl = 0;
+    const int n_chunks = (n_ent + 31) / 32;
+    if (n_chunks > 0) find_chunk(0);
+    __syncwarp();
+    for (int c = 0; c < n_chunks; ++c) {
+      if (c + 1 < n_chunks) find_chunk(c + 1);
+      if (lane == 0) {
+        for (int x = c * 32; x < min(n_ent, c * 32 + 32) && ok; ++x) {
+          const int kb = cols[x];
+          const int64_t tile_idx = ((static_cast<int64_t>(b) * a.Hq + h) * a.ds_nnz + sSlot[(c & 1) * 32 + (x & 31)]) * 2;
+          const int st = x % kSt;
+          if (x >= kSt) ok = mbar_wait(bars + B_E + st, ((x / kSt) - 1) & 1, a.error_word, 81);
+          if (!ok) break;
+          mbar_expect_tx(bars + B_F + st, SM::kDs2 + kTile);
+          uint8_t* dA = smem + SM::oA + st * SM::kDs2;
+#pragma unroll
+          for (int half = 0; half < 2; ++half)
+            asm volatile(
+                "cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes.L2::cache_hint [%0], [%1, {%3, %4}], [%2], %5;" ::"r"(
+                    smem_u32(dA + half * (SM::kDs2 / 2))),
+                "l"(reinterpret_cast<uint64_t>(&tm_ds)), "r"(smem_u32(bars + B_F + st)), "r"(0),
+                "r"(static_cast<int>((tile_idx + half) * 128)), "l"(evict_first)
+                : "memory");
+          tma_load_rows<D, 128>(smem + SM::oK + st * kTile, &tm_k, bars + B_F + st, 0, kb * 128, hk, b);
+          nl = x + 1;
+        }
+      }
+      ok = __all_sync(0xffffffffu, ok);
+      if (!ok) break;
+    }
+    if (lane == 0)
+      for (int x = max(nl - kSt, 0); x < nl; ++x) mbar_wait(bars + B_F + x % kSt, (x / kSt) & 1, a.error_word, 82);
+  } else if (warp == 5) {
+    // ------------------------------ MMA issuer ---------------------------------------------
+    const bool lead = elect_one();
+    constexpr uint32_t idesc = make_idesc_bf16(128, D, 1, 1);   // A = dS^T and B = K, both MN-major
+    const uint32_t hi = desc_hi(1024);
+    const uint32_t a_lo0 = desc_lo(smem_u32(smem + SM::oA), SM::kDs2 / 2), k_lo0 = desc_lo(smem_u32(smem + SM::oK), BwdTile<D>::kBox);
+    bool ok = true;
+#pragma unroll 1
+    for (int x = 0; x < n_ent; ++x) {
+      const int st = x % kSt;
+      ok = ok && mbar_wait(bars + B_F + st, (x / kSt) & 1, a.error_word, 83);
+      if (ok) {
+        tc_fence_after();
+        const uint32_t a_lo = a_lo0 + st * (SM::kDs2 >> 4), b_lo = k_lo0 + st * (kTile >> 4);
+#pragma unroll
+        for (int kk = 0; kk < 8; ++kk)
+          if (lead) mma_ss2(tmem, a_lo + kk * (2048 >> 4), b_lo + kk * (2048 >> 4), hi, idesc, (x > 0) || (kk > 0));
+      }
+      if (lead) mma_commit(bars + B_E + st);
+    }
+    if (lead) mma_commit(bars + B_DONE);
+    mbar_wait(bars + B_DONE, 0, a.error_word, 84);           // nothing of mine is still running at exit
+  } else {
+    // ------------------------------ epilogue: dQ * scale -> bf16 ----------------------------
+    const int r = warp * 32 + lane;
+    const int qi = t * 128 + r;
+    bool ok = true;
+    if (n_ent > 0) ok = mbar_wait_warp(bars + B_DONE, 0, a.error_word, 85);
+    if (ok) {
+      tc_fence_after();
+      const uint32_t lane_addr = tmem + (static_cast<uint32_t>(warp * 32) << 16);
+      __nv_bfloat16* dq_row = a.out0 + b * a.s0[0] + h * a.s0[1] + static_cast<int64_t>(qi) * a.s0[2];
+      if (n_ent > 0) {
+        store_acc_cols<D>(lane_addr, dq_row, a.scale, qi < a.L);
+      } else if (qi < a.L) {
+#pragma unroll
+        for (int x = 0; x < D; x += 8) *reinterpret_cast<uint4*>(dq_row + x) = make_uint4(0, 0, 0, 0);
+      }
+    }
+  }
+  tc_fence_before();
+  __syncthreads();
+  if (warp == 5) tmem_dealloc(tmem, D);
 }
 
 }  // namespace lg

@@ -64,6 +64,7 @@ struct WsLayout {
   // position, the ticket + arrival counters (cleared at every call), and dQ in fp32
   size_t kt_rank, kt_tile_of, kt_pos, sem, dq_acc;
   size_t sem_bytes;
+  size_t ds_buf;                                 // backward that keeps dS only: the dS^T tiles (0 otherwise)
   size_t total;
 };
 WsLayout ws_layout(const Resolved& r, bool want_bwd);
@@ -80,8 +81,18 @@ lg_status prepare_workspace(const Resolved& r, const WsLayout& w, uint8_t* ws, i
 lg_status make_tmap(CUtensorMap* out, const void* base, int B, int H, int L, int D, const int64_t strides[3],
                     int box_rows);
 
-// Which backward runs for this problem: the single sweep (lg_bwd_fused.cuh) or the two passes (lg_bwd.cuh).
-bool bwd_is_fused(const Resolved& r);
+// Which backward runs for this problem.
+enum BwdVariant {
+  kBwdTwoPass = 0,   // dK/dV pass, then a dQ pass that recomputes S and dP (lg_bwd.cuh)
+  kBwdFused = 1,     // one sweep; the parts of dQ are added in a fixed order through counters (lg_bwd_fused.cuh)
+  kBwdKeepDs = 2     // dK/dV pass that also writes dS^T to the workspace, then dQ = dS K (lg_bwd.cuh)
+};
+BwdVariant bwd_variant(const Resolved& r);
+inline bool bwd_is_fused(const Resolved& r) { return bwd_variant(r) == kBwdFused; }
+// bytes of the dS^T buffer of the kBwdKeepDs variant
+size_t ds_buffer_bytes(const Resolved& r);
+
+lg_status make_tmap_ds(CUtensorMap* out, const void* base, int64_t rows);
 
 lg_status check_arch();
 inline bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15) == 0; }

@@ -96,11 +96,12 @@ def test_block_index_bit_exact(lg, cfg):
         assert np.array_equal(g.cpu().numpy(), r), name
 
 
-@pytest.mark.parametrize("variant", ["fused", "two_pass"])
+@pytest.mark.parametrize("variant", ["fused", "two_pass", "keep_ds"])
 @pytest.mark.parametrize("cfg", SMALL, ids=lambda c: c.name)
 def test_fwd_bwd_parity_small(lg, cfg, variant, monkeypatch):
-    """Both backward variants (the single sweep that adds the parts of dQ in a fixed order, and the two
-    passes) on every small pattern; with D = 64 both names run the two passes."""
+    """The backward variants (the two passes; the dK/dV pass that keeps dS for a one-product dQ pass; the
+    single sweep that adds the parts of dQ in a fixed order) on every small pattern.  Where a variant does
+    not apply (keeping dS needs 128-token blocks, the single sweep D = 128) the name runs the two passes."""
     monkeypatch.setenv("LG_BWD_VARIANT", variant)
     p = lg.params_of(cfg)
     inp = synth.make_attn_inputs(cfg, "cuda", seed=0, with_do=True)
@@ -121,7 +122,7 @@ def test_fwd_bwd_parity_small(lg, cfg, variant, monkeypatch):
         _assert_close(synth.to_f64(dv[b]), dV, TOL_G, "dV")
 
 
-@pytest.mark.parametrize("variant", ["fused", "two_pass"])
+@pytest.mark.parametrize("variant", ["fused", "two_pass", "keep_ds"])
 @pytest.mark.parametrize("cfg", [SMALL[5], replace(synth.CFG1, name="rep_window", L=8192, D=128, Hq=8, Hkv=4, block=128,
                                                    sink_tokens=128, window_tokens=1024)], ids=lambda c: c.name)
 def test_bitwise_reproducible(lg, cfg, variant, monkeypatch):
