@@ -243,6 +243,7 @@ def bench_attn(lg, cfg, warmup, steps, want_bwd, profile_kernels=False):
                                               dv=dv, workspace=ws)
         out["bwd_ms"] = time_cuda(f_bwd, warmup, steps)
         out["bwd_tflops"] = flops(cfg, False, True) / out["bwd_ms"] / 1e9
+        out["bwd_variant"] = lg.bwd_variant_name(p)
         out["fwd_bwd_ms"] = out["fwd_ms"] + out["bwd_ms"]
         out["fwd_bwd_tflops"] = flops(cfg) / out["fwd_bwd_ms"] / 1e9
         if profile_kernels:
@@ -422,7 +423,8 @@ def main():
                 "peak_source": "%s sustained bf16 matmul" % peaks["source"],
                 "frac_of_nominal_2250": achieved / NOMINAL_BF16_TFLOPS,
                 "kernel_ms": kernel_ms,
-                "note": "algorithmic FLOPs per launch: fwd 4D, dK/dV pass 8D, dQ pass 2D per visible pair"}
+                "note": "algorithmic FLOPs per launch: fwd 4D, dK/dV pass 8D, dQ pass 2D per visible pair (the dQ pass of "
+                        "the keep_ds variant is one product that reads dS back from HBM: it is bandwidth-bound)"}
 
     mhz = clk.get("sm_mhz")
     line = {"metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
@@ -431,6 +433,7 @@ def main():
             "config": {"workload": cfg.name, "B": cfg.B, "Hq": cfg.Hq, "Hkv": cfg.Hkv, "L": cfg.L, "D": cfg.D,
                        "block": cfg.block, "sink_tokens": cfg.sink_tokens, "window_tokens": cfg.window_tokens,
                        "useful_flop_per_step": flops(cfg), "parallelism": "replicas x%d" % world,
+                       "bwd_variant": lg.bwd_variant_name(p),
                        "l2": "inputs (8.6 GB) far larger than L2; no flush",
                        "lists": "block lists and tile schedules built once before the timed region "
                                 "(lg_sparse_attn_prepare, %.3f ms); a step = forward + backward kernels" % index_ms},

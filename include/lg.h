@@ -145,6 +145,16 @@ lg_status lg_sparse_attn_bwd(const lg_attn_params* p, const void* q, const void*
                              void* dq, void* dk, void* dv,
                              void* workspace, size_t workspace_bytes, void* stream);
 
+/* Which of its two equivalent backward variants lg_sparse_attn_bwd runs for `p` (the workspace size
+ * reflects the choice): 0 = two passes, the dQ pass recomputing S and dP; 2 = the dK/dV pass also
+ * writes dS (bf16, 2 bytes per visible pair and query head) to the workspace and the dQ pass is the
+ * single product dQ = dS K.  The second is chosen for 128-token blocks when that buffer takes at most
+ * 48 GB (environment: LG_KEEP_DS_MAX_GB) and the block lists are shared by the batch; the environment
+ * variable LG_BWD_VARIANT = two_pass | keep_ds overrides the choice.  Both give bitwise reproducible
+ * results; they differ from one another in the last bits (dS is rounded to bf16 once either way, but the
+ * order of the fp32 sums differs).  < 0 = lg_status.  (The paper has no counterpart.)            */
+int32_t lg_sparse_attn_bwd_variant(const lg_attn_params* p);
+
 /* Same computation as lg_sparse_attn_bwd; in addition the CUDA events of the caller are recorded on
  * `stream` around its kernels: events[0] before the first one, events[1] after the pre-pass
  * (delta), events[2] after the dK/dV pass, events[3] after the dQ pass.  `events` is a HOST array

@@ -56,6 +56,7 @@ SYMBOLS = {
     "lg_build_block_index": (C.c_int, [C.POINTER(AttnParams), _vp, _vp, _vp, _vp, C.POINTER(C.c_int64), _vp]),
     "lg_sparse_attn_workspace_bytes": (_sz, [C.POINTER(AttnParams), C.c_int]),
     "lg_sparse_attn_prepare": (C.c_int, [C.POINTER(AttnParams), _vp, _sz, C.c_int, _vp]),
+    "lg_sparse_attn_bwd_variant": (C.c_int32, [C.POINTER(AttnParams)]),
     "lg_sparse_attn_fwd": (C.c_int, [C.POINTER(AttnParams), _vp, _vp, _vp, _vp, _vp, _vp, _sz, _vp]),
     "lg_sparse_attn_bwd": (C.c_int, [C.POINTER(AttnParams)] + [_vp] * 9 + [_vp, _sz, _vp]),
     "lg_sparse_attn_bwd_marked": (C.c_int, [C.POINTER(AttnParams)] + [_vp] * 9 + [_vp, _sz, _vp, C.POINTER(_vp)]),
@@ -176,6 +177,14 @@ def lg_sparse_attn_prepare(p: AttnParams, workspace: torch.Tensor, want_bwd: boo
                                                  _stream()), "lg_sparse_attn_prepare")
     p.lists_prepared = 1
     return p
+
+
+def bwd_variant_name(p: AttnParams) -> str:
+    """Which backward variant lg_sparse_attn_bwd runs for these parameters."""
+    v = load_library().lg_sparse_attn_bwd_variant(C.byref(p))
+    if v < 0:
+        raise LgError(int(v), "lg_sparse_attn_bwd_variant")
+    return {0: "two_pass", 2: "keep_ds"}[int(v)]
 
 
 def lg_sparse_attn_fwd(p: AttnParams, q, k, v, o=None, lse=None, workspace=None):

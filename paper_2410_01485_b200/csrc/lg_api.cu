@@ -113,29 +113,27 @@ lg_status resolve(const lg_attn_params* p, Resolved* r) {
   return LG_OK;
 }
 
-// Three backward variants compute the same gradients (see BwdVariant).  The two passes run everywhere.
+// Two backward variants compute the same gradients (see BwdVariant).  The two passes run everywhere.
 // Keeping dS trades workspace and HBM traffic (2 bytes per visible pair, written once and read once, on
 // a memory system the attention kernels otherwise leave idle) for the two recomputed products of the dQ
-// pass; it is the default where it applies: 128-token blocks, no per-sequence lists, and a dS buffer of
-// at most LG_KEEP_DS_MAX_GB (default 48) gigabytes.  The single sweep needs D = 128 and is only chosen
-// explicitly: its ordered fp32 additions into dQ cost more than the recomputation they save.
-// LG_BWD_VARIANT = two_pass | keep_ds | fused overrides the choice (read at every call; it must not
-// change between a size query, a prepare and the calls that use them).
-size_t ds_buffer_bytes(const Resolved& r) {
-  return static_cast<size_t>(r.B) * r.Hq * static_cast<size_t>(r.nnz) * (r.block / 64) * (128 * 128);
+// pass.  It is the default for 128-token blocks (with 64-token blocks the two variants were measured
+// equal) when the lists are shared by the batch and the dS buffer takes at most LG_KEEP_DS_MAX_GB
+// (default 48) gigabytes.  LG_BWD_VARIANT = two_pass | keep_ds overrides the choice (read at every call;
+// it must not change between a size query, a prepare and the calls that use them).
+size_t ds_buffer_bytes(const Resolved& r) {   // every tile of 64 queries x 128 keys, plus one tile of zeros at the end
+  return (static_cast<size_t>(r.B) * r.Hq * static_cast<size_t>(r.nnz) * (r.block / 64) + 1) * (128 * 128);
 }
 
 BwdVariant bwd_variant(const Resolved& r) {
   const char* env = getenv("LG_BWD_VARIANT");
   if (env && strcmp(env, "two_pass") == 0) return kBwdTwoPass;
-  if (env && strcmp(env, "fused") == 0) return r.D == 128 ? kBwdFused : kBwdTwoPass;
   // the stored tiles are addressed by 32-bit row coordinates of a tensor map
-  const bool can_keep = r.block == 128 && !(r.doc_start != nullptr && r.B > 1) &&
-                        ds_buffer_bytes(r) / 128 < (1ull << 31);
+  const bool can_keep = !(r.doc_start != nullptr && r.B > 1) && ds_buffer_bytes(r) / 128 < (1ull << 31);
   if (env && strcmp(env, "keep_ds") == 0) return can_keep ? kBwdKeepDs : kBwdTwoPass;
   double max_gb = 48.0;
   if (const char* m = getenv("LG_KEEP_DS_MAX_GB")) max_gb = atof(m);
-  return (can_keep && static_cast<double>(ds_buffer_bytes(r)) <= max_gb * 1e9) ? kBwdKeepDs : kBwdTwoPass;
+  return (can_keep && r.block == 128 && static_cast<double>(ds_buffer_bytes(r)) <= max_gb * 1e9) ? kBwdKeepDs
+                                                                                                  : kBwdTwoPass;
 }
 
 WsLayout ws_layout(const Resolved& r, bool want_bwd) {
@@ -165,16 +163,12 @@ WsLayout ws_layout(const Resolved& r, bool want_bwd) {
     w.kt_off = take((static_cast<size_t>(r.n_ktiles) + 1) * 4);
     if (r.doc_start) w.doc_end = take(static_cast<size_t>(r.B) * r.L * 4);
     w.delta = take(static_cast<size_t>(r.B) * r.Hq * align_up(r.L, 128) * 8);   // rows padded to whole tiles   // two planes: -LSE * log2 e and -delta per query row
-    if (bwd_is_fused(r)) {
-      const size_t Lp = align_up(r.L, 128);
-      w.kt_rank = take(nnz * 4);
+    if (bwd_variant(r) == kBwdKeepDs) {
       w.kt_tile_of = take(nB * 4);
-      w.kt_pos = take(static_cast<size_t>(r.n_ktiles) * 4);
-      w.sem_bytes = (64 + static_cast<size_t>(r.B) * r.Hq * (Lp / 64) * 4) * 4;   // ticket + four counters per (head, 64-row group)
-      w.sem = take(w.sem_bytes);
-      w.dq_acc = take(static_cast<size_t>(r.B) * r.Hq * Lp * r.D * 4);
+      w.dq_cnt = take(static_cast<size_t>(r.n_qtiles) * 4);
+      w.dq_ent = take(nnz * 3 * 4);
+      w.ds_buf = take(ds_buffer_bytes(r));
     }
-    if (bwd_variant(r) == kBwdKeepDs) w.ds_buf = take(ds_buffer_bytes(r));
   }
   w.total = off;
   return w;
@@ -245,12 +239,11 @@ lg_status prepare_workspace(const Resolved& r, const WsLayout& w, uint8_t* ws, i
     kv_tile_merge_kernel<<<(nt + 127) / 128, 128, 0, stream>>>(i32(w.col_ptr), i32(w.row_idx), i32(w.kt_cols),
                                                                i32(w.kt_off), R, nt, i32(w.kt_cnt), i32(w.kt_ent)); note_launch();
     tile_order_kernel<<<(nt + 127) / 128, 128, 0, stream>>>(i32(w.kt_cnt), nt, i32(w.kt_order)); note_launch();
-    if (bwd_is_fused(r)) {   // order of the dQ parts: rank of every (kv tile, query block) entry
+    if (bwd_variant(r) == kBwdKeepDs) {   // which dS tiles each query tile reads back
       kv_tile_of_kernel<<<(nt * R + 127) / 128, 128, 0, stream>>>(i32(w.kt_cols), R, nt, i32(w.kt_tile_of)); note_launch();
-      tile_pos_kernel<<<(nt + 127) / 128, 128, 0, stream>>>(i32(w.kt_order), nt, i32(w.kt_pos)); note_launch();
-      kv_tile_rank_kernel<<<nt, 128, 0, stream>>>(i32(w.row_ptr), i32(w.col_idx), i32(w.kt_tile_of), i32(w.kt_pos),
-                                                  i32(w.kt_cols), i32(w.kt_off), i32(w.kt_cnt), i32(w.kt_ent), R,
-                                                  i32(w.kt_rank)); note_launch();
+      dq_sched_kernel<<<(r.n_qtiles + 63) / 64, 64, 0, stream>>>(i32(w.row_ptr), i32(w.col_idx), i32(w.kt_tile_of),
+                                                                  i32(w.kt_off), i32(w.kt_cnt), i32(w.kt_ent), R, nB,
+                                                                  r.n_qtiles, i32(w.dq_cnt), i32(w.dq_ent)); note_launch();
     }
     if (r.doc_start) {
       const int64_t n = static_cast<int64_t>(r.B) * r.L;
@@ -474,6 +467,12 @@ size_t lg_sparse_attn_workspace_bytes(const lg_attn_params* p, int want_bwd) {
   Resolved r;
   if (resolve(p, &r) != LG_OK) return 0;
   return attn_workspace_total(r, want_bwd != 0);
+}
+
+int32_t lg_sparse_attn_bwd_variant(const lg_attn_params* p) {
+  Resolved r;
+  lg_status s = resolve(p, &r);
+  return s == LG_OK ? static_cast<int32_t>(bwd_variant(r)) : static_cast<int32_t>(s);
 }
 
 lg_status lg_sparse_attn_prepare(const lg_attn_params* p, void* workspace, size_t workspace_bytes, int want_bwd,

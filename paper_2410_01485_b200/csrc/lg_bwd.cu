@@ -1,5 +1,5 @@
 // Launch of the backward attention kernels: delta pre-pass, dK/dV pass, dQ pass.
-#include "lg_bwd_fused.cuh"
+#include "lg_bwd.cuh"
 #include "lg_host.h"
 
 namespace lg {
@@ -35,50 +35,8 @@ static lg_status launch_bwd_t(const Resolved& r, const WsLayout& w, const void* 
   a.scale = r.scale;
   a.scale_log2 = r.scale * 1.4426950408889634f;
   a.ds_nnz = r.nnz;
-  a.aux0 = a.aux1 = a.aux2 = nullptr;
   constexpr int smem = BwdSmem<D, BS>::kTotal;
   const BwdVariant variant = bwd_variant(r);
-
-  if constexpr (D == 128) {
-    if (bwd_is_fused(r)) {
-      // ---- single sweep: dK, dV and the parts of dQ, then dQ -> bf16 -----------------------
-      CUtensorMap tq, tk, tv, tdo;
-      if ((s = make_tmap(&tq, q, r.B, r.Hq, r.L, D, r.qs, BS)) != LG_OK) return s;
-      if ((s = make_tmap(&tdo, d_o, r.B, r.Hq, r.L, D, r.os, BS)) != LG_OK) return s;
-      if ((s = make_tmap(&tk, k, r.B, r.Hkv, r.L, D, r.ks, BS)) != LG_OK) return s;
-      if ((s = make_tmap(&tv, v, r.B, r.Hkv, r.L, D, r.vs, BS)) != LG_OK) return s;
-      a.tile_off = reinterpret_cast<const int32_t*>(ws + w.kt_off);
-      a.tile_cols = reinterpret_cast<const int32_t*>(ws + w.kt_cols);
-      a.tile_cnt = reinterpret_cast<const int32_t*>(ws + w.kt_cnt);
-      a.tile_ent = reinterpret_cast<const int32_t*>(ws + w.kt_ent);
-      a.order = reinterpret_cast<const int32_t*>(ws + w.kt_order);
-      a.out0 = static_cast<__nv_bfloat16*>(dk);
-      a.out1 = static_cast<__nv_bfloat16*>(dv);
-      for (int i = 0; i < 3; ++i) { a.s0[i] = r.ks[i]; a.s1[i] = r.vs[i]; }
-      FusedArgs fa;
-      fa.b = a;
-      fa.tile_rank = reinterpret_cast<const int32_t*>(ws + w.kt_rank);
-      fa.dq_acc = reinterpret_cast<float*>(ws + w.dq_acc);
-      fa.sem = reinterpret_cast<unsigned int*>(ws + w.sem);
-      fa.n64 = a.Lp / 64;
-      fa.n_tiles = r.n_ktiles;
-      // the ticket and the arrival counters start every call at zero (a memset node, not a kernel)
-      if (cudaMemsetAsync(ws + w.sem, 0, w.sem_bytes, stream) != cudaSuccess) return LG_ERR_CUDA;
-      auto kern = bwd_fused_kernel<D, BS>;
-      constexpr int fsmem = FusedSmem<D, BS>::kTotal;
-      if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, fsmem) != cudaSuccess)
-        return LG_ERR_CUDA;
-      dim3 grid(r.B * r.Hkv, r.n_ktiles);
-      kern<<<grid, kFuThreads, fsmem, stream>>>(tq, tk, tv, tdo, fa); note_launch();
-      if (marks) cudaEventRecord(marks[2], stream);
-      const int64_t n_rows = static_cast<int64_t>(r.B) * r.Hq * r.L;
-      const int64_t threads = n_rows * (D / 8);
-      dq_convert_kernel<D><<<static_cast<unsigned>((threads + 255) / 256), 256, 0, stream>>>(
-          fa.dq_acc, static_cast<__nv_bfloat16*>(dq), r.qs[0], r.qs[1], r.qs[2], r.Hq, r.L, a.Lp, n_rows, r.scale); note_launch();
-      if (marks) cudaEventRecord(marks[3], stream);
-      return cudaGetLastError() == cudaSuccess ? LG_OK : LG_ERR_CUDA;
-    }
-  }
 
   // ---- dK / dV pass -------------------------------------------------------------------
   {
@@ -97,6 +55,8 @@ static lg_status launch_bwd_t(const Resolved& r, const WsLayout& w, const void* 
     for (int i = 0; i < 3; ++i) { a.s0[i] = r.ks[i]; a.s1[i] = r.vs[i]; }
     dim3 grid(r.B * r.Hkv, r.n_ktiles);
     if (variant == kBwdKeepDs) {
+      // the tile of zeros that stands in for a half of a query tile a kv tile has no entry for
+      if (cudaMemsetAsync(ws + w.ds_buf + ds_buffer_bytes(r) - 128 * 128, 0, 128 * 128, stream) != cudaSuccess) return LG_ERR_CUDA;
       CUtensorMap tds;
       if ((s = make_tmap_ds(&tds, ws + w.ds_buf, static_cast<int64_t>(ds_buffer_bytes(r) / 128))) != LG_OK) return s;
       auto kern = bwd_dkdv_kernel<D, BS, true>;
@@ -112,32 +72,27 @@ static lg_status launch_bwd_t(const Resolved& r, const WsLayout& w, const void* 
     }
     if (marks) cudaEventRecord(marks[2], stream);
   }
-  if constexpr (BS == 128) {
-    if (variant == kBwdKeepDs) {
-      // ---- dQ = scale * dS K from the kept tiles ------------------------------------------
-      CUtensorMap tk, tds;
-      if ((s = make_tmap(&tk, k, r.B, r.Hkv, r.L, D, r.ks, 128)) != LG_OK) return s;
-      if ((s = make_tmap_ds(&tds, ws + w.ds_buf, static_cast<int64_t>(ds_buffer_bytes(r) / 128))) != LG_OK) return s;
-      a.tile_off = reinterpret_cast<const int32_t*>(ws + w.row_ptr);
-      a.tile_ent = reinterpret_cast<const int32_t*>(ws + w.col_idx);
-      a.tile_cols = nullptr;
-      a.tile_cnt = nullptr;
-      a.order = reinterpret_cast<const int32_t*>(ws + w.qt_order);
-      a.aux0 = reinterpret_cast<const int32_t*>(ws + w.col_ptr);
-      a.aux1 = reinterpret_cast<const int32_t*>(ws + w.row_idx);
-      a.aux2 = reinterpret_cast<const int32_t*>(ws + w.kt_off);
-      a.out0 = static_cast<__nv_bfloat16*>(dq);
-      a.out1 = nullptr;
-      for (int i = 0; i < 3; ++i) { a.s0[i] = r.qs[i]; a.s1[i] = 0; }
-      auto kern = bwd_dq_from_ds_kernel<D>;
-      constexpr int smem_q = DqDsSmem<D>::kTotal;
-      if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, smem_q) != cudaSuccess)
-        return LG_ERR_CUDA;
-      dim3 grid(r.B * r.Hq, r.n_qtiles);
-      kern<<<grid, kDq2Threads, smem_q, stream>>>(tk, tds, a); note_launch();
-      if (marks) cudaEventRecord(marks[3], stream);
-      return cudaGetLastError() == cudaSuccess ? LG_OK : LG_ERR_CUDA;
-    }
+  if (variant == kBwdKeepDs) {
+    // ---- dQ = scale * dS K from the kept tiles --------------------------------------------
+    CUtensorMap tk, tds;
+    if ((s = make_tmap(&tk, k, r.B, r.Hkv, r.L, D, r.ks, BS)) != LG_OK) return s;
+    if ((s = make_tmap_ds(&tds, ws + w.ds_buf, static_cast<int64_t>(ds_buffer_bytes(r) / 128))) != LG_OK) return s;
+    a.tile_off = reinterpret_cast<const int32_t*>(ws + w.row_ptr);
+    a.tile_ent = reinterpret_cast<const int32_t*>(ws + w.dq_ent);
+    a.tile_cols = reinterpret_cast<const int32_t*>(ws + w.kt_cols);
+    a.tile_cnt = reinterpret_cast<const int32_t*>(ws + w.dq_cnt);
+    a.order = reinterpret_cast<const int32_t*>(ws + w.qt_order);
+    a.out0 = static_cast<__nv_bfloat16*>(dq);
+    a.out1 = nullptr;
+    for (int i = 0; i < 3; ++i) { a.s0[i] = r.qs[i]; a.s1[i] = 0; }
+    auto kern = bwd_dq_from_ds_kernel<D, BS>;
+    constexpr int smem_q = DqDsSmem<D>::kTotal;
+    if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, smem_q) != cudaSuccess)
+      return LG_ERR_CUDA;
+    dim3 grid(r.B * r.Hq, r.n_qtiles);
+    kern<<<grid, kDq2Threads, smem_q, stream>>>(tk, tds, a); note_launch();
+    if (marks) cudaEventRecord(marks[3], stream);
+    return cudaGetLastError() == cudaSuccess ? LG_OK : LG_ERR_CUDA;
   }
   // ---- dQ pass ------------------------------------------------------------------------
   {

@@ -56,9 +56,6 @@ struct BwdArgs {
   // ds_buf as a tile of [128 keys][64 queries] bf16; tile index = ((b * Hq + h) * ds_nnz + schedule
   // position of the (kv tile, query block) entry) * (block / 64) + half.  The dQ pass then reads them back.
   int64_t ds_nnz;
-  const int32_t* aux0;       // dQ-from-dS pass: col_ptr (CSC)        } to find where a (query block, key block)
-  const int32_t* aux1;       //                  row_idx (CSC)        } pair sits in its kv tile's schedule
-  const int32_t* aux2;       //                  start of each kv tile's schedule
 };
 
 // ---- stat = -(LSE * log2 e) and -rowsum(dO * O), stored negated (they are only ever subtracted),
@@ -472,9 +469,12 @@ constexpr int kKvNB = 128 / kKvHalf;                       // (half-)steps per s
 constexpr int kKvCols = kKvHalf / (kKvEwWarps / 4);        // queries of a half-step per element-wise thread
 
 // kSpill: the pass also writes dS^T (bf16) of every half-step to global memory (tm_ds: the buffer as
-// rows of 64 queries, boxes of 128 key rows, 128-byte swizzle), so that the dQ pass is one product per
-// step, dQ += dS K, instead of recomputing S and dP (bwd_dq_from_ds_kernel).  The element-wise warps put
-// dS^T into shared memory as well as tensor memory; the thread that issues dK sends the tile on its way.
+// rows of 64 queries, boxes of 128 key rows, 128-byte swizzle; in memory the tiles are plain row-major
+// [128 keys][64 queries]), so that the dQ pass is one product per step, dQ += dS K, instead of
+// recomputing S and dP (bwd_dq_from_ds_kernel).  The element-wise warps put dS^T into shared memory as
+// well as tensor memory and a store warp sends the tiles on their way with TMA.  (Storing the 32 bytes of
+// every thread straight from its registers was measured 20 % slower: 32 separate cache lines per
+// instruction keep the load/store unit busy.)
 template <int D, int BS, bool kSpill>
 __global__ void __launch_bounds__(kKvThreads + (kSpill ? 32 : 0), 1)
 bwd_dkdv_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUtensorMap tm_k,
@@ -848,7 +848,7 @@ bwd_dkdv_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
       }
       if constexpr (C == 16) tmem_st8(dp_addr, dsreg); else tmem_st16(dp_addr, dsreg);                               // dS^T over my own dP^T columns
       if constexpr (kSpill) {
-        static_assert(!kSpill || (C == 16 && kKvNB == 2), "the spilled tile is laid out for half-steps of 64 queries");
+        static_assert(!kSpill || (C == 16 && kKvNB == 2), "the kept tiles are laid out for half-steps of 64 queries");
         // ... and into this half's tile in shared memory: my 16 queries are two 16-byte chunks of my key's
         // 128-byte row (128-byte swizzle, the layout the stored tensor map expects).  The tile is free once
         // the store of the half-step two before this one has read it.
@@ -903,30 +903,34 @@ bwd_dkdv_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
 }
 
 // ============================== dQ from the kept dS ===========================================
-// dQ(128 queries x D) = scale * sum over the active key blocks of dS(128 queries x 128 keys) K(128 keys x D),
-// with dS^T read back from the tiles the dK/dV pass left in global memory (two tiles of 64 queries per
-// step): one product per step, no exponentials, nothing recomputed.  The kernel is a plain pipelined
-// contraction -- warp 4 loads (three stages of dS^T + K), warp 5 issues, warps 0-3 write the result --
-// and is bound by the HBM reads of dS.  128-token blocks only.
+// dQ(128 queries x D) = scale * sum over the kv tiles of the row of dS(128 queries x 128 keys) K(128 keys x D),
+// with dS^T read back from the tiles the dK/dV pass left in global memory (one tile of [128 keys][64
+// queries] per half of the query tile; a half without an entry in that kv tile reads the tile of zeros):
+// one product per step, no exponentials, nothing recomputed.  The kernel is a plain pipelined
+// contraction -- warp 4 loads (a ring of dS^T tile pairs and a ring of K tiles), warp 5 issues, warps
+// 0-3 write the result -- and is bound by the HBM reads of dS.
 template <int D>
 struct DqDsSmem {
   static constexpr int kTile = BwdTile<D>::kBytes;
   static constexpr int kDs2 = 2 * 128 * 128;                   // dS^T of a step: two tiles of [128 keys][64 queries]
-  static constexpr int kStages = 3;
+  static constexpr int kAStages = (D == 128) ? 4 : 5;          // dS^T comes from HBM: the deeper ring
+  static constexpr int kKStages = 3;                           // K comes from the L2
   static constexpr int oA = 0;
-  static constexpr int oK = kStages * kDs2;
-  static constexpr int oBar = oK + kStages * kTile;
-  static constexpr int kTotal = oBar + 512;
+  static constexpr int oK = kAStages * kDs2;
+  static constexpr int oBar = oK + kKStages * kTile;
+  static constexpr int kTotal = oBar + 256;
 };
 constexpr int kDq2Threads = 6 * 32;
 
-template <int D>
+template <int D, int BS>
 __global__ void __launch_bounds__(kDq2Threads, 1)
 bwd_dq_from_ds_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__ CUtensorMap tm_ds, const BwdArgs a) {
   using SM = DqDsSmem<D>;
-  constexpr int kSt = SM::kStages;
+  constexpr int kAS = SM::kAStages, kKS = SM::kKStages;
+  constexpr int R = 128 / BS;
   constexpr int kTile = SM::kTile;
-  enum { B_F = 0, B_E = kSt, B_DONE = 2 * kSt, B_COUNT = 2 * kSt + 1 };
+  enum { B_AF = 0, B_AE = kAS, B_KF = 2 * kAS, B_KE = 2 * kAS + kKS, B_DONE = 2 * kAS + 2 * kKS, B_COUNT = B_DONE + 1 };
+  static_assert(B_COUNT * 8 + 8 <= 256, "barrier area too small");
   extern __shared__ __align__(1024) uint8_t smem[];
   uint64_t* bars = reinterpret_cast<uint64_t*>(smem + SM::oBar);
   uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + B_COUNT);
@@ -939,12 +943,13 @@ bwd_dq_from_ds_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_con
   if (!lists_match(a.error_word, a.expect_fp, a.expect_fp2, 80u)) return;
   unsigned int abort_word = 0;
   if (tid == 0) abort_word = *reinterpret_cast<volatile unsigned int*>(a.error_word);
-  const int t = a.order[blockIdx.y];                       // query tile = query block (128 rows)
+  const int t = a.order[blockIdx.y];                       // query tile (128 rows)
   const int b = blockIdx.x / a.Hq, h = blockIdx.x % a.Hq, hk = h / a.G;
-  const int e0 = a.tile_off[t], n_ent = a.tile_off[t + 1] - e0;   // CSR row of the block
-  const int32_t* cols = a.tile_ent + e0;                    // its key blocks, ascending
+  const int n_ent = a.tile_cnt[t];
+  const int32_t* ent = a.tile_ent + 3 * static_cast<int64_t>(a.tile_off[R * t]);   // (kv tile, tile of half 0, tile of half 1)
   if (tid == 0) {
-    for (int i = 0; i < kSt; ++i) { mbar_init(bars + B_F + i, 1); mbar_init(bars + B_E + i, 1); }
+    for (int i = 0; i < kAS; ++i) { mbar_init(bars + B_AF + i, 1); mbar_init(bars + B_AE + i, 1); }
+    for (int i = 0; i < kKS; ++i) { mbar_init(bars + B_KF + i, 1); mbar_init(bars + B_KE + i, 1); }
     mbar_init(bars + B_DONE, 1);
     mbar_fence_init();
     tmem_slot[1] = abort_word;
@@ -963,59 +968,50 @@ bwd_dq_from_ds_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_con
   }
   if (warp == 4) {
     // ------------------------------ TMA producer ------------------------------------------
-    // Where a (query block, key block) pair sits in the key block's schedule takes a bisection of its
-    // CSC column: a chain of dependent loads.  The whole warp does 32 entries at a time, one chunk ahead
-    // of the lane that issues the copies, so that the chain is never on the critical path.
-    int32_t* sSlot = reinterpret_cast<int32_t*>(bars + B_COUNT + 1);   // [2][32] schedule positions
-    auto find_chunk = [&](int c) {
-      const int x = c * 32 + lane;
-      if (x < n_ent) {
-        const int kb = cols[x];
-        int lo = a.aux0[kb], hi = a.aux0[kb + 1];
-        const int c0 = lo;
-        while (lo < hi) {
-          const int mid = (lo + hi) >> 1;
-          if (a.aux1[mid] < t) lo = mid + 1; else hi = mid;
-        }
-        sSlot[(c & 1) * 32 + lane] = a.aux2[kb] + (lo - c0);
-      }
-    };
-    if (lane == 0) { tma_prefetch_desc(&tm_k); tma_prefetch_desc(&tm_ds); }
-    uint64_t evict_first;
-    asm volatile("createpolicy.fractional.L2::evict_first.b64 %0, 1.0;" : "=l"(evict_first));   // dS tiles are read once
-    bool ok = true;
-    int nl = 0;
-    const int n_chunks = (n_ent + 31) / 32;
-    if (n_chunks > 0) find_chunk(0);
-    __syncwarp();
-    for (int c = 0; c < n_chunks; ++c) {
-      if (c + 1 < n_chunks) find_chunk(c + 1);
-      if (lane == 0) {
-        for (int x = c * 32; x < min(n_ent, c * 32 + 32) && ok; ++x) {
-          const int kb = cols[x];
-          const int64_t tile_idx = ((static_cast<int64_t>(b) * a.Hq + h) * a.ds_nnz + sSlot[(c & 1) * 32 + (x & 31)]) * 2;
-          const int st = x % kSt;
-          if (x >= kSt) ok = mbar_wait(bars + B_E + st, ((x / kSt) - 1) & 1, a.error_word, 81);
-          if (!ok) break;
-          mbar_expect_tx(bars + B_F + st, SM::kDs2 + kTile);
-          uint8_t* dA = smem + SM::oA + st * SM::kDs2;
+    if (lane == 0) {
+      tma_prefetch_desc(&tm_k); tma_prefetch_desc(&tm_ds);
+      uint64_t evict_first;
+      asm volatile("createpolicy.fractional.L2::evict_first.b64 %0, 1.0;" : "=l"(evict_first));   // dS tiles are read once
+      const int64_t head_base = (static_cast<int64_t>(b) * a.Hq + h) * a.ds_nnz * (BS / 64);
+      const int64_t zero_tile = static_cast<int64_t>(gridDim.x) * a.ds_nnz * (BS / 64);              // the tile after the last head's
+      bool ok = true;
+      int nl = 0;
+      int e_T = n_ent > 0 ? ent[0] : 0, e_h0 = n_ent > 0 ? ent[1] : 0, e_h1 = n_ent > 0 ? ent[2] : 0;
+      for (int x = 0; x < n_ent; ++x) {
+        const int T = e_T, h0 = e_h0, h1 = e_h1;
+        if (x + 1 < n_ent) { e_T = ent[3 * x + 3]; e_h0 = ent[3 * x + 4]; e_h1 = ent[3 * x + 5]; }   // read ahead
+        const int sa = x % kAS, sk = x % kKS;
+        if (x >= kAS) ok = mbar_wait(bars + B_AE + sa, ((x / kAS) - 1) & 1, a.error_word, 81);
+        if (!ok) break;
+        mbar_expect_tx(bars + B_AF + sa, SM::kDs2);
+        uint8_t* dA = smem + SM::oA + sa * SM::kDs2;
 #pragma unroll
-          for (int half = 0; half < 2; ++half)
-            asm volatile(
-                "cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes.L2::cache_hint [%0], [%1, {%3, %4}], [%2], %5;" ::"r"(
-                    smem_u32(dA + half * (SM::kDs2 / 2))),
-                "l"(reinterpret_cast<uint64_t>(&tm_ds)), "r"(smem_u32(bars + B_F + st)), "r"(0),
-                "r"(static_cast<int>((tile_idx + half) * 128)), "l"(evict_first)
-                : "memory");
-          tma_load_rows<D, 128>(smem + SM::oK + st * kTile, &tm_k, bars + B_F + st, 0, kb * 128, hk, b);
-          nl = x + 1;
+        for (int half = 0; half < 2; ++half) {
+          const int hx = half ? h1 : h0;
+          const int64_t tile_idx = hx >= 0 ? head_base + hx : zero_tile;
+          asm volatile(
+              "cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes.L2::cache_hint [%0], [%1, {%3, %4}], [%2], %5;" ::"r"(
+                  smem_u32(dA + half * (SM::kDs2 / 2))),
+              "l"(reinterpret_cast<uint64_t>(&tm_ds)), "r"(smem_u32(bars + B_AF + sa)), "r"(0),
+              "r"(static_cast<int>(tile_idx * 128)), "l"(evict_first)
+              : "memory");
         }
+        if (x >= kKS) ok = mbar_wait(bars + B_KE + sk, ((x / kKS) - 1) & 1, a.error_word, 86);
+        if (!ok) break;
+        mbar_expect_tx(bars + B_KF + sk, kTile);
+        uint8_t* dK = smem + SM::oK + sk * kTile;
+        if (BS == 128) {
+          tma_load_rows<D, 128>(dK, &tm_k, bars + B_KF + sk, 0, T * 128, hk, b);
+        } else {   // the tile's two pattern columns need not be neighbours (a missing one: its dS rows are zero)
+          const int ca = a.tile_cols[2 * T], cb = a.tile_cols[2 * T + 1];
+          tma_load_rows<D, 64>(dK, &tm_k, bars + B_KF + sk, 0, ca * 64, hk, b);
+          tma_load_rows<D, 64>(dK, &tm_k, bars + B_KF + sk, 1, (cb >= 0 ? cb : ca) * 64, hk, b);
+        }
+        nl = x + 1;
       }
-      ok = __all_sync(0xffffffffu, ok);
-      if (!ok) break;
+      for (int x = max(nl - kAS, 0); x < nl; ++x) mbar_wait(bars + B_AF + x % kAS, (x / kAS) & 1, a.error_word, 82);
+      for (int x = max(nl - kKS, 0); x < nl; ++x) mbar_wait(bars + B_KF + x % kKS, (x / kKS) & 1, a.error_word, 87);
     }
-    if (lane == 0)
-      for (int x = max(nl - kSt, 0); x < nl; ++x) mbar_wait(bars + B_F + x % kSt, (x / kSt) & 1, a.error_word, 82);
   } else if (warp == 5) {
     // ------------------------------ MMA issuer ---------------------------------------------
     const bool lead = elect_one();
@@ -1025,16 +1021,17 @@ bwd_dq_from_ds_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_con
     bool ok = true;
 #pragma unroll 1
     for (int x = 0; x < n_ent; ++x) {
-      const int st = x % kSt;
-      ok = ok && mbar_wait(bars + B_F + st, (x / kSt) & 1, a.error_word, 83);
+      const int sa = x % kAS, sk = x % kKS;
+      ok = ok && mbar_wait(bars + B_AF + sa, (x / kAS) & 1, a.error_word, 83);
+      ok = ok && mbar_wait(bars + B_KF + sk, (x / kKS) & 1, a.error_word, 88);
       if (ok) {
         tc_fence_after();
-        const uint32_t a_lo = a_lo0 + st * (SM::kDs2 >> 4), b_lo = k_lo0 + st * (kTile >> 4);
+        const uint32_t a_lo = a_lo0 + sa * (SM::kDs2 >> 4), b_lo = k_lo0 + sk * (kTile >> 4);
 #pragma unroll
         for (int kk = 0; kk < 8; ++kk)
           if (lead) mma_ss2(tmem, a_lo + kk * (2048 >> 4), b_lo + kk * (2048 >> 4), hi, idesc, (x > 0) || (kk > 0));
       }
-      if (lead) mma_commit(bars + B_E + st);
+      if (lead) { mma_commit(bars + B_AE + sa); mma_commit(bars + B_KE + sk); }
     }
     if (lead) mma_commit(bars + B_DONE);
     mbar_wait(bars + B_DONE, 0, a.error_word, 84);           // nothing of mine is still running at exit

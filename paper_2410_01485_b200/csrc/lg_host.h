@@ -60,11 +60,8 @@ struct WsLayout {
   size_t kt_cols, kt_off;                        // members of each kv tile, start of its schedule
   size_t doc_end;                                // int32 [B, L]: end of each token's document (bwd with documents only)
   size_t delta;                                  // 2 x float [B, Hq, L]: -LSE * log2 e, then -delta (bwd only)
-  // fused backward only (0 otherwise): rank of every kv-tile schedule entry, column -> tile, tile -> launch
-  // position, the ticket + arrival counters (cleared at every call), and dQ in fp32
-  size_t kt_rank, kt_tile_of, kt_pos, sem, dq_acc;
-  size_t sem_bytes;
-  size_t ds_buf;                                 // backward that keeps dS only: the dS^T tiles (0 otherwise)
+  // backward that keeps dS only (0 otherwise): pattern column -> kv tile, the schedule of its dQ pass, the dS^T tiles
+  size_t kt_tile_of, dq_cnt, dq_ent, ds_buf;
   size_t total;
 };
 WsLayout ws_layout(const Resolved& r, bool want_bwd);
@@ -83,12 +80,10 @@ lg_status make_tmap(CUtensorMap* out, const void* base, int B, int H, int L, int
 
 // Which backward runs for this problem.
 enum BwdVariant {
-  kBwdTwoPass = 0,   // dK/dV pass, then a dQ pass that recomputes S and dP (lg_bwd.cuh)
-  kBwdFused = 1,     // one sweep; the parts of dQ are added in a fixed order through counters (lg_bwd_fused.cuh)
-  kBwdKeepDs = 2     // dK/dV pass that also writes dS^T to the workspace, then dQ = dS K (lg_bwd.cuh)
+  kBwdTwoPass = 0,   // dK/dV pass, then a dQ pass that recomputes S and dP
+  kBwdKeepDs = 2     // dK/dV pass that also writes dS^T to the workspace, then a dQ pass that is one product: dQ = dS K
 };
 BwdVariant bwd_variant(const Resolved& r);
-inline bool bwd_is_fused(const Resolved& r) { return bwd_variant(r) == kBwdFused; }
 // bytes of the dS^T buffer of the kBwdKeepDs variant
 size_t ds_buffer_bytes(const Resolved& r);
 

@@ -207,56 +207,64 @@ __global__ void kv_tile_merge_kernel(const int32_t* __restrict__ col_ptr, const 
   tile_cnt[t] = n;
 }
 
-// ---- order of the dQ contributions in the fused backward --------------------------------------
-// In the fused backward every kv tile adds its part of dQ to the rows of the query blocks it
-// visits; the parts of one query block are added in the launch order of the kv tiles that hold
-// a column of its row.  rank[e] of schedule entry e = (tile t, query block qb) is the number of
-// OTHER kv tiles with an active column in row qb that come before t in that order: the tile's
-// part is the rank-th one (0 = it initialises the rows).
-//   tile_of[kb] = kv tile of pattern column kb;  pos[t] = launch position of tile t.
+// tile_of[kb] = kv tile of pattern column kb
 __global__ void kv_tile_of_kernel(const int32_t* __restrict__ cols, int R, int n_tiles, int32_t* __restrict__ tile_of) {
   const int c = blockIdx.x * blockDim.x + threadIdx.x;
   if (c >= n_tiles * R) return;
   const int kb = cols[c];
   if (kb >= 0) tile_of[kb] = c / R;
 }
-__global__ void tile_pos_kernel(const int32_t* __restrict__ order, int n_tiles, int32_t* __restrict__ pos) {
-  const int i = blockIdx.x * blockDim.x + threadIdx.x;
-  if (i < n_tiles) pos[order[i]] = i;
-}
-// grid = kv tiles, block = 128 threads striding over the tile's entries
-__global__ void kv_tile_rank_kernel(const int32_t* __restrict__ row_ptr, const int32_t* __restrict__ col_idx,
-                                    const int32_t* __restrict__ tile_of, const int32_t* __restrict__ pos,
-                                    const int32_t* __restrict__ cols, const int32_t* __restrict__ off,
-                                    const int32_t* __restrict__ tile_cnt, const int32_t* __restrict__ tile_ent, int R,
-                                    int32_t* __restrict__ rank) {
-  const int t = blockIdx.x;
-  const int my_pos = pos[t];
-  const int n = tile_cnt[t];
-  for (int e = threadIdx.x; e < n; e += blockDim.x) {
-    const int qb = tile_ent[off[t] + e] >> 2;
-    const int r0 = row_ptr[qb], r1 = row_ptr[qb + 1];
-    int count = 0;
-    for (int x = r0; x < r1; ++x) {
-      const int kb = col_idx[x];
-      const int u = tile_of[kb];
-      if (u == t || pos[u] >= my_pos) continue;
-      if (R == 2) {   // a tile with both columns in this row counts once: at its smaller column
-        const int ca = cols[2 * u], cb = cols[2 * u + 1];
-        const int other = (kb == ca) ? cb : ca;
-        if (other >= 0 && other < kb) {
-          int lo = r0, hi = r1;            // is `other` in the (ascending) row?
-          while (lo < hi) {
-            const int mid = (lo + hi) >> 1;
-            if (col_idx[mid] < other) lo = mid + 1; else hi = mid;
-          }
-          if (lo < r1 && col_idx[lo] == other) continue;
-        }
-      }
-      ++count;
+
+// ---- schedule of the dQ pass that reads the kept dS tiles -------------------------------------
+// The dK/dV pass leaves, per (kv tile T, entry e = query block qb of T's schedule), dS^T tiles of 64
+// queries: numbered (off[T] + e) * (block / 64) + half.  A query tile of 128 rows needs, for every kv
+// tile with an active column in the row(s) of its query block(s), the two tiles of its two 64-row halves
+// (-1: that half has no entry in T, its dS is zero).  One thread per query tile; entries (T, h0, h1) at
+// dq_ent[3 * (row_ptr[R t] + i)], kv tiles ascending.
+__global__ void dq_sched_kernel(const int32_t* __restrict__ row_ptr, const int32_t* __restrict__ col_idx,
+                                const int32_t* __restrict__ tile_of, const int32_t* __restrict__ off,
+                                const int32_t* __restrict__ tile_cnt, const int32_t* __restrict__ tile_ent, int R, int nB,
+                                int n_qtiles, int32_t* __restrict__ dq_cnt, int32_t* __restrict__ dq_ent) {
+  const int t = blockIdx.x * blockDim.x + threadIdx.x;
+  if (t >= n_qtiles) return;
+  int32_t* out = dq_ent + 3 * static_cast<int64_t>(row_ptr[R * t]);
+  int n = 0;
+  for (int m = 0; m < R; ++m) {          // distinct kv tiles of the tile's query blocks, kept ascending
+    const int qb = R * t + m;
+    if (qb >= nB) break;
+    for (int x = row_ptr[qb]; x < row_ptr[qb + 1]; ++x) {
+      const int T = tile_of[col_idx[x]];
+      int pos = 0;
+      while (pos < n && out[3 * pos] < T) ++pos;
+      if (pos < n && out[3 * pos] == T) continue;
+      for (int y = n; y > pos; --y) out[3 * y] = out[3 * (y - 1)];
+      out[3 * pos] = T;
+      ++n;
     }
-    rank[off[t] + e] = count;
   }
+  auto find = [&](int T, int qb) {       // index of query block qb in T's schedule (ascending), or -1
+    if (qb >= nB) return -1;
+    int lo = 0, hi = tile_cnt[T];
+    const int32_t* ent = tile_ent + off[T];
+    while (lo < hi) {
+      const int mid = (lo + hi) >> 1;
+      if ((ent[mid] >> 2) < qb) lo = mid + 1; else hi = mid;
+    }
+    return (lo < tile_cnt[T] && (ent[lo] >> 2) == qb) ? lo : -1;
+  };
+  for (int i = 0; i < n; ++i) {
+    const int T = out[3 * i];
+    if (R == 1) {
+      const int e = find(T, t);
+      out[3 * i + 1] = (off[T] + e) * 2;
+      out[3 * i + 2] = (off[T] + e) * 2 + 1;
+    } else {
+      const int e0 = find(T, 2 * t), e1 = find(T, 2 * t + 1);
+      out[3 * i + 1] = e0 >= 0 ? off[T] + e0 : -1;
+      out[3 * i + 2] = e1 >= 0 ? off[T] + e1 : -1;
+    }
+  }
+  dq_cnt[t] = n;
 }
 
 // doc_end[b][j] = end (one past the last token) of the document token j belongs to, from

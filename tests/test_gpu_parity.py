@@ -96,12 +96,11 @@ def test_block_index_bit_exact(lg, cfg):
         assert np.array_equal(g.cpu().numpy(), r), name
 
 
-@pytest.mark.parametrize("variant", ["fused", "two_pass", "keep_ds"])
+@pytest.mark.parametrize("variant", ["two_pass", "keep_ds"])
 @pytest.mark.parametrize("cfg", SMALL, ids=lambda c: c.name)
 def test_fwd_bwd_parity_small(lg, cfg, variant, monkeypatch):
-    """The backward variants (the two passes; the dK/dV pass that keeps dS for a one-product dQ pass; the
-    single sweep that adds the parts of dQ in a fixed order) on every small pattern.  Where a variant does
-    not apply (keeping dS needs 128-token blocks, the single sweep D = 128) the name runs the two passes."""
+    """Both backward variants (the two passes; the dK/dV pass that keeps dS for a one-product dQ pass) on
+    every small pattern, 64- and 128-token blocks, GQA, ragged lengths."""
     monkeypatch.setenv("LG_BWD_VARIANT", variant)
     p = lg.params_of(cfg)
     inp = synth.make_attn_inputs(cfg, "cuda", seed=0, with_do=True)
@@ -122,13 +121,12 @@ def test_fwd_bwd_parity_small(lg, cfg, variant, monkeypatch):
         _assert_close(synth.to_f64(dv[b]), dV, TOL_G, "dV")
 
 
-@pytest.mark.parametrize("variant", ["fused", "two_pass", "keep_ds"])
+@pytest.mark.parametrize("variant", ["two_pass", "keep_ds"])
 @pytest.mark.parametrize("cfg", [SMALL[5], replace(synth.CFG1, name="rep_window", L=8192, D=128, Hq=8, Hkv=4, block=128,
                                                    sink_tokens=128, window_tokens=1024)], ids=lambda c: c.name)
 def test_bitwise_reproducible(lg, cfg, variant, monkeypatch):
-    """Same inputs, same bits, run after run: single writers in the two passes; in the single sweep the parts
-    of dQ that several kv tiles add to the same rows arrive in a fixed order (the second case has 64 kv tiles
-    per head in flight at once, so the order would show if it were left to chance)."""
+    """Same inputs, same bits, run after run: every output tile has a single writer and a fixed order of
+    accumulation, in both backward variants."""
     monkeypatch.setenv("LG_BWD_VARIANT", variant)
     p = lg.params_of(cfg)
     inp = synth.make_attn_inputs(cfg, "cuda", seed=1, with_do=True)
