@@ -663,7 +663,9 @@ lg_status lg_last_status(void* workspace, void* stream) {
   if (word[0] != 0 || word[1] != 0) {
     if (cudaMemset(workspace, 0, sizeof(word)) != cudaSuccess) return LG_ERR_CUDA;
     const unsigned int first = word[1] != 0 ? word[1] : word[0];
-    return (first >> 24) == 3u ? LG_ERR_WORKSPACE : LG_ERR_DEVICE_TIMEOUT;
+    // 3: lists of another pattern; 4 (checked builds): a schedule value out of range -- either way the workspace is not
+    // what the call needs
+    return ((first >> 24) == 3u || (first >> 24) == 4u) ? LG_ERR_WORKSPACE : LG_ERR_DEVICE_TIMEOUT;
   }
   return LG_OK;
 }

@@ -27,6 +27,7 @@ static lg_status launch_bwd_t(const Resolved& r, const WsLayout& w, const void* 
   a.stat_plane = static_cast<int64_t>(r.B) * r.Hq * a.Lp;
   a.error_word = r.error_word ? r.error_word : reinterpret_cast<unsigned int*>(ws);
   a.expect_fp = r.expect_fp;
+  a.n_tiles = r.n_ktiles; a.nB = r.pat.nB; a.n_list = static_cast<int>(r.nnz);   // (all three kernels walk ceil(L / 128) tiles)
   a.expect_fp2 = r.expect_fp2;
   a.L = r.L; a.Hq = r.Hq; a.Hkv = r.Hkv; a.G = r.G;
   a.exact_w = r.exact_w; a.ns = r.pat.ns;

@@ -46,6 +46,7 @@ struct BwdArgs {
   __nv_bfloat16* out1;       // unused | dV
   unsigned int* error_word;  // first word of the workspace header
   unsigned long long expect_fp, expect_fp2;   // fingerprints of the lists this call was told the workspace holds (0: built by the call itself)
+  int n_tiles, nB, n_list;   // sizes of the schedule arrays: tiles, pattern blocks, entries (bounds of the checked build)
   int64_t s0[3], s1[3];      // strides of out0 / out1 (batch, head, token; elements)
   int L, Hq, Hkv, G;
   int exact_w, ns;           // token-exact window (0: off) and number of sink blocks
@@ -199,10 +200,11 @@ bwd_dq_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ 
   // has a wait already given up in this call?  (read now, so that it travels with the schedule loads below)
   unsigned int abort_word = 0;
   if (tid == 0) abort_word = *reinterpret_cast<volatile unsigned int*>(a.error_word);
-  const int tile = a.order[blockIdx.y];
+  const int tile = checked(a.order[blockIdx.y], 0, a.n_tiles - 1, a.error_word, 110);
   const int b = blockIdx.x / a.Hq, h = blockIdx.x % a.Hq, hk = h / a.G;
-  const int n_ent = a.tile_cnt[tile];
-  const int32_t* ent = a.tile_ent + a.tile_off[tile * R];
+  const int ent_off = checked(a.tile_off[tile * R], 0, a.n_list, a.error_word, 111);
+  const int n_ent = checked(a.tile_cnt[tile], 0, a.n_list - ent_off, a.error_word, 112);
+  const int32_t* ent = a.tile_ent + ent_off;
   const int row0 = tile * 128;
   const int n_steps = (BS == 128) ? n_ent : (n_ent + 1) / 2;
 
@@ -510,12 +512,14 @@ bwd_dkdv_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
   // has a wait already given up in this call?  (read now, so that it travels with the schedule loads below)
   unsigned int abort_word = 0;
   if (tid == 0) abort_word = *reinterpret_cast<volatile unsigned int*>(a.error_word);
-  const int tile = a.order[blockIdx.y];
+  const int tile = checked(a.order[blockIdx.y], 0, a.n_tiles - 1, a.error_word, 120);
   const int b = blockIdx.x / a.Hkv, hk = blockIdx.x % a.Hkv;
-  const int n_ent = a.tile_cnt[tile];
-  const int32_t* ent = a.tile_ent + a.tile_off[tile];
+  const int ent_off = checked(a.tile_off[tile], 0, a.n_list, a.error_word, 121);
+  const int n_ent = checked(a.tile_cnt[tile], 0, a.n_list - ent_off, a.error_word, 122);
+  const int32_t* ent = a.tile_ent + ent_off;
   // key blocks of the tile's members (with 64-token blocks the two members need not be neighbours)
-  const int kb_a = a.tile_cols[R * tile], kb_b = (R == 2) ? a.tile_cols[R * tile + 1] : -1;
+  const int kb_a = checked(a.tile_cols[R * tile], 0, a.nB - 1, a.error_word, 123);
+  const int kb_b = (R == 2) ? checked(a.tile_cols[R * tile + 1], -1, a.nB - 1, a.error_word, 124) : -1;
   const int n_items = n_ent * a.G;
   const int n_hs = (BS == 128) ? kKvNB * n_items : (kKvNB == 2 ? n_items : (n_items + 1) / 2);    // half-steps
   const int n_steps = (n_hs + kKvNB - 1) / kKvNB;          // 128-row tiles streamed
@@ -576,7 +580,7 @@ bwd_dkdv_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
       auto next_item = [&](int& hq, int& qrow, int& entry) {
         entry = ent[e];
         hq = hk * a.G + grp;
-        qrow = (entry >> 2) * BS;
+        qrow = checked(entry >> 2, 0, a.nB - 1, a.error_word, 125) * BS;   // (also the address of the item's statistics)
         if (++e == n_ent) { e = 0; ++grp; }
       };
       for (int j = 0; j < n_steps; ++j) {
@@ -738,7 +742,7 @@ bwd_dkdv_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
         if (!ok) break;
         const int item = (BS == 128) ? j : hs;
         const int g = item / n_ent, e = item - g * n_ent;
-        const int64_t tile_idx = ((static_cast<int64_t>(b) * a.Hq + hk * a.G + g) * a.ds_nnz + a.tile_off[tile] + e) *
+        const int64_t tile_idx = ((static_cast<int64_t>(b) * a.Hq + hk * a.G + g) * a.ds_nnz + ent_off + e) *
                                      (BS / 64) + (BS == 128 ? half : 0);
         asm volatile("cp.async.bulk.tensor.2d.global.shared::cta.bulk_group.L2::cache_hint [%0, {%2, %3}], [%1], %4;" ::"l"(
                          reinterpret_cast<uint64_t>(&tm_ds)), "r"(smem_u32(sDS + half * SM::kDs)), "r"(0),
@@ -943,10 +947,11 @@ bwd_dq_from_ds_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_con
   if (!lists_match(a.error_word, a.expect_fp, a.expect_fp2, 80u)) return;
   unsigned int abort_word = 0;
   if (tid == 0) abort_word = *reinterpret_cast<volatile unsigned int*>(a.error_word);
-  const int t = a.order[blockIdx.y];                       // query tile (128 rows)
+  const int t = checked(a.order[blockIdx.y], 0, a.n_tiles - 1, a.error_word, 130);   // query tile (128 rows)
   const int b = blockIdx.x / a.Hq, h = blockIdx.x % a.Hq, hk = h / a.G;
-  const int n_ent = a.tile_cnt[t];
-  const int32_t* ent = a.tile_ent + 3 * static_cast<int64_t>(a.tile_off[R * t]);   // (kv tile, tile of half 0, tile of half 1)
+  const int ent_off = checked(a.tile_off[R * t], 0, a.n_list, a.error_word, 131);
+  const int n_ent = checked(a.tile_cnt[t], 0, a.n_list - ent_off, a.error_word, 132);
+  const int32_t* ent = a.tile_ent + 3 * static_cast<int64_t>(ent_off);   // (kv tile, tile of half 0, tile of half 1)
   if (tid == 0) {
     for (int i = 0; i < kAS; ++i) { mbar_init(bars + B_AF + i, 1); mbar_init(bars + B_AE + i, 1); }
     for (int i = 0; i < kKS; ++i) { mbar_init(bars + B_KF + i, 1); mbar_init(bars + B_KE + i, 1); }
@@ -978,7 +983,7 @@ bwd_dq_from_ds_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_con
       int nl = 0;
       int e_T = n_ent > 0 ? ent[0] : 0, e_h0 = n_ent > 0 ? ent[1] : 0, e_h1 = n_ent > 0 ? ent[2] : 0;
       for (int x = 0; x < n_ent; ++x) {
-        const int T = e_T, h0 = e_h0, h1 = e_h1;
+        const int T = checked(e_T, 0, a.nB - 1, a.error_word, 133), h0 = e_h0, h1 = e_h1;   // (with 64-token blocks T indexes the tiles' column pairs; nB bounds it from above)
         if (x + 1 < n_ent) { e_T = ent[3 * x + 3]; e_h0 = ent[3 * x + 4]; e_h1 = ent[3 * x + 5]; }   // read ahead
         const int sa = x % kAS, sk = x % kKS;
         if (x >= kAS) ok = mbar_wait(bars + B_AE + sa, ((x / kAS) - 1) & 1, a.error_word, 81);

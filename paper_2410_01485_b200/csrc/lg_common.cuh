@@ -10,7 +10,8 @@ namespace lg {
 // ---- workspace header (first 256 bytes of every workspace) ---------------------------
 struct WsHeader {
   unsigned int error_word;         // 0 = ok; else (code << 24) | site.  code 1: a wait gave up, 2: shared memory
-                                   // misaligned, 3: the workspace does not hold the lists the call was told it holds
+                                   // misaligned, 3: the workspace does not hold the lists the call was told it holds,
+                                   // 4: a schedule value out of range (checked builds only)
   unsigned int latched;            // an error word that a later call found unread and kept for lg_last_status
   unsigned long long magic;        // kWsMagic once the header has been initialised by a call
   unsigned long long fingerprint;  // which pattern the lists and schedules below were built for (0: none)
@@ -28,6 +29,22 @@ __device__ __forceinline__ bool lists_match(unsigned int* error_word, unsigned l
   if (have == fp || have == fp2) return true;
   if (threadIdx.x == 0) atomicCAS(error_word, 0u, (3u << 24) | site);
   return false;
+}
+
+// Checked builds (-DLG_DEBUG): every value read from a schedule or list that is later used as an index, an
+// offset or an address passes through here.  A value outside [lo, hi] is recorded in the status word
+// (code 4, with the site) and replaced by the nearest bound, so that a damaged workspace shows up as a
+// status instead of a fault.  In normal builds this is the identity.
+__device__ __forceinline__ int checked(int v, int lo, int hi, unsigned int* error_word, unsigned int site) {
+#ifdef LG_DEBUG
+  if (v < lo || v > hi) {
+    atomicCAS(error_word, 0u, (4u << 24) | site);
+    return v < lo ? lo : hi;
+  }
+#else
+  (void)lo; (void)hi; (void)error_word; (void)site;
+#endif
+  return v;
 }
 
 constexpr long long kWaitLimitCycles = 4000000000ll;   // ~2 s of SM clock: a wait that long gave up

@@ -563,6 +563,38 @@ static int choose_nsplit(const lg_decode_params* p) {
 // Batches of up to kDecFlatMaxB sequences take the flattened one-wave schedule.
 static bool decode_is_flat(const lg_decode_params* p) { return p->B <= kDecFlatMaxB; }
 
+// What a decode call needs to know about its device, looked up once per device: the SM count, and
+// that the streaming kernels may use their large dynamic shared memory.  (A serving loop makes this call
+// every 50 microseconds; the runtime queries cost a noticeable part of that on the host.)
+namespace {
+constexpr int kMaxDecodeDevices = 64;
+struct DecodeDeviceInfo { int sms = 0; bool ready = false; };
+DecodeDeviceInfo g_decode_dev[kMaxDecodeDevices];
+std::mutex g_decode_dev_mutex;
+
+lg_status decode_device_info(int* sms_out) {
+  int dev = -1;
+  if (cudaGetDevice(&dev) != cudaSuccess) return LG_ERR_CUDA;
+  if (dev < 0 || dev >= kMaxDecodeDevices) return LG_ERR_UNSUPPORTED;
+  std::lock_guard<std::mutex> lock(g_decode_dev_mutex);
+  DecodeDeviceInfo& d = g_decode_dev[dev];
+  if (!d.ready) {
+    const lg_status arch = check_arch();                     // the kernels are built for sm_100a only
+    if (arch != LG_OK) return arch;
+    if (cudaDeviceGetAttribute(&d.sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess) return LG_ERR_CUDA;
+    const int big = 227 * 1024;   // the kernels are launched with what they need, which is below this
+    if (cudaFuncSetAttribute(decode_stream_kernel<128>, cudaFuncAttributeMaxDynamicSharedMemorySize, big) != cudaSuccess ||
+        cudaFuncSetAttribute(decode_stream_kernel<64>, cudaFuncAttributeMaxDynamicSharedMemorySize, big) != cudaSuccess ||
+        cudaFuncSetAttribute(decode_split_kernel<128>, cudaFuncAttributeMaxDynamicSharedMemorySize, big) != cudaSuccess ||
+        cudaFuncSetAttribute(decode_split_kernel<64>, cudaFuncAttributeMaxDynamicSharedMemorySize, big) != cudaSuccess)
+      return LG_ERR_CUDA;
+    d.ready = true;
+  }
+  *sms_out = d.sms;
+  return LG_OK;
+}
+}  // namespace
+
 static size_t decode_part_bytes(const lg_decode_params* p, int nsplit) {
   const int HG = (p->Hq / p->Hkv + kDecHeads - 1) / kDecHeads;
   return static_cast<size_t>(p->B) * p->Hkv * HG * nsplit * kDecHeads * (p->D + 2) * sizeof(float);
@@ -626,7 +658,8 @@ lg_status lg_sparse_decode(const lg_decode_params* p, const void* q, const void*
       (reinterpret_cast<uintptr_t>(workspace) & 255))
     return LG_ERR_INVALID_ARG;
   if (workspace_bytes < lg_sparse_decode_workspace_bytes(p)) return LG_ERR_WORKSPACE;
-  if ((s = check_arch()) != LG_OK) return s;
+  int sms = 0;
+  if ((s = decode_device_info(&sms)) != LG_OK) return s;
   cudaStream_t st = static_cast<cudaStream_t>(stream);
   DecodeArgs a;
   a.q = static_cast<const __nv_bfloat16*>(q);
@@ -646,10 +679,6 @@ lg_status lg_sparse_decode(const lg_decode_params* p, const void* q, const void*
   a.scale_log2 = scale * 1.4426950408889634f;
   a.B = p->B;
   if (decode_is_flat(p)) {
-    int dev = 0, sms = 0;
-    if (cudaGetDevice(&dev) != cudaSuccess ||
-        cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess)
-      return LG_ERR_CUDA;
     // as many CTAs per SM as shared memory allows (at most two), fewer when the cache is too small to
     // give each warp a couple of tiles
     const int64_t units = static_cast<int64_t>(p->B) * a.Hkv * a.HG;
@@ -672,14 +701,8 @@ lg_status lg_sparse_decode(const lg_decode_params* p, const void* q, const void*
     a.part = reinterpret_cast<float*>(static_cast<uint8_t*>(workspace) + sizeof(WsHeader) + count_bytes);
     const int smem_flat = kDecWarps * kDecStages * 2 * kDecTile * p->D * 2 + (p->B + 1) * static_cast<int>(sizeof(int));
     if (p->D == 128) {
-      if (cudaFuncSetAttribute(decode_stream_kernel<128>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem_flat) !=
-          cudaSuccess)
-        return LG_ERR_CUDA;
       decode_stream_kernel<128><<<static_cast<unsigned>(n_cta), kDecWarps * 32, smem_flat, st>>>(a); note_launch();
     } else {
-      if (cudaFuncSetAttribute(decode_stream_kernel<64>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem_flat) !=
-          cudaSuccess)
-        return LG_ERR_CUDA;
       decode_stream_kernel<64><<<static_cast<unsigned>(n_cta), kDecWarps * 32, smem_flat, st>>>(a); note_launch();
     }
     return cudaGetLastError() == cudaSuccess ? LG_OK : LG_ERR_CUDA;
@@ -689,15 +712,9 @@ lg_status lg_sparse_decode(const lg_decode_params* p, const void* q, const void*
   dim3 grid(a.nsplit, a.Hkv * a.HG, p->B);
   const int smem = kDecWarps * kDecStages * 2 * kDecTile * p->D * 2;
   if (p->D == 128) {
-    if (cudaFuncSetAttribute(decode_split_kernel<128>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem) !=
-        cudaSuccess)
-      return LG_ERR_CUDA;
     decode_split_kernel<128><<<grid, kDecWarps * 32, smem, st>>>(a); note_launch();
     decode_merge_kernel<128><<<p->B * a.Hkv * a.HG, 128, 0, st>>>(a); note_launch();
   } else {
-    if (cudaFuncSetAttribute(decode_split_kernel<64>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem) !=
-        cudaSuccess)
-      return LG_ERR_CUDA;
     decode_split_kernel<64><<<grid, kDecWarps * 32, smem, st>>>(a); note_launch();
     decode_merge_kernel<64><<<p->B * a.Hkv * a.HG, 128, 0, st>>>(a); note_launch();
   }

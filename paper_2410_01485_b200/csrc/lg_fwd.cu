@@ -21,6 +21,7 @@ static lg_status launch_fwd_t(const Resolved& r, const WsLayout& w, const void* 
   a.lse = lse;
   a.error_word = r.error_word ? r.error_word : reinterpret_cast<unsigned int*>(ws);
   a.expect_fp = r.expect_fp;
+  a.n_tiles = r.n_stiles; a.nB = r.pat.nB; a.n_list = static_cast<int>(r.nnz);
   a.expect_fp2 = r.expect_fp2;
   for (int i = 0; i < 3; ++i) a.o_strides[i] = r.os[i];
   a.L = r.L; a.Hq = r.Hq; a.G = r.G;

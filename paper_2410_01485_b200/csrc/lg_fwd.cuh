@@ -33,6 +33,7 @@ struct FwdArgs {
   float* lse;                // [B, Hq, L]
   unsigned int* error_word;  // first word of the workspace header
   unsigned long long expect_fp, expect_fp2;   // fingerprints of the lists this call was told the workspace holds (0: built by the call itself)
+  int n_tiles, nB, n_list;   // sizes of the schedule arrays: tiles, pattern blocks, entries (bounds of the checked build)
   int64_t o_strides[3];      // batch, head, token (elements)
   int L, Hq, G;              // G = Hq / Hkv
   int q_start, Lq;           // queries exist for rows [q_start, q_start + Lq) of the L key positions only
@@ -94,10 +95,11 @@ fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUt
   // has a wait already given up in this call?  (read now, so that it travels with the schedule loads below)
   unsigned int abort_word = 0;
   if (tid == 0) abort_word = *reinterpret_cast<volatile unsigned int*>(a.error_word);
-  const int tile = a.order[blockIdx.y];
+  const int tile = checked(a.order[blockIdx.y], 0, a.n_tiles - 1, a.error_word, 100);
   const int b = blockIdx.x / a.Hq, h = blockIdx.x % a.Hq, hk = h / a.G;
-  const int n_ent = a.tile_cnt[tile];
-  const int32_t* ent = a.tile_ent + a.tile_off[tile * R4];
+  const int ent_off = checked(a.tile_off[tile * R4], 0, a.n_list, a.error_word, 101);
+  const int n_ent = checked(a.tile_cnt[tile], 0, a.n_list - ent_off, a.error_word, 102);
+  const int32_t* ent = a.tile_ent + ent_off;
   const int row0 = tile * 256;
   const int n_steps = (BS == 128) ? n_ent : (n_ent + 1) / 2;
   if (row0 + 256 <= a.q_start) return;   // no query lives in this super-tile (uniform over the CTA)
