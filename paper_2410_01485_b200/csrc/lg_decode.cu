@@ -582,11 +582,14 @@ lg_status decode_device_info(int* sms_out) {
     const lg_status arch = check_arch();                     // the kernels are built for sm_100a only
     if (arch != LG_OK) return arch;
     if (cudaDeviceGetAttribute(&d.sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess) return LG_ERR_CUDA;
-    const int big = 227 * 1024;   // the kernels are launched with what they need, which is below this
-    if (cudaFuncSetAttribute(decode_stream_kernel<128>, cudaFuncAttributeMaxDynamicSharedMemorySize, big) != cudaSuccess ||
-        cudaFuncSetAttribute(decode_stream_kernel<64>, cudaFuncAttributeMaxDynamicSharedMemorySize, big) != cudaSuccess ||
-        cudaFuncSetAttribute(decode_split_kernel<128>, cudaFuncAttributeMaxDynamicSharedMemorySize, big) != cudaSuccess ||
-        cudaFuncSetAttribute(decode_split_kernel<64>, cudaFuncAttributeMaxDynamicSharedMemorySize, big) != cudaSuccess)
+    // the most dynamic shared memory a launch of each kernel can ask for: the tile pipelines of the
+    // warps, plus (flattened schedule) the prefix array of the largest batch it takes
+    auto pipe = [](int D) { return kDecWarps * kDecStages * 2 * kDecTile * D * 2; };
+    const int cum = (kDecFlatMaxB + 1) * static_cast<int>(sizeof(int));
+    if (cudaFuncSetAttribute(decode_stream_kernel<128>, cudaFuncAttributeMaxDynamicSharedMemorySize, pipe(128) + cum) != cudaSuccess ||
+        cudaFuncSetAttribute(decode_stream_kernel<64>, cudaFuncAttributeMaxDynamicSharedMemorySize, pipe(64) + cum) != cudaSuccess ||
+        cudaFuncSetAttribute(decode_split_kernel<128>, cudaFuncAttributeMaxDynamicSharedMemorySize, pipe(128)) != cudaSuccess ||
+        cudaFuncSetAttribute(decode_split_kernel<64>, cudaFuncAttributeMaxDynamicSharedMemorySize, pipe(64)) != cudaSuccess)
       return LG_ERR_CUDA;
     d.ready = true;
   }
