@@ -121,14 +121,14 @@ lg_status resolve(const lg_attn_params* p, Resolved* r) {
 // (default 48) gigabytes.  LG_BWD_VARIANT = two_pass | keep_ds overrides the choice (read at every call;
 // it must not change between a size query, a prepare and the calls that use them).
 size_t ds_buffer_bytes(const Resolved& r) {   // every tile of 64 queries x 128 keys, plus one tile of zeros at the end
-  return (static_cast<size_t>(r.B) * r.Hq * static_cast<size_t>(r.nnz) * (r.block / 64) + 1) * (128 * 128);
+  return (static_cast<size_t>(r.B) * r.Hq * static_cast<size_t>(r.nnz) * (r.block / 64) + 1) * static_cast<size_t>(128 * 64 * 2);
 }
 
 BwdVariant bwd_variant(const Resolved& r) {
   const char* env = getenv("LG_BWD_VARIANT");
   if (env && strcmp(env, "two_pass") == 0) return kBwdTwoPass;
-  // the stored tiles are addressed by 32-bit row coordinates of a tensor map
-  const bool can_keep = !(r.doc_start != nullptr && r.B > 1) && ds_buffer_bytes(r) / 128 < (1ull << 31);
+  // (per-sequence lists have no common tile numbering)
+  const bool can_keep = !(r.doc_start != nullptr && r.B > 1);
   if (env && strcmp(env, "keep_ds") == 0) return can_keep ? kBwdKeepDs : kBwdTwoPass;
   double max_gb = 48.0;
   if (const char* m = getenv("LG_KEEP_DS_MAX_GB")) max_gb = atof(m);
@@ -287,20 +287,6 @@ lg_status make_tmap(CUtensorMap* out, const void* base, int B, int H, int L, int
   return rc == CUDA_SUCCESS ? LG_OK : LG_ERR_CUDA;
 }
 
-
-// dS^T buffer of the backward that keeps dS: rows of 64 bf16 (128 bytes), boxes of 128 rows, 128-byte swizzle
-lg_status make_tmap_ds(CUtensorMap* out, const void* base, int64_t rows) {
-  EncodeTiledFn fn = get_encode_fn();
-  if (!fn) return LG_ERR_CUDA;
-  cuuint64_t dims[2] = {64, static_cast<cuuint64_t>(rows)};
-  cuuint64_t gstr[1] = {128};
-  cuuint32_t box[2] = {64, 128};
-  cuuint32_t estr[2] = {1, 1};
-  CUresult rc = fn(out, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(base), dims, gstr, box, estr,
-                   CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
-                   CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
-  return rc == CUDA_SUCCESS ? LG_OK : LG_ERR_CUDA;
-}
 
 // ---- chunk served against a sink + window ring ----------------------------------------------
 // Time-ordered copy of what the ring holds, followed by the chunk: K_lin, V_lin [B, Hkv, Lc, D]

@@ -36,6 +36,7 @@ static lg_status launch_bwd_t(const Resolved& r, const WsLayout& w, const void* 
   a.scale = r.scale;
   a.scale_log2 = r.scale * 1.4426950408889634f;
   a.ds_nnz = r.nnz;
+  a.ds_buf = reinterpret_cast<__nv_bfloat16*>(ws + w.ds_buf);
   constexpr int smem = BwdSmem<D, BS>::kTotal;
   const BwdVariant variant = bwd_variant(r);
 
@@ -57,27 +58,23 @@ static lg_status launch_bwd_t(const Resolved& r, const WsLayout& w, const void* 
     dim3 grid(r.B * r.Hkv, r.n_ktiles);
     if (variant == kBwdKeepDs) {
       // the tile of zeros that stands in for a half of a query tile a kv tile has no entry for
-      if (cudaMemsetAsync(ws + w.ds_buf + ds_buffer_bytes(r) - 128 * 128, 0, 128 * 128, stream) != cudaSuccess) return LG_ERR_CUDA;
-      CUtensorMap tds;
-      if ((s = make_tmap_ds(&tds, ws + w.ds_buf, static_cast<int64_t>(ds_buffer_bytes(r) / 128))) != LG_OK) return s;
+      if (cudaMemsetAsync(ws + w.ds_buf + ds_buffer_bytes(r) - kDsTileBytes, 0, kDsTileBytes, stream) != cudaSuccess) return LG_ERR_CUDA;
       auto kern = bwd_dkdv_kernel<D, BS, true>;
-      constexpr int smem_k = BwdSmem<D, BS, true>::kTotal;
-      if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, smem_k) != cudaSuccess)
+      if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, smem) != cudaSuccess)
         return LG_ERR_CUDA;
-      kern<<<grid, kKvThreads + 32, smem_k, stream>>>(tq, tk, tv, tdo, tds, a); note_launch();
+      kern<<<grid, kKvThreads, smem, stream>>>(tq, tk, tv, tdo, a); note_launch();
     } else {
       auto kern = bwd_dkdv_kernel<D, BS, false>;
       if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, smem) != cudaSuccess)
         return LG_ERR_CUDA;
-      kern<<<grid, kKvThreads, smem, stream>>>(tq, tk, tv, tdo, tq /* unused */, a); note_launch();
+      kern<<<grid, kKvThreads, smem, stream>>>(tq, tk, tv, tdo, a); note_launch();
     }
     if (marks) cudaEventRecord(marks[2], stream);
   }
   if (variant == kBwdKeepDs) {
     // ---- dQ = scale * dS K from the kept tiles --------------------------------------------
-    CUtensorMap tk, tds;
+    CUtensorMap tk;
     if ((s = make_tmap(&tk, k, r.B, r.Hkv, r.L, D, r.ks, BS)) != LG_OK) return s;
-    if ((s = make_tmap_ds(&tds, ws + w.ds_buf, static_cast<int64_t>(ds_buffer_bytes(r) / 128))) != LG_OK) return s;
     a.tile_off = reinterpret_cast<const int32_t*>(ws + w.row_ptr);
     a.tile_ent = reinterpret_cast<const int32_t*>(ws + w.dq_ent);
     a.tile_cols = reinterpret_cast<const int32_t*>(ws + w.kt_cols);
@@ -91,7 +88,7 @@ static lg_status launch_bwd_t(const Resolved& r, const WsLayout& w, const void* 
     if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, smem_q) != cudaSuccess)
       return LG_ERR_CUDA;
     dim3 grid(r.B * r.Hq, r.n_qtiles);
-    kern<<<grid, kDq2Threads, smem_q, stream>>>(tk, tds, a); note_launch();
+    kern<<<grid, kDq2Threads, smem_q, stream>>>(tk, a); note_launch();
     if (marks) cudaEventRecord(marks[3], stream);
     return cudaGetLastError() == cudaSuccess ? LG_OK : LG_ERR_CUDA;
   }

@@ -54,10 +54,16 @@ struct BwdArgs {
   const int32_t* doc_end;    // [B, L] end of each token's document (null together with doc_start)
   float scale, scale_log2;
   // dK/dV pass that also keeps dS (see bwd_dkdv_kernel): dS^T of every half-step of 64 queries goes to
-  // ds_buf as a tile of [128 keys][64 queries] bf16; tile index = ((b * Hq + h) * ds_nnz + schedule
-  // position of the (kv tile, query block) entry) * (block / 64) + half.  The dQ pass then reads them back.
+  // ds_buf as a tile of 16 KB; tile index = ((b * Hq + h) * ds_nnz + schedule position of the (kv tile,
+  // query block) entry) * (block / 64) + half.  The dQ pass then reads them back.  Inside a tile the
+  // element (key k, query q) sits at byte (q / 8) * 2048 + k * 16 + (q % 8) * 2: eight queries of one key
+  // are 16 contiguous bytes, the 128 keys of such a group follow one another -- the un-swizzled
+  // core-matrix layout of a tensor-core operand whose M (query) index is the contiguous one, and a
+  // layout in which the 32 key rows of a warp write 512 contiguous bytes per store instruction.
   int64_t ds_nnz;
+  __nv_bfloat16* ds_buf;
 };
+constexpr int kDsTileBytes = 128 * 64 * 2;
 
 // ---- stat = -(LSE * log2 e) and -rowsum(dO * O), stored negated (they are only ever subtracted),
 // each in a plane of its own: the dK/dV pass fetches four neighbouring queries' values of one kind
@@ -103,17 +109,15 @@ struct BwdTile {
   static constexpr int kBytes = (D / 64) * kBox;
 };
 
-template <int D, int BS, bool kSpill = false>
+template <int D, int BS>
 struct BwdSmem {
   static constexpr int kTile = BwdTile<D>::kBytes;
-  static constexpr int kDs = 128 * 128;                          // a dS^T tile: 128 keys x 64 queries bf16
-  static constexpr int kAStages = kSpill ? 2 : 3;   // operand read by the first and the last MMA of a step (K | Q)
+  static constexpr int kAStages = 3;   // operand read by the first and the last MMA of a step (K | Q)
   static constexpr int kBStages = 2;   // operand read by adjacent MMAs (V | dO)
   static constexpr int oFix0 = 0, oFix1 = kTile;
   static constexpr int oA = 2 * kTile;
   static constexpr int oB = oA + kAStages * kTile;
-  static constexpr int oDS = oB + kBStages * kTile;              // [2] dS^T tiles on their way to global memory (kSpill)
-  static constexpr int oStat = oDS + (kSpill ? 2 * kDs : 0);     // dK/dV pass: [2 stages][2 planes][128] floats
+  static constexpr int oStat = oB + kBStages * kTile;            // dK/dV pass: [2 stages][2 planes][128] floats
   static constexpr int oBar = oStat + 2 * 128 * 8;
   static constexpr int kBarBytes = 512;                          // mbarriers, the TMEM slot and the step's schedule entries
   static constexpr int kTotal = oBar + kBarBytes;
@@ -453,48 +457,47 @@ bwd_dq_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ 
 // worked in two half-steps of 64 queries.  TMEM columns: S^T of the even / odd half-step at
 // 0 / 64 (P^T written as bf16 over it), dP^T at 128 / 192 (dS^T over it), dV at 256, dK at 384:
 // both score tiles are double-buffered, so the S^T of the next half-step is computed while the
-// exponentials of this one are evaluated.  Sixteen element-wise warps (four groups of 16
-// streamed queries) and two issuing threads on different scheduler partitions: thread A issues
-// S^T and dV (dV reads P^T from the S^T columns, so the S^T that overwrites them follows it in
-// the same queue), thread B issues dP^T and dK likewise.
-#ifndef LG_KV_EW_WARPS
-#define LG_KV_EW_WARPS 16
-#endif
-constexpr int kKvEwWarps = LG_KV_EW_WARPS;
+// exponentials of this one are evaluated.  Sixteen element-wise warps in two teams of eight: team t
+// works the half-steps t, t + 2, ... (the t-th half of every step; its threads take 32 of the 64
+// streamed queries each), so that on every scheduler partition two warps are in the arithmetic of one
+// half-step while the other two sit in the loads, stores, fences and barrier round trips of the next
+// -- with all sixteen warps on the same half-step those latencies were paid one after the other and
+// the element-wise path, not the tensor pipe, set the pace.  Two issuing threads on different
+// scheduler partitions: thread A issues S^T and dV (dV reads P^T from the S^T columns, so the S^T
+// that overwrites them follows it in the same queue), thread B issues dP^T and dK likewise.
+constexpr int kKvEwWarps = 16;
+constexpr int kKvTeamWarps = kKvEwWarps / 2;
 constexpr int kKvTmaWarp = kKvEwWarps, kKvMmaWarpA = kKvEwWarps + 1, kKvMmaWarpB = kKvEwWarps + 2;
 constexpr int kKvThreads = (kKvEwWarps + 3) * 32;
-#ifndef LG_KV_HALF
-#define LG_KV_HALF 64
-#endif
-constexpr int kKvHalf = LG_KV_HALF;                        // queries of a (half-)step: 64, or 128 = whole steps, single buffers
-constexpr int kKvNB = 128 / kKvHalf;                       // (half-)steps per step = score buffers in rotation
-constexpr int kKvCols = kKvHalf / (kKvEwWarps / 4);        // queries of a half-step per element-wise thread
+constexpr int kKvHalf = 64;                                // queries of a half-step
+constexpr int kKvNB = 128 / kKvHalf;                       // half-steps per step = score buffers in rotation = teams
+constexpr int kKvCols = kKvHalf / (kKvTeamWarps / 4);      // queries of a half-step per element-wise thread
 
-// kSpill: the pass also writes dS^T (bf16) of every half-step to global memory (tm_ds: the buffer as
-// rows of 64 queries, boxes of 128 key rows, 128-byte swizzle; in memory the tiles are plain row-major
-// [128 keys][64 queries]), so that the dQ pass is one product per step, dQ += dS K, instead of
-// recomputing S and dP (bwd_dq_from_ds_kernel).  The element-wise warps put dS^T into shared memory as
-// well as tensor memory and a store warp sends the tiles on their way with TMA.  (Storing the 32 bytes of
-// every thread straight from its registers was measured 20 % slower: 32 separate cache lines per
-// instruction keep the load/store unit busy.)
+// kSpill: the pass also writes dS^T (bf16) of every half-step to global memory (BwdArgs::ds_buf), so
+// that the dQ pass is one product per step, dQ += dS K, instead of recomputing S and dP
+// (bwd_dq_from_ds_kernel).  Every element-wise thread stores the 64 bytes it holds (32 queries of its
+// key) straight from its registers: in the tile layout described at BwdArgs::ds_buf a warp's store
+// instruction covers 512 contiguous bytes.  (Staging the tiles in shared memory for a TMA store cost
+// a shared-memory ring stage of Q, a proxy fence and two barrier round trips per half-step; storing
+// rows of a [key][query] layout from registers touched 32 separate cache lines per instruction.)
 template <int D, int BS, bool kSpill>
-__global__ void __launch_bounds__(kKvThreads + (kSpill ? 32 : 0), 1)
+__global__ void __launch_bounds__(kKvThreads, 1)
 bwd_dkdv_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUtensorMap tm_k,
-                const __grid_constant__ CUtensorMap tm_v, const __grid_constant__ CUtensorMap tm_do,
-                const __grid_constant__ CUtensorMap tm_ds, const BwdArgs a) {
-  using SM = BwdSmem<D, BS, kSpill>;
+                const __grid_constant__ CUtensorMap tm_v, const __grid_constant__ CUtensorMap tm_do, const BwdArgs a) {
+  using SM = BwdSmem<D, BS>;
   constexpr int kQS = SM::kAStages;
   constexpr int R = 128 / BS;
   constexpr uint32_t kColS = 0, kColDP = 128, kColDV = 256, kColDK = 384;
   constexpr int kTile = SM::kTile;
   enum { B_FIX = 0, B_QF = 1, B_QE = 4, B_OF = 7, B_OE = 9, B_SF = 11, B_DPF = 13, B_PF = 15, B_DSF = 17,
-         B_DONE = 19, B_DRAIN = 20, B_STF = 22, B_STE = 24, B_DSE = 26, B_DSS = 28, B_COUNT = 30 };
+         B_DONE = 19, B_DRAIN = 20, B_STF = 22, B_STE = 24, B_COUNT = 26 };
 
   extern __shared__ __align__(1024) uint8_t smem[];
   uint64_t* bars = reinterpret_cast<uint64_t*>(smem + SM::oBar);
   uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + B_COUNT);
   int32_t* sEnt = reinterpret_cast<int32_t*>(bars + B_COUNT + 1);   // [2][2]: entries of a step's items
-  static_assert((B_COUNT + 1) * 8 + 16 <= SM::kBarBytes, "barrier area too small");
+  int64_t* sTile = reinterpret_cast<int64_t*>(bars + B_COUNT + 3);  // [2][2]: dS tile index of a step's items (kSpill)
+  static_assert((B_COUNT + 3) * 8 + 32 <= SM::kBarBytes, "barrier area too small");
   const int tid = threadIdx.x, lane = tid & 31;
   const int warp = __shfl_sync(0xffffffffu, tid >> 5, 0);   // same value, known to be warp-uniform
   if ((smem_u32(smem) & 1023u) != 0) {
@@ -506,7 +509,6 @@ bwd_dkdv_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
   uint8_t* sV = smem + SM::oFix1;
   uint8_t* sQ = smem + SM::oA;     // [3]
   uint8_t* sDO = smem + SM::oB;    // [2]
-  uint8_t* sDS = smem + SM::oDS;   // [2] (kSpill)
   float* sStat = reinterpret_cast<float*>(smem + SM::oStat);   // [2 stages][-LSE2 | -delta][128 queries]
 
   // has a wait already given up in this call?  (read now, so that it travels with the schedule loads below)
@@ -535,13 +537,11 @@ bwd_dkdv_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
       mbar_init(bars + B_OE + i, 2);      // dP^T (thread B) and dV (thread A) both read the dO tile
       mbar_init(bars + B_SF + i, 1);
       mbar_init(bars + B_DPF + i, 1);
-      mbar_init(bars + B_PF + i, kKvEwWarps);
-      mbar_init(bars + B_DSF + i, kKvEwWarps);
+      mbar_init(bars + B_PF + i, kKvTeamWarps);
+      mbar_init(bars + B_DSF + i, kKvTeamWarps);
       mbar_init(bars + B_DRAIN + i, 1);
       mbar_init(bars + B_STF + i, 1);
-      mbar_init(bars + B_STE + i, kKvEwWarps);
-      mbar_init(bars + B_DSE + i, 1);
-      mbar_init(bars + B_DSS + i, kKvEwWarps);
+      mbar_init(bars + B_STE + i, kKvEwWarps);   // every warp once per step, after its team's half
     }
     mbar_init(bars + B_DONE, 2);          // the last dV and the last dK
     mbar_fence_init();
@@ -577,22 +577,25 @@ bwd_dkdv_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
       bool ok = true;
       int nq = 0, no = 0, nst = 0;   // loads started
       int grp = 0, e = 0;            // (query head within the group, entry) of the next item
-      auto next_item = [&](int& hq, int& qrow, int& entry) {
+      auto next_item = [&](int& hq, int& qrow, int& entry, int64_t& ds_tile) {
         entry = ent[e];
         hq = hk * a.G + grp;
         qrow = checked(entry >> 2, 0, a.nB - 1, a.error_word, 125) * BS;   // (also the address of the item's statistics)
+        ds_tile = ((static_cast<int64_t>(b) * a.Hq + hq) * a.ds_nnz + ent_off + e) * (BS / 64);
         if (++e == n_ent) { e = 0; ++grp; }
       };
       for (int j = 0; j < n_steps; ++j) {
         const int sq = j % kQS, so = j & 1;
         int h0, r0, e0, h1, r1, e1;
-        next_item(h0, r0, e0);
-        h1 = h0; r1 = r0; e1 = e0 & ~3;                         // a missing second item repeats the first block, as nobody's member
-        if (BS == 64 && 2 * j + 1 < n_items) next_item(h1, r1, e1);
+        int64_t t0, t1;
+        next_item(h0, r0, e0, t0);
+        h1 = h0; r1 = r0; e1 = e0 & ~3; t1 = t0 + 1;            // a missing second item repeats the first block, as nobody's member
+        if (BS == 64 && 2 * j + 1 < n_items) next_item(h1, r1, e1, t1);
         if (j >= 2) ok = mbar_wait(bars + B_STE + so, ((j / 2) - 1) & 1, a.error_word, 40);
         if (!ok) break;
         sEnt[so * 2] = e0;
         sEnt[so * 2 + 1] = e1;
+        if (kSpill) { sTile[so * 2] = t0; sTile[so * 2 + 1] = t1; }   // (128-token blocks: the two halves of the one item)
         mbar_expect_tx(bars + B_STF + so, 2 * 128 * 4);         // (release: publishes the entries as well)
         {
           const float* st0 = a.stat + (static_cast<int64_t>(b) * a.Hq + h0) * a.Lp + r0;
@@ -725,40 +728,11 @@ bwd_dkdv_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
       if (lead) { mma_commit(bars + B_DONE); mma_commit(bars + B_DRAIN + 1); }
       mbar_wait(bars + B_DRAIN + 1, 0, a.error_word, 7);
     }
-  } else if (kSpill && warp == kKvMmaWarpB + 1) {
-    // ------------------------------ store warp: dS^T tiles -> global memory (kSpill) ----------
-    // The element-wise warps leave dS^T of every half-step in shared memory as well; this thread sends the
-    // tile on its way and tells them when its buffer may be written again.  Items = (query head g of the
-    // group, entry e) in schedule order; one tile of 64 queries per half-step.
-    if (lane == 0) {
-      uint64_t evict_first;
-      // (written once, read once by the dQ pass: marked evict-first so that the stream does not push the
-      // Q / dO tiles, which every kv tile of a window re-reads, out of the L2)
-      asm volatile("createpolicy.fractional.L2::evict_first.b64 %0, 1.0;" : "=l"(evict_first));
-      bool ok = true;
-      for (int hs = 0; hs < n_hs && ok; ++hs) {
-        const int j = hs / kKvNB, half = hs % kKvNB;
-        ok = mbar_wait(bars + B_DSS + half, j & 1, a.error_word, 43);
-        if (!ok) break;
-        const int item = (BS == 128) ? j : hs;
-        const int g = item / n_ent, e = item - g * n_ent;
-        const int64_t tile_idx = ((static_cast<int64_t>(b) * a.Hq + hk * a.G + g) * a.ds_nnz + ent_off + e) *
-                                     (BS / 64) + (BS == 128 ? half : 0);
-        asm volatile("cp.async.bulk.tensor.2d.global.shared::cta.bulk_group.L2::cache_hint [%0, {%2, %3}], [%1], %4;" ::"l"(
-                         reinterpret_cast<uint64_t>(&tm_ds)), "r"(smem_u32(sDS + half * SM::kDs)), "r"(0),
-                     "r"(static_cast<int>(tile_idx * 128)), "l"(evict_first) : "memory");
-        asm volatile("cp.async.bulk.commit_group;" ::: "memory");
-        if (hs >= 1) {   // the tile of the half-step before this one has been read out of its buffer
-          asm volatile("cp.async.bulk.wait_group.read 1;" ::: "memory");
-          mbar_arrive(bars + B_DSE + ((hs - 1) & 1));
-        }
-      }
-      asm volatile("cp.async.bulk.wait_group 0;" ::: "memory");   // my stores have left shared memory and landed
-    }
   } else {
     // ------------------------------ element-wise warps ------------------------------------
     constexpr int C = kKvCols;
-    const int g = warp >> 2;                                // group of C streamed queries
+    const int half = warp / kKvTeamWarps;                   // team = the half of every step it works
+    const int g = (warp >> 2) % (kKvTeamWarps / 4);         // group of C streamed queries within the half-step
     const int r = (warp & 3) * 32 + lane;                   // key row in the tile == TMEM lane
     const int member = (R == 1) ? 0 : (r / BS);
     const int kb_mine = (R == 2 && member) ? kb_b : kb_a;
@@ -768,15 +742,15 @@ bwd_dkdv_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
     const int dend = (a.doc_end && kb_mine >= 0 && kj < a.L) ? a.doc_end[static_cast<int64_t>(b) * a.L + kj] : a.L;
     const uint32_t lane_addr = tmem + (static_cast<uint32_t>((warp & 3) * 32) << 16);
     const uint64_t scale2 = f32x2(a.scale_log2, a.scale_log2);
+    uint64_t evict_first = 0;
+    if (kSpill) asm volatile("createpolicy.fractional.L2::evict_first.b64 %0, 1.0;" : "=l"(evict_first));
     bool ok = true;
 #pragma unroll 1
-    for (int hs = 0; hs < n_hs; ++hs) {
-      const int j = hs / kKvNB, half = hs % kKvNB;
-      if (half == 0) {
-        ok = mbar_wait(bars + B_STF + (j & 1), (j >> 1) & 1, a.error_word, 4);   // statistics and entries of step j
-        ok = __all_sync(0xffffffffu, ok);
-        if (!ok) break;
-      }
+    for (int hs = half; hs < n_hs; hs += kKvNB) {
+      const int j = hs / kKvNB;
+      ok = mbar_wait(bars + B_STF + (j & 1), (j >> 1) & 1, a.error_word, 4);   // statistics and entries of step j
+      ok = __all_sync(0xffffffffu, ok);
+      if (!ok) break;
       // -LSE2 and -delta of my C queries, four to a load
       const float4* st_l = reinterpret_cast<const float4*>(sStat + (j & 1) * 256 + half * kKvHalf + g * C);
       const float4* st_d = st_l + 128 / 4;
@@ -855,29 +829,19 @@ bwd_dkdv_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
       }
       if constexpr (C == 16) tmem_st8(dp_addr, dsreg); else tmem_st16(dp_addr, dsreg);                               // dS^T over my own dP^T columns
       if constexpr (kSpill) {
-        static_assert(!kSpill || (C == 16 && kKvNB == 2), "the kept tiles are laid out for half-steps of 64 queries");
-        // ... and into this half's tile in shared memory: my 16 queries are two 16-byte chunks of my key's
-        // 128-byte row (128-byte swizzle, the layout the stored tensor map expects).  The tile is free once
-        // the store of the half-step two before this one has read it.
-        if (j >= 1) {
-          ok = mbar_wait(bars + B_DSE + half, (j - 1) & 1, a.error_word, 42);
-          ok = __all_sync(0xffffffffu, ok);
-          if (!ok) break;
-        }
-        const uint32_t base = smem_u32(sDS) + half * SM::kDs + r * 128;
-        asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(base + (((2 * g) ^ (r & 7)) << 4)), "r"(dsreg[0]),
-                     "r"(dsreg[1]), "r"(dsreg[2]), "r"(dsreg[3]) : "memory");
-        asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(base + (((2 * g + 1) ^ (r & 7)) << 4)), "r"(dsreg[4]),
-                     "r"(dsreg[5]), "r"(dsreg[6]), "r"(dsreg[7]) : "memory");
-        fence_proxy_async_smem();
-        __syncwarp();
-        if (lane == 0) mbar_arrive(bars + B_DSS + half);
+        static_assert(!kSpill || (C == 32 && kKvNB == 2), "the kept tiles are laid out for half-steps of 64 queries");
+        // ... and to this half-step's tile in global memory: my 32 queries are four 16-byte groups of my
+        // key.  (Written once, read once by the dQ pass: marked evict-first so that the stream does not
+        // push the Q / dO tiles, which every kv tile of a window re-reads, out of the L2.)
+        uint8_t* dst = reinterpret_cast<uint8_t*>(a.ds_buf) + sTile[(j & 1) * 2 + half] * kDsTileBytes + (4 * g) * 2048 + r * 16;
+#pragma unroll
+        for (int i = 0; i < 4; ++i)
+          asm volatile("st.global.L2::cache_hint.v4.b32 [%0], {%1, %2, %3, %4}, %5;" ::"l"(dst + i * 2048),
+                       "r"(dsreg[4 * i]), "r"(dsreg[4 * i + 1]), "r"(dsreg[4 * i + 2]), "r"(dsreg[4 * i + 3]), "l"(evict_first) : "memory");
       }
       ew_publish(bars + B_DSF + half);
-      if (closes_step(hs)) {   // this warp is done with the statistics of step j
-        __syncwarp();
-        if (lane == 0) mbar_arrive(bars + B_STE + (j & 1));
-      }
+      __syncwarp();   // this warp is done with the statistics of step j
+      if (lane == 0) mbar_arrive(bars + B_STE + (j & 1));
     }
     // ---- epilogue: dV, dK * scale -> bf16 ---------------------------------------------------
     if (ok && n_hs > 0) {
@@ -888,12 +852,13 @@ bwd_dkdv_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
       tc_fence_after();
       constexpr int kEpi = 32;                               // output columns per thread
       const bool mine = kj < a.L;                            // keys past L take part in the loads only
-      if (kb_mine >= 0 && g * kEpi < D) {
-        __nv_bfloat16* dk_row = a.out0 + b * a.s0[0] + hk * a.s0[1] + static_cast<int64_t>(kj) * a.s0[2] + g * kEpi;
-        __nv_bfloat16* dv_row = a.out1 + b * a.s1[0] + hk * a.s1[1] + static_cast<int64_t>(kj) * a.s1[2] + g * kEpi;
+      const int ge = warp >> 2;                              // the sixteen warps share the D output columns
+      if (kb_mine >= 0 && ge * kEpi < D) {
+        __nv_bfloat16* dk_row = a.out0 + b * a.s0[0] + hk * a.s0[1] + static_cast<int64_t>(kj) * a.s0[2] + ge * kEpi;
+        __nv_bfloat16* dv_row = a.out1 + b * a.s1[0] + hk * a.s1[1] + static_cast<int64_t>(kj) * a.s1[2] + ge * kEpi;
         if (n_hs > 0) {
-          store_acc_cols<kEpi>(lane_addr + kColDV + g * kEpi, dv_row, 1.0f, mine);
-          store_acc_cols<kEpi>(lane_addr + kColDK + g * kEpi, dk_row, a.scale, mine);
+          store_acc_cols<kEpi>(lane_addr + kColDV + ge * kEpi, dv_row, 1.0f, mine);
+          store_acc_cols<kEpi>(lane_addr + kColDK + ge * kEpi, dk_row, a.scale, mine);
         } else if (mine) {
 #pragma unroll
           for (int x = 0; x < kEpi; x += 8) {
@@ -911,15 +876,16 @@ bwd_dkdv_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
 
 // ============================== dQ from the kept dS ===========================================
 // dQ(128 queries x D) = scale * sum over the kv tiles of the row of dS(128 queries x 128 keys) K(128 keys x D),
-// with dS^T read back from the tiles the dK/dV pass left in global memory (one tile of [128 keys][64
-// queries] per half of the query tile; a half without an entry in that kv tile reads the tile of zeros):
+// with dS^T read back from the tiles the dK/dV pass left in global memory (one tile of 64 queries x 128
+// keys per half of the query tile, in the core-matrix layout described at BwdArgs::ds_buf, copied as it
+// is and used as an un-swizzled operand; a half without an entry in that kv tile reads the tile of zeros):
 // one product per step, no exponentials, nothing recomputed.  The kernel is a plain pipelined
 // contraction -- warp 4 loads (a ring of dS^T tile pairs and a ring of K tiles), warp 5 issues, warps
 // 0-3 write the result -- and is bound by the HBM reads of dS.
 template <int D>
 struct DqDsSmem {
   static constexpr int kTile = BwdTile<D>::kBytes;
-  static constexpr int kDs2 = 2 * 128 * 128;                   // dS^T of a step: two tiles of [128 keys][64 queries]
+  static constexpr int kDs2 = 2 * kDsTileBytes;                // dS^T of a step: the tiles of the two halves of the query tile
   static constexpr int kAStages = (D == 128) ? 4 : 5;          // dS^T comes from HBM: the deeper ring
   static constexpr int kKStages = 3;                           // K comes from the L2
   static constexpr int oA = 0;
@@ -931,7 +897,7 @@ constexpr int kDq2Threads = 6 * 32;
 
 template <int D, int BS>
 __global__ void __launch_bounds__(kDq2Threads, 1)
-bwd_dq_from_ds_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__ CUtensorMap tm_ds, const BwdArgs a) {
+bwd_dq_from_ds_kernel(const __grid_constant__ CUtensorMap tm_k, const BwdArgs a) {
   using SM = DqDsSmem<D>;
   constexpr int kAS = SM::kAStages, kKS = SM::kKStages;
   constexpr int R = 128 / BS;
@@ -977,7 +943,7 @@ bwd_dq_from_ds_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_con
   if (warp == 4) {
     // ------------------------------ TMA producer ------------------------------------------
     if (lane == 0) {
-      tma_prefetch_desc(&tm_k); tma_prefetch_desc(&tm_ds);
+      tma_prefetch_desc(&tm_k);
       uint64_t evict_first;
       asm volatile("createpolicy.fractional.L2::evict_first.b64 %0, 1.0;" : "=l"(evict_first));   // dS tiles are read once
       const int64_t head_base = (static_cast<int64_t>(b) * a.Hq + h) * a.ds_nnz * (BS / 64);
@@ -997,12 +963,8 @@ bwd_dq_from_ds_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_con
         for (int half = 0; half < 2; ++half) {
           const int hx = half ? h1 : h0;
           const int64_t tile_idx = hx >= 0 ? head_base + hx : zero_tile;
-          asm volatile(
-              "cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes.L2::cache_hint [%0], [%1, {%3, %4}], [%2], %5;" ::"r"(
-                  smem_u32(dA + half * (SM::kDs2 / 2))),
-              "l"(reinterpret_cast<uint64_t>(&tm_ds)), "r"(smem_u32(bars + B_AF + sa)), "r"(0),
-              "r"(static_cast<int>(tile_idx * 128)), "l"(evict_first)
-              : "memory");
+          bulk_load_hint(dA + half * kDsTileBytes, reinterpret_cast<const uint8_t*>(a.ds_buf) + tile_idx * kDsTileBytes,
+                         kDsTileBytes, bars + B_AF + sa, evict_first);
         }
         if (x >= kKS) ok = mbar_wait(bars + B_KE + sk, ((x / kKS) - 1) & 1, a.error_word, 86);
         if (!ok) break;
@@ -1025,7 +987,9 @@ bwd_dq_from_ds_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_con
     const bool lead = elect_one();
     constexpr uint32_t idesc = make_idesc_bf16(128, D, 1, 1);   // A = dS^T and B = K, both MN-major
     const uint32_t hi = desc_hi(1024);
-    const uint32_t a_lo0 = desc_lo(smem_u32(smem + SM::oA), SM::kDs2 / 2), k_lo0 = desc_lo(smem_u32(smem + SM::oK), BwdTile<D>::kBox);
+    // A without swizzle: groups of 8 keys are 128 bytes apart (leading offset), groups of 8 queries 2048 bytes (stride offset)
+    const uint32_t a_hi = desc_hi(2048, 0);
+    const uint32_t a_lo0 = desc_lo(smem_u32(smem + SM::oA), 128), k_lo0 = desc_lo(smem_u32(smem + SM::oK), BwdTile<D>::kBox);
     bool ok = true;
 #pragma unroll 1
     for (int x = 0; x < n_ent; ++x) {
@@ -1037,7 +1001,7 @@ bwd_dq_from_ds_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_con
         const uint32_t a_lo = a_lo0 + sa * (SM::kDs2 >> 4), b_lo = k_lo0 + sk * (kTile >> 4);
 #pragma unroll
         for (int kk = 0; kk < 8; ++kk)
-          if (lead) mma_ss2(tmem, a_lo + kk * (2048 >> 4), b_lo + kk * (2048 >> 4), hi, idesc, (x > 0) || (kk > 0));
+          if (lead) mma_ss2x(tmem, a_lo + kk * (256 >> 4), a_hi, b_lo + kk * (2048 >> 4), hi, idesc, (x > 0) || (kk > 0));
       }
       if (lead) { mma_commit(bars + B_AE + sa); mma_commit(bars + B_KE + sk); }
     }

@@ -87,7 +87,6 @@ BwdVariant bwd_variant(const Resolved& r);
 // bytes of the dS^T buffer of the kBwdKeepDs variant
 size_t ds_buffer_bytes(const Resolved& r);
 
-lg_status make_tmap_ds(CUtensorMap* out, const void* base, int64_t rows);
 
 lg_status check_arch();
 inline bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15) == 0; }
