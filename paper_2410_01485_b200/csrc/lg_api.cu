@@ -116,9 +116,9 @@ lg_status resolve(const lg_attn_params* p, Resolved* r) {
 // Two backward variants compute the same gradients (see BwdVariant).  The two passes run everywhere.
 // Keeping dS trades workspace and HBM traffic (2 bytes per visible pair, written once and read once, on
 // a memory system the attention kernels otherwise leave idle) for the two recomputed products of the dQ
-// pass.  It is the default for 128-token blocks (with 64-token blocks the two variants were measured
-// equal) when the lists are shared by the batch and the dS buffer takes at most LG_KEEP_DS_MAX_GB
-// (default 48) gigabytes.  LG_BWD_VARIANT = two_pass | keep_ds overrides the choice (read at every call;
+// pass.  It is the default when the lists are shared by the batch and the dS buffer takes at most
+// LG_KEEP_DS_MAX_GB (default 48) gigabytes; the buffer is block-granular, so a strided pattern with
+// 64-token blocks, whose kv tiles pair columns with different rows, can need twice its visible pairs.  LG_BWD_VARIANT = two_pass | keep_ds overrides the choice (read at every call;
 // it must not change between a size query, a prepare and the calls that use them).
 size_t ds_buffer_bytes(const Resolved& r) {   // every tile of 64 queries x 128 keys, plus one tile of zeros at the end
   return (static_cast<size_t>(r.B) * r.Hq * static_cast<size_t>(r.nnz) * (r.block / 64) + 1) * static_cast<size_t>(128 * 64 * 2);
@@ -132,8 +132,7 @@ BwdVariant bwd_variant(const Resolved& r) {
   if (env && strcmp(env, "keep_ds") == 0) return can_keep ? kBwdKeepDs : kBwdTwoPass;
   double max_gb = 48.0;
   if (const char* m = getenv("LG_KEEP_DS_MAX_GB")) max_gb = atof(m);
-  return (can_keep && r.block == 128 && static_cast<double>(ds_buffer_bytes(r)) <= max_gb * 1e9) ? kBwdKeepDs
-                                                                                                  : kBwdTwoPass;
+  return (can_keep && static_cast<double>(ds_buffer_bytes(r)) <= max_gb * 1e9) ? kBwdKeepDs : kBwdTwoPass;
 }
 
 WsLayout ws_layout(const Resolved& r, bool want_bwd) {

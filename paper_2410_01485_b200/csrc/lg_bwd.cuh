@@ -584,22 +584,47 @@ bwd_dkdv_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
         ds_tile = ((static_cast<int64_t>(b) * a.Hq + hq) * a.ds_nnz + ent_off + e) * (BS / 64);
         if (++e == n_ent) { e = 0; ++grp; }
       };
-      for (int j = 0; j < n_steps; ++j) {
-        const int sq = j % kQS, so = j & 1;
-        int h0, r0, e0, h1, r1, e1;
-        int64_t t0, t1;
-        next_item(h0, r0, e0, t0);
-        h1 = h0; r1 = r0; e1 = e0 & ~3; t1 = t0 + 1;            // a missing second item repeats the first block, as nobody's member
-        if (BS == 64 && 2 * j + 1 < n_items) next_item(h1, r1, e1, t1);
+      // Each load is started as soon as its ring slot is free, in the order in which the slots come
+      // free: dO of step j (its slot is released when the dV and dP^T products of step j - 2 are done),
+      // the statistics of step j (released by the element-wise warps at the end of step j - 2), then Q
+      // of step j + 1 (three stages: the slot of step j - 2, released by its dK product).  Q is the first
+      // operand a step needs -- S^T of step j + 1 is issued early in step j -- hence the step of lead.
+      struct Item { int h, r, e; int64_t t; };
+      auto step_items = [&](int j, Item& i0, Item& i1) {
+        next_item(i0.h, i0.r, i0.e, i0.t);
+        i1 = i0; i1.e = i0.e & ~3; i1.t = i0.t + 1;             // a missing second item repeats the first block, as nobody's member
+        if (BS == 64 && 2 * j + 1 < n_items) next_item(i1.h, i1.r, i1.e, i1.t);
+      };
+      auto load_q = [&](int j, const Item& i0, const Item& i1) {
+        const int sq = j % kQS;
+        if (j >= kQS) ok = mbar_wait(bars + B_QE + sq, ((j / kQS) - 1) & 1, a.error_word, 11);
+        if (!ok) return;
+        mbar_expect_tx(bars + B_QF + sq, kTile);
+        tma_load_rows<D, BS>(sQ + sq * kTile, &tm_q, bars + B_QF + sq, 0, i0.r, i0.h, b);
+        if (BS == 64) tma_load_rows<D, BS>(sQ + sq * kTile, &tm_q, bars + B_QF + sq, 1, i1.r, i1.h, b);
+        nq = j + 1;
+      };
+      Item c0, c1, n0, n1;   // items of step j and of step j + 1
+      if (n_steps > 0) { step_items(0, n0, n1); load_q(0, n0, n1); }
+      for (int j = 0; j < n_steps && ok; ++j) {
+        const int so = j & 1;
+        c0 = n0; c1 = n1;
+        if (j + 1 < n_steps) step_items(j + 1, n0, n1);
+        if (j >= 2) ok = mbar_wait(bars + B_OE + so, ((j / 2) - 1) & 1, a.error_word, 12);
+        if (!ok) break;
+        mbar_expect_tx(bars + B_OF + so, kTile);
+        tma_load_rows<D, BS>(sDO + so * kTile, &tm_do, bars + B_OF + so, 0, c0.r, c0.h, b);
+        if (BS == 64) tma_load_rows<D, BS>(sDO + so * kTile, &tm_do, bars + B_OF + so, 1, c1.r, c1.h, b);
+        no = j + 1;
         if (j >= 2) ok = mbar_wait(bars + B_STE + so, ((j / 2) - 1) & 1, a.error_word, 40);
         if (!ok) break;
-        sEnt[so * 2] = e0;
-        sEnt[so * 2 + 1] = e1;
-        if (kSpill) { sTile[so * 2] = t0; sTile[so * 2 + 1] = t1; }   // (128-token blocks: the two halves of the one item)
+        sEnt[so * 2] = c0.e;
+        sEnt[so * 2 + 1] = c1.e;
+        if (kSpill) { sTile[so * 2] = c0.t; sTile[so * 2 + 1] = c1.t; }   // (128-token blocks: the two halves of the one item)
         mbar_expect_tx(bars + B_STF + so, 2 * 128 * 4);         // (release: publishes the entries as well)
         {
-          const float* st0 = a.stat + (static_cast<int64_t>(b) * a.Hq + h0) * a.Lp + r0;
-          const float* st1 = a.stat + (static_cast<int64_t>(b) * a.Hq + h1) * a.Lp + r1;
+          const float* st0 = a.stat + (static_cast<int64_t>(b) * a.Hq + c0.h) * a.Lp + c0.r;
+          const float* st1 = a.stat + (static_cast<int64_t>(b) * a.Hq + c1.h) * a.Lp + c1.r;
 #pragma unroll
           for (int pl = 0; pl < 2; ++pl) {
             float* dst = sStat + (so * 2 + pl) * 128;
@@ -612,18 +637,7 @@ bwd_dkdv_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
           }
         }
         nst = j + 1;
-        if (j >= kQS) ok = mbar_wait(bars + B_QE + sq, ((j / kQS) - 1) & 1, a.error_word, 11);
-        if (!ok) break;
-        mbar_expect_tx(bars + B_QF + sq, kTile);
-        tma_load_rows<D, BS>(sQ + sq * kTile, &tm_q, bars + B_QF + sq, 0, r0, h0, b);
-        if (BS == 64) tma_load_rows<D, BS>(sQ + sq * kTile, &tm_q, bars + B_QF + sq, 1, r1, h1, b);
-        nq = j + 1;
-        if (j >= 2) ok = mbar_wait(bars + B_OE + so, ((j / 2) - 1) & 1, a.error_word, 12);
-        if (!ok) break;
-        mbar_expect_tx(bars + B_OF + so, kTile);
-        tma_load_rows<D, BS>(sDO + so * kTile, &tm_do, bars + B_OF + so, 0, r0, h0, b);
-        if (BS == 64) tma_load_rows<D, BS>(sDO + so * kTile, &tm_do, bars + B_OF + so, 1, r1, h1, b);
-        no = j + 1;
+        if (j + 1 < n_steps) load_q(j + 1, n0, n1);
       }
       mbar_wait(bars + B_FIX, 0, a.error_word, 16);
       for (int j = max(nq - kQS, 0); j < nq; ++j) mbar_wait(bars + B_QF + j % kQS, (j / kQS) & 1, a.error_word, 17);

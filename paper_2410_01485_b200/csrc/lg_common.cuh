@@ -116,6 +116,8 @@ __device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, unsign
 // every lane.
 __device__ __forceinline__ bool mbar_wait_warp(uint64_t* bar, uint32_t parity, unsigned int* error_word,
                                                uint32_t site) {
+  // common case: the phase is over already and every lane sees that with one probe of its own
+  if (__all_sync(0xffffffffu, mbar_try_wait(bar, parity))) return true;
   bool ok = true;
   if (lane_id() == 0) ok = mbar_wait(bar, parity, error_word, site);
   ok = __all_sync(0xffffffffu, ok);

@@ -15,9 +15,10 @@
 //   S_0(0) S_1(0) | PV_0(0) S_0(1) | PV_1(0) S_1(1) | PV_0(1) S_0(2) | ...
 // so the two halves of a slot form a double buffer: while the softmax works on one half the
 // tensor pipe computes the other, and the second slot fills what is left.  The online softmax
-// advances half by half.  The running maximum is only raised (and O rescaled) when it grew by
-// more than 2^8; until then probabilities are expressed relative to the older maximum, which
-// fp32 / bf16 hold easily.
+// advances half by half.  A row's reference (the maximum its probabilities are expressed relative
+// to) only moves, and O is only rescaled, when a half's probabilities sum to more than 2^8;
+// until then they are relative to the older reference, which fp32 / bf16 hold easily, and the
+// row maximum is not computed at all.
 #pragma once
 #include <cuda.h>
 #include "lg_common.cuh"
@@ -49,7 +50,7 @@ struct FwdArgs {
 
 constexpr int kFwdTmaWarp = 8, kFwdMmaWarp0 = 9;
 constexpr int kFwdThreads = 11 * 32;
-constexpr float kFwdRescaleThreshold = 8.0f;   // log2 units
+constexpr float kFwdMaxProb = 256.0f;   // a half's probabilities may grow to this (relative to the row's reference) before the reference moves
 template <int D>
 struct FwdSmem {
   static constexpr int kBox = 128 * 128;               // one 64-column box of 128 rows
@@ -308,22 +309,48 @@ fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUt
           for (int x = 0; x < 64; ++x)
             v[x] = (x < lim && x >= lo) ? v[x] : 0xff800000u;   // -inf: the exponential below gives exactly 0
         }
-        float mx;
-        {
-          float m0 = -INFINITY, m1 = -INFINITY, m2 = -INFINITY, m3 = -INFINITY;
+        // Probabilities relative to the reference as it stands; the row maximum is only looked at when
+        // that cannot be right: the row has no reference yet, or the sum of the half's probabilities
+        // (an upper bound of each of them) passes 2^8.  Otherwise every probability is below 2^8 and the
+        // reference stays -- the maximum, its 32 instructions per row and the vote are off the common path.
+        uint32_t preg[32];
+        float psum;
+        auto exp_half = [&](float neg_m) {
+          float q0 = 0.f, q1 = 0.f, q2 = 0.f, q3 = 0.f;   // independent partial sums
 #pragma unroll
-          for (int x = 0; x < 64; x += 8) {
-            m0 = max3(m0, __uint_as_float(v[x + 0]), __uint_as_float(v[x + 1]));
-            m1 = max3(m1, __uint_as_float(v[x + 2]), __uint_as_float(v[x + 3]));
-            m2 = max3(m2, __uint_as_float(v[x + 4]), __uint_as_float(v[x + 5]));
-            m3 = max3(m3, __uint_as_float(v[x + 6]), __uint_as_float(v[x + 7]));
+          for (int x = 0; x < 64; x += 4) {
+            const float x0 = fmaf(__uint_as_float(v[x]), a.scale_log2, neg_m);
+            const float x1 = fmaf(__uint_as_float(v[x + 1]), a.scale_log2, neg_m);
+            const float x2 = fmaf(__uint_as_float(v[x + 2]), a.scale_log2, neg_m);
+            const float x3 = fmaf(__uint_as_float(v[x + 3]), a.scale_log2, neg_m);
+            const float e0 = fast_exp2(x0), e1 = fast_exp2(x1), e2 = fast_exp2(x2), e3 = fast_exp2(x3);
+            q0 += e0; q1 += e1; q2 += e2; q3 += e3;
+            preg[x >> 1] = pack_bf16(e0, e1);
+            preg[(x >> 1) + 1] = pack_bf16(e2, e3);
           }
-          mx = fmaxf(fmaxf(m0, m1), fmaxf(m2, m3));
-        }
-        const float m_new = fmaxf(m_ref, mx * a.scale_log2);
-        // raise the reference only when it would grow by more than the threshold (or is still unset)
-        const bool raise = (m_new > m_ref + kFwdRescaleThreshold) || (m_ref == -INFINITY && m_new > -INFINITY);
-        if (__any_sync(0xffffffffu, raise)) {
+          psum = (q0 + q2) + (q1 + q3);
+        };
+        const bool unset = (m_ref == -INFINITY);
+        exp_half(unset ? 0.f : -m_ref);
+        // (an unset reference with every column masked gives zeros and stays unset; NaN compares false
+        // and cannot appear: masked scores are -inf, whose exponential is 0)
+        const bool look = unset ? (lim > lo) : !(psum <= kFwdMaxProb);
+        if (__any_sync(0xffffffffu, look)) {
+          float mx;
+          {
+            float m0 = -INFINITY, m1 = -INFINITY, m2 = -INFINITY, m3 = -INFINITY;
+#pragma unroll
+            for (int x = 0; x < 64; x += 8) {
+              m0 = max3(m0, __uint_as_float(v[x + 0]), __uint_as_float(v[x + 1]));
+              m1 = max3(m1, __uint_as_float(v[x + 2]), __uint_as_float(v[x + 3]));
+              m2 = max3(m2, __uint_as_float(v[x + 4]), __uint_as_float(v[x + 5]));
+              m3 = max3(m3, __uint_as_float(v[x + 6]), __uint_as_float(v[x + 7]));
+            }
+            mx = fmaxf(fmaxf(m0, m1), fmaxf(m2, m3));
+          }
+          // the rows that asked move their reference to the maximum seen so far (the others keep theirs)
+          const float m_new = fmaxf(m_ref, mx * a.scale_log2);
+          const bool raise = look && m_new > m_ref;
           const float alpha = raise ? fast_exp2(m_ref - m_new) : 1.f;   // m_ref = -inf -> 0
           if (raise) { m_ref = m_new; l_run *= alpha; }
           if (p0 + p1 > 0) {   // O already holds products: wait for them, then rescale my row
@@ -340,22 +367,9 @@ fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUt
               tmem_st16(my_o + c * 16, oreg);
             }
           }
+          exp_half((m_ref == -INFINITY) ? 0.f : -m_ref);
         }
-        const float neg_m = (m_ref == -INFINITY) ? 0.f : -m_ref;
-        uint32_t preg[32];
-        float q0 = 0.f, q1 = 0.f, q2 = 0.f, q3 = 0.f;   // independent partial sums
-#pragma unroll
-        for (int x = 0; x < 64; x += 4) {
-          const float x0 = fmaf(__uint_as_float(v[x]), a.scale_log2, neg_m);
-          const float x1 = fmaf(__uint_as_float(v[x + 1]), a.scale_log2, neg_m);
-          const float x2 = fmaf(__uint_as_float(v[x + 2]), a.scale_log2, neg_m);
-          const float x3 = fmaf(__uint_as_float(v[x + 3]), a.scale_log2, neg_m);
-          const float p0 = fast_exp2(x0), p1 = fast_exp2(x1), p2 = fast_exp2(x2), p3 = fast_exp2(x3);
-          q0 += p0; q1 += p1; q2 += p2; q3 += p3;
-          preg[x >> 1] = pack_bf16(p0, p1);
-          preg[(x >> 1) + 1] = pack_bf16(p2, p3);
-        }
-        l_run += (q0 + q2) + (q1 + q3);
+        l_run += psum;
         tmem_st32(my_s + hf * 64, preg);   // P over the first columns of this half's S
         tmem_st_wait();
         tc_fence_before();
