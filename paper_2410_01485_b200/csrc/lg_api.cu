@@ -117,11 +117,10 @@ lg_status resolve(const lg_attn_params* p, Resolved* r) {
 // Keeping dS trades workspace and HBM traffic (2 bytes per visible pair, written once and read once, on
 // a memory system the attention kernels otherwise leave idle) for the two recomputed products of the dQ
 // pass.  It is the default when the lists are shared by the batch and the dS buffer takes at most
-// LG_KEEP_DS_MAX_GB (default 48) gigabytes; the buffer is block-granular, so a strided pattern with
-// 64-token blocks, whose kv tiles pair columns with different rows, can need twice its visible pairs.  LG_BWD_VARIANT = two_pass | keep_ds overrides the choice (read at every call;
+// LG_KEEP_DS_MAX_GB (default 48) gigabytes (the buffer holds every block of the pattern in full).  LG_BWD_VARIANT = two_pass | keep_ds overrides the choice (read at every call;
 // it must not change between a size query, a prepare and the calls that use them).
-size_t ds_buffer_bytes(const Resolved& r) {   // every tile of 64 queries x 128 keys, plus one tile of zeros at the end
-  return (static_cast<size_t>(r.B) * r.Hq * static_cast<size_t>(r.nnz) * (r.block / 64) + 1) * static_cast<size_t>(128 * 64 * 2);
+size_t ds_buffer_bytes(const Resolved& r) {   // 2 bytes per pair of every block of the pattern and query head, plus one tile of zeros at the end
+  return static_cast<size_t>(r.B) * r.Hq * static_cast<size_t>(r.nnz) * r.block * r.block * 2 + 128 * 64 * 2;
 }
 
 BwdVariant bwd_variant(const Resolved& r) {
@@ -165,7 +164,7 @@ WsLayout ws_layout(const Resolved& r, bool want_bwd) {
     if (bwd_variant(r) == kBwdKeepDs) {
       w.kt_tile_of = take(nB * 4);
       w.dq_cnt = take(static_cast<size_t>(r.n_qtiles) * 4);
-      w.dq_ent = take(nnz * 3 * 4);
+      w.dq_ent = take(nnz * kDqEntInts * 4);
       w.ds_buf = take(ds_buffer_bytes(r));
     }
   }
@@ -240,8 +239,8 @@ lg_status prepare_workspace(const Resolved& r, const WsLayout& w, uint8_t* ws, i
     tile_order_kernel<<<(nt + 127) / 128, 128, 0, stream>>>(i32(w.kt_cnt), nt, i32(w.kt_order)); note_launch();
     if (bwd_variant(r) == kBwdKeepDs) {   // which dS tiles each query tile reads back
       kv_tile_of_kernel<<<(nt * R + 127) / 128, 128, 0, stream>>>(i32(w.kt_cols), R, nt, i32(w.kt_tile_of)); note_launch();
-      dq_sched_kernel<<<(r.n_qtiles + 63) / 64, 64, 0, stream>>>(i32(w.row_ptr), i32(w.col_idx), i32(w.kt_tile_of),
-                                                                  i32(w.kt_off), i32(w.kt_cnt), i32(w.kt_ent), R, nB,
+      dq_sched_kernel<<<(r.n_qtiles + 63) / 64, 64, 0, stream>>>(i32(w.row_ptr), i32(w.col_idx), i32(w.col_ptr),
+                                                                  i32(w.row_idx), i32(w.kt_tile_of), i32(w.kt_cols), R, nB,
                                                                   r.n_qtiles, i32(w.dq_cnt), i32(w.dq_ent)); note_launch();
     }
     if (r.doc_start) {

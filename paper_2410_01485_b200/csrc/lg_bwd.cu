@@ -37,6 +37,7 @@ static lg_status launch_bwd_t(const Resolved& r, const WsLayout& w, const void* 
   a.scale_log2 = r.scale * 1.4426950408889634f;
   a.ds_nnz = r.nnz;
   a.ds_buf = reinterpret_cast<__nv_bfloat16*>(ws + w.ds_buf);
+  a.col_ptr = reinterpret_cast<const int32_t*>(ws + w.col_ptr);
   constexpr int smem = BwdSmem<D, BS>::kTotal;
   const BwdVariant variant = bwd_variant(r);
 
@@ -58,7 +59,7 @@ static lg_status launch_bwd_t(const Resolved& r, const WsLayout& w, const void* 
     dim3 grid(r.B * r.Hkv, r.n_ktiles);
     if (variant == kBwdKeepDs) {
       // the tile of zeros that stands in for a half of a query tile a kv tile has no entry for
-      if (cudaMemsetAsync(ws + w.ds_buf + ds_buffer_bytes(r) - kDsTileBytes, 0, kDsTileBytes, stream) != cudaSuccess) return LG_ERR_CUDA;
+      if (cudaMemsetAsync(ws + w.ds_buf + ds_buffer_bytes(r) - 128 * 64 * 2, 0, 128 * 64 * 2, stream) != cudaSuccess) return LG_ERR_CUDA;
       auto kern = bwd_dkdv_kernel<D, BS, true>;
       if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, smem) != cudaSuccess)
         return LG_ERR_CUDA;

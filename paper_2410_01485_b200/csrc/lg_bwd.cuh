@@ -53,17 +53,20 @@ struct BwdArgs {
   const int32_t* doc_start;  // [B, L] first position of each token's document, or null
   const int32_t* doc_end;    // [B, L] end of each token's document (null together with doc_start)
   float scale, scale_log2;
-  // dK/dV pass that also keeps dS (see bwd_dkdv_kernel): dS^T of every half-step of 64 queries goes to
-  // ds_buf as a tile of 16 KB; tile index = ((b * Hq + h) * ds_nnz + schedule position of the (kv tile,
-  // query block) entry) * (block / 64) + half.  The dQ pass then reads them back.  Inside a tile the
-  // element (key k, query q) sits at byte (q / 8) * 2048 + k * 16 + (q % 8) * 2: eight queries of one key
-  // are 16 contiguous bytes, the 128 keys of such a group follow one another -- the un-swizzled
-  // core-matrix layout of a tensor-core operand whose M (query) index is the contiguous one, and a
-  // layout in which the 32 key rows of a warp write 512 contiguous bytes per store instruction.
+  // dK/dV pass that also keeps dS (see bwd_dkdv_kernel): dS^T of every block of the pattern goes to ds_buf
+  // in tiles of 64 queries x KT keys, KT = the block size: with p = the block's position in the column
+  // lists (col_ptr[column] + rank of the query block in the column), a head's tiles are 2 p and 2 p + 1
+  // (the block's two 64-query halves, 16 KB each) with 128-token blocks and p (8 KB) with 64-token
+  // blocks; head (b, h) starts at tile (b * Hq + h) * ds_nnz * (block / 64).  The dQ pass reads them back.
+  // Inside a tile the element (key k, query q) sits at byte (q / 8) * 16 KT + k * 16 + (q % 8) * 2: eight
+  // queries of one key are 16 contiguous bytes, the KT keys of such a group follow one another -- the
+  // un-swizzled core-matrix layout of a tensor-core operand whose M (query) index is the contiguous one,
+  // and a layout in which the 32 key rows of a warp write 512 contiguous bytes per store instruction.
   int64_t ds_nnz;
   __nv_bfloat16* ds_buf;
+  const int32_t* col_ptr;    // column lists of the pattern (dK/dV pass that keeps dS: positions of its blocks)
 };
-constexpr int kDsTileBytes = 128 * 64 * 2;
+template <int BS> constexpr int kDsTileBytes = BS * 64 * 2;
 
 // ---- stat = -(LSE * log2 e) and -rowsum(dO * O), stored negated (they are only ever subtracted),
 // each in a plane of its own: the dK/dV pass fetches four neighbouring queries' values of one kind
@@ -496,8 +499,8 @@ bwd_dkdv_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
   uint64_t* bars = reinterpret_cast<uint64_t*>(smem + SM::oBar);
   uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + B_COUNT);
   int32_t* sEnt = reinterpret_cast<int32_t*>(bars + B_COUNT + 1);   // [2][2]: entries of a step's items
-  int64_t* sTile = reinterpret_cast<int64_t*>(bars + B_COUNT + 3);  // [2][2]: dS tile index of a step's items (kSpill)
-  static_assert((B_COUNT + 3) * 8 + 32 <= SM::kBarBytes, "barrier area too small");
+  int64_t* sTile = reinterpret_cast<int64_t*>(bars + B_COUNT + 3);  // [2][2][2]: dS tile of (half-step, member) of a step (kSpill)
+  static_assert((B_COUNT + 3) * 8 + 64 <= SM::kBarBytes, "barrier area too small");
   const int tid = threadIdx.x, lane = tid & 31;
   const int warp = __shfl_sync(0xffffffffu, tid >> 5, 0);   // same value, known to be warp-uniform
   if ((smem_u32(smem) & 1023u) != 0) {
@@ -577,23 +580,31 @@ bwd_dkdv_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
       bool ok = true;
       int nq = 0, no = 0, nst = 0;   // loads started
       int grp = 0, e = 0;            // (query head within the group, entry) of the next item
-      auto next_item = [&](int& hq, int& qrow, int& entry, int64_t& ds_tile) {
+      // positions, in the column lists, of the members' next blocks: the entries that carry a member's bit
+      // are that column's query blocks in ascending order
+      const int pos_a0 = (kSpill && kb_a >= 0) ? a.col_ptr[kb_a] : 0, pos_b0 = (kSpill && kb_b >= 0) ? a.col_ptr[kb_b] : 0;
+      int pos_a = pos_a0, pos_b = pos_b0;
+      auto next_item = [&](int& hq, int& qrow, int& entry, int64_t& ta, int64_t& tb) {
         entry = ent[e];
         hq = hk * a.G + grp;
         qrow = checked(entry >> 2, 0, a.nB - 1, a.error_word, 125) * BS;   // (also the address of the item's statistics)
-        ds_tile = ((static_cast<int64_t>(b) * a.Hq + hq) * a.ds_nnz + ent_off + e) * (BS / 64);
-        if (++e == n_ent) { e = 0; ++grp; }
+        const int64_t head_base = (static_cast<int64_t>(b) * a.Hq + hq) * a.ds_nnz;
+        ta = (head_base + pos_a) * (BS / 64);
+        tb = (head_base + pos_b) * (BS / 64);
+        pos_a += entry & 1;
+        pos_b += (entry >> 1) & 1;
+        if (++e == n_ent) { e = 0; ++grp; pos_a = pos_a0; pos_b = pos_b0; }
       };
       // Each load is started as soon as its ring slot is free, in the order in which the slots come
       // free: dO of step j (its slot is released when the dV and dP^T products of step j - 2 are done),
       // the statistics of step j (released by the element-wise warps at the end of step j - 2), then Q
       // of step j + 1 (three stages: the slot of step j - 2, released by its dK product).  Q is the first
       // operand a step needs -- S^T of step j + 1 is issued early in step j -- hence the step of lead.
-      struct Item { int h, r, e; int64_t t; };
+      struct Item { int h, r, e; int64_t ta, tb; };
       auto step_items = [&](int j, Item& i0, Item& i1) {
-        next_item(i0.h, i0.r, i0.e, i0.t);
-        i1 = i0; i1.e = i0.e & ~3; i1.t = i0.t + 1;             // a missing second item repeats the first block, as nobody's member
-        if (BS == 64 && 2 * j + 1 < n_items) next_item(i1.h, i1.r, i1.e, i1.t);
+        next_item(i0.h, i0.r, i0.e, i0.ta, i0.tb);
+        i1 = i0; i1.e = i0.e & ~3; i1.ta = i0.ta + 1;           // a missing second item repeats the first block, as nobody's member
+        if (BS == 64 && 2 * j + 1 < n_items) next_item(i1.h, i1.r, i1.e, i1.ta, i1.tb);
       };
       auto load_q = [&](int j, const Item& i0, const Item& i1) {
         const int sq = j % kQS;
@@ -620,7 +631,10 @@ bwd_dkdv_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
         if (!ok) break;
         sEnt[so * 2] = c0.e;
         sEnt[so * 2 + 1] = c1.e;
-        if (kSpill) { sTile[so * 2] = c0.t; sTile[so * 2 + 1] = c1.t; }   // (128-token blocks: the two halves of the one item)
+        if (kSpill) {   // (128-token blocks: the two halves of the one item are neighbouring tiles)
+          sTile[so * 4] = c0.ta; sTile[so * 4 + 1] = c0.tb;
+          sTile[so * 4 + 2] = c1.ta; sTile[so * 4 + 3] = c1.tb;
+        }
         mbar_expect_tx(bars + B_STF + so, 2 * 128 * 4);         // (release: publishes the entries as well)
         {
           const float* st0 = a.stat + (static_cast<int64_t>(b) * a.Hq + c0.h) * a.Lp + c0.r;
@@ -847,11 +861,15 @@ bwd_dkdv_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
         // ... and to this half-step's tile in global memory: my 32 queries are four 16-byte groups of my
         // key.  (Written once, read once by the dQ pass: marked evict-first so that the stream does not
         // push the Q / dO tiles, which every kv tile of a window re-reads, out of the L2.)
-        uint8_t* dst = reinterpret_cast<uint8_t*>(a.ds_buf) + sTile[(j & 1) * 2 + half] * kDsTileBytes + (4 * g) * 2048 + r * 16;
+        // (a member the entry does not list has no block, hence no tile: its dS is zero and stays unwritten)
+        if (on) {
+          uint8_t* dst = reinterpret_cast<uint8_t*>(a.ds_buf) + sTile[(j & 1) * 4 + half * 2 + member] * kDsTileBytes<BS> +
+                         (4 * g) * (16 * BS) + (r & (BS - 1)) * 16;
 #pragma unroll
-        for (int i = 0; i < 4; ++i)
-          asm volatile("st.global.L2::cache_hint.v4.b32 [%0], {%1, %2, %3, %4}, %5;" ::"l"(dst + i * 2048),
-                       "r"(dsreg[4 * i]), "r"(dsreg[4 * i + 1]), "r"(dsreg[4 * i + 2]), "r"(dsreg[4 * i + 3]), "l"(evict_first) : "memory");
+          for (int i = 0; i < 4; ++i)
+            asm volatile("st.global.L2::cache_hint.v4.b32 [%0], {%1, %2, %3, %4}, %5;" ::"l"(dst + i * (16 * BS)),
+                         "r"(dsreg[4 * i]), "r"(dsreg[4 * i + 1]), "r"(dsreg[4 * i + 2]), "r"(dsreg[4 * i + 3]), "l"(evict_first) : "memory");
+        }
       }
       ew_publish(bars + B_DSF + half);
       __syncwarp();   // this warp is done with the statistics of step j
@@ -890,16 +908,17 @@ bwd_dkdv_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
 
 // ============================== dQ from the kept dS ===========================================
 // dQ(128 queries x D) = scale * sum over the kv tiles of the row of dS(128 queries x 128 keys) K(128 keys x D),
-// with dS^T read back from the tiles the dK/dV pass left in global memory (one tile of 64 queries x 128
-// keys per half of the query tile, in the core-matrix layout described at BwdArgs::ds_buf, copied as it
-// is and used as an un-swizzled operand; a half without an entry in that kv tile reads the tile of zeros):
+// with dS^T read back from the tiles the dK/dV pass left in global memory (per kv tile of the row the two
+// tiles of 64 queries x 128 keys, or the four of 64 x 64, that make up the 128 x 128 product, in the
+// core-matrix layout described at BwdArgs::ds_buf, copied as they are and used as an un-swizzled operand;
+// where the pattern has no block the tile of zeros is read):
 // one product per step, no exponentials, nothing recomputed.  The kernel is a plain pipelined
 // contraction -- warp 4 loads (a ring of dS^T tile pairs and a ring of K tiles), warp 5 issues, warps
 // 0-3 write the result -- and is bound by the HBM reads of dS.
 template <int D>
 struct DqDsSmem {
   static constexpr int kTile = BwdTile<D>::kBytes;
-  static constexpr int kDs2 = 2 * kDsTileBytes;                // dS^T of a step: the tiles of the two halves of the query tile
+  static constexpr int kDs2 = 128 * 128 * 2;                   // dS^T of a step: [key half (64-token blocks)][query half][8 queries][keys][8 queries]
   static constexpr int kAStages = (D == 128) ? 4 : 5;          // dS^T comes from HBM: the deeper ring
   static constexpr int kKStages = 3;                           // K comes from the L2
   static constexpr int oA = 0;
@@ -934,7 +953,7 @@ bwd_dq_from_ds_kernel(const __grid_constant__ CUtensorMap tm_k, const BwdArgs a)
   const int b = blockIdx.x / a.Hq, h = blockIdx.x % a.Hq, hk = h / a.G;
   const int ent_off = checked(a.tile_off[R * t], 0, a.n_list, a.error_word, 131);
   const int n_ent = checked(a.tile_cnt[t], 0, a.n_list - ent_off, a.error_word, 132);
-  const int32_t* ent = a.tile_ent + 3 * static_cast<int64_t>(ent_off);   // (kv tile, tile of half 0, tile of half 1)
+  const int32_t* ent = a.tile_ent + kDqEntInts * static_cast<int64_t>(ent_off);   // (kv tile, dS tiles of its quarters)
   if (tid == 0) {
     for (int i = 0; i < kAS; ++i) { mbar_init(bars + B_AF + i, 1); mbar_init(bars + B_AE + i, 1); }
     for (int i = 0; i < kKS; ++i) { mbar_init(bars + B_KF + i, 1); mbar_init(bars + B_KE + i, 1); }
@@ -960,25 +979,34 @@ bwd_dq_from_ds_kernel(const __grid_constant__ CUtensorMap tm_k, const BwdArgs a)
       tma_prefetch_desc(&tm_k);
       uint64_t evict_first;
       asm volatile("createpolicy.fractional.L2::evict_first.b64 %0, 1.0;" : "=l"(evict_first));   // dS tiles are read once
+      constexpr int E = kDqEntInts, NT = (BS == 128) ? 2 : 4;   // tiles per step
       const int64_t head_base = (static_cast<int64_t>(b) * a.Hq + h) * a.ds_nnz * (BS / 64);
       const int64_t zero_tile = static_cast<int64_t>(gridDim.x) * a.ds_nnz * (BS / 64);              // the tile after the last head's
       bool ok = true;
       int nl = 0;
-      int e_T = n_ent > 0 ? ent[0] : 0, e_h0 = n_ent > 0 ? ent[1] : 0, e_h1 = n_ent > 0 ? ent[2] : 0;
+      int e_next[E];
+#pragma unroll
+      for (int i = 0; i < E; ++i) e_next[i] = n_ent > 0 ? ent[i] : 0;
       for (int x = 0; x < n_ent; ++x) {
-        const int T = checked(e_T, 0, a.nB - 1, a.error_word, 133), h0 = e_h0, h1 = e_h1;   // (with 64-token blocks T indexes the tiles' column pairs; nB bounds it from above)
-        if (x + 1 < n_ent) { e_T = ent[3 * x + 3]; e_h0 = ent[3 * x + 4]; e_h1 = ent[3 * x + 5]; }   // read ahead
+        int e_cur[E];
+#pragma unroll
+        for (int i = 0; i < E; ++i) e_cur[i] = e_next[i];
+        const int T = checked(e_cur[0], 0, a.nB - 1, a.error_word, 133);   // (with 64-token blocks T indexes the tiles' column pairs; nB bounds it from above)
+        if (x + 1 < n_ent) {   // read ahead
+#pragma unroll
+          for (int i = 0; i < E; ++i) e_next[i] = ent[E * (x + 1) + i];
+        }
         const int sa = x % kAS, sk = x % kKS;
         if (x >= kAS) ok = mbar_wait(bars + B_AE + sa, ((x / kAS) - 1) & 1, a.error_word, 81);
         if (!ok) break;
         mbar_expect_tx(bars + B_AF + sa, SM::kDs2);
         uint8_t* dA = smem + SM::oA + sa * SM::kDs2;
 #pragma unroll
-        for (int half = 0; half < 2; ++half) {
-          const int hx = half ? h1 : h0;
+        for (int i = 0; i < NT; ++i) {   // i = 2 * key half + query half: the order of the schedule entry and of the stage
+          const int hx = checked(e_cur[1 + i], -1, static_cast<int>(a.ds_nnz * (BS / 64)) - 1, a.error_word, 134);
           const int64_t tile_idx = hx >= 0 ? head_base + hx : zero_tile;
-          bulk_load_hint(dA + half * kDsTileBytes, reinterpret_cast<const uint8_t*>(a.ds_buf) + tile_idx * kDsTileBytes,
-                         kDsTileBytes, bars + B_AF + sa, evict_first);
+          bulk_load_hint(dA + i * kDsTileBytes<BS>, reinterpret_cast<const uint8_t*>(a.ds_buf) + tile_idx * kDsTileBytes<BS>,
+                         kDsTileBytes<BS>, bars + B_AF + sa, evict_first);
         }
         if (x >= kKS) ok = mbar_wait(bars + B_KE + sk, ((x / kKS) - 1) & 1, a.error_word, 86);
         if (!ok) break;
@@ -1001,8 +1029,9 @@ bwd_dq_from_ds_kernel(const __grid_constant__ CUtensorMap tm_k, const BwdArgs a)
     const bool lead = elect_one();
     constexpr uint32_t idesc = make_idesc_bf16(128, D, 1, 1);   // A = dS^T and B = K, both MN-major
     const uint32_t hi = desc_hi(1024);
-    // A without swizzle: groups of 8 keys are 128 bytes apart (leading offset), groups of 8 queries 2048 bytes (stride offset)
-    const uint32_t a_hi = desc_hi(2048, 0);
+    // A without swizzle: groups of 8 keys are 128 bytes apart (leading offset), groups of 8 queries 16 bytes x
+    // the keys of a tile (stride offset); with 64-token blocks the key halves of a step are 16 KB apart
+    const uint32_t a_hi = desc_hi(16 * BS, 0);
     const uint32_t a_lo0 = desc_lo(smem_u32(smem + SM::oA), 128), k_lo0 = desc_lo(smem_u32(smem + SM::oK), BwdTile<D>::kBox);
     bool ok = true;
 #pragma unroll 1
@@ -1015,7 +1044,9 @@ bwd_dq_from_ds_kernel(const __grid_constant__ CUtensorMap tm_k, const BwdArgs a)
         const uint32_t a_lo = a_lo0 + sa * (SM::kDs2 >> 4), b_lo = k_lo0 + sk * (kTile >> 4);
 #pragma unroll
         for (int kk = 0; kk < 8; ++kk)
-          if (lead) mma_ss2x(tmem, a_lo + kk * (256 >> 4), a_hi, b_lo + kk * (2048 >> 4), hi, idesc, (x > 0) || (kk > 0));
+          if (lead)
+            mma_ss2x(tmem, a_lo + (BS == 128 ? kk * (256 >> 4) : (kk >> 2) * (16384 >> 4) + (kk & 3) * (256 >> 4)), a_hi,
+                     b_lo + kk * (2048 >> 4), hi, idesc, (x > 0) || (kk > 0));
       }
       if (lead) { mma_commit(bars + B_AE + sa); mma_commit(bars + B_KE + sk); }
     }

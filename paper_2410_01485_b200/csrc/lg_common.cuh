@@ -17,6 +17,7 @@ struct WsHeader {
   unsigned long long fingerprint;  // which pattern the lists and schedules below were built for (0: none)
   unsigned int pad[58];
 };
+constexpr int kDqEntInts = 5;   // ints per entry of the schedule of the dQ pass that reads dS back (dq_sched_kernel)
 constexpr unsigned long long kWsMagic = 0x4c47575348445231ull;   // "LGWSHDR1"
 static_assert(sizeof(WsHeader) == 256, "header size");
 

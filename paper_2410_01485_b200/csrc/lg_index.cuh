@@ -216,18 +216,22 @@ __global__ void kv_tile_of_kernel(const int32_t* __restrict__ cols, int R, int n
 }
 
 // ---- schedule of the dQ pass that reads the kept dS tiles -------------------------------------
-// The dK/dV pass leaves, per (kv tile T, entry e = query block qb of T's schedule), dS^T tiles of 64
-// queries: numbered (off[T] + e) * (block / 64) + half.  A query tile of 128 rows needs, for every kv
-// tile with an active column in the row(s) of its query block(s), the two tiles of its two 64-row halves
-// (-1: that half has no entry in T, its dS is zero).  One thread per query tile; entries (T, h0, h1) at
-// dq_ent[3 * (row_ptr[R t] + i)], kv tiles ascending.
+// The dK/dV pass leaves one dS tile per block of the pattern and 64-row half of its query block, numbered by
+// the block's position p in the column lists (col_ptr[c] + rank of the query block in column c):
+// 128-token blocks: tiles 2 p and 2 p + 1 (128 keys x 64 queries each); 64-token blocks: tile p (64 keys x
+// 64 queries).  A query tile of 128 rows needs, for every kv tile T with an active column in the row(s) of
+// its query block(s), the four quarters (64-row half m, 64-key half n) of its 128 x 128 product; entry =
+// (T, tile of (m, n) at 1 + 2 n + m), -1 where the pattern has no block (that quarter of dS is zero).  With
+// 128-token blocks only n = 0 is used: the tiles of the two halves.  One thread per query tile; entries at
+// dq_ent[kDqEntInts * (row_ptr[R t] + i)], kv tiles ascending.
 __global__ void dq_sched_kernel(const int32_t* __restrict__ row_ptr, const int32_t* __restrict__ col_idx,
-                                const int32_t* __restrict__ tile_of, const int32_t* __restrict__ off,
-                                const int32_t* __restrict__ tile_cnt, const int32_t* __restrict__ tile_ent, int R, int nB,
+                                const int32_t* __restrict__ col_ptr, const int32_t* __restrict__ row_idx,
+                                const int32_t* __restrict__ tile_of, const int32_t* __restrict__ cols, int R, int nB,
                                 int n_qtiles, int32_t* __restrict__ dq_cnt, int32_t* __restrict__ dq_ent) {
   const int t = blockIdx.x * blockDim.x + threadIdx.x;
   if (t >= n_qtiles) return;
-  int32_t* out = dq_ent + 3 * static_cast<int64_t>(row_ptr[R * t]);
+  constexpr int E = kDqEntInts;
+  int32_t* out = dq_ent + E * static_cast<int64_t>(row_ptr[R * t]);
   int n = 0;
   for (int m = 0; m < R; ++m) {          // distinct kv tiles of the tile's query blocks, kept ascending
     const int qb = R * t + m;
@@ -235,33 +239,33 @@ __global__ void dq_sched_kernel(const int32_t* __restrict__ row_ptr, const int32
     for (int x = row_ptr[qb]; x < row_ptr[qb + 1]; ++x) {
       const int T = tile_of[col_idx[x]];
       int pos = 0;
-      while (pos < n && out[3 * pos] < T) ++pos;
-      if (pos < n && out[3 * pos] == T) continue;
-      for (int y = n; y > pos; --y) out[3 * y] = out[3 * (y - 1)];
-      out[3 * pos] = T;
+      while (pos < n && out[E * pos] < T) ++pos;
+      if (pos < n && out[E * pos] == T) continue;
+      for (int y = n; y > pos; --y) out[E * y] = out[E * (y - 1)];
+      out[E * pos] = T;
       ++n;
     }
   }
-  auto find = [&](int T, int qb) {       // index of query block qb in T's schedule (ascending), or -1
-    if (qb >= nB) return -1;
-    int lo = 0, hi = tile_cnt[T];
-    const int32_t* ent = tile_ent + off[T];
+  auto find = [&](int c, int qb) {       // position of block (row qb, column c) in the column lists, or -1
+    if (c < 0 || qb >= nB) return -1;
+    int lo = col_ptr[c], hi = col_ptr[c + 1];
+    const int end = hi;
     while (lo < hi) {
       const int mid = (lo + hi) >> 1;
-      if ((ent[mid] >> 2) < qb) lo = mid + 1; else hi = mid;
+      if (row_idx[mid] < qb) lo = mid + 1; else hi = mid;
     }
-    return (lo < tile_cnt[T] && (ent[lo] >> 2) == qb) ? lo : -1;
+    return (lo < end && row_idx[lo] == qb) ? lo : -1;
   };
   for (int i = 0; i < n; ++i) {
-    const int T = out[3 * i];
+    const int T = out[E * i];
     if (R == 1) {
-      const int e = find(T, t);
-      out[3 * i + 1] = (off[T] + e) * 2;
-      out[3 * i + 2] = (off[T] + e) * 2 + 1;
+      const int p = find(cols[T], t);
+      out[E * i + 1] = p >= 0 ? 2 * p : -1;
+      out[E * i + 2] = p >= 0 ? 2 * p + 1 : -1;
+      out[E * i + 3] = out[E * i + 4] = -1;
     } else {
-      const int e0 = find(T, 2 * t), e1 = find(T, 2 * t + 1);
-      out[3 * i + 1] = e0 >= 0 ? off[T] + e0 : -1;
-      out[3 * i + 2] = e1 >= 0 ? off[T] + e1 : -1;
+      for (int nn = 0; nn < 2; ++nn)
+        for (int m = 0; m < 2; ++m) out[E * i + 1 + 2 * nn + m] = find(cols[2 * T + nn], 2 * t + m);
     }
   }
   dq_cnt[t] = n;
