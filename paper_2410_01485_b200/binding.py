@@ -335,6 +335,27 @@ def lg_sparse_decode(p: DecodeParams, q, k_cache, v_cache, n_tokens, o=None, lse
     return o, lse
 
 
+def decode_call(p: DecodeParams, q, k_cache, v_cache, n_tokens, o, lse, workspace):
+    """lg_sparse_decode on fixed buffers (a serving loop's): the arguments are marshalled once, the returned
+    function takes no arguments, launches on the stream that is current when it is called and returns
+    nothing (the results are in o, lse).  The tensors must stay alive and in place."""
+    assert q.is_contiguous() and k_cache.is_contiguous() and v_cache.is_contiguous()
+    fn = load_library().lg_sparse_decode
+    args = (C.byref(p), C.c_void_p(q.data_ptr()), C.c_void_p(k_cache.data_ptr()), C.c_void_p(v_cache.data_ptr()),
+            C.c_void_p(n_tokens.data_ptr()), C.c_void_p(o.data_ptr()),
+            C.c_void_p(lse.data_ptr() if lse is not None else None), C.c_void_p(workspace.data_ptr()),
+            C.c_size_t(workspace.numel()))
+    keep = (p, q, k_cache, v_cache, n_tokens, o, lse, workspace)
+    current_stream = torch.cuda.current_stream
+
+    def call(_keep=keep):
+        code = fn(*args, C.c_void_p(current_stream().cuda_stream))
+        if code != LG_OK:
+            raise LgError(code, "lg_sparse_decode")
+
+    return call
+
+
 def chunk_prefill_workspace(p: DecodeParams, T: int, n_tokens_before: int, device="cuda") -> torch.Tensor:
     n = load_library().lg_chunk_prefill_workspace_bytes(C.byref(p), T, n_tokens_before)
     if n == 0:

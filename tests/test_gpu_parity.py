@@ -542,6 +542,14 @@ def test_decode_cfg5_as_stated(lg):
         assert np.isfinite(oo).all()
         _assert_close(synth.to_f64(o[b]), oo, TOL_O, "cfg5 decode o b%d" % b)
         assert np.abs(synth.to_f64(lse[b]) - ll).max() <= TOL_LSE
+    # the call with arguments marshalled once (what the bench times per host call) is the same call
+    o2, lse2 = torch.zeros_like(o), torch.zeros_like(lse)
+    step = lg.decode_call(p, q, kc, vc, n_t, o2, lse2, ws)
+    step()
+    step()
+    torch.cuda.synchronize()
+    assert lg.lg_last_status(ws) == 0
+    assert torch.equal(o2, o) and torch.equal(lse2, lse)
 
 
 def test_decode_cfg5_dense_comparator_131072(lg):
