@@ -14,7 +14,7 @@ static lg_status launch_bwd_t(const Resolved& r, const WsLayout& w, const void* 
   {
     const int Lp = static_cast<int>(align_up(r.L, 128));
     const int n_bh = r.B * r.Hq;
-    const int rows_per_block = 256 / (D / 8);
+    const int rows_per_block = 256 / (D / 8) * kDeltaRowsPerThread;
     dim3 grid((Lp + rows_per_block - 1) / rows_per_block, n_bh < 65535 ? n_bh : 65535);
     delta_kernel<D><<<grid, 256, 0, stream>>>(
         static_cast<const __nv_bfloat16*>(o), static_cast<const __nv_bfloat16*>(d_o), lse, stat, r.os[0], r.os[1],

@@ -71,36 +71,48 @@ template <int BS> constexpr int kDsTileBytes = BS * 64 * 2;
 // ---- stat = -(LSE * log2 e) and -rowsum(dO * O), stored negated (they are only ever subtracted),
 // each in a plane of its own: the dK/dV pass fetches four neighbouring queries' values of one kind
 // with a single 16-byte shared-memory load ---------------------------------------------------------
+constexpr int kDeltaRowsPerThread = 4;   // rows a thread works, their loads issued together
 template <int D>
 __global__ void delta_kernel(const __nv_bfloat16* __restrict__ o, const __nv_bfloat16* __restrict__ d_o,
                              const float* __restrict__ lse, float* __restrict__ stat, int64_t sb, int64_t sh,
                              int64_t sl, int Hq, int n_bh, int L, int Lp, int64_t plane) {
   // grid.x walks the padded rows of a head (rows i >= L exist only in `stat`, as zeros), grid.y the heads
   constexpr int TPR = D / 8;   // threads per row, 16 bytes each
-  const int i = blockIdx.x * (blockDim.x / TPR) + threadIdx.x / TPR;
+  constexpr int U = kDeltaRowsPerThread;
+  const int rows = blockDim.x / TPR;                       // rows per pass of the block
+  const int i0 = blockIdx.x * (rows * U) + threadIdx.x / TPR;
   const int ch = threadIdx.x % TPR;
   for (int bh = blockIdx.y; bh < n_bh; bh += gridDim.y) {
-    float acc = 0.f;
-    const bool real = i < L;
-    if (real) {
-      const int h = bh % Hq, b = bh / Hq;
-      const int64_t off = b * sb + h * sh + static_cast<int64_t>(i) * sl + ch * 8;
-      const uint4 ov = *reinterpret_cast<const uint4*>(o + off);
-      const uint4 dv = *reinterpret_cast<const uint4*>(d_o + off);
-      const __nv_bfloat162* op = reinterpret_cast<const __nv_bfloat162*>(&ov);
-      const __nv_bfloat162* dp = reinterpret_cast<const __nv_bfloat162*>(&dv);
+    const int h = bh % Hq, b = bh / Hq;
+    uint4 ov[U], dv[U];
+#pragma unroll
+    for (int u = 0; u < U; ++u) {
+      const int i = i0 + u * rows;
+      ov[u] = dv[u] = make_uint4(0, 0, 0, 0);
+      if (i < L) {
+        const int64_t off = b * sb + h * sh + static_cast<int64_t>(i) * sl + ch * 8;
+        ov[u] = *reinterpret_cast<const uint4*>(o + off);
+        dv[u] = *reinterpret_cast<const uint4*>(d_o + off);
+      }
+    }
+#pragma unroll
+    for (int u = 0; u < U; ++u) {
+      const int i = i0 + u * rows;
+      const __nv_bfloat162* op = reinterpret_cast<const __nv_bfloat162*>(&ov[u]);
+      const __nv_bfloat162* dp = reinterpret_cast<const __nv_bfloat162*>(&dv[u]);
+      float acc = 0.f;
 #pragma unroll
       for (int x = 0; x < 4; ++x) {
         const float2 a = __bfloat1622float2(op[x]), c = __bfloat1622float2(dp[x]);
         acc += a.x * c.x + a.y * c.y;
       }
-    }
 #pragma unroll
-    for (int s = TPR / 2; s > 0; s >>= 1) acc += __shfl_xor_sync(0xffffffffu, acc, s);
-    if (i < Lp && ch == 0) {
-      const int64_t row = static_cast<int64_t>(bh) * Lp + i;
-      stat[row] = real ? -lse[static_cast<int64_t>(bh) * L + i] * 1.4426950408889634f : 0.f;
-      stat[plane + row] = -acc;
+      for (int s = TPR / 2; s > 0; s >>= 1) acc += __shfl_xor_sync(0xffffffffu, acc, s);
+      if (i < Lp && ch == 0) {
+        const int64_t row = static_cast<int64_t>(bh) * Lp + i;
+        stat[row] = i < L ? -lse[static_cast<int64_t>(bh) * L + i] * 1.4426950408889634f : 0.f;
+        stat[plane + row] = -acc;
+      }
     }
   }
 }

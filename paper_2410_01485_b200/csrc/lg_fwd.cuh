@@ -298,6 +298,7 @@ fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUt
         const int lo_abs = (a.exact_w > 0 && (e >> 4) >= a.ns) ? max(dstart, win_lo) : dstart;
         const int lo = min(max(lo_abs - key0, 0), 64);
 
+        const bool masked = __any_sync(0xffffffffu, lim < 64 || lo > 0);   // (voted before the wait: off the chain)
         ok = mbar_wait_warp(bars + B_SF + s * 2 + hf, (hf ? p1 : p0) & 1, a.error_word, 12);
         if (!ok) break;
         tc_fence_after();
@@ -305,7 +306,7 @@ fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUt
         tmem_ld32(my_s + hf * 64, v);
         tmem_ld32(my_s + hf * 64 + 32, v + 32);
         tmem_ld_wait();
-        if (__any_sync(0xffffffffu, lim < 64 || lo > 0)) {
+        if (masked) {
 #pragma unroll
           for (int x = 0; x < 64; ++x)
             v[x] = (x < lim && x >= lo) ? v[x] : 0xff800000u;   // -inf: the exponential below gives exactly 0

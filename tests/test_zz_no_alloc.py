@@ -67,3 +67,35 @@ def test_static_decode_matches_workspace_decode_twice(lib):
         assert (o.float() - o_ref.float()).abs().max().item() <= TOL_O
         assert (lse - lse_ref).abs().max().item() <= TOL_LSE
         assert torch.equal(o, o_ref) and torch.equal(lse, lse_ref)   # same kernels, same order: same bits
+
+
+@pytest.mark.gpu
+def test_static_decode_second_shape_over_the_first_ones_leftovers_and_no_allocation(lib):
+    """Two problems of different shape, one after the other, share the fixed array: the second (other batch,
+    head counts, head dimension and lengths, hence other units, counters and record layout) must not be
+    disturbed by what the first left there.  And the call requests no device memory: the bytes the driver
+    reports free and the bytes torch has handed out are the same before and after it."""
+    g = torch.Generator(device="cuda").manual_seed(11)
+    shapes = [(4, 64, 8, 128, 128, 4096, [5000, 4224, 777, 131072]),   # the headline head layout, split units
+              (3, 12, 4, 64, 64, 512, [600, 1, 300])]                   # other B / Hkv / G / D / capacity
+    for B, Hq, Hkv, D, sink, W, n_list in shapes:
+        p = lg.decode_params(B, Hq, Hkv, D, sink, W)
+        cap = sink + W
+        q = torch.randn(B, Hq, D, generator=g, device="cuda").to(torch.bfloat16)
+        kc = torch.randn(B, Hkv, cap, D, generator=g, device="cuda").to(torch.bfloat16)
+        vc = torch.randn(B, Hkv, cap, D, generator=g, device="cuda").to(torch.bfloat16)
+        n_t = torch.tensor(n_list, dtype=torch.int64, device="cuda")
+        o_ref, lse_ref = lg.lg_sparse_decode(p, q, kc, vc, n_t)
+        o = torch.full_like(q, float("nan"))
+        lse = torch.full((B, Hq), float("nan"), dtype=torch.float32, device="cuda")
+        lg.lg_sparse_decode_static(p, q, kc, vc, n_t, o, lse)      # (first call of a shape: one-time set-up of the device's facts)
+        torch.cuda.synchronize()
+        free0, _ = torch.cuda.mem_get_info()
+        held0, reserved0 = torch.cuda.memory_allocated(), torch.cuda.memory_reserved()
+        o.fill_(float("nan")); lse.fill_(float("nan"))
+        lg.lg_sparse_decode_static(p, q, kc, vc, n_t, o, lse)
+        torch.cuda.synchronize()
+        free1, _ = torch.cuda.mem_get_info()
+        assert free1 == free0, "the call changed the device's free memory by %d bytes" % (free0 - free1)
+        assert torch.cuda.memory_allocated() == held0 and torch.cuda.memory_reserved() == reserved0
+        assert torch.equal(o, o_ref) and torch.equal(lse, lse_ref)
