@@ -113,12 +113,26 @@ lg_status resolve(const lg_attn_params* p, Resolved* r) {
   return LG_OK;
 }
 
+// SMs of the current device (looked up once per device)
+int sm_count() {
+  static int cached[64];
+  int dev = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return -1;
+  if (cached[dev] == 0) {
+    int n = 0;
+    if (cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || n <= 0) return -1;
+    cached[dev] = n;
+  }
+  return cached[dev];
+}
+
 // Two backward variants compute the same gradients (see BwdVariant).  The two passes run everywhere.
 // Keeping dS trades workspace and HBM traffic (2 bytes per visible pair, written once and read once, on
 // a memory system the attention kernels otherwise leave idle) for the two recomputed products of the dQ
 // pass.  It is the default when the lists are shared by the batch and the dS buffer takes at most
-// LG_KEEP_DS_MAX_GB (default 48) gigabytes (the buffer holds every block of the pattern in full).  LG_BWD_VARIANT = two_pass | keep_ds overrides the choice (read at every call;
-// it must not change between a size query, a prepare and the calls that use them).
+// LG_KEEP_DS_MAX_GB (default 48) gigabytes (the buffer holds every block of the pattern in full).
+// LG_BWD_VARIANT = two_pass | keep_ds overrides the choice (read at every call; it must not change between
+// a size query, a prepare and the calls that use them).
 size_t ds_buffer_bytes(const Resolved& r) {   // 2 bytes per pair of every block of the pattern and query head, plus one tile of zeros at the end
   return static_cast<size_t>(r.B) * r.Hq * static_cast<size_t>(r.nnz) * r.block * r.block * 2 + 128 * 64 * 2;
 }

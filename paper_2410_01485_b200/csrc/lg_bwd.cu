@@ -57,6 +57,8 @@ static lg_status launch_bwd_t(const Resolved& r, const WsLayout& w, const void* 
     a.out1 = static_cast<__nv_bfloat16*>(dv);
     for (int i = 0; i < 3; ++i) { a.s0[i] = r.ks[i]; a.s1[i] = r.vs[i]; }
     dim3 grid(r.B * r.Hkv, r.n_ktiles);
+    a.ahead = sm_count();   // one CTA per SM
+    if (a.ahead < 0) return LG_ERR_CUDA;
     if (variant == kBwdKeepDs) {
       // the tile of zeros that stands in for a half of a query tile a kv tile has no entry for
       if (cudaMemsetAsync(ws + w.ds_buf + ds_buffer_bytes(r) - 128 * 64 * 2, 0, 128 * 64 * 2, stream) != cudaSuccess) return LG_ERR_CUDA;

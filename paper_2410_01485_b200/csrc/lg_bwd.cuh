@@ -65,6 +65,7 @@ struct BwdArgs {
   int64_t ds_nnz;
   __nv_bfloat16* ds_buf;
   const int32_t* col_ptr;    // column lists of the pattern (dK/dV pass that keeps dS: positions of its blocks)
+  int ahead;                 // dK/dV pass: CTAs that run at a time (see prefetch_successor), 0: no prefetch
 };
 template <int BS> constexpr int kDsTileBytes = BS * 64 * 2;
 
@@ -613,6 +614,28 @@ bwd_dkdv_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
       // the statistics of step j (released by the element-wise warps at the end of step j - 2), then Q
       // of step j + 1 (three stages: the slot of step j - 2, released by its dK product).  Q is the first
       // operand a step needs -- S^T of step j + 1 is issued early in step j -- hence the step of lead.
+      // CTAs start in launch order as SMs come free, and the tiles of a pattern's band take the same time:
+      // the CTA `ahead` places after this one starts about when this one ends, on some SM.  Its K and V
+      // tiles are first touched by it and would come from HBM at the head of its critical path; asked for
+      // now (once this tile's first loads are on their way and this thread mostly waits), they are in the L2
+      // by then.  A hint only: nothing waits for it and a wrong guess costs two tile reads.
+      auto prefetch_successor = [&]() {
+        if (a.ahead <= 0) return;
+        const int64_t w = static_cast<int64_t>(blockIdx.y) * gridDim.x + blockIdx.x + a.ahead;
+        if (w >= static_cast<int64_t>(gridDim.x) * gridDim.y) return;
+        const int t2 = checked(a.order[w / gridDim.x], 0, a.n_tiles - 1, a.error_word, 126);
+        const int x2 = static_cast<int>(w % gridDim.x), b2 = x2 / a.Hkv, hk2 = x2 % a.Hkv;
+#pragma unroll
+        for (int m = 0; m < R; ++m) {
+          const int kb2 = checked(a.tile_cols[R * t2 + m], -1, a.nB - 1, a.error_word, 127);
+          if (kb2 < 0) continue;
+#pragma unroll
+          for (int x = 0; x < D / 64; ++x) {
+            tma_prefetch_l2_4d(&tm_k, x * 64, kb2 * BS, hk2, b2);
+            tma_prefetch_l2_4d(&tm_v, x * 64, kb2 * BS, hk2, b2);
+          }
+        }
+      };
       struct Item { int h, r, e; int64_t ta, tb; };
       auto step_items = [&](int j, Item& i0, Item& i1) {
         next_item(i0.h, i0.r, i0.e, i0.ta, i0.tb);
@@ -665,6 +688,7 @@ bwd_dkdv_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
         }
         nst = j + 1;
         if (j + 1 < n_steps) load_q(j + 1, n0, n1);
+        if (j == 2) prefetch_successor();
       }
       mbar_wait(bars + B_FIX, 0, a.error_word, 16);
       for (int j = max(nq - kQS, 0); j < nq; ++j) mbar_wait(bars + B_QF + j % kQS, (j / kQS) & 1, a.error_word, 17);
