@@ -617,8 +617,9 @@ bwd_dkdv_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
       // CTAs start in launch order as SMs come free, and the tiles of a pattern's band take the same time:
       // the CTA `ahead` places after this one starts about when this one ends, on some SM.  Its K and V
       // tiles are first touched by it and would come from HBM at the head of its critical path; asked for
-      // now (once this tile's first loads are on their way and this thread mostly waits), they are in the L2
-      // by then.  A hint only: nothing waits for it and a wrong guess costs two tile reads.
+      // a few steps before this tile ends (earlier, the stream of dS stores has pushed them out of the L2
+      // again by the time they are wanted: + 25 % of DRAM reads in the profile), they are in the L2 by then.
+      // A hint only: nothing waits for it and a wrong guess costs two tile reads.
       auto prefetch_successor = [&]() {
         if (a.ahead <= 0) return;
         const int64_t w = static_cast<int64_t>(blockIdx.y) * gridDim.x + blockIdx.x + a.ahead;
@@ -688,7 +689,7 @@ bwd_dkdv_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
         }
         nst = j + 1;
         if (j + 1 < n_steps) load_q(j + 1, n0, n1);
-        if (j == 2) prefetch_successor();
+        if (j + 1 == (n_steps > 8 ? n_steps - 8 : 1)) prefetch_successor();   // a few steps before this tile ends
       }
       mbar_wait(bars + B_FIX, 0, a.error_word, 16);
       for (int j = max(nq - kQS, 0); j < nq; ++j) mbar_wait(bars + B_QF + j % kQS, (j / kQS) & 1, a.error_word, 17);
