@@ -335,21 +335,22 @@ def lg_sparse_decode(p: DecodeParams, q, k_cache, v_cache, n_tokens, o=None, lse
     return o, lse
 
 
-def decode_call(p: DecodeParams, q, k_cache, v_cache, n_tokens, o, lse, workspace):
-    """lg_sparse_decode on fixed buffers (a serving loop's): the arguments are marshalled once, the returned
-    function takes no arguments, launches on the stream that is current when it is called and returns
-    nothing (the results are in o, lse).  The tensors must stay alive and in place."""
+def decode_call(p: DecodeParams, q, k_cache, v_cache, n_tokens, o, lse, workspace, stream=None):
+    """lg_sparse_decode on fixed buffers (a serving loop's): every argument is marshalled once, the stream
+    included (`stream`, default: the stream that is current now).  The returned function takes no arguments,
+    launches on that stream and returns nothing (the results are in o, lse).  The tensors must stay alive
+    and in place."""
     assert q.is_contiguous() and k_cache.is_contiguous() and v_cache.is_contiguous()
     fn = load_library().lg_sparse_decode
+    handle = (torch.cuda.current_stream() if stream is None else stream).cuda_stream
     args = (C.byref(p), C.c_void_p(q.data_ptr()), C.c_void_p(k_cache.data_ptr()), C.c_void_p(v_cache.data_ptr()),
             C.c_void_p(n_tokens.data_ptr()), C.c_void_p(o.data_ptr()),
             C.c_void_p(lse.data_ptr() if lse is not None else None), C.c_void_p(workspace.data_ptr()),
-            C.c_size_t(workspace.numel()))
+            C.c_size_t(workspace.numel()), C.c_void_p(handle))
     keep = (p, q, k_cache, v_cache, n_tokens, o, lse, workspace)
-    current_stream = torch.cuda.current_stream
 
     def call(_keep=keep):
-        code = fn(*args, C.c_void_p(current_stream().cuda_stream))
+        code = fn(*args)
         if code != LG_OK:
             raise LgError(code, "lg_sparse_decode")
 
