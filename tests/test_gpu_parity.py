@@ -837,10 +837,13 @@ DOC_CASES = [
 ]
 
 
+@pytest.mark.parametrize("variant", ["two_pass", "keep_ds"])
 @pytest.mark.parametrize("cfg", DOC_CASES, ids=lambda c: c.name)
-def test_documents_fwd_bwd_parity(lg, cfg):
+def test_documents_fwd_bwd_parity(lg, cfg, variant, monkeypatch):
     """Packed documents (no key of an earlier document) on top of every pattern: forward and backward against
-    the oracle; document lengths are seeded, differ per batch element, and include very short documents."""
+    the oracle; document lengths are seeded, differ per batch element, and include very short documents.
+    Both backward variants (with per-sequence lists, B > 1, the library takes the two passes either way)."""
+    monkeypatch.setenv("LG_BWD_VARIANT", variant)
     ds = torch.stack([synth.make_doc_start(cfg.L, seed=7 + b, mean_len=150) for b in range(cfg.B)]).cuda()
     first = int((ds[0] == 0).sum())                        # cut the first document of sequence 0 into 1 + 2 + rest
     assert first > 3
@@ -904,10 +907,13 @@ RAGGED = [
 ]
 
 
+@pytest.mark.parametrize("variant", ["two_pass", "keep_ds"])
 @pytest.mark.parametrize("cfg", RAGGED, ids=lambda c: c.name)
-def test_partial_last_block_parity(lg, cfg):
+def test_partial_last_block_parity(lg, cfg, variant, monkeypatch):
     """L that ends inside a block (odd lengths included): lists bit-exact, forward and backward against the
-    oracle, and nothing written past L (outputs live in buffers with a sentinel row after the end)."""
+    oracle, and nothing written past L (outputs live in buffers with a sentinel row after the end); both
+    backward variants."""
+    monkeypatch.setenv("LG_BWD_VARIANT", variant)
     p = lg.params_of(cfg)
     got = lg.lg_build_block_index(p)
     ref = O.block_lists(O.Pattern.of(cfg))
