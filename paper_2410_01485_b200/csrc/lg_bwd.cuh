@@ -849,10 +849,9 @@ bwd_dkdv_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
                                 f32x2(l4.x, l4.y)), x0, x1);
           f32x2_split(fma_f32x2(f32x2(__uint_as_float(sreg[c + 2]), __uint_as_float(sreg[c + 3])), scale2,
                                 f32x2(l4.z, l4.w)), x2, x3);
-          // half of the exponentials on the exponential unit, half as a polynomial on the FMA pipe: all
-          // sixteen warps reach this point together, and the unit alone would need 512 cycles for the half-step
-          float v0 = fast_exp2(x0), v1 = fast_exp2(x1), v2, v3;
-          poly_exp2_x2(x2, x3, v2, v3);
+          // (all on the exponential unit: with the two teams the element-wise warps have slack, and under
+          // the power cap the instructions of a polynomial on the FMA pipe cost more than the unit's cycles)
+          float v0 = fast_exp2(x0), v1 = fast_exp2(x1), v2 = fast_exp2(x2), v3 = fast_exp2(x3);
           if (masked) {
             v0 = (c >= xmin && c < xmax) ? v0 : 0.f;
             v1 = (c + 1 >= xmin && c + 1 < xmax) ? v1 : 0.f;

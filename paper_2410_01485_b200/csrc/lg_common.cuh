@@ -318,27 +318,6 @@ __device__ __forceinline__ uint64_t mul_f32x2(uint64_t a, uint64_t b) {
   asm("mul.rn.f32x2 %0, %1, %2;" : "=l"(d) : "l"(a), "l"(b));
   return d;
 }
-// 2^x for a pair of values on the FMA / ALU pipes instead of the exponential unit (which delivers 16
-// results per clock and SM and is what the element-wise warps of the backward queue up for): round to
-// the nearest integer with the 1.5 * 2^23 trick, a cubic for 2^f on f in [-0.5, 0.5] (relative error
-// below 8e-5, far inside the bf16 rounding that follows), and the integer added into the exponent field.
-// Inputs below -125 (masked scores) are clamped; their results are tiny and get masked or rounded away.
-__device__ __forceinline__ void poly_exp2_x2(float x0, float x1, float& y0, float& y1) {
-  const float magic = 12582912.0f;
-  const uint64_t x = f32x2(fmaxf(x0, -125.f), fmaxf(x1, -125.f));
-  const uint64_t t = add_f32x2(x, f32x2(magic, magic));
-  const uint64_t xr = add_f32x2(t, f32x2(-magic, -magic));
-  const uint64_t f = fma_f32x2(xr, f32x2(-1.f, -1.f), x);
-  uint64_t p = fma_f32x2(f32x2(0.05508868396282196f, 0.05508868396282196f), f, f32x2(0.24260404706001282f, 0.24260404706001282f));
-  p = fma_f32x2(p, f, f32x2(0.6932762265205383f, 0.6932762265205383f));
-  p = fma_f32x2(p, f, f32x2(0.9999289512634277f, 0.9999289512634277f));
-  float t0, t1, p0, p1;
-  f32x2_split(t, t0, t1);
-  f32x2_split(p, p0, p1);
-  y0 = __int_as_float(__float_as_int(p0) + (__float_as_int(t0) << 23));
-  y1 = __int_as_float(__float_as_int(p1) + (__float_as_int(t1) << 23));
-}
-
 __device__ __forceinline__ float max3(float a, float b, float c) {
   float d;
   asm("max.f32 %0, %1, %2, %3;" : "=f"(d) : "f"(a), "f"(b), "f"(c));
