@@ -919,21 +919,28 @@ bwd_dkdv_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
     }
     if (ok) {
       tc_fence_after();
-      constexpr int kEpi = 32;                               // output columns per thread
-      const bool mine = kj < a.L;                            // keys past L take part in the loads only
-      const int ge = warp >> 2;                              // the sixteen warps share the D output columns
-      if (kb_mine >= 0 && ge * kEpi < D) {
-        __nv_bfloat16* dk_row = a.out0 + b * a.s0[0] + hk * a.s0[1] + static_cast<int64_t>(kj) * a.s0[2] + ge * kEpi;
-        __nv_bfloat16* dv_row = a.out1 + b * a.s1[0] + hk * a.s1[1] + static_cast<int64_t>(kj) * a.s1[2] + ge * kEpi;
+      // The sixteen warps share the output: warp group ge takes 64 columns of one accumulator (dV first, then
+      // dK) for its 32 keys.  The rows leave through the Q ring (every load into it has been consumed by the
+      // products that are now done), 4 KB per warp, so that the stores cover whole rows (store_acc_64cols).
+      constexpr int kParts = D / 64;
+      const int ge = warp >> 2;
+      if (kb_mine >= 0 && ge < 2 * kParts) {
+        const bool is_dk = ge >= kParts;
+        const int part = ge % kParts;
+        const int64_t* st = is_dk ? a.s0 : a.s1;
+        __nv_bfloat16* base = (is_dk ? a.out0 : a.out1) + b * st[0] + hk * st[1] + part * 64;
+        const int64_t row_stride = st[2];
         if (n_hs > 0) {
-          store_acc_cols<kEpi>(lane_addr + kColDV + ge * kEpi, dv_row, 1.0f, mine);
-          store_acc_cols<kEpi>(lane_addr + kColDK + ge * kEpi, dk_row, a.scale, mine);
-        } else if (mine) {
+          const int r_first = (warp & 3) * 32;
+          store_acc_64cols(lane_addr + (is_dk ? kColDK : kColDV) + part * 64, sQ + warp * 4096, is_dk ? a.scale : 1.0f,
+                           [&](int r2) -> __nv_bfloat16* {
+                             const int rr = r_first + r2;
+                             const int k2 = kb_mine * BS + (R == 2 ? (rr & (BS - 1)) : rr);   // keys past L take part in the loads only
+                             return k2 < a.L ? base + static_cast<int64_t>(k2) * row_stride : nullptr;
+                           });
+        } else if (kj < a.L) {
 #pragma unroll
-          for (int x = 0; x < kEpi; x += 8) {
-            *reinterpret_cast<uint4*>(dk_row + x) = make_uint4(0, 0, 0, 0);
-            *reinterpret_cast<uint4*>(dv_row + x) = make_uint4(0, 0, 0, 0);
-          }
+          for (int x = 0; x < 64; x += 8) *reinterpret_cast<uint4*>(base + static_cast<int64_t>(kj) * row_stride + x) = make_uint4(0, 0, 0, 0);
         }
       }
     }

@@ -329,4 +329,43 @@ __device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
   return r;
 }
 
+// Epilogue of an accumulator tile: fp32 columns [taddr, taddr + 64) of this warp's 32 tensor-memory lanes
+// (lane = row), times `mul`, as bf16 to global rows.  A thread holds a whole row, so storing straight from its
+// registers makes every store instruction of the warp touch 32 rows (32 separate 16-byte pieces); the
+// rows go through `stage` (4 KB of shared memory of this warp's own, 16-byte chunks XOR-swizzled by the row)
+// instead, and every store instruction then writes four whole 128-byte rows.  row_ptr(r) = where the 64
+// columns of row r (0 .. 31 of this warp) go, or nullptr for a row that is not stored.  The whole warp calls.
+template <typename RowPtr>
+__device__ __forceinline__ void store_acc_64cols(uint32_t taddr, uint8_t* stage, float mul, RowPtr row_ptr) {
+  const uint32_t lane = lane_id();
+  const uint32_t sbase = smem_u32(stage);
+#pragma unroll
+  for (int c = 0; c < 2; ++c) {
+    uint32_t reg[32];
+    tmem_ld32(taddr + c * 32, reg);
+    tmem_ld_wait();
+#pragma unroll
+    for (int x = 0; x < 4; ++x) {
+      const uint32_t w0 = pack_bf16(__uint_as_float(reg[8 * x + 0]) * mul, __uint_as_float(reg[8 * x + 1]) * mul);
+      const uint32_t w1 = pack_bf16(__uint_as_float(reg[8 * x + 2]) * mul, __uint_as_float(reg[8 * x + 3]) * mul);
+      const uint32_t w2 = pack_bf16(__uint_as_float(reg[8 * x + 4]) * mul, __uint_as_float(reg[8 * x + 5]) * mul);
+      const uint32_t w3 = pack_bf16(__uint_as_float(reg[8 * x + 6]) * mul, __uint_as_float(reg[8 * x + 7]) * mul);
+      asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(sbase + lane * 128 + (((4 * c + x) ^ (lane & 7)) << 4)),
+                   "r"(w0), "r"(w1), "r"(w2), "r"(w3) : "memory");
+    }
+  }
+  __syncwarp();
+#pragma unroll
+  for (int k = 0; k < 8; ++k) {
+    const uint32_t row = 4 * k + (lane >> 3), ch = lane & 7;
+    uint4 v;
+    asm volatile("ld.shared.v4.b32 {%0, %1, %2, %3}, [%4];" : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w)
+                 : "r"(sbase + row * 128 + ((ch ^ (row & 7)) << 4)) : "memory");
+    __nv_bfloat16* dst = row_ptr(static_cast<int>(row));
+    if (dst) *reinterpret_cast<uint4*>(dst + ch * 8) = v;
+  }
+  __syncwarp();   // the stage may be written again
+}
+
+
 }  // namespace lg

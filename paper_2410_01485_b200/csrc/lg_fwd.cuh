@@ -388,23 +388,17 @@ fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUt
       const bool mine = qi < a.L && qi >= a.q_start;
       tc_fence_after();
       const float inv_l = l_run > 0.f ? 1.f / l_run : 0.f;
-      __nv_bfloat16* orow =
-          a.o + b * a.o_strides[0] + h * a.o_strides[1] + static_cast<int64_t>(qi - a.q_start) * a.o_strides[2];
+      // rows leave through the slot's own Q tile (its last S product is done: it precedes the last P V in
+      // the issuer's queue), 4 KB per warp, so that the stores cover whole rows (store_acc_64cols)
+      uint8_t* stage = sQ + s * kTile + (warp & 3) * 4096;
+      const int q_first = row0 + s * 128 + (warp & 3) * 32;        // the warp's first row
+      __nv_bfloat16* obase = a.o + b * a.o_strides[0] + h * a.o_strides[1];
 #pragma unroll
-      for (int c = 0; c < D / 32; ++c) {
-        uint32_t oreg[32];
-        tmem_ld32(my_o + c * 32, oreg);
-        tmem_ld_wait();
-#pragma unroll
-        for (int x = 0; x < 32; x += 8) {
-          uint4 v4;
-          v4.x = pack_bf16(__uint_as_float(oreg[x + 0]) * inv_l, __uint_as_float(oreg[x + 1]) * inv_l);
-          v4.y = pack_bf16(__uint_as_float(oreg[x + 2]) * inv_l, __uint_as_float(oreg[x + 3]) * inv_l);
-          v4.z = pack_bf16(__uint_as_float(oreg[x + 4]) * inv_l, __uint_as_float(oreg[x + 5]) * inv_l);
-          v4.w = pack_bf16(__uint_as_float(oreg[x + 6]) * inv_l, __uint_as_float(oreg[x + 7]) * inv_l);
-          if (mine) *reinterpret_cast<uint4*>(orow + c * 32 + x) = v4;
-        }
-      }
+      for (int c = 0; c < D / 64; ++c)
+        store_acc_64cols(my_o + c * 64, stage, inv_l, [&](int r2) -> __nv_bfloat16* {
+          const int q2 = q_first + r2;
+          return (q2 < a.L && q2 >= a.q_start) ? obase + static_cast<int64_t>(q2 - a.q_start) * a.o_strides[2] + c * 64 : nullptr;
+        });
       if (mine)
         a.lse[(static_cast<int64_t>(b) * a.Hq + h) * a.Lq + qi - a.q_start] =
             l_run > 0.f ? (m_ref + log2f(l_run)) * 0.6931471805599453f : -INFINITY;
