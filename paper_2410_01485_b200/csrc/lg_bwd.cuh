@@ -1107,7 +1107,14 @@ bwd_dq_from_ds_kernel(const __grid_constant__ CUtensorMap tm_k, const BwdArgs a)
       const uint32_t lane_addr = tmem + (static_cast<uint32_t>(warp * 32) << 16);
       __nv_bfloat16* dq_row = a.out0 + b * a.s0[0] + h * a.s0[1] + static_cast<int64_t>(qi) * a.s0[2];
       if (n_ent > 0) {
-        store_acc_cols<D>(lane_addr, dq_row, a.scale, qi < a.L);
+        // through the dS ring (every tile loaded into it has been consumed): whole rows per store instruction
+        __nv_bfloat16* base = a.out0 + b * a.s0[0] + h * a.s0[1];
+#pragma unroll
+        for (int c = 0; c < D / 64; ++c)
+          store_acc_64cols(lane_addr + c * 64, smem + SM::oA + warp * 4096, a.scale, [&](int r2) -> __nv_bfloat16* {
+            const int q2 = t * 128 + warp * 32 + r2;
+            return q2 < a.L ? base + static_cast<int64_t>(q2) * a.s0[2] + c * 64 : nullptr;
+          });
       } else if (qi < a.L) {
 #pragma unroll
         for (int x = 0; x < D; x += 8) *reinterpret_cast<uint4*>(dq_row + x) = make_uint4(0, 0, 0, 0);
