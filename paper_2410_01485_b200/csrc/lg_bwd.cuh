@@ -149,28 +149,6 @@ __device__ __forceinline__ void tma_load_rows(uint8_t* dst, const CUtensorMap* t
     tma_load_4d(dst + x * BwdTile<D>::kBox + (BS == 64 ? half * (64 * 128) : 0), tm, bar, x * 64, row, head, batch);
 }
 
-// fp32 accumulator columns [c0, c0 + n) of this thread's TMEM lane -> bf16 row (times mul)
-template <int N>
-__device__ __forceinline__ void store_acc_cols(uint32_t taddr, __nv_bfloat16* dst, float mul, bool do_store) {
-#pragma unroll
-  for (int c = 0; c < N / 32; ++c) {
-    uint32_t reg[32];
-    tmem_ld32(taddr + c * 32, reg);
-    tmem_ld_wait();
-    if (do_store) {
-#pragma unroll
-      for (int x = 0; x < 32; x += 8) {
-        uint4 v4;
-        v4.x = pack_bf16(__uint_as_float(reg[x + 0]) * mul, __uint_as_float(reg[x + 1]) * mul);
-        v4.y = pack_bf16(__uint_as_float(reg[x + 2]) * mul, __uint_as_float(reg[x + 3]) * mul);
-        v4.z = pack_bf16(__uint_as_float(reg[x + 4]) * mul, __uint_as_float(reg[x + 5]) * mul);
-        v4.w = pack_bf16(__uint_as_float(reg[x + 6]) * mul, __uint_as_float(reg[x + 7]) * mul);
-        *reinterpret_cast<uint4*>(dst + c * 32 + x) = v4;
-      }
-    }
-  }
-}
-
 // A warp of element-wise threads finished writing tensor memory: publish it to the MMA thread.
 __device__ __forceinline__ void ew_publish(uint64_t* bar) {
   tmem_st_wait();
@@ -451,14 +429,18 @@ bwd_dq_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ 
     }
     if (ok) {
       tc_fence_after();
-      constexpr int kEpi = 32;                     // output columns per thread
-      if (g * kEpi < D) {                          // warp-uniform; rows past L take part in the loads only
-        __nv_bfloat16* dq_row = a.out0 + b * a.s0[0] + h * a.s0[1] + static_cast<int64_t>(qi) * a.s0[2] + g * kEpi;
+      if (g * 64 < D) {                            // warp-uniform: warp group g takes 64 output columns
+        __nv_bfloat16* base = a.out0 + b * a.s0[0] + h * a.s0[1] + g * 64;
         if (n_steps > 0) {
-          store_acc_cols<kEpi>(lane_addr + kColDQ + g * kEpi, dq_row, a.scale, qi < a.L);
+          // through the K ring (every tile loaded into it has been consumed): whole rows per store instruction;
+          // rows past L take part in the loads only
+          const int q_first = qi - lane;
+          store_acc_64cols(lane_addr + kColDQ + g * 64, smem + SM::oA + warp * 4096, a.scale, [&](int r2) -> __nv_bfloat16* {
+            return q_first + r2 < a.L ? base + static_cast<int64_t>(q_first + r2) * a.s0[2] : nullptr;
+          });
         } else if (qi < a.L) {
 #pragma unroll
-          for (int x = 0; x < kEpi; x += 8) *reinterpret_cast<uint4*>(dq_row + x) = make_uint4(0, 0, 0, 0);
+          for (int x = 0; x < 64; x += 8) *reinterpret_cast<uint4*>(base + static_cast<int64_t>(qi) * a.s0[2] + x) = make_uint4(0, 0, 0, 0);
         }
       }
     }
