@@ -820,7 +820,8 @@ bwd_dkdv_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
       float p[C];
       {
         uint32_t sreg[C];
-        if constexpr (C == 16) tmem_ld16(s_addr, sreg); else tmem_ld32(s_addr, sreg);
+#pragma unroll
+        for (int c = 0; c < C; c += 32) tmem_ld32(s_addr + c, sreg + c);
         tmem_ld_wait();
         const bool masked = __any_sync(0xffffffffu, xmin > 0 || xmax < C);
 #pragma unroll
@@ -848,7 +849,7 @@ bwd_dkdv_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
         uint32_t preg[C / 2];
 #pragma unroll
         for (int c = 0; c < C; c += 2) preg[c >> 1] = pack_bf16(p[c], p[c + 1]);
-        if constexpr (C == 16) tmem_st8(s_addr, preg); else tmem_st16(s_addr, preg);                               // P^T over my own S^T columns
+        if constexpr (C == 32) tmem_st16(s_addr, preg); else tmem_st32(s_addr, preg);   // P^T over my own S^T columns
         ew_publish(bars + B_PF + half);
       }
       ok = mbar_wait(bars + B_DPF + half, j & 1, a.error_word, 2);
@@ -857,35 +858,39 @@ bwd_dkdv_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
       tc_fence_after();
       uint32_t dsreg[C / 2];
       {
-        uint32_t dreg[C];
-        if constexpr (C == 16) tmem_ld16(dp_addr, dreg); else tmem_ld32(dp_addr, dreg);
-        tmem_ld_wait();
 #pragma unroll
-        for (int x = 0; x < C; x += 4) {
-          const float4 d4 = st_d[x >> 2];
-          float d0, d1, d2, d3;
-          f32x2_split(mul_f32x2(f32x2(p[x], p[x + 1]),
-                                add_f32x2(f32x2(__uint_as_float(dreg[x]), __uint_as_float(dreg[x + 1])),
-                                          f32x2(d4.x, d4.y))), d0, d1);
-          f32x2_split(mul_f32x2(f32x2(p[x + 2], p[x + 3]),
-                                add_f32x2(f32x2(__uint_as_float(dreg[x + 2]), __uint_as_float(dreg[x + 3])),
-                                          f32x2(d4.z, d4.w))), d2, d3);
-          dsreg[x >> 1] = pack_bf16(d0, d1);
-          dsreg[(x >> 1) + 1] = pack_bf16(d2, d3);
+        for (int c0 = 0; c0 < C; c0 += 32) {   // 32 columns at a time: their dP^T leaves the registers before the next 32 arrive
+          uint32_t dreg[32];
+          tmem_ld32(dp_addr + c0, dreg);
+          tmem_ld_wait();
+#pragma unroll
+          for (int y = 0; y < 32; y += 4) {
+            const int x = c0 + y;
+            const float4 d4 = st_d[x >> 2];
+            float d0, d1, d2, d3;
+            f32x2_split(mul_f32x2(f32x2(p[x], p[x + 1]),
+                                  add_f32x2(f32x2(__uint_as_float(dreg[y]), __uint_as_float(dreg[y + 1])),
+                                            f32x2(d4.x, d4.y))), d0, d1);
+            f32x2_split(mul_f32x2(f32x2(p[x + 2], p[x + 3]),
+                                  add_f32x2(f32x2(__uint_as_float(dreg[y + 2]), __uint_as_float(dreg[y + 3])),
+                                            f32x2(d4.z, d4.w))), d2, d3);
+            dsreg[x >> 1] = pack_bf16(d0, d1);
+            dsreg[(x >> 1) + 1] = pack_bf16(d2, d3);
+          }
         }
       }
-      if constexpr (C == 16) tmem_st8(dp_addr, dsreg); else tmem_st16(dp_addr, dsreg);                               // dS^T over my own dP^T columns
+      if constexpr (C == 32) tmem_st16(dp_addr, dsreg); else tmem_st32(dp_addr, dsreg);   // dS^T over my own dP^T columns
       if constexpr (kSpill) {
-        static_assert(!kSpill || (C == 32 && kKvNB == 2), "the kept tiles are laid out for half-steps of 64 queries");
-        // ... and to this half-step's tile in global memory: my 32 queries are four 16-byte groups of my
+        static_assert(!kSpill || ((C == 32 || C == 64) && kKvNB == 2), "the kept tiles are laid out for half-steps of 64 queries");
+        // ... and to this half-step's tile in global memory: my C queries are C / 8 16-byte groups of my
         // key.  (Written once, read once by the dQ pass: marked evict-first so that the stream does not
         // push the Q / dO tiles, which every kv tile of a window re-reads, out of the L2.)
         // (a member the entry does not list has no block, hence no tile: its dS is zero and stays unwritten)
         if (on) {
           uint8_t* dst = reinterpret_cast<uint8_t*>(a.ds_buf) + sTile[(j & 1) * 4 + half * 2 + member] * kDsTileBytes<BS> +
-                         (4 * g) * (16 * BS) + (r & (BS - 1)) * 16;
+                         (C / 8 * g) * (16 * BS) + (r & (BS - 1)) * 16;
 #pragma unroll
-          for (int i = 0; i < 4; ++i)
+          for (int i = 0; i < C / 8; ++i)
             asm volatile("st.global.L2::cache_hint.v4.b32 [%0], {%1, %2, %3, %4}, %5;" ::"l"(dst + i * (16 * BS)),
                          "r"(dsreg[4 * i]), "r"(dsreg[4 * i + 1]), "r"(dsreg[4 * i + 2]), "r"(dsreg[4 * i + 3]), "l"(evict_first) : "memory");
         }
@@ -904,25 +909,28 @@ bwd_dkdv_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
       // The sixteen warps share the output: warp group ge takes 64 columns of one accumulator (dV first, then
       // dK) for its 32 keys.  The rows leave through the Q ring (every load into it has been consumed by the
       // products that are now done), 4 KB per warp, so that the stores cover whole rows (store_acc_64cols).
-      constexpr int kParts = D / 64;
+      constexpr int kParts = D / 64, kGroups = kKvEwWarps / 4;
       const int ge = warp >> 2;
-      if (kb_mine >= 0 && ge < 2 * kParts) {
-        const bool is_dk = ge >= kParts;
-        const int part = ge % kParts;
-        const int64_t* st = is_dk ? a.s0 : a.s1;
-        __nv_bfloat16* base = (is_dk ? a.out0 : a.out1) + b * st[0] + hk * st[1] + part * 64;
-        const int64_t row_stride = st[2];
-        if (n_hs > 0) {
-          const int r_first = (warp & 3) * 32;
-          store_acc_64cols(lane_addr + (is_dk ? kColDK : kColDV) + part * 64, sQ + warp * 4096, is_dk ? a.scale : 1.0f,
-                           [&](int r2) -> __nv_bfloat16* {
-                             const int rr = r_first + r2;
-                             const int k2 = kb_mine * BS + (R == 2 ? (rr & (BS - 1)) : rr);   // keys past L take part in the loads only
-                             return k2 < a.L ? base + static_cast<int64_t>(k2) * row_stride : nullptr;
-                           });
-        } else if (kj < a.L) {
+      if (kb_mine >= 0) {
 #pragma unroll
-          for (int x = 0; x < 64; x += 8) *reinterpret_cast<uint4*>(base + static_cast<int64_t>(kj) * row_stride + x) = make_uint4(0, 0, 0, 0);
+        for (int pi = ge; pi < 2 * kParts; pi += kGroups) {      // warp-uniform
+          const bool is_dk = pi >= kParts;
+          const int part = pi % kParts;
+          const int64_t* st = is_dk ? a.s0 : a.s1;
+          __nv_bfloat16* base = (is_dk ? a.out0 : a.out1) + b * st[0] + hk * st[1] + part * 64;
+          const int64_t row_stride = st[2];
+          if (n_hs > 0) {
+            const int r_first = (warp & 3) * 32;
+            store_acc_64cols(lane_addr + (is_dk ? kColDK : kColDV) + part * 64, sQ + warp * 4096, is_dk ? a.scale : 1.0f,
+                             [&](int r2) -> __nv_bfloat16* {
+                               const int rr = r_first + r2;
+                               const int k2 = kb_mine * BS + (R == 2 ? (rr & (BS - 1)) : rr);   // keys past L take part in the loads only
+                               return k2 < a.L ? base + static_cast<int64_t>(k2) * row_stride : nullptr;
+                             });
+          } else if (kj < a.L) {
+#pragma unroll
+            for (int x = 0; x < 64; x += 8) *reinterpret_cast<uint4*>(base + static_cast<int64_t>(kj) * row_stride + x) = make_uint4(0, 0, 0, 0);
+          }
         }
       }
     }
