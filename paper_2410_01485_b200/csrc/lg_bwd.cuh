@@ -66,6 +66,7 @@ struct BwdArgs {
   __nv_bfloat16* ds_buf;
   const int32_t* col_ptr;    // column lists of the pattern (dK/dV pass that keeps dS: positions of its blocks)
   int ahead;                 // dK/dV pass: CTAs that run at a time (see prefetch_successor), 0: no prefetch
+  int head_group;            // dK/dV pass: kv heads whose CTAs run side by side (cta_coords); >= gridDim.x: all of them
 };
 template <int BS> constexpr int kDsTileBytes = BS * 64 * 2;
 
@@ -513,8 +514,10 @@ bwd_dkdv_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
   // has a wait already given up in this call?  (read now, so that it travels with the schedule loads below)
   unsigned int abort_word = 0;
   if (tid == 0) abort_word = *reinterpret_cast<volatile unsigned int*>(a.error_word);
-  const int tile = checked(a.order[blockIdx.y], 0, a.n_tiles - 1, a.error_word, 120);
-  const int b = blockIdx.x / a.Hkv, hk = blockIdx.x % a.Hkv;
+  int cta_x, cta_y;   // (batch, kv head) and launch rank of this CTA's kv tile
+  cta_coords(static_cast<long long>(blockIdx.y) * gridDim.x + blockIdx.x, gridDim.x, gridDim.y, a.head_group, cta_x, cta_y);
+  const int tile = checked(a.order[cta_y], 0, a.n_tiles - 1, a.error_word, 120);
+  const int b = cta_x / a.Hkv, hk = cta_x % a.Hkv;
   const int ent_off = checked(a.tile_off[tile], 0, a.n_list, a.error_word, 121);
   const int n_ent = checked(a.tile_cnt[tile], 0, a.n_list - ent_off, a.error_word, 122);
   const int32_t* ent = a.tile_ent + ent_off;
@@ -606,8 +609,10 @@ bwd_dkdv_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
         if (a.ahead <= 0) return;
         const int64_t w = static_cast<int64_t>(blockIdx.y) * gridDim.x + blockIdx.x + a.ahead;
         if (w >= static_cast<int64_t>(gridDim.x) * gridDim.y) return;
-        const int t2 = checked(a.order[w / gridDim.x], 0, a.n_tiles - 1, a.error_word, 126);
-        const int x2 = static_cast<int>(w % gridDim.x), b2 = x2 / a.Hkv, hk2 = x2 % a.Hkv;
+        int x2, y2;
+        cta_coords(w, gridDim.x, gridDim.y, a.head_group, x2, y2);
+        const int t2 = checked(a.order[y2], 0, a.n_tiles - 1, a.error_word, 126);
+        const int b2 = x2 / a.Hkv, hk2 = x2 % a.Hkv;
 #pragma unroll
         for (int m = 0; m < R; ++m) {
           const int kb2 = checked(a.tile_cols[R * t2 + m], -1, a.nB - 1, a.error_word, 127);

@@ -288,6 +288,27 @@ __device__ __forceinline__ void tmem_st32(uint32_t taddr, const uint32_t* r) {
 }
 __device__ __forceinline__ void tmem_st_wait() { asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory"); }
 
+// ---- which (head, launch rank) a CTA works ----------------------------------------------
+// CTAs start in the order of their linear index (x fastest).  With x = head, the CTAs that run at one time
+// spread over all heads, a handful of tiles each, and the operand tiles that neighbouring tiles of one
+// head share (the window's K / V in the forward, its Q / dO in the dK/dV pass) have to stay in the L2 for
+// every head at once: 80 MB at 32 heads, more than the L2 holds of it (measured at cfg 3: 22.9 GB of DRAM
+// reads in the dK/dV pass against 4.3 GB of operands; 4.6 GB with groups of four).  Heads can therefore be
+// taken in groups of `group`: linear index w -> group w / (group * n_y), and inside a group the heads
+// alternate and the ranks advance, so that 148 CTAs cover ~ 37 neighbouring tiles of 4 heads.  The host
+// asks for it where the tiles of a head take about the same time (sink + window well below the sequence
+// length); where their lengths differ widely (strided combs, full causal) the longest-first launch order
+// over all heads matters more, and group = n_x leaves it as it is.
+constexpr int kHeadGroup = 4;
+__device__ __forceinline__ void cta_coords(long long w, int n_x, int n_y, int group, int& x, int& y) {
+  const long long per_group = static_cast<long long>(group) * n_y;
+  const int grp = static_cast<int>(w / per_group);
+  const int rem = static_cast<int>(w - grp * per_group);
+  const int size = min(group, n_x - grp * group);   // the last group may be smaller
+  x = grp * group + rem % size;
+  y = rem / size;
+}
+
 // ---- small math helpers --------------------------------------------------------------
 __device__ __forceinline__ float fast_exp2(float x) {
   float y;

@@ -30,6 +30,7 @@ static lg_status launch_fwd_t(const Resolved& r, const WsLayout& w, const void* 
   a.win_block = r.win_block; a.win_phase = r.win_phase;
   a.doc_start = r.doc_start;
   a.scale_log2 = r.scale * 1.4426950408889634f;
+  a.head_group = head_group(r, r.B * r.Hq);
   auto kern = fwd_kernel<D, BS>;
   constexpr int smem = FwdSmem<D>::kTotal;
   if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, smem) != cudaSuccess) return LG_ERR_CUDA;

@@ -86,6 +86,7 @@ enum BwdVariant {
 BwdVariant bwd_variant(const Resolved& r);
 // bytes of the dS^T buffer of the kBwdKeepDs variant
 int sm_count();   // SMs of the current device, < 0 on failure
+int head_group(const Resolved& r, int n_x);
 size_t ds_buffer_bytes(const Resolved& r);
 
 
