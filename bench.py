@@ -210,7 +210,7 @@ def dram_traffic_record(kernel: str):
     """DRAM bytes per launch of `kernel` from the committed ncu summary, or None when the kernel sources
     have changed since that capture (the record carries a hash of them)."""
     import hashlib
-    path = os.path.join(ROOT, "profiles", "dram_traffic_cfg3_small.json")
+    path = os.path.join(ROOT, "profiles", "dram_traffic_cfg3.json")
     if not os.path.exists(path):
         return None, "no record"
     with open(path) as f:
@@ -221,8 +221,6 @@ def dram_traffic_record(kernel: str):
             h.update(f.read())
     if h.hexdigest() != rec["sources_sha256"]:
         return None, "kernel sources changed since the capture %s" % rec["capture"]
-    if kernel not in rec["dram_bytes_per_launch"]:
-        return None, "kernel not in the capture %s" % rec["capture"]
     return rec, rec["capture"]
 
 
@@ -416,12 +414,14 @@ def main():
     dom = max(("fwd", "bwd_dkdv", "bwd_dq"), key=lambda n: kern[n][0])
     achieved = kern[dom][1] / kern[dom][0] / 1e9
     # dram__bytes_read + dram__bytes_write of one launch come from the committed ncu summary of the same kernels
-    # on the 8-head x 32K case of this pattern, scaled by the (head, token) units of this workload; null once
-    # the kernel sources differ from the ones that were captured
+    # on this very workload (a single-pass capture; no scaling: the L2 behaves differently at other sizes);
+    # null for a workload that was not captured and once the kernel sources differ from the captured ones
     rec, rec_note = dram_traffic_record(dom)
     traffic = None
     if rec is not None:
-        traffic = rec["dram_bytes_per_launch"][dom] * (cfg.B * cfg.Hq * cfg.L) / float(rec["units_head_tokens"])
+        traffic = rec["workloads"].get(cfg.name, {}).get(dom)
+        if traffic is None:
+            rec_note = "workload %s is not in the capture %s" % (cfg.name, rec["capture"])
     kernel_ms = {k: v[0] for k, v in kern.items()}
     kernel_ms["index_build_once"] = index_ms
     roofline = {"bound": "tensor", "kernel": dom, "achieved": achieved, "peak": peaks["bf16_sustained"],
