@@ -59,6 +59,7 @@ static lg_status launch_bwd_t(const Resolved& r, const WsLayout& w, const void* 
     dim3 grid(r.B * r.Hkv, r.n_ktiles);
     a.ahead = sm_count();   // one CTA per SM
     a.head_group = head_group(r, r.B * r.Hkv);
+    a.descending = r.mode != LG_MODE_SINK_WINDOW;   // combs and full causal attention
     if (a.ahead < 0) return LG_ERR_CUDA;
     if (variant == kBwdKeepDs) {
       // the tile of zeros that stands in for a half of a query tile a kv tile has no entry for

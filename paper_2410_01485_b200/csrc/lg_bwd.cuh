@@ -67,6 +67,7 @@ struct BwdArgs {
   const int32_t* col_ptr;    // column lists of the pattern (dK/dV pass that keeps dS: positions of its blocks)
   int ahead;                 // dK/dV pass: CTAs that run at a time (see prefetch_successor), 0: no prefetch
   int head_group;            // dK/dV pass: kv heads whose CTAs run side by side (cta_coords); >= gridDim.x: all of them
+  int descending;            // dK/dV pass: walk a tile's entries from the last query block down (see the producer)
 };
 template <int BS> constexpr int kDsTileBytes = BS * 64 * 2;
 
@@ -575,14 +576,23 @@ bwd_dkdv_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
       }
       // Besides the tiles, each step gets the softmax statistics of its 128 queries and the
       // schedule entries of its items, so that the element-wise warps read neither global memory
-      // nor the schedule.  Items run query head by query head through the tile's entries.
+      // nor the schedule.
       bool ok = true;
       int nq = 0, no = 0, nst = 0;   // loads started
-      int grp = 0, e = 0;            // (query head within the group, entry) of the next item
+      // Items: the tile's entries in order, and for every entry the query heads of the group one after the
+      // other.  The order is ascending (from the tile's own diagonal upwards) where the tiles of a head take
+      // about the same time, and DESCENDING, from the last query block down, where they do not (a.descending:
+      // strided combs, full causal attention): every tile of a comb column needs every later row of every
+      // head, and walking down from the last row the kv tiles of a kv head that run at one time stream the
+      // same Q / dO tiles at the same time, whatever their own first row is, and share them in the L2 (cfg 4:
+      // 127 -> 92 GB of DRAM reads in the pass; its operands are 5 GB, but tiles that start later are on
+      // rows of their own again).
+      const int e_step = a.descending ? -1 : 1;
+      int grp = 0, e = a.descending ? n_ent - 1 : 0;    // (query head within the group, entry) of the next item
       // positions, in the column lists, of the members' next blocks: the entries that carry a member's bit
-      // are that column's query blocks in ascending order
-      const int pos_a0 = (kSpill && kb_a >= 0) ? a.col_ptr[kb_a] : 0, pos_b0 = (kSpill && kb_b >= 0) ? a.col_ptr[kb_b] : 0;
-      int pos_a = pos_a0, pos_b = pos_b0;
+      // are that column's query blocks in the same order
+      auto col_first = [&](int kb) { return (!kSpill || kb < 0) ? 0 : (a.descending ? a.col_ptr[kb + 1] - 1 : a.col_ptr[kb]); };
+      int pos_a = col_first(kb_a), pos_b = col_first(kb_b);
       auto next_item = [&](int& hq, int& qrow, int& entry, int64_t& ta, int64_t& tb) {
         entry = ent[e];
         hq = hk * a.G + grp;
@@ -590,9 +600,7 @@ bwd_dkdv_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
         const int64_t head_base = (static_cast<int64_t>(b) * a.Hq + hq) * a.ds_nnz;
         ta = (head_base + pos_a) * (BS / 64);
         tb = (head_base + pos_b) * (BS / 64);
-        pos_a += entry & 1;
-        pos_b += (entry >> 1) & 1;
-        if (++e == n_ent) { e = 0; ++grp; pos_a = pos_a0; pos_b = pos_b0; }
+        if (++grp == a.G) { grp = 0; pos_a += e_step * (entry & 1); pos_b += e_step * ((entry >> 1) & 1); e += e_step; }
       };
       // Each load is started as soon as its ring slot is free, in the order in which the slots come
       // free: dO of step j (its slot is released when the dV and dP^T products of step j - 2 are done),
