@@ -113,11 +113,13 @@ lg_status resolve(const lg_attn_params* p, Resolved* r) {
   return LG_OK;
 }
 
-// Heads whose CTAs the forward and the dK/dV pass run side by side (cta_coords): groups where the tiles of a
-// head take about the same time -- sink + window, the window at most a quarter of the sequence -- and all
-// n_x heads together otherwise (combs and full causal attention need the longest-first order over all heads).
+// Heads whose CTAs the forward and the backward passes run side by side (cta_coords): groups of four where
+// the tiles of a head take about the same time -- sink + window, the window at most a quarter of the
+// sequence --, two heads at a time for full causal attention, and all n_x heads together otherwise (combs
+// need the longest-first order over all heads).
 int head_group(const Resolved& r, int n_x) {
   const bool uniform = r.mode == LG_MODE_SINK_WINDOW && static_cast<long long>(r.pat.nw + r.pat.ns) * 4 <= r.pat.nB;
+  if (r.mode == LG_MODE_FULL_CAUSAL) return kHeadGroupFull < n_x ? kHeadGroupFull : n_x;
   return uniform && n_x > kHeadGroup ? kHeadGroup : n_x;
 }
 

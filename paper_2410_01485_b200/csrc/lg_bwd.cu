@@ -112,6 +112,7 @@ static lg_status launch_bwd_t(const Resolved& r, const WsLayout& w, const void* 
     a.out0 = static_cast<__nv_bfloat16*>(dq);
     a.out1 = nullptr;
     for (int i = 0; i < 3; ++i) { a.s0[i] = r.qs[i]; a.s1[i] = 0; }
+    a.head_group = head_group(r, r.B * r.Hq);
     auto kern = bwd_dq_kernel<D, BS>;
     if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, smem) != cudaSuccess)
       return LG_ERR_CUDA;

@@ -201,8 +201,10 @@ bwd_dq_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ 
   // has a wait already given up in this call?  (read now, so that it travels with the schedule loads below)
   unsigned int abort_word = 0;
   if (tid == 0) abort_word = *reinterpret_cast<volatile unsigned int*>(a.error_word);
-  const int tile = checked(a.order[blockIdx.y], 0, a.n_tiles - 1, a.error_word, 110);
-  const int b = blockIdx.x / a.Hq, h = blockIdx.x % a.Hq, hk = h / a.G;
+  int cta_x, cta_y;   // (batch, query head) and launch rank of this CTA's query tile
+  cta_coords(static_cast<long long>(blockIdx.y) * gridDim.x + blockIdx.x, gridDim.x, gridDim.y, a.head_group, cta_x, cta_y);
+  const int tile = checked(a.order[cta_y], 0, a.n_tiles - 1, a.error_word, 110);
+  const int b = cta_x / a.Hq, h = cta_x % a.Hq, hk = h / a.G;
   const int ent_off = checked(a.tile_off[tile * R], 0, a.n_list, a.error_word, 111);
   const int n_ent = checked(a.tile_cnt[tile], 0, a.n_list - ent_off, a.error_word, 112);
   const int32_t* ent = a.tile_ent + ent_off;
