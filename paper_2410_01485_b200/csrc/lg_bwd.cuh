@@ -68,6 +68,7 @@ struct BwdArgs {
   int ahead;                 // dK/dV pass: CTAs that run at a time (see prefetch_successor), 0: no prefetch
   int head_group;            // dK/dV pass: kv heads whose CTAs run side by side (cta_coords); >= gridDim.x: all of them
   int descending;            // dK/dV pass: walk a tile's entries from the last query block down (see the producer)
+  int n_long;                // dK/dV pass: launch ranks taken in head groups (cta_coords2); >= gridDim.y: all of them
 };
 template <int BS> constexpr int kDsTileBytes = BS * 64 * 2;
 
@@ -518,7 +519,7 @@ bwd_dkdv_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
   unsigned int abort_word = 0;
   if (tid == 0) abort_word = *reinterpret_cast<volatile unsigned int*>(a.error_word);
   int cta_x, cta_y;   // (batch, kv head) and launch rank of this CTA's kv tile
-  cta_coords(static_cast<long long>(blockIdx.y) * gridDim.x + blockIdx.x, gridDim.x, gridDim.y, a.head_group, cta_x, cta_y);
+  cta_coords2(static_cast<long long>(blockIdx.y) * gridDim.x + blockIdx.x, gridDim.x, gridDim.y, a.head_group, a.n_long, cta_x, cta_y);
   const int tile = checked(a.order[cta_y], 0, a.n_tiles - 1, a.error_word, 120);
   const int b = cta_x / a.Hkv, hk = cta_x % a.Hkv;
   const int ent_off = checked(a.tile_off[tile], 0, a.n_list, a.error_word, 121);
@@ -620,7 +621,7 @@ bwd_dkdv_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
         const int64_t w = static_cast<int64_t>(blockIdx.y) * gridDim.x + blockIdx.x + a.ahead;
         if (w >= static_cast<int64_t>(gridDim.x) * gridDim.y) return;
         int x2, y2;
-        cta_coords(w, gridDim.x, gridDim.y, a.head_group, x2, y2);
+        cta_coords2(w, gridDim.x, gridDim.y, a.head_group, a.n_long, x2, y2);
         const int t2 = checked(a.order[y2], 0, a.n_tiles - 1, a.error_word, 126);
         const int b2 = x2 / a.Hkv, hk2 = x2 % a.Hkv;
 #pragma unroll

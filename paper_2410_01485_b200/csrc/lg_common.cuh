@@ -302,8 +302,10 @@ __device__ __forceinline__ void tmem_st_wait() { asm volatile("tcgen05.wait::st.
 // pass): with two heads at a time the tiles that run together share what they stream, and the DRAM reads
 // of the three kernels at 128K fall from 0.5 / 1.1 / 0.5 TB to 5 / 8 / 7 GB (fwd + bwd 664 -> 523 ms).
 // Strided combs keep all heads side by side (group = n_x): a few very long tiles per head make the
-// longest-first launch order over all heads worth more.
+// longest-first launch order over all heads worth more; only the dK/dV pass without grouped queries takes
+// its comb tiles two heads at a time (cta_coords2).
 constexpr int kHeadGroup = 4;
+constexpr int kHeadGroupCombs = 2;  // strided pattern, dK/dV pass: the comb tiles of this many kv heads at a time
 constexpr int kHeadGroupFull = 2;   // full causal attention: every tile of a head streams the same rows from the same end
 __device__ __forceinline__ void cta_coords(long long w, int n_x, int n_y, int group, int& x, int& y) {
   const long long per_group = static_cast<long long>(group) * n_y;
@@ -312,6 +314,15 @@ __device__ __forceinline__ void cta_coords(long long w, int n_x, int n_y, int gr
   const int size = min(group, n_x - grp * group);   // the last group may be smaller
   x = grp * group + rem % size;
   y = rem / size;
+}
+// The same with two regions of launch ranks: the first n_long ranks in groups of `group` heads, the rest with
+// all heads side by side (a strided pattern's few long comb tiles per head, and the many short ones behind
+// them, which fill the tail whatever head the last long tile belongs to).
+__device__ __forceinline__ void cta_coords2(long long w, int n_x, int n_y, int group, int n_long, int& x, int& y) {
+  const long long first = static_cast<long long>(n_x) * n_long;
+  if (n_long >= n_y || w < first) { cta_coords(w, n_x, n_long < n_y ? n_long : n_y, group, x, y); return; }
+  x = static_cast<int>((w - first) % n_x);
+  y = n_long + static_cast<int>((w - first) / n_x);
 }
 
 // ---- small math helpers --------------------------------------------------------------

@@ -75,6 +75,9 @@ SMALL = [
     replace(synth.CFG1, name="window_ge_L", L=512, sink_tokens=0, window_tokens=512, Hq=3, Hkv=1, D=128),
     replace(synth.CFG1, name="strided_bs128", mode=synth.MODE_STRIDED_LOCAL, stride_blocks=3, local_blocks=1,
             block=128, L=1536, D=64, Hq=2, Hkv=2),
+    # comb tiles taken two heads at a time in the dK/dV pass: odd head count, comb columns that do not fill their last tile
+    replace(synth.CFG1, name="strided_5heads", mode=synth.MODE_STRIDED_LOCAL, stride_blocks=4, local_blocks=1,
+            L=64 * 23, D=128, Hq=5, Hkv=5),
     # token-exact window edge (the mask the rolling-buffer decode applies)
     replace(synth.CFG1, name="exact_bs64", window_exact=True, D=128, L=640),
     replace(synth.CFG1, name="exact_bs128_gqa2", window_exact=True, block=128, sink_tokens=128, window_tokens=256,
