@@ -78,6 +78,11 @@ SMALL = [
     # comb tiles taken two heads at a time in the dK/dV pass: odd head count, comb columns that do not fill their last tile
     replace(synth.CFG1, name="strided_5heads", mode=synth.MODE_STRIDED_LOCAL, stride_blocks=4, local_blocks=1,
             L=64 * 23, D=128, Hq=5, Hkv=5),
+    # heads taken in groups by the launch order (two for full causal attention, four where sink + window is at most
+    # a quarter of the sequence) with a last group that is not full, over batch entries and grouped queries
+    replace(synth.CFG1, name="full_causal_3heads", mode=synth.MODE_FULL_CAUSAL, L=1024, D=128, Hq=3, Hkv=3),
+    replace(synth.CFG1, name="uniform_b2_3heads", L=1024, sink_tokens=64, window_tokens=64, D=128, Hq=3, Hkv=3, B=2),
+    replace(synth.CFG1, name="uniform_gqa2_10heads", L=1280, sink_tokens=64, window_tokens=128, D=64, Hq=10, Hkv=5),
     # token-exact window edge (the mask the rolling-buffer decode applies)
     replace(synth.CFG1, name="exact_bs64", window_exact=True, D=128, L=640),
     replace(synth.CFG1, name="exact_bs128_gqa2", window_exact=True, block=128, sink_tokens=128, window_tokens=256,
