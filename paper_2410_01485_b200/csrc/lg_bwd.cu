@@ -104,8 +104,11 @@ static lg_status launch_bwd_t(const Resolved& r, const WsLayout& w, const void* 
     constexpr int smem_q = DqDsSmem<D>::kTotal;
     if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, smem_q) != cudaSuccess)
       return LG_ERR_CUDA;
-    dim3 grid(r.B * r.Hq, r.n_qtiles);
-    kern<<<grid, kDq2Threads, smem_q, stream>>>(tk, a); note_launch();
+    const int n_sm = sm_count();
+    if (n_sm <= 0) return LG_ERR_CUDA;
+    const long long n_items = static_cast<long long>(r.B) * r.Hq * r.n_qtiles;
+    const int n_cta = static_cast<int>(n_items < n_sm ? n_items : n_sm);   // one CTA per SM, each working every n_cta-th item
+    kern<<<n_cta, kDq2Threads, smem_q, stream>>>(tk, a, r.B * r.Hq, r.n_qtiles); note_launch();
     if (marks) cudaEventRecord(marks[3], stream);
     return cudaGetLastError() == cudaSuccess ? LG_OK : LG_ERR_CUDA;
   }

@@ -969,24 +969,34 @@ template <int D>
 struct DqDsSmem {
   static constexpr int kTile = BwdTile<D>::kBytes;
   static constexpr int kDs2 = 128 * 128 * 2;                   // dS^T of a step: [key half (64-token blocks)][query half][8 queries][keys][8 queries]
-  static constexpr int kAStages = (D == 128) ? 4 : 5;          // dS^T comes from HBM: the deeper ring
+  static constexpr int kAStages = (D == 128) ? 3 : 5;          // dS^T comes from HBM: the deeper ring
   static constexpr int kKStages = 3;                           // K comes from the L2
+  static constexpr int kStage = 4 * 4096;                      // the epilogue's rows, 4 KB per warp (store_acc_64cols)
   static constexpr int oA = 0;
   static constexpr int oK = kAStages * kDs2;
-  static constexpr int oBar = oK + kKStages * kTile;
+  static constexpr int oStage = oK + kKStages * kTile;
+  static constexpr int oBar = oStage + kStage;
   static constexpr int kTotal = oBar + 256;
 };
 constexpr int kDq2Threads = 6 * 32;
 
+// One CTA per SM, each working the (head, query tile) items  c, c + gridDim.x, ...  of the launch order (head
+// fastest, tiles longest first).  The three roles run through the items on their own: the rings carry on from
+// one item to the next and the accumulator alternates between two column ranges, so that the loads and the
+// products of an item run while the rows of the one before leave -- with one item per CTA, the 2-4 us between
+// an item's last load and the first load of the CTA that followed left the memory system idle for a seventh of
+// the pass.
 template <int D, int BS>
 __global__ void __launch_bounds__(kDq2Threads, 1)
-bwd_dq_from_ds_kernel(const __grid_constant__ CUtensorMap tm_k, const BwdArgs a) {
+bwd_dq_from_ds_kernel(const __grid_constant__ CUtensorMap tm_k, const BwdArgs a, const int n_heads, const int n_ranks) {
   using SM = DqDsSmem<D>;
   constexpr int kAS = SM::kAStages, kKS = SM::kKStages;
   constexpr int R = 128 / BS;
   constexpr int kTile = SM::kTile;
-  enum { B_AF = 0, B_AE = kAS, B_KF = 2 * kAS, B_KE = 2 * kAS + kKS, B_DONE = 2 * kAS + 2 * kKS, B_COUNT = B_DONE + 1 };
+  enum { B_AF = 0, B_AE = kAS, B_KF = 2 * kAS, B_KE = 2 * kAS + kKS, B_DONE = 2 * kAS + 2 * kKS, B_FREE = B_DONE + 2,
+         B_ALL = B_FREE + 2, B_COUNT = B_ALL + 1 };
   static_assert(B_COUNT * 8 + 8 <= 256, "barrier area too small");
+  static_assert(SM::kTotal <= 227 * 1024, "shared memory");
   extern __shared__ __align__(1024) uint8_t smem[];
   uint64_t* bars = reinterpret_cast<uint64_t*>(smem + SM::oBar);
   uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + B_COUNT);
@@ -999,20 +1009,17 @@ bwd_dq_from_ds_kernel(const __grid_constant__ CUtensorMap tm_k, const BwdArgs a)
   if (!lists_match(a.error_word, a.expect_fp, a.expect_fp2, 80u)) return;
   unsigned int abort_word = 0;
   if (tid == 0) abort_word = *reinterpret_cast<volatile unsigned int*>(a.error_word);
-  const int t = checked(a.order[blockIdx.y], 0, a.n_tiles - 1, a.error_word, 130);   // query tile (128 rows)
-  const int b = blockIdx.x / a.Hq, h = blockIdx.x % a.Hq, hk = h / a.G;
-  const int ent_off = checked(a.tile_off[R * t], 0, a.n_list, a.error_word, 131);
-  const int n_ent = checked(a.tile_cnt[t], 0, a.n_list - ent_off, a.error_word, 132);
-  const int32_t* ent = a.tile_ent + kDqEntInts * static_cast<int64_t>(ent_off);   // (kv tile, dS tiles of its quarters)
+  const long long n_items = static_cast<long long>(n_heads) * n_ranks;
   if (tid == 0) {
     for (int i = 0; i < kAS; ++i) { mbar_init(bars + B_AF + i, 1); mbar_init(bars + B_AE + i, 1); }
     for (int i = 0; i < kKS; ++i) { mbar_init(bars + B_KF + i, 1); mbar_init(bars + B_KE + i, 1); }
-    mbar_init(bars + B_DONE, 1);
+    for (int i = 0; i < 2; ++i) { mbar_init(bars + B_DONE + i, 1); mbar_init(bars + B_FREE + i, 4); }
+    mbar_init(bars + B_ALL, 1);
     mbar_fence_init();
     tmem_slot[1] = abort_word;
   }
   if (warp == 5) {
-    tmem_alloc(tmem_slot, D);
+    tmem_alloc(tmem_slot, 2 * D);
     tmem_relinquish();
   }
   tc_fence_before();
@@ -1020,9 +1027,21 @@ bwd_dq_from_ds_kernel(const __grid_constant__ CUtensorMap tm_k, const BwdArgs a)
   tc_fence_after();
   const uint32_t tmem = *tmem_slot;
   if (tmem_slot[1] != 0) {
-    if (warp == 5) tmem_dealloc(tmem, D);
+    if (warp == 5) tmem_dealloc(tmem, 2 * D);
     return;
   }
+  // item w of the launch order: (batch entry, head), query tile and its schedule entries
+  struct Item { int b, h, t, n_ent; const int32_t* ent; };
+  auto item_of = [&](long long w) {
+    Item it;
+    const int x = static_cast<int>(w % n_heads), y = static_cast<int>(w / n_heads);
+    it.b = x / a.Hq; it.h = x % a.Hq;
+    it.t = checked(a.order[y], 0, a.n_tiles - 1, a.error_word, 130);   // query tile (128 rows)
+    const int ent_off = checked(a.tile_off[R * it.t], 0, a.n_list, a.error_word, 131);
+    it.n_ent = checked(a.tile_cnt[it.t], 0, a.n_list - ent_off, a.error_word, 132);
+    it.ent = a.tile_ent + kDqEntInts * static_cast<int64_t>(ent_off);   // (kv tile, dS tiles of its quarters)
+    return it;
+  };
   if (warp == 4) {
     // ------------------------------ TMA producer ------------------------------------------
     if (lane == 0) {
@@ -1030,49 +1049,57 @@ bwd_dq_from_ds_kernel(const __grid_constant__ CUtensorMap tm_k, const BwdArgs a)
       uint64_t evict_first;
       asm volatile("createpolicy.fractional.L2::evict_first.b64 %0, 1.0;" : "=l"(evict_first));   // dS tiles are read once
       constexpr int E = kDqEntInts, NT = (BS == 128) ? 2 : 4;   // tiles per step
-      const int64_t head_base = (static_cast<int64_t>(b) * a.Hq + h) * a.ds_nnz * (BS / 64);
-      const int64_t zero_tile = static_cast<int64_t>(gridDim.x) * a.ds_nnz * (BS / 64);              // the tile after the last head's
+      const int64_t zero_tile = static_cast<int64_t>(n_heads) * a.ds_nnz * (BS / 64);                // the tile after the last head's
       bool ok = true;
-      int nl = 0;
-      int e_next[E];
+      int g = 0;   // steps loaded so far, over all items: ring slots and barrier phases follow it
+      for (long long w = blockIdx.x; w < n_items && ok; w += gridDim.x) {
+        const Item it = item_of(w);
+        const int hk = it.h / a.G;
+        const int64_t head_base = (static_cast<int64_t>(it.b) * a.Hq + it.h) * a.ds_nnz * (BS / 64);
+        int e_next[E];
 #pragma unroll
-      for (int i = 0; i < E; ++i) e_next[i] = n_ent > 0 ? ent[i] : 0;
-      for (int x = 0; x < n_ent; ++x) {
-        int e_cur[E];
+        for (int i = 0; i < E; ++i) e_next[i] = it.n_ent > 0 ? it.ent[i] : 0;
+        for (int x = 0; x < it.n_ent; ++x) {
+          int e_cur[E];
 #pragma unroll
-        for (int i = 0; i < E; ++i) e_cur[i] = e_next[i];
-        const int T = checked(e_cur[0], 0, a.nB - 1, a.error_word, 133);   // (with 64-token blocks T indexes the tiles' column pairs; nB bounds it from above)
-        if (x + 1 < n_ent) {   // read ahead
+          for (int i = 0; i < E; ++i) e_cur[i] = e_next[i];
+          const int T = checked(e_cur[0], 0, a.nB - 1, a.error_word, 133);   // (with 64-token blocks T indexes the tiles' column pairs; nB bounds it from above)
+          if (x + 1 < it.n_ent) {   // read ahead
 #pragma unroll
-          for (int i = 0; i < E; ++i) e_next[i] = ent[E * (x + 1) + i];
+            for (int i = 0; i < E; ++i) e_next[i] = it.ent[E * (x + 1) + i];
+          }
+          const int sa = g % kAS, sk = g % kKS;
+          if (g >= kAS) ok = mbar_wait(bars + B_AE + sa, ((g / kAS) - 1) & 1, a.error_word, 81);
+          if (!ok) break;
+          mbar_expect_tx(bars + B_AF + sa, SM::kDs2);
+          uint8_t* dA = smem + SM::oA + sa * SM::kDs2;
+#pragma unroll
+          for (int i = 0; i < NT; ++i) {   // i = 2 * key half + query half: the order of the schedule entry and of the stage
+            const int hx = checked(e_cur[1 + i], -1, static_cast<int>(a.ds_nnz * (BS / 64)) - 1, a.error_word, 134);
+            const int64_t tile_idx = hx >= 0 ? head_base + hx : zero_tile;
+            bulk_load_hint(dA + i * kDsTileBytes<BS>, reinterpret_cast<const uint8_t*>(a.ds_buf) + tile_idx * kDsTileBytes<BS>,
+                           kDsTileBytes<BS>, bars + B_AF + sa, evict_first);
+          }
+          if (g >= kKS) ok = mbar_wait(bars + B_KE + sk, ((g / kKS) - 1) & 1, a.error_word, 86);
+          if (!ok) {   // the dS tiles just asked for: let them land before the CTA leaves
+            mbar_wait(bars + B_AF + sa, (g / kAS) & 1, a.error_word, 82);
+            break;
+          }
+          mbar_expect_tx(bars + B_KF + sk, kTile);
+          uint8_t* dK = smem + SM::oK + sk * kTile;
+          if (BS == 128) {
+            tma_load_rows<D, 128>(dK, &tm_k, bars + B_KF + sk, 0, T * 128, hk, it.b);
+          } else {   // the tile's two pattern columns need not be neighbours (a missing one: its dS rows are zero)
+            const int ca = a.tile_cols[2 * T], cb = a.tile_cols[2 * T + 1];
+            tma_load_rows<D, 64>(dK, &tm_k, bars + B_KF + sk, 0, ca * 64, hk, it.b);
+            tma_load_rows<D, 64>(dK, &tm_k, bars + B_KF + sk, 1, (cb >= 0 ? cb : ca) * 64, hk, it.b);
+          }
+          ++g;
         }
-        const int sa = x % kAS, sk = x % kKS;
-        if (x >= kAS) ok = mbar_wait(bars + B_AE + sa, ((x / kAS) - 1) & 1, a.error_word, 81);
-        if (!ok) break;
-        mbar_expect_tx(bars + B_AF + sa, SM::kDs2);
-        uint8_t* dA = smem + SM::oA + sa * SM::kDs2;
-#pragma unroll
-        for (int i = 0; i < NT; ++i) {   // i = 2 * key half + query half: the order of the schedule entry and of the stage
-          const int hx = checked(e_cur[1 + i], -1, static_cast<int>(a.ds_nnz * (BS / 64)) - 1, a.error_word, 134);
-          const int64_t tile_idx = hx >= 0 ? head_base + hx : zero_tile;
-          bulk_load_hint(dA + i * kDsTileBytes<BS>, reinterpret_cast<const uint8_t*>(a.ds_buf) + tile_idx * kDsTileBytes<BS>,
-                         kDsTileBytes<BS>, bars + B_AF + sa, evict_first);
-        }
-        if (x >= kKS) ok = mbar_wait(bars + B_KE + sk, ((x / kKS) - 1) & 1, a.error_word, 86);
-        if (!ok) break;
-        mbar_expect_tx(bars + B_KF + sk, kTile);
-        uint8_t* dK = smem + SM::oK + sk * kTile;
-        if (BS == 128) {
-          tma_load_rows<D, 128>(dK, &tm_k, bars + B_KF + sk, 0, T * 128, hk, b);
-        } else {   // the tile's two pattern columns need not be neighbours (a missing one: its dS rows are zero)
-          const int ca = a.tile_cols[2 * T], cb = a.tile_cols[2 * T + 1];
-          tma_load_rows<D, 64>(dK, &tm_k, bars + B_KF + sk, 0, ca * 64, hk, b);
-          tma_load_rows<D, 64>(dK, &tm_k, bars + B_KF + sk, 1, (cb >= 0 ? cb : ca) * 64, hk, b);
-        }
-        nl = x + 1;
       }
-      for (int x = max(nl - kAS, 0); x < nl; ++x) mbar_wait(bars + B_AF + x % kAS, (x / kAS) & 1, a.error_word, 82);
-      for (int x = max(nl - kKS, 0); x < nl; ++x) mbar_wait(bars + B_KF + x % kKS, (x / kKS) & 1, a.error_word, 87);
+      // every load asked for has landed before the CTA leaves
+      for (int x = max(g - kAS, 0); x < g; ++x) mbar_wait(bars + B_AF + x % kAS, (x / kAS) & 1, a.error_word, 82);
+      for (int x = max(g - kKS, 0); x < g; ++x) mbar_wait(bars + B_KF + x % kKS, (x / kKS) & 1, a.error_word, 87);
     }
   } else if (warp == 5) {
     // ------------------------------ MMA issuer ---------------------------------------------
@@ -1084,44 +1111,61 @@ bwd_dq_from_ds_kernel(const __grid_constant__ CUtensorMap tm_k, const BwdArgs a)
     const uint32_t a_hi = desc_hi(16 * BS, 0);
     const uint32_t a_lo0 = desc_lo(smem_u32(smem + SM::oA), 128), k_lo0 = desc_lo(smem_u32(smem + SM::oK), BwdTile<D>::kBox);
     bool ok = true;
+    int g = 0, n_acc = 0;   // steps consumed and accumulators filled so far, over all items
 #pragma unroll 1
-    for (int x = 0; x < n_ent; ++x) {
-      const int sa = x % kAS, sk = x % kKS;
-      ok = ok && mbar_wait(bars + B_AF + sa, (x / kAS) & 1, a.error_word, 83);
-      ok = ok && mbar_wait(bars + B_KF + sk, (x / kKS) & 1, a.error_word, 88);
-      if (ok) {
-        tc_fence_after();
-        const uint32_t a_lo = a_lo0 + sa * (SM::kDs2 >> 4), b_lo = k_lo0 + sk * (kTile >> 4);
+    for (long long w = blockIdx.x; w < n_items && ok; w += gridDim.x) {
+      const Item it = item_of(w);
+      if (it.n_ent == 0) continue;
+      const uint32_t acc = tmem + (n_acc & 1) * D;
+      // the rows of the item that used this accumulator two items ago have been read
+      if (n_acc >= 2) ok = mbar_wait(bars + B_FREE + (n_acc & 1), ((n_acc >> 1) - 1) & 1, a.error_word, 89);
+#pragma unroll 1
+      for (int x = 0; x < it.n_ent && ok; ++x, ++g) {
+        const int sa = g % kAS, sk = g % kKS;
+        ok = ok && mbar_wait(bars + B_AF + sa, (g / kAS) & 1, a.error_word, 83);
+        ok = ok && mbar_wait(bars + B_KF + sk, (g / kKS) & 1, a.error_word, 88);
+        if (ok) {
+          tc_fence_after();
+          const uint32_t a_lo = a_lo0 + sa * (SM::kDs2 >> 4), b_lo = k_lo0 + sk * (kTile >> 4);
 #pragma unroll
-        for (int kk = 0; kk < 8; ++kk)
-          if (lead)
-            mma_ss2x(tmem, a_lo + (BS == 128 ? kk * (256 >> 4) : (kk >> 2) * (16384 >> 4) + (kk & 3) * (256 >> 4)), a_hi,
-                     b_lo + kk * (2048 >> 4), hi, idesc, (x > 0) || (kk > 0));
+          for (int kk = 0; kk < 8; ++kk)
+            if (lead)
+              mma_ss2x(acc, a_lo + (BS == 128 ? kk * (256 >> 4) : (kk >> 2) * (16384 >> 4) + (kk & 3) * (256 >> 4)), a_hi,
+                       b_lo + kk * (2048 >> 4), hi, idesc, (x > 0) || (kk > 0));
+        }
+        if (lead) { mma_commit(bars + B_AE + sa); mma_commit(bars + B_KE + sk); }
       }
-      if (lead) { mma_commit(bars + B_AE + sa); mma_commit(bars + B_KE + sk); }
+      if (lead) mma_commit(bars + B_DONE + (n_acc & 1));
+      ++n_acc;
     }
-    if (lead) mma_commit(bars + B_DONE);
-    mbar_wait(bars + B_DONE, 0, a.error_word, 84);           // nothing of mine is still running at exit
+    if (lead) mma_commit(bars + B_ALL);
+    mbar_wait(bars + B_ALL, 0, a.error_word, 84);           // nothing of mine is still running at exit
   } else {
     // ------------------------------ epilogue: dQ * scale -> bf16 ----------------------------
-    const int r = warp * 32 + lane;
-    const int qi = t * 128 + r;
     bool ok = true;
-    if (n_ent > 0) ok = mbar_wait_warp(bars + B_DONE, 0, a.error_word, 85);
-    if (ok) {
-      tc_fence_after();
-      const uint32_t lane_addr = tmem + (static_cast<uint32_t>(warp * 32) << 16);
-      __nv_bfloat16* dq_row = a.out0 + b * a.s0[0] + h * a.s0[1] + static_cast<int64_t>(qi) * a.s0[2];
-      if (n_ent > 0) {
-        // through the dS ring (every tile loaded into it has been consumed): whole rows per store instruction
-        __nv_bfloat16* base = a.out0 + b * a.s0[0] + h * a.s0[1];
+    int n_acc = 0;
+    for (long long w = blockIdx.x; w < n_items && ok; w += gridDim.x) {
+      const Item it = item_of(w);
+      const int qi = it.t * 128 + warp * 32 + lane;
+      __nv_bfloat16* base = a.out0 + it.b * a.s0[0] + it.h * a.s0[1];
+      if (it.n_ent > 0) {
+        ok = mbar_wait_warp(bars + B_DONE + (n_acc & 1), (n_acc >> 1) & 1, a.error_word, 85);
+        if (!ok) break;
+        tc_fence_after();
+        const uint32_t lane_addr = tmem + (n_acc & 1) * D + (static_cast<uint32_t>(warp * 32) << 16);
+        // through 4 KB of shared memory per warp: whole rows per store instruction
 #pragma unroll
         for (int c = 0; c < D / 64; ++c)
-          store_acc_64cols(lane_addr + c * 64, smem + SM::oA + warp * 4096, a.scale, [&](int r2) -> __nv_bfloat16* {
-            const int q2 = t * 128 + warp * 32 + r2;
+          store_acc_64cols(lane_addr + c * 64, smem + SM::oStage + warp * 4096, a.scale, [&](int r2) -> __nv_bfloat16* {
+            const int q2 = it.t * 128 + warp * 32 + r2;
             return q2 < a.L ? base + static_cast<int64_t>(q2) * a.s0[2] + c * 64 : nullptr;
           });
+        tc_fence_before();
+        __syncwarp();
+        if (lane == 0) mbar_arrive(bars + B_FREE + (n_acc & 1));   // the accumulator may be filled again
+        ++n_acc;
       } else if (qi < a.L) {
+        __nv_bfloat16* dq_row = base + static_cast<int64_t>(qi) * a.s0[2];
 #pragma unroll
         for (int x = 0; x < D; x += 8) *reinterpret_cast<uint4*>(dq_row + x) = make_uint4(0, 0, 0, 0);
       }
@@ -1129,7 +1173,7 @@ bwd_dq_from_ds_kernel(const __grid_constant__ CUtensorMap tm_k, const BwdArgs a)
   }
   tc_fence_before();
   __syncthreads();
-  if (warp == 5) tmem_dealloc(tmem, D);
+  if (warp == 5) tmem_dealloc(tmem, 2 * D);
 }
 
 }  // namespace lg
