@@ -149,7 +149,8 @@ lg_status lg_sparse_attn_bwd(const lg_attn_params* p, const void* q, const void*
  * reflects the choice): 0 = two passes, the dQ pass recomputing S and dP; 2 = the dK/dV pass also
  * writes dS (bf16, 2 bytes per pair of every block of the pattern and query head) to the workspace and
  * the dQ pass is the single product dQ = dS K.  The second is chosen when that buffer takes at most
- * 48 GB (environment: LG_KEEP_DS_MAX_GB) and the block lists are shared by the batch; the environment
+ * 40 % of the current device's memory (or LG_KEEP_DS_MAX_GB gigabytes, where the environment sets it;
+ * 48 GB where no device can be asked) and the block lists are shared by the batch; the environment
  * variable LG_BWD_VARIANT = two_pass | keep_ds overrides the choice.  Both give bitwise reproducible
  * results; they differ from one another in the last bits (dS is rounded to bf16 once either way, but the
  * order of the fp32 sums differs).  < 0 = lg_status.  (The paper has no counterpart.)            */

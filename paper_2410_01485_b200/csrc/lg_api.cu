@@ -140,11 +140,27 @@ int sm_count() {
 // Keeping dS trades workspace and HBM traffic (2 bytes per visible pair, written once and read once, on
 // a memory system the attention kernels otherwise leave idle) for the two recomputed products of the dQ
 // pass.  It is the default when the lists are shared by the batch and the dS buffer takes at most
-// LG_KEEP_DS_MAX_GB (default 48) gigabytes (the buffer holds every block of the pattern in full).
+// LG_KEEP_DS_MAX_GB gigabytes (the buffer holds every block of the pattern in full); without the variable
+// the limit is 40 % of the current device's memory (77 GB of a B200's 192e9 bytes: 64 query heads of the
+// strided pattern at 128K, 73 GB, still keep dS), 48 GB where no device can be asked.
 // LG_BWD_VARIANT = two_pass | keep_ds overrides the choice (read at every call; it must not change between
 // a size query, a prepare and the calls that use them).
 size_t ds_buffer_bytes(const Resolved& r) {   // 2 bytes per pair of every block of the pattern and query head, plus one tile of zeros at the end
   return static_cast<size_t>(r.B) * r.Hq * static_cast<size_t>(r.nnz) * r.block * r.block * 2 + 128 * 64 * 2;
+}
+
+// largest dS buffer the default choice accepts, in bytes
+double keep_ds_limit() {
+  if (const char* m = getenv("LG_KEEP_DS_MAX_GB")) return atof(m) * 1e9;
+  static double cached[64];
+  int dev = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) { cudaGetLastError(); return 48e9; }
+  if (cached[dev] == 0.0) {
+    size_t free_b = 0, total_b = 0;
+    if (cudaMemGetInfo(&free_b, &total_b) != cudaSuccess || total_b == 0) { cudaGetLastError(); return 48e9; }
+    cached[dev] = 0.4 * static_cast<double>(total_b);
+  }
+  return cached[dev];
 }
 
 BwdVariant bwd_variant(const Resolved& r) {
@@ -153,9 +169,7 @@ BwdVariant bwd_variant(const Resolved& r) {
   // (per-sequence lists have no common tile numbering)
   const bool can_keep = !(r.doc_start != nullptr && r.B > 1);
   if (env && strcmp(env, "keep_ds") == 0) return can_keep ? kBwdKeepDs : kBwdTwoPass;
-  double max_gb = 48.0;
-  if (const char* m = getenv("LG_KEEP_DS_MAX_GB")) max_gb = atof(m);
-  return (can_keep && static_cast<double>(ds_buffer_bytes(r)) <= max_gb * 1e9) ? kBwdKeepDs : kBwdTwoPass;
+  return (can_keep && static_cast<double>(ds_buffer_bytes(r)) <= keep_ds_limit()) ? kBwdKeepDs : kBwdTwoPass;
 }
 
 WsLayout ws_layout(const Resolved& r, bool want_bwd) {

@@ -61,16 +61,18 @@ static lg_status launch_bwd_t(const Resolved& r, const WsLayout& w, const void* 
     a.head_group = head_group(r, r.B * r.Hkv);
     a.n_long = r.n_ktiles;
     a.descending = r.mode != LG_MODE_SINK_WINDOW;   // combs and full causal attention
-    if (r.mode == LG_MODE_STRIDED_LOCAL && r.pat.stride > 1 && r.Hq == r.Hkv) {
+    if (r.mode == LG_MODE_STRIDED_LOCAL && r.pat.stride > 1) {
       // the comb columns (every stride-th) are the longest and share kv tiles among themselves: those tiles,
-      // two heads at a time, walk down the same rows together; the short tiles follow with all heads side by
-      // side (stride-64 setting, 32 heads: dK/dV pass 6.3 -> 5.9 ms).  With grouped-query attention a tile
-      // already streams each row for all query heads of its group and the pass is far from the DRAM bound
-      // (64 / 8 heads at 128K: 34.4-34.9 ms before, 34.9-35.7 ms with two kv heads at a time), so it is left alone.
+      // a few heads at a time, walk down the same rows together; the short tiles follow with all heads side
+      // by side (stride-64 setting, 32 heads, two at a time: dK/dV pass 6.3 -> 5.9 ms).  With grouped-query
+      // attention a tile streams each row for all query heads of its group; four kv heads at a time were
+      // measured best there (64 / 8 heads at 128K, dS kept: 40.5-41.7 -> 39.8-39.9 ms, two at a time 40.8-41.1;
+      // recomputing dQ pass: 34.4-34.9 -> 33.9-35.2 ms, two at a time 34.9-35.7).
       const int n_comb = (r.pat.nB + r.pat.stride - 1) / r.pat.stride, per_tile = 128 / r.block;
       a.n_long = (n_comb + per_tile - 1) / per_tile;
       if (a.n_long > r.n_ktiles) a.n_long = r.n_ktiles;
-      a.head_group = r.B * r.Hkv > kHeadGroupCombs ? kHeadGroupCombs : r.B * r.Hkv;
+      const int comb_group = r.Hq == r.Hkv ? kHeadGroupCombs : kHeadGroupCombsGqa;
+      a.head_group = r.B * r.Hkv > comb_group ? comb_group : r.B * r.Hkv;
     }
     if (a.ahead < 0) return LG_ERR_CUDA;
     if (variant == kBwdKeepDs) {

@@ -302,10 +302,11 @@ __device__ __forceinline__ void tmem_st_wait() { asm volatile("tcgen05.wait::st.
 // pass): with two heads at a time the tiles that run together share what they stream, and the DRAM reads
 // of the three kernels at 128K fall from 0.5 / 1.1 / 0.5 TB to 5 / 8 / 7 GB (fwd + bwd 664 -> 523 ms).
 // Strided combs keep all heads side by side (group = n_x): a few very long tiles per head make the
-// longest-first launch order over all heads worth more; only the dK/dV pass without grouped queries takes
-// its comb tiles two heads at a time (cta_coords2).
+// longest-first launch order over all heads worth more; only the dK/dV pass takes its comb tiles two or four
+// heads at a time (cta_coords2).
 constexpr int kHeadGroup = 4;
-constexpr int kHeadGroupCombs = 2;  // strided pattern, dK/dV pass: the comb tiles of this many kv heads at a time
+constexpr int kHeadGroupCombs = 2;     // strided pattern, dK/dV pass: the comb tiles of this many kv heads at a time
+constexpr int kHeadGroupCombsGqa = 4;  // the same with grouped queries
 constexpr int kHeadGroupFull = 2;   // full causal attention: every tile of a head streams the same rows from the same end
 __device__ __forceinline__ void cta_coords(long long w, int n_x, int n_y, int group, int& x, int& y) {
   const long long per_group = static_cast<long long>(group) * n_y;

@@ -322,7 +322,9 @@ def test_cfg3_train_128k(lg):
     _check_keys(cfg, inp, dk, dv, kv_heads=groups, key_ranges=ranges)
 
 
-def test_cfg4_strided_gqa_128k(lg):
+@pytest.mark.parametrize("variant", ["keep_ds", "two_pass"])
+def test_cfg4_strided_gqa_128k(lg, monkeypatch, variant):
+    monkeypatch.setenv("LG_BWD_VARIANT", variant)   # (keeping dS takes a 73 GB buffer: the default on a 180 GB device)
     cfg = synth.CFG4
     inp = synth.make_attn_inputs(cfg, "cuda", seed=0)
     p = lg.params_of(cfg)
