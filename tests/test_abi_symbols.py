@@ -46,6 +46,33 @@ def test_nnz_and_sizes_on_host(lib):
     assert binding.lg_block_index_nnz(strided) == 139770
 
 
+def test_backward_variant_follows_the_ds_buffer_and_the_environment(lib, monkeypatch):
+    """Which backward a call takes is host logic: dS is kept while its buffer (2 bytes per pair of the pattern's
+    blocks and query head) is within the limit, and the workspace grows by that buffer."""
+    cfg3 = binding.attn_params(1, 32, 32, 131072, 128, 128, binding.MODE_SINK_WINDOW, sink_tokens=128, window_tokens=4096)
+    nnz = binding.lg_block_index_nnz(cfg3)
+    ds_bytes = 32 * nnz * 128 * 128 * 2                       # 34.9e9
+    assert 34.8e9 < ds_bytes < 35.0e9
+    monkeypatch.delenv("LG_BWD_VARIANT", raising=False)
+    sizes = {}
+    for cap, want in (("34", 0), ("36", 2)):                  # just below and just above the buffer
+        monkeypatch.setenv("LG_KEEP_DS_MAX_GB", cap)
+        assert lib.lg_sparse_attn_bwd_variant(C.byref(cfg3)) == want
+        sizes[want] = lib.lg_sparse_attn_workspace_bytes(C.byref(cfg3), 1)
+    assert ds_bytes <= sizes[2] - sizes[0] < ds_bytes + (1 << 20)
+    monkeypatch.setenv("LG_BWD_VARIANT", "two_pass")          # the explicit choice wins over the limit
+    assert lib.lg_sparse_attn_bwd_variant(C.byref(cfg3)) == 0
+    monkeypatch.setenv("LG_BWD_VARIANT", "keep_ds")
+    monkeypatch.setenv("LG_KEEP_DS_MAX_GB", "1")
+    assert lib.lg_sparse_attn_bwd_variant(C.byref(cfg3)) == 2
+    # without either variable the limit is 40 % of the device's memory, 48 GB where there is no device:
+    # the 34.9 GB of this config are kept either way
+    monkeypatch.delenv("LG_BWD_VARIANT")
+    monkeypatch.delenv("LG_KEEP_DS_MAX_GB")
+    assert lib.lg_sparse_attn_bwd_variant(C.byref(cfg3)) == 2
+    assert lib.lg_sparse_attn_bwd_variant(None) < 0
+
+
 @pytest.mark.parametrize("mutate", [
     lambda p: setattr(p, "Hkv", 3),                 # Hq % Hkv != 0
     lambda p: setattr(p, "L", 0),                   # empty sequence
